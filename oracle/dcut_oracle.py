@@ -1,0 +1,256 @@
+"""ctypes front end of the CPU oracle (`dcut_oracle.c`).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
+It marshals numpy / torch-CPU arrays to the C functions and does no arithmetic of its own
+(what each C function computes, and the passage of the paper it follows, is in the C file).
+It imports nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dcut_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the library is missing or older than its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-Wall", "-shared", "-fPIC",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Info(C.Structure):
+    _fields_ = [("n_star", C.c_int32), ("t_total", C.c_int32), ("candidate", C.c_int32),
+                ("closure_ok", C.c_int32), ("sum_fixed", C.c_int64), ("objective", C.c_double),
+                ("sum_f64", C.c_double)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+    return _lib
+
+
+def _p(a, typ):
+    if a is None:
+        return None
+    return a.ctypes.data_as(C.POINTER(typ))
+
+
+def _i32(a):
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _bf16_bits(t) -> np.ndarray:
+    """A torch bf16 CPU tensor (or a uint16 array of bf16 bit patterns) as contiguous uint16."""
+    if isinstance(t, np.ndarray):
+        assert t.dtype == np.uint16
+        return np.ascontiguousarray(t)
+    import torch
+    assert t.dtype == torch.bfloat16 and t.device.type == "cpu"
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def scores(conf: np.ndarray) -> np.ndarray:
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    B, g = conf.shape
+    out = np.empty((B, g), dtype=np.float32)
+    rc = lib().oracle_scores(_p(conf, C.c_float), B, g, _p(out, C.c_float))
+    assert rc == 0, rc
+    return out
+
+
+def budget(B: int, gamma: int, num: int, den: int) -> int:
+    k = C.c_int(0)
+    rc = lib().oracle_budget(B, gamma, num, den, C.byref(k))
+    if rc != 0:
+        raise ValueError(f"oracle_budget rc={rc}")
+    return k.value
+
+
+@dataclass
+class SelectResult:
+    depths: np.ndarray
+    cu_q: np.ndarray
+    tok_req: np.ndarray
+    tok_pos: np.ndarray
+    tok_id: np.ndarray
+    ranks: np.ndarray      # [B, gamma] global rank of every draft position
+    scores: np.ndarray     # [B, gamma] fp32
+    n_star: int
+    t_total: int
+    candidate: int
+    closure_ok: bool
+    sum_fixed: int
+    objective: float
+    sum_f64: float
+
+
+class OracleError(RuntimeError):
+    def __init__(self, rc):
+        super().__init__(f"oracle rc={rc}")
+        self.rc = rc
+
+
+def select(conf, draft_ids, bonus_ids, ctx_lens, cost_ms, bucket_K: Optional[Sequence[int]] = None) -> SelectResult:
+    """Dense mode when bucket_K is None (cost_ms indexed by packed length T), else bucket mode
+    (cost_ms per bucket)."""
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    B, g = conf.shape
+    draft_ids, bonus_ids, ctx_lens = _i32(draft_ids).reshape(B, g), _i32(bonus_ids), _i32(ctx_lens)
+    cost_ms = np.ascontiguousarray(cost_ms, dtype=np.float32)
+    cap = B * (g + 1)
+    depths = np.zeros(B, np.int32)
+    cu_q = np.zeros(B + 1, np.int32)
+    tok_req = np.full(max(cap, 1), -1, np.int32)
+    tok_pos = np.full(max(cap, 1), -1, np.int32)
+    tok_id = np.full(max(cap, 1), -1, np.int32)
+    ranks = np.zeros((B, g), np.int32)
+    sc = np.zeros((B, g), np.float32)
+    info = _Info()
+    bk = None if bucket_K is None else _i32(bucket_K)
+    rc = lib().oracle_select(_p(conf, C.c_float), B, g, _p(draft_ids, C.c_int32), _p(bonus_ids, C.c_int32),
+                             _p(ctx_lens, C.c_int32), 0 if bk is None else 1, _p(cost_ms, C.c_float),
+                             len(cost_ms), _p(bk, C.c_int32), _p(depths, C.c_int32), _p(cu_q, C.c_int32),
+                             _p(tok_req, C.c_int32), _p(tok_pos, C.c_int32), _p(tok_id, C.c_int32),
+                             _p(ranks, C.c_int32), _p(sc, C.c_float), C.byref(info))
+    if rc != 0:
+        raise OracleError(rc)
+    T = info.t_total
+    return SelectResult(depths, cu_q, tok_req[:T], tok_pos[:T], tok_id[:T], ranks, sc, info.n_star, T,
+                        info.candidate, bool(info.closure_ok), info.sum_fixed, info.objective, info.sum_f64)
+
+
+def verify_attn(q, k_cache, v_cache, block_table, ctx_lens, cu_q, n_q_heads, n_kv_heads, head_dim,
+                page_size, scale=None, sample_tok=None, sample_head=None):
+    """Returns (out, lse) in float64: [T, Hq, Dh], [T, Hq], or [n, Dh], [n] for sampled rows."""
+    qb, kb, vb = _bf16_bits(q), _bf16_bits(k_cache), _bf16_bits(v_cache)
+    bt = _i32(block_table)
+    B = bt.shape[0]
+    ctx_lens, cu_q = _i32(ctx_lens), _i32(cu_q)
+    T = int(cu_q[B])
+    if scale is None:
+        scale = 1.0 / np.sqrt(head_dim)
+    if sample_tok is not None:
+        st, sh = _i32(sample_tok), _i32(sample_head)
+        n = len(st)
+        out = np.empty((n, head_dim), np.float64)
+        lse = np.empty((n,), np.float64)
+    else:
+        st = sh = None
+        n = 0
+        out = np.empty((T, n_q_heads, head_dim), np.float64)
+        lse = np.empty((T, n_q_heads), np.float64)
+    f = lib().oracle_verify_attn
+    f.argtypes = [C.c_void_p] * 6 + [C.c_int] * 6 + [C.c_double, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                                     C.c_void_p]
+    rc = f(qb.ctypes.data, kb.ctypes.data, vb.ctypes.data, bt.ctypes.data, ctx_lens.ctypes.data,
+           cu_q.ctypes.data, B, n_q_heads, n_kv_heads, head_dim, page_size, bt.shape[1], float(scale),
+           None if st is None else st.ctypes.data, None if sh is None else sh.ctypes.data, n,
+           out.ctypes.data, lse.ctypes.data)
+    if rc != 0:
+        raise OracleError(rc)
+    return out, lse
+
+
+@dataclass
+class AcceptResult:
+    accept_len: np.ndarray
+    bonus: np.ndarray
+    out_tokens: np.ndarray
+    n_accepted_total: int
+    argmax: np.ndarray
+
+
+def accept(logits, draft_ids, cu_q, gamma: int) -> AcceptResult:
+    lb = _bf16_bits(logits)
+    T, V = lb.shape
+    cu_q = _i32(cu_q)
+    B = len(cu_q) - 1
+    assert int(cu_q[B]) <= T
+    draft_ids = _i32(draft_ids).reshape(B, gamma)
+    al = np.zeros(B, np.int32)
+    bo = np.zeros(B, np.int32)
+    ot = np.zeros((B, gamma + 1), np.int32)
+    tot = C.c_int32(0)
+    am = np.zeros(max(int(cu_q[B]), 1), np.int32)
+    f = lib().oracle_accept
+    f.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 5
+    rc = f(lb.ctypes.data, V, draft_ids.ctypes.data, cu_q.ctypes.data, B, gamma, al.ctypes.data,
+           bo.ctypes.data, ot.ctypes.data, C.addressof(tot), am.ctypes.data)
+    if rc != 0:
+        raise OracleError(rc)
+    return AcceptResult(al, bo, ot, tot.value, am[: int(cu_q[B])])
+
+
+# ---- decoder-layer pieces ---------------------------------------------------------------------
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    out = np.empty(x.shape, np.uint16)
+    f = lib().oracle_round_bf16
+    f.argtypes = [C.c_void_p, C.c_long, C.c_void_p]
+    f.restype = None
+    f(x.ctypes.data, x.size, out.ctypes.data)
+    return out
+
+
+def rmsnorm(x, gain, eps: float) -> np.ndarray:
+    xb, gb = _bf16_bits(x), _bf16_bits(gain)
+    rows, hidden = xb.shape
+    y = np.empty((rows, hidden), np.float64)
+    f = lib().oracle_rmsnorm
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_double, C.c_void_p]
+    assert f(xb.ctypes.data, gb.ctypes.data, rows, hidden, float(eps), y.ctypes.data) == 0
+    return y
+
+
+def linear(a, w) -> np.ndarray:
+    ab, wb = _bf16_bits(a), _bf16_bits(w)
+    M, K = ab.shape
+    N, K2 = wb.shape
+    assert K == K2
+    c = np.empty((M, N), np.float64)
+    f = lib().oracle_linear
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
+    assert f(ab.ctypes.data, wb.ctypes.data, M, N, K, c.ctypes.data) == 0
+    return c
+
+
+def rope(x, pos, theta: float) -> np.ndarray:
+    xb = _bf16_bits(x)
+    rows, heads, dh = xb.shape
+    pos = _i32(pos)
+    y = np.empty((rows, heads, dh), np.float64)
+    f = lib().oracle_rope
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_double, C.c_void_p]
+    assert f(xb.ctypes.data, pos.ctypes.data, rows, heads, dh, float(theta), y.ctypes.data) == 0
+    return y
+
+
+def swiglu(g, u) -> np.ndarray:
+    gb, ub = _bf16_bits(g), _bf16_bits(u)
+    y = np.empty(gb.shape, np.float64)
+    f = lib().oracle_swiglu
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
+    assert f(gb.ctypes.data, ub.ctypes.data, gb.size, y.ctypes.data) == 0
+    return y
