@@ -1,0 +1,158 @@
+/*
+ * libdcut.so - the verify hot path of D-cut (adaptive verification-depth pruning for batched
+ * speculative decoding) as hand-written sm_100a kernels behind a plain C ABI.
+ *
+ * Vocabulary.  B requests; gamma draft tokens per request (the paper's D); c_{i,k} the drafter's
+ * confidence at depth k = 1..gamma; p_{i,k} = prod_{t<=k} c_{i,t} the prefix score (the paper's
+ * s_{i,k}, Eq. 3); d_i the kept depth (the paper's n_i); N the number of kept draft positions over
+ * the batch; T = B + N the packed verification length (the paper's budget K); L_i the number of
+ * tokens request i already has in the KV cache.
+ *
+ * Conventions.
+ *   - Every pointer argument is marked HOST or DEVICE.  Device buffers are owned by the caller
+ *     (any allocator); the library never frees or keeps them beyond the call.
+ *   - Calls that take a `stream` are asynchronous on that CUDA stream (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and never synchronise it.
+ *   - The context owns only its scratch memory, allocated once in dcut_create from dcut_limits;
+ *     no call on the hot path allocates.  One context serves one stream at a time: calls that
+ *     overlap on the GPU share the scratch and race.
+ *   - Every call returns a dcut_status.  Errors the host can see (null pointer, a size over the
+ *     limits, a bad cost table) are returned before anything is launched.  Nothing aborts or traps;
+ *     dcut_last_error gives a message for the last failing call on that context.
+ *   - bf16 tensors are passed as const void* / void* (2 bytes per element, row-major).
+ *   - KV cache layout, for K and for V: [num_pages, n_kv_heads, page_size, head_dim] bf16, so the
+ *     (page, kv head) tile is one contiguous block.  The cache base must be 128-byte aligned.
+ *     Position j of request i lives in page block_table[i][j / page_size], slot j % page_size.
+ */
+#ifndef DCUT_H_
+#define DCUT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dcut_ctx dcut_ctx;
+
+typedef enum {
+    DCUT_OK = 0,
+    DCUT_EINVAL = 1,    /* null pointer, negative size, unsupported shape                        */
+    DCUT_ECAPACITY = 2, /* a size exceeds what dcut_limits reserved                               */
+    DCUT_ECUDA = 3,     /* a CUDA runtime / driver call failed (message in dcut_last_error)       */
+    DCUT_ECOST = 4,     /* cost table missing, too short, or holding a value <= 0, NaN or inf     */
+    DCUT_EDEVICE = 5    /* a kernel reported an error through the device status word             */
+} dcut_status;
+
+typedef struct {
+    int max_B;             /* requests per step                                  */
+    int max_gamma;         /* draft tokens per request; max_B * max_gamma <= 8192 */
+    int n_q_heads;         /* query heads (multiple of n_kv_heads, group <= 16)   */
+    int n_kv_heads;
+    int head_dim;          /* 64 or 128                                          */
+    int page_size;         /* 16                                                 */
+    int max_pages_per_req; /* columns of the block table that may be used        */
+    int vocab;             /* largest vocabulary dcut_accept will see            */
+    int hidden;            /* decoder-layer calls only, else 0                   */
+    int intermediate;      /* decoder-layer calls only, else 0                   */
+} dcut_limits;
+
+/* Result record of dcut_select, written to DEVICE memory (16-byte aligned). */
+typedef struct {
+    int32_t n_star;    /* kept draft positions N*                                              */
+    int32_t t_total;   /* packed length T = B + N*                                             */
+    int32_t candidate; /* index of the winning candidate: N* (dense mode) or the bucket index  */
+    int32_t reserved;
+    int64_t sum_fixed; /* B * 2^40 + sum over the kept positions of floor(p * 2^40)            */
+    double objective;  /* sum_fixed / cost of the winning candidate                            */
+} dcut_select_info;
+
+/* Context.  `device` is the CUDA device ordinal; the context's scratch lives there.
+ * dcut_create allocates; dcut_destroy frees (synchronises the device). */
+dcut_status dcut_create(dcut_ctx** ctx, const dcut_limits* limits, int device);
+dcut_status dcut_destroy(dcut_ctx* ctx);
+const char* dcut_last_error(const dcut_ctx* ctx);
+
+/*
+ * Runtime cost table (Section 3.3, Appendix C "Cost-table profiling protocol"): the latency of a
+ * speculative step as a function of how many positions are verified.  HOST pointers, copied.
+ *
+ * Dense form: cost_ms[T] for packed lengths T = 0..n-1.  dcut_select then searches every
+ * N = 0..B*gamma and needs n > B*(gamma+1).
+ * Bucket form (the paper's Eq. 4-5): n_buckets budgets K[r] (strictly ascending,
+ * B <= K[r] <= B*(gamma+1), total positions including the B bonus positions) and their costs;
+ * valid for exactly this B and gamma.  n_buckets <= 64.
+ * Any cost <= 0, NaN or inf gives DCUT_ECOST.  Setting one form replaces the other.
+ */
+dcut_status dcut_set_cost_dense(dcut_ctx* ctx, const float* cost_ms, int n);
+dcut_status dcut_set_cost_buckets(dcut_ctx* ctx, int B, int gamma, const int* K, const float* cost_ms,
+                                  int n_buckets);
+
+/* Eq. 4: K = max(B, ceil(num/den * B * (gamma+1))), in exact integer arithmetic.  Host only. */
+dcut_status dcut_budget_from_ratio(int B, int gamma, int num, int den, int* K);
+
+/*
+ * Cross-request depth selection (Eq. 3-5; Algorithm 1 steps 2-12; Appendix A, contiguous prefix;
+ * Appendix C, packing).
+ *   p_{i,k} = p_{i,k-1} * clamp(c_{i,k}, 0, 1) in fp32, left to right, p_{i,0} = 1 (NaN counts as 0);
+ *   the B*gamma draft positions are ranked by (p descending, depth ascending, request ascending);
+ *   for each candidate N the objective is (B*2^40 + sum of floor(p*2^40) over the top N) / cost,
+ *   one fp64 divide; the largest objective wins, the smallest N among equals;
+ *   d_i = number of kept positions of request i (a contiguous prefix); cu_q = exclusive prefix sum
+ *   of 1 + d_i; packed tokens are request-major, bonus first: tok_req = i, tok_pos = L_i + t,
+ *   tok_id = z_{i,t}.
+ * DEVICE in:  conf fp32 [B,gamma]; draft_ids i32 [B,gamma]; bonus_ids i32 [B]; ctx_lens i32 [B]
+ *             (draft_ids / bonus_ids / ctx_lens may be NULL if tok_id / tok_pos are NULL).
+ * DEVICE out: depths i32 [B]; cu_q i32 [B+1]; tok_req, tok_pos, tok_id i32 [B*(gamma+1)] (entries
+ *             past T are set to -1; each may be NULL); info (may be NULL); scores_out fp32
+ *             [B,gamma] and ranks_out i32 [B,gamma] (global rank of every draft position), or NULL.
+ * Errors: DCUT_ECOST if no table is set, the dense table is shorter than B*(gamma+1)+1, or the
+ * bucket table was set for another (B, gamma); DCUT_ECAPACITY if B*gamma > 8192 or over limits.
+ */
+dcut_status dcut_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
+                        const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q, int* tok_req,
+                        int* tok_pos, int* tok_id, dcut_select_info* info, float* scores_out,
+                        int* ranks_out, void* stream);
+
+/*
+ * Ragged causal multi-token verification attention over the paged cache (Appendix C: each kept
+ * position is scored against its accepted prefix; Section 1: B*(D+1) tokens verified per step).
+ * For request i, packed token t = 0..d_i (d_i = cu_q[i+1]-cu_q[i]-1), query head h:
+ *   out = softmax_j( q . k_j * scale ) v_j  over cache positions j = 0 .. L_i + t,
+ * reading kv head h / (n_q_heads / n_kv_heads).  The K/V of the 1 + d_i new tokens must already
+ * be in the cache at positions L_i .. L_i + d_i.  bf16 in, fp32 accumulate, bf16 out.
+ * DEVICE in:  q bf16 [T, n_q_heads, head_dim]; k_cache, v_cache (layout above, num_pages pages);
+ *             block_table i32 [B, block_table_stride]; ctx_lens i32 [B] (= L_i); cu_q i32 [B+1].
+ * DEVICE out: out bf16 [T, n_q_heads, head_dim]; lse fp32 [T, n_q_heads] (natural log of the
+ *             softmax denominator, scale applied) or NULL.
+ * T is read on the device from cu_q[B]; T_cap is a host-known upper bound used to size launches
+ * (T_cap <= max_B*(max_gamma+1)).  Shapes come from dcut_limits.  Split-KV partial results live
+ * in the context's scratch.
+ */
+dcut_status dcut_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                             long long num_pages, const int* block_table, int block_table_stride,
+                             const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
+                             void* out, float* lse, void* stream);
+
+/*
+ * Greedy acceptance (Section 3.1-3.2: sequential acceptance, A_i = 1 + min(L_i, n_i), bonus token).
+ * Row cu_q[i]+t of the packed logits predicts z_{i,t+1}.  a_{i,t} = argmax over the vocabulary
+ * (lowest index among equal maxima; NaN never wins; an all-NaN row gives 0);
+ * m_i = longest prefix with a_{i,t} = draft_ids[i][t], t < d_i; bonus_i = a_{i,m_i}.
+ * DEVICE in:  logits bf16 [T, V]; draft_ids i32 [B,gamma]; cu_q i32 [B+1].
+ * DEVICE out: accept_len i32 [B] (= m_i); bonus i32 [B]; out_tokens i32 [B,gamma+1] (m_i drafts,
+ *             the bonus, then -1), may be NULL; n_accepted_total i32 [1] = sum (m_i + 1), may be NULL.
+ * Per-row partial maxima live in the context's scratch.
+ */
+dcut_status dcut_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
+                        int B, int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
+                        int* n_accepted_total, void* stream);
+
+/* Reads the device status word (0 = no kernel reported an error) after synchronising `stream`,
+ * and clears it.  A non-zero code also makes this call return DCUT_EDEVICE. */
+dcut_status dcut_poll_device_status(dcut_ctx* ctx, int* code, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DCUT_H_ */

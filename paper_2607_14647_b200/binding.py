@@ -1,0 +1,202 @@
+"""Thin ctypes binding of libdcut.so: argument marshalling only.
+
+Each function has the name and meaning of the C entry point declared in include/dcut.h; tensors
+are torch CUDA tensors whose `data_ptr()` is passed through, the stream is torch's current
+stream.  There is no CPU fallback: importing this module without a built library raises, and
+every call runs the CUDA kernels.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdcut.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is not built; run `python -m paper_2607_14647_b200.build` "
+                      "(needs nvcc; there is no fallback path)")
+_lib = C.CDLL(LIB_PATH)
+
+OK, EINVAL, ECAPACITY, ECUDA, ECOST, EDEVICE = range(6)
+STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_ECOST", "DCUT_EDEVICE"]
+
+EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
+           "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_poll_device_status"]
+
+
+class Limits(C.Structure):
+    _fields_ = [(n, C.c_int) for n in ("max_B", "max_gamma", "n_q_heads", "n_kv_heads", "head_dim", "page_size",
+                                       "max_pages_per_req", "vocab", "hidden", "intermediate")]
+
+
+class SelectInfo(C.Structure):
+    _fields_ = [("n_star", C.c_int32), ("t_total", C.c_int32), ("candidate", C.c_int32), ("reserved", C.c_int32),
+                ("sum_fixed", C.c_int64), ("objective", C.c_double)]
+
+
+_vp, _i, _ll, _f = C.c_void_p, C.c_int, C.c_longlong, C.c_float
+_lib.dcut_create.argtypes = [C.POINTER(_vp), C.POINTER(Limits), _i]
+_lib.dcut_destroy.argtypes = [_vp]
+_lib.dcut_last_error.argtypes = [_vp]
+_lib.dcut_last_error.restype = C.c_char_p
+_lib.dcut_set_cost_dense.argtypes = [_vp, _vp, _i]
+_lib.dcut_set_cost_buckets.argtypes = [_vp, _i, _i, _vp, _vp, _i]
+_lib.dcut_budget_from_ratio.argtypes = [_i, _i, _i, _i, C.POINTER(_i)]
+_lib.dcut_select.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
+_lib.dcut_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _i, _i, _f, _vp, _vp, _vp]
+_lib.dcut_accept.argtypes = [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
+_lib.dcut_poll_device_status.argtypes = [_vp, C.POINTER(_i), _vp]
+
+
+class DcutError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {msg}")
+        self.status = status
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def budget_from_ratio(B: int, gamma: int, num: int, den: int) -> int:
+    k = _i(0)
+    st = _lib.dcut_budget_from_ratio(B, gamma, num, den, C.byref(k))
+    if st != OK:
+        raise DcutError(st, "dcut_budget_from_ratio")
+    return k.value
+
+
+@dataclass
+class SelectOut:
+    depths: torch.Tensor
+    cu_q: torch.Tensor
+    tok_req: torch.Tensor
+    tok_pos: torch.Tensor
+    tok_id: torch.Tensor
+    info: torch.Tensor       # int64 [4] view of dcut_select_info: see `read_info`
+    scores: Optional[torch.Tensor]
+    ranks: Optional[torch.Tensor]
+
+
+def read_info(info: torch.Tensor) -> SelectInfo:
+    """Copies the device record to the host (synchronises)."""
+    raw = info.cpu().numpy().tobytes()
+    return SelectInfo.from_buffer_copy(raw)
+
+
+class Context:
+    """Owns a dcut_ctx.  Calls are asynchronous on torch's current stream."""
+
+    def __init__(self, max_B: int, max_gamma: int, n_q_heads: int = 0, n_kv_heads: int = 0, head_dim: int = 0,
+                 page_size: int = 16, max_pages_per_req: int = 0, vocab: int = 0, hidden: int = 0,
+                 intermediate: int = 0, device: Optional[int] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libdcut needs a CUDA device (sm_100a); there is no CPU path")
+        self.device = torch.cuda.current_device() if device is None else device
+        self.limits = Limits(max_B, max_gamma, n_q_heads, n_kv_heads, head_dim, page_size, max_pages_per_req,
+                             vocab, hidden, intermediate)
+        self._h = _vp(None)
+        st = _lib.dcut_create(C.byref(self._h), C.byref(self.limits), self.device)
+        if st != OK:
+            msg = _lib.dcut_last_error(self._h).decode() if self._h else "dcut_create"
+            _lib.dcut_destroy(self._h)
+            self._h = _vp(None)
+            raise DcutError(st, msg)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _lib.dcut_destroy(self._h)
+            self._h = _vp(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st != OK:
+            raise DcutError(st, _lib.dcut_last_error(self._h).decode())
+
+    # -- cost model (host arrays) ------------------------------------------------------------
+    def set_cost_dense(self, cost_ms: Sequence[float]):
+        a = np.ascontiguousarray(cost_ms, dtype=np.float32)
+        self._check(_lib.dcut_set_cost_dense(self._h, a.ctypes.data, len(a)))
+
+    def set_cost_buckets(self, B: int, gamma: int, K: Sequence[int], cost_ms: Sequence[float]):
+        k = np.ascontiguousarray(K, dtype=np.int32)
+        a = np.ascontiguousarray(cost_ms, dtype=np.float32)
+        assert len(k) == len(a)
+        self._check(_lib.dcut_set_cost_buckets(self._h, B, gamma, k.ctypes.data, a.ctypes.data, len(a)))
+
+    # -- hot path ------------------------------------------------------------------------------
+    def select(self, conf, draft_ids, bonus_ids, ctx_lens, out: Optional[SelectOut] = None,
+               want_scores: bool = False, want_ranks: bool = False) -> SelectOut:
+        B, gamma = conf.shape
+        dev = conf.device
+        if out is None:
+            cap = B * (gamma + 1)
+            i32 = dict(dtype=torch.int32, device=dev)
+            out = SelectOut(torch.empty(B, **i32), torch.empty(B + 1, **i32), torch.empty(cap, **i32),
+                            torch.empty(cap, **i32), torch.empty(cap, **i32),
+                            torch.zeros(4, dtype=torch.int64, device=dev),
+                            torch.empty((B, gamma), dtype=torch.float32, device=dev) if want_scores else None,
+                            torch.empty((B, gamma), **i32) if want_ranks else None)
+        self._check(_lib.dcut_select(self._h, _ptr(conf, torch.float32), B, gamma, _ptr(draft_ids, torch.int32),
+                                     _ptr(bonus_ids, torch.int32), _ptr(ctx_lens, torch.int32),
+                                     _ptr(out.depths), _ptr(out.cu_q), _ptr(out.tok_req), _ptr(out.tok_pos),
+                                     _ptr(out.tok_id), _ptr(out.info), _ptr(out.scores), _ptr(out.ranks), _stream()))
+        return out
+
+    def verify_attn(self, q, k_cache, v_cache, block_table, ctx_lens, cu_q, T_cap: int, scale: Optional[float] = None,
+                    out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B = ctx_lens.shape[0]
+        if out is None:
+            out = torch.empty_like(q)
+        if scale is None:
+            scale = 1.0 / float(np.sqrt(self.limits.head_dim))
+        self._check(_lib.dcut_verify_attn(self._h, _ptr(q, torch.bfloat16), _ptr(k_cache, torch.bfloat16),
+                                          _ptr(v_cache, torch.bfloat16), k_cache.shape[0],
+                                          _ptr(block_table, torch.int32), block_table.shape[1],
+                                          _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32), B, T_cap,
+                                          float(scale), _ptr(out, torch.bfloat16), _ptr(lse, torch.float32),
+                                          _stream()))
+        return out
+
+    def accept(self, logits, draft_ids, cu_q, T_cap: int, out_tokens: bool = True):
+        B, gamma = draft_ids.shape
+        V = logits.shape[1]
+        i32 = dict(dtype=torch.int32, device=logits.device)
+        accept_len, bonus = torch.empty(B, **i32), torch.empty(B, **i32)
+        toks = torch.empty((B, gamma + 1), **i32) if out_tokens else None
+        total = torch.empty(1, **i32)
+        self.accept_into(logits, draft_ids, cu_q, T_cap, accept_len, bonus, toks, total)
+        return accept_len, bonus, toks, total
+
+    def accept_into(self, logits, draft_ids, cu_q, T_cap, accept_len, bonus, out_tokens, total):
+        B, gamma = draft_ids.shape
+        self._check(_lib.dcut_accept(self._h, _ptr(logits, torch.bfloat16), logits.shape[1],
+                                     _ptr(draft_ids, torch.int32), _ptr(cu_q, torch.int32), B, gamma, T_cap,
+                                     _ptr(accept_len), _ptr(bonus), _ptr(out_tokens), _ptr(total), _stream()))
+
+    def poll_device_status(self) -> int:
+        code = _i(0)
+        st = _lib.dcut_poll_device_status(self._h, C.byref(code), _stream())
+        if st not in (OK, EDEVICE):
+            self._check(st)
+        return code.value

@@ -1,0 +1,174 @@
+// dcut_accept: greedy acceptance (Sections 3.1-3.2: A_i = 1 + min(L_i, n_i) and the bonus token).
+//
+// Two launches.
+//   accept_argmax_kernel  HBM-bound scan of the bf16 logits [T, V].  Each row is cut into
+//       segments, one CTA per (segment, row), so small batches still fill 148 SMs.  Threads read
+//       16-byte vectors with streaming loads, several in flight per thread, and keep (max, first
+//       index); the CTA result is merged into one 64-bit word per row with atomicMax on
+//       (ordered value << 32 | ~index): the largest value wins and, among equals, the lowest
+//       index, whatever order the CTAs finish in.
+//   accept_match_kernel   one thread per request: longest matching prefix, bonus token, emitted
+//       tokens, total; clears the per-row words for the next call.
+#include "dcut_internal.h"
+
+namespace {
+
+constexpr int kArgmaxThreads = 256;
+constexpr int kUnroll = 4;
+
+__device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+// value order as an unsigned integer: larger float <=> larger code; every non-NaN code is > 0
+__device__ __forceinline__ unsigned int ordered_bits(float f) {
+    if (f == 0.0f) f = 0.0f;   // -0 and +0 are the same value
+    const unsigned int b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+__device__ __forceinline__ void take(float f, int idx, float& best, int& bidx) {
+    if (f > best) {   // strict: the first of equal values stays; NaN never passes
+        best = f;
+        bidx = idx;
+    }
+}
+
+__device__ __forceinline__ void take8(const uint4& v, int base, float& best, int& bidx) {
+    const unsigned int w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        take(__uint_as_float(w[e] << 16), base + 2 * e, best, bidx);
+        take(__uint_as_float(w[e] & 0xffff0000u), base + 2 * e + 1, best, bidx);
+    }
+}
+
+__global__ void __launch_bounds__(kArgmaxThreads) accept_argmax_kernel(
+    const unsigned short* __restrict__ logits, int V, const int* __restrict__ cu_q, int B, int seg_elems,
+    unsigned long long* __restrict__ row_key) {
+    const int row = blockIdx.y;
+    if (row >= cu_q[B]) return;
+    const int start = blockIdx.x * seg_elems;
+    if (start >= V) return;
+    const int end = min(V, start + seg_elems);
+    const unsigned short* rp = logits + (size_t)row * V;
+    float best = -INFINITY;
+    int bidx = -1;
+
+    // scalar head up to the first 16-byte boundary, vector body, scalar tail
+    const unsigned long long addr = (unsigned long long)(rp + start);
+    int head = (int)(((16 - (addr & 15)) & 15) >> 1);
+    if (head > end - start) head = end - start;
+    const int body0 = start + head;
+    const int nvec = (end - body0) >> 3;
+    const int tail0 = body0 + (nvec << 3);
+    if ((int)threadIdx.x < head)
+        take(__uint_as_float((unsigned int)rp[start + threadIdx.x] << 16), start + threadIdx.x, best, bidx);
+    const uint4* vp = reinterpret_cast<const uint4*>(rp + body0);
+    int v = threadIdx.x;
+    for (; v + (kUnroll - 1) * kArgmaxThreads < nvec; v += kUnroll * kArgmaxThreads) {
+        uint4 x[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) x[u] = ld_stream_v4(vp + v + u * kArgmaxThreads);
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) take8(x[u], body0 + ((v + u * kArgmaxThreads) << 3), best, bidx);
+    }
+    for (; v < nvec; v += kArgmaxThreads) take8(ld_stream_v4(vp + v), body0 + (v << 3), best, bidx);
+    // a thread's indices ascend except for the tail, which lies past every body index
+    if ((int)threadIdx.x < end - tail0)
+        take(__uint_as_float((unsigned int)rp[tail0 + threadIdx.x] << 16), tail0 + threadIdx.x, best, bidx);
+
+    unsigned long long key = 0;   // 0 = nothing above -inf seen
+    if (bidx >= 0) key = ((unsigned long long)ordered_bits(best) << 32) | (unsigned long long)(0xffffffffu - (unsigned int)bidx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+    }
+    __shared__ unsigned long long wk[kArgmaxThreads / 32];
+    if ((threadIdx.x & 31) == 0) wk[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < kArgmaxThreads / 32; ++w) key = wk[w] > key ? wk[w] : key;
+        if (key) atomicMax(row_key + row, key);
+    }
+}
+
+// rows whose maximum is -inf (or that hold only NaN) leave key 0: the first non-NaN index, else 0
+__device__ int slow_first_valid(const unsigned short* rp, int V) {
+    for (int v = 0; v < V; ++v) {
+        const float f = __uint_as_float((unsigned int)rp[v] << 16);
+        if (f == f) return v;
+    }
+    return 0;
+}
+
+__global__ void __launch_bounds__(1024) accept_match_kernel(
+    const unsigned short* __restrict__ logits, int V, const int* __restrict__ draft_ids,
+    const int* __restrict__ cu_q, int B, int gamma, unsigned long long* __restrict__ row_key,
+    int* __restrict__ accept_len, int* __restrict__ bonus, int* __restrict__ out_tokens,
+    int* __restrict__ n_accepted_total) {
+    __shared__ int total_s;
+    if (threadIdx.x == 0) total_s = 0;
+    __syncthreads();
+    int local = 0;
+    for (int i = threadIdx.x; i < B; i += blockDim.x) {
+        const int a = cu_q[i], d = cu_q[i + 1] - a - 1;
+        int m = -1, bon = 0;
+        for (int t = 0; t <= d; ++t) {
+            const unsigned long long key = row_key[a + t];
+            row_key[a + t] = 0;
+            if (m >= 0) continue;   // already stopped: only clearing
+            const int am = key ? (int)(0xffffffffu - (unsigned int)key) : slow_first_valid(logits + (size_t)(a + t) * V, V);
+            if (t == d || am != draft_ids[(size_t)i * gamma + t]) {
+                m = t;
+                bon = am;
+            }
+        }
+        accept_len[i] = m;
+        bonus[i] = bon;
+        if (out_tokens) {
+            int* o = out_tokens + (size_t)i * (gamma + 1);
+            for (int t = 0; t <= gamma; ++t) o[t] = t < m ? draft_ids[(size_t)i * gamma + t] : (t == m ? bon : -1);
+        }
+        local += m + 1;
+    }
+    if (local) atomicAdd(&total_s, local);
+    __syncthreads();
+    if (threadIdx.x == 0 && n_accepted_total) *n_accepted_total = total_s;
+}
+
+}  // namespace
+
+dcut_status dcut_init_accept(dcut_ctx* ctx) {
+    (void)ctx;
+    return DCUT_OK;
+}
+
+dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids,
+                               const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
+                               int* out_tokens, int* n_accepted_total, unsigned long long* row_key,
+                               cudaStream_t stream) {
+    // segments: at least ~16 KB each, and enough CTAs for a few waves over the SMs
+    const int want_ctas = ctx->sm_count * 16;
+    int splits = (want_ctas + T_cap - 1) / T_cap;
+    const int max_splits = (V + 8191) / 8192;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    int seg = (V + splits - 1) / splits;
+    seg = (seg + 7) & ~7;
+    splits = (V + seg - 1) / seg;
+    dim3 grid(splits, T_cap);
+    accept_argmax_kernel<<<grid, kArgmaxThreads, 0, stream>>>(static_cast<const unsigned short*>(logits), V, cu_q,
+                                                            B, seg, row_key);
+    dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_argmax_kernel");
+    if (st != DCUT_OK) return st;
+    accept_match_kernel<<<1, 1024, 0, stream>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B,
+                                               gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total);
+    return dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_match_kernel");
+}

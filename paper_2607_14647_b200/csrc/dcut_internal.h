@@ -1,0 +1,82 @@
+// Internal declarations shared by the translation units of libdcut.so (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dcut.h"
+
+#define DCUT_MAX_KEYS 8192      // B * gamma handled by the single-CTA selector
+#define DCUT_MAX_BUCKETS 64
+
+// device status word codes (dcut_poll_device_status)
+#define DCUT_DEV_OK 0
+#define DCUT_DEV_ATTN_WAIT_TIMEOUT 1   // a bounded mbarrier wait in the attention kernel gave up
+#define DCUT_DEV_BAD_PAGE 2            // a block-table entry outside [0, num_pages)
+
+// One split-KV work item of the attention kernel: one (request, kv head, page range).
+struct __align__(16) AttnItem {
+    int32_t req;
+    int32_t kv_head;
+    int32_t page_begin;   // first page index (within the request's block-table row)
+    int32_t page_end;     // one past the last
+    int32_t chunk;        // which chunk of this request
+    int32_t n_chunks;     // how many chunks the request has
+    int32_t part_row;     // first row of this item's partial results in the scratch
+    int32_t pad;
+};
+
+struct dcut_ctx {
+    dcut_limits lim;
+    int device;
+    int sm_count;
+    char err[512];
+
+    // cost model
+    float* d_cost;          // dense: [cost_n]; bucket: [n_buckets]
+    int* d_bucket_K;        // [DCUT_MAX_BUCKETS]
+    int cost_n;             // entries of the dense table (0 = none)
+    int cost_cap;           // allocated floats
+    int n_buckets;          // > 0: bucket mode
+    int bucket_B, bucket_gamma;
+
+    // attention scratch
+    AttnItem* d_items;      // [max_items]
+    int* d_plan;            // [8] plan header: n_items, chunk_pages, ...
+    int* d_req_part;        // [max_B * 2]: first partial row / n_chunks per request
+    float* d_part_o;        // [part_rows_cap, head_dim] fp32
+    float* d_part_lse;      // [part_rows_cap]
+    int max_items;
+    long long part_rows_cap;
+    int target_items;
+
+    // accept scratch
+    unsigned long long* d_row_key;   // [max_T] packed (ordered max, ~index); zero between calls
+
+    int* d_status;          // device status word
+
+    // tensor-map encoder (driver entry point fetched through the runtime)
+    void* encode_tiled;
+};
+
+dcut_status dcut_fail(dcut_ctx* ctx, dcut_status st, const char* fmt, ...);
+dcut_status dcut_check_cuda(dcut_ctx* ctx, cudaError_t e, const char* what);
+
+// per-device set-up (function attributes), called from dcut_create with the device current
+dcut_status dcut_init_select(dcut_ctx* ctx);
+dcut_status dcut_init_accept(dcut_ctx* ctx);
+dcut_status dcut_init_verify_attn(dcut_ctx* ctx);
+
+// kernel launchers (one per translation unit)
+dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
+                               const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q,
+                               int* tok_req, int* tok_pos, int* tok_id, dcut_select_info* info,
+                               float* scores_out, int* ranks_out, cudaStream_t stream);
+dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids,
+                               const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
+                               int* out_tokens, int* n_accepted_total, unsigned long long* row_key,
+                               cudaStream_t stream);
+dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                    long long num_pages, const int* block_table, int block_table_stride,
+                                    const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
+                                    void* out, float* lse, cudaStream_t stream);

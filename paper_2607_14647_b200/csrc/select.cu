@@ -1,0 +1,307 @@
+// dcut_select: cross-request depth selection in one CTA (Eq. 3-5, Algorithm 1).
+//
+// The whole problem (at most 8192 draft positions, 32 KB of confidences) fits one SM's shared
+// memory, and every step depends on the one before, so the kernel is latency-bound: one CTA of
+// 1024 threads, no global round trips between the steps.
+//   1. prefix products, one thread per request, fp32, left to right           (Eq. 3)
+//   2. 64-bit keys (inverted score bits | depth | request) and a bitonic sort in shared memory:
+//      ascending key order = score descending, depth ascending, request ascending
+//   3. block-wide scan of the fixed-point scores floor(p * 2^40) in int64 (exact in any order)
+//   4. objective (B*2^40 + Q_N) / cost for every candidate N, fp64 divide, block argmax with
+//      ties toward the smallest N                                            (Eq. 4-5)
+//   5. depths by counting kept keys per request, cu_q by a block scan, packed token metadata
+#include <limits.h>
+
+#include "dcut_internal.h"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+
+struct SelectArgs {
+    const float* conf;
+    const int* draft_ids;
+    const int* bonus_ids;
+    const int* ctx_lens;
+    const float* cost;      // dense: cost[T]; bucket: cost[c]
+    const int* bucket_K;    // bucket mode only
+    int n_buckets;          // 0 = dense
+    int B, gamma, npad;
+    int* depths;
+    int* cu_q;
+    int* tok_req;
+    int* tok_pos;
+    int* tok_id;
+    dcut_select_info* info;
+    float* scores_out;
+    int* ranks_out;
+};
+
+__device__ __forceinline__ float clamp_conf(float c) {
+    if (!(c == c)) return 0.0f;
+    if (c < 0.0f) return 0.0f;
+    if (c > 1.0f) return 1.0f;
+    return c;
+}
+
+template <typename T>
+__device__ __forceinline__ T warp_inclusive_scan(T v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        T u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
+
+// exclusive scan of one value per thread over the CTA; returns the exclusive prefix and writes the
+// CTA total to *total_out (same value in every thread).  `ws` is a [kWarps + 1] shared array.
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T v, T* ws, T* total_out) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    T inc = warp_inclusive_scan(v, lane);
+    if (lane == 31) ws[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        T w = ws[lane];
+        T winc = warp_inclusive_scan(w, lane);
+        ws[lane] = winc - w;
+        if (lane == 31) ws[kWarps] = winc;
+    }
+    __syncthreads();
+    T res = ws[warp] + inc - v;
+    *total_out = ws[kWarps];
+    __syncthreads();
+    return res;
+}
+
+struct Best {
+    double obj;
+    int N;
+    int cand;
+};
+
+__device__ __forceinline__ bool better(const Best& a, const Best& b) {   // is a better than b
+    return a.obj > b.obj || (a.obj == b.obj && a.N < b.N);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int B = a.B, gamma = a.gamma, n = B * gamma, npad = a.npad;
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);          // [npad]
+    long long* qs = reinterpret_cast<long long*>(keys + npad);                       // [npad + 1]
+    int* depth_s = reinterpret_cast<int*>(qs + npad + 1);                            // [B]
+    int* cu_s = depth_s + B;                                                         // [B + 1]
+    __shared__ long long ws64[kWarps + 1];
+    __shared__ int ws32[kWarps + 1];
+    __shared__ Best wbest[kWarps];
+    __shared__ Best best_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // 1. prefix scores and sort keys
+    for (int i = tid; i < B; i += kThreads) {
+        float p = 1.0f;
+        for (int k = 0; k < gamma; ++k) {
+            p = __fmul_rn(p, clamp_conf(a.conf[(size_t)i * gamma + k]));
+            if (p == 0.0f) p = 0.0f;   // -0 -> +0
+            if (a.scores_out) a.scores_out[(size_t)i * gamma + k] = p;
+            const unsigned int bits = __float_as_uint(p);
+            keys[i * gamma + k] = ((unsigned long long)(0xffffffffu - bits) << 32) |
+                                  ((unsigned long long)k << 16) | (unsigned long long)i;
+        }
+    }
+    for (int r = n + tid; r < npad; r += kThreads) keys[r] = ~0ull;
+    for (int i = tid; i < B; i += kThreads) depth_s[i] = 0;
+    __syncthreads();
+
+    // 2. bitonic sort, ascending
+    for (int k = 2; k <= npad; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = tid; t < (npad >> 1); t += kThreads) {
+                const int i = 2 * t - (t & (j - 1));
+                const int l = i + j;
+                const bool up = (i & k) == 0;
+                const unsigned long long x = keys[i], y = keys[l];
+                if ((x > y) == up) {
+                    keys[i] = y;
+                    keys[l] = x;
+                }
+            }
+            __syncthreads();
+        }
+    }
+
+    // 3. fixed-point prefix sums Q[0..n]; ranks
+    {
+        const int per = (npad + kThreads - 1) / kThreads;
+        const int r0 = tid * per;
+        long long local = 0;
+        for (int e = 0; e < per; ++e) {
+            const int r = r0 + e;
+            if (r < n) {
+                const unsigned long long key = keys[r];
+                const float p = __uint_as_float(0xffffffffu - (unsigned int)(key >> 32));
+                local += __double2ll_rz((double)p * 1099511627776.0);
+                if (a.ranks_out) {
+                    const int i = (int)(key & 0xffffu), k = (int)((key >> 16) & 0xffffu);
+                    a.ranks_out[(size_t)i * gamma + k] = r;
+                }
+            }
+        }
+        long long total;
+        long long run = block_exclusive_scan<long long>(local, ws64, &total);
+        if (tid == 0) qs[0] = 0;
+        for (int e = 0; e < per; ++e) {
+            const int r = r0 + e;
+            if (r < n) {
+                const float p = __uint_as_float(0xffffffffu - (unsigned int)(keys[r] >> 32));
+                run += __double2ll_rz((double)p * 1099511627776.0);
+                qs[r + 1] = run;
+            }
+        }
+    }
+    __syncthreads();
+
+    // 4. objective over the candidates
+    {
+        const long long bfix = (long long)B << 40;
+        Best b = {-1.0, INT_MAX, -1};
+        const int n_cand = a.n_buckets > 0 ? a.n_buckets : n + 1;
+        for (int c = tid; c < n_cand; c += kThreads) {
+            int N;
+            float cost;
+            if (a.n_buckets > 0) {
+                N = a.bucket_K[c] - B;
+                cost = a.cost[c];
+            } else {
+                N = c;
+                cost = a.cost[B + N];
+            }
+            Best cur = {__ddiv_rn(__ll2double_rn(bfix + qs[N]), (double)cost), N, c};
+            if (better(cur, b)) b = cur;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            Best other;
+            other.obj = __shfl_xor_sync(0xffffffffu, b.obj, o);
+            other.N = __shfl_xor_sync(0xffffffffu, b.N, o);
+            other.cand = __shfl_xor_sync(0xffffffffu, b.cand, o);
+            if (better(other, b)) b = other;
+        }
+        if (lane == 0) wbest[warp] = b;
+        __syncthreads();
+        if (warp == 0) {
+            b = wbest[lane];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                Best other;
+                other.obj = __shfl_xor_sync(0xffffffffu, b.obj, o);
+                other.N = __shfl_xor_sync(0xffffffffu, b.N, o);
+                other.cand = __shfl_xor_sync(0xffffffffu, b.cand, o);
+                if (better(other, b)) b = other;
+            }
+            if (lane == 0) best_s = b;
+        }
+        __syncthreads();
+    }
+    const int n_star = best_s.N;
+
+    // 5. depths, cu_q, packed token metadata
+    for (int r = tid; r < n_star; r += kThreads) atomicAdd(&depth_s[(int)(keys[r] & 0xffffu)], 1);
+    __syncthreads();
+    {
+        const int per = (B + kThreads - 1) / kThreads;
+        const int i0 = tid * per;
+        int local = 0;
+        for (int e = 0; e < per; ++e)
+            if (i0 + e < B) local += 1 + depth_s[i0 + e];
+        int total;
+        int run = block_exclusive_scan<int>(local, ws32, &total);
+        for (int e = 0; e < per; ++e) {
+            const int i = i0 + e;
+            if (i < B) {
+                cu_s[i] = run;
+                a.cu_q[i] = run;
+                a.depths[i] = depth_s[i];
+                run += 1 + depth_s[i];
+            }
+        }
+        if (tid == 0) {
+            cu_s[B] = total;
+            a.cu_q[B] = total;
+        }
+    }
+    __syncthreads();
+    const int T = cu_s[B];
+    const int cap = B * (gamma + 1);
+    for (int idx = tid; idx < cap; idx += kThreads) {
+        const int i = idx / (gamma + 1), t = idx - i * (gamma + 1);
+        if (t <= depth_s[i]) {
+            const int pos = cu_s[i] + t;
+            if (a.tok_req) a.tok_req[pos] = i;
+            if (a.tok_pos) a.tok_pos[pos] = a.ctx_lens[i] + t;
+            if (a.tok_id) a.tok_id[pos] = (t == 0) ? a.bonus_ids[i] : a.draft_ids[(size_t)i * gamma + t - 1];
+        }
+        if (idx >= T) {
+            if (a.tok_req) a.tok_req[idx] = -1;
+            if (a.tok_pos) a.tok_pos[idx] = -1;
+            if (a.tok_id) a.tok_id[idx] = -1;
+        }
+    }
+    if (tid == 0 && a.info) {
+        dcut_select_info out;
+        out.n_star = n_star;
+        out.t_total = T;
+        out.candidate = best_s.cand;
+        out.reserved = 0;
+        out.sum_fixed = ((long long)B << 40) + qs[n_star];
+        out.objective = best_s.obj;
+        *a.info = out;
+    }
+}
+
+size_t select_smem_bytes(int B, int npad) {
+    return sizeof(unsigned long long) * (size_t)npad + sizeof(long long) * (size_t)(npad + 1) +
+           sizeof(int) * (size_t)(2 * B + 1) + 16;
+}
+
+}  // namespace
+
+// Per-device set-up: the selector may use up to ~192 KB of dynamic shared memory.
+dcut_status dcut_init_select(dcut_ctx* ctx) {
+    cudaError_t e = cudaFuncSetAttribute(dcut_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)select_smem_bytes(DCUT_MAX_KEYS, DCUT_MAX_KEYS));
+    return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(select)");
+}
+
+dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
+                               const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q,
+                               int* tok_req, int* tok_pos, int* tok_id, dcut_select_info* info,
+                               float* scores_out, int* ranks_out, cudaStream_t stream) {
+    const int n = B * gamma;
+    int npad = 32;
+    while (npad < n) npad <<= 1;
+    SelectArgs a;
+    a.conf = conf;
+    a.draft_ids = draft_ids;
+    a.bonus_ids = bonus_ids;
+    a.ctx_lens = ctx_lens;
+    a.cost = ctx->d_cost;
+    a.bucket_K = ctx->d_bucket_K;
+    a.n_buckets = ctx->n_buckets;
+    a.B = B;
+    a.gamma = gamma;
+    a.npad = npad;
+    a.depths = depths;
+    a.cu_q = cu_q;
+    a.tok_req = tok_req;
+    a.tok_pos = tok_pos;
+    a.tok_id = tok_id;
+    a.info = info;
+    a.scores_out = scores_out;
+    a.ranks_out = ranks_out;
+    const size_t smem = select_smem_bytes(B, npad);
+    dcut_select_kernel<<<1, kThreads, smem, stream>>>(a);
+    return dcut_check_cuda(ctx, cudaGetLastError(), "launch dcut_select_kernel");
+}

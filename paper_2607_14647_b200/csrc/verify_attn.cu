@@ -1,0 +1,700 @@
+// dcut_verify_attn: ragged causal multi-token attention over a paged bf16 KV cache.
+//
+// HBM-bound by design: every K/V byte of every request is read once per step, so the kernel is
+// organised around keeping ~100 KB of page loads in flight per SM and doing the (small) matrix
+// work out of shared memory on the warp-level tensor-core path.
+//
+//   attn_plan_kernel     one CTA.  Cuts every request's page list into near-equal chunks so the
+//                        batch gives a few work items per SM (flash-decoding split-KV); an item is
+//                        one (request, kv head, page range).
+//   attn_split_kernel    one CTA per item: 15 consumer warps + 1 producer warp.
+//       producer         reads the block table and issues TMA tile loads (2-D tensor map over the
+//                        cache seen as [rows of one token, head_dim], 128-byte swizzle) into a ring
+//                        of page stages, each guarded by a full/empty mbarrier pair.
+//       consumers        the item's query tile is (1 + d_i) * group rows (every query token of the
+//                        request times the q heads sharing this kv head), cut into 16-row m-tiles.
+//                        Warp w owns m-tile (w mod MT) and page slot (w div MT): it runs
+//                        S = Q K^T, online softmax and O += P V for its m-tile on every
+//                        nslots-th page (mma.sync m16n8k16 bf16, fp32 accumulate, ldmatrix from the
+//                        swizzled tiles).  Small query tiles therefore spread pages over warps,
+//                        large ones spread rows.
+//       epilogue         the slots' (m, l, O) are merged through shared memory; a request with one
+//                        chunk writes bf16 output directly, otherwise normalised fp32 partials + LSE.
+//   attn_combine_kernel  merges the chunks of multi-chunk requests.
+//
+// Every mbarrier wait is bounded; on expiry the CTA sets the device status word and leaves.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "dcut_internal.h"
+
+namespace {
+
+constexpr int kConsumerWarps = 15;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kThreads = kConsumerThreads + 32;
+constexpr int kStages = 17;
+constexpr int kPage = 16;          // tokens per page
+constexpr int kMaxMTiles = 9;      // query rows per item <= 144
+constexpr int kPlanThreads = 1024;
+constexpr long long kSpinLimit = 1ll << 22;
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait: false if the phase did not complete within the spin limit
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (long long it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 4096) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void consumer_bar() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+}
+
+// byte offset of 16-byte chunk `c16` (0 .. DH/8-1) of token/row `r` (0..15) inside a swizzled
+// [DH/64][16][64] bf16 tile (what two 64-column TMA boxes with 128-byte swizzle produce)
+__device__ __forceinline__ uint32_t tile_off(int r, int c16) {
+    return (uint32_t)(((c16 >> 3) << 11) + (r << 7) + (((c16 & 7) ^ (r & 7)) << 4));
+}
+
+// ------------------------------------------------------------------------------------------------
+// plan
+
+struct PlanArgs {
+    const int* ctx_lens;
+    const int* cu_q;
+    int B, n_q_heads, n_kv_heads;
+    int target_items, min_chunk_pages, max_items;
+    long long part_rows_cap;
+    AttnItem* items;
+    int* plan;       // [0] n_items, [1] chunk_pages, [2] total_pages, [3] partial rows used
+    int* req_part;   // [B][2]: first partial row, n_chunks
+};
+
+template <typename T>
+__device__ __forceinline__ T plan_warp_scan(T v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        T u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += u;
+    }
+    return v;
+}
+
+__device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = plan_warp_scan(v, lane);
+    if (lane == 31) ws[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = ws[lane];
+        int winc = plan_warp_scan(w, lane);
+        ws[lane] = winc - w;
+        if (lane == 31) ws[32] = winc;
+    }
+    __syncthreads();
+    int res = ws[warp] + inc - v;
+    *total = ws[32];
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
+    __shared__ int ws[33];
+    const int tid = threadIdx.x;
+    const int per = (a.B + kPlanThreads - 1) / kPlanThreads;
+    const int i0 = tid * per;
+    int local = 0;
+    for (int e = 0; e < per; ++e) {
+        const int i = i0 + e;
+        if (i < a.B) {
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            local += (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+        }
+    }
+    int total_pages;
+    plan_block_exclusive_scan(local, ws, &total_pages);
+    long long units = (long long)total_pages * a.n_kv_heads;
+    int chunk_pages = (int)((units + a.target_items - 1) / a.target_items);
+    if (chunk_pages < a.min_chunk_pages) chunk_pages = a.min_chunk_pages;
+
+    int my_items = 0, my_rows = 0;
+    for (int e = 0; e < per; ++e) {
+        const int i = i0 + e;
+        if (i < a.B) {
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+            const int nc = (pages + chunk_pages - 1) / chunk_pages;
+            my_items += nc * a.n_kv_heads;
+            if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
+        }
+    }
+    int n_items, n_rows;
+    int item_off = plan_block_exclusive_scan(my_items, ws, &n_items);
+    int row_off = plan_block_exclusive_scan(my_rows, ws, &n_rows);
+    const bool overflow = n_items > a.max_items || (long long)n_rows > a.part_rows_cap;
+    if (tid == 0) {
+        a.plan[0] = overflow ? 0 : n_items;
+        a.plan[1] = chunk_pages;
+        a.plan[2] = total_pages;
+        a.plan[3] = n_rows;
+        a.plan[4] = overflow ? 1 : 0;
+    }
+    if (overflow) return;
+    const int group = a.n_q_heads / a.n_kv_heads;
+    for (int e = 0; e < per; ++e) {
+        const int i = i0 + e;
+        if (i < a.B) {
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+            const int nc = (pages + chunk_pages - 1) / chunk_pages;
+            const int cp = (pages + nc - 1) / nc;   // near-equal chunks
+            const int M = (d + 1) * group;
+            a.req_part[2 * i] = row_off;
+            a.req_part[2 * i + 1] = nc;
+            for (int c = 0; c < nc; ++c)
+                for (int h = 0; h < a.n_kv_heads; ++h) {
+                    AttnItem it;
+                    it.req = i;
+                    it.kv_head = h;
+                    it.page_begin = c * cp;
+                    it.page_end = min(pages, (c + 1) * cp);
+                    it.chunk = c;
+                    it.n_chunks = nc;
+                    it.part_row = nc > 1 ? row_off + (c * a.n_kv_heads + h) * M : -1;
+                    it.pad = 0;
+                    a.items[item_off + c * a.n_kv_heads + h] = it;
+                }
+            item_off += nc * a.n_kv_heads;
+            if (nc > 1) row_off += nc * (d + 1) * a.n_q_heads;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// split-KV attention
+
+struct AttnArgs {
+    const __nv_bfloat16* q;
+    const int* block_table;
+    int block_table_stride;
+    const int* ctx_lens;
+    const int* cu_q;
+    const AttnItem* items;
+    const int* plan;
+    int n_q_heads, n_kv_heads;
+    long long num_pages;
+    float scale_log2;          // softmax scale * log2(e)
+    __nv_bfloat16* out;
+    float* lse;                // [T, Hq] or null
+    float* part_o;
+    float* part_lse;
+    int* status;
+};
+
+template <int DH>
+struct SmemLayout {
+    static constexpr int kHalves = DH / 64;
+    static constexpr int kPageBytes = kPage * DH * 2;            // one K or V page tile
+    static constexpr int kStageBytes = 2 * kPageBytes;
+    static constexpr int kRingBytes = kStages * kStageBytes;
+    static constexpr int kQBytes = kMaxMTiles * 16 * DH * 2;
+    static constexpr int kMergeStride = DH + 8;                  // floats per merged row
+    static constexpr int kMergeBytes = kConsumerWarps * 16 * kMergeStride * 4;
+    static constexpr int kMLBytes = kConsumerWarps * 16 * 2 * 4;
+    static constexpr int kBarBytes = 2 * kStages * 8;
+    static constexpr int kRingOrMerge = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;
+    static constexpr int kTotal = kRingOrMerge + kQBytes + kMLBytes + kBarBytes + 1024 /* alignment slack */;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, AttnArgs a) {
+    using L = SmemLayout<DH>;
+    if ((int)blockIdx.x >= a.plan[0]) return;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* ring = smem;
+    unsigned char* q_s = smem + L::kRingOrMerge;
+    float* ml_s = reinterpret_cast<float*>(q_s + L::kQBytes);
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(ml_s) + L::kMLBytes);
+    __shared__ int abort_s;
+
+    const AttnItem item = a.items[blockIdx.x];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int req = item.req, kvh = item.kv_head;
+    const int group = a.n_q_heads / a.n_kv_heads;
+    const int q0 = a.cu_q[req];
+    const int depth = a.cu_q[req + 1] - q0 - 1;
+    const int ctx_len = a.ctx_lens[req];
+    const int M = (depth + 1) * group;
+    const int MT = (M + 15) >> 4;
+    const int nslots = kConsumerWarps / MT;
+    const int n_pages = item.page_end - item.page_begin;
+
+    const uint32_t full_bar = smem_u32(bars);
+    const uint32_t empty_bar = smem_u32(bars + kStages);
+    if (tid == 0) {
+        abort_s = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, MT);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ---------------------------------------------------------------- producer warp
+        const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
+        int my_page = 0;
+        for (int p = 0; p < n_pages; ++p) {
+            if ((p & 31) == 0) my_page = (p + lane < n_pages) ? bt[p + lane] : 0;
+            int page_id = __shfl_sync(0xffffffffu, my_page, p & 31);
+            const int stage = p % kStages;
+            int ok = 1;
+            if (lane == 0) {
+                if (p >= kStages) ok = mbar_wait(empty_bar + 8 * stage, ((p / kStages) - 1) & 1) ? 1 : 0;
+                if (ok && *(volatile int*)&abort_s) ok = 0;
+                if (ok) {
+                    if (page_id < 0 || page_id >= a.num_pages) {
+                        atomicExch(a.status, DCUT_DEV_BAD_PAGE);
+                        page_id = 0;
+                    }
+                    const uint32_t bar = full_bar + 8 * stage;
+                    const uint32_t dst = smem_u32(ring + stage * L::kStageBytes);
+                    const int row = (page_id * a.n_kv_heads + kvh) * kPage;
+                    mbar_arrive_expect_tx(bar, L::kStageBytes);
+#pragma unroll
+                    for (int h = 0; h < L::kHalves; ++h) {
+                        tma_load_2d(dst + h * 2048, &k_map, h * 64, row, bar);
+                        tma_load_2d(dst + L::kPageBytes + h * 2048, &v_map, h * 64, row, bar);
+                    }
+                } else {
+                    atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
+                    *(volatile int*)&abort_s = 1;
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+        }
+        return;
+    }
+
+    // -------------------------------------------------------------------- consumer warps
+    // stage the query tile: row R = t * group + hl  <->  q[(q0 + t), kvh * group + hl, :]
+    {
+        constexpr int kChunks = DH / 8;
+        const int rows_padded = MT * 16;
+        for (int idx = tid; idx < rows_padded * kChunks; idx += kConsumerThreads) {
+            const int R = idx / kChunks, c16 = idx - R * kChunks;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (R < M) {
+                const int t = R / group, hl = R - t * group;
+                v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * DH + c16 * 8);
+            }
+            *reinterpret_cast<uint4*>(q_s + (R >> 4) * (16 * DH * 2) + tile_off(R & 15, c16)) = v;
+        }
+    }
+    consumer_bar();
+
+    const int mt = warp % MT, slot = warp / MT;
+    const bool active = slot < nslots;
+    float o[DH / 8][4];
+#pragma unroll
+    for (int j = 0; j < DH / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.0f, 0.0f};
+    bool aborted = false;
+
+    if (active) {
+        uint32_t qf[DH / 16][4];
+        {
+            const int mat = lane >> 3;
+            const int r = ((mat & 1) << 3) + (lane & 7);
+            const uint32_t qbase = smem_u32(q_s + mt * (16 * DH * 2));
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks) ldmatrix_x4(qbase + tile_off(r, 2 * ks + (mat >> 1)), qf[ks]);
+        }
+        // causal limit per row: query token t sees cache positions j <= ctx_len + t
+        const int R_lo = mt * 16 + (lane >> 2), R_hi = R_lo + 8;
+        const int jmax_lo = ctx_len + min(R_lo, M - 1) / group;
+        const int jmax_hi = ctx_len + min(R_hi, M - 1) / group;
+        // per-lane ldmatrix row/chunk selectors
+        const int kmat = lane >> 3;
+        const int k_tok = ((kmat >> 1) << 3) + (lane & 7);
+        const int k_chunk = kmat & 1;
+        const int v_tok = ((kmat & 1) << 3) + (lane & 7);
+        const int v_chunk = kmat >> 1;
+
+        for (int p = slot; p < n_pages; p += nslots) {
+            const int stage = p % kStages;
+            if (!mbar_wait(full_bar + 8 * stage, (p / kStages) & 1)) {
+                aborted = true;
+                break;
+            }
+            const uint32_t k_base = smem_u32(ring + stage * L::kStageBytes);
+            const uint32_t v_base = k_base + L::kPageBytes;
+
+            float s[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.0f;
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks) {
+                uint32_t kf[4];
+                ldmatrix_x4(k_base + tile_off(k_tok, 2 * ks + k_chunk), kf);
+                mma_bf16(s[0], qf[ks], kf[0], kf[1]);
+                mma_bf16(s[1], qf[ks], kf[2], kf[3]);
+            }
+            // scale to the log2 domain, mask
+            const int j0 = (item.page_begin + p) * kPage + ((lane & 3) << 1);
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int j = j0 + nt * 8 + (e & 1);
+                    const int jmax = (e < 2) ? jmax_lo : jmax_hi;
+                    s[nt][e] = (j <= jmax) ? s[nt][e] * a.scale_log2 : -INFINITY;
+                }
+            }
+            // online softmax for the two rows this thread holds
+            float mx[2] = {fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])),
+                           fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]))};
+            float alpha[2], msafe[2];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+                const float m_new = fmaxf(m_run[r], mx[r]);
+                msafe[r] = (m_new == -INFINITY) ? 0.0f : m_new;
+                alpha[r] = exp2f(m_run[r] - msafe[r]);
+                m_run[r] = m_new;
+            }
+            float ps[2][4];
+#pragma unroll
+            for (int nt = 0; nt < 2; ++nt) {
+                ps[nt][0] = exp2f(s[nt][0] - msafe[0]);
+                ps[nt][1] = exp2f(s[nt][1] - msafe[0]);
+                ps[nt][2] = exp2f(s[nt][2] - msafe[1]);
+                ps[nt][3] = exp2f(s[nt][3] - msafe[1]);
+            }
+            l_run[0] = l_run[0] * alpha[0] + (ps[0][0] + ps[0][1] + ps[1][0] + ps[1][1]);
+            l_run[1] = l_run[1] * alpha[1] + (ps[0][2] + ps[0][3] + ps[1][2] + ps[1][3]);
+            if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
+#pragma unroll
+                for (int j = 0; j < DH / 8; ++j) {
+                    o[j][0] *= alpha[0];
+                    o[j][1] *= alpha[0];
+                    o[j][2] *= alpha[1];
+                    o[j][3] *= alpha[1];
+                }
+            }
+            uint32_t pf[4] = {pack_bf16(ps[0][0], ps[0][1]), pack_bf16(ps[0][2], ps[0][3]),
+                              pack_bf16(ps[1][0], ps[1][1]), pack_bf16(ps[1][2], ps[1][3])};
+#pragma unroll
+            for (int jj = 0; jj < DH / 16; ++jj) {
+                uint32_t vf[4];
+                ldmatrix_x4_trans(v_base + tile_off(v_tok, 2 * jj + v_chunk), vf);
+                mma_bf16(o[2 * jj], pf, vf[0], vf[1]);
+                mma_bf16(o[2 * jj + 1], pf, vf[2], vf[3]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+        }
+    }
+    if (aborted) {
+        atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
+        *(volatile int*)&abort_s = 1;
+    }
+
+    // -------------------------------------------------------------------- merge the slots
+    consumer_bar();   // every page has been consumed: the ring can be reused
+    float* merge = reinterpret_cast<float*>(ring);
+    if (active) {
+        float* mo = merge + (size_t)warp * 16 * L::kMergeStride;
+        const int r_lo = lane >> 2, c0 = (lane & 3) << 1;
+#pragma unroll
+        for (int j = 0; j < DH / 8; ++j) {
+            *reinterpret_cast<float2*>(mo + r_lo * L::kMergeStride + j * 8 + c0) = make_float2(o[j][0], o[j][1]);
+            *reinterpret_cast<float2*>(mo + (r_lo + 8) * L::kMergeStride + j * 8 + c0) = make_float2(o[j][2], o[j][3]);
+        }
+        if ((lane & 3) == 0) {
+            ml_s[(warp * 16 + r_lo) * 2] = m_run[0];
+            ml_s[(warp * 16 + r_lo) * 2 + 1] = l_run[0];
+            ml_s[(warp * 16 + r_lo + 8) * 2] = m_run[1];
+            ml_s[(warp * 16 + r_lo + 8) * 2 + 1] = l_run[1];
+        }
+    }
+    consumer_bar();
+    if (*(volatile int*)&abort_s) return;
+    {
+        constexpr int kVec = DH / 4;   // float4 per row
+        for (int idx = tid; idx < M * kVec; idx += kConsumerThreads) {
+            const int R = idx / kVec, c4 = idx - R * kVec;
+            const int tile = R >> 4, r = R & 15;
+            float m_all = -INFINITY;
+            for (int sl = 0; sl < nslots; ++sl) m_all = fmaxf(m_all, ml_s[((sl * MT + tile) * 16 + r) * 2]);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            float l_all = 0.0f;
+            for (int sl = 0; sl < nslots; ++sl) {
+                const int w = sl * MT + tile;
+                const float m_w = ml_s[(w * 16 + r) * 2];
+                const float wgt = (m_w == -INFINITY) ? 0.0f : exp2f(m_w - m_all);
+                l_all += wgt * ml_s[(w * 16 + r) * 2 + 1];
+                const float4 v = *reinterpret_cast<const float4*>(merge + ((size_t)w * 16 + r) * L::kMergeStride + c4 * 4);
+                acc.x += wgt * v.x;
+                acc.y += wgt * v.y;
+                acc.z += wgt * v.z;
+                acc.w += wgt * v.w;
+            }
+            const float inv = l_all > 0.0f ? 1.0f / l_all : 0.0f;
+            acc.x *= inv;
+            acc.y *= inv;
+            acc.z *= inv;
+            acc.w *= inv;
+            const float lse_nat = l_all > 0.0f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+            const int t = R / group, hl = R - t * group;
+            const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+            if (item.n_chunks == 1) {
+                uint2 pk;
+                pk.x = pack_bf16(acc.x, acc.y);
+                pk.y = pack_bf16(acc.z, acc.w);
+                *reinterpret_cast<uint2*>(a.out + orow * DH + c4 * 4) = pk;
+                if (a.lse && c4 == 0) a.lse[orow] = lse_nat;
+            } else {
+                const size_t prow = (size_t)item.part_row + R;
+                *reinterpret_cast<float4*>(a.part_o + prow * DH + c4 * 4) = acc;
+                if (c4 == 0) a.part_lse[prow] = lse_nat;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// combine the chunks of multi-chunk requests: one warp per (token, q head)
+
+struct CombineArgs {
+    const int* cu_q;
+    const int* req_part;
+    const float* part_o;
+    const float* part_lse;
+    const int* plan;
+    int B, n_q_heads, n_kv_heads;
+    __nv_bfloat16* out;
+    float* lse;
+};
+
+template <int DH>
+__global__ void __launch_bounds__(256) attn_combine_kernel(CombineArgs a) {
+    if (a.plan[4]) return;
+    const int T = a.cu_q[a.B];
+    const int gw = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
+    const int lane = threadIdx.x & 31;
+    if (gw >= T * a.n_q_heads) return;
+    const int tok = gw / a.n_q_heads, h = gw - tok * a.n_q_heads;
+    int lo = 0, hi = a.B;   // request with cu_q[i] <= tok < cu_q[i+1]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (a.cu_q[mid] <= tok) lo = mid; else hi = mid;
+    }
+    const int req = lo;
+    const int nc = a.req_part[2 * req + 1];
+    if (nc <= 1) return;
+    const int group = a.n_q_heads / a.n_kv_heads;
+    const int q0 = a.cu_q[req];
+    const int M = (a.cu_q[req + 1] - q0) * group;
+    const int kvh = h / group;
+    const int R = (tok - q0) * group + (h - kvh * group);
+    const size_t base = (size_t)a.req_part[2 * req];
+    float m_all = -INFINITY;
+    for (int c = 0; c < nc; ++c) m_all = fmaxf(m_all, a.part_lse[base + (size_t)(c * a.n_kv_heads + kvh) * M + R]);
+    constexpr int kPer = DH / 32;
+    float acc[kPer];
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) acc[e] = 0.0f;
+    float wsum = 0.0f;
+    for (int c = 0; c < nc; ++c) {
+        const size_t prow = base + (size_t)(c * a.n_kv_heads + kvh) * M + R;
+        const float l = a.part_lse[prow];
+        const float w = (l == -INFINITY) ? 0.0f : __expf(l - m_all);
+        wsum += w;
+        const float* po = a.part_o + prow * DH + lane * kPer;
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) acc[e] += w * po[e];
+    }
+    const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+    __nv_bfloat16* op = a.out + ((size_t)tok * a.n_q_heads + h) * DH + lane * kPer;
+#pragma unroll
+    for (int e = 0; e < kPer; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+    if (a.lse && lane == 0) a.lse[(size_t)tok * a.n_q_heads + h] = wsum > 0.0f ? m_all + logf(wsum) : -INFINITY;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+dcut_status make_cache_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, long long num_pages) {
+    const int DH = ctx->lim.head_dim;
+    cuuint64_t dims[2] = {(cuuint64_t)DH, (cuuint64_t)num_pages * ctx->lim.n_kv_heads * kPage};
+    cuuint64_t strides[1] = {(cuuint64_t)DH * 2};
+    cuuint32_t box[2] = {64, kPage};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return dcut_fail(ctx, DCUT_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+    return DCUT_OK;
+}
+
+template <int DH>
+dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm, const AttnArgs& aa,
+                     const CombineArgs& ca, int T_cap, cudaStream_t stream) {
+    attn_split_kernel<DH><<<ctx->max_items, kThreads, SmemLayout<DH>::kTotal, stream>>>(km, vm, aa);
+    dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_split_kernel");
+    if (st != DCUT_OK) return st;
+    const long long warps = (long long)T_cap * ctx->lim.n_q_heads;
+    const int blocks = (int)((warps + 7) / 8);
+    attn_combine_kernel<DH><<<blocks, 256, 0, stream>>>(ca);
+    return dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_combine_kernel");
+}
+
+}  // namespace
+
+dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
+    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SmemLayout<128>::kTotal);
+    if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 128)");
+    e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             SmemLayout<64>::kTotal);
+    if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 64)");
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+        return dcut_fail(ctx, DCUT_ECUDA, "cuTensorMapEncodeTiled entry point not available");
+    ctx->encode_tiled = fn;
+    return DCUT_OK;
+}
+
+dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
+                                    long long num_pages, const int* block_table, int block_table_stride,
+                                    const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
+                                    void* out, float* lse, cudaStream_t stream) {
+    CUtensorMap km, vm;
+    dcut_status st = make_cache_map(ctx, &km, k_cache, num_pages);
+    if (st != DCUT_OK) return st;
+    st = make_cache_map(ctx, &vm, v_cache, num_pages);
+    if (st != DCUT_OK) return st;
+
+    PlanArgs pa;
+    pa.ctx_lens = ctx_lens;
+    pa.cu_q = cu_q;
+    pa.B = B;
+    pa.n_q_heads = ctx->lim.n_q_heads;
+    pa.n_kv_heads = ctx->lim.n_kv_heads;
+    pa.target_items = ctx->target_items;
+    pa.min_chunk_pages = 8;
+    pa.max_items = ctx->max_items;
+    pa.part_rows_cap = ctx->part_rows_cap;
+    pa.items = ctx->d_items;
+    pa.plan = ctx->d_plan;
+    pa.req_part = ctx->d_req_part;
+    attn_plan_kernel<<<1, kPlanThreads, 0, stream>>>(pa);
+    st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_plan_kernel");
+    if (st != DCUT_OK) return st;
+
+    AttnArgs aa;
+    aa.q = static_cast<const __nv_bfloat16*>(q);
+    aa.block_table = block_table;
+    aa.block_table_stride = block_table_stride;
+    aa.ctx_lens = ctx_lens;
+    aa.cu_q = cu_q;
+    aa.items = ctx->d_items;
+    aa.plan = ctx->d_plan;
+    aa.n_q_heads = ctx->lim.n_q_heads;
+    aa.n_kv_heads = ctx->lim.n_kv_heads;
+    aa.num_pages = num_pages;
+    aa.scale_log2 = scale * 1.4426950408889634f;
+    aa.out = static_cast<__nv_bfloat16*>(out);
+    aa.lse = lse;
+    aa.part_o = ctx->d_part_o;
+    aa.part_lse = ctx->d_part_lse;
+    aa.status = ctx->d_status;
+
+    CombineArgs ca;
+    ca.cu_q = cu_q;
+    ca.req_part = ctx->d_req_part;
+    ca.part_o = ctx->d_part_o;
+    ca.part_lse = ctx->d_part_lse;
+    ca.plan = ctx->d_plan;
+    ca.B = B;
+    ca.n_q_heads = ctx->lim.n_q_heads;
+    ca.n_kv_heads = ctx->lim.n_kv_heads;
+    ca.out = static_cast<__nv_bfloat16*>(out);
+    ca.lse = lse;
+
+    if (ctx->lim.head_dim == 128) return launch_t<128>(ctx, km, vm, aa, ca, T_cap, stream);
+    return launch_t<64>(ctx, km, vm, aa, ca, T_cap, stream);
+}

@@ -1,0 +1,143 @@
+"""dcut_verify_attn against the oracle: |err| <= 1e-2 + 1e-2 |ref| element by element on small
+cases spanning several tiles and ragged tails, and on sampled rows at the full workload sizes."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dcut_oracle as orc
+from paper_2607_14647_b200 import workloads as wl
+from tests.gpu_helpers import attn_tolerance_ok, dev, make_ctx
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, sel, kv, depths, want_lse=True):
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req)
+    q = wl.q_rows(cfg, depths)
+    cu = wl.cu_q_from_depths(depths)
+    T = int(cu[-1])
+    lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device="cuda") if want_lse else None
+    out = ctx.verify_attn(dev(q), dev(kv.k_cache), dev(kv.v_cache), dev(kv.block_table), dev(sel.ctx_lens), dev(cu),
+                          cfg.t_cap, lse=lse)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    ctx.close()
+    return q, cu, out.float().cpu().numpy(), None if lse is None else lse.cpu().numpy()
+
+
+def _full_compare(cfg, sel, kv, depths):
+    q, cu, out, lse = _run(cfg, sel, kv, depths)
+    ref, ref_lse = orc.verify_attn(q, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, cu,
+                                   cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.page_size)
+    ok, worst = attn_tolerance_ok(out, ref)
+    assert ok, f"worst err/limit {worst}"
+    np.testing.assert_allclose(lse, ref_lse, rtol=2e-3, atol=2e-3)
+    return worst
+
+
+@pytest.mark.parametrize("depths", [[16, 16, 16, 16], [0, 0, 0, 0], [0, 3, 16, 7], [1, 2, 4, 15]])
+def test_tiny_config_every_element(depths):
+    cfg = wl.config(0)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    _full_compare(cfg, sel, kv, np.array(depths, np.int32))
+
+
+@pytest.mark.parametrize("shape", [dict(n_q_heads=32, n_kv_heads=8, head_dim=128), dict(n_q_heads=16, n_kv_heads=2, head_dim=128),
+                                   dict(n_q_heads=8, n_kv_heads=8, head_dim=64), dict(n_q_heads=6, n_kv_heads=2, head_dim=64)])
+def test_mid_size_every_element(shape):
+    """Contexts from 1 to ~1500 tokens: single-page requests, many chunks, ragged last pages."""
+    cfg = wl.custom_config(B=12, gamma=16, ctx_lo=0, ctx_hi=1500, **shape)
+    sel = wl.select_inputs(cfg)
+    sel.ctx_lens[:4] = [0, 1, 15, 16]                       # degenerate and page-boundary contexts
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    rng = np.random.default_rng(1)
+    for depths in (rng.integers(0, 17, cfg.B).astype(np.int32), np.full(cfg.B, 16, np.int32), np.zeros(cfg.B, np.int32)):
+        _full_compare(cfg, sel, kv, depths)
+
+
+def test_unused_slots_are_never_read():
+    cfg = wl.custom_config(B=6, gamma=16, n_q_heads=8, n_kv_heads=2, head_dim=128, ctx_lo=10, ctx_hi=300)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    depths = np.array([0, 5, 16, 2, 9, 1], np.int32)
+    for i in range(cfg.B):                                  # poison everything past the deepest kept position
+        n_slots = ((int(sel.ctx_lens[i]) + cfg.gamma + 1 + 15) // 16) * 16
+        for j in range(int(sel.ctx_lens[i]) + int(depths[i]) + 1, n_slots):
+            kv.k_cache[kv.block_table[i, j // 16], :, j % 16] = 3.0e4
+            kv.v_cache[kv.block_table[i, j // 16], :, j % 16] = 3.0e4
+    _full_compare(cfg, sel, kv, depths)
+
+
+def _sampled_compare(cfg, sel, kv, depths, n_samples, seed=0):
+    q, cu, out, lse = _run(cfg, sel, kv, depths)
+    T = int(cu[-1])
+    rng = np.random.default_rng(seed)
+    tok = rng.integers(0, T, n_samples).astype(np.int32)
+    head = rng.integers(0, cfg.n_q_heads, n_samples).astype(np.int32)
+    # always include the first and last token of the longest and the shortest request
+    order = np.argsort(sel.ctx_lens)
+    extra = [cu[order[0]], cu[order[0] + 1] - 1, cu[order[-1]], cu[order[-1] + 1] - 1]
+    tok[: len(extra)] = extra
+    ref, ref_lse = orc.verify_attn(q, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, cu, cfg.n_q_heads,
+                                   cfg.n_kv_heads, cfg.head_dim, cfg.page_size, sample_tok=tok, sample_head=head)
+    ok, worst = attn_tolerance_ok(out[tok, head], ref)
+    assert ok, f"worst err/limit {worst}"
+    np.testing.assert_allclose(lse[tok, head], ref_lse, rtol=2e-3, atol=2e-3)
+    assert np.isfinite(out).all()
+
+
+def _pruned_depths(cfg, sel):
+    return orc.select(sel.conf, sel.draft_ids, sel.bonus_ids, sel.ctx_lens,
+                      wl.cost_table_linear(cfg.t_cap + 1, 0.2, 0.0006)).depths
+
+
+@pytest.mark.parametrize("idx", [1, 2])
+def test_full_size_configs_sampled(idx):
+    cfg = wl.config(idx)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    for depths in (_pruned_depths(cfg, sel), np.full(cfg.B, cfg.gamma, np.int32), np.zeros(cfg.B, np.int32)):
+        _sampled_compare(cfg, sel, kv, depths, 192)
+
+
+def test_b256_long_tail_sampled():
+    cfg = wl.config(3)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    _sampled_compare(cfg, sel, kv, _pruned_depths(cfg, sel), 160)
+    _sampled_compare(cfg, sel, kv, np.full(cfg.B, cfg.gamma, np.int32), 96, seed=1)
+
+
+def test_repeated_runs_are_bit_identical():
+    cfg = wl.custom_config(B=8, gamma=16, n_q_heads=32, n_kv_heads=8, head_dim=128, ctx_lo=100, ctx_hi=3000)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    depths = np.array([3, 16, 0, 8, 12, 1, 5, 16], np.int32)
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req)
+    args = (dev(wl.q_rows(cfg, depths)), dev(kv.k_cache), dev(kv.v_cache), dev(kv.block_table), dev(sel.ctx_lens),
+            dev(wl.cu_q_from_depths(depths)), cfg.t_cap)
+    first = ctx.verify_attn(*args).clone()
+    for _ in range(10):
+        assert torch.equal(ctx.verify_attn(*args), first)
+    ctx.close()
+
+
+def test_argument_errors():
+    from paper_2607_14647_b200 import binding
+    cfg = wl.config(0)
+    with pytest.raises(binding.DcutError) as e:
+        binding.Context(max_B=4, max_gamma=16, n_q_heads=4, n_kv_heads=1, head_dim=96, max_pages_per_req=4)
+    assert e.value.status == binding.EINVAL
+    with pytest.raises(binding.DcutError) as e:
+        binding.Context(max_B=4, max_gamma=16, n_q_heads=32, n_kv_heads=2, head_dim=128, max_pages_per_req=4)
+    assert e.value.status == binding.ECAPACITY                 # 17 * 16 query rows per kv head
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req - 1)
+    depths = np.zeros(cfg.B, np.int32)
+    with pytest.raises(binding.DcutError) as e:
+        ctx.verify_attn(dev(wl.q_rows(cfg, depths)), dev(kv.k_cache), dev(kv.v_cache), dev(kv.block_table),
+                        dev(sel.ctx_lens), dev(wl.cu_q_from_depths(depths)), cfg.t_cap)
+    assert e.value.status == binding.ECAPACITY
+    ctx.close()
