@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the D-cut verify hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl dcut|reference] [--config 2]
+
+A step is one pass of the whole hot path over one batch of synthetic input: dcut_select ->
+dcut_verify_attn -> dcut_accept.  The headline value is accepted tokens/s of the D-cut-pruned arm
+at B = 64 (workload 2); the full-gamma and gamma = 0 arms, the attention roofline, the end-to-end
+number from host buffers and the CPU oracle's throughput ride along in the same JSON line.
+
+`--impl reference` times the CPU oracle (test infrastructure, run as it stands) on a bounded
+sample of the same workload.  With N > 1 every rank runs an independent replica of the workload
+(the path has no cross-GPU exchange); the value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_14647_b200 import workloads as wl  # noqa: E402
+
+METRIC = "accepted_tokens_per_s_per_verify_step_B64"
+UNIT = "tokens/s"
+L2_BYTES = 126e6
+# DRAM bytes per algorithmic byte of attn_split_kernel measured with ncu (profiles/); None until captured
+ATTN_TRAFFIC_RATIO = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="dcut", choices=["dcut", "reference"])
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--cost-points", type=int, default=18)
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------ helpers
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.path = tempfile.mktemp(prefix="dcut_clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [r.strip().split(",") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.strip().lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return world, rank, local
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    """The slowest rank's value (the only cross-rank exchange of the benchmark)."""
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda" if dist.get_backend() == "nccl" else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
+
+
+def attn_algorithmic_bytes(cfg, ctx_lens: np.ndarray, depths: np.ndarray) -> int:
+    """K and V of every visible cache position once, Q read, O written, block-table entries."""
+    kv_tokens = int((ctx_lens.astype(np.int64) + depths + 1).sum())
+    T = int((depths.astype(np.int64) + 1).sum())
+    pages = int(((ctx_lens.astype(np.int64) + depths + 1 + cfg.page_size - 1) // cfg.page_size).sum())
+    return (kv_tokens * cfg.n_kv_heads * cfg.head_dim * 2 * 2 + 2 * T * cfg.n_q_heads * cfg.head_dim * 2
+            + pages * 4 * cfg.n_kv_heads)
+
+
+def peaks() -> dict:
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample(cfg, sel, kv, q_all, logits_all, cost, seconds: float):
+    """Times the oracle, as it stands, on a bounded sample: selection for the whole batch, then
+    attention and acceptance request by request until `seconds` of CPU time are used."""
+    from oracle import dcut_oracle as orc
+    t0 = time.perf_counter()
+    r = orc.select(sel.conf, sel.draft_ids, sel.bonus_ids, sel.ctx_lens, cost)
+    done, accepted = 0, 0
+    for i in range(cfg.B):
+        d = int(r.depths[i])
+        cu1 = np.array([0, d + 1], np.int32)
+        orc.verify_attn(q_all[i, : d + 1].contiguous(), kv.k_cache, kv.v_cache, kv.block_table[i: i + 1],
+                        sel.ctx_lens[i: i + 1], cu1, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.page_size)
+        a = orc.accept(logits_all[i, : d + 1].contiguous(), sel.draft_ids[i: i + 1], cu1, cfg.gamma)
+        accepted += a.n_accepted_total
+        done += 1
+        if time.perf_counter() - t0 > seconds:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": accepted / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"selection for all {cfg.B} requests, attention + acceptance for the first {done} of {cfg.B} "
+                      f"requests ({accepted} accepted tokens in {dt:.1f} s)"}, dt, done, accepted
+
+
+def host_inputs(cfg):
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    full = np.full(cfg.B, cfg.gamma, np.int32)
+    q_all = wl.q_rows(cfg, full).view(cfg.B, cfg.gamma + 1, cfg.n_q_heads, cfg.head_dim)
+    logits_all = wl.logits_rows(cfg, sel, full).view(cfg.B, cfg.gamma + 1, cfg.vocab)
+    return sel, kv, q_all, logits_all
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = wl.config(args.config)
+    sel, kv, q_all, logits_all = host_inputs(cfg)
+    cost = wl.cost_table_for(cfg)
+    per_step = max(2.0, min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(cfg, sel, kv, q_all, logits_all, cost, per_step)
+    times, toks, info = [], [], None
+    for _ in range(args.steps):
+        info, dt, _, acc = oracle_sample(cfg, sel, kv, q_all, logits_all, cost, per_step)
+        times.append(dt)
+        toks.append(acc)
+    value = sum(toks) / sum(times)
+    info["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"configs[{cfg.index}] {cfg.name}: B={cfg.B} gamma={cfg.gamma} "
+                                   f"{cfg.n_q_heads}q/{cfg.n_kv_heads}kv Dh={cfg.head_dim} V={cfg.vocab}",
+                       "cost_table": "linear stand-in (no GPU profile in this arm)"},
+            "cpu_baseline": info,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ GPU arm
+
+def run_dcut(args):
+    world, rank, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    from paper_2607_14647_b200 import binding
+
+    cfg = wl.config(args.config)
+    sel, kv, q_all, logits_all = host_inputs(cfg)
+    dev = torch.device("cuda", local)
+    d_conf = torch.from_numpy(sel.conf).to(dev)
+    d_draft = torch.from_numpy(sel.draft_ids).to(dev)
+    d_bonus = torch.from_numpy(sel.bonus_ids).to(dev)
+    d_ctx = torch.from_numpy(sel.ctx_lens).to(dev)
+    d_bt = torch.from_numpy(kv.block_table).to(dev)
+    d_k, d_v = kv.k_cache.to(dev), kv.v_cache.to(dev)
+    d_q_all = q_all.to(dev).view(cfg.t_cap, cfg.n_q_heads, cfg.head_dim)
+    d_logits_all = logits_all.to(dev).view(cfg.t_cap, cfg.vocab)
+    ctx = binding.Context(max_B=cfg.B, max_gamma=cfg.gamma, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                          head_dim=cfg.head_dim, page_size=cfg.page_size, max_pages_per_req=kv.max_pages_per_req,
+                          vocab=cfg.vocab)
+    cap = cfg.t_cap
+    sel_out = None
+
+    def pack(depths_np):
+        """Gathers the kept rows (i, t <= d_i) of the unpacked device tensors (set-up, not timed)."""
+        idx = np.concatenate([i * (cfg.gamma + 1) + np.arange(d + 1) for i, d in enumerate(depths_np)])
+        idx_t = torch.from_numpy(idx).to(dev)
+        return d_q_all.index_select(0, idx_t).contiguous(), d_logits_all.index_select(0, idx_t).contiguous()
+
+    res = {}
+
+    def step(qp, lp, bufs):
+        nonlocal sel_out
+        sel_out = ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=sel_out)
+        ctx.verify_attn(qp, d_k, d_v, d_bt, d_ctx, sel_out.cu_q, cap, out=bufs["attn_out"])
+        ctx.accept_into(lp, d_draft, sel_out.cu_q, cap, bufs["accept_len"], bufs["bonus"], bufs["out_tokens"],
+                        bufs["total"])
+
+    def make_bufs(T):
+        i32 = dict(dtype=torch.int32, device=dev)
+        return dict(attn_out=torch.empty((T, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev),
+                    accept_len=torch.empty(cfg.B, **i32), bonus=torch.empty(cfg.B, **i32),
+                    out_tokens=torch.empty((cfg.B, cfg.gamma + 1), **i32), total=torch.empty(1, **i32))
+
+    def depths_now():
+        step_sel = ctx.select(d_conf, d_draft, d_bonus, d_ctx)
+        torch.cuda.synchronize()
+        return step_sel.depths.cpu().numpy()
+
+    # ---- cost table: step latency against the packed length T, profiled on this GPU ---------------
+    grid = sorted(set(int(round(x)) for x in np.linspace(cfg.B, cap, args.cost_points)))
+    prof = []
+    for T in grid:
+        ctx.set_cost_buckets(cfg.B, cfg.gamma, [T], [1.0])
+        d = depths_now()
+        qp, lp = pack(d)
+        bufs = make_bufs(T)
+        for _ in range(3):
+            step(qp, lp, bufs)
+        ts = []
+        for _ in range(7):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            step(qp, lp, bufs)
+            e1.record()
+            e1.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        prof.append(statistics.median(ts))
+        del qp, lp, bufs
+    cost = np.interp(np.arange(cap + 1), grid, prof)
+    cost = np.maximum.accumulate(cost).astype(np.float32)          # non-decreasing in T
+
+    arms = {"pruned": cost, "full_gamma": np.ones(cap + 1, np.float32),
+            "gamma0": (1.0 + 10.0 * np.maximum(0, np.arange(cap + 1) - cfg.B)).astype(np.float32)}
+    sampler = ClockSampler(local) if rank == 0 else None
+    for name, table in arms.items():
+        ctx.set_cost_dense(table)
+        d = depths_now()
+        qp, lp = pack(d)
+        T = int(d.sum()) + cfg.B
+        bufs = make_bufs(T)
+        for _ in range(max(3, args.warmup)):
+            step(qp, lp, bufs)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        barrier(world)
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record()
+        for k in range(args.steps):
+            nonlocal_sel = ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=sel_out)
+            ev[k][0].record()
+            ctx.verify_attn(qp, d_k, d_v, d_bt, d_ctx, nonlocal_sel.cu_q, cap, out=bufs["attn_out"])
+            ev[k][1].record()
+            ctx.accept_into(lp, d_draft, nonlocal_sel.cu_q, cap, bufs["accept_len"], bufs["bonus"],
+                            bufs["out_tokens"], bufs["total"])
+        end.record()
+        barrier(world)
+        total_ms = max_over_ranks(start.elapsed_time(end), world)
+        attn_ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+        accepted = int(bufs["total"].item())
+        assert ctx.poll_device_status() == 0
+        res[name] = dict(T=T, accepted=accepted, ms_per_step=total_ms / args.steps, attn_ms=attn_ms,
+                         tokens_per_s=world * accepted / (total_ms / args.steps * 1e-3),
+                         attn_bytes=attn_algorithmic_bytes(cfg, sel.ctx_lens, d), depths=d)
+        del qp, lp, bufs
+    clocks = sampler.stop() if sampler else {}
+
+    # ---- end to end from host buffers ---------------------------------------------------------
+    ctx.set_cost_dense(cost)
+    pin = lambda t: t.contiguous().pin_memory()
+    h = dict(conf=pin(torch.from_numpy(sel.conf)), draft=pin(torch.from_numpy(sel.draft_ids)),
+             bonus=pin(torch.from_numpy(sel.bonus_ids)), ctx=pin(torch.from_numpy(sel.ctx_lens)),
+             bt=pin(torch.from_numpy(kv.block_table)), q=pin(q_all), logits=pin(logits_all))
+    hout = ctx.host_step_outputs(cfg.B, cfg.gamma)
+    call = lambda: ctx.verify_step_host(h["conf"], h["draft"], h["bonus"], h["ctx"], h["bt"], h["q"], h["logits"],
+                                        d_k, d_v, out=hout)
+    for _ in range(3):
+        call()
+    barrier(world)
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        call()
+    barrier(world)
+    e2e_s = max_over_ranks(time.perf_counter() - t0, world) / args.e2e_steps
+    e2e_accepted = int(hout["n_accepted_total"].item())
+    assert e2e_accepted == res["pruned"]["accepted"], (e2e_accepted, res["pruned"]["accepted"])
+
+    if rank != 0:
+        return
+    pk = peaks()
+    p = res["pruned"]
+    achieved = p["attn_bytes"] / (p["attn_ms"] * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": p["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": p["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"configs[{cfg.index}] {cfg.name}: B={cfg.B} gamma={cfg.gamma} {cfg.n_q_heads}q/"
+                               f"{cfg.n_kv_heads}kv Dh={cfg.head_dim} page={cfg.page_size} V={cfg.vocab} "
+                               f"ctx {cfg.ctx_lo}-{cfg.ctx_hi}",
+                   "arm": "D-cut pruned (dense cost table profiled on this GPU)",
+                   "l2": f"inputs exceed L2: each step streams {p['attn_bytes'] / 1e6:.0f} MB of KV and "
+                         f"{p['T'] * cfg.vocab * 2 / 1e6:.0f} MB of logits once (L2 is 126 MB)",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "arms": {k: {"T": v["T"], "accepted_tokens": v["accepted"], "ms_per_step": round(v["ms_per_step"], 4),
+                     "attn_ms": round(v["attn_ms"], 4), "tokens_per_s": round(v["tokens_per_s"], 1),
+                     "attn_gbs": round(v["attn_bytes"] / (v["attn_ms"] * 1e-3) / 1e9, 1)} for k, v in res.items()},
+        "roofline": {"kernel": "dcut_verify_attn (plan + split + combine launches)", "bound": "hbm",
+                     "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(achieved / pk["hbm_gbs"], 4), "peak_source": f"of {pk['source']}",
+                     "frac_of_8000_nominal": round(achieved / 8000.0, 4),
+                     "algorithmic_bytes_per_launch": p["attn_bytes"],
+                     "traffic": None if ATTN_TRAFFIC_RATIO is None else int(ATTN_TRAFFIC_RATIO * p["attn_bytes"])},
+        "e2e": {"value": world * e2e_accepted / e2e_s, "unit": UNIT, "ms_per_step": round(e2e_s * 1e3, 4),
+                "h2d_bytes_per_step": hout["h2d_bytes"], "d2h_bytes_per_step": hout["d2h_bytes"],
+                "api": "dcut_verify_step_host (pinned host buffers; KV cache resident)"},
+        "gpu_launches": 6 * args.steps,
+        "cost_table_ms": {str(t): round(c, 4) for t, c in zip(grid, prof)},
+        "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        info, *_ = oracle_sample(cfg, sel, kv, q_all, logits_all, cost, args.cpu_seconds)
+        line["cpu_baseline"] = info
+    print(json.dumps(line))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_dcut(args)
+
+
+if __name__ == "__main__":
+    main()

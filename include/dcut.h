@@ -148,6 +148,47 @@ dcut_status dcut_accept(dcut_ctx* ctx, const void* logits, int V, const int* dra
                         int B, int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
                         int* n_accepted_total, void* stream);
 
+/*
+ * One whole verify step from HOST buffers: select, packing, verification attention, acceptance
+ * (Algorithm 1 followed by the target's accept step), with every host<->device copy inside the call.
+ * The packed shape is resolved on the host, as the paper's own system does (Section 5, limitation
+ * paragraph): after dcut_select the call reads cu_q back, then copies only the kept prefix of every
+ * request's query and logits rows to the device, runs dcut_verify_attn and dcut_accept, copies the
+ * results back and synchronises `stream` before returning.
+ * HOST in (pinned memory recommended): conf fp32 [B,gamma]; draft_ids i32 [B,gamma]; bonus_ids i32
+ *   [B]; ctx_lens i32 [B]; block_table i32 [B, block_table_stride]; q_rows bf16
+ *   [B, gamma+1, n_q_heads, head_dim] and logits_rows bf16 [B, gamma+1, vocab]: the row of every block
+ *   position (i, t), of which the kept ones t <= d_i are used.
+ * DEVICE in: k_cache, v_cache (resident state, layout above), num_pages.
+ * HOST out: depths, accept_len, bonus i32 [B]; out_tokens i32 [B, gamma+1]; n_accepted_total i32
+ *   [1]; attn_out bf16 [T, n_q_heads, head_dim] or NULL; h2d_bytes / d2h_bytes (bytes copied, or NULL).
+ * Uses the cost table set on the context.  The first call (and a call with a larger vocab) allocates
+ * device staging buffers; later calls allocate nothing.
+ */
+typedef struct {
+    int B, gamma, vocab, block_table_stride;
+    long long num_pages;
+    float scale;
+    const float* conf;
+    const int* draft_ids;
+    const int* bonus_ids;
+    const int* ctx_lens;
+    const int* block_table;
+    const void* q_rows;
+    const void* logits_rows;
+    const void* k_cache;
+    const void* v_cache;
+    int* depths;
+    int* accept_len;
+    int* bonus;
+    int* out_tokens;
+    int* n_accepted_total;
+    void* attn_out;
+    long long* h2d_bytes;
+    long long* d2h_bytes;
+} dcut_host_step;
+dcut_status dcut_verify_step_host(dcut_ctx* ctx, const dcut_host_step* step, void* stream);
+
 /* Reads the device status word (0 = no kernel reported an error) after synchronising `stream`,
  * and clears it.  A non-zero code also makes this call return DCUT_EDEVICE. */
 dcut_status dcut_poll_device_status(dcut_ctx* ctx, int* code, void* stream);

@@ -27,7 +27,8 @@ OK, EINVAL, ECAPACITY, ECUDA, ECOST, EDEVICE = range(6)
 STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_ECOST", "DCUT_EDEVICE"]
 
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
-           "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_poll_device_status"]
+           "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
+           "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -41,6 +42,17 @@ class SelectInfo(C.Structure):
 
 
 _vp, _i, _ll, _f = C.c_void_p, C.c_int, C.c_longlong, C.c_float
+
+
+class HostStep(C.Structure):
+    _fields_ = [("B", _i), ("gamma", _i), ("vocab", _i), ("block_table_stride", _i), ("num_pages", _ll),
+                ("scale", _f)] + [(n, _vp) for n in (
+                    "conf", "draft_ids", "bonus_ids", "ctx_lens", "block_table", "q_rows", "logits_rows", "k_cache",
+                    "v_cache", "depths", "accept_len", "bonus", "out_tokens", "n_accepted_total", "attn_out",
+                    "h2d_bytes", "d2h_bytes")]
+
+
+_lib.dcut_verify_step_host.argtypes = [_vp, C.POINTER(HostStep), _vp]
 _lib.dcut_create.argtypes = [C.POINTER(_vp), C.POINTER(Limits), _i]
 _lib.dcut_destroy.argtypes = [_vp]
 _lib.dcut_last_error.argtypes = [_vp]
@@ -193,6 +205,39 @@ class Context:
         self._check(_lib.dcut_accept(self._h, _ptr(logits, torch.bfloat16), logits.shape[1],
                                      _ptr(draft_ids, torch.int32), _ptr(cu_q, torch.int32), B, gamma, T_cap,
                                      _ptr(accept_len), _ptr(bonus), _ptr(out_tokens), _ptr(total), _stream()))
+
+    def verify_step_host(self, conf, draft_ids, bonus_ids, ctx_lens, block_table, q_rows, logits_rows, k_cache,
+                         v_cache, out: Optional[dict] = None, scale: Optional[float] = None, want_attn_out=False):
+        """Whole step from HOST tensors (CPU torch tensors, ideally pinned); k_cache / v_cache are the
+        device-resident cache.  Returns a dict of CPU tensors plus the bytes copied each way."""
+        B, gamma = conf.shape
+        V = logits_rows.shape[-1]
+        for t in (conf, draft_ids, bonus_ids, ctx_lens, block_table, q_rows, logits_rows):
+            assert not t.is_cuda and t.is_contiguous()
+        if out is None:
+            out = self.host_step_outputs(B, gamma, want_attn_out)
+        if scale is None:
+            scale = 1.0 / float(np.sqrt(self.limits.head_dim))
+        h2d, d2h = _ll(0), _ll(0)
+        hs = HostStep(B, gamma, V, block_table.shape[1], k_cache.shape[0], float(scale), conf.data_ptr(),
+                      draft_ids.data_ptr(), bonus_ids.data_ptr(), ctx_lens.data_ptr(), block_table.data_ptr(),
+                      q_rows.data_ptr(), logits_rows.data_ptr(), _ptr(k_cache, torch.bfloat16),
+                      _ptr(v_cache, torch.bfloat16), out["depths"].data_ptr(), out["accept_len"].data_ptr(),
+                      out["bonus"].data_ptr(), out["out_tokens"].data_ptr(), out["n_accepted_total"].data_ptr(),
+                      out["attn_out"].data_ptr() if out.get("attn_out") is not None else None,
+                      C.addressof(h2d), C.addressof(d2h))
+        self._check(_lib.dcut_verify_step_host(self._h, C.byref(hs), _stream()))
+        out["h2d_bytes"], out["d2h_bytes"] = h2d.value, d2h.value
+        return out
+
+    def host_step_outputs(self, B: int, gamma: int, want_attn_out: bool = False) -> dict:
+        pin = dict(dtype=torch.int32, pin_memory=True)
+        out = dict(depths=torch.zeros(B, **pin), accept_len=torch.zeros(B, **pin), bonus=torch.zeros(B, **pin),
+                   out_tokens=torch.zeros((B, gamma + 1), **pin), n_accepted_total=torch.zeros(1, **pin), attn_out=None)
+        if want_attn_out:
+            out["attn_out"] = torch.zeros((B * (gamma + 1), self.limits.n_q_heads, self.limits.head_dim),
+                                          dtype=torch.bfloat16, pin_memory=True)
+        return out
 
     def poll_device_status(self) -> int:
         code = _i(0)

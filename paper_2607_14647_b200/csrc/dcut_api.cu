@@ -53,6 +53,18 @@ void free_all(dcut_ctx* c) {
     cudaFree(c->d_part_lse);
     cudaFree(c->d_row_key);
     cudaFree(c->d_status);
+    cudaFree(c->hs_conf);
+    cudaFree(c->hs_draft);
+    cudaFree(c->hs_bonus);
+    cudaFree(c->hs_ctx_lens);
+    cudaFree(c->hs_block_table);
+    cudaFree(c->hs_depths);
+    cudaFree(c->hs_cu_q);
+    cudaFree(c->hs_accept);
+    cudaFree(c->hs_q);
+    cudaFree(c->hs_out);
+    cudaFree(c->hs_logits);
+    if (c->hs_host_cu_q) cudaFreeHost(c->hs_host_cu_q);
 }
 
 }  // namespace
@@ -254,3 +266,100 @@ dcut_status dcut_poll_device_status(dcut_ctx* c, int* code, void* stream) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Whole step from host buffers.
+
+namespace {
+
+dcut_status ensure_host_step_buffers(dcut_ctx* c, int V) {
+    if (c->hs_ready && c->hs_vocab >= V) return DCUT_OK;
+    const dcut_limits& l = c->lim;
+    const size_t max_T = (size_t)l.max_B * (l.max_gamma + 1);
+    const size_t keys = (size_t)l.max_B * l.max_gamma;
+    dcut_status st;
+    if (!c->hs_ready) {
+        if ((st = dmalloc(c, &c->hs_conf, keys, "cudaMalloc(step conf)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_draft, keys, "cudaMalloc(step draft)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_bonus, l.max_B, "cudaMalloc(step bonus)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_ctx_lens, l.max_B, "cudaMalloc(step ctx_lens)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_block_table, (size_t)l.max_B * l.max_pages_per_req, "cudaMalloc(step block table)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_depths, l.max_B, "cudaMalloc(step depths)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_cu_q, (size_t)l.max_B + 1, "cudaMalloc(step cu_q)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_accept, (size_t)l.max_B * (l.max_gamma + 3) + 4, "cudaMalloc(step accept)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_q, max_T * l.n_q_heads * l.head_dim, "cudaMalloc(step q)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->hs_out, max_T * l.n_q_heads * l.head_dim, "cudaMalloc(step out)")) != DCUT_OK) return st;
+        cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&c->hs_host_cu_q), sizeof(int) * ((size_t)l.max_B + 1));
+        if (e != cudaSuccess) return dcut_check_cuda(c, e, "cudaMallocHost(step cu_q)");
+    }
+    if (c->hs_logits) cudaFree(c->hs_logits);
+    c->hs_logits = nullptr;
+    if ((st = dmalloc(c, &c->hs_logits, max_T * (size_t)V, "cudaMalloc(step logits)")) != DCUT_OK) return st;
+    c->hs_vocab = V;
+    c->hs_ready = 1;
+    return DCUT_OK;
+}
+
+}  // namespace
+
+extern "C" dcut_status dcut_verify_step_host(dcut_ctx* c, const dcut_host_step* s, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (!s || !s->conf || !s->draft_ids || !s->bonus_ids || !s->ctx_lens || !s->block_table || !s->q_rows ||
+        !s->logits_rows || !s->k_cache || !s->v_cache || !s->depths || !s->accept_len || !s->bonus || !s->out_tokens ||
+        !s->n_accepted_total)
+        return dcut_fail(c, DCUT_EINVAL, "null pointer in dcut_host_step");
+    const int B = s->B, g = s->gamma, V = s->vocab;
+    const dcut_limits& l = c->lim;
+    if (B < 1 || g < 1 || V < 1) return dcut_fail(c, DCUT_EINVAL, "need B, gamma, vocab >= 1");
+    if (B > l.max_B || g > l.max_gamma || s->block_table_stride > l.max_pages_per_req || s->block_table_stride < 1)
+        return dcut_fail(c, DCUT_ECAPACITY, "B, gamma or block_table_stride exceed the limits");
+    if (l.n_q_heads <= 0) return dcut_fail(c, DCUT_EINVAL, "context was created without attention shapes");
+    dcut_status st = ensure_host_step_buffers(c, V);
+    if (st != DCUT_OK) return st;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const size_t q_row = (size_t)l.n_q_heads * l.head_dim * 2, lg_row = (size_t)V * 2;
+#define DCUT_CP(dst, src, bytes, kind)                                                                   \
+    if ((st = dcut_check_cuda(c, cudaMemcpyAsync(dst, src, bytes, kind, cs), "cudaMemcpyAsync(step)")) != DCUT_OK) return st
+    DCUT_CP(c->hs_conf, s->conf, sizeof(float) * B * g, cudaMemcpyHostToDevice);
+    DCUT_CP(c->hs_draft, s->draft_ids, sizeof(int) * B * g, cudaMemcpyHostToDevice);
+    DCUT_CP(c->hs_bonus, s->bonus_ids, sizeof(int) * B, cudaMemcpyHostToDevice);
+    DCUT_CP(c->hs_ctx_lens, s->ctx_lens, sizeof(int) * B, cudaMemcpyHostToDevice);
+    DCUT_CP(c->hs_block_table, s->block_table, sizeof(int) * (size_t)B * s->block_table_stride, cudaMemcpyHostToDevice);
+    st = dcut_select(c, c->hs_conf, B, g, nullptr, nullptr, nullptr, c->hs_depths, c->hs_cu_q, nullptr, nullptr, nullptr,
+                     nullptr, nullptr, nullptr, stream);
+    if (st != DCUT_OK) return st;
+    // the packed shape is resolved on the host: read cu_q back, then copy only the kept prefixes
+    DCUT_CP(c->hs_host_cu_q, c->hs_cu_q, sizeof(int) * (B + 1), cudaMemcpyDeviceToHost);
+    if ((st = dcut_check_cuda(c, cudaStreamSynchronize(cs), "cudaStreamSynchronize(step)")) != DCUT_OK) return st;
+    const int* cu = c->hs_host_cu_q;
+    long long h2d = (long long)(sizeof(float) + sizeof(int)) * B * g + 2ll * sizeof(int) * B +
+                    (long long)sizeof(int) * B * s->block_table_stride;
+    for (int i = 0; i < B; ++i) {
+        const size_t rows = (size_t)(cu[i + 1] - cu[i]);
+        DCUT_CP(reinterpret_cast<char*>(c->hs_q) + (size_t)cu[i] * q_row,
+                static_cast<const char*>(s->q_rows) + (size_t)i * (g + 1) * q_row, rows * q_row, cudaMemcpyHostToDevice);
+        DCUT_CP(reinterpret_cast<char*>(c->hs_logits) + (size_t)cu[i] * lg_row,
+                static_cast<const char*>(s->logits_rows) + (size_t)i * (g + 1) * lg_row, rows * lg_row, cudaMemcpyHostToDevice);
+        h2d += (long long)(rows * (q_row + lg_row));
+    }
+    const int T_cap = B * (g + 1);
+    st = dcut_verify_attn(c, c->hs_q, s->k_cache, s->v_cache, s->num_pages, c->hs_block_table, s->block_table_stride,
+                          c->hs_ctx_lens, c->hs_cu_q, B, T_cap, s->scale, c->hs_out, nullptr, stream);
+    if (st != DCUT_OK) return st;
+    int* acc = c->hs_accept;            // [B] accept_len, [B] bonus, [B*(g+1)] tokens, [1] total
+    st = dcut_accept(c, c->hs_logits, V, c->hs_draft, c->hs_cu_q, B, g, T_cap, acc, acc + B, acc + 2 * B,
+                     acc + 2 * B + B * (g + 1), stream);
+    if (st != DCUT_OK) return st;
+    DCUT_CP(s->depths, c->hs_depths, sizeof(int) * B, cudaMemcpyDeviceToHost);
+    DCUT_CP(s->accept_len, acc, sizeof(int) * B, cudaMemcpyDeviceToHost);
+    DCUT_CP(s->bonus, acc + B, sizeof(int) * B, cudaMemcpyDeviceToHost);
+    DCUT_CP(s->out_tokens, acc + 2 * B, sizeof(int) * B * (g + 1), cudaMemcpyDeviceToHost);
+    DCUT_CP(s->n_accepted_total, acc + 2 * B + B * (g + 1), sizeof(int), cudaMemcpyDeviceToHost);
+    if (s->attn_out) DCUT_CP(s->attn_out, c->hs_out, (size_t)cu[B] * q_row, cudaMemcpyDeviceToHost);
+#undef DCUT_CP
+    if ((st = dcut_check_cuda(c, cudaStreamSynchronize(cs), "cudaStreamSynchronize(step end)")) != DCUT_OK) return st;
+    if (s->h2d_bytes) *s->h2d_bytes = h2d;
+    if (s->d2h_bytes)
+        *s->d2h_bytes = (long long)sizeof(int) * (B + 1 + 3 * B + B * (g + 1) + 1) + (s->attn_out ? (long long)cu[B] * q_row : 0);
+    return DCUT_OK;
+}

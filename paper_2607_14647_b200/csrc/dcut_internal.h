@@ -57,6 +57,13 @@ struct dcut_ctx {
 
     // tensor-map encoder (driver entry point fetched through the runtime)
     void* encode_tiled;
+
+    // staging of dcut_verify_step_host (allocated by its first call)
+    int hs_ready, hs_vocab;
+    float* hs_conf;
+    int *hs_draft, *hs_bonus, *hs_ctx_lens, *hs_block_table, *hs_depths, *hs_cu_q, *hs_accept;
+    unsigned short *hs_q, *hs_out, *hs_logits;
+    int* hs_host_cu_q;      // pinned
 };
 
 dcut_status dcut_fail(dcut_ctx* ctx, dcut_status st, const char* fmt, ...);
