@@ -8,15 +8,15 @@
 //                        batch gives a few work items per SM (flash-decoding split-KV); an item is
 //                        one (request, kv head, page range).
 //   attn_split_kernel    one CTA per item: 15 consumer warps + 1 producer warp.
-//       producer         reads the block table and issues TMA tile loads (2-D tensor map over the
-//                        cache seen as [rows of one token, head_dim], 128-byte swizzle) into a ring
-//                        of page stages, each guarded by a full/empty mbarrier pair.
+//       producer         four lanes read the block table and issue TMA tile loads (3-D tensor map over
+//                        the cache, one 4 KB box per (page, kv head) tile, 128-byte swizzle) into a
+//                        ring of page stages, each guarded by a full/empty mbarrier pair.
 //       consumers        the item's query tile is (1 + d_i) * group rows (every query token of the
 //                        request times the q heads sharing this kv head), cut into 16-row m-tiles.
 //                        Warp w owns m-tile (w mod MT) and page slot (w div MT): it runs
 //                        S = Q K^T, online softmax and O += P V for its m-tile on every
 //                        nslots-th page (mma.sync m16n8k16 bf16, fp32 accumulate, ldmatrix from the
-//                        swizzled tiles).  Small query tiles therefore spread pages over warps,
+//                        swizzled tiles); it still waits on and releases every stage in order.  Small query tiles therefore spread pages over warps,
 //                        large ones spread rows.
 //       epilogue         the slots' (m, l, O) are merged through shared memory; a request with one
 //                        chunk writes bf16 output directly, otherwise normalised fp32 partials + LSE.
@@ -33,11 +33,13 @@ namespace {
 constexpr int kConsumerWarps = 15;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
-constexpr int kStages = 17;
+constexpr int kStages = 20;        // multiple of kProducerLanes
+constexpr int kProducerLanes = 4;  // lanes of the producer warp that each stream every 4th page
+static_assert(kStages % kProducerLanes == 0, "a stage must always be refilled by the same producer lane");
 constexpr int kPage = 16;          // tokens per page
 constexpr int kMaxMTiles = 9;      // query rows per item <= 144
 constexpr int kPlanThreads = 1024;
-constexpr long long kSpinLimit = 1ll << 22;
+constexpr int kSpinLimit = 1 << 21;   // bounded waits: ~1 s, then the CTA reports and leaves
 
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -65,18 +67,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// bounded wait: false if the phase did not complete within the spin limit
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (long long it = 0; it < kSpinLimit; ++it) {
+// bounded wait: false if the phase did not complete within the spin limit, or another warp of the
+// CTA has already given up
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag) {
+    for (int it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (it > 4096) __nanosleep(64);
+        if (it > 4096) {
+            __nanosleep(128);
+            if ((it & 255) == 0 && *abort_flag) return false;
+        }
     }
     return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+// one (page, kv head) tile: box {64 columns, 16 token rows, head_dim/64 column halves}
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int row, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
@@ -290,7 +297,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         abort_s = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, MT);
+            mbar_init(empty_bar + 8 * s, MT * nslots);   // every working consumer warp releases every stage
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -299,37 +306,35 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
 
     if (warp == kConsumerWarps) {
         // ---------------------------------------------------------------- producer warp
-        const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
-        int my_page = 0;
-        for (int p = 0; p < n_pages; ++p) {
-            if ((p & 31) == 0) my_page = (p + lane < n_pages) ? bt[p + lane] : 0;
-            int page_id = __shfl_sync(0xffffffffu, my_page, p & 31);
-            const int stage = p % kStages;
-            int ok = 1;
-            if (lane == 0) {
-                if (p >= kStages) ok = mbar_wait(empty_bar + 8 * stage, ((p / kStages) - 1) & 1) ? 1 : 0;
-                if (ok && *(volatile int*)&abort_s) ok = 0;
-                if (ok) {
-                    if (page_id < 0 || page_id >= a.num_pages) {
-                        atomicExch(a.status, DCUT_DEV_BAD_PAGE);
-                        page_id = 0;
-                    }
-                    const uint32_t bar = full_bar + 8 * stage;
-                    const uint32_t dst = smem_u32(ring + stage * L::kStageBytes);
-                    const int row = (page_id * a.n_kv_heads + kvh) * kPage;
-                    mbar_arrive_expect_tx(bar, L::kStageBytes);
-#pragma unroll
-                    for (int h = 0; h < L::kHalves; ++h) {
-                        tma_load_2d(dst + h * 2048, &k_map, h * 64, row, bar);
-                        tma_load_2d(dst + L::kPageBytes + h * 2048, &v_map, h * 64, row, bar);
-                    }
-                } else {
-                    atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
+        // Lanes 0..kProducerLanes-1 each stream pages lane, lane + kProducerLanes, ... on their own:
+        // one lane's issue latency (block-table read, empty wait, expect_tx, two tile loads) is then
+        // overlapped with the others'.  kStages is a multiple of kProducerLanes, so every stage is
+        // always refilled by the same lane and its waits stay ordered.
+        if (lane < kProducerLanes) {
+            const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
+            int next = lane < n_pages ? bt[lane] : 0;
+            for (int p = lane; p < n_pages; p += kProducerLanes) {
+                int page_id = next;
+                if (p + kProducerLanes < n_pages) next = bt[p + kProducerLanes];
+                const int stage = p % kStages;
+                bool ok = true;
+                if (p >= kStages) ok = mbar_wait(empty_bar + 8 * stage, ((p / kStages) - 1) & 1, &abort_s);
+                if (!ok || *(volatile int*)&abort_s) {
+                    if (!ok) atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
                     *(volatile int*)&abort_s = 1;
+                    break;
                 }
+                if (page_id < 0 || page_id >= a.num_pages) {
+                    atomicExch(a.status, DCUT_DEV_BAD_PAGE);
+                    page_id = 0;
+                }
+                const uint32_t bar = full_bar + 8 * stage;
+                const uint32_t dst = smem_u32(ring + stage * L::kStageBytes);
+                const int row = (page_id * a.n_kv_heads + kvh) * kPage;
+                mbar_arrive_expect_tx(bar, L::kStageBytes);
+                tma_load_tile(dst, &k_map, row, bar);
+                tma_load_tile(dst + L::kPageBytes, &v_map, row, bar);
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
         }
         return;
     }
@@ -380,12 +385,24 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         const int v_tok = ((kmat & 1) << 3) + (lane & 7);
         const int v_chunk = kmat >> 1;
 
-        for (int p = slot; p < n_pages; p += nslots) {
-            const int stage = p % kStages;
-            if (!mbar_wait(full_bar + 8 * stage, (p / kStages) & 1)) {
+        // Every working warp walks every stage in order (wait full, release empty) and computes only on
+        // its slot's pages.  Walking all stages keeps each warp within one ring cycle of the producer,
+        // which the one-bit phase parity of the mbarrier waits relies on.
+        int stage = 0, parity = 0, mine = slot;
+        for (int p = 0; p < n_pages; ++p, ++stage) {
+            if (stage == kStages) {
+                stage = 0;
+                parity ^= 1;
+            }
+            if (!mbar_wait(full_bar + 8 * stage, parity, &abort_s)) {
                 aborted = true;
                 break;
             }
+            if (p != mine) {
+                if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
+                continue;
+            }
+            mine += nslots;
             const uint32_t k_base = smem_u32(ring + stage * L::kStageBytes);
             const uint32_t v_base = k_base + L::kPageBytes;
 
@@ -595,13 +612,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 dcut_status make_cache_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, long long num_pages) {
+    // The cache seen as a 3-D tensor {64 columns, token rows, head_dim / 64 column halves}: one box
+    // {64, 16, halves} is a whole (page, kv head) tile and lands in shared memory as
+    // [half][16 rows][64 columns] with the 128-byte swizzle the ldmatrix addressing expects.
     const int DH = ctx->lim.head_dim;
-    cuuint64_t dims[2] = {(cuuint64_t)DH, (cuuint64_t)num_pages * ctx->lim.n_kv_heads * kPage};
-    cuuint64_t strides[1] = {(cuuint64_t)DH * 2};
-    cuuint32_t box[2] = {64, kPage};
-    cuuint32_t estr[2] = {1, 1};
+    cuuint64_t dims[3] = {64, (cuuint64_t)num_pages * ctx->lim.n_kv_heads * kPage, (cuuint64_t)(DH / 64)};
+    cuuint64_t strides[2] = {(cuuint64_t)DH * 2, 128};
+    cuuint32_t box[3] = {64, kPage, (cuuint32_t)(DH / 64)};
+    cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return dcut_fail(ctx, DCUT_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
