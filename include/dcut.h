@@ -27,6 +27,7 @@
 #ifndef DCUT_H_
 #define DCUT_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -147,6 +148,35 @@ dcut_status dcut_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, 
 dcut_status dcut_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
                         int B, int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
                         int* n_accepted_total, void* stream);
+
+/*
+ * dcut_accept without any allocation.  (The paper has no counterpart: this entry point exists for
+ * the way the library gets embedded, not for the method.)
+ *
+ * Who needs it: code that runs inside a serving process after the engine has handed nearly all of
+ * the GPU's memory to its KV-cache pool, where a cudaMalloc (and therefore dcut_create) can simply
+ * fail; and code on a latency-critical path that is not allowed to call the allocator at all,
+ * because cudaMalloc / cudaFree may synchronise the whole device.  Such callers cannot own a
+ * dcut_ctx, so this call takes none: the per-row scratch of dcut_accept (one 64-bit word per packed
+ * logits row) lives in a fixed array inside the library image, DCUT_ACCEPT_STATIC_MAX_ROWS words
+ * (64 KB) on every GPU that loads the library, held until the process exits.
+ *
+ * Same arguments, same results and same DEVICE / caller-owned buffers as dcut_accept; the device that
+ * holds the buffers must be current.  T_cap > DCUT_ACCEPT_STATIC_MAX_ROWS returns DCUT_ECAPACITY
+ * (use dcut_accept then).  errbuf (HOST, may be NULL) receives a message when the status is not
+ * DCUT_OK.  The call never calls cudaMalloc, cudaFree or any allocating routine; it issues one
+ * cudaMemsetAsync and two kernels on `stream`.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, which can
+ * make the runtime load the library's device code); make that first call outside any stream
+ * capture.  All calls on a device share the one array, and it keeps what the previous call left, so
+ * every call clears the words it is going to use first.  Two calls that overlap on the GPU (different
+ * streams, or several threads) race on the array and give wrong results: serialise them.
+ */
+#define DCUT_ACCEPT_STATIC_MAX_ROWS 8192
+dcut_status dcut_accept_static(const void* logits, int V, const int* draft_ids, const int* cu_q, int B,
+                               int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
+                               int* n_accepted_total, void* stream, char* errbuf, size_t errbuf_len);
 
 /*
  * One whole verify step from HOST buffers: select, packing, verification attention, acceptance

@@ -28,7 +28,7 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
-           "dcut_poll_device_status"]
+           "dcut_accept_static", "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -66,6 +66,10 @@ _lib.dcut_accept.argtypes = [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, 
 _lib.dcut_poll_device_status.argtypes = [_vp, C.POINTER(_i), _vp]
 
 
+_lib.dcut_accept_static.argtypes = [_vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, C.c_char_p, C.c_size_t]
+ACCEPT_STATIC_MAX_ROWS = 8192
+
+
 class DcutError(RuntimeError):
     def __init__(self, status: int, msg: str):
         super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {msg}")
@@ -91,6 +95,18 @@ def budget_from_ratio(B: int, gamma: int, num: int, den: int) -> int:
     if st != OK:
         raise DcutError(st, "dcut_budget_from_ratio")
     return k.value
+
+
+def accept_static(logits, draft_ids, cu_q, T_cap: int, accept_len, bonus, out_tokens, total):
+    """dcut_accept_static: acceptance for callers that may not allocate (no context, fixed scratch inside the
+    library, at most ACCEPT_STATIC_MAX_ROWS packed rows).  All tensors are the caller's CUDA tensors."""
+    B, gamma = draft_ids.shape
+    err = C.create_string_buffer(256)
+    st = _lib.dcut_accept_static(_ptr(logits, torch.bfloat16), logits.shape[1], _ptr(draft_ids, torch.int32),
+                                 _ptr(cu_q, torch.int32), B, gamma, T_cap, _ptr(accept_len), _ptr(bonus),
+                                 _ptr(out_tokens), _ptr(total), _stream(), err, len(err))
+    if st != OK:
+        raise DcutError(st, err.value.decode())
 
 
 @dataclass

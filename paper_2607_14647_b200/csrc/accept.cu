@@ -172,3 +172,103 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
                                                gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total);
     return dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_match_kernel");
 }
+
+// ---------------------------------------------------------------------------------------------
+// dcut_accept_static: the same two kernels, with the per-row words in a fixed device array that
+// is part of the library image instead of a context allocation.
+
+#include <mutex>
+#include <stdio.h>
+
+namespace {
+
+// One 64-bit word per packed logits row.  Every GPU that loads this library carries these 64 KB
+// until the process exits.
+__device__ __align__(256) static unsigned long long g_static_row_key[DCUT_ACCEPT_STATIC_MAX_ROWS];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+unsigned long long* g_static_ptr[kMaxDevices];   // device address of g_static_row_key, per device ordinal
+int g_static_sms[kMaxDevices];
+
+void static_msg(char* buf, size_t len, const char* fmt, long long a = 0, long long b = 0) {
+    if (buf && len) snprintf(buf, len, fmt, a, b);
+}
+
+}  // namespace
+
+extern "C" dcut_status dcut_accept_static(const void* logits, int V, const int* draft_ids, const int* cu_q, int B,
+                                          int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
+                                          int* n_accepted_total, void* stream, char* errbuf, size_t errbuf_len) {
+    if (!logits || !draft_ids || !cu_q || !accept_len || !bonus) {
+        static_msg(errbuf, errbuf_len, "dcut_accept_static: null pointer argument");
+        return DCUT_EINVAL;
+    }
+    if (B < 1 || gamma < 1 || V < 1 || T_cap < B) {
+        static_msg(errbuf, errbuf_len, "dcut_accept_static: need B, gamma, V >= 1 and T_cap >= B");
+        return DCUT_EINVAL;
+    }
+    if (T_cap > DCUT_ACCEPT_STATIC_MAX_ROWS || B > 1024 * 64) {
+        static_msg(errbuf, errbuf_len,
+                   "dcut_accept_static: T_cap = %lld packed rows exceed the fixed scratch of %lld rows; use dcut_accept",
+                   T_cap, DCUT_ACCEPT_STATIC_MAX_ROWS);
+        return DCUT_ECAPACITY;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        static_msg(errbuf, errbuf_len, "dcut_accept_static: cudaGetDevice failed or device ordinal %lld out of range", dev);
+        return DCUT_ECUDA;
+    }
+    unsigned long long* keys = nullptr;
+    int sms = 0;
+    {
+        // set-up, once per device and with that device current: in host code the array's name is only a
+        // handle, so its device address has to be asked for before a kernel can be given it
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            unsigned long long* p = nullptr;
+            e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_row_key);
+            if (e != cudaSuccess || !p) {
+                static_msg(errbuf, errbuf_len, "dcut_accept_static: cudaGetSymbolAddress failed (error %lld)", (long long)e);
+                return DCUT_ECUDA;
+            }
+            int n = 0;
+            e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess || n < 1) {
+                static_msg(errbuf, errbuf_len, "dcut_accept_static: cannot read the SM count (error %lld)", (long long)e);
+                return DCUT_ECUDA;
+            }
+            g_static_sms[dev] = n;
+            g_static_ptr[dev] = p;
+        }
+        keys = g_static_ptr[dev];
+        sms = g_static_sms[dev];
+    }
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the last call (of any caller) left: the words must start at zero
+    e = cudaMemsetAsync(keys, 0, sizeof(unsigned long long) * (size_t)T_cap, cs);
+    if (e != cudaSuccess) {
+        static_msg(errbuf, errbuf_len, "dcut_accept_static: cudaMemsetAsync failed (error %lld)", (long long)e);
+        return DCUT_ECUDA;
+    }
+    int splits = (sms * 16 + T_cap - 1) / T_cap;
+    const int max_splits = (V + 8191) / 8192;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    int seg = (V + splits - 1) / splits;
+    seg = (seg + 7) & ~7;
+    splits = (V + seg - 1) / seg;
+    dim3 grid(splits, T_cap);
+    accept_argmax_kernel<<<grid, kArgmaxThreads, 0, cs>>>(static_cast<const unsigned short*>(logits), V, cu_q, B, seg, keys);
+    if ((e = cudaGetLastError()) == cudaSuccess) {
+        accept_match_kernel<<<1, 1024, 0, cs>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma,
+                                               keys, accept_len, bonus, out_tokens, n_accepted_total);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        static_msg(errbuf, errbuf_len, "dcut_accept_static: kernel launch failed (error %lld)", (long long)e);
+        return DCUT_ECUDA;
+    }
+    return DCUT_OK;
+}
