@@ -8,15 +8,16 @@
 //                        batch gives a few work items per SM (flash-decoding split-KV); an item is
 //                        one (request, kv head, page range).
 //   attn_split_kernel    one CTA per item: 15 consumer warps + 1 producer warp.
-//       producer         four lanes read the block table and issue TMA tile loads (3-D tensor map over
+//       producer         a few lanes read the block table and issue TMA tile loads (3-D tensor map over
 //                        the cache, one 4 KB box per (page, kv head) tile, 128-byte swizzle) into a
-//                        ring of page stages, each guarded by a full/empty mbarrier pair.
+//                        ring of page stages, each guarded by a full/empty mbarrier pair.  The ring is
+//                        cut into one sub-ring per page slot.
 //       consumers        the item's query tile is (1 + d_i) * group rows (every query token of the
 //                        request times the q heads sharing this kv head), cut into 16-row m-tiles.
 //                        Warp w owns m-tile (w mod MT) and page slot (w div MT): it runs
 //                        S = Q K^T, online softmax and O += P V for its m-tile on every
 //                        nslots-th page (mma.sync m16n8k16 bf16, fp32 accumulate, ldmatrix from the
-//                        swizzled tiles); it still waits on and releases every stage in order.  Small query tiles therefore spread pages over warps,
+//                        swizzled tiles), taking them in order from its slot's sub-ring.  Small query tiles therefore spread pages over warps,
 //                        large ones spread rows.
 //       epilogue         the slots' (m, l, O) are merged through shared memory; a request with one
 //                        chunk writes bf16 output directly, otherwise normalised fp32 partials + LSE.
@@ -33,9 +34,8 @@ namespace {
 constexpr int kConsumerWarps = 15;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kThreads = kConsumerThreads + 32;
-constexpr int kStages = 20;        // multiple of kProducerLanes
-constexpr int kProducerLanes = 4;  // lanes of the producer warp that each stream every 4th page
-static_assert(kStages % kProducerLanes == 0, "a stage must always be refilled by the same producer lane");
+constexpr int kStages = 20;        // page stages in the ring (8 KB each at head_dim 128)
+constexpr int kMaxProducerLanes = 6;
 constexpr int kPage = 16;          // tokens per page
 constexpr int kMaxMTiles = 9;      // query rows per item <= 144
 constexpr int kPlanThreads = 1024;
@@ -105,6 +105,12 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+// 2^x on the special-function unit (2 ulp; -inf -> 0); far inside the output tolerance of bf16
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ void consumer_bar() {
     asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
@@ -290,6 +296,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const int MT = (M + 15) >> 4;
     const int nslots = kConsumerWarps / MT;
     const int n_pages = item.page_end - item.page_begin;
+    // The ring is cut into one sub-ring of `depth_s` stages per page slot: page p belongs to slot
+    // p % nslots and is the (p / nslots)-th page of that slot, so a stage is filled and drained by the
+    // same warps in order, which is what the one-bit phase parity of the mbarrier waits needs.
+    const int depth_s = kStages / nslots;
+    const int ring_n = nslots * depth_s;
 
     const uint32_t full_bar = smem_u32(bars);
     const uint32_t empty_bar = smem_u32(bars + kStages);
@@ -297,7 +308,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         abort_s = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, MT * nslots);   // every working consumer warp releases every stage
+            mbar_init(empty_bar + 8 * s, MT);   // the m-tile warps of the stage's slot
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -306,19 +317,23 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
 
     if (warp == kConsumerWarps) {
         // ---------------------------------------------------------------- producer warp
-        // Lanes 0..kProducerLanes-1 each stream pages lane, lane + kProducerLanes, ... on their own:
-        // one lane's issue latency (block-table read, empty wait, expect_tx, two tile loads) is then
-        // overlapped with the others'.  kStages is a multiple of kProducerLanes, so every stage is
-        // always refilled by the same lane and its waits stay ordered.
-        if (lane < kProducerLanes) {
+        // Lanes 0..G-1 each stream pages lane, lane + G, ... on their own, so one lane's issue latency
+        // (block-table read, empty wait, expect_tx, two tile loads) overlaps the others'.  G divides the
+        // number of stages in use: every stage is then always refilled by the same lane, whose waits on
+        // that stage are ordered.
+        int G = kMaxProducerLanes;
+        while (ring_n % G) --G;
+        if (lane < G) {
             const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
             int next = lane < n_pages ? bt[lane] : 0;
-            for (int p = lane; p < n_pages; p += kProducerLanes) {
+            for (int p = lane; p < n_pages; p += G) {
                 int page_id = next;
-                if (p + kProducerLanes < n_pages) next = bt[p + kProducerLanes];
-                const int stage = p % kStages;
+                if (p + G < n_pages) next = bt[p + G];
+                const int q = p / nslots, sl = p - q * nslots;   // q-th page of slot sl
+                const int use = q / depth_s, r = q - use * depth_s;
+                const int stage = sl * depth_s + r;
                 bool ok = true;
-                if (p >= kStages) ok = mbar_wait(empty_bar + 8 * stage, ((p / kStages) - 1) & 1, &abort_s);
+                if (use > 0) ok = mbar_wait(empty_bar + 8 * stage, (use - 1) & 1, &abort_s);
                 if (!ok || *(volatile int*)&abort_s) {
                     if (!ok) atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
                     *(volatile int*)&abort_s = 1;
@@ -385,24 +400,19 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
         const int v_tok = ((kmat & 1) << 3) + (lane & 7);
         const int v_chunk = kmat >> 1;
 
-        // Every working warp walks every stage in order (wait full, release empty) and computes only on
-        // its slot's pages.  Walking all stages keeps each warp within one ring cycle of the producer,
-        // which the one-bit phase parity of the mbarrier waits relies on.
-        int stage = 0, parity = 0, mine = slot;
-        for (int p = 0; p < n_pages; ++p, ++stage) {
-            if (stage == kStages) {
-                stage = 0;
-                parity ^= 1;
-            }
+        // this warp's pages: slot, slot + nslots, ... through the slot's own sub-ring
+        const float c_log2 = a.scale_log2;
+        int r_stage = 0, parity = 0;
+        for (int p = slot; p < n_pages; p += nslots) {
+            const int stage = slot * depth_s + r_stage;
             if (!mbar_wait(full_bar + 8 * stage, parity, &abort_s)) {
                 aborted = true;
                 break;
             }
-            if (p != mine) {
-                if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
-                continue;
+            if (++r_stage == depth_s) {
+                r_stage = 0;
+                parity ^= 1;
             }
-            mine += nslots;
             const uint32_t k_base = smem_u32(ring + stage * L::kStageBytes);
             const uint32_t v_base = k_base + L::kPageBytes;
 
@@ -416,37 +426,41 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
                 mma_bf16(s[0], qf[ks], kf[0], kf[1]);
                 mma_bf16(s[1], qf[ks], kf[2], kf[3]);
             }
-            // scale to the log2 domain, mask
+            // causal mask: only pages that reach past the cached context can hold hidden positions
             const int j0 = (item.page_begin + p) * kPage + ((lane & 3) << 1);
+            if ((item.page_begin + p) * kPage + kPage - 1 > ctx_len) {
 #pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
+                for (int nt = 0; nt < 2; ++nt) {
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int j = j0 + nt * 8 + (e & 1);
-                    const int jmax = (e < 2) ? jmax_lo : jmax_hi;
-                    s[nt][e] = (j <= jmax) ? s[nt][e] * a.scale_log2 : -INFINITY;
+                    for (int e = 0; e < 4; ++e) {
+                        const int j = j0 + nt * 8 + (e & 1);
+                        const int jmax = (e < 2) ? jmax_lo : jmax_hi;
+                        if (j > jmax) s[nt][e] = -INFINITY;
+                    }
                 }
             }
-            // online softmax for the two rows this thread holds
+            // online softmax for the two rows this thread holds; running max kept on the raw scores,
+            // the softmax scale folded into the exponent: p = 2^(s*c - m*c)
             float mx[2] = {fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])),
                            fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]))};
-            float alpha[2], msafe[2];
+            float alpha[2], mc[2];
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
                 mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
                 const float m_new = fmaxf(m_run[r], mx[r]);
-                msafe[r] = (m_new == -INFINITY) ? 0.0f : m_new;
-                alpha[r] = exp2f(m_run[r] - msafe[r]);
+                const float msafe = (m_new == -INFINITY) ? 0.0f : m_new;
+                alpha[r] = fast_exp2((m_run[r] - msafe) * c_log2);
+                mc[r] = msafe * c_log2;
                 m_run[r] = m_new;
             }
             float ps[2][4];
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
-                ps[nt][0] = exp2f(s[nt][0] - msafe[0]);
-                ps[nt][1] = exp2f(s[nt][1] - msafe[0]);
-                ps[nt][2] = exp2f(s[nt][2] - msafe[1]);
-                ps[nt][3] = exp2f(s[nt][3] - msafe[1]);
+                ps[nt][0] = fast_exp2(fmaf(s[nt][0], c_log2, -mc[0]));
+                ps[nt][1] = fast_exp2(fmaf(s[nt][1], c_log2, -mc[0]));
+                ps[nt][2] = fast_exp2(fmaf(s[nt][2], c_log2, -mc[1]));
+                ps[nt][3] = fast_exp2(fmaf(s[nt][3], c_log2, -mc[1]));
             }
             l_run[0] = l_run[0] * alpha[0] + (ps[0][0] + ps[0][1] + ps[1][0] + ps[1][1]);
             l_run[1] = l_run[1] * alpha[1] + (ps[0][2] + ps[0][3] + ps[1][2] + ps[1][3]);
@@ -514,7 +528,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             for (int sl = 0; sl < nslots; ++sl) {
                 const int w = sl * MT + tile;
                 const float m_w = ml_s[(w * 16 + r) * 2];
-                const float wgt = (m_w == -INFINITY) ? 0.0f : exp2f(m_w - m_all);
+                const float wgt = (m_w == -INFINITY) ? 0.0f : exp2f((m_w - m_all) * a.scale_log2);
                 l_all += wgt * ml_s[(w * 16 + r) * 2 + 1];
                 const float4 v = *reinterpret_cast<const float4*>(merge + ((size_t)w * 16 + r) * L::kMergeStride + c4 * 4);
                 acc.x += wgt * v.x;
@@ -527,7 +541,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
             acc.y *= inv;
             acc.z *= inv;
             acc.w *= inv;
-            const float lse_nat = l_all > 0.0f ? (m_all + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+            const float lse_nat = l_all > 0.0f ? (m_all * a.scale_log2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
             const int t = R / group, hl = R - t * group;
             const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
             if (item.n_chunks == 1) {
