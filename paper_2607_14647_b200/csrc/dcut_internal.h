@@ -13,6 +13,7 @@
 #define DCUT_DEV_OK 0
 #define DCUT_DEV_ATTN_WAIT_TIMEOUT 1   // a bounded mbarrier wait in the attention kernel gave up
 #define DCUT_DEV_BAD_PAGE 2            // a block-table entry outside [0, num_pages)
+#define DCUT_DEV_PLAN_OVERFLOW 3       // the attention work list did not fit the context's scratch
 
 // One split-KV work item of the attention kernel: one (request, kv head, page range).
 struct __align__(16) AttnItem {
@@ -20,10 +21,12 @@ struct __align__(16) AttnItem {
     int32_t kv_head;
     int32_t page_begin;   // first page index (within the request's block-table row)
     int32_t page_end;     // one past the last
-    int32_t chunk;        // which chunk of this request
     int32_t n_chunks;     // how many chunks the request has
-    int32_t part_row;     // first row of this item's partial results in the scratch
-    int32_t pad;
+    int32_t part_row;     // first row of this item's partial results in the scratch (-1: writes the output)
+    int32_t q0;           // cu_q[req]: first packed token of the request
+    int32_t depth;        // d_i
+    int32_t ctx_len;      // L_i
+    int32_t pad[3];
 };
 
 struct dcut_ctx {

@@ -129,8 +129,9 @@ struct PlanArgs {
     const int* ctx_lens;
     const int* cu_q;
     int B, n_q_heads, n_kv_heads;
-    int target_items, min_chunk_pages, max_items;
+    int target_items, min_chunk_pages, max_items, npad;
     long long part_rows_cap;
+    int* status;
     AttnItem* items;
     int* plan;       // [0] n_items, [1] chunk_pages, [2] total_pages, [3] partial rows used
     int* req_part;   // [B][2]: first partial row, n_chunks
@@ -164,29 +165,64 @@ __device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* to
     return res;
 }
 
+// Requests are ordered by the estimated duration of their items, longest first, so the CTAs that
+// start last are the short ones (the hardware hands items to SMs in index order as SMs free up).
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
+    extern __shared__ unsigned long long order[];   // [npad] (inverted cost << 32 | request), sorted ascending
     __shared__ int ws[33];
+    __shared__ int total_s;
     const int tid = threadIdx.x;
-    const int per = (a.B + kPlanThreads - 1) / kPlanThreads;
-    const int i0 = tid * per;
+    const int group = a.n_q_heads / a.n_kv_heads;
+    if (tid == 0) total_s = 0;
+    __syncthreads();
     int local = 0;
-    for (int e = 0; e < per; ++e) {
-        const int i = i0 + e;
-        if (i < a.B) {
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            local += (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-        }
+    for (int i = tid; i < a.B; i += kPlanThreads) {
+        const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+        local += (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
     }
-    int total_pages;
-    plan_block_exclusive_scan(local, ws, &total_pages);
-    long long units = (long long)total_pages * a.n_kv_heads;
+    if (local) atomicAdd(&total_s, local);
+    __syncthreads();
+    const int total_pages = total_s;
+    const long long units = (long long)total_pages * a.n_kv_heads;
     int chunk_pages = (int)((units + a.target_items - 1) / a.target_items);
     if (chunk_pages < a.min_chunk_pages) chunk_pages = a.min_chunk_pages;
 
+    for (int i = tid; i < a.npad; i += kPlanThreads) {
+        unsigned long long key = ~0ull;
+        if (i < a.B) {
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+            const int nc = (pages + chunk_pages - 1) / chunk_pages;
+            const int cp = (pages + nc - 1) / nc;
+            const int MT = ((d + 1) * group + 15) >> 4;
+            // per page: memory-bound below about two m-tiles, then time grows with the m-tiles
+            const unsigned int cost = (unsigned int)cp * (unsigned int)max(7, 3 * MT);
+            key = ((unsigned long long)(0xffffffffu - cost) << 32) | (unsigned int)i;
+        }
+        order[i] = key;
+    }
+    __syncthreads();
+    for (int k = 2; k <= a.npad; k <<= 1)
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = tid; t < (a.npad >> 1); t += kPlanThreads) {
+                const int i = 2 * t - (t & (j - 1)), l = i + j;
+                const bool up = (i & k) == 0;
+                const unsigned long long x = order[i], y = order[l];
+                if ((x > y) == up) {
+                    order[i] = y;
+                    order[l] = x;
+                }
+            }
+            __syncthreads();
+        }
+
+    const int per = (a.B + kPlanThreads - 1) / kPlanThreads;
+    const int j0 = tid * per;
     int my_items = 0, my_rows = 0;
     for (int e = 0; e < per; ++e) {
-        const int i = i0 + e;
-        if (i < a.B) {
+        const int j = j0 + e;
+        if (j < a.B) {
+            const int i = (int)(order[j] & 0xffffffffu);
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
             const int nc = (pages + chunk_pages - 1) / chunk_pages;
@@ -204,14 +240,17 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
         a.plan[2] = total_pages;
         a.plan[3] = n_rows;
         a.plan[4] = overflow ? 1 : 0;
+        if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
     }
     if (overflow) return;
-    const int group = a.n_q_heads / a.n_kv_heads;
     for (int e = 0; e < per; ++e) {
-        const int i = i0 + e;
-        if (i < a.B) {
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+        const int j = j0 + e;
+        if (j < a.B) {
+            const int i = (int)(order[j] & 0xffffffffu);
+            const int q0 = a.cu_q[i];
+            const int d = a.cu_q[i + 1] - q0 - 1;
+            const int ctx_len = a.ctx_lens[i];
+            const int pages = (ctx_len + d + 1 + kPage - 1) / kPage;
             const int nc = (pages + chunk_pages - 1) / chunk_pages;
             const int cp = (pages + nc - 1) / nc;   // near-equal chunks
             const int M = (d + 1) * group;
@@ -224,10 +263,12 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
                     it.kv_head = h;
                     it.page_begin = c * cp;
                     it.page_end = min(pages, (c + 1) * cp);
-                    it.chunk = c;
                     it.n_chunks = nc;
                     it.part_row = nc > 1 ? row_off + (c * a.n_kv_heads + h) * M : -1;
-                    it.pad = 0;
+                    it.q0 = q0;
+                    it.depth = d;
+                    it.ctx_len = ctx_len;
+                    it.pad[0] = it.pad[1] = it.pad[2] = 0;
                     a.items[item_off + c * a.n_kv_heads + h] = it;
                 }
             item_off += nc * a.n_kv_heads;
@@ -259,7 +300,6 @@ struct AttnArgs {
 
 template <int DH>
 struct SmemLayout {
-    static constexpr int kHalves = DH / 64;
     static constexpr int kPageBytes = kPage * DH * 2;            // one K or V page tile
     static constexpr int kStageBytes = 2 * kPageBytes;
     static constexpr int kRingBytes = kStages * kStageBytes;
@@ -289,9 +329,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int req = item.req, kvh = item.kv_head;
     const int group = a.n_q_heads / a.n_kv_heads;
-    const int q0 = a.cu_q[req];
-    const int depth = a.cu_q[req + 1] - q0 - 1;
-    const int ctx_len = a.ctx_lens[req];
+    const int q0 = item.q0, depth = item.depth, ctx_len = item.ctx_len;
     const int M = (depth + 1) * group;
     const int MT = (M + 15) >> 4;
     const int nslots = kConsumerWarps / MT;
@@ -568,27 +606,22 @@ struct CombineArgs {
     const float* part_o;
     const float* part_lse;
     const int* plan;
-    int B, n_q_heads, n_kv_heads;
+    int B, n_q_heads, n_kv_heads, tokens_per_req;
     __nv_bfloat16* out;
     float* lse;
 };
 
 template <int DH>
 __global__ void __launch_bounds__(256) attn_combine_kernel(CombineArgs a) {
+    // grid: x = request * (gamma_max + 1) + block position t, y = group of 8 q heads; warp = one head
     if (a.plan[4]) return;
-    const int T = a.cu_q[a.B];
-    const int gw = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
-    const int lane = threadIdx.x & 31;
-    if (gw >= T * a.n_q_heads) return;
-    const int tok = gw / a.n_q_heads, h = gw - tok * a.n_q_heads;
-    int lo = 0, hi = a.B;   // request with cu_q[i] <= tok < cu_q[i+1]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (a.cu_q[mid] <= tok) lo = mid; else hi = mid;
-    }
-    const int req = lo;
+    const int req = blockIdx.x / a.tokens_per_req, t = blockIdx.x - req * a.tokens_per_req;
     const int nc = a.req_part[2 * req + 1];
     if (nc <= 1) return;
+    const int lane = threadIdx.x & 31;
+    const int h = blockIdx.y * 8 + (threadIdx.x >> 5);
+    if (h >= a.n_q_heads || t >= a.cu_q[req + 1] - a.cu_q[req]) return;
+    const int tok = a.cu_q[req] + t;
     const int group = a.n_q_heads / a.n_kv_heads;
     const int q0 = a.cu_q[req];
     const int M = (a.cu_q[req + 1] - q0) * group;
@@ -648,9 +681,9 @@ dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm
     attn_split_kernel<DH><<<ctx->max_items, kThreads, SmemLayout<DH>::kTotal, stream>>>(km, vm, aa);
     dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_split_kernel");
     if (st != DCUT_OK) return st;
-    const long long warps = (long long)T_cap * ctx->lim.n_q_heads;
-    const int blocks = (int)((warps + 7) / 8);
-    attn_combine_kernel<DH><<<blocks, 256, 0, stream>>>(ca);
+    (void)T_cap;
+    dim3 cgrid(ca.B * ca.tokens_per_req, (ctx->lim.n_q_heads + 7) / 8);
+    attn_combine_kernel<DH><<<cgrid, 256, 0, stream>>>(ca);
     return dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_combine_kernel");
 }
 
@@ -663,6 +696,8 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
     e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              SmemLayout<64>::kTotal);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 64)");
+    e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS);
+    if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn plan)");
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
@@ -690,12 +725,15 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.n_kv_heads = ctx->lim.n_kv_heads;
     pa.target_items = ctx->target_items;
     pa.min_chunk_pages = 8;
+    pa.npad = 32;
+    while (pa.npad < B) pa.npad <<= 1;
+    pa.status = ctx->d_status;
     pa.max_items = ctx->max_items;
     pa.part_rows_cap = ctx->part_rows_cap;
     pa.items = ctx->d_items;
     pa.plan = ctx->d_plan;
     pa.req_part = ctx->d_req_part;
-    attn_plan_kernel<<<1, kPlanThreads, 0, stream>>>(pa);
+    attn_plan_kernel<<<1, kPlanThreads, sizeof(unsigned long long) * pa.npad, stream>>>(pa);
     st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_plan_kernel");
     if (st != DCUT_OK) return st;
 
@@ -726,6 +764,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     ca.B = B;
     ca.n_q_heads = ctx->lim.n_q_heads;
     ca.n_kv_heads = ctx->lim.n_kv_heads;
+    ca.tokens_per_req = ctx->lim.max_gamma + 1;
     ca.out = static_cast<__nv_bfloat16*>(out);
     ca.lse = lse;
 
