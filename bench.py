@@ -34,8 +34,9 @@ from paper_2607_14647_b200 import workloads as wl  # noqa: E402
 METRIC = "accepted_tokens_per_s_per_verify_step_B64"
 UNIT = "tokens/s"
 L2_BYTES = 126e6
-# DRAM bytes per algorithmic byte of attn_split_kernel measured with ncu (profiles/); None until captured
-ATTN_TRAFFIC_RATIO = None
+# DRAM bytes per algorithmic byte of attn_split_kernel, from the ncu capture on workload 1 summarised under
+# profiles/ (1.03 at gamma = 0 to 1.07 at full gamma); the kernel's traffic is proportional to the KV streamed
+ATTN_TRAFFIC_RATIO = 1.05
 
 
 def parse_args():
