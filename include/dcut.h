@@ -150,6 +150,49 @@ dcut_status dcut_accept(dcut_ctx* ctx, const void* logits, int V, const int* dra
                         int* n_accepted_total, void* stream);
 
 /*
+ * Dense projection on the tensor cores: out[T, N] = a[T, K] . w[N, K]^T  (bf16 in, fp32 accumulate, bf16 out),
+ * over the ragged packed batch (T = cu_q[B] read on the device, T_cap the host-known bound).  This is the
+ * building block of dcut_layer_forward, exported for tests and measurements.
+ *   mode 0: plain.   mode 1: out = residual + a . w^T (residual bf16 [T, N]).
+ *   mode 2: SwiGLU, out[T, N] = silu(a . w^T) * (a . w2^T) with w = gate weight, w2 = up weight, both [N, K].
+ * DEVICE pointers; a must have room for T_cap rows (rows past T are read and ignored).  Requirements: K a
+ * multiple of 64; N a multiple of 256 (128 in mode 2); all bases 128-byte aligned.
+ */
+dcut_status dcut_gemm_bf16(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
+                           const int* cu_q, int B, int T_cap, void* out, const void* residual, void* stream);
+
+/*
+ * One pre-norm decoder layer of the target model over the packed verification batch (the full-layer workload:
+ * the paper's verification forward is this layer repeated; Section 1 and Appendix C):
+ *   n  = RMSNorm(x) * g_attn;  [q|k|v] = n . w_qkv^T;  rotate-half RoPE (angle = position * theta^(-2e/Dh)) on q, k;
+ *   the new K (after RoPE) and V are written into the paged cache at position tok_pos = L_i + t;
+ *   a  = dcut_verify_attn(q, cache);  h1 = x + a . w_o^T;
+ *   n2 = RMSNorm(h1) * g_mlp;  y = h1 + (silu(n2 . w_gate^T) * (n2 . w_up^T)) . w_down^T.
+ * No biases, no q/k norm.  bf16 tensors, fp32 accumulation; intermediate tensors are rounded to bf16 where they
+ * are materialised (n, qkv, q/k after RoPE, a, h1, n2, the SwiGLU product, y).
+ * DEVICE in: x bf16 [T, hidden]; weights (w_qkv [(Hq+2Hkv)*Dh, hidden] rows = q heads, k heads, v heads;
+ *   w_o [hidden, Hq*Dh]; w_gate, w_up [intermediate, hidden]; w_down [hidden, intermediate]; g_attn, g_mlp
+ *   [hidden]); block_table, ctx_lens, cu_q, tok_req, tok_pos as written by dcut_select.
+ * DEVICE in/out: k_cache, v_cache (the step's new tokens are appended).   DEVICE out: y bf16 [T, hidden].
+ * Shapes come from dcut_limits (hidden, intermediate > 0).  Workspace lives in the context.
+ */
+typedef struct {
+    const void* w_qkv;
+    const void* w_o;
+    const void* w_gate;
+    const void* w_up;
+    const void* w_down;
+    const void* g_attn;
+    const void* g_mlp;
+    float rms_eps;
+    float rope_theta;
+} dcut_layer_weights;
+dcut_status dcut_layer_forward(dcut_ctx* ctx, const dcut_layer_weights* weights, const void* x, void* y, void* k_cache,
+                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                               int T_cap, void* stream);
+
+/*
  * dcut_accept without any allocation.  (The paper has no counterpart: this entry point exists for
  * the way the library gets embedded, not for the method.)
  *

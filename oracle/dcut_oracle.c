@@ -452,3 +452,11 @@ int oracle_num_threads(void) {
     return 1;
 #endif
 }
+
+/* SwiGLU on double inputs (the product is the only tensor the GPU materialises, so gate and up are
+ * not rounded in between): y = g / (1 + exp(-g)) * u */
+int oracle_swiglu_f64(const double* g, const double* u, long n, double* y) {
+    if (!g || !u || !y) return ORACLE_EINVAL;
+    for (long i = 0; i < n; ++i) y[i] = g[i] / (1.0 + exp(-g[i])) * u[i];
+    return ORACLE_OK;
+}

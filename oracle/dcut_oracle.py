@@ -254,3 +254,54 @@ def swiglu(g, u) -> np.ndarray:
     f.argtypes = [C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
     assert f(gb.ctypes.data, ub.ctypes.data, gb.size, y.ctypes.data) == 0
     return y
+
+
+def swiglu_f64(g: np.ndarray, u: np.ndarray) -> np.ndarray:
+    g = np.ascontiguousarray(g, np.float64)
+    u = np.ascontiguousarray(u, np.float64)
+    y = np.empty(g.shape, np.float64)
+    f = lib().oracle_swiglu_f64
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_long, C.c_void_p]
+    assert f(g.ctypes.data, u.ctypes.data, g.size, y.ctypes.data) == 0
+    return y
+
+
+def _as_bf16_tensor(bits: np.ndarray):
+    import torch
+    return torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16)
+
+
+def layer_forward(x, w, k_cache, v_cache, block_table, ctx_lens, depths, n_q_heads, n_kv_heads, head_dim, page_size,
+                  rms_eps, rope_theta):
+    """One pre-norm decoder layer on the packed batch, composed from the C pieces in double precision and
+    rounded to bf16 exactly where the GPU path materialises a tensor: n, qkv, q/k after RoPE, attention
+    output, h1, n2, the SwiGLU product, y.  `w` has w_qkv, w_o, w_gate, w_up, w_down, g_attn, g_mlp (torch bf16).
+    The K/V of the new tokens are written into COPIES of the caches at positions L_i + t.  Returns a dict of the
+    stages (torch bf16) plus the updated cache copies."""
+    import torch
+    depths = np.asarray(depths, np.int32)
+    B = len(depths)
+    cu = np.zeros(B + 1, np.int32)
+    np.cumsum(depths.astype(np.int64) + 1, out=cu[1:])
+    T = int(cu[-1])
+    pos = np.concatenate([int(ctx_lens[i]) + np.arange(depths[i] + 1) for i in range(B)]).astype(np.int32)
+    req = np.concatenate([np.full(depths[i] + 1, i) for i in range(B)])
+    rb = lambda a: _as_bf16_tensor(round_bf16(a))
+    n = rb(rmsnorm(x, w["g_attn"], rms_eps))
+    qkv = rb(linear(n, w["w_qkv"]))
+    q_w, kv_w = n_q_heads * head_dim, n_kv_heads * head_dim
+    q = rb(rope(qkv[:, :q_w].reshape(T, n_q_heads, head_dim).contiguous(), pos, rope_theta))
+    k = rb(rope(qkv[:, q_w:q_w + kv_w].reshape(T, n_kv_heads, head_dim).contiguous(), pos, rope_theta))
+    v = qkv[:, q_w + kv_w:].reshape(T, n_kv_heads, head_dim)
+    kc, vc = k_cache.clone(), v_cache.clone()
+    for r in range(T):
+        page = int(block_table[req[r], pos[r] // page_size])
+        kc[page, :, pos[r] % page_size] = k[r]
+        vc[page, :, pos[r] % page_size] = v[r]
+    attn, _ = verify_attn(q, kc, vc, block_table, ctx_lens, cu, n_q_heads, n_kv_heads, head_dim, page_size)
+    a = rb(attn.reshape(T, q_w))
+    h1 = rb(linear(a, w["w_o"]) + x.double().numpy())
+    n2 = rb(rmsnorm(h1, w["g_mlp"], rms_eps))
+    act = rb(swiglu_f64(linear(n2, w["w_gate"]), linear(n2, w["w_up"])))
+    y = rb(linear(act, w["w_down"]) + h1.double().numpy())
+    return dict(n=n, qkv=qkv, q=q, k=k, attn=a, h1=h1, n2=n2, act=act, y=y, k_cache=kc, v_cache=vc, cu_q=cu, pos=pos)

@@ -28,7 +28,7 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
-           "dcut_accept_static", "dcut_poll_device_status"]
+           "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -68,6 +68,16 @@ _lib.dcut_poll_device_status.argtypes = [_vp, C.POINTER(_i), _vp]
 
 _lib.dcut_accept_static.argtypes = [_vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, C.c_char_p, C.c_size_t]
 ACCEPT_STATIC_MAX_ROWS = 8192
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [(n, _vp) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")] + \
+               [("rms_eps", _f), ("rope_theta", _f)]
+
+
+_lib.dcut_gemm_bf16.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _vp, _vp]
+_lib.dcut_layer_forward.argtypes = [_vp, C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _vp, _vp,
+                                    _i, _i, _vp]
 
 
 class DcutError(RuntimeError):
@@ -254,6 +264,28 @@ class Context:
             out["attn_out"] = torch.zeros((B * (gamma + 1), self.limits.n_q_heads, self.limits.head_dim),
                                           dtype=torch.bfloat16, pin_memory=True)
         return out
+
+    def gemm_bf16(self, a, w, cu_q, T_cap: int, out, mode: int = 0, w2=None, residual=None):
+        """out[T, N] = a[T, K] . w[N, K]^T; mode 1 adds `residual`; mode 2 is SwiGLU with gate w and up w2."""
+        B = cu_q.shape[0] - 1
+        N, K = w.shape
+        self._check(_lib.dcut_gemm_bf16(self._h, _ptr(a, torch.bfloat16), _ptr(w, torch.bfloat16),
+                                        _ptr(w2, torch.bfloat16), mode, N, K, _ptr(cu_q, torch.int32), B, T_cap,
+                                        _ptr(out, torch.bfloat16), _ptr(residual, torch.bfloat16), _stream()))
+        return out
+
+    def layer_forward(self, weights: dict, x, y, k_cache, v_cache, block_table, ctx_lens, cu_q, tok_req, tok_pos,
+                      T_cap: int, rms_eps: float = 1e-6, rope_theta: float = 1e6):
+        """dcut_layer_forward; `weights` maps w_qkv, w_o, w_gate, w_up, w_down, g_attn, g_mlp to CUDA bf16 tensors."""
+        lw = LayerWeights(*[_ptr(weights[n], torch.bfloat16) for n in
+                            ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")], rms_eps, rope_theta)
+        B = ctx_lens.shape[0]
+        self._check(_lib.dcut_layer_forward(self._h, C.byref(lw), _ptr(x, torch.bfloat16), _ptr(y, torch.bfloat16),
+                                            _ptr(k_cache, torch.bfloat16), _ptr(v_cache, torch.bfloat16),
+                                            k_cache.shape[0], _ptr(block_table, torch.int32), block_table.shape[1],
+                                            _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32),
+                                            _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32), B, T_cap, _stream()))
+        return y
 
     def poll_device_status(self) -> int:
         code = _i(0)

@@ -53,6 +53,15 @@ void free_all(dcut_ctx* c) {
     cudaFree(c->d_part_lse);
     cudaFree(c->d_row_key);
     cudaFree(c->d_status);
+    cudaFree(c->ly_norm);
+    cudaFree(c->ly_qkv);
+    cudaFree(c->ly_q);
+    cudaFree(c->ly_attn);
+    cudaFree(c->ly_h1);
+    cudaFree(c->ly_norm2);
+    cudaFree(c->ly_act);
+    cudaFree(c->ly_inv_freq);
+    dcut_free_layer(c);
     cudaFree(c->hs_conf);
     cudaFree(c->hs_draft);
     cudaFree(c->hs_bonus);
@@ -125,6 +134,22 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
         if ((st = dmalloc(c, &c->d_part_lse, (size_t)c->part_rows_cap, "cudaMalloc(part_lse)")) != DCUT_OK) return st;
         if ((st = dcut_init_verify_attn(c)) != DCUT_OK) return st;
     }
+    if (lim->hidden > 0) {
+        if (!has_attn) return dcut_fail(c, DCUT_EINVAL, "the decoder layer needs the attention shapes");
+        const int q_w = lim->n_q_heads * lim->head_dim, qkv_w = (lim->n_q_heads + 2 * lim->n_kv_heads) * lim->head_dim;
+        if (lim->hidden % 256 || lim->intermediate % 128 || lim->intermediate < 128 || qkv_w % 256 || q_w % 64)
+            return dcut_fail(c, DCUT_EINVAL, "layer shapes: hidden %% 256, intermediate %% 128, (Hq+2Hkv)*Dh %% 256 must be 0");
+        const size_t mt = (size_t)max_T;
+        if ((st = dmalloc(c, &c->ly_norm, mt * lim->hidden, "cudaMalloc(layer norm)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_qkv, mt * qkv_w, "cudaMalloc(layer qkv)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_q, mt * q_w, "cudaMalloc(layer q)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_attn, mt * q_w, "cudaMalloc(layer attn)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_h1, mt * lim->hidden, "cudaMalloc(layer h1)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_norm2, mt * lim->hidden, "cudaMalloc(layer norm2)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_act, mt * lim->intermediate, "cudaMalloc(layer act)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_inv_freq, (size_t)lim->head_dim / 2, "cudaMalloc(inv_freq)")) != DCUT_OK) return st;
+    }
+    if (has_attn && (st = dcut_init_layer(c)) != DCUT_OK) return st;
     return dcut_check_cuda(c, cudaDeviceSynchronize(), "cudaDeviceSynchronize(create)");
 }
 
@@ -244,6 +269,54 @@ dcut_status dcut_accept(dcut_ctx* c, const void* logits, int V, const int* draft
     if (reinterpret_cast<uintptr_t>(logits) & 1) return dcut_fail(c, DCUT_EINVAL, "logits must be 2-byte aligned");
     return dcut_launch_accept(c, logits, V, draft_ids, cu_q, B, gamma, T_cap, accept_len, bonus, out_tokens,
                               n_accepted_total, c->d_row_key, static_cast<cudaStream_t>(stream));
+}
+
+dcut_status dcut_gemm_bf16(dcut_ctx* c, const void* a, const void* w, const void* w2, int mode, int N, int K,
+                           const int* cu_q, int B, int T_cap, void* out, const void* residual, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (!c->layer_maps) return dcut_fail(c, DCUT_EINVAL, "context was created without attention shapes (no tensor-map encoder)");
+    if (!a || !w || !cu_q || !out || (mode == 2 && !w2) || (mode == 1 && !residual) || mode < 0 || mode > 2)
+        return dcut_fail(c, DCUT_EINVAL, "null pointer or bad mode");
+    if (B < 1 || T_cap < 1 || K < 64 || K % 64 || N < 1 || N % (mode == 2 ? 128 : 256))
+        return dcut_fail(c, DCUT_EINVAL, "need K %% 64 == 0 and N %% 256 == 0 (128 in SwiGLU mode)");
+    if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(out) |
+         reinterpret_cast<uintptr_t>(w2) | reinterpret_cast<uintptr_t>(residual)) & 127)
+        return dcut_fail(c, DCUT_EINVAL, "operands must be 128-byte aligned");
+    return dcut_launch_gemm(c, a, w, w2, mode, N, K, cu_q, B, T_cap, out, residual, static_cast<cudaStream_t>(stream));
+}
+
+dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
+                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                               int T_cap, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (c->lim.hidden <= 0 || !c->ly_norm) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
+    if (!w || !w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down || !w->g_attn || !w->g_mlp || !x || !y ||
+        !k_cache || !v_cache || !block_table || !ctx_lens || !cu_q || !tok_req || !tok_pos)
+        return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (B < 1 || T_cap < B || B > c->lim.max_B || T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
+        return dcut_fail(c, DCUT_ECAPACITY, "B = %d, T_cap = %d outside the limits", B, T_cap);
+    if (block_table_stride < 1 || block_table_stride > c->lim.max_pages_per_req)
+        return dcut_fail(c, DCUT_ECAPACITY, "block_table_stride = %d outside [1, %d]", block_table_stride, c->lim.max_pages_per_req);
+    if (!(w->rope_theta > 1.0f) || !(w->rms_eps >= 0.0f)) return dcut_fail(c, DCUT_EINVAL, "rope_theta must exceed 1, rms_eps >= 0");
+    const uintptr_t al = reinterpret_cast<uintptr_t>(w->w_qkv) | reinterpret_cast<uintptr_t>(w->w_o) |
+                         reinterpret_cast<uintptr_t>(w->w_gate) | reinterpret_cast<uintptr_t>(w->w_up) |
+                         reinterpret_cast<uintptr_t>(w->w_down) | reinterpret_cast<uintptr_t>(k_cache) |
+                         reinterpret_cast<uintptr_t>(v_cache);
+    if ((al & 127) || ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) |
+                        reinterpret_cast<uintptr_t>(w->g_attn) | reinterpret_cast<uintptr_t>(w->g_mlp)) & 15))
+        return dcut_fail(c, DCUT_EINVAL, "weights and caches must be 128-byte aligned, x / y / gains 16-byte aligned");
+    if (c->ly_theta != w->rope_theta) {   // first call (or a new theta): build the inverse-frequency table in fp64
+        const int half = c->lim.head_dim / 2;
+        float tab[128];
+        for (int e = 0; e < half; ++e) tab[e] = (float)pow((double)w->rope_theta, -2.0 * e / c->lim.head_dim);
+        dcut_status st = dcut_check_cuda(c, cudaMemcpyAsync(c->ly_inv_freq, tab, sizeof(float) * half, cudaMemcpyHostToDevice,
+                                                            static_cast<cudaStream_t>(stream)), "cudaMemcpyAsync(inv_freq)");
+        if (st != DCUT_OK) return st;
+        c->ly_theta = w->rope_theta;
+    }
+    return dcut_launch_layer(c, w, x, y, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q,
+                             tok_req, tok_pos, B, T_cap, static_cast<cudaStream_t>(stream));
 }
 
 dcut_status dcut_poll_device_status(dcut_ctx* c, int* code, void* stream) {

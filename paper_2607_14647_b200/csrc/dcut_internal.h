@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libdcut.so (not installed).
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -14,6 +15,7 @@
 #define DCUT_DEV_ATTN_WAIT_TIMEOUT 1   // a bounded mbarrier wait in the attention kernel gave up
 #define DCUT_DEV_BAD_PAGE 2            // a block-table entry outside [0, num_pages)
 #define DCUT_DEV_PLAN_OVERFLOW 3       // the attention work list did not fit the context's scratch
+#define DCUT_DEV_GEMM_WAIT_TIMEOUT 4    // a bounded mbarrier wait in the GEMM kernel gave up
 
 // One split-KV work item of the attention kernel: one (request, kv head, page range).
 struct __align__(16) AttnItem {
@@ -61,6 +63,12 @@ struct dcut_ctx {
     // tensor-map encoder (driver entry point fetched through the runtime)
     void* encode_tiled;
 
+    // decoder-layer workspace (hidden > 0 only), all [max_T, width] bf16
+    __nv_bfloat16 *ly_norm, *ly_qkv, *ly_q, *ly_attn, *ly_h1, *ly_norm2, *ly_act;
+    float* ly_inv_freq;     // [head_dim / 2]
+    float ly_theta;         // theta the table was built for (0 = none yet)
+    void* layer_maps;       // cached tensor maps (layer.cu)
+
     // staging of dcut_verify_step_host (allocated by its first call)
     int hs_ready, hs_vocab;
     float* hs_conf;
@@ -76,6 +84,8 @@ dcut_status dcut_check_cuda(dcut_ctx* ctx, cudaError_t e, const char* what);
 dcut_status dcut_init_select(dcut_ctx* ctx);
 dcut_status dcut_init_accept(dcut_ctx* ctx);
 dcut_status dcut_init_verify_attn(dcut_ctx* ctx);
+dcut_status dcut_init_layer(dcut_ctx* ctx);
+void dcut_free_layer(dcut_ctx* ctx);
 
 // kernel launchers (one per translation unit)
 dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
@@ -90,3 +100,9 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
                                     long long num_pages, const int* block_table, int block_table_stride,
                                     const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
                                     void* out, float* lse, cudaStream_t stream);
+dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
+                             const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream);
+dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
+                              void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                              const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                              int T_cap, cudaStream_t stream);

@@ -1,0 +1,485 @@
+// dcut_layer_forward: one pre-norm decoder layer over the ragged packed batch (full-layer workload).
+//
+//   h1 = x + Wo . Attn(RoPE(Wqkv . RMSNorm(x)))        y = h1 + Wd . (SiLU(Wg . n2) * (Wu . n2)),  n2 = RMSNorm(h1)
+//
+// Kernels in this file
+//   rmsnorm_kernel        one CTA per packed token, fp32 sum of squares, bf16 out
+//   rope_append_kernel    rotate-half RoPE on q and k heads, K/V of the new tokens written into the paged cache at
+//                         position L_i + t, q written as the attention kernel's [T, Hq, Dh] input
+//   gemm_tcgen05_kernel   C[M, N] = A[M, K] . B[N, K]^T on the 5th-generation tensor cores: 128 x 256 output tile
+//                         per CTA, accumulator in tensor memory (256 fp32 columns), operands staged by TMA into a
+//                         4-stage ring of 128-byte-swizzled K-major tiles (BK = 64), one thread issuing
+//                         tcgen05.mma (M128 N256 K16) and releasing stages with tcgen05.commit, four epilogue warps
+//                         reading the accumulator with tcgen05.ld.  Epilogues: plain bf16, + residual, or SwiGLU
+//                         (the B tile is 128 gate rows followed by the 128 matching up rows, so silu(g) * u is
+//                         formed in registers and the [T, 2I] intermediate never exists).
+// M is ragged and known only on the device (T = cu_q[B]): grids are sized for T_cap, CTAs past T leave at once,
+// rows past T are computed on whatever the buffers hold and never stored.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "dcut_internal.h"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, kGemmStages = 4;
+constexpr int kATile = BM * BK * 2;            // 16 KB
+constexpr int kBTile = BN * BK * 2;            // 32 KB
+constexpr int kGemmStageBytes = kATile + kBTile;
+constexpr int kGemmThreads = 192;              // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int kTmemCols = 256;
+constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256 /* barriers, tmem ptr */;
+constexpr int kWaitLimit = 1 << 22;
+
+enum GemmMode { kPlain = 0, kResidual = 1, kSwiGLU = 2 };
+
+// ------------------------------------------------------------------------------------------------ PTX
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (int it = 0; it < kWaitLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 8192) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] . B[smem desc]^T, M128 N256 K16, bf16 in, fp32 accumulate
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with the 128-byte
+// swizzle: 8-row groups are 1024 bytes apart (stride byte offset), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffff) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                               // leading byte offset: unused with this swizzle
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
+    d |= (uint64_t)1 << 46;                               // descriptor version
+    d |= (uint64_t)2 << 61;                               // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = 256, M = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// ------------------------------------------------------------------------------------------------ GEMM
+
+struct GemmArgs {
+    const int* cu_q;   // T = cu_q[B]
+    int B;
+    int N_out;         // columns of the output (kSwiGLU: the intermediate size I; otherwise N)
+    int K;
+    __nv_bfloat16* out;
+    const __nv_bfloat16* residual;   // [T, N_out] or null
+    int* status;
+};
+
+template <int MODE>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
+                    const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
+    const int T = g.cu_q[g.B];
+    const int m0 = blockIdx.x * BM;
+    if (m0 >= T) return;
+    const int n_tile = blockIdx.y;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGemmStages + 1);
+    const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
+    const uint32_t accum_bar = smem_u32(bars + 2 * kGemmStages);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_kb = g.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGemmStages; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        mbar_init(accum_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // tensor memory: 256 columns for the 128 x 256 fp32 accumulator
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool failed = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ TMA producer
+            for (int kb = 0; kb < n_kb; ++kb) {
+                const int s = kb % kGemmStages;
+                if (kb >= kGemmStages && !mbar_wait(empty_bar + 8 * s, ((kb / kGemmStages) - 1) & 1)) {
+                    failed = true;
+                    break;
+                }
+                const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
+                const uint32_t bar = full_bar + 8 * s;
+                mbar_arrive_expect_tx(bar, kGemmStageBytes);
+                tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
+                if (MODE == kSwiGLU) {   // 128 gate rows, then the 128 up rows of the same features
+                    tma_load_2d(b_dst, &b_map, kb * BK, n_tile * (BN / 2), bar);
+                    tma_load_2d(b_dst + kBTile / 2, &b2_map, kb * BK, n_tile * (BN / 2), bar);
+                } else {
+                    tma_load_2d(b_dst, &b_map, kb * BK, n_tile * BN, bar);
+                    tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ MMA issuer
+            for (int kb = 0; kb < n_kb; ++kb) {
+                const int s = kb % kGemmStages;
+                if (!mbar_wait(full_bar + 8 * s, (kb / kGemmStages) & 1)) {
+                    failed = true;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
+                const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
+                    tc_mma(tmem_base, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+                tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
+            }
+            tc_commit(accum_bar);                   // accumulator complete
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int quarter = warp & 3;               // tensor-memory lanes 32 * quarter .. + 31
+        const int row = m0 + quarter * 32 + lane;
+        if (!mbar_wait(accum_bar, 0)) failed = true;
+        tc_fence_after();
+        if (!failed) {
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            if (MODE == kSwiGLU) {
+                __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + (size_t)n_tile * (BN / 2);
+#pragma unroll 1
+                for (int c = 0; c < BN / 2; c += 32) {
+                    uint32_t gt[32], up[32];
+                    tc_ld32(t_row + c, gt);
+                    tc_ld32(t_row + BN / 2 + c, up);
+                    tc_wait_ld();
+                    if (row < T) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float g0 = __uint_as_float(gt[e + 2 * j]), g1 = __uint_as_float(gt[e + 2 * j + 1]);
+                                const float u0 = __uint_as_float(up[e + 2 * j]), u1 = __uint_as_float(up[e + 2 * j + 1]);
+                                w[j] = pack_bf16(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+                            }
+                            *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+            } else {
+                __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + (size_t)n_tile * BN;
+                const __nv_bfloat16* rrow = MODE == kResidual ? g.residual + (size_t)row * g.N_out + (size_t)n_tile * BN : nullptr;
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t acc[32];
+                    tc_ld32(t_row + c, acc);
+                    tc_wait_ld();
+                    if (row < T) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint4 res = make_uint4(0, 0, 0, 0);
+                            if (MODE == kResidual) res = *reinterpret_cast<const uint4*>(rrow + c + e);
+                            const uint32_t rw[4] = {res.x, res.y, res.z, res.w};
+                            uint32_t w[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                w[j] = pack_bf16(__uint_as_float(acc[e + 2 * j]) + bf_lo(rw[j]),
+                                                 __uint_as_float(acc[e + 2 * j + 1]) + bf_hi(rw[j]));
+                            *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    if (failed) atomicExch(g.status, DCUT_DEV_GEMM_WAIT_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ RMSNorm
+
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
+                                                      const int* __restrict__ cu_q, int B, int hidden, float eps,
+                                                      __nv_bfloat16* __restrict__ y) {
+    const int row = blockIdx.x;
+    if (row >= cu_q[B]) return;
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * hidden);
+    const uint4* gr = reinterpret_cast<const uint4*>(gain);
+    uint4* yr = reinterpret_cast<uint4*>(y + (size_t)row * hidden);
+    const int nvec = hidden >> 3;
+    float ss = 0.0f;
+    for (int v = threadIdx.x; v < nvec; v += 256) {
+        const uint4 a = xr[v];
+        const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) ss += bf_lo(w[j]) * bf_lo(w[j]) + bf_hi(w[j]) * bf_hi(w[j]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    __shared__ float wsum[8];
+    if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.0f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += wsum[w];
+    const float inv = rsqrtf(tot / (float)hidden + eps);
+    for (int v = threadIdx.x; v < nvec; v += 256) {
+        const uint4 a = xr[v], gq = gr[v];
+        const uint32_t w[4] = {a.x, a.y, a.z, a.w}, gw[4] = {gq.x, gq.y, gq.z, gq.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[j] = pack_bf16(bf_lo(w[j]) * inv * bf_lo(gw[j]), bf_hi(w[j]) * inv * bf_hi(gw[j]));
+        yr[v] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ RoPE + KV append
+
+struct RopeArgs {
+    const __nv_bfloat16* qkv;   // [T, (Hq + 2 Hkv) * Dh]: q heads, k heads, v heads
+    const int* cu_q;
+    const int* tok_req;
+    const int* tok_pos;
+    const int* block_table;
+    int block_table_stride;
+    const float* inv_freq;      // [Dh / 2] = theta^(-2e/Dh)
+    int B, n_q_heads, n_kv_heads, head_dim;
+    long long num_pages;
+    __nv_bfloat16* q_out;       // [T, Hq, Dh]
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    int* status;
+};
+
+__global__ void __launch_bounds__(256) rope_append_kernel(RopeArgs a) {
+    const int tok = blockIdx.x;
+    if (tok >= a.cu_q[a.B]) return;
+    const int Dh = a.head_dim, half = Dh >> 1;
+    const int req = a.tok_req[tok], pos = a.tok_pos[tok];
+    int page = a.block_table[(size_t)req * a.block_table_stride + pos / 16];
+    if (page < 0 || page >= a.num_pages) {
+        if (threadIdx.x == 0) atomicExch(a.status, DCUT_DEV_BAD_PAGE);
+        return;
+    }
+    const int slot = pos & 15;
+    const int row_w = (a.n_q_heads + 2 * a.n_kv_heads) * Dh;
+    const __nv_bfloat16* row = a.qkv + (size_t)tok * row_w;
+    const int n_rot = (a.n_q_heads + a.n_kv_heads) * half;   // rotated pairs of the q and k heads
+    for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
+        const int h = idx / half, e = idx - h * half;
+        float sn, cs;
+        sincosf((float)pos * a.inv_freq[e], &sn, &cs);
+        const float x0 = __bfloat162float(row[h * Dh + e]), x1 = __bfloat162float(row[h * Dh + e + half]);
+        const __nv_bfloat16 y0 = __float2bfloat16_rn(x0 * cs - x1 * sn), y1 = __float2bfloat16_rn(x1 * cs + x0 * sn);
+        if (h < a.n_q_heads) {
+            __nv_bfloat16* q = a.q_out + ((size_t)tok * a.n_q_heads + h) * Dh;
+            q[e] = y0;
+            q[e + half] = y1;
+        } else {
+            __nv_bfloat16* k = a.k_cache + (((size_t)page * a.n_kv_heads + (h - a.n_q_heads)) * 16 + slot) * Dh;
+            k[e] = y0;
+            k[e + half] = y1;
+        }
+    }
+    const __nv_bfloat16* vrow = row + (a.n_q_heads + a.n_kv_heads) * Dh;
+    for (int idx = threadIdx.x; idx < a.n_kv_heads * Dh; idx += blockDim.x) {
+        const int h = idx / Dh, e = idx - h * Dh;
+        a.v_cache[(((size_t)page * a.n_kv_heads + h) * 16 + slot) * Dh + e] = vrow[idx];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// K-major bf16 matrix [rows, cols] as a 2-D tensor map with a {64 columns, box_rows} box and 128-byte swizzle
+dcut_status make_kmajor_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return dcut_fail(ctx, DCUT_ECUDA, "cuTensorMapEncodeTiled failed for a GEMM operand (%d)", (int)r);
+    return DCUT_OK;
+}
+
+template <int MODE>
+dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& b2, int n_tiles,
+                        int T_cap, const GemmArgs& g, cudaStream_t stream) {
+    dim3 grid((T_cap + BM - 1) / BM, n_tiles);
+    gemm_tcgen05_kernel<MODE><<<grid, kGemmThreads, kGemmSmem, stream>>>(a, b, b2, g);
+    return dcut_check_cuda(ctx, cudaGetLastError(), "launch gemm_tcgen05_kernel");
+}
+
+struct LayerMaps {
+    const void* w[5];
+    CUtensorMap m[5];   // w_qkv, w_o, w_gate, w_up, w_down
+    CUtensorMap act[4]; // norm out, attention out, norm-2 out, mlp activation
+    bool act_ready;
+};
+
+}  // namespace
+
+dcut_status dcut_init_layer(dcut_ctx* ctx) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(gemm)");
+    ctx->layer_maps = calloc(1, sizeof(LayerMaps));
+    return ctx->layer_maps ? DCUT_OK : dcut_fail(ctx, DCUT_EINVAL, "out of host memory");
+}
+
+void dcut_free_layer(dcut_ctx* ctx) { free(ctx->layer_maps); }
+
+dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
+                             const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream) {
+    // generic entry used by dcut_gemm_bf16 (tests, benchmarks): encodes its maps on every call
+    CUtensorMap am, bm, b2m;
+    dcut_status st = make_kmajor_map(ctx, &am, a, T_cap, K, BM);
+    if (st != DCUT_OK) return st;
+    const int rows_w = mode == kSwiGLU ? N : N;
+    if ((st = make_kmajor_map(ctx, &bm, w, rows_w, K, BN / 2)) != DCUT_OK) return st;
+    b2m = bm;
+    if (mode == kSwiGLU && (st = make_kmajor_map(ctx, &b2m, w2, rows_w, K, BN / 2)) != DCUT_OK) return st;
+    GemmArgs g;
+    g.cu_q = cu_q;
+    g.B = B;
+    g.N_out = N;
+    g.K = K;
+    g.out = static_cast<__nv_bfloat16*>(out);
+    g.residual = static_cast<const __nv_bfloat16*>(residual);
+    g.status = ctx->d_status;
+    if (mode == kSwiGLU) return launch_gemm<kSwiGLU>(ctx, am, bm, b2m, N / (BN / 2), T_cap, g, stream);
+    if (mode == kResidual) return launch_gemm<kResidual>(ctx, am, bm, b2m, N / BN, T_cap, g, stream);
+    return launch_gemm<kPlain>(ctx, am, bm, b2m, N / BN, T_cap, g, stream);
+}
+
+dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
+                              void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                              const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                              int T_cap, cudaStream_t stream) {
+    const dcut_limits& l = ctx->lim;
+    const int H = l.hidden, I = l.intermediate, Dh = l.head_dim;
+    const int qkv_w = (l.n_q_heads + 2 * l.n_kv_heads) * Dh, q_w = l.n_q_heads * Dh;
+    const int max_T = l.max_B * (l.max_gamma + 1);
+    LayerMaps* lm = static_cast<LayerMaps*>(ctx->layer_maps);
+    dcut_status st;
+    if (!lm->act_ready) {
+        if ((st = make_kmajor_map(ctx, &lm->act[0], ctx->ly_norm, max_T, H, BM)) != DCUT_OK) return st;
+        if ((st = make_kmajor_map(ctx, &lm->act[1], ctx->ly_attn, max_T, q_w, BM)) != DCUT_OK) return st;
+        if ((st = make_kmajor_map(ctx, &lm->act[2], ctx->ly_norm2, max_T, H, BM)) != DCUT_OK) return st;
+        if ((st = make_kmajor_map(ctx, &lm->act[3], ctx->ly_act, max_T, I, BM)) != DCUT_OK) return st;
+        lm->act_ready = true;
+    }
+    const void* wp[5] = {w->w_qkv, w->w_o, w->w_gate, w->w_up, w->w_down};
+    const long long wr[5] = {qkv_w, H, I, I, H}, wc[5] = {H, q_w, H, H, I};
+    for (int i = 0; i < 5; ++i)
+        if (lm->w[i] != wp[i]) {
+            if ((st = make_kmajor_map(ctx, &lm->m[i], wp[i], wr[i], wc[i], BN / 2)) != DCUT_OK) return st;
+            lm->w[i] = wp[i];
+        }
+    GemmArgs g;
+    g.cu_q = cu_q;
+    g.B = B;
+    g.status = ctx->d_status;
+
+    // 1. n = RMSNorm(x)
+    rmsnorm_kernel<<<T_cap, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w->g_attn),
+                                              cu_q, B, H, w->rms_eps, ctx->ly_norm);
+    // 2. qkv = n . Wqkv^T
+    g.N_out = qkv_w; g.K = H; g.out = ctx->ly_qkv; g.residual = nullptr;
+    if ((st = launch_gemm<kPlain>(ctx, lm->act[0], lm->m[0], lm->m[0], qkv_w / BN, T_cap, g, stream)) != DCUT_OK) return st;
+    // 3. RoPE, append the new K/V to the paged cache
+    RopeArgs r;
+    r.qkv = ctx->ly_qkv; r.cu_q = cu_q; r.tok_req = tok_req; r.tok_pos = tok_pos; r.block_table = block_table;
+    r.block_table_stride = block_table_stride; r.inv_freq = ctx->ly_inv_freq; r.B = B; r.n_q_heads = l.n_q_heads;
+    r.n_kv_heads = l.n_kv_heads; r.head_dim = Dh; r.num_pages = num_pages; r.q_out = ctx->ly_q;
+    r.k_cache = static_cast<__nv_bfloat16*>(k_cache); r.v_cache = static_cast<__nv_bfloat16*>(v_cache); r.status = ctx->d_status;
+    rope_append_kernel<<<T_cap, 256, 0, stream>>>(r);
+    if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch rope_append_kernel")) != DCUT_OK) return st;
+    // 4. attention
+    st = dcut_launch_verify_attn(ctx, ctx->ly_q, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens,
+                                 cu_q, B, T_cap, 1.0f / sqrtf((float)Dh), ctx->ly_attn, nullptr, stream);
+    if (st != DCUT_OK) return st;
+    // 5. h1 = x + attn . Wo^T
+    g.N_out = H; g.K = q_w; g.out = ctx->ly_h1; g.residual = static_cast<const __nv_bfloat16*>(x);
+    if ((st = launch_gemm<kResidual>(ctx, lm->act[1], lm->m[1], lm->m[1], H / BN, T_cap, g, stream)) != DCUT_OK) return st;
+    // 6. n2 = RMSNorm(h1)
+    rmsnorm_kernel<<<T_cap, 256, 0, stream>>>(ctx->ly_h1, static_cast<const __nv_bfloat16*>(w->g_mlp), cu_q, B, H, w->rms_eps, ctx->ly_norm2);
+    // 7. act = SiLU(n2 . Wg^T) * (n2 . Wu^T)
+    g.N_out = I; g.K = H; g.out = ctx->ly_act; g.residual = nullptr;
+    if ((st = launch_gemm<kSwiGLU>(ctx, lm->act[2], lm->m[2], lm->m[3], I / (BN / 2), T_cap, g, stream)) != DCUT_OK) return st;
+    // 8. y = h1 + act . Wd^T
+    g.N_out = H; g.K = I; g.out = static_cast<__nv_bfloat16*>(y); g.residual = ctx->ly_h1;
+    return launch_gemm<kResidual>(ctx, lm->act[3], lm->m[4], lm->m[4], H / BN, T_cap, g, stream);
+}

@@ -1,0 +1,114 @@
+"""Decoder-layer path against the oracle: the tcgen05 GEMM by itself (all three epilogues), RMSNorm + RoPE + cache
+append through the whole layer on a small shape (every element, every stage that is visible), and the full-layer
+workload on a sub-batch of requests the oracle can afford.  Tolerance 2e-2 + 2e-2 |ref| (bf16 tensors, fp32
+accumulation over K up to 12 288; the paper gives none)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dcut_oracle as orc
+from paper_2607_14647_b200 import workloads as wl
+from tests.gpu_helpers import dev, make_ctx
+
+pytestmark = pytest.mark.gpu
+
+
+def _close(got, want, what):
+    got = got.float().cpu().numpy().astype(np.float64)
+    want = want.float().numpy().astype(np.float64) if isinstance(want, torch.Tensor) else np.asarray(want, np.float64)
+    err = np.abs(got - want)
+    lim = 2e-2 + 2e-2 * np.abs(want)
+    assert (err <= lim).all(), f"{what}: worst err/limit {(err / lim).max():.2f} at {np.unravel_index((err / lim).argmax(), err.shape)}"
+
+
+def _bf(rng, shape, scale=1.0):
+    return torch.from_numpy((rng.standard_normal(shape, dtype=np.float32) * scale)).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("T,N,K", [(1, 256, 64), (100, 256, 128), (128, 512, 512), (129, 256, 1024), (300, 768, 4096),
+                                   (517, 256, 12288)])
+def test_gemm_plain_and_residual(T, N, K):
+    rng = np.random.default_rng(T + N + K)
+    cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
+    ctx = make_ctx(cfg, max_pages=1, vocab=0)
+    T_cap = max(T, 2)
+    a, w, res = _bf(rng, (T_cap, K)), _bf(rng, (N, K), 0.05), _bf(rng, (T_cap, N))
+    cu = dev(np.array([0, T], np.int32))
+    out = torch.full((T_cap, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(w), cu, T_cap, out)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    ref = orc.linear(a[:T], w)
+    _close(out[:T], ref, "plain")
+    assert (out[T:] == 7.0).all()                      # rows past T are never stored
+    out2 = torch.empty((T_cap, N), dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(w), cu, T_cap, out2, mode=1, residual=dev(res))
+    _close(out2[:T], ref + res[:T].double().numpy(), "residual")
+    ctx.close()
+
+
+@pytest.mark.parametrize("T,I,K", [(70, 128, 256), (260, 384, 512), (131, 1024, 4096)])
+def test_gemm_swiglu(T, I, K):
+    rng = np.random.default_rng(T + I + K)
+    cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
+    ctx = make_ctx(cfg, max_pages=1, vocab=0)
+    a, wg, wu = _bf(rng, (T, K)), _bf(rng, (I, K), 0.05), _bf(rng, (I, K), 0.05)
+    out = torch.empty((T, I), dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(wg), dev(np.array([0, T], np.int32)), T, out, mode=2, w2=dev(wu))
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    _close(out, orc.swiglu_f64(orc.linear(a, wg), orc.linear(a, wu)), "swiglu")
+    ctx.close()
+
+
+def _layer_case(cfg, depths, hidden, inter, sub=None):
+    """Runs the GPU layer on the whole batch and the oracle on the requests in `sub` (default: all)."""
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    w = wl.layer_weights(cfg, hidden, inter)
+    wd = {n: getattr(w, n) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")}
+    x = wl.layer_x_rows(cfg, depths, hidden)
+    cu = wl.cu_q_from_depths(depths)
+    tok_req = np.concatenate([np.full(d + 1, i) for i, d in enumerate(depths)]).astype(np.int32)
+    tok_pos = np.concatenate([sel.ctx_lens[i] + np.arange(d + 1) for i, d in enumerate(depths)]).astype(np.int32)
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req, hidden=hidden, intermediate=inter, vocab=0)
+    d_k, d_v = dev(kv.k_cache), dev(kv.v_cache)
+    y = torch.empty((int(cu[-1]), hidden), dtype=torch.bfloat16, device="cuda")
+    ctx.layer_forward({k: dev(v) for k, v in wd.items()}, dev(x), y, d_k, d_v, dev(kv.block_table), dev(sel.ctx_lens),
+                      dev(cu), dev(tok_req), dev(tok_pos), cfg.t_cap, cfg.rms_eps, cfg.rope_theta)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    ctx.close()
+    sub = list(range(cfg.B)) if sub is None else sub
+    rows = np.concatenate([np.arange(cu[i], cu[i + 1]) for i in sub])
+    ref = orc.layer_forward(x[rows], wd, kv.k_cache, kv.v_cache, kv.block_table[sub], sel.ctx_lens[sub], depths[sub],
+                            cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.page_size, cfg.rms_eps, cfg.rope_theta)
+    _close(y[rows], ref["y"], "layer output y")
+    # the appended K/V of the new tokens (the rest of the cache must be untouched)
+    kc, vc = d_k.cpu(), d_v.cpu()
+    for n_, i in enumerate(sub):
+        for t in range(depths[i] + 1):
+            pos = int(sel.ctx_lens[i]) + t
+            page = kv.block_table[i, pos // 16]
+            _close(kc[page, :, pos % 16], ref["k_cache"][page, :, pos % 16], "appended K")
+            _close(vc[page, :, pos % 16], ref["v_cache"][page, :, pos % 16], "appended V")
+    if len(sub) == cfg.B:
+        touched = torch.zeros(kc.shape[0], dtype=torch.bool)
+        for i in range(cfg.B):
+            for t in range(depths[i] + 1):
+                touched[kv.block_table[i, (int(sel.ctx_lens[i]) + t) // 16]] = True
+        assert torch.equal(kc[~touched], kv.k_cache[~touched]) and torch.equal(vc[~touched], kv.v_cache[~touched])
+
+
+def test_small_layer_every_element():
+    cfg = wl.custom_config(B=6, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128, ctx_lo=5, ctx_hi=400,
+                           conf_kind="skew_halves")
+    _layer_case(cfg, np.array([16, 0, 3, 9, 1, 16], np.int32), hidden=512, inter=1024)
+
+
+def test_full_layer_workload_on_sampled_requests():
+    cfg = wl.config(4)
+    sel = wl.select_inputs(cfg)
+    depths = orc.select(sel.conf, sel.draft_ids, sel.bonus_ids, sel.ctx_lens,
+                        wl.cost_table_linear(cfg.t_cap + 1, 0.5, 0.001)).depths
+    _layer_case(cfg, depths, cfg.hidden, cfg.intermediate, sub=[0, 1, 37])
