@@ -56,49 +56,63 @@ def parse_args():
 # ------------------------------------------------------------------------------------------------ helpers
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+    """Samples the SM clock and the throttle reasons through NVML (read-only) from a thread while the timed
+    region runs; falls back to one nvidia-smi query if NVML is not importable."""
+    REASONS = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4}
 
-    def __init__(self, index: int):
-        self.path = tempfile.mktemp(prefix="dcut_clocks_", suffix=".csv")
-        self.proc = None
+    def __init__(self, index: int, period_s: float = 0.005):
+        import threading
+        self.sm, self.reasons, self.max_mhz, self.index = [], set(), None, index
+        self._stop = threading.Event()
+        self._thread = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            # CUDA_VISIBLE_DEVICES remaps ordinals: find the NVML device by the CUDA device's UUID
+            uuid = str(torch.cuda.get_device_properties(index).uuid)
+            self._h = None
+            for i in range(pynvml.nvmlDeviceGetCount()):
+                h = pynvml.nvmlDeviceGetHandleByIndex(i)
+                u = pynvml.nvmlDeviceGetUUID(h)
+                u = u.decode() if isinstance(u, bytes) else u
+                if uuid in u:
+                    self._h = h
+            if self._h is None:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self._thread = threading.Thread(target=self._run, args=(period_s,), daemon=True)
+            self._thread.start()
         except Exception:
-            self.proc = None
+            self._nv = None
+
+    def _run(self, period_s):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for name, bit in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(period_s)
 
     def stop(self) -> dict:
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        try:
-            rows = [r.strip().split(",") for r in open(self.path) if r.strip()]
-            os.unlink(self.path)
-        except Exception:
-            return out
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in rows:
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join(timeout=2)
+        if not self.sm:      # fallback: a single nvidia-smi reading taken now
             try:
-                sm.append(float(r[0]))
-                mx.append(float(r[1]))
-                for n, v in zip(names, r[3:7]):
-                    if v.strip().lower().startswith("active"):
-                        reasons.add(n)
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=clocks.sm,clocks.max.sm",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=20).stdout
+                a, b = out.strip().split(",")
+                return {"sm_mhz": float(a), "sm_max_mhz": float(b), "reasons": [], "samples": 1, "source": "nvidia-smi"}
             except Exception:
-                continue
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
-        return out
+                return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.sm), "sm_min_mhz": min(self.sm), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm), "source": "nvml"}
 
 
 def dist_setup(n_gpus: int):
@@ -180,6 +194,13 @@ def host_inputs(cfg):
     return sel, kv, q_all, logits_all
 
 
+def layer_flops(cfg, T: int) -> float:
+    """Dense-projection flops of one layer for T packed tokens (2 * T * parameters)."""
+    qkv_w = (cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim
+    params = qkv_w * cfg.hidden + cfg.hidden * cfg.n_q_heads * cfg.head_dim + 3 * cfg.intermediate * cfg.hidden
+    return 2.0 * T * params
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -229,30 +250,45 @@ def run_dcut(args):
     d_k, d_v = kv.k_cache.to(dev), kv.v_cache.to(dev)
     d_q_all = q_all.to(dev).view(cfg.t_cap, cfg.n_q_heads, cfg.head_dim)
     d_logits_all = logits_all.to(dev).view(cfg.t_cap, cfg.vocab)
+    is_layer = cfg.hidden > 0
     ctx = binding.Context(max_B=cfg.B, max_gamma=cfg.gamma, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
                           head_dim=cfg.head_dim, page_size=cfg.page_size, max_pages_per_req=kv.max_pages_per_req,
-                          vocab=cfg.vocab)
+                          vocab=cfg.vocab, hidden=cfg.hidden, intermediate=cfg.intermediate)
     cap = cfg.t_cap
     sel_out = None
+    if is_layer:
+        lw = wl.layer_weights(cfg)
+        d_w = {n: getattr(lw, n).to(dev) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")}
+        d_x_all = wl.layer_x_rows(cfg, np.full(cfg.B, cfg.gamma, np.int32)).to(dev)
 
     def pack(depths_np):
         """Gathers the kept rows (i, t <= d_i) of the unpacked device tensors (set-up, not timed)."""
         idx = np.concatenate([i * (cfg.gamma + 1) + np.arange(d + 1) for i, d in enumerate(depths_np)])
         idx_t = torch.from_numpy(idx).to(dev)
-        return d_q_all.index_select(0, idx_t).contiguous(), d_logits_all.index_select(0, idx_t).contiguous()
+        first = d_x_all if is_layer else d_q_all
+        return first.index_select(0, idx_t).contiguous(), d_logits_all.index_select(0, idx_t).contiguous()
 
     res = {}
+
+    def middle(qp, so, bufs):
+        """The verification forward between selection and acceptance: attention, or the whole decoder layer."""
+        if is_layer:
+            ctx.layer_forward(d_w, qp, bufs["attn_out"], d_k, d_v, d_bt, d_ctx, so.cu_q, so.tok_req, so.tok_pos, cap,
+                              cfg.rms_eps, cfg.rope_theta)
+        else:
+            ctx.verify_attn(qp, d_k, d_v, d_bt, d_ctx, so.cu_q, cap, out=bufs["attn_out"])
 
     def step(qp, lp, bufs):
         nonlocal sel_out
         sel_out = ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=sel_out)
-        ctx.verify_attn(qp, d_k, d_v, d_bt, d_ctx, sel_out.cu_q, cap, out=bufs["attn_out"])
+        middle(qp, sel_out, bufs)
         ctx.accept_into(lp, d_draft, sel_out.cu_q, cap, bufs["accept_len"], bufs["bonus"], bufs["out_tokens"],
                         bufs["total"])
 
     def make_bufs(T):
         i32 = dict(dtype=torch.int32, device=dev)
-        return dict(attn_out=torch.empty((T, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device=dev),
+        mid = (T, cfg.hidden) if is_layer else (T, cfg.n_q_heads, cfg.head_dim)
+        return dict(attn_out=torch.empty(mid, dtype=torch.bfloat16, device=dev),
                     accept_len=torch.empty(cfg.B, **i32), bonus=torch.empty(cfg.B, **i32),
                     out_tokens=torch.empty((cfg.B, cfg.gamma + 1), **i32), total=torch.empty(1, **i32))
 
@@ -302,7 +338,7 @@ def run_dcut(args):
         for k in range(args.steps):
             nonlocal_sel = ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=sel_out)
             ev[k][0].record()
-            ctx.verify_attn(qp, d_k, d_v, d_bt, d_ctx, nonlocal_sel.cu_q, cap, out=bufs["attn_out"])
+            middle(qp, nonlocal_sel, bufs)
             ev[k][1].record()
             ctx.accept_into(lp, d_draft, nonlocal_sel.cu_q, cap, bufs["accept_len"], bufs["bonus"],
                             bufs["out_tokens"], bufs["total"])
@@ -320,23 +356,59 @@ def run_dcut(args):
 
     # ---- end to end from host buffers ---------------------------------------------------------
     ctx.set_cost_dense(cost)
-    pin = lambda t: t.contiguous().pin_memory()
-    h = dict(conf=pin(torch.from_numpy(sel.conf)), draft=pin(torch.from_numpy(sel.draft_ids)),
-             bonus=pin(torch.from_numpy(sel.bonus_ids)), ctx=pin(torch.from_numpy(sel.ctx_lens)),
-             bt=pin(torch.from_numpy(kv.block_table)), q=pin(q_all), logits=pin(logits_all))
-    hout = ctx.host_step_outputs(cfg.B, cfg.gamma)
-    call = lambda: ctx.verify_step_host(h["conf"], h["draft"], h["bonus"], h["ctx"], h["bt"], h["q"], h["logits"],
-                                        d_k, d_v, out=hout)
-    for _ in range(3):
-        call()
-    barrier(world)
-    t0 = time.perf_counter()
-    for _ in range(args.e2e_steps):
-        call()
-    barrier(world)
-    e2e_s = max_over_ranks(time.perf_counter() - t0, world) / args.e2e_steps
-    e2e_accepted = int(hout["n_accepted_total"].item())
-    assert e2e_accepted == res["pruned"]["accepted"], (e2e_accepted, res["pruned"]["accepted"])
+    e2e = None
+    if not is_layer:
+        pin = lambda t: t.contiguous().pin_memory()
+        h = dict(conf=pin(torch.from_numpy(sel.conf)), draft=pin(torch.from_numpy(sel.draft_ids)),
+                 bonus=pin(torch.from_numpy(sel.bonus_ids)), ctx=pin(torch.from_numpy(sel.ctx_lens)),
+                 bt=pin(torch.from_numpy(kv.block_table)), q=pin(q_all), logits=pin(logits_all))
+        hout = ctx.host_step_outputs(cfg.B, cfg.gamma)
+        call = lambda: ctx.verify_step_host(h["conf"], h["draft"], h["bonus"], h["ctx"], h["bt"], h["q"], h["logits"],
+                                            d_k, d_v, out=hout)
+        for _ in range(3):
+            call()
+        barrier(world)
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            call()
+        barrier(world)
+        e2e_s = max_over_ranks(time.perf_counter() - t0, world) / args.e2e_steps
+        e2e_accepted = int(hout["n_accepted_total"].item())
+        assert e2e_accepted == res["pruned"]["accepted"], (e2e_accepted, res["pruned"]["accepted"])
+        e2e = {"value": world * e2e_accepted / e2e_s, "unit": UNIT, "ms_per_step": round(e2e_s * 1e3, 4),
+               "h2d_bytes_per_step": hout["h2d_bytes"], "d2h_bytes_per_step": hout["d2h_bytes"],
+               "api": "dcut_verify_step_host (pinned host buffers; KV cache resident)"}
+
+    # ---- the four projections of the layer, timed alone (tensor roofline) ---------------------------
+    gemm = None
+    if is_layer and rank == 0:
+        gemm = {}
+        qkv_w, q_w = (cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim, cfg.n_q_heads * cfg.head_dim
+        for arm in ("pruned", "full_gamma"):
+            T = res[arm]["T"]
+            cu1 = torch.tensor([0, T], dtype=torch.int32, device=dev)
+            rows = {}
+            for name, (w, w2, mode, K, N) in {"qkv": (d_w["w_qkv"], None, 0, cfg.hidden, qkv_w),
+                                              "o": (d_w["w_o"], None, 1, q_w, cfg.hidden),
+                                              "gate_up_swiglu": (d_w["w_gate"], d_w["w_up"], 2, cfg.hidden, cfg.intermediate),
+                                              "down": (d_w["w_down"], None, 1, cfg.intermediate, cfg.hidden)}.items():
+                a_in = torch.randn((cap, K), device=dev, dtype=torch.float32).to(torch.bfloat16)
+                outb = torch.empty((cap, N), dtype=torch.bfloat16, device=dev)
+                resb = torch.zeros((cap, N), dtype=torch.bfloat16, device=dev) if mode == 1 else None
+                for _ in range(3):
+                    ctx.gemm_bf16(a_in, w, cu1, cap, outb, mode=mode, w2=w2, residual=resb)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(20):
+                    ctx.gemm_bf16(a_in, w, cu1, cap, outb, mode=mode, w2=w2, residual=resb)
+                e1.record()
+                e1.synchronize()
+                ms = e0.elapsed_time(e1) / 20
+                fl = 2.0 * T * K * N * (2 if mode == 2 else 1)
+                rows[name] = {"ms": round(ms, 4), "tflops": round(fl / ms / 1e9, 1)}
+            tot_ms = sum(r["ms"] for r in rows.values())
+            rows["all"] = {"ms": round(tot_ms, 4), "tflops": round(layer_flops(cfg, T) / tot_ms / 1e9, 1)}
+            gemm[arm] = rows
 
     if rank != 0:
         return
@@ -363,14 +435,22 @@ def run_dcut(args):
                      "frac_of_8000_nominal": round(achieved / 8000.0, 4),
                      "algorithmic_bytes_per_launch": p["attn_bytes"],
                      "traffic": None if ATTN_TRAFFIC_RATIO is None else int(ATTN_TRAFFIC_RATIO * p["attn_bytes"])},
-        "e2e": {"value": world * e2e_accepted / e2e_s, "unit": UNIT, "ms_per_step": round(e2e_s * 1e3, 4),
-                "h2d_bytes_per_step": hout["h2d_bytes"], "d2h_bytes_per_step": hout["d2h_bytes"],
-                "api": "dcut_verify_step_host (pinned host buffers; KV cache resident)"},
-        "gpu_launches": 6 * args.steps,
+        "e2e": e2e,
+        "gpu_launches": (14 if is_layer else 6) * args.steps,
         "cost_table_ms": {str(t): round(c, 4) for t, c in zip(grid, prof)},
         "clocks": clocks,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if is_layer:
+        pkj = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+        tf_peak = float(pkj.get("bf16_tflops", 1590.0))
+        line["config"]["arm"] += "; verification forward = one decoder layer (dcut_layer_forward)"
+        line["layer"] = {"gemm_alone": gemm, "flops_per_token": layer_flops(cfg, 1)}
+        g = gemm["full_gamma"]["all"]
+        line["roofline_tensor"] = {"kernel": "gemm_tcgen05_kernel (4 projections of the layer, full-gamma arm, timed alone)",
+                                   "bound": "tensor", "achieved": g["tflops"], "peak": tf_peak, "unit": "TFLOP/s",
+                                   "frac": round(g["tflops"] / tf_peak, 4),
+                                   "peak_source": "of measured (burst)" if pkj else "of fallback", "traffic": None}
+    if world == 1 and not args.no_cpu_baseline and not is_layer:
         info, *_ = oracle_sample(cfg, sel, kv, q_all, logits_all, cost, args.cpu_seconds)
         line["cpu_baseline"] = info
     print(json.dumps(line))
