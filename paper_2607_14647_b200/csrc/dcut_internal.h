@@ -54,6 +54,7 @@ struct dcut_ctx {
     int max_items;
     long long part_rows_cap;
     int target_items;
+    int attn_tc_min_rows;   // items with at least this many query rows (and <= 128) use the tcgen05 kernel
 
     // accept scratch
     unsigned long long* d_row_key;   // [max_T] packed (ordered max, ~index); zero between calls

@@ -26,6 +26,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA sets the device status word and leaves.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <stdlib.h>
 
 #include "dcut_internal.h"
 
@@ -129,7 +130,7 @@ struct PlanArgs {
     const int* ctx_lens;
     const int* cu_q;
     int B, n_q_heads, n_kv_heads;
-    int target_items, min_chunk_pages, max_items, npad;
+    int target_items, min_chunk_pages, max_items, npad, tc_min_rows;
     long long part_rows_cap;
     int* status;
     AttnItem* items;
@@ -268,7 +269,8 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
                     it.q0 = q0;
                     it.depth = d;
                     it.ctx_len = ctx_len;
-                    it.pad[0] = it.pad[1] = it.pad[2] = 0;
+                    it.pad[0] = (M >= a.tc_min_rows && M <= 128) ? 1 : 0;   // which kernel takes the item
+                    it.pad[1] = it.pad[2] = 0;
                     a.items[item_off + c * a.n_kv_heads + h] = it;
                 }
             item_off += nc * a.n_kv_heads;
@@ -326,6 +328,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     __shared__ int abort_s;
 
     const AttnItem item = a.items[blockIdx.x];
+    if (item.pad[0]) return;   // many query rows: handled by the tcgen05 kernel
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int req = item.req, kvh = item.kv_head;
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -597,6 +600,355 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// tcgen05 variant of the split kernel for items with many query rows (head_dim 128, rows <= 128).
+//
+// With 3+ m-tiles the warp-level MMA path is bound by the tensor pipe and by operand traffic through
+// registers, not by HBM.  Here the query tile is padded to 128 rows (row = tensor-memory lane) and lives in
+// tensor memory for the whole item; pages are handled in groups of four (64 keys):
+//   S[128, 64]  = Q . K_group^T     8 MMAs (M128 N64 K16): A = Q from tensor memory, B = the group's K tiles,
+//                 which TMA lays out contiguously so the 64 key rows form one K-major operand;
+//                 accumulator in tensor memory, double-buffered;
+//   softmax     128 threads, one per row: tcgen05.ld of the row, mask, running max and sum without any
+//                 shuffle; P goes back as bf16 into the columns S occupied (tcgen05.st), so it never
+//                 touches shared memory; O is only rescaled when a row's maximum grows by more than 2^8;
+//   O[128, 128] += P . V_page       one MMA (M128 N128 K16) per page: A = P from tensor memory, B = the V tile
+//                 read MN-major (transposed by its descriptor); accumulator in tensor memory for the item.
+// Both MMAs therefore stream only K and V from shared memory.  Warp 0: TMA producer (4 lanes, one page of
+// every group each), warp 1: MMA issuer and tensor-memory owner, warps 2-5: softmax + epilogue.
+constexpr int kTcGroupStages = 4;                  // ring of page groups
+constexpr int kTcThreads = 192;
+constexpr int kTcPageBytes = kPage * 128 * 2;      // 4 KB: one K or V page tile
+constexpr int kTcGroupBytes = 8 * kTcPageBytes;    // K of 4 pages (16 KB, [half][64 rows][64]) + V of 4 pages
+constexpr int kTcSmem = kTcGroupStages * kTcGroupBytes + 1024 + 256;
+constexpr int kTcCols = 512;                       // O: 0..127, S/P buffers: 128..191 and 192..255, Q: 256..319
+constexpr int kTcColS = 128, kTcColQ = 256;
+constexpr float kRescaleLog2 = 8.0f;
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[tmem] . B[smem descriptor]
+__device__ __forceinline__ void tc_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+          "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+          "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+
+// K-major tile with 128-byte rows and 128-byte swizzle: 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3ffff) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+// MN-major tile (rows = K index, 128 bytes = 64 consecutive MN elements per row): the next 64 MN elements are
+// 2048 bytes on (leading byte offset), the next 8 K rows 1024 bytes on (stride byte offset)
+__device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
+    return (uint64_t)((addr & 0x3ffff) >> 4) | ((uint64_t)(2048 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+           ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// instruction descriptors: fp32 accumulate, bf16 operands, M = 128; QK^T: B K-major, N = 16 per page in the group;
+// PV: B MN-major, N = 128
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16) | ((128u >> 3) << 17);
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant__ CUtensorMap v_map, AttnArgs a) {
+    if ((int)blockIdx.x >= a.plan[0]) return;
+    const AttnItem item = a.items[blockIdx.x];
+    if (!item.pad[0]) return;                      // handled by the warp-level kernel
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    unsigned char* ring = smem;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(ring + kTcGroupStages * kTcGroupBytes);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcGroupStages + 6);
+    __shared__ int abort_s;
+    const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kTcGroupStages);
+    const uint32_t s_full = smem_u32(bars + 2 * kTcGroupStages), p_full = s_full + 16, pv_done = s_full + 32;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int req = item.req, kvh = item.kv_head;
+    const int group = a.n_q_heads / a.n_kv_heads;
+    const int q0 = item.q0, ctx_len = item.ctx_len;
+    const int M = (item.depth + 1) * group;
+    const int n_pages = item.page_end - item.page_begin;
+    const int n_groups = (n_pages + 3) >> 2;
+
+    if (tid == 0) {
+        abort_s = 0;
+        for (int s = 0; s < kTcGroupStages; ++s) {
+            mbar_init(full_bar + 8 * s, 4);          // one arrival per page slot of the group
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(s_full + 8 * b, 1);
+            mbar_init(p_full + 8 * b, 128);
+            mbar_init(pv_done + 8 * b, 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTcCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_o = *tmem_slot;
+    bool failed = false;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        // lane l loads page l of every group; the group's full barrier takes four arrivals, so a lane whose
+        // page does not exist (last group) still arrives, without bytes
+        if (lane < 4) {
+            const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
+            int next = lane < n_pages ? bt[lane] : 0;
+            for (int g = 0; g < n_groups; ++g) {
+                const int p = 4 * g + lane;
+                int page_id = next;
+                if (p + 4 < n_pages) next = bt[p + 4];
+                const int gs = g % kTcGroupStages, use = g / kTcGroupStages;
+                if ((use > 0 && !mbar_wait(empty_bar + 8 * gs, (use - 1) & 1, &abort_s)) || *(volatile int*)&abort_s) {
+                    failed = true;
+                    break;
+                }
+                const uint32_t bar = full_bar + 8 * gs;
+                if (p >= n_pages) {
+                    mbar_arrive(bar);
+                    continue;
+                }
+                if (page_id < 0 || page_id >= a.num_pages) {
+                    atomicExch(a.status, DCUT_DEV_BAD_PAGE);
+                    page_id = 0;
+                }
+                const uint32_t dst = smem_u32(ring + gs * kTcGroupBytes);
+                const int row = (page_id * a.n_kv_heads + kvh) * kPage;
+                mbar_arrive_expect_tx(bar, 2 * kTcPageBytes);
+                tma_load_2d(dst + lane * 2048, &k2_map, 0, row, bar);            // K columns 0..63 of the page
+                tma_load_2d(dst + 8192 + lane * 2048, &k2_map, 64, row, bar);    // K columns 64..127
+                tma_load_tile(dst + 4 * kTcPageBytes + lane * kTcPageBytes, &v_map, row, bar);
+            }
+        }
+    } else {
+        const uint32_t tmem_q = tmem_o + kTcColQ;
+        if (warp >= 2) {
+            // the query tile goes to tensor memory: thread = row R = lane of tensor memory, 128 bf16 = 64 words
+            const int R = (warp & 3) * 32 + lane;
+            uint32_t qw[64];
+            if (R < M) {
+                const int t = R / group, hl = R - t * group;
+                const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128);
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const uint4 v = src[c];
+                    qw[4 * c] = v.x; qw[4 * c + 1] = v.y; qw[4 * c + 2] = v.z; qw[4 * c + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) qw[c] = 0;
+            }
+            const uint32_t t_q = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
+            tc_st32(t_q, qw);
+            tc_st32(t_q + 32, qw + 32);
+            tc_wait_st();
+            tc_fence_before();
+        }
+        asm volatile("bar.sync 1, 160;" ::: "memory");                      // MMA warp + softmax warps
+        if (warp == 1) {
+            if (lane == 0) {
+                // ------------------------------------------------------------ MMA issuer
+                tc_fence_after();
+                auto issue_qk = [&](int g) -> bool {
+                    const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages;
+                    if (!mbar_wait(full_bar + 8 * gs, (g / kTcGroupStages) & 1, &abort_s)) return false;
+                    tc_fence_after();
+                    const uint32_t k_addr = smem_u32(ring + gs * kTcGroupBytes);
+                    const uint32_t d = tmem_o + kTcColS + 64 * (g & 1);
+                    const uint32_t idesc = kIdescBase | ((uint32_t)(np * kPage >> 3) << 17);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)    // 16 head-dim elements = 8 words of Q, 32 bytes along a K row
+                            tc_mma_ts(d, tmem_q + (h * 4 + ks) * 8, desc_kmajor(k_addr + h * 8192) + 2 * ks, idesc, (h | ks) ? 1u : 0u);
+                    tc_commit(s_full + 8 * (g & 1));
+                    return true;
+                };
+                bool ok = issue_qk(0);
+                for (int g = 0; ok && g < n_groups; ++g) {
+                    if (g + 1 < n_groups) {
+                        // the S/P buffer of group g+1 was last used by group g-1
+                        if (g >= 1 && !mbar_wait(pv_done + 8 * ((g + 1) & 1), ((g - 1) >> 1) & 1, &abort_s)) { ok = false; break; }
+                        if (!issue_qk(g + 1)) { ok = false; break; }
+                    }
+                    if (!mbar_wait(p_full + 8 * (g & 1), (g >> 1) & 1, &abort_s)) { ok = false; break; }
+                    tc_fence_after();
+                    const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages;
+                    const uint32_t v_addr = smem_u32(ring + gs * kTcGroupBytes) + 4 * kTcPageBytes;
+                    const uint32_t tmem_p = tmem_o + kTcColS + 64 * (g & 1);
+                    for (int j = 0; j < np; ++j)           // 16 keys = 8 words of P
+                        tc_mma_ts(tmem_o, tmem_p + 8 * j, desc_mnmajor(v_addr + j * kTcPageBytes), kIdescPV, (g | j) ? 1u : 0u);
+                    tc_commit(empty_bar + 8 * gs);         // the group's K and V tiles are free again
+                    tc_commit(pv_done + 8 * (g & 1));
+                }
+                if (!ok) failed = true;
+            }
+        } else {
+            // ---------------------------------------------------------------- softmax + epilogue, thread = row
+            const int R = (warp & 3) * 32 + lane;
+            const uint32_t t_lane = tmem_o + ((uint32_t)((warp & 3) * 32) << 16);
+            const int jmax = ctx_len + min(R, M - 1) / group;           // last visible cache position
+            const float c = a.scale_log2;
+            float m_run = -INFINITY, l_run = 0.0f;
+            for (int g = 0; g < n_groups; ++g) {
+                if (!mbar_wait(s_full + 8 * (g & 1), (g >> 1) & 1, &abort_s)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t t_s = t_lane + kTcColS + 64 * (g & 1);
+                uint32_t sr[64];
+                tc_ld32(t_s, sr);
+                tc_ld32(t_s + 32, sr + 32);
+                tc_wait_ld();
+                const int ncols = min(4, n_pages - 4 * g) * kPage;
+                const int j0 = (item.page_begin + 4 * g) * kPage;
+                float mx = -INFINITY;
+                if (ncols < 64 || j0 + 63 > ctx_len) {                  // a partial group or one that holds hidden keys
+                    const int lim = min(ncols - 1, jmax - j0);          // columns 0..lim are visible
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) {
+                        const float v = e <= lim ? __uint_as_float(sr[e]) : -INFINITY;
+                        sr[e] = __float_as_uint(v);
+                        mx = fmaxf(mx, v);
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sr[e]));
+                }
+                // the running maximum only moves (and O is only rescaled) when it would grow by more than 2^8
+                float alpha = 1.0f;
+                bool moved = false;
+                if (mx > m_run && (m_run == -INFINITY || (mx - m_run) * c > kRescaleLog2)) {
+                    alpha = fast_exp2((m_run - mx) * c);                  // 0 when nothing was visible before
+                    m_run = mx;
+                    l_run *= alpha;
+                    moved = g > 0;
+                }
+                if (g > 0 && __any_sync(0xffffffffu, moved)) {
+                    // O is being updated by the previous group's MMAs: wait for them, then scale this warp's rows
+                    if (!mbar_wait(pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, &abort_s)) { failed = true; break; }
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int cc = 0; cc < 128; cc += 32) {
+                        uint32_t o[32];
+                        tc_ld32(t_lane + cc, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tc_st32(t_lane + cc, o);
+                    }
+                    tc_wait_st();
+                }
+                const float mc = (m_run == -INFINITY ? 0.0f : m_run) * c;
+                float sum = 0.0f;
+                uint32_t pw[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), c, -mc));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), c, -mc));
+                    sum += p0 + p1;
+                    pw[e] = pack_bf16(p0, p1);
+                }
+                l_run += sum;
+                tc_st32(t_s, pw);                                       // P over the columns S occupied
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(p_full + 8 * (g & 1));
+            }
+            // epilogue: the item's O row, normalised
+            if (!failed && !mbar_wait(pv_done + 8 * ((n_groups - 1) & 1), ((n_groups - 1) >> 1) & 1, &abort_s)) failed = true;
+            tc_fence_after();
+            if (!failed) {
+                const float inv = l_run > 0.0f ? 1.0f / l_run : 0.0f;
+                const float lse_nat = l_run > 0.0f ? (m_run * c + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+                const int t = R / group, hl = R - t * group;
+                const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+#pragma unroll 1
+                for (int cc = 0; cc < 128; cc += 32) {
+                    uint32_t o[32];
+                    tc_ld32(t_lane + cc, o);
+                    tc_wait_ld();
+                    if (R < M) {
+                        if (item.n_chunks == 1) {
+#pragma unroll
+                            for (int e = 0; e < 32; e += 8) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    w[j] = pack_bf16(__uint_as_float(o[e + 2 * j]) * inv, __uint_as_float(o[e + 2 * j + 1]) * inv);
+                                *reinterpret_cast<uint4*>(a.out + orow * 128 + cc + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        } else {
+                            float* po = a.part_o + ((size_t)item.part_row + R) * 128 + cc;
+#pragma unroll
+                            for (int e = 0; e < 32; e += 4)
+                                *reinterpret_cast<float4*>(po + e) =
+                                    make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
+                                                __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+                        }
+                    }
+                }
+                if (R < M) {
+                    if (item.n_chunks == 1) {
+                        if (a.lse) a.lse[orow] = lse_nat;
+                    } else {
+                        a.part_lse[(size_t)item.part_row + R] = lse_nat;
+                    }
+                }
+            }
+        }
+    }
+    if (failed) {
+        atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
+        *(volatile int*)&abort_s = 1;
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_o), "n"(kTcCols) : "memory");
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // combine the chunks of multi-chunk requests: one warp per (token, q head)
 
@@ -676,11 +1028,15 @@ dcut_status make_cache_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, lo
 }
 
 template <int DH>
-dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm, const AttnArgs& aa,
+dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& k2m, const AttnArgs& aa,
                      const CombineArgs& ca, int T_cap, cudaStream_t stream) {
+    dcut_status st;
+    if (DH == 128 && ctx->attn_tc_min_rows <= 128) {
+        attn_tc_kernel<<<ctx->max_items, kTcThreads, kTcSmem, stream>>>(k2m, vm, aa);
+        if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_tc_kernel")) != DCUT_OK) return st;
+    }
     attn_split_kernel<DH><<<ctx->max_items, kThreads, SmemLayout<DH>::kTotal, stream>>>(km, vm, aa);
-    dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_split_kernel");
-    if (st != DCUT_OK) return st;
+    if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_split_kernel")) != DCUT_OK) return st;
     (void)T_cap;
     dim3 cgrid(ca.B * ca.tokens_per_req, (ctx->lim.n_q_heads + 7) / 8);
     attn_combine_kernel<DH><<<cgrid, 256, 0, stream>>>(ca);
@@ -696,6 +1052,12 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
     e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              SmemLayout<64>::kTotal);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 64)");
+    e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+    if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn tc)");
+    {
+        const char* env = getenv("DCUT_ATTN_TC_MIN_ROWS");   // query rows from which an item goes to the tcgen05 kernel
+        ctx->attn_tc_min_rows = env ? atoi(env) : 33;
+    }
     e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn plan)");
     void* fn = nullptr;
@@ -711,11 +1073,22 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
                                     long long num_pages, const int* block_table, int block_table_stride,
                                     const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
                                     void* out, float* lse, cudaStream_t stream) {
-    CUtensorMap km, vm;
+    CUtensorMap km, vm, k2m;
     dcut_status st = make_cache_map(ctx, &km, k_cache, num_pages);
     if (st != DCUT_OK) return st;
     st = make_cache_map(ctx, &vm, v_cache, num_pages);
     if (st != DCUT_OK) return st;
+    k2m = km;
+    if (ctx->lim.head_dim == 128) {   // the K cache as a plain 2-D matrix of token rows, {64 columns, 16 rows} boxes
+        cuuint64_t dims[2] = {128, (cuuint64_t)num_pages * ctx->lim.n_kv_heads * kPage};
+        cuuint64_t strides[1] = {256};
+        cuuint32_t box[2] = {64, kPage}, estr[2] = {1, 1};
+        CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+            &k2m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(k_cache), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return dcut_fail(ctx, DCUT_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+    }
 
     PlanArgs pa;
     pa.ctx_lens = ctx_lens;
@@ -728,6 +1101,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.npad = 32;
     while (pa.npad < B) pa.npad <<= 1;
     pa.status = ctx->d_status;
+    pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
     pa.max_items = ctx->max_items;
     pa.part_rows_cap = ctx->part_rows_cap;
     pa.items = ctx->d_items;
@@ -768,6 +1142,6 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     ca.out = static_cast<__nv_bfloat16*>(out);
     ca.lse = lse;
 
-    if (ctx->lim.head_dim == 128) return launch_t<128>(ctx, km, vm, aa, ca, T_cap, stream);
-    return launch_t<64>(ctx, km, vm, aa, ca, T_cap, stream);
+    if (ctx->lim.head_dim == 128) return launch_t<128>(ctx, km, vm, k2m, aa, ca, T_cap, stream);
+    return launch_t<64>(ctx, km, vm, k2m, aa, ca, T_cap, stream);
 }
