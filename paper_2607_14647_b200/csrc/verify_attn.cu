@@ -27,6 +27,12 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdlib.h>
+#ifdef DCUT_PROFILE_TC
+#include <stdio.h>
+#define TCP(...) __VA_ARGS__
+#else
+#define TCP(...)
+#endif
 
 #include "dcut_internal.h"
 
@@ -71,6 +77,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // bounded wait: false if the phase did not complete within the spin limit, or another warp of the
 // CTA has already given up
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
     for (int it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it > 4096) {
@@ -315,11 +323,9 @@ struct SmemLayout {
 };
 
 template <int DH>
-__global__ void __launch_bounds__(kThreads, 1)
-attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map, AttnArgs a) {
+__device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnArgs& a,
+                                           const AttnItem& item, unsigned char* smem_raw) {
     using L = SmemLayout<DH>;
-    if ((int)blockIdx.x >= a.plan[0]) return;
-    extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* ring = smem;
     unsigned char* q_s = smem + L::kRingOrMerge;
@@ -327,8 +333,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(ml_s) + L::kMLBytes);
     __shared__ int abort_s;
 
-    const AttnItem item = a.items[blockIdx.x];
-    if (item.pad[0]) return;   // many query rows: handled by the tcgen05 kernel
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int req = item.req, kvh = item.kv_head;
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -617,13 +621,15 @@ attn_split_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_consta
 //                 read MN-major (transposed by its descriptor); accumulator in tensor memory for the item.
 // Both MMAs therefore stream only K and V from shared memory.  Warp 0: TMA producer (4 lanes, one page of
 // every group each), warp 1: MMA issuer and tensor-memory owner, warps 2-5: softmax + epilogue.
-constexpr int kTcGroupStages = 4;                  // ring of page groups
-constexpr int kTcThreads = 192;
+constexpr int kTcGroupStages = 6;                  // ring of page groups (192 KB in flight)
+constexpr int kTcSBufs = 3;                        // S/P buffers in tensor memory: groups in flight between QK^T and PV
+constexpr int kTcSoftmaxThreads = 256;             // two threads per row, 32 columns each
+constexpr int kTcThreads = 64 + kTcSoftmaxThreads;
 constexpr int kTcPageBytes = kPage * 128 * 2;      // 4 KB: one K or V page tile
 constexpr int kTcGroupBytes = 8 * kTcPageBytes;    // K of 4 pages (16 KB, [half][64 rows][64]) + V of 4 pages
 constexpr int kTcSmem = kTcGroupStages * kTcGroupBytes + 1024 + 256;
-constexpr int kTcCols = 512;                       // O: 0..127, S/P buffers: 128..191 and 192..255, Q: 256..319
-constexpr int kTcColS = 128, kTcColQ = 256;
+constexpr int kTcCols = 512;                       // O: 0..127, S/P buffers: 128..319, Q: 320..383
+constexpr int kTcColS = 128, kTcColQ = kTcColS + 64 * kTcSBufs;
 constexpr float kRescaleLog2 = 8.0f;
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -658,6 +664,13 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]), "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -682,19 +695,18 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescBase | (1u << 16) | ((128u >> 3) << 17);
 
-__global__ void __launch_bounds__(kTcThreads, 1)
-attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant__ CUtensorMap v_map, AttnArgs a) {
-    if ((int)blockIdx.x >= a.plan[0]) return;
-    const AttnItem item = a.items[blockIdx.x];
-    if (!item.pad[0]) return;                      // handled by the warp-level kernel
-    extern __shared__ unsigned char smem_raw[];
+__device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtensorMap& v_map, const AttnArgs& a,
+                                        const AttnItem& item, unsigned char* smem_raw) {
+    // runs inside a CTA of kThreads threads; only the first kTcThreads take part (CTA-wide syncs count them only)
+    if ((int)threadIdx.x >= kTcThreads) return;
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned char* ring = smem;
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(ring + kTcGroupStages * kTcGroupBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcGroupStages + 6);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcGroupStages + 3 * kTcSBufs);
     __shared__ int abort_s;
+    __shared__ float xch[2][2][128];   // [group parity][column half][row]: partial row maxima; [0][h][r] also the final sums
     const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kTcGroupStages);
-    const uint32_t s_full = smem_u32(bars + 2 * kTcGroupStages), p_full = s_full + 16, pv_done = s_full + 32;
+    const uint32_t s_full = smem_u32(bars + 2 * kTcGroupStages), p_full = s_full + 8 * kTcSBufs, pv_done = p_full + 8 * kTcSBufs;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int req = item.req, kvh = item.kv_head;
@@ -710,9 +722,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant
             mbar_init(full_bar + 8 * s, 4);          // one arrival per page slot of the group
             mbar_init(empty_bar + 8 * s, 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kTcSBufs; ++b) {
             mbar_init(s_full + 8 * b, 1);
-            mbar_init(p_full + 8 * b, 128);
+            mbar_init(p_full + 8 * b, kTcSoftmaxThreads);
             mbar_init(pv_done + 8 * b, 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -723,7 +735,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
-    __syncthreads();
+    asm volatile("bar.sync 0, %0;" ::"n"(kTcThreads) : "memory");
     tc_fence_after();
     const uint32_t tmem_o = *tmem_slot;
     bool failed = false;
@@ -735,15 +747,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant
         if (lane < 4) {
             const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
             int next = lane < n_pages ? bt[lane] : 0;
+            TCP(long long t_we = 0; long long t_all = clock64();)
             for (int g = 0; g < n_groups; ++g) {
                 const int p = 4 * g + lane;
                 int page_id = next;
                 if (p + 4 < n_pages) next = bt[p + 4];
                 const int gs = g % kTcGroupStages, use = g / kTcGroupStages;
+                TCP(long long c0 = clock64();)
                 if ((use > 0 && !mbar_wait(empty_bar + 8 * gs, (use - 1) & 1, &abort_s)) || *(volatile int*)&abort_s) {
                     failed = true;
                     break;
                 }
+                TCP(t_we += clock64() - c0;)
                 const uint32_t bar = full_bar + 8 * gs;
                 if (p >= n_pages) {
                     mbar_arrive(bar);
@@ -760,150 +775,192 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant
                 tma_load_2d(dst + 8192 + lane * 2048, &k2_map, 64, row, bar);    // K columns 64..127
                 tma_load_tile(dst + 4 * kTcPageBytes + lane * kTcPageBytes, &v_map, row, bar);
             }
+            TCP(if (blockIdx.x == 0 && lane == 0) printf("producer: groups %d total %lld wait_empty %lld\n", n_groups, clock64() - t_all, t_we);)
         }
     } else {
         const uint32_t tmem_q = tmem_o + kTcColQ;
+        const int quarter = warp & 3, half = (warp - 2) >> 2;     // softmax warps: lane quarter of tensor memory, column half
         if (warp >= 2) {
-            // the query tile goes to tensor memory: thread = row R = lane of tensor memory, 128 bf16 = 64 words
-            const int R = (warp & 3) * 32 + lane;
-            uint32_t qw[64];
+            // the query tile goes to tensor memory: row R = lane of tensor memory, 128 bf16 = 64 words, 32 per thread
+            const int R = quarter * 32 + lane;
+            uint32_t qw[32];
             if (R < M) {
                 const int t = R / group, hl = R - t * group;
-                const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128);
+                const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * half;
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
+                for (int c = 0; c < 8; ++c) {
                     const uint4 v = src[c];
                     qw[4 * c] = v.x; qw[4 * c + 1] = v.y; qw[4 * c + 2] = v.z; qw[4 * c + 3] = v.w;
                 }
             } else {
 #pragma unroll
-                for (int c = 0; c < 64; ++c) qw[c] = 0;
+                for (int c = 0; c < 32; ++c) qw[c] = 0;
             }
-            const uint32_t t_q = tmem_q + ((uint32_t)((warp & 3) * 32) << 16);
-            tc_st32(t_q, qw);
-            tc_st32(t_q + 32, qw + 32);
+            tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * half, qw);
             tc_wait_st();
             tc_fence_before();
         }
-        asm volatile("bar.sync 1, 160;" ::: "memory");                      // MMA warp + softmax warps
+        asm volatile("bar.sync 1, %0;" ::"n"(32 + kTcSoftmaxThreads) : "memory");   // MMA warp + softmax warps
         if (warp == 1) {
             if (lane == 0) {
                 // ------------------------------------------------------------ MMA issuer
                 tc_fence_after();
+                TCP(long long t_wf = 0, t_qk = 0, t_wpv = 0, t_wp = 0, t_pv = 0; long long t_all = clock64();)
                 auto issue_qk = [&](int g) -> bool {
-                    const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages;
+                    const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages, b = g % kTcSBufs;
+                    TCP(long long c0 = clock64();)
                     if (!mbar_wait(full_bar + 8 * gs, (g / kTcGroupStages) & 1, &abort_s)) return false;
                     tc_fence_after();
+                    TCP(long long c1 = clock64(); t_wf += c1 - c0;)
                     const uint32_t k_addr = smem_u32(ring + gs * kTcGroupBytes);
-                    const uint32_t d = tmem_o + kTcColS + 64 * (g & 1);
+                    const uint32_t d = tmem_o + kTcColS + 64 * b;
                     const uint32_t idesc = kIdescBase | ((uint32_t)(np * kPage >> 3) << 17);
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks)    // 16 head-dim elements = 8 words of Q, 32 bytes along a K row
                             tc_mma_ts(d, tmem_q + (h * 4 + ks) * 8, desc_kmajor(k_addr + h * 8192) + 2 * ks, idesc, (h | ks) ? 1u : 0u);
-                    tc_commit(s_full + 8 * (g & 1));
+                    tc_commit(s_full + 8 * b);
+                    TCP(t_qk += clock64() - c1;)
                     return true;
                 };
-                bool ok = issue_qk(0);
+                // QK^T runs kTcSBufs - 1 groups ahead of PV
+                bool ok = true;
+                for (int g = 0; ok && g < kTcSBufs - 1 && g < n_groups; ++g) ok = issue_qk(g);
                 for (int g = 0; ok && g < n_groups; ++g) {
-                    if (g + 1 < n_groups) {
-                        // the S/P buffer of group g+1 was last used by group g-1
-                        if (g >= 1 && !mbar_wait(pv_done + 8 * ((g + 1) & 1), ((g - 1) >> 1) & 1, &abort_s)) { ok = false; break; }
-                        if (!issue_qk(g + 1)) { ok = false; break; }
+                    const int ga = g + kTcSBufs - 1;
+                    if (ga < n_groups) {
+                        // its S/P buffer was last used by group g-1
+                        TCP(long long c0 = clock64();)
+                        if (g >= 1 && !mbar_wait(pv_done + 8 * (ga % kTcSBufs), ((g - 1) / kTcSBufs) & 1, &abort_s)) { ok = false; break; }
+                        TCP(t_wpv += clock64() - c0;)
+                        if (!issue_qk(ga)) { ok = false; break; }
                     }
-                    if (!mbar_wait(p_full + 8 * (g & 1), (g >> 1) & 1, &abort_s)) { ok = false; break; }
+                    const int b = g % kTcSBufs;
+                    TCP(long long c2 = clock64();)
+                    if (!mbar_wait(p_full + 8 * b, (g / kTcSBufs) & 1, &abort_s)) { ok = false; break; }
                     tc_fence_after();
+                    TCP(long long c3 = clock64(); t_wp += c3 - c2;)
                     const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages;
                     const uint32_t v_addr = smem_u32(ring + gs * kTcGroupBytes) + 4 * kTcPageBytes;
-                    const uint32_t tmem_p = tmem_o + kTcColS + 64 * (g & 1);
+                    const uint32_t tmem_p = tmem_o + kTcColS + 64 * b;
                     for (int j = 0; j < np; ++j)           // 16 keys = 8 words of P
                         tc_mma_ts(tmem_o, tmem_p + 8 * j, desc_mnmajor(v_addr + j * kTcPageBytes), kIdescPV, (g | j) ? 1u : 0u);
                     tc_commit(empty_bar + 8 * gs);         // the group's K and V tiles are free again
-                    tc_commit(pv_done + 8 * (g & 1));
+                    tc_commit(pv_done + 8 * b);
+                    TCP(t_pv += clock64() - c3;)
                 }
+                TCP(if (blockIdx.x == 0) printf("mma: groups %d total %lld | wait_full %lld qk_issue %lld wait_pvdone %lld wait_p %lld pv_issue %lld\n", n_groups, clock64() - t_all, t_wf, t_qk, t_wpv, t_wp, t_pv);)
                 if (!ok) failed = true;
             }
         } else {
-            // ---------------------------------------------------------------- softmax + epilogue, thread = row
-            const int R = (warp & 3) * 32 + lane;
-            const uint32_t t_lane = tmem_o + ((uint32_t)((warp & 3) * 32) << 16);
+            // ---------------------------------------------------------------- softmax + epilogue
+            // row R = tensor-memory lane; this thread owns columns [32 * half, 32 * half + 32) of every S tile
+            const int R = quarter * 32 + lane;
+            const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
             const int jmax = ctx_len + min(R, M - 1) / group;           // last visible cache position
             const float c = a.scale_log2;
             float m_run = -INFINITY, l_run = 0.0f;
+            // A failed wait never leaves the loop early: the two threads of a row meet at a named barrier every group,
+            // so a thread that has given up keeps walking (skipping the tensor-memory work) until the loop ends.
+            TCP(long long t_ws = 0, t_wk = 0, t_bar = 0;)
             for (int g = 0; g < n_groups; ++g) {
-                if (!mbar_wait(s_full + 8 * (g & 1), (g >> 1) & 1, &abort_s)) { failed = true; break; }
-                tc_fence_after();
-                const uint32_t t_s = t_lane + kTcColS + 64 * (g & 1);
-                uint32_t sr[64];
-                tc_ld32(t_s, sr);
-                tc_ld32(t_s + 32, sr + 32);
-                tc_wait_ld();
-                const int ncols = min(4, n_pages - 4 * g) * kPage;
-                const int j0 = (item.page_begin + 4 * g) * kPage;
-                float mx = -INFINITY;
-                if (ncols < 64 || j0 + 63 > ctx_len) {                  // a partial group or one that holds hidden keys
-                    const int lim = min(ncols - 1, jmax - j0);          // columns 0..lim are visible
+                const int b = g % kTcSBufs;
+                TCP(long long c0 = clock64();)
+                if (!failed && !mbar_wait(s_full + 8 * b, (g / kTcSBufs) & 1, &abort_s)) failed = true;
+                failed = __any_sync(0xffffffffu, failed);
+                TCP(long long c1 = clock64(); t_ws += c1 - c0;)
+                const uint32_t t_s = t_lane + kTcColS + 64 * b;
+                uint32_t sr[32];
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                if (!failed) {
+                    tc_fence_after();
+                    tc_ld32(t_s + 32 * half, sr);
+                    tc_wait_ld();
+                    const int ncols = min(4, n_pages - 4 * g) * kPage;
+                    const int j0 = (item.page_begin + 4 * g) * kPage + 32 * half;
+                    if (ncols < 64 || j0 + 31 > ctx_len) {                  // a partial group or one that holds hidden keys
+                        const int lim = min(ncols - 32 * half - 1, jmax - j0);   // own columns 0..lim are visible
 #pragma unroll
-                    for (int e = 0; e < 64; ++e) {
-                        const float v = e <= lim ? __uint_as_float(sr[e]) : -INFINITY;
-                        sr[e] = __float_as_uint(v);
-                        mx = fmaxf(mx, v);
+                        for (int e = 0; e < 32; ++e) {
+                            const float v = e <= lim ? __uint_as_float(sr[e]) : -INFINITY;
+                            sr[e] = __float_as_uint(v);
+                            mx4[e & 3] = fmaxf(mx4[e & 3], v);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sr[e]));
                     }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sr[e]));
                 }
+                // the two threads of a row exchange their partial maxima
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                xch[g & 1][half][R] = mx;
+                TCP(long long c4 = clock64();)
+                asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
+                TCP(t_bar += clock64() - c4;)
+                mx = fmaxf(mx, xch[g & 1][half ^ 1][R]);
                 // the running maximum only moves (and O is only rescaled) when it would grow by more than 2^8
                 float alpha = 1.0f;
                 bool moved = false;
-                if (mx > m_run && (m_run == -INFINITY || (mx - m_run) * c > kRescaleLog2)) {
+                if (!failed && mx > m_run && (m_run == -INFINITY || (mx - m_run) * c > kRescaleLog2)) {
                     alpha = fast_exp2((m_run - mx) * c);                  // 0 when nothing was visible before
                     m_run = mx;
                     l_run *= alpha;
                     moved = g > 0;
                 }
                 if (g > 0 && __any_sync(0xffffffffu, moved)) {
-                    // O is being updated by the previous group's MMAs: wait for them, then scale this warp's rows
-                    if (!mbar_wait(pv_done + 8 * ((g - 1) & 1), ((g - 1) >> 1) & 1, &abort_s)) { failed = true; break; }
-                    tc_fence_after();
+                    // O is being updated by the previous group's MMAs: wait for them, then scale this thread's half row
+                    if (!mbar_wait(pv_done + 8 * ((g - 1) % kTcSBufs), ((g - 1) / kTcSBufs) & 1, &abort_s)) failed = true;
+                    failed = __any_sync(0xffffffffu, failed);
+                    if (!failed) {
+                        tc_fence_after();
 #pragma unroll 1
-                    for (int cc = 0; cc < 128; cc += 32) {
-                        uint32_t o[32];
-                        tc_ld32(t_lane + cc, o);
-                        tc_wait_ld();
+                        for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
+                            uint32_t o[32];
+                            tc_ld32(t_lane + cc, o);
+                            tc_wait_ld();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tc_st32(t_lane + cc, o);
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tc_st32(t_lane + cc, o);
+                        }
+                        tc_wait_st();
                     }
-                    tc_wait_st();
                 }
-                const float mc = (m_run == -INFINITY ? 0.0f : m_run) * c;
-                float sum = 0.0f;
-                uint32_t pw[32];
+                if (!failed) {
+                    const float mc = (m_run == -INFINITY ? 0.0f : m_run) * c;
+                    float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                    uint32_t pw[16];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), c, -mc));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), c, -mc));
-                    sum += p0 + p1;
-                    pw[e] = pack_bf16(p0, p1);
+                    for (int e = 0; e < 16; ++e) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), c, -mc));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), c, -mc));
+                        sum4[e & 3] += p0 + p1;
+                        pw[e] = pack_bf16(p0, p1);
+                    }
+                    l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    tc_st16(t_s + 16 * half, pw);                           // P over the columns S occupied
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(p_full + 8 * b);
                 }
-                l_run += sum;
-                tc_st32(t_s, pw);                                       // P over the columns S occupied
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(p_full + 8 * (g & 1));
+                TCP(t_wk += clock64() - c1;)
             }
-            // epilogue: the item's O row, normalised
-            if (!failed && !mbar_wait(pv_done + 8 * ((n_groups - 1) & 1), ((n_groups - 1) >> 1) & 1, &abort_s)) failed = true;
+            TCP(if (blockIdx.x == 0 && R == 0) printf("softmax half %d: wait_s %lld work %lld (pair barrier %lld)\n", half, t_ws, t_wk, t_bar);)
+            // epilogue: the item's O row, normalised; this thread writes columns [64 * half, 64 * half + 64)
+            if (!failed && !mbar_wait(pv_done + 8 * ((n_groups - 1) % kTcSBufs), ((n_groups - 1) / kTcSBufs) & 1, &abort_s)) failed = true;
+            failed = __any_sync(0xffffffffu, failed);
             tc_fence_after();
+            asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");   // every exchange read of the last group is done
+            xch[0][half][R] = l_run;
+            asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
+            l_run += xch[0][half ^ 1][R];
             if (!failed) {
                 const float inv = l_run > 0.0f ? 1.0f / l_run : 0.0f;
                 const float lse_nat = l_run > 0.0f ? (m_run * c + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
                 const int t = R / group, hl = R - t * group;
                 const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
 #pragma unroll 1
-                for (int cc = 0; cc < 128; cc += 32) {
+                for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
                     uint32_t o[32];
                     tc_ld32(t_lane + cc, o);
                     tc_wait_ld();
@@ -927,7 +984,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant
                         }
                     }
                 }
-                if (R < M) {
+                if (R < M && half == 0) {
                     if (item.n_chunks == 1) {
                         if (a.lse) a.lse[orow] = lse_nat;
                     } else {
@@ -942,11 +999,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap k2_map, const __grid_constant
         *(volatile int*)&abort_s = 1;
     }
     tc_fence_before();
-    __syncthreads();
+    asm volatile("bar.sync 0, %0;" ::"n"(kTcThreads) : "memory");
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_o), "n"(kTcCols) : "memory");
     }
+}
+
+// One CTA per work item; the item says which of the two paths takes it.
+template <int DH>
+__global__ void __launch_bounds__(kThreads, 1)
+attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
+                 const __grid_constant__ CUtensorMap k2_map, AttnArgs a) {
+    if ((int)blockIdx.x >= a.plan[0]) return;
+    extern __shared__ unsigned char smem_raw[];
+    const AttnItem item = a.items[blockIdx.x];
+    if (DH == 128 && item.pad[0])
+        tc_item(k2_map, v_map, a, item, smem_raw);
+    else
+        split_item<DH>(k_map, v_map, a, item, smem_raw);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1030,13 +1101,10 @@ dcut_status make_cache_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, lo
 template <int DH>
 dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& k2m, const AttnArgs& aa,
                      const CombineArgs& ca, int T_cap, cudaStream_t stream) {
-    dcut_status st;
-    if (DH == 128 && ctx->attn_tc_min_rows <= 128) {
-        attn_tc_kernel<<<ctx->max_items, kTcThreads, kTcSmem, stream>>>(k2m, vm, aa);
-        if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_tc_kernel")) != DCUT_OK) return st;
-    }
-    attn_split_kernel<DH><<<ctx->max_items, kThreads, SmemLayout<DH>::kTotal, stream>>>(km, vm, aa);
-    if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_split_kernel")) != DCUT_OK) return st;
+    constexpr int kSmem = (DH == 128 && kTcSmem > SmemLayout<DH>::kTotal) ? kTcSmem : SmemLayout<DH>::kTotal;
+    attn_item_kernel<DH><<<ctx->max_items, kThreads, kSmem, stream>>>(km, vm, k2m, aa);
+    dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_item_kernel");
+    if (st != DCUT_OK) return st;
     (void)T_cap;
     dim3 cgrid(ca.B * ca.tokens_per_req, (ctx->lim.n_q_heads + 7) / 8);
     attn_combine_kernel<DH><<<cgrid, 256, 0, stream>>>(ca);
@@ -1046,14 +1114,11 @@ dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm
 }  // namespace
 
 dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
-    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         SmemLayout<128>::kTotal);
+    constexpr int kSmem128 = kTcSmem > SmemLayout<128>::kTotal ? kTcSmem : SmemLayout<128>::kTotal;
+    cudaError_t e = cudaFuncSetAttribute(attn_item_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem128);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 128)");
-    e = cudaFuncSetAttribute(attn_split_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             SmemLayout<64>::kTotal);
+    e = cudaFuncSetAttribute(attn_item_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout<64>::kTotal);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 64)");
-    e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
-    if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn tc)");
     {
         const char* env = getenv("DCUT_ATTN_TC_MIN_ROWS");   // query rows from which an item goes to the tcgen05 kernel
         ctx->attn_tc_min_rows = env ? atoi(env) : 33;
