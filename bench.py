@@ -50,6 +50,7 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch the step's kernels one by one instead of replaying a CUDA graph")
     return ap.parse_args()
 
 
@@ -331,6 +332,7 @@ def run_dcut(args):
         bufs = make_bufs(T)
         for _ in range(max(3, args.warmup)):
             step(qp, lp, bufs)
+        # (a) kernel-by-kernel launches, with events around the verification forward (attention roofline)
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
         barrier(world)
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -344,11 +346,29 @@ def run_dcut(args):
                             bufs["out_tokens"], bufs["total"])
         end.record()
         barrier(world)
-        total_ms = max_over_ranks(start.elapsed_time(end), world)
+        eager_ms = max_over_ranks(start.elapsed_time(end), world)
         attn_ms = statistics.mean(a.elapsed_time(b) for a, b in ev)
+        total_ms = eager_ms
+        # (b) the same step captured once in a CUDA graph and replayed: the packed length is read on the device,
+        # so one graph serves whatever depth vector the selector produces
+        if not args.no_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step(qp, lp, bufs)
+            for _ in range(3):
+                graph.replay()
+            barrier(world)
+            start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            start.record()
+            for k in range(args.steps):
+                graph.replay()
+            end.record()
+            barrier(world)
+            total_ms = max_over_ranks(start.elapsed_time(end), world)
+            del graph
         accepted = int(bufs["total"].item())
         assert ctx.poll_device_status() == 0
-        res[name] = dict(T=T, accepted=accepted, ms_per_step=total_ms / args.steps, attn_ms=attn_ms,
+        res[name] = dict(T=T, accepted=accepted, ms_per_step=total_ms / args.steps, eager_ms=eager_ms / args.steps, attn_ms=attn_ms,
                          tokens_per_s=world * accepted / (total_ms / args.steps * 1e-3),
                          attn_bytes=attn_algorithmic_bytes(cfg, sel.ctx_lens, d), depths=d)
         del qp, lp, bufs
@@ -423,10 +443,12 @@ def run_dcut(args):
                                f"{cfg.n_kv_heads}kv Dh={cfg.head_dim} page={cfg.page_size} V={cfg.vocab} "
                                f"ctx {cfg.ctx_lo}-{cfg.ctx_hi}",
                    "arm": "D-cut pruned (dense cost table profiled on this GPU)",
+                   "launch": "kernel by kernel" if args.no_graph else "one CUDA graph of the step, replayed each step",
                    "l2": f"inputs exceed L2: each step streams {p['attn_bytes'] / 1e6:.0f} MB of KV and "
                          f"{p['T'] * cfg.vocab * 2 / 1e6:.0f} MB of logits once (L2 is 126 MB)",
                    "parallelism": "replicas only" if world > 1 else "1 GPU"},
         "arms": {k: {"T": v["T"], "accepted_tokens": v["accepted"], "ms_per_step": round(v["ms_per_step"], 4),
+                     "ms_per_step_kernel_by_kernel": round(v["eager_ms"], 4),
                      "attn_ms": round(v["attn_ms"], 4), "tokens_per_s": round(v["tokens_per_s"], 1),
                      "attn_gbs": round(v["attn_bytes"] / (v["attn_ms"] * 1e-3) / 1e9, 1)} for k, v in res.items()},
         "roofline": {"kernel": "dcut_verify_attn (plan + split + combine launches)", "bound": "hbm",

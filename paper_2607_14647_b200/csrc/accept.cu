@@ -7,7 +7,7 @@
 //       index); the CTA result is merged into one 64-bit word per row with atomicMax on
 //       (ordered value << 32 | ~index): the largest value wins and, among equals, the lowest
 //       index, whatever order the CTAs finish in.
-//   accept_match_kernel   one thread per request: longest matching prefix, bonus token, emitted
+//   accept_match_kernel   one warp per request: longest matching prefix, bonus token, emitted
 //       tokens, total; clears the per-row words for the next call.
 #include "dcut_internal.h"
 
@@ -108,6 +108,8 @@ __device__ int slow_first_valid(const unsigned short* rp, int V) {
     return 0;
 }
 
+// One warp per request: the lanes fetch the row results of t = lane, lane + 32, ... together, a ballot finds the
+// first row whose argmax differs from the draft (or the last row), and the per-row words are cleared on the way.
 __global__ void __launch_bounds__(1024) accept_match_kernel(
     const unsigned short* __restrict__ logits, int V, const int* __restrict__ draft_ids,
     const int* __restrict__ cu_q, int B, int gamma, unsigned long long* __restrict__ row_key,
@@ -116,27 +118,37 @@ __global__ void __launch_bounds__(1024) accept_match_kernel(
     __shared__ int total_s;
     if (threadIdx.x == 0) total_s = 0;
     __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     int local = 0;
-    for (int i = threadIdx.x; i < B; i += blockDim.x) {
+    for (int i = warp; i < B; i += n_warps) {
         const int a = cu_q[i], d = cu_q[i + 1] - a - 1;
         int m = -1, bon = 0;
-        for (int t = 0; t <= d; ++t) {
-            const unsigned long long key = row_key[a + t];
-            row_key[a + t] = 0;
-            if (m >= 0) continue;   // already stopped: only clearing
-            const int am = key ? (int)(0xffffffffu - (unsigned int)key) : slow_first_valid(logits + (size_t)(a + t) * V, V);
-            if (t == d || am != draft_ids[(size_t)i * gamma + t]) {
-                m = t;
-                bon = am;
+        for (int t0 = 0; t0 <= d; t0 += 32) {
+            const int t = t0 + lane;
+            int am = 0;
+            bool stop = false;
+            if (t <= d) {
+                const unsigned long long key = row_key[a + t];
+                row_key[a + t] = 0;
+                am = key ? (int)(0xffffffffu - (unsigned int)key) : slow_first_valid(logits + (size_t)(a + t) * V, V);
+                stop = (t == d) || am != draft_ids[(size_t)i * gamma + t];
+            }
+            const unsigned int mask = __ballot_sync(0xffffffffu, stop);
+            if (m < 0 && mask) {
+                const int first = __ffs(mask) - 1;
+                m = t0 + first;
+                bon = __shfl_sync(0xffffffffu, am, first);
             }
         }
-        accept_len[i] = m;
-        bonus[i] = bon;
+        if (lane == 0) {
+            accept_len[i] = m;
+            bonus[i] = bon;
+            local += m + 1;
+        }
         if (out_tokens) {
             int* o = out_tokens + (size_t)i * (gamma + 1);
-            for (int t = 0; t <= gamma; ++t) o[t] = t < m ? draft_ids[(size_t)i * gamma + t] : (t == m ? bon : -1);
+            for (int t = lane; t <= gamma; t += 32) o[t] = t < m ? draft_ids[(size_t)i * gamma + t] : (t == m ? bon : -1);
         }
-        local += m + 1;
     }
     if (local) atomicAdd(&total_s, local);
     __syncthreads();

@@ -99,11 +99,15 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     __shared__ Best best_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    // 1. prefix scores and sort keys
+    // 1. prefix scores and sort keys.  The confidences come in through shared memory with coalesced loads
+    // (the later prefix-sum array is free at this point), so the per-request product chain reads no global memory.
+    float* conf_s = reinterpret_cast<float*>(qs);
+    for (int e = tid; e < n; e += kThreads) conf_s[e] = a.conf[e];
+    __syncthreads();
     for (int i = tid; i < B; i += kThreads) {
         float p = 1.0f;
         for (int k = 0; k < gamma; ++k) {
-            p = __fmul_rn(p, clamp_conf(a.conf[(size_t)i * gamma + k]));
+            p = __fmul_rn(p, clamp_conf(conf_s[i * gamma + k]));
             if (p == 0.0f) p = 0.0f;   // -0 -> +0
             if (a.scores_out) a.scores_out[(size_t)i * gamma + k] = p;
             const unsigned int bits = __float_as_uint(p);
