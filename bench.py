@@ -451,7 +451,7 @@ def run_dcut(args):
                      "ms_per_step_kernel_by_kernel": round(v["eager_ms"], 4),
                      "attn_ms": round(v["attn_ms"], 4), "tokens_per_s": round(v["tokens_per_s"], 1),
                      "attn_gbs": round(v["attn_bytes"] / (v["attn_ms"] * 1e-3) / 1e9, 1)} for k, v in res.items()},
-        "roofline": {"kernel": "dcut_verify_attn (plan + split + combine launches)", "bound": "hbm",
+        "roofline": {"kernel": "dcut_verify_attn (attn_plan_kernel + attn_item_kernel + attn_combine_kernel)", "bound": "hbm",
                      "achieved": round(achieved, 1), "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": round(achieved / pk["hbm_gbs"], 4), "peak_source": f"of {pk['source']}",
                      "frac_of_8000_nominal": round(achieved / 8000.0, 4),
