@@ -8,7 +8,7 @@
 //                         position L_i + t, q written as the attention kernel's [T, Hq, Dh] input
 //   gemm_tcgen05_kernel   C[M, N] = A[M, K] . B[N, K]^T on the 5th-generation tensor cores: 128 x 256 output tile
 //                         per CTA, accumulator in tensor memory (256 fp32 columns), operands staged by TMA into a
-//                         4-stage ring of 128-byte-swizzled K-major tiles (BK = 64), one thread issuing
+//                         4-stage ring of 128-byte-swizzled K-major tiles (BK = 64), one elected lane issuing
 //                         tcgen05.mma (M128 N256 K16) and releasing stages with tcgen05.commit, four epilogue warps
 //                         reading the accumulator with tcgen05.ld.  Epilogues: plain bf16, + residual, or SwiGLU
 //                         (the B tile is 128 gate rows followed by the 128 matching up rows, so silu(g) * u is
@@ -61,6 +61,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+// One lane of a converged warp.  Issuing tcgen05 / TMA instructions under this predicate (rather than under
+// `lane == 0`) lets the compiler keep their operands in uniform registers; measured on B200 this halves the
+// cycles per tcgen05.mma of the issuing thread.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -156,14 +164,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     bool failed = false;
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ TMA producer
-            for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % kGemmStages;
-                if (kb >= kGemmStages && !mbar_wait(empty_bar + 8 * s, ((kb / kGemmStages) - 1) & 1)) {
-                    failed = true;
-                    break;
-                }
+        // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
+        for (int kb = 0; kb < n_kb; ++kb) {
+            const int s = kb % kGemmStages;
+            if (kb >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kb / kGemmStages) - 1) & 1))) {
+                failed = true;
+                break;
+            }
+            if (elect_one()) {
                 const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
                 const uint32_t bar = full_bar + 8 * s;
                 mbar_arrive_expect_tx(bar, kGemmStageBytes);
@@ -176,17 +184,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                     tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
                 }
             }
+            __syncwarp();
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ------------------------------------------------------------ MMA issuer
-            for (int kb = 0; kb < n_kb; ++kb) {
-                const int s = kb % kGemmStages;
-                if (!mbar_wait(full_bar + 8 * s, (kb / kGemmStages) & 1)) {
-                    failed = true;
-                    break;
-                }
-                tc_fence_after();
+        // ---------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
+        for (int kb = 0; kb < n_kb; ++kb) {
+            const int s = kb % kGemmStages;
+            if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kb / kGemmStages) & 1))) {
+                failed = true;
+                break;
+            }
+            tc_fence_after();
+            if (elect_one()) {
                 const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
                 const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
 #pragma unroll
@@ -194,8 +203,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                     tc_mma(tmem_base, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
                 tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
             }
-            tc_commit(accum_bar);                   // accumulator complete
+            __syncwarp();
         }
+        if (elect_one()) tc_commit(accum_bar);      // accumulator complete
+        __syncwarp();
     } else {
         // ---------------------------------------------------------------- epilogue warps
         const int quarter = warp & 3;               // tensor-memory lanes 32 * quarter .. + 31

@@ -632,6 +632,14 @@ constexpr int kTcCols = 512;                       // O: 0..127, S/P buffers: 12
 constexpr int kTcColS = 128, kTcColQ = kTcColS + 64 * kTcSBufs;
 constexpr float kRescaleLog2 = 8.0f;
 
+// One lane of a converged warp.  Issuing tcgen05.mma / tcgen05.commit under this predicate (not under `lane == 0`)
+// lets the compiler keep the operands in uniform registers: on B200 the issuing thread then needs ~47 cycles for
+// an M128 N64 K16 MMA with A in tensor memory and ~73 for N128, against 96+ from a lane-0-only branch.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -802,57 +810,60 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
         }
         asm volatile("bar.sync 1, %0;" ::"n"(32 + kTcSoftmaxThreads) : "memory");   // MMA warp + softmax warps
         if (warp == 1) {
-            if (lane == 0) {
-                // ------------------------------------------------------------ MMA issuer
+            // ---------------------------------------------------------------- MMA issuer
+            // The whole warp walks the schedule and waits on the barriers; one elected lane issues.
+            tc_fence_after();
+            auto issue_qk = [&](int g) -> bool {
+                const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages, b = g % kTcSBufs;
+                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * gs, (g / kTcGroupStages) & 1, &abort_s))) return false;
                 tc_fence_after();
-                TCP(long long t_wf = 0, t_qk = 0, t_wpv = 0, t_wp = 0, t_pv = 0; long long t_all = clock64();)
-                auto issue_qk = [&](int g) -> bool {
-                    const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages, b = g % kTcSBufs;
-                    TCP(long long c0 = clock64();)
-                    if (!mbar_wait(full_bar + 8 * gs, (g / kTcGroupStages) & 1, &abort_s)) return false;
-                    tc_fence_after();
-                    TCP(long long c1 = clock64(); t_wf += c1 - c0;)
+                if (elect_one()) {
                     const uint32_t k_addr = smem_u32(ring + gs * kTcGroupBytes);
                     const uint32_t d = tmem_o + kTcColS + 64 * b;
                     const uint32_t idesc = kIdescBase | ((uint32_t)(np * kPage >> 3) << 17);
+                    const uint64_t dk0 = desc_kmajor(k_addr), dk1 = desc_kmajor(k_addr + 8192);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int ks = 0; ks < 4; ++ks)    // 16 head-dim elements = 8 words of Q, 32 bytes along a K row
+                        tc_mma_ts(d, tmem_q + ks * 8, dk0 + 2 * ks, idesc, ks ? 1u : 0u);
 #pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)    // 16 head-dim elements = 8 words of Q, 32 bytes along a K row
-                            tc_mma_ts(d, tmem_q + (h * 4 + ks) * 8, desc_kmajor(k_addr + h * 8192) + 2 * ks, idesc, (h | ks) ? 1u : 0u);
+                    for (int ks = 0; ks < 4; ++ks)
+                        tc_mma_ts(d, tmem_q + (4 + ks) * 8, dk1 + 2 * ks, idesc, 1u);
                     tc_commit(s_full + 8 * b);
-                    TCP(t_qk += clock64() - c1;)
-                    return true;
-                };
-                // QK^T runs kTcSBufs - 1 groups ahead of PV
-                bool ok = true;
-                for (int g = 0; ok && g < kTcSBufs - 1 && g < n_groups; ++g) ok = issue_qk(g);
-                for (int g = 0; ok && g < n_groups; ++g) {
-                    const int ga = g + kTcSBufs - 1;
-                    if (ga < n_groups) {
-                        // its S/P buffer was last used by group g-1
-                        TCP(long long c0 = clock64();)
-                        if (g >= 1 && !mbar_wait(pv_done + 8 * (ga % kTcSBufs), ((g - 1) / kTcSBufs) & 1, &abort_s)) { ok = false; break; }
-                        TCP(t_wpv += clock64() - c0;)
-                        if (!issue_qk(ga)) { ok = false; break; }
-                    }
-                    const int b = g % kTcSBufs;
-                    TCP(long long c2 = clock64();)
-                    if (!mbar_wait(p_full + 8 * b, (g / kTcSBufs) & 1, &abort_s)) { ok = false; break; }
-                    tc_fence_after();
-                    TCP(long long c3 = clock64(); t_wp += c3 - c2;)
+                }
+                __syncwarp();
+                return true;
+            };
+            // QK^T runs kTcSBufs - 1 groups ahead of PV
+            bool ok = true;
+            for (int g = 0; ok && g < kTcSBufs - 1 && g < n_groups; ++g) ok = issue_qk(g);
+            for (int g = 0; ok && g < n_groups; ++g) {
+                const int ga = g + kTcSBufs - 1;
+                if (ga < n_groups) {
+                    // its S/P buffer was last used by group g-1
+                    if (g >= 1 && !__all_sync(0xffffffffu, mbar_wait(pv_done + 8 * (ga % kTcSBufs), ((g - 1) / kTcSBufs) & 1, &abort_s))) { ok = false; break; }
+                    if (!issue_qk(ga)) { ok = false; break; }
+                }
+                const int b = g % kTcSBufs;
+                if (!__all_sync(0xffffffffu, mbar_wait(p_full + 8 * b, (g / kTcSBufs) & 1, &abort_s))) { ok = false; break; }
+                tc_fence_after();
+                if (elect_one()) {
                     const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages;
-                    const uint32_t v_addr = smem_u32(ring + gs * kTcGroupBytes) + 4 * kTcPageBytes;
                     const uint32_t tmem_p = tmem_o + kTcColS + 64 * b;
-                    for (int j = 0; j < np; ++j)           // 16 keys = 8 words of P
-                        tc_mma_ts(tmem_o, tmem_p + 8 * j, desc_mnmajor(v_addr + j * kTcPageBytes), kIdescPV, (g | j) ? 1u : 0u);
+                    const uint64_t dv = desc_mnmajor(smem_u32(ring + gs * kTcGroupBytes) + 4 * kTcPageBytes);
+                    if (np == 4) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)        // 16 keys = 8 words of P; the next V tile is 4 KB = 256 units on
+                            tc_mma_ts(tmem_o, tmem_p + 8 * j, dv + 256 * j, kIdescPV, (g | j) ? 1u : 0u);
+                    } else {
+                        for (int j = 0; j < np; ++j)
+                            tc_mma_ts(tmem_o, tmem_p + 8 * j, dv + 256 * j, kIdescPV, (g | j) ? 1u : 0u);
+                    }
                     tc_commit(empty_bar + 8 * gs);         // the group's K and V tiles are free again
                     tc_commit(pv_done + 8 * b);
-                    TCP(t_pv += clock64() - c3;)
                 }
-                TCP(if (blockIdx.x == 0) printf("mma: groups %d total %lld | wait_full %lld qk_issue %lld wait_pvdone %lld wait_p %lld pv_issue %lld\n", n_groups, clock64() - t_all, t_wf, t_qk, t_wpv, t_wp, t_pv);)
-                if (!ok) failed = true;
+                __syncwarp();
             }
+            if (!ok) failed = true;
         } else {
             // ---------------------------------------------------------------- softmax + epilogue
             // row R = tensor-memory lane; this thread owns columns [32 * half, 32 * half + 32) of every S tile
