@@ -122,7 +122,7 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
     if ((st = dcut_init_accept(c)) != DCUT_OK) return st;
     if (has_attn) {
         const char* env = getenv("DCUT_ATTN_TARGET_ITEMS");
-        c->target_items = env ? atoi(env) : c->sm_count * 4;
+        c->target_items = env ? atoi(env) : c->sm_count * 2;   // requests are only cut when the batch has fewer (request, head) pairs than that
         if (c->target_items < 1) c->target_items = 1;
         c->max_items = lim->max_B * lim->n_kv_heads + c->target_items;
         const int group = lim->n_q_heads / lim->n_kv_heads;

@@ -162,7 +162,7 @@ __device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* to
     if (lane == 31) ws[warp] = inc;
     __syncthreads();
     if (warp == 0) {
-        int w = ws[lane];
+        int w = lane < (int)(blockDim.x >> 5) ? ws[lane] : 0;
         int winc = plan_warp_scan(w, lane);
         ws[lane] = winc - w;
         if (lane == 31) ws[32] = winc;
@@ -180,12 +180,12 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     extern __shared__ unsigned long long order[];   // [npad] (inverted cost << 32 | request), sorted ascending
     __shared__ int ws[33];
     __shared__ int total_s;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, nthr = blockDim.x;   // 256 threads for small batches: cheaper barriers
     const int group = a.n_q_heads / a.n_kv_heads;
     if (tid == 0) total_s = 0;
     __syncthreads();
     int local = 0;
-    for (int i = tid; i < a.B; i += kPlanThreads) {
+    for (int i = tid; i < a.B; i += nthr) {
         const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
         local += (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
     }
@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     int chunk_pages = (int)((units + a.target_items - 1) / a.target_items);
     if (chunk_pages < a.min_chunk_pages) chunk_pages = a.min_chunk_pages;
 
-    for (int i = tid; i < a.npad; i += kPlanThreads) {
+    for (int i = tid; i < a.npad; i += nthr) {
         unsigned long long key = ~0ull;
         if (i < a.B) {
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     __syncthreads();
     for (int k = 2; k <= a.npad; k <<= 1)
         for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < (a.npad >> 1); t += kPlanThreads) {
+            for (int t = tid; t < (a.npad >> 1); t += nthr) {
                 const int i = 2 * t - (t & (j - 1)), l = i + j;
                 const bool up = (i & k) == 0;
                 const unsigned long long x = order[i], y = order[l];
@@ -225,7 +225,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             __syncthreads();
         }
 
-    const int per = (a.B + kPlanThreads - 1) / kPlanThreads;
+    const int per = (a.B + nthr - 1) / nthr;
     const int j0 = tid * per;
     int my_items = 0, my_rows = 0;
     for (int e = 0; e < per; ++e) {
@@ -1132,7 +1132,7 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 64)");
     {
         const char* env = getenv("DCUT_ATTN_TC_MIN_ROWS");   // query rows from which an item goes to the tcgen05 kernel
-        ctx->attn_tc_min_rows = env ? atoi(env) : 33;
+        ctx->attn_tc_min_rows = env ? atoi(env) : 17;
     }
     e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn plan)");
@@ -1183,7 +1183,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.items = ctx->d_items;
     pa.plan = ctx->d_plan;
     pa.req_part = ctx->d_req_part;
-    attn_plan_kernel<<<1, kPlanThreads, sizeof(unsigned long long) * pa.npad, stream>>>(pa);
+    attn_plan_kernel<<<1, B <= 256 ? 256 : kPlanThreads, sizeof(unsigned long long) * pa.npad, stream>>>(pa);
     st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_plan_kernel");
     if (st != DCUT_OK) return st;
 
