@@ -138,7 +138,7 @@ struct PlanArgs {
     const int* ctx_lens;
     const int* cu_q;
     int B, n_q_heads, n_kv_heads;
-    int target_items, min_chunk_pages, max_items, npad, tc_min_rows;
+    int target_items, min_chunk_pages, max_items, npad, tc_min_rows, max_item_rows;
     long long part_rows_cap;
     int* status;
     AttnItem* items;
@@ -235,7 +235,8 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
             const int nc = (pages + chunk_pages - 1) / chunk_pages;
-            my_items += nc * a.n_kv_heads;
+            const int n_rb = ((d + 1) * group + a.max_item_rows - 1) / a.max_item_rows;
+            my_items += nc * a.n_kv_heads * n_rb;
             if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
         }
     }
@@ -265,23 +266,29 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             const int M = (d + 1) * group;
             a.req_part[2 * i] = row_off;
             a.req_part[2 * i + 1] = nc;
+            // a query tile above max_item_rows rows (head_dim 128: the 128 lanes of tensor memory) is cut into row
+            // blocks, each its own item over the same pages
+            const int n_rb = (M + a.max_item_rows - 1) / a.max_item_rows;
             for (int c = 0; c < nc; ++c)
-                for (int h = 0; h < a.n_kv_heads; ++h) {
-                    AttnItem it;
-                    it.req = i;
-                    it.kv_head = h;
-                    it.page_begin = c * cp;
-                    it.page_end = min(pages, (c + 1) * cp);
-                    it.n_chunks = nc;
-                    it.part_row = nc > 1 ? row_off + (c * a.n_kv_heads + h) * M : -1;
-                    it.q0 = q0;
-                    it.depth = d;
-                    it.ctx_len = ctx_len;
-                    it.pad[0] = (M >= a.tc_min_rows && M <= 128) ? 1 : 0;   // which kernel takes the item
-                    it.pad[1] = it.pad[2] = 0;
-                    a.items[item_off + c * a.n_kv_heads + h] = it;
-                }
-            item_off += nc * a.n_kv_heads;
+                for (int h = 0; h < a.n_kv_heads; ++h)
+                    for (int rb = 0; rb < n_rb; ++rb) {
+                        const int row0 = rb * a.max_item_rows, rows = min(a.max_item_rows, M - row0);
+                        AttnItem it;
+                        it.req = i;
+                        it.kv_head = h;
+                        it.page_begin = c * cp;
+                        it.page_end = min(pages, (c + 1) * cp);
+                        it.n_chunks = nc;
+                        it.part_row = nc > 1 ? row_off + (c * a.n_kv_heads + h) * M + row0 : -1;
+                        it.q0 = q0;
+                        it.depth = d;
+                        it.ctx_len = ctx_len;
+                        it.pad[0] = (rows >= a.tc_min_rows && rows <= 128) ? 1 : 0;   // which path takes the item
+                        it.pad[1] = row0;    // first query row of the item within the request's tile
+                        it.pad[2] = rows;    // query rows of the item
+                        a.items[item_off + (c * a.n_kv_heads + h) * n_rb + rb] = it;
+                    }
+            item_off += nc * a.n_kv_heads * n_rb;
             if (nc > 1) row_off += nc * (d + 1) * a.n_q_heads;
         }
     }
@@ -336,8 +343,8 @@ __device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUten
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int req = item.req, kvh = item.kv_head;
     const int group = a.n_q_heads / a.n_kv_heads;
-    const int q0 = item.q0, depth = item.depth, ctx_len = item.ctx_len;
-    const int M = (depth + 1) * group;
+    const int q0 = item.q0, ctx_len = item.ctx_len;
+    const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile: row0 .. row0 + M - 1
     const int MT = (M + 15) >> 4;
     const int nslots = kConsumerWarps / MT;
     const int n_pages = item.page_end - item.page_begin;
@@ -408,7 +415,7 @@ __device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUten
             const int R = idx / kChunks, c16 = idx - R * kChunks;
             uint4 v = make_uint4(0, 0, 0, 0);
             if (R < M) {
-                const int t = R / group, hl = R - t * group;
+                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
                 v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * DH + c16 * 8);
             }
             *reinterpret_cast<uint4*>(q_s + (R >> 4) * (16 * DH * 2) + tile_off(R & 15, c16)) = v;
@@ -436,8 +443,8 @@ __device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUten
         }
         // causal limit per row: query token t sees cache positions j <= ctx_len + t
         const int R_lo = mt * 16 + (lane >> 2), R_hi = R_lo + 8;
-        const int jmax_lo = ctx_len + min(R_lo, M - 1) / group;
-        const int jmax_hi = ctx_len + min(R_hi, M - 1) / group;
+        const int jmax_lo = ctx_len + (row0 + min(R_lo, M - 1)) / group;
+        const int jmax_hi = ctx_len + (row0 + min(R_hi, M - 1)) / group;
         // per-lane ldmatrix row/chunk selectors
         const int kmat = lane >> 3;
         const int k_tok = ((kmat >> 1) << 3) + (lane & 7);
@@ -587,7 +594,7 @@ __device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUten
             acc.z *= inv;
             acc.w *= inv;
             const float lse_nat = l_all > 0.0f ? (m_all * a.scale_log2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
-            const int t = R / group, hl = R - t * group;
+            const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
             const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
             if (item.n_chunks == 1) {
                 uint2 pk;
@@ -720,7 +727,7 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
     const int req = item.req, kvh = item.kv_head;
     const int group = a.n_q_heads / a.n_kv_heads;
     const int q0 = item.q0, ctx_len = item.ctx_len;
-    const int M = (item.depth + 1) * group;
+    const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile
     const int n_pages = item.page_end - item.page_begin;
     const int n_groups = (n_pages + 3) >> 2;
 
@@ -793,7 +800,7 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
             const int R = quarter * 32 + lane;
             uint32_t qw[32];
             if (R < M) {
-                const int t = R / group, hl = R - t * group;
+                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
                 const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * half;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
@@ -869,7 +876,7 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
             // row R = tensor-memory lane; this thread owns columns [32 * half, 32 * half + 32) of every S tile
             const int R = quarter * 32 + lane;
             const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
-            const int jmax = ctx_len + min(R, M - 1) / group;           // last visible cache position
+            const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
             const float c = a.scale_log2;
             float m_run = -INFINITY, l_run = 0.0f;
             // A failed wait never leaves the loop early: the two threads of a row meet at a named barrier every group,
@@ -968,7 +975,7 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
             if (!failed) {
                 const float inv = l_run > 0.0f ? 1.0f / l_run : 0.0f;
                 const float lse_nat = l_run > 0.0f ? (m_run * c + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-                const int t = R / group, hl = R - t * group;
+                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
                 const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
 #pragma unroll 1
                 for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
@@ -1178,6 +1185,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     while (pa.npad < B) pa.npad <<= 1;
     pa.status = ctx->d_status;
     pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
+    pa.max_item_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? 128 : 144;
     pa.max_items = ctx->max_items;
     pa.part_rows_cap = ctx->part_rows_cap;
     pa.items = ctx->d_items;
