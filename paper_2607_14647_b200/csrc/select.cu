@@ -4,7 +4,8 @@
 // memory, and every step depends on the one before, so the kernel is latency-bound: one CTA of
 // 1024 threads, no global round trips between the steps.
 //   1. prefix products, one thread per request, fp32, left to right           (Eq. 3)
-//   2. 64-bit keys (inverted score bits | depth | request) and a bitonic sort in shared memory:
+//   2. 64-bit keys (inverted score bits | depth | request) and a bitonic sort held in registers (warp shuffles
+//      for short distances, a double-buffered shared array for long ones):
 //      ascending key order = score descending, depth ascending, request ascending
 //   3. block-wide scan of the fixed-point scores floor(p * 2^40) in int64 (exact in any order)
 //   4. objective (B*2^40 + Q_N) / cost for every candidate N, fp64 divide, block argmax with
@@ -13,6 +14,12 @@
 #include <limits.h>
 
 #include "dcut_internal.h"
+#ifdef DCUT_PROFILE_SEL
+#include <stdio.h>
+#define SELP(...) __VA_ARGS__
+#else
+#define SELP(...)
+#endif
 
 namespace {
 
@@ -76,6 +83,77 @@ __device__ __forceinline__ T block_exclusive_scan(T v, T* ws, T* total_out) {
     return res;
 }
 
+// keep the smaller (or larger) of own and partner key
+__device__ __forceinline__ unsigned long long cx(unsigned long long mine, unsigned long long other, bool keep_min) {
+    return ((mine < other) == keep_min) ? mine : other;
+}
+
+template <int E>
+__device__ __forceinline__ void sort_keys_e(unsigned long long* keys, unsigned long long (*xbuf)[kThreads], int npad) {
+    const int tid = threadIdx.x;
+    unsigned long long k[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int idx = e * kThreads + tid;
+        k[e] = idx < npad ? keys[idx] : ~0ull;
+    }
+    __syncthreads();
+    int p = 0;
+    constexpr int S = E * kThreads;
+    for (int kk = 2; kk <= S; kk <<= 1) {
+        for (int j = kk >> 1; j > 0; j >>= 1) {
+            if (j >= kThreads) {                      // partner in the same thread
+#pragma unroll
+                for (int je = E / 2; je >= 1; je >>= 1) {
+                    if (j == je * kThreads) {
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            if ((e & je) == 0) {
+                                const int idx = e * kThreads + tid;
+                                const bool up = (idx & kk) == 0;
+                                const unsigned long long a = k[e], b = k[e | je];
+                                const bool swap = (a > b) == up;
+                                k[e] = swap ? b : a;
+                                k[e | je] = swap ? a : b;
+                            }
+                        }
+                    }
+                }
+            } else if (j >= 32) {                     // partner in another warp: through shared memory
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    xbuf[p][tid] = k[e];
+                    __syncthreads();
+                    const unsigned long long other = xbuf[p][tid ^ j];
+                    const int idx = e * kThreads + tid;
+                    k[e] = cx(k[e], other, ((idx & kk) == 0) == ((tid & j) == 0));
+                    p ^= 1;
+                }
+            } else {                                  // partner in the same warp
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, k[e], j);
+                    const int idx = e * kThreads + tid;
+                    k[e] = cx(k[e], other, ((idx & kk) == 0) == ((tid & j) == 0));
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int idx = e * kThreads + tid;
+        if (idx < npad) keys[idx] = k[e];
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ void sort_keys(unsigned long long* keys, unsigned long long (*xbuf)[kThreads], int npad) {
+    if (npad <= kThreads) sort_keys_e<1>(keys, xbuf, npad);
+    else if (npad <= 2 * kThreads) sort_keys_e<2>(keys, xbuf, npad);
+    else if (npad <= 4 * kThreads) sort_keys_e<4>(keys, xbuf, npad);
+    else sort_keys_e<8>(keys, xbuf, npad);
+}
+
 struct Best {
     double obj;
     int N;
@@ -93,12 +171,14 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     long long* qs = reinterpret_cast<long long*>(keys + npad);                       // [npad + 1]
     int* depth_s = reinterpret_cast<int*>(qs + npad + 1);                            // [B]
     int* cu_s = depth_s + B;                                                         // [B + 1]
+    __shared__ unsigned long long xbuf[2][kThreads];
     __shared__ long long ws64[kWarps + 1];
     __shared__ int ws32[kWarps + 1];
     __shared__ Best wbest[kWarps];
     __shared__ Best best_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    SELP(long long t0 = clock64();)
     // 1. prefix scores and sort keys.  The confidences come in through shared memory with coalesced loads
     // (the later prefix-sum array is free at this point), so the per-request product chain reads no global memory.
     float* conf_s = reinterpret_cast<float*>(qs);
@@ -119,23 +199,12 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     for (int i = tid; i < B; i += kThreads) depth_s[i] = 0;
     __syncthreads();
 
-    // 2. bitonic sort, ascending
-    for (int k = 2; k <= npad; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < (npad >> 1); t += kThreads) {
-                const int i = 2 * t - (t & (j - 1));
-                const int l = i + j;
-                const bool up = (i & k) == 0;
-                const unsigned long long x = keys[i], y = keys[l];
-                if ((x > y) == up) {
-                    keys[i] = y;
-                    keys[l] = x;
-                }
-            }
-            __syncthreads();
-        }
-    }
-
+    SELP(long long t1 = clock64();)
+    // 2. bitonic sort, ascending, over S = max(npad, 1024) keys held in registers: thread t owns elements
+    // e * 1024 + t.  Compare-exchange distances below 32 go through warp shuffles, distances 32..512 through a
+    // double-buffered shared array (one barrier per stage), distances >= 1024 stay inside the thread.
+    sort_keys(keys, xbuf, npad);
+    SELP(long long t2 = clock64();)
     // 3. fixed-point prefix sums Q[0..n]; ranks
     {
         const int per = (npad + kThreads - 1) / kThreads;
@@ -167,6 +236,7 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     }
     __syncthreads();
 
+    SELP(long long t3 = clock64();)
     // 4. objective over the candidates
     {
         const long long bfix = (long long)B << 40;
@@ -211,6 +281,7 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     }
     const int n_star = best_s.N;
 
+    SELP(long long t4 = clock64();)
     // 5. depths, cu_q, packed token metadata
     for (int r = tid; r < n_star; r += kThreads) atomicAdd(&depth_s[(int)(keys[r] & 0xffffu)], 1);
     __syncthreads();
@@ -253,6 +324,7 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
             if (a.tok_id) a.tok_id[idx] = -1;
         }
     }
+    SELP(if (tid == 0) printf("select cycles: load+products %lld sort %lld scan %lld objective %lld depths+meta %lld\n", t1 - t0, t2 - t1, t3 - t2, t4 - t3, clock64() - t4);)
     if (tid == 0 && a.info) {
         dcut_select_info out;
         out.n_star = n_star;
