@@ -468,7 +468,10 @@ def run_dcut(args):
         line["config"]["arm"] += "; verification forward = one decoder layer (dcut_layer_forward)"
         line["layer"] = {"gemm_alone": gemm, "flops_per_token": layer_flops(cfg, 1)}
         g = gemm["full_gamma"]["all"]
-        line["roofline_tensor"] = {"kernel": "gemm_tcgen05_kernel (4 projections of the layer, full-gamma arm, timed alone)",
+        for v in line["arms"].values():   # here the timed middle stage is the whole layer, not attention alone
+            v["forward_ms"] = v.pop("attn_ms")
+            v.pop("attn_gbs")
+        line["roofline"] = line["roofline_tensor"] = {"kernel": "gemm_tcgen05_kernel (4 projections of the layer, full-gamma arm, timed alone)",
                                    "bound": "tensor", "achieved": g["tflops"], "peak": tf_peak, "unit": "TFLOP/s",
                                    "frac": round(g["tflops"] / tf_peak, 4),
                                    "peak_source": "of measured (burst)" if pkj else "of fallback", "traffic": None}

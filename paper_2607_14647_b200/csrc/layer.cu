@@ -28,7 +28,7 @@ constexpr int kATile = BM * BK * 2;            // 16 KB
 constexpr int kBTile = BN * BK * 2;            // 32 KB
 constexpr int kGemmStageBytes = kATile + kBTile;
 constexpr int kGemmThreads = 192;              // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
-constexpr int kTmemCols = 256;
+constexpr int kTmemCols = 512;              // two 128 x 256 fp32 accumulators
 constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256 /* barriers, tmem ptr */;
 constexpr int kWaitLimit = 1 << 22;
 
@@ -61,6 +61,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // One lane of a converged warp.  Issuing tcgen05 / TMA instructions under this predicate (rather than under
 // `lane == 0`) lets the compiler keep their operands in uniform registers; measured on B200 this halves the
@@ -122,25 +125,29 @@ struct GemmArgs {
     int B;
     int N_out;         // columns of the output (kSwiGLU: the intermediate size I; otherwise N)
     int K;
+    int n_tiles;       // output tiles along N
     __nv_bfloat16* out;
     const __nv_bfloat16* residual;   // [T, N_out] or null
     int* status;
 };
 
+// Persistent: a CTA walks the output tiles b, b + gridDim.x, ... (m fastest, so the CTAs running together share
+// weight tiles in L2).  The operand ring and its barriers simply continue across tiles; the accumulator is
+// double-buffered in tensor memory (2 x 256 columns), so the epilogue of one tile overlaps the main loop of the next.
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                     const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
     const int T = g.cu_q[g.B];
-    const int m0 = blockIdx.x * BM;
-    if (m0 >= T) return;
-    const int n_tile = blockIdx.y;
+    const int m_tiles = (T + BM - 1) / BM;
+    const int n_work = m_tiles * g.n_tiles;
+    if ((int)blockIdx.x >= n_work) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGemmStages + 1);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGemmStages + 4);
     const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
-    const uint32_t accum_bar = smem_u32(bars + 2 * kGemmStages);
+    const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages), acc_empty = acc_full + 16;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_kb = g.K / BK;
 
@@ -149,11 +156,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
             mbar_init(full_bar + 8 * s, 1);
             mbar_init(empty_bar + 8 * s, 1);
         }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full + 8 * b, 1);
+            mbar_init(acc_empty + 8 * b, 128);   // the four epilogue warps
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {   // tensor memory: 256 columns for the 128 x 256 fp32 accumulator
+    if (warp == 1) {   // tensor memory: two 128 x 256 fp32 accumulators
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -165,56 +175,78 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
-        for (int kb = 0; kb < n_kb; ++kb) {
-            const int s = kb % kGemmStages;
-            if (kb >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kb / kGemmStages) - 1) & 1))) {
-                failed = true;
-                break;
-            }
-            if (elect_one()) {
-                const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
-                const uint32_t bar = full_bar + 8 * s;
-                mbar_arrive_expect_tx(bar, kGemmStageBytes);
-                tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
-                if (MODE == kSwiGLU) {   // 128 gate rows, then the 128 up rows of the same features
-                    tma_load_2d(b_dst, &b_map, kb * BK, n_tile * (BN / 2), bar);
-                    tma_load_2d(b_dst + kBTile / 2, &b2_map, kb * BK, n_tile * (BN / 2), bar);
-                } else {
-                    tma_load_2d(b_dst, &b_map, kb * BK, n_tile * BN, bar);
-                    tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
+        int kc = 0;   // k-blocks issued so far, over all tiles
+        for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x) {
+            const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
+            for (int kb = 0; kb < n_kb; ++kb, ++kc) {
+                const int s = kc % kGemmStages;
+                if (kc >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kGemmStages) - 1) & 1))) {
+                    failed = true;
+                    break;
                 }
+                if (elect_one()) {
+                    const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
+                    const uint32_t bar = full_bar + 8 * s;
+                    mbar_arrive_expect_tx(bar, kGemmStageBytes);
+                    tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
+                    if (MODE == kSwiGLU) {   // 128 gate rows, then the 128 up rows of the same features
+                        tma_load_2d(b_dst, &b_map, kb * BK, n_tile * (BN / 2), bar);
+                        tma_load_2d(b_dst + kBTile / 2, &b2_map, kb * BK, n_tile * (BN / 2), bar);
+                    } else {
+                        tma_load_2d(b_dst, &b_map, kb * BK, n_tile * BN, bar);
+                        tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
+                    }
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
-        for (int kb = 0; kb < n_kb; ++kb) {
-            const int s = kb % kGemmStages;
-            if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kb / kGemmStages) & 1))) {
+        int kc = 0, it = 0;
+        for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
+            const int acc = it & 1;
+            // the epilogue must have drained this accumulator (used by tile it - 2)
+            if (it >= 2 && !__all_sync(0xffffffffu, mbar_wait(acc_empty + 8 * acc, ((it >> 1) - 1) & 1))) {
                 failed = true;
                 break;
             }
             tc_fence_after();
-            if (elect_one()) {
-                const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
-                const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
+            const uint32_t tmem_d = tmem_base + acc * BN;
+            for (int kb = 0; kb < n_kb; ++kb, ++kc) {
+                const int s = kc % kGemmStages;
+                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kGemmStages) & 1))) {
+                    failed = true;
+                    break;
+                }
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
+                    const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
 #pragma unroll
-                for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
-                    tc_mma(tmem_base, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
-                tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
+                    for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
+                        tc_mma(tmem_d, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+                    tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
+                }
+                __syncwarp();
             }
+            if (failed) break;
+            if (elect_one()) tc_commit(acc_full + 8 * acc);   // accumulator complete
             __syncwarp();
         }
-        if (elect_one()) tc_commit(accum_bar);      // accumulator complete
-        __syncwarp();
     } else {
         // ---------------------------------------------------------------- epilogue warps
         const int quarter = warp & 3;               // tensor-memory lanes 32 * quarter .. + 31
-        const int row = m0 + quarter * 32 + lane;
-        if (!mbar_wait(accum_bar, 0)) failed = true;
-        tc_fence_after();
-        if (!failed) {
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        int it = 0;
+        for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
+            const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
+            const int acc = it & 1;
+            const int row = m0 + quarter * 32 + lane;
+            if (!mbar_wait(acc_full + 8 * acc, (it >> 1) & 1)) {
+                failed = true;
+                break;
+            }
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
             if (MODE == kSwiGLU) {
                 __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + (size_t)n_tile * (BN / 2);
 #pragma unroll 1
@@ -226,14 +258,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                     if (row < T) {
 #pragma unroll
                         for (int e = 0; e < 32; e += 8) {
-                            uint32_t w[4];
+                            uint32_t o[4];
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const float g0 = __uint_as_float(gt[e + 2 * j]), g1 = __uint_as_float(gt[e + 2 * j + 1]);
                                 const float u0 = __uint_as_float(up[e + 2 * j]), u1 = __uint_as_float(up[e + 2 * j + 1]);
-                                w[j] = pack_bf16(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+                                o[j] = pack_bf16(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
                             }
-                            *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                            *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
                 }
@@ -242,8 +274,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                 const __nv_bfloat16* rrow = MODE == kResidual ? g.residual + (size_t)row * g.N_out + (size_t)n_tile * BN : nullptr;
 #pragma unroll 1
                 for (int c = 0; c < BN; c += 32) {
-                    uint32_t acc[32];
-                    tc_ld32(t_row + c, acc);
+                    uint32_t av[32];
+                    tc_ld32(t_row + c, av);
                     tc_wait_ld();
                     if (row < T) {
 #pragma unroll
@@ -251,16 +283,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                             uint4 res = make_uint4(0, 0, 0, 0);
                             if (MODE == kResidual) res = *reinterpret_cast<const uint4*>(rrow + c + e);
                             const uint32_t rw[4] = {res.x, res.y, res.z, res.w};
-                            uint32_t w[4];
+                            uint32_t o[4];
 #pragma unroll
                             for (int j = 0; j < 4; ++j)
-                                w[j] = pack_bf16(__uint_as_float(acc[e + 2 * j]) + bf_lo(rw[j]),
-                                                 __uint_as_float(acc[e + 2 * j + 1]) + bf_hi(rw[j]));
-                            *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                                o[j] = pack_bf16(__uint_as_float(av[e + 2 * j]) + bf_lo(rw[j]),
+                                                 __uint_as_float(av[e + 2 * j + 1]) + bf_hi(rw[j]));
+                            *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
                 }
             }
+            // this accumulator may be overwritten once all four epilogue warps have read it
+            tc_fence_before();
+            mbar_arrive(acc_empty + 8 * acc);
         }
     }
     if (failed) atomicExch(g.status, DCUT_DEV_GEMM_WAIT_TIMEOUT);
@@ -387,8 +422,11 @@ dcut_status make_kmajor_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, l
 template <int MODE>
 dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& b2, int n_tiles,
                         int T_cap, const GemmArgs& g, cudaStream_t stream) {
-    dim3 grid((T_cap + BM - 1) / BM, n_tiles);
-    gemm_tcgen05_kernel<MODE><<<grid, kGemmThreads, kGemmSmem, stream>>>(a, b, b2, g);
+    GemmArgs ga = g;
+    ga.n_tiles = n_tiles;
+    const int n_work = ((T_cap + BM - 1) / BM) * n_tiles;
+    const int grid = n_work < ctx->sm_count ? n_work : ctx->sm_count;   // persistent: at most one CTA per SM
+    gemm_tcgen05_kernel<MODE><<<grid, kGemmThreads, kGemmSmem, stream>>>(a, b, b2, ga);
     return dcut_check_cuda(ctx, cudaGetLastError(), "launch gemm_tcgen05_kernel");
 }
 
