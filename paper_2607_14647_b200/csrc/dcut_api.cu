@@ -124,7 +124,14 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
         const char* env = getenv("DCUT_ATTN_TARGET_ITEMS");
         c->target_items = env ? atoi(env) : c->sm_count * 2;   // requests are only cut when the batch has fewer (request, head) pairs than that
         if (c->target_items < 1) c->target_items = 1;
-        c->max_items = 2 * (lim->max_B * lim->n_kv_heads + c->target_items);   // x2: query tiles above 128 rows are cut in two
+        env = getenv("DCUT_ATTN_TAIL_REQ_DIV");
+        c->attn_tail_req_div = env ? atoi(env) : 0;
+        env = getenv("DCUT_ATTN_TAIL_MIN_PAGES");
+        c->attn_tail_min_pages = env ? atoi(env) : 32;
+        if (c->attn_tail_min_pages < 8) c->attn_tail_min_pages = 8;
+        // whole-batch cut (<= target_items + pairs) + tail cut (<= target_items + pairs); x2: query tiles above 128
+        // rows are cut in two
+        c->max_items = 2 * (2 * lim->max_B * lim->n_kv_heads + 2 * c->target_items);
         const int group = lim->n_q_heads / lim->n_kv_heads;
         c->part_rows_cap = (long long)c->max_items * (lim->max_gamma + 1) * group;
         if ((st = dmalloc(c, &c->d_items, c->max_items, "cudaMalloc(items)")) != DCUT_OK) return st;

@@ -54,6 +54,8 @@ struct dcut_ctx {
     int max_items;
     long long part_rows_cap;
     int target_items;
+    int attn_tail_req_div;  // the shortest max(1, B / this) requests are cut finer (0: none)
+    int attn_tail_min_pages;
     int attn_tc_min_rows;   // items with at least this many query rows (and <= 128) use the tcgen05 kernel
 
     // accept scratch

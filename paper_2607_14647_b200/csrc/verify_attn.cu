@@ -27,6 +27,25 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdlib.h>
+#ifdef DCUT_PROFILE_STAMPS
+// profiling builds only: wall-clock stamps (ns) of the three kernels of one call
+__device__ unsigned long long g_attn_stamps[8];   // plan start/end, item first start/last end, combine first start/last end, item first-CTA-after-wait
+__device__ __forceinline__ unsigned long long gtime() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define STAMP_MIN(i) do { if (threadIdx.x == 0) atomicMin(&g_attn_stamps[i], gtime()); } while (0)
+#define STAMP_MAX(i) do { if (threadIdx.x == 0) atomicMax(&g_attn_stamps[i], gtime()); } while (0)
+extern "C" void dcut_debug_attn_stamps(unsigned long long* out) {
+    cudaMemcpyFromSymbol(out, g_attn_stamps, sizeof(unsigned long long) * 8);
+    unsigned long long init[8] = {~0ull, 0, ~0ull, 0, ~0ull, 0, ~0ull, 0};
+    cudaMemcpyToSymbol(g_attn_stamps, init, sizeof(init));
+}
+#else
+#define STAMP_MIN(i)
+#define STAMP_MAX(i)
+#endif
 #ifdef DCUT_PROFILE_TC
 #include <stdio.h>
 #define TCP(...) __VA_ARGS__
@@ -139,6 +158,7 @@ struct PlanArgs {
     const int* cu_q;
     int B, n_q_heads, n_kv_heads;
     int target_items, min_chunk_pages, max_items, npad, tc_min_rows, max_item_rows;
+    int tail_req_div, tail_min_pages;   // the shortest B / tail_req_div requests are cut finer (0: none)
     long long part_rows_cap;
     int* status;
     AttnItem* items;
@@ -179,10 +199,15 @@ __device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* to
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     extern __shared__ unsigned long long order[];   // [npad] (inverted cost << 32 | request), sorted ascending
     __shared__ int ws[33];
-    __shared__ int total_s;
+    __shared__ int total_s, tail_s;
     const int tid = threadIdx.x, nthr = blockDim.x;   // 256 threads for small batches: cheaper barriers
+    STAMP_MIN(0);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the item kernel's CTAs may take their SMs now
     const int group = a.n_q_heads / a.n_kv_heads;
-    if (tid == 0) total_s = 0;
+    if (tid == 0) {
+        total_s = 0;
+        tail_s = 0;
+    }
     __syncthreads();
     int local = 0;
     for (int i = tid; i < a.B; i += nthr) {
@@ -225,6 +250,20 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             __syncthreads();
         }
 
+    // The items that start last decide how unevenly the SMs finish: the requests at the end of the order are cut
+    // into about target_items pieces altogether, so every SM ends on a short item.
+    const int n_tail = a.tail_req_div > 0 ? (a.B + a.tail_req_div - 1) / a.tail_req_div : 0;
+    const int tail_from = a.B - n_tail;
+    for (int j = tail_from + tid; j < a.B; j += nthr) {
+        const int i = (int)(order[j] & 0xffffffffu);
+        const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+        atomicAdd(&tail_s, (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage);
+    }
+    __syncthreads();
+    int tail_chunk = (int)(((long long)tail_s * a.n_kv_heads + a.target_items - 1) / a.target_items);
+    if (tail_chunk < a.tail_min_pages) tail_chunk = a.tail_min_pages;
+    if (tail_chunk > chunk_pages) tail_chunk = chunk_pages;
+
     const int per = (a.B + nthr - 1) / nthr;
     const int j0 = tid * per;
     int my_items = 0, my_rows = 0;
@@ -234,7 +273,8 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             const int i = (int)(order[j] & 0xffffffffu);
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-            const int nc = (pages + chunk_pages - 1) / chunk_pages;
+            const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
+            const int nc = (pages + cpj - 1) / cpj;
             const int n_rb = ((d + 1) * group + a.max_item_rows - 1) / a.max_item_rows;
             my_items += nc * a.n_kv_heads * n_rb;
             if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
@@ -250,6 +290,9 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
         a.plan[2] = total_pages;
         a.plan[3] = n_rows;
         a.plan[4] = overflow ? 1 : 0;
+#ifdef DCUT_PROFILE_STAMPS
+        atomicMax(&g_attn_stamps[1], gtime());
+#endif
         if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
     }
     if (overflow) return;
@@ -261,7 +304,8 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             const int d = a.cu_q[i + 1] - q0 - 1;
             const int ctx_len = a.ctx_lens[i];
             const int pages = (ctx_len + d + 1 + kPage - 1) / kPage;
-            const int nc = (pages + chunk_pages - 1) / chunk_pages;
+            const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
+            const int nc = (pages + cpj - 1) / cpj;
             const int cp = (pages + nc - 1) / nc;   // near-equal chunks
             const int M = (d + 1) * group;
             a.req_part[2 * i] = row_off;
@@ -1029,6 +1073,12 @@ template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                  const __grid_constant__ CUtensorMap k2_map, AttnArgs a) {
+    // launched with programmatic stream serialization: the CTAs may become resident while the plan kernel still
+    // runs, so nothing it writes is read before this wait
+    STAMP_MIN(2);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    STAMP_MIN(6);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if ((int)blockIdx.x >= a.plan[0]) return;
     extern __shared__ unsigned char smem_raw[];
     const AttnItem item = a.items[blockIdx.x];
@@ -1036,6 +1086,7 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
         tc_item(k2_map, v_map, a, item, smem_raw);
     else
         split_item<DH>(k_map, v_map, a, item, smem_raw);
+    STAMP_MAX(3);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1053,14 +1104,18 @@ struct CombineArgs {
 };
 
 template <int DH>
-__global__ void __launch_bounds__(256) attn_combine_kernel(CombineArgs a) {
-    // grid: x = request * (gamma_max + 1) + block position t, y = group of 8 q heads; warp = one head
+__global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
+    // grid: x = request * (gamma_max + 1) + block position t, y = group of blockDim.x / 32 q heads; warp = one head.
+    // Launched with programmatic stream serialization (see attn_item_kernel).
+    STAMP_MIN(4);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    STAMP_MAX(5);
     if (a.plan[4]) return;
     const int req = blockIdx.x / a.tokens_per_req, t = blockIdx.x - req * a.tokens_per_req;
     const int nc = a.req_part[2 * req + 1];
     if (nc <= 1) return;
     const int lane = threadIdx.x & 31;
-    const int h = blockIdx.y * 8 + (threadIdx.x >> 5);
+    const int h = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (h >= a.n_q_heads || t >= a.cu_q[req + 1] - a.cu_q[req]) return;
     const int tok = a.cu_q[req] + t;
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -1120,13 +1175,26 @@ template <int DH>
 dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& k2m, const AttnArgs& aa,
                      const CombineArgs& ca, int T_cap, cudaStream_t stream) {
     constexpr int kSmem = (DH == 128 && kTcSmem > SmemLayout<DH>::kTotal) ? kTcSmem : SmemLayout<DH>::kTotal;
-    attn_item_kernel<DH><<<ctx->max_items, kThreads, kSmem, stream>>>(km, vm, k2m, aa);
-    dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_item_kernel");
+    // Both kernels may be scheduled before their predecessor has finished (they wait on the device before reading
+    // its results), which hides the launch latency between the three kernels of the call.
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(ctx->max_items);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = kSmem;
+    lc.stream = stream;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    dcut_status st = dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, attn_item_kernel<DH>, km, vm, k2m, aa), "launch attn_item_kernel");
     if (st != DCUT_OK) return st;
     (void)T_cap;
-    dim3 cgrid(ca.B * ca.tokens_per_req, (ctx->lim.n_q_heads + 7) / 8);
-    attn_combine_kernel<DH><<<cgrid, 256, 0, stream>>>(ca);
-    return dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_combine_kernel");
+    const int heads_per_cta = ctx->lim.n_q_heads < 32 ? ((ctx->lim.n_q_heads + 7) / 8) * 8 : 32;
+    lc.gridDim = dim3(ca.B * ca.tokens_per_req, (ctx->lim.n_q_heads + heads_per_cta - 1) / heads_per_cta);
+    lc.blockDim = dim3(32 * heads_per_cta);
+    lc.dynamicSmemBytes = 0;
+    return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, attn_combine_kernel<DH>, ca), "launch attn_combine_kernel");
 }
 
 }  // namespace
@@ -1181,6 +1249,8 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.n_kv_heads = ctx->lim.n_kv_heads;
     pa.target_items = ctx->target_items;
     pa.min_chunk_pages = 8;
+    pa.tail_req_div = ctx->attn_tail_req_div;
+    pa.tail_min_pages = ctx->attn_tail_min_pages;
     pa.npad = 32;
     while (pa.npad < B) pa.npad <<= 1;
     pa.status = ctx->d_status;
