@@ -135,7 +135,7 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
         const int group = lim->n_q_heads / lim->n_kv_heads;
         c->part_rows_cap = (long long)c->max_items * (lim->max_gamma + 1) * group;
         if ((st = dmalloc(c, &c->d_items, c->max_items, "cudaMalloc(items)")) != DCUT_OK) return st;
-        if ((st = dmalloc(c, &c->d_plan, 8, "cudaMalloc(plan)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->d_plan, 16, "cudaMalloc(plan)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->d_req_part, 2 * (size_t)lim->max_B, "cudaMalloc(req_part)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->d_part_o, (size_t)c->part_rows_cap * lim->head_dim, "cudaMalloc(part_o)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->d_part_lse, (size_t)c->part_rows_cap, "cudaMalloc(part_lse)")) != DCUT_OK) return st;

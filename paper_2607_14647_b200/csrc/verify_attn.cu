@@ -1,29 +1,30 @@
 // dcut_verify_attn: ragged causal multi-token attention over a paged bf16 KV cache.
 //
-// HBM-bound by design: every K/V byte of every request is read once per step, so the kernel is
-// organised around keeping ~100 KB of page loads in flight per SM and doing the (small) matrix
-// work out of shared memory on the warp-level tensor-core path.
+// HBM-bound by design: every K/V byte of every request is read once per step, so the kernels are organised around
+// keeping 100-200 KB of page loads in flight per SM, all the time.
 //
-//   attn_plan_kernel     one CTA.  Cuts every request's page list into near-equal chunks so the
-//                        batch gives a few work items per SM (flash-decoding split-KV); an item is
-//                        one (request, kv head, page range).
-//   attn_split_kernel    one CTA per item: 15 consumer warps + 1 producer warp.
-//       producer         a few lanes read the block table and issue TMA tile loads (3-D tensor map over
-//                        the cache, one 4 KB box per (page, kv head) tile, 128-byte swizzle) into a
-//                        ring of page stages, each guarded by a full/empty mbarrier pair.  The ring is
-//                        cut into one sub-ring per page slot.
-//       consumers        the item's query tile is (1 + d_i) * group rows (every query token of the
-//                        request times the q heads sharing this kv head), cut into 16-row m-tiles.
-//                        Warp w owns m-tile (w mod MT) and page slot (w div MT): it runs
-//                        S = Q K^T, online softmax and O += P V for its m-tile on every
-//                        nslots-th page (mma.sync m16n8k16 bf16, fp32 accumulate, ldmatrix from the
-//                        swizzled tiles), taking them in order from its slot's sub-ring.  Small query tiles therefore spread pages over warps,
-//                        large ones spread rows.
-//       epilogue         the slots' (m, l, O) are merged through shared memory; a request with one
-//                        chunk writes bf16 output directly, otherwise normalised fp32 partials + LSE.
-//   attn_combine_kernel  merges the chunks of multi-chunk requests.
+//   attn_plan_kernel     one CTA.  Cuts the requests' page lists into work items (flash-decoding split-KV, only when the
+//                        batch has fewer (request, kv head) pairs than two per SM); an item is one (request, kv head,
+//                        page range, block of query rows).  Items go to one of two queues, each ordered longest first:
+//                        query tiles of 17+ rows to the tcgen05 queue, smaller ones to the warp-level queue.
+//   attn_item_kernel     persistent, one CTA per SM.  A CTA claims items from the tcgen05 queue, then from the warp-level
+//                        queue, through a global counter.  In both phases the TMA producer warp claims the next item as
+//                        soon as it has issued the current item's last load and keeps streaming into the same ring of
+//                        stages (stages, tensor-memory buffers and their mbarriers are numbered through consecutive
+//                        items), so the loads never pause at an item boundary.
+//       tcgen05 phase    Q and P in tensor memory, page groups of four (64 keys), S = Q K^T and O += P V as tcgen05.mma,
+//                        softmax by two threads per row (see tc_phase).
+//       warp-level phase 8 consumer warps + 1 producer warp; the query tile is cut into 16-row m-tiles, warp w owns
+//                        m-tile (w mod MT) and page slot (w div MT) and runs S = Q K^T, online softmax and O += P V on
+//                        every nslots-th page (mma.sync m16n8k16 bf16, fp32 accumulate, ldmatrix from the swizzled
+//                        tiles), in order from its slot's sub-ring; the slots' (m, l, O) are merged through shared
+//                        memory (see mma_phase).
+//       output           an item of an uncut request writes bf16 output directly, otherwise normalised fp32 partials
+//                        and their log-sum-exp.
+//   attn_combine_kernel  merges the chunks of cut requests.
 //
-// Every mbarrier wait is bounded; on expiry the CTA sets the device status word and leaves.
+// The three kernels are chained with programmatic dependent launch.  Every mbarrier wait is bounded; on expiry the CTA
+// sets the device status word and every role leaves at a point where none is left waiting at a named barrier.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdlib.h>
@@ -57,13 +58,13 @@ extern "C" void dcut_debug_attn_stamps(unsigned long long* out) {
 
 namespace {
 
-constexpr int kConsumerWarps = 15;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kThreads = kConsumerThreads + 32;
-constexpr int kStages = 20;        // page stages in the ring (8 KB each at head_dim 128)
-constexpr int kMaxProducerLanes = 6;
-constexpr int kPage = 16;          // tokens per page
-constexpr int kMaxMTiles = 9;      // query rows per item <= 144
+constexpr int kThreads = 320;        // tcgen05 phase: TMA warp, MMA warp, 8 softmax warps; warp-level phase: 8 consumer warps + 1 producer
+constexpr int kMmaWarps = 8;         // consumer warps of the warp-level MMA phase
+constexpr int kMmaThreads = kMmaWarps * 32;
+constexpr int kMmaStages = 16;       // page stages in its ring (8 KB each at head_dim 128)
+constexpr int kMaxProducerLanes = 8;
+constexpr int kPage = 16;            // tokens per page
+constexpr int kMaxMTiles = 8;        // query rows per item <= 128
 constexpr int kPlanThreads = 1024;
 constexpr int kSpinLimit = 1 << 21;   // bounded waits: ~1 s, then the CTA reports and leaves
 
@@ -140,10 +141,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void consumer_bar() {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
-}
-
 // byte offset of 16-byte chunk `c16` (0 .. DH/8-1) of token/row `r` (0..15) inside a swizzled
 // [DH/64][16][64] bf16 tile (what two 64-column TMA boxes with 128-byte swizzle produce)
 __device__ __forceinline__ uint32_t tile_off(int r, int c16) {
@@ -162,7 +159,7 @@ struct PlanArgs {
     long long part_rows_cap;
     int* status;
     AttnItem* items;
-    int* plan;       // [0] n_items, [1] chunk_pages, [2] total_pages, [3] partial rows used
+    int* plan;       // [0] n_items, [1] chunk_pages, [2] total_pages, [3] partial rows used, [4] overflow, [5] n_tc, [8], [9] queue heads
     int* req_part;   // [B][2]: first partial row, n_chunks
 };
 
@@ -266,7 +263,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
 
     const int per = (a.B + nthr - 1) / nthr;
     const int j0 = tid * per;
-    int my_items = 0, my_rows = 0;
+    int my_tc = 0, my_mma = 0, my_rows = 0;
     for (int e = 0; e < per; ++e) {
         const int j = j0 + e;
         if (j < a.B) {
@@ -275,14 +272,23 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
             const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
             const int nc = (pages + cpj - 1) / cpj;
-            const int n_rb = ((d + 1) * group + a.max_item_rows - 1) / a.max_item_rows;
-            my_items += nc * a.n_kv_heads * n_rb;
+            // row blocks of the query tile: full blocks of max_item_rows rows and one remainder; each goes to the
+            // tcgen05 queue or to the warp-level queue by its number of rows
+            const int M = (d + 1) * group;
+            const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
+            const int tc_rb = (a.max_item_rows >= a.tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= a.tc_min_rows) ? 1 : 0);
+            const int n_rb = n_full + (rem > 0 ? 1 : 0);
+            my_tc += nc * a.n_kv_heads * tc_rb;
+            my_mma += nc * a.n_kv_heads * (n_rb - tc_rb);
             if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
         }
     }
-    int n_items, n_rows;
-    int item_off = plan_block_exclusive_scan(my_items, ws, &n_items);
+    int n_tc, n_mma, n_rows;
+    int tc_off = plan_block_exclusive_scan(my_tc, ws, &n_tc);
+    int mma_off = plan_block_exclusive_scan(my_mma, ws, &n_mma);
     int row_off = plan_block_exclusive_scan(my_rows, ws, &n_rows);
+    const int n_items = n_tc + n_mma;
+    mma_off += n_tc;
     const bool overflow = n_items > a.max_items || (long long)n_rows > a.part_rows_cap;
     if (tid == 0) {
         a.plan[0] = overflow ? 0 : n_items;
@@ -290,6 +296,9 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
         a.plan[2] = total_pages;
         a.plan[3] = n_rows;
         a.plan[4] = overflow ? 1 : 0;
+        a.plan[5] = overflow ? 0 : n_tc;     // items [0, n_tc): tcgen05 queue; [n_tc, n_items): warp-level queue
+        a.plan[8] = 0;                       // next item of the tcgen05 queue (claimed by the CTAs of the item kernel)
+        a.plan[9] = overflow ? 0 : n_tc;     // next item of the warp-level queue
 #ifdef DCUT_PROFILE_STAMPS
         atomicMax(&g_attn_stamps[1], gtime());
 #endif
@@ -327,334 +336,16 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
                         it.q0 = q0;
                         it.depth = d;
                         it.ctx_len = ctx_len;
-                        it.pad[0] = (rows >= a.tc_min_rows && rows <= 128) ? 1 : 0;   // which path takes the item
-                        it.pad[1] = row0;    // first query row of the item within the request's tile
-                        it.pad[2] = rows;    // query rows of the item
-                        a.items[item_off + (c * a.n_kv_heads + h) * n_rb + rb] = it;
+                        const bool tc = rows >= a.tc_min_rows;
+                        it.pad[0] = tc ? 1 : 0;   // which queue the item is in
+                        it.pad[1] = row0;         // first query row of the item within the request's tile
+                        it.pad[2] = rows;         // query rows of the item
+                        a.items[tc ? tc_off++ : mma_off++] = it;
                     }
-            item_off += nc * a.n_kv_heads * n_rb;
             if (nc > 1) row_off += nc * (d + 1) * a.n_q_heads;
         }
     }
 }
-
-// ------------------------------------------------------------------------------------------------
-// split-KV attention
-
-struct AttnArgs {
-    const __nv_bfloat16* q;
-    const int* block_table;
-    int block_table_stride;
-    const int* ctx_lens;
-    const int* cu_q;
-    const AttnItem* items;
-    const int* plan;
-    int n_q_heads, n_kv_heads;
-    long long num_pages;
-    float scale_log2;          // softmax scale * log2(e)
-    __nv_bfloat16* out;
-    float* lse;                // [T, Hq] or null
-    float* part_o;
-    float* part_lse;
-    int* status;
-};
-
-template <int DH>
-struct SmemLayout {
-    static constexpr int kPageBytes = kPage * DH * 2;            // one K or V page tile
-    static constexpr int kStageBytes = 2 * kPageBytes;
-    static constexpr int kRingBytes = kStages * kStageBytes;
-    static constexpr int kQBytes = kMaxMTiles * 16 * DH * 2;
-    static constexpr int kMergeStride = DH + 8;                  // floats per merged row
-    static constexpr int kMergeBytes = kConsumerWarps * 16 * kMergeStride * 4;
-    static constexpr int kMLBytes = kConsumerWarps * 16 * 2 * 4;
-    static constexpr int kBarBytes = 2 * kStages * 8;
-    static constexpr int kRingOrMerge = kRingBytes > kMergeBytes ? kRingBytes : kMergeBytes;
-    static constexpr int kTotal = kRingOrMerge + kQBytes + kMLBytes + kBarBytes + 1024 /* alignment slack */;
-};
-
-template <int DH>
-__device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnArgs& a,
-                                           const AttnItem& item, unsigned char* smem_raw) {
-    using L = SmemLayout<DH>;
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned char* ring = smem;
-    unsigned char* q_s = smem + L::kRingOrMerge;
-    float* ml_s = reinterpret_cast<float*>(q_s + L::kQBytes);
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(ml_s) + L::kMLBytes);
-    __shared__ int abort_s;
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int req = item.req, kvh = item.kv_head;
-    const int group = a.n_q_heads / a.n_kv_heads;
-    const int q0 = item.q0, ctx_len = item.ctx_len;
-    const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile: row0 .. row0 + M - 1
-    const int MT = (M + 15) >> 4;
-    const int nslots = kConsumerWarps / MT;
-    const int n_pages = item.page_end - item.page_begin;
-    // The ring is cut into one sub-ring of `depth_s` stages per page slot: page p belongs to slot
-    // p % nslots and is the (p / nslots)-th page of that slot, so a stage is filled and drained by the
-    // same warps in order, which is what the one-bit phase parity of the mbarrier waits needs.
-    const int depth_s = kStages / nslots;
-    const int ring_n = nslots * depth_s;
-
-    const uint32_t full_bar = smem_u32(bars);
-    const uint32_t empty_bar = smem_u32(bars + kStages);
-    if (tid == 0) {
-        abort_s = 0;
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, MT);   // the m-tile warps of the stage's slot
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-
-    if (warp == kConsumerWarps) {
-        // ---------------------------------------------------------------- producer warp
-        // Lanes 0..G-1 each stream pages lane, lane + G, ... on their own, so one lane's issue latency
-        // (block-table read, empty wait, expect_tx, two tile loads) overlaps the others'.  G divides the
-        // number of stages in use: every stage is then always refilled by the same lane, whose waits on
-        // that stage are ordered.
-        int G = kMaxProducerLanes;
-        while (ring_n % G) --G;
-        if (lane < G) {
-            const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
-            int next = lane < n_pages ? bt[lane] : 0;
-            for (int p = lane; p < n_pages; p += G) {
-                int page_id = next;
-                if (p + G < n_pages) next = bt[p + G];
-                const int q = p / nslots, sl = p - q * nslots;   // q-th page of slot sl
-                const int use = q / depth_s, r = q - use * depth_s;
-                const int stage = sl * depth_s + r;
-                bool ok = true;
-                if (use > 0) ok = mbar_wait(empty_bar + 8 * stage, (use - 1) & 1, &abort_s);
-                if (!ok || *(volatile int*)&abort_s) {
-                    if (!ok) atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
-                    *(volatile int*)&abort_s = 1;
-                    break;
-                }
-                if (page_id < 0 || page_id >= a.num_pages) {
-                    atomicExch(a.status, DCUT_DEV_BAD_PAGE);
-                    page_id = 0;
-                }
-                const uint32_t bar = full_bar + 8 * stage;
-                const uint32_t dst = smem_u32(ring + stage * L::kStageBytes);
-                const int row = (page_id * a.n_kv_heads + kvh) * kPage;
-                mbar_arrive_expect_tx(bar, L::kStageBytes);
-                tma_load_tile(dst, &k_map, row, bar);
-                tma_load_tile(dst + L::kPageBytes, &v_map, row, bar);
-            }
-        }
-        return;
-    }
-
-    // -------------------------------------------------------------------- consumer warps
-    // stage the query tile: row R = t * group + hl  <->  q[(q0 + t), kvh * group + hl, :]
-    {
-        constexpr int kChunks = DH / 8;
-        const int rows_padded = MT * 16;
-        for (int idx = tid; idx < rows_padded * kChunks; idx += kConsumerThreads) {
-            const int R = idx / kChunks, c16 = idx - R * kChunks;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (R < M) {
-                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
-                v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * DH + c16 * 8);
-            }
-            *reinterpret_cast<uint4*>(q_s + (R >> 4) * (16 * DH * 2) + tile_off(R & 15, c16)) = v;
-        }
-    }
-    consumer_bar();
-
-    const int mt = warp % MT, slot = warp / MT;
-    const bool active = slot < nslots;
-    float o[DH / 8][4];
-#pragma unroll
-    for (int j = 0; j < DH / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
-    float m_run[2] = {-INFINITY, -INFINITY};
-    float l_run[2] = {0.0f, 0.0f};
-    bool aborted = false;
-
-    if (active) {
-        uint32_t qf[DH / 16][4];
-        {
-            const int mat = lane >> 3;
-            const int r = ((mat & 1) << 3) + (lane & 7);
-            const uint32_t qbase = smem_u32(q_s + mt * (16 * DH * 2));
-#pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) ldmatrix_x4(qbase + tile_off(r, 2 * ks + (mat >> 1)), qf[ks]);
-        }
-        // causal limit per row: query token t sees cache positions j <= ctx_len + t
-        const int R_lo = mt * 16 + (lane >> 2), R_hi = R_lo + 8;
-        const int jmax_lo = ctx_len + (row0 + min(R_lo, M - 1)) / group;
-        const int jmax_hi = ctx_len + (row0 + min(R_hi, M - 1)) / group;
-        // per-lane ldmatrix row/chunk selectors
-        const int kmat = lane >> 3;
-        const int k_tok = ((kmat >> 1) << 3) + (lane & 7);
-        const int k_chunk = kmat & 1;
-        const int v_tok = ((kmat & 1) << 3) + (lane & 7);
-        const int v_chunk = kmat >> 1;
-
-        // this warp's pages: slot, slot + nslots, ... through the slot's own sub-ring
-        const float c_log2 = a.scale_log2;
-        int r_stage = 0, parity = 0;
-        for (int p = slot; p < n_pages; p += nslots) {
-            const int stage = slot * depth_s + r_stage;
-            if (!mbar_wait(full_bar + 8 * stage, parity, &abort_s)) {
-                aborted = true;
-                break;
-            }
-            if (++r_stage == depth_s) {
-                r_stage = 0;
-                parity ^= 1;
-            }
-            const uint32_t k_base = smem_u32(ring + stage * L::kStageBytes);
-            const uint32_t v_base = k_base + L::kPageBytes;
-
-            float s[2][4];
-#pragma unroll
-            for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.0f;
-#pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) {
-                uint32_t kf[4];
-                ldmatrix_x4(k_base + tile_off(k_tok, 2 * ks + k_chunk), kf);
-                mma_bf16(s[0], qf[ks], kf[0], kf[1]);
-                mma_bf16(s[1], qf[ks], kf[2], kf[3]);
-            }
-            // causal mask: only pages that reach past the cached context can hold hidden positions
-            const int j0 = (item.page_begin + p) * kPage + ((lane & 3) << 1);
-            if ((item.page_begin + p) * kPage + kPage - 1 > ctx_len) {
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int j = j0 + nt * 8 + (e & 1);
-                        const int jmax = (e < 2) ? jmax_lo : jmax_hi;
-                        if (j > jmax) s[nt][e] = -INFINITY;
-                    }
-                }
-            }
-            // online softmax for the two rows this thread holds; running max kept on the raw scores,
-            // the softmax scale folded into the exponent: p = 2^(s*c - m*c)
-            float mx[2] = {fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])),
-                           fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]))};
-            float alpha[2], mc[2];
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-                mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-                const float m_new = fmaxf(m_run[r], mx[r]);
-                const float msafe = (m_new == -INFINITY) ? 0.0f : m_new;
-                alpha[r] = fast_exp2((m_run[r] - msafe) * c_log2);
-                mc[r] = msafe * c_log2;
-                m_run[r] = m_new;
-            }
-            float ps[2][4];
-#pragma unroll
-            for (int nt = 0; nt < 2; ++nt) {
-                ps[nt][0] = fast_exp2(fmaf(s[nt][0], c_log2, -mc[0]));
-                ps[nt][1] = fast_exp2(fmaf(s[nt][1], c_log2, -mc[0]));
-                ps[nt][2] = fast_exp2(fmaf(s[nt][2], c_log2, -mc[1]));
-                ps[nt][3] = fast_exp2(fmaf(s[nt][3], c_log2, -mc[1]));
-            }
-            l_run[0] = l_run[0] * alpha[0] + (ps[0][0] + ps[0][1] + ps[1][0] + ps[1][1]);
-            l_run[1] = l_run[1] * alpha[1] + (ps[0][2] + ps[0][3] + ps[1][2] + ps[1][3]);
-            if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
-#pragma unroll
-                for (int j = 0; j < DH / 8; ++j) {
-                    o[j][0] *= alpha[0];
-                    o[j][1] *= alpha[0];
-                    o[j][2] *= alpha[1];
-                    o[j][3] *= alpha[1];
-                }
-            }
-            uint32_t pf[4] = {pack_bf16(ps[0][0], ps[0][1]), pack_bf16(ps[0][2], ps[0][3]),
-                              pack_bf16(ps[1][0], ps[1][1]), pack_bf16(ps[1][2], ps[1][3])};
-#pragma unroll
-            for (int jj = 0; jj < DH / 16; ++jj) {
-                uint32_t vf[4];
-                ldmatrix_x4_trans(v_base + tile_off(v_tok, 2 * jj + v_chunk), vf);
-                mma_bf16(o[2 * jj], pf, vf[0], vf[1]);
-                mma_bf16(o[2 * jj + 1], pf, vf[2], vf[3]);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
-        }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
-        }
-    }
-    if (aborted) {
-        atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
-        *(volatile int*)&abort_s = 1;
-    }
-
-    // -------------------------------------------------------------------- merge the slots
-    consumer_bar();   // every page has been consumed: the ring can be reused
-    float* merge = reinterpret_cast<float*>(ring);
-    if (active) {
-        float* mo = merge + (size_t)warp * 16 * L::kMergeStride;
-        const int r_lo = lane >> 2, c0 = (lane & 3) << 1;
-#pragma unroll
-        for (int j = 0; j < DH / 8; ++j) {
-            *reinterpret_cast<float2*>(mo + r_lo * L::kMergeStride + j * 8 + c0) = make_float2(o[j][0], o[j][1]);
-            *reinterpret_cast<float2*>(mo + (r_lo + 8) * L::kMergeStride + j * 8 + c0) = make_float2(o[j][2], o[j][3]);
-        }
-        if ((lane & 3) == 0) {
-            ml_s[(warp * 16 + r_lo) * 2] = m_run[0];
-            ml_s[(warp * 16 + r_lo) * 2 + 1] = l_run[0];
-            ml_s[(warp * 16 + r_lo + 8) * 2] = m_run[1];
-            ml_s[(warp * 16 + r_lo + 8) * 2 + 1] = l_run[1];
-        }
-    }
-    consumer_bar();
-    if (*(volatile int*)&abort_s) return;
-    {
-        constexpr int kVec = DH / 4;   // float4 per row
-        for (int idx = tid; idx < M * kVec; idx += kConsumerThreads) {
-            const int R = idx / kVec, c4 = idx - R * kVec;
-            const int tile = R >> 4, r = R & 15;
-            float m_all = -INFINITY;
-            for (int sl = 0; sl < nslots; ++sl) m_all = fmaxf(m_all, ml_s[((sl * MT + tile) * 16 + r) * 2]);
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            float l_all = 0.0f;
-            for (int sl = 0; sl < nslots; ++sl) {
-                const int w = sl * MT + tile;
-                const float m_w = ml_s[(w * 16 + r) * 2];
-                const float wgt = (m_w == -INFINITY) ? 0.0f : exp2f((m_w - m_all) * a.scale_log2);
-                l_all += wgt * ml_s[(w * 16 + r) * 2 + 1];
-                const float4 v = *reinterpret_cast<const float4*>(merge + ((size_t)w * 16 + r) * L::kMergeStride + c4 * 4);
-                acc.x += wgt * v.x;
-                acc.y += wgt * v.y;
-                acc.z += wgt * v.z;
-                acc.w += wgt * v.w;
-            }
-            const float inv = l_all > 0.0f ? 1.0f / l_all : 0.0f;
-            acc.x *= inv;
-            acc.y *= inv;
-            acc.z *= inv;
-            acc.w *= inv;
-            const float lse_nat = l_all > 0.0f ? (m_all * a.scale_log2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
-            const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
-            const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
-            if (item.n_chunks == 1) {
-                uint2 pk;
-                pk.x = pack_bf16(acc.x, acc.y);
-                pk.y = pack_bf16(acc.z, acc.w);
-                *reinterpret_cast<uint2*>(a.out + orow * DH + c4 * 4) = pk;
-                if (a.lse && c4 == 0) a.lse[orow] = lse_nat;
-            } else {
-                const size_t prow = (size_t)item.part_row + R;
-                *reinterpret_cast<float4*>(a.part_o + prow * DH + c4 * 4) = acc;
-                if (c4 == 0) a.part_lse[prow] = lse_nat;
-            }
-        }
-    }
-}
-
 
 // ------------------------------------------------------------------------------------------------
 // tcgen05 variant of the split kernel for items with many query rows (head_dim 128, rows <= 128).
@@ -675,10 +366,10 @@ __device__ __forceinline__ void split_item(const CUtensorMap& k_map, const CUten
 constexpr int kTcGroupStages = 6;                  // ring of page groups (192 KB in flight)
 constexpr int kTcSBufs = 3;                        // S/P buffers in tensor memory: groups in flight between QK^T and PV
 constexpr int kTcSoftmaxThreads = 256;             // two threads per row, 32 columns each
-constexpr int kTcThreads = 64 + kTcSoftmaxThreads;
+static_assert(kThreads == 64 + kTcSoftmaxThreads, "roles of the tcgen05 phase");
 constexpr int kTcPageBytes = kPage * 128 * 2;      // 4 KB: one K or V page tile
 constexpr int kTcGroupBytes = 8 * kTcPageBytes;    // K of 4 pages (16 KB, [half][64 rows][64]) + V of 4 pages
-constexpr int kTcSmem = kTcGroupStages * kTcGroupBytes + 1024 + 256;
+constexpr int kTcRingBytes = kTcGroupStages * kTcGroupBytes;
 constexpr int kTcCols = 512;                       // O: 0..127, S/P buffers: 128..319, Q: 320..383
 constexpr int kTcColS = 128, kTcColQ = kTcColS + 64 * kTcSBufs;
 constexpr float kRescaleLog2 = 8.0f;
@@ -754,119 +445,536 @@ __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = kIdescBase | (1u << 16) | ((128u >> 3) << 17);
 
-__device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtensorMap& v_map, const AttnArgs& a,
-                                        const AttnItem& item, unsigned char* smem_raw) {
-    // runs inside a CTA of kThreads threads; only the first kTcThreads take part (CTA-wide syncs count them only)
-    if ((int)threadIdx.x >= kTcThreads) return;
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+// ------------------------------------------------------------------------------------------------
+// persistent item kernel: shared declarations
+
+struct AttnArgs {
+    const __nv_bfloat16* q;
+    const int* block_table;
+    int block_table_stride;
+    const int* ctx_lens;
+    const int* cu_q;
+    const AttnItem* items;
+    int* plan;
+    int n_q_heads, n_kv_heads;
+    long long num_pages;
+    float scale_log2;          // softmax scale * log2(e)
+    __nv_bfloat16* out;
+    float* lse;                // [T, Hq] or null
+    float* part_o;
+    float* part_lse;
+    int* status;
+};
+
+// Control block of a CTA (shared memory, behind the data region).  Every cross-role hand-over goes through an
+// mbarrier with a bounded wait; the two phases of the kernel use separate scheduler barriers.
+struct __align__(16) Ctrl {
+    unsigned long long ring_full[kMmaStages], ring_empty[kMmaStages];   // the tcgen05 phase uses the first kTcGroupStages
+    unsigned long long s_full[kTcSBufs], p_full[kTcSBufs], pv_done[kTcSBufs];
+    unsigned long long q_ready, o_free;
+    unsigned long long sched_full[2][2], sched_empty[2][2];             // [phase][slot]
+    unsigned long long geom_a, geom_b;                                  // ring re-initialisation of the warp-level phase
+    AttnItem item[2];
+    int item_idx[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+#define ABORTED(c) (*(volatile int*)&(c)->abort)
+
+template <int DH>
+struct MmaSmem {
+    static constexpr int kPageBytes = kPage * DH * 2;            // one K or V page tile
+    static constexpr int kStageBytes = 2 * kPageBytes;
+    static constexpr int kRingBytes = kMmaStages * kStageBytes;
+    static constexpr int kQBytes = kMaxMTiles * 16 * DH * 2;
+    static constexpr int kMergeStride = DH + 8;                  // floats per merged row
+    static constexpr int kMergeBytes = kMmaWarps * 16 * kMergeStride * 4;
+    static constexpr int kMergeOrQ = kMergeBytes > kQBytes ? kMergeBytes : kQBytes;   // Q staging reuses the merge buffer
+    static constexpr int kMLBytes = kMmaWarps * 16 * 2 * 4;
+    static constexpr int kTotal = kRingBytes + kMergeOrQ + kMLBytes;
+};
+
+// barrier + OR-reduction over the threads of a named barrier: the result is the same in every thread
+__device__ __forceinline__ bool bar_any(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %3, 0;\n\t"
+        "barrier.cta.red.or.pred q, %1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(id), "r"(nthreads), "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
+// Scheduler, producer side (whole warp, converged): claims the next item of the phase from the global counter and
+// posts it in slot n & 1 of the CTA's queue.  idx = -1 when the phase has no items left.
+__device__ __forceinline__ bool sched_fetch(Ctrl* c, const AttnArgs& a, int phase, int n, int* counter, int end,
+                                            AttnItem& it, int& idx) {
+    const int slot = n & 1, lane = threadIdx.x & 31;
+    if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(smem_u32(&c->sched_empty[phase][slot]), ((n >> 1) - 1) & 1, &c->abort)))
+        return false;
+    int i = 0;
+    if (lane == 0) i = atomicAdd(counter, 1);
+    i = __shfl_sync(0xffffffffu, i, 0);
+    idx = i < end ? i : -1;
+    if (idx >= 0) it = a.items[idx];
+    if (lane == 0) {
+        c->item_idx[slot] = idx;
+        if (idx >= 0) c->item[slot] = it;
+        mbar_arrive(smem_u32(&c->sched_full[phase][slot]));
+    }
+    __syncwarp();
+    return true;
+}
+// consumer side: idx = -2 when the wait gave up
+__device__ __forceinline__ int sched_wait(Ctrl* c, int phase, int n, AttnItem& it) {
+    if (!mbar_wait(smem_u32(&c->sched_full[phase][n & 1]), (n >> 1) & 1, &c->abort)) return -2;
+    const int idx = c->item_idx[n & 1];
+    if (idx >= 0) it = c->item[n & 1];
+    return idx;
+}
+__device__ __forceinline__ void sched_release(Ctrl* c, int phase, int n) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(smem_u32(&c->sched_empty[phase][n & 1]));
+}
+
+// ------------------------------------------------------------------------------------------------
+// warp-level MMA phase (items with few query rows, or any item when head_dim is not 128)
+//
+// kMmaWarps consumer warps + one producer warp.  The ring of page stages is cut into one sub-ring per page slot
+// (nslots = kMmaWarps / m-tiles of the item); pages are numbered through consecutive items, so the producer keeps
+// loading the next item's pages while the consumers still merge the current one.  Only when the number of m-tiles
+// changes between two items is the ring drained and its barriers set up again.
+
+template <int DH>
+__device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnArgs& a,
+                                          unsigned char* smem, Ctrl* c, int* counter, int end) {
+    using L = MmaSmem<DH>;
     unsigned char* ring = smem;
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(ring + kTcGroupStages * kTcGroupBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kTcGroupStages + 3 * kTcSBufs);
-    __shared__ int abort_s;
-    __shared__ float xch[2][2][128];   // [group parity][column half][row]: partial row maxima; [0][h][r] also the final sums
-    const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kTcGroupStages);
-    const uint32_t s_full = smem_u32(bars + 2 * kTcGroupStages), p_full = s_full + 8 * kTcSBufs, pv_done = p_full + 8 * kTcSBufs;
-
+    float* merge = reinterpret_cast<float*>(smem + L::kRingBytes);
+    unsigned char* q_s = smem + L::kRingBytes;
+    float* ml_s = reinterpret_cast<float*>(smem + L::kRingBytes + L::kMergeOrQ);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int req = item.req, kvh = item.kv_head;
     const int group = a.n_q_heads / a.n_kv_heads;
-    const int q0 = item.q0, ctx_len = item.ctx_len;
-    const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile
-    const int n_pages = item.page_end - item.page_begin;
-    const int n_groups = (n_pages + 3) >> 2;
+    const uint32_t full_bar = smem_u32(c->ring_full), empty_bar = smem_u32(c->ring_empty);
+    const uint32_t geom_a = smem_u32(&c->geom_a), geom_b = smem_u32(&c->geom_b);
+    constexpr int kPhase = 1;
 
-    if (tid == 0) {
-        abort_s = 0;
-        for (int s = 0; s < kTcGroupStages; ++s) {
-            mbar_init(full_bar + 8 * s, 4);          // one arrival per page slot of the group
-            mbar_init(empty_bar + 8 * s, 1);
-        }
-        for (int b = 0; b < kTcSBufs; ++b) {
-            mbar_init(s_full + 8 * b, 1);
-            mbar_init(p_full + 8 * b, kTcSoftmaxThreads);
-            mbar_init(pv_done + 8 * b, 1);
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTcCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    asm volatile("bar.sync 0, %0;" ::"n"(kTcThreads) : "memory");
-    tc_fence_after();
-    const uint32_t tmem_o = *tmem_slot;
+    if (warp > kMmaWarps) return;               // spare warps of the CTA
+
+    AttnItem item;
+    int cur_mt = -1, n_geom = 0;
+    long long P0 = 0;                           // pages of the earlier items since the ring was last set up
     bool failed = false;
+
+    if (warp == kMmaWarps) {
+        // ---------------------------------------------------------------- producer warp
+        for (int n = 0;; ++n) {
+            int idx;
+            if (!sched_fetch(c, a, kPhase, n, counter, end, item, idx)) {
+                failed = true;
+                break;
+            }
+            if (idx < 0) break;
+            const int MT = (item.pad[2] + 15) >> 4;
+            const int nslots = kMmaWarps / MT, depth_s = kMmaStages / nslots, ring_n = nslots * depth_s;
+            if (MT != cur_mt) {
+                // every consumer has finished the previous item (nothing of this one is in flight yet)
+                if (lane == 0) mbar_arrive(geom_a);
+                if (!__all_sync(0xffffffffu, mbar_wait(geom_b, n_geom & 1, &c->abort))) {
+                    failed = true;
+                    break;
+                }
+                ++n_geom;
+                cur_mt = MT;
+                P0 = 0;
+            }
+            const int n_pages = item.page_end - item.page_begin;
+            int G = kMaxProducerLanes;
+            while (ring_n % G) --G;
+            if (lane < G) {
+                // lane l issues the pages whose running number is l modulo G: a stage is always refilled by the
+                // same lane, whose waits on it are therefore ordered
+                const int* bt = a.block_table + (size_t)item.req * a.block_table_stride + item.page_begin;
+                int p = (int)(((long long)lane - P0 % G + G) % G);
+                int next = p < n_pages ? bt[p] : 0;
+                for (; p < n_pages; p += G) {
+                    int page_id = next;
+                    if (p + G < n_pages) next = bt[p + G];
+                    const long long P = P0 + p;
+                    const int in_ring = (int)(P % ring_n);
+                    const long long use = P / ring_n;
+                    const int sl = in_ring % nslots, r = in_ring / nslots;   // r-th stage of slot sl
+                    const int stage = sl * depth_s + r;
+                    if (use > 0 && !mbar_wait(empty_bar + 8 * stage, (uint32_t)((use - 1) & 1), &c->abort)) {
+                        failed = true;
+                        break;
+                    }
+                    if (page_id < 0 || page_id >= a.num_pages) {
+                        atomicExch(a.status, DCUT_DEV_BAD_PAGE);
+                        page_id = 0;
+                    }
+                    const uint32_t bar = full_bar + 8 * stage;
+                    const uint32_t dst = smem_u32(ring + stage * L::kStageBytes);
+                    const int row = (page_id * a.n_kv_heads + item.kv_head) * kPage;
+                    mbar_arrive_expect_tx(bar, L::kStageBytes);
+                    tma_load_tile(dst, &k_map, row, bar);
+                    tma_load_tile(dst + L::kPageBytes, &v_map, row, bar);
+                }
+            }
+            __syncwarp();
+            if (__any_sync(0xffffffffu, failed) || c->abort) {
+                failed = true;
+                break;
+            }
+            P0 += n_pages;
+        }
+        if (failed) {
+            atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
+            c->abort = 1;
+        }
+        return;
+    }
+
+    // -------------------------------------------------------------------- consumer warps
+    int r_stage = 0, parity = 0;                // position of this warp in its slot's sub-ring
+    for (int n = 0;; ++n) {
+        const int idx = sched_wait(c, kPhase, n, item);
+        if (idx == -2) failed = true;
+        if (bar_any(1, kMmaThreads, failed || c->abort)) break;   // also: the previous merge has been read by everyone
+        if (idx < 0) break;
+        const int q0 = item.q0, ctx_len = item.ctx_len, kvh = item.kv_head;
+        const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile
+        const int MT = (M + 15) >> 4;
+        const int nslots = kMmaWarps / MT, depth_s = kMmaStages / nslots;
+        const int n_pages = item.page_end - item.page_begin;
+        if (MT != cur_mt) {
+            // set the ring up for this number of m-tiles; the producer waits for it before it loads anything
+            __syncwarp();
+            if (lane == 0) mbar_arrive(geom_a);
+            if (tid == 0) {
+                if (mbar_wait(geom_a, n_geom & 1, &c->abort)) {
+                    for (int s = 0; s < kMmaStages; ++s) {
+                        asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(full_bar + 8 * s) : "memory");
+                        asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(empty_bar + 8 * s) : "memory");
+                        mbar_init(full_bar + 8 * s, 1);
+                        mbar_init(empty_bar + 8 * s, MT);   // the m-tile warps of the stage's slot
+                    }
+                    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    mbar_arrive(geom_b);
+                } else {
+                    c->abort = 1;
+                }
+            }
+            if (!mbar_wait(geom_b, n_geom & 1, &c->abort)) failed = true;
+            ++n_geom;
+            cur_mt = MT;
+            P0 = 0;
+            r_stage = 0;
+            parity = 0;
+        }
+        // stage the query tile: row R = t * group + hl  <->  q[(q0 + t), kvh * group + hl, :]
+        {
+            constexpr int kChunks = DH / 8;
+            const int rows_padded = MT * 16;
+            for (int i = tid; i < rows_padded * kChunks; i += kMmaThreads) {
+                const int R = i / kChunks, c16 = i - R * kChunks;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (R < M) {
+                    const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
+                    v = *reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * DH + c16 * 8);
+                }
+                *reinterpret_cast<uint4*>(q_s + (R >> 4) * (16 * DH * 2) + tile_off(R & 15, c16)) = v;
+            }
+        }
+        if (bar_any(1, kMmaThreads, failed)) break;
+
+        const int mt = warp % MT, slot = warp / MT;
+        const bool active = slot < nslots;
+        float o[DH / 8][4];
+#pragma unroll
+        for (int j = 0; j < DH / 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
+        float m_run[2] = {-INFINITY, -INFINITY};
+        float l_run[2] = {0.0f, 0.0f};
+
+        if (active) {
+            uint32_t qf[DH / 16][4];
+            {
+                const int mat = lane >> 3;
+                const int r = ((mat & 1) << 3) + (lane & 7);
+                const uint32_t qbase = smem_u32(q_s + mt * (16 * DH * 2));
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) ldmatrix_x4(qbase + tile_off(r, 2 * ks + (mat >> 1)), qf[ks]);
+            }
+            // causal limit per row: query token t sees cache positions j <= ctx_len + t
+            const int R_lo = mt * 16 + (lane >> 2), R_hi = R_lo + 8;
+            const int jmax_lo = ctx_len + (row0 + min(R_lo, M - 1)) / group;
+            const int jmax_hi = ctx_len + (row0 + min(R_hi, M - 1)) / group;
+            // per-lane ldmatrix row/chunk selectors
+            const int kmat = lane >> 3;
+            const int k_tok = ((kmat >> 1) << 3) + (lane & 7);
+            const int k_chunk = kmat & 1;
+            const int v_tok = ((kmat & 1) << 3) + (lane & 7);
+            const int v_chunk = kmat >> 1;
+
+            // this warp's pages of the item: running number = slot modulo nslots, in order through the slot's sub-ring
+            const float c_log2 = a.scale_log2;
+            for (int p = (int)(((long long)slot - P0 % nslots + nslots) % nslots); p < n_pages; p += nslots) {
+                const int stage = slot * depth_s + r_stage;
+                if (!mbar_wait(full_bar + 8 * stage, parity, &c->abort)) {
+                    failed = true;
+                    break;
+                }
+                if (++r_stage == depth_s) {
+                    r_stage = 0;
+                    parity ^= 1;
+                }
+                const uint32_t k_base = smem_u32(ring + stage * L::kStageBytes);
+                const uint32_t v_base = k_base + L::kPageBytes;
+
+                float s[2][4];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.0f;
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks) {
+                    uint32_t kf[4];
+                    ldmatrix_x4(k_base + tile_off(k_tok, 2 * ks + k_chunk), kf);
+                    mma_bf16(s[0], qf[ks], kf[0], kf[1]);
+                    mma_bf16(s[1], qf[ks], kf[2], kf[3]);
+                }
+                // causal mask: only pages that reach past the cached context can hold hidden positions
+                const int j0 = (item.page_begin + p) * kPage + ((lane & 3) << 1);
+                if ((item.page_begin + p) * kPage + kPage - 1 > ctx_len) {
+#pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int j = j0 + nt * 8 + (e & 1);
+                            const int jmax = (e < 2) ? jmax_lo : jmax_hi;
+                            if (j > jmax) s[nt][e] = -INFINITY;
+                        }
+                    }
+                }
+                // online softmax for the two rows this thread holds; running max kept on the raw scores,
+                // the softmax scale folded into the exponent: p = 2^(s*c - m*c)
+                float mx[2] = {fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])),
+                               fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]))};
+                float alpha[2], mc[2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                    mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+                    const float m_new = fmaxf(m_run[r], mx[r]);
+                    const float msafe = (m_new == -INFINITY) ? 0.0f : m_new;
+                    alpha[r] = fast_exp2((m_run[r] - msafe) * c_log2);
+                    mc[r] = msafe * c_log2;
+                    m_run[r] = m_new;
+                }
+                float ps[2][4];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) {
+                    ps[nt][0] = fast_exp2(fmaf(s[nt][0], c_log2, -mc[0]));
+                    ps[nt][1] = fast_exp2(fmaf(s[nt][1], c_log2, -mc[0]));
+                    ps[nt][2] = fast_exp2(fmaf(s[nt][2], c_log2, -mc[1]));
+                    ps[nt][3] = fast_exp2(fmaf(s[nt][3], c_log2, -mc[1]));
+                }
+                l_run[0] = l_run[0] * alpha[0] + (ps[0][0] + ps[0][1] + ps[1][0] + ps[1][1]);
+                l_run[1] = l_run[1] * alpha[1] + (ps[0][2] + ps[0][3] + ps[1][2] + ps[1][3]);
+                if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
+#pragma unroll
+                    for (int j = 0; j < DH / 8; ++j) {
+                        o[j][0] *= alpha[0];
+                        o[j][1] *= alpha[0];
+                        o[j][2] *= alpha[1];
+                        o[j][3] *= alpha[1];
+                    }
+                }
+                uint32_t pf[4] = {pack_bf16(ps[0][0], ps[0][1]), pack_bf16(ps[0][2], ps[0][3]),
+                                  pack_bf16(ps[1][0], ps[1][1]), pack_bf16(ps[1][2], ps[1][3])};
+#pragma unroll
+                for (int jj = 0; jj < DH / 16; ++jj) {
+                    uint32_t vf[4];
+                    ldmatrix_x4_trans(v_base + tile_off(v_tok, 2 * jj + v_chunk), vf);
+                    mma_bf16(o[2 * jj], pf, vf[0], vf[1]);
+                    mma_bf16(o[2 * jj + 1], pf, vf[2], vf[3]);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar + 8 * stage);
+            }
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+                l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+            }
+        }
+        if (failed) c->abort = 1;
+        P0 += n_pages;
+
+        // ---------------------------------------------------------------- merge the slots
+        // (the merge buffer is not part of the ring: the producer is already loading the next item)
+        if (active) {
+            float* mo = merge + (size_t)warp * 16 * L::kMergeStride;
+            const int r_lo = lane >> 2, c0 = (lane & 3) << 1;
+#pragma unroll
+            for (int j = 0; j < DH / 8; ++j) {
+                *reinterpret_cast<float2*>(mo + r_lo * L::kMergeStride + j * 8 + c0) = make_float2(o[j][0], o[j][1]);
+                *reinterpret_cast<float2*>(mo + (r_lo + 8) * L::kMergeStride + j * 8 + c0) = make_float2(o[j][2], o[j][3]);
+            }
+            if ((lane & 3) == 0) {
+                ml_s[(warp * 16 + r_lo) * 2] = m_run[0];
+                ml_s[(warp * 16 + r_lo) * 2 + 1] = l_run[0];
+                ml_s[(warp * 16 + r_lo + 8) * 2] = m_run[1];
+                ml_s[(warp * 16 + r_lo + 8) * 2 + 1] = l_run[1];
+            }
+        }
+        if (bar_any(1, kMmaThreads, failed || ABORTED(c))) break;
+        {
+            constexpr int kVec = DH / 4;   // float4 per row
+            for (int i = tid; i < M * kVec; i += kMmaThreads) {
+                const int R = i / kVec, c4 = i - R * kVec;
+                const int tile = R >> 4, r = R & 15;
+                float m_all = -INFINITY;
+                for (int sl = 0; sl < nslots; ++sl) m_all = fmaxf(m_all, ml_s[((sl * MT + tile) * 16 + r) * 2]);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float l_all = 0.0f;
+                for (int sl = 0; sl < nslots; ++sl) {
+                    const int w = sl * MT + tile;
+                    const float m_w = ml_s[(w * 16 + r) * 2];
+                    const float wgt = (m_w == -INFINITY) ? 0.0f : exp2f((m_w - m_all) * a.scale_log2);
+                    l_all += wgt * ml_s[(w * 16 + r) * 2 + 1];
+                    const float4 v = *reinterpret_cast<const float4*>(merge + ((size_t)w * 16 + r) * L::kMergeStride + c4 * 4);
+                    acc.x += wgt * v.x;
+                    acc.y += wgt * v.y;
+                    acc.z += wgt * v.z;
+                    acc.w += wgt * v.w;
+                }
+                const float inv = l_all > 0.0f ? 1.0f / l_all : 0.0f;
+                acc.x *= inv;
+                acc.y *= inv;
+                acc.z *= inv;
+                acc.w *= inv;
+                const float lse_nat = l_all > 0.0f ? (m_all * a.scale_log2 + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
+                const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+                if (item.n_chunks == 1) {
+                    uint2 pk;
+                    pk.x = pack_bf16(acc.x, acc.y);
+                    pk.y = pack_bf16(acc.z, acc.w);
+                    *reinterpret_cast<uint2*>(a.out + orow * DH + c4 * 4) = pk;
+                    if (a.lse && c4 == 0) a.lse[orow] = lse_nat;
+                } else {
+                    const size_t prow = (size_t)item.part_row + R;
+                    *reinterpret_cast<float4*>(a.part_o + prow * DH + c4 * 4) = acc;
+                    if (c4 == 0) a.part_lse[prow] = lse_nat;
+                }
+            }
+        }
+        sched_release(c, kPhase, n);
+    }
+    if (failed) {
+        atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
+        c->abort = 1;
+    }
+}
+
+// One persistent pass over the tcgen05-path items of this CTA.  Ring stages, S/P buffers and their barriers are
+// numbered through consecutive items (running group number), so the producer streams the next item's pages while the
+// current item is still being finished; only Q and O (single-buffered in tensor memory) serialise at an item boundary,
+// through the q_ready and o_free barriers.
+__device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtensorMap& v_map, const AttnArgs& a,
+                                         unsigned char* ring, Ctrl* c, float (*xch)[2][128], float (*xl)[128],
+                                         int* counter, int end) {
+    constexpr int kPhase = 0;
+    const uint32_t full_bar = smem_u32(c->ring_full), empty_bar = smem_u32(c->ring_empty);
+    const uint32_t s_full = smem_u32(c->s_full), p_full = smem_u32(c->p_full), pv_done = smem_u32(c->pv_done);
+    const uint32_t q_ready = smem_u32(&c->q_ready), o_free = smem_u32(&c->o_free);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int group = a.n_q_heads / a.n_kv_heads;
+    const uint32_t tmem_o = c->tmem_base;
+    AttnItem item;
+    bool failed = false;
+    int G0 = 0;                                  // groups of the earlier items: running group number = G0 + g
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
-        // lane l loads page l of every group; the group's full barrier takes four arrivals, so a lane whose
-        // page does not exist (last group) still arrives, without bytes
-        if (lane < 4) {
-            const int* bt = a.block_table + (size_t)req * a.block_table_stride + item.page_begin;
-            int next = lane < n_pages ? bt[lane] : 0;
+        // The whole warp walks the groups; lanes 0-3 look up the group's four pages one group ahead, and one elected
+        // lane issues all of the group's tile loads (uniform operands: a divergent lane needs about twice as long per
+        // load, which made the producer the slowest role).
+        for (int n = 0;; ++n) {
+            int idx;
+            if (!sched_fetch(c, a, kPhase, n, counter, end, item, idx)) {
+                failed = true;
+                break;
+            }
+            if (idx < 0) break;
+            const int n_pages = item.page_end - item.page_begin;
+            const int n_groups = (n_pages + 3) >> 2;
+            const int* bt = a.block_table + (size_t)item.req * a.block_table_stride + item.page_begin;
+            int next = (lane < 4 && lane < n_pages) ? bt[lane] : 0;
             TCP(long long t_we = 0; long long t_all = clock64();)
             for (int g = 0; g < n_groups; ++g) {
-                const int p = 4 * g + lane;
                 int page_id = next;
-                if (p + 4 < n_pages) next = bt[p + 4];
-                const int gs = g % kTcGroupStages, use = g / kTcGroupStages;
+                const int pn = 4 * (g + 1) + lane;
+                if (lane < 4 && pn < n_pages) next = bt[pn];
+                const int gc = G0 + g, gs = gc % kTcGroupStages, use = gc / kTcGroupStages;
                 TCP(long long c0 = clock64();)
-                if ((use > 0 && !mbar_wait(empty_bar + 8 * gs, (use - 1) & 1, &abort_s)) || *(volatile int*)&abort_s) {
+                if (use > 0 && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * gs, (use - 1) & 1, &c->abort))) {
                     failed = true;
                     break;
                 }
                 TCP(t_we += clock64() - c0;)
-                const uint32_t bar = full_bar + 8 * gs;
-                if (p >= n_pages) {
-                    mbar_arrive(bar);
-                    continue;
-                }
-                if (page_id < 0 || page_id >= a.num_pages) {
+                const int np = min(4, n_pages - 4 * g);
+                if (lane < np && (page_id < 0 || page_id >= a.num_pages)) {
                     atomicExch(a.status, DCUT_DEV_BAD_PAGE);
                     page_id = 0;
                 }
-                const uint32_t dst = smem_u32(ring + gs * kTcGroupBytes);
-                const int row = (page_id * a.n_kv_heads + kvh) * kPage;
-                mbar_arrive_expect_tx(bar, 2 * kTcPageBytes);
-                tma_load_2d(dst + lane * 2048, &k2_map, 0, row, bar);            // K columns 0..63 of the page
-                tma_load_2d(dst + 8192 + lane * 2048, &k2_map, 64, row, bar);    // K columns 64..127
-                tma_load_tile(dst + 4 * kTcPageBytes + lane * kTcPageBytes, &v_map, row, bar);
+                const int row = (page_id * a.n_kv_heads + item.kv_head) * kPage;
+                const int r0 = __shfl_sync(0xffffffffu, row, 0), r1 = __shfl_sync(0xffffffffu, row, 1);
+                const int r2 = __shfl_sync(0xffffffffu, row, 2), r3 = __shfl_sync(0xffffffffu, row, 3);
+                if (elect_one()) {
+                    const uint32_t bar = full_bar + 8 * gs;
+                    const uint32_t dst = smem_u32(ring + gs * kTcGroupBytes);
+                    mbar_arrive_expect_tx(bar, (uint32_t)np * 2 * kTcPageBytes);
+                    const int rows[4] = {r0, r1, r2, r3};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        if (j < np) {
+                            tma_load_2d(dst + j * 2048, &k2_map, 0, rows[j], bar);            // K columns 0..63 of page j
+                            tma_load_2d(dst + 8192 + j * 2048, &k2_map, 64, rows[j], bar);    // K columns 64..127
+                            tma_load_tile(dst + 4 * kTcPageBytes + j * kTcPageBytes, &v_map, rows[j], bar);
+                        }
+                }
+                __syncwarp();
             }
             TCP(if (blockIdx.x == 0 && lane == 0) printf("producer: groups %d total %lld wait_empty %lld\n", n_groups, clock64() - t_all, t_we);)
-        }
-    } else {
-        const uint32_t tmem_q = tmem_o + kTcColQ;
-        const int quarter = warp & 3, half = (warp - 2) >> 2;     // softmax warps: lane quarter of tensor memory, column half
-        if (warp >= 2) {
-            // the query tile goes to tensor memory: row R = lane of tensor memory, 128 bf16 = 64 words, 32 per thread
-            const int R = quarter * 32 + lane;
-            uint32_t qw[32];
-            if (R < M) {
-                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
-                const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * half;
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const uint4 v = src[c];
-                    qw[4 * c] = v.x; qw[4 * c + 1] = v.y; qw[4 * c + 2] = v.z; qw[4 * c + 3] = v.w;
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) qw[c] = 0;
+            if (failed || ABORTED(c)) {
+                failed = true;
+                break;
             }
-            tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * half, qw);
-            tc_wait_st();
-            tc_fence_before();
+            G0 += n_groups;
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(32 + kTcSoftmaxThreads) : "memory");   // MMA warp + softmax warps
-        if (warp == 1) {
-            // ---------------------------------------------------------------- MMA issuer
-            // The whole warp walks the schedule and waits on the barriers; one elected lane issues.
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        // The whole warp walks the schedule and waits on the barriers; one elected lane issues.
+        const uint32_t tmem_q = tmem_o + kTcColQ;
+        for (int n = 0; !failed; ++n) {
+            const int idx = sched_wait(c, kPhase, n, item);
+            if (idx == -2) failed = true;
+            if (__any_sync(0xffffffffu, failed) || idx < 0) break;
+            const int n_pages = item.page_end - item.page_begin;
+            const int n_groups = (n_pages + 3) >> 2;
+            // this item's query tile is in tensor memory
+            if (!__all_sync(0xffffffffu, mbar_wait(q_ready, n & 1, &c->abort))) {
+                failed = true;
+                break;
+            }
             tc_fence_after();
             auto issue_qk = [&](int g) -> bool {
-                const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages, b = g % kTcSBufs;
-                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * gs, (g / kTcGroupStages) & 1, &abort_s))) return false;
+                const int gc = G0 + g;
+                const int np = min(4, n_pages - 4 * g), gs = gc % kTcGroupStages, b = gc % kTcSBufs;
+                // the S/P buffer was last used by the running group gc - kTcSBufs
+                if (gc >= kTcSBufs && !__all_sync(0xffffffffu, mbar_wait(pv_done + 8 * b, ((gc / kTcSBufs) - 1) & 1, &c->abort))) return false;
+                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * gs, (gc / kTcGroupStages) & 1, &c->abort))) return false;
                 tc_fence_after();
                 if (elect_one()) {
                     const uint32_t k_addr = smem_u32(ring + gs * kTcGroupBytes);
@@ -889,16 +997,14 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
             for (int g = 0; ok && g < kTcSBufs - 1 && g < n_groups; ++g) ok = issue_qk(g);
             for (int g = 0; ok && g < n_groups; ++g) {
                 const int ga = g + kTcSBufs - 1;
-                if (ga < n_groups) {
-                    // its S/P buffer was last used by group g-1
-                    if (g >= 1 && !__all_sync(0xffffffffu, mbar_wait(pv_done + 8 * (ga % kTcSBufs), ((g - 1) / kTcSBufs) & 1, &abort_s))) { ok = false; break; }
-                    if (!issue_qk(ga)) { ok = false; break; }
-                }
-                const int b = g % kTcSBufs;
-                if (!__all_sync(0xffffffffu, mbar_wait(p_full + 8 * b, (g / kTcSBufs) & 1, &abort_s))) { ok = false; break; }
+                if (ga < n_groups && !issue_qk(ga)) { ok = false; break; }
+                const int gc = G0 + g, b = gc % kTcSBufs;
+                if (!__all_sync(0xffffffffu, mbar_wait(p_full + 8 * b, (gc / kTcSBufs) & 1, &c->abort))) { ok = false; break; }
+                // the first PV of an item overwrites O: the previous item's epilogue must have read it
+                if (g == 0 && n > 0 && !__all_sync(0xffffffffu, mbar_wait(o_free, (n - 1) & 1, &c->abort))) { ok = false; break; }
                 tc_fence_after();
                 if (elect_one()) {
-                    const int np = min(4, n_pages - 4 * g), gs = g % kTcGroupStages;
+                    const int np = min(4, n_pages - 4 * g), gs = gc % kTcGroupStages;
                     const uint32_t tmem_p = tmem_o + kTcColS + 64 * b;
                     const uint64_t dv = desc_mnmajor(smem_u32(ring + gs * kTcGroupBytes) + 4 * kTcPageBytes);
                     if (np == 4) {
@@ -914,22 +1020,63 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
                 }
                 __syncwarp();
             }
-            if (!ok) failed = true;
-        } else {
-            // ---------------------------------------------------------------- softmax + epilogue
-            // row R = tensor-memory lane; this thread owns columns [32 * half, 32 * half + 32) of every S tile
-            const int R = quarter * 32 + lane;
-            const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
+            if (!ok) {
+                failed = true;
+                break;
+            }
+            sched_release(c, kPhase, n);
+            G0 += n_groups;
+        }
+    } else if (warp < 2 + kTcSoftmaxThreads / 32) {
+        // ---------------------------------------------------------------- softmax + epilogue
+        // row R = tensor-memory lane; this thread owns columns [32 * half, 32 * half + 32) of every S tile.
+        // The two threads of a row meet at a named barrier every group, so a thread whose wait has given up keeps
+        // walking (skipping the tensor-memory work) until a point where both leave together.
+        const uint32_t tmem_q = tmem_o + kTcColQ;
+        const int quarter = warp & 3, half = (warp - 2) >> 2;     // lane quarter of tensor memory, column half
+        const int R = quarter * 32 + lane;
+        const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
+        const float cs = a.scale_log2;
+        for (int n = 0;; ++n) {
+            const int idx = sched_wait(c, kPhase, n, item);
+            if (idx == -2) failed = true;
+            if (bar_any(2 + quarter, 64, failed || ABORTED(c))) {
+                failed = true;
+                break;
+            }
+            if (idx < 0) break;
+            const int q0 = item.q0, ctx_len = item.ctx_len, kvh = item.kv_head;
+            const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile
+            const int n_pages = item.page_end - item.page_begin;
+            const int n_groups = (n_pages + 3) >> 2;
+            {
+                // the query tile goes to tensor memory (every QK^T of the previous item has completed: its last
+                // s_full was seen): row R = lane of tensor memory, 128 bf16 = 64 words, 32 per thread
+                uint32_t qw[32];
+                if (R < M) {
+                    const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
+                    const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * half;
+#pragma unroll
+                    for (int cc = 0; cc < 8; ++cc) {
+                        const uint4 v = src[cc];
+                        qw[4 * cc] = v.x; qw[4 * cc + 1] = v.y; qw[4 * cc + 2] = v.z; qw[4 * cc + 3] = v.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int cc = 0; cc < 32; ++cc) qw[cc] = 0;
+                }
+                tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * half, qw);
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(q_ready);
+            }
             const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
-            const float c = a.scale_log2;
             float m_run = -INFINITY, l_run = 0.0f;
-            // A failed wait never leaves the loop early: the two threads of a row meet at a named barrier every group,
-            // so a thread that has given up keeps walking (skipping the tensor-memory work) until the loop ends.
             TCP(long long t_ws = 0, t_wk = 0, t_bar = 0;)
             for (int g = 0; g < n_groups; ++g) {
-                const int b = g % kTcSBufs;
+                const int gc = G0 + g, b = gc % kTcSBufs;
                 TCP(long long c0 = clock64();)
-                if (!failed && !mbar_wait(s_full + 8 * b, (g / kTcSBufs) & 1, &abort_s)) failed = true;
+                if (!failed && !mbar_wait(s_full + 8 * b, (gc / kTcSBufs) & 1, &c->abort)) failed = true;
                 failed = __any_sync(0xffffffffu, failed);
                 TCP(long long c1 = clock64(); t_ws += c1 - c0;)
                 const uint32_t t_s = t_lane + kTcColS + 64 * b;
@@ -956,23 +1103,23 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
                 }
                 // the two threads of a row exchange their partial maxima
                 float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                xch[g & 1][half][R] = mx;
+                xch[gc & 1][half][R] = mx;
                 TCP(long long c4 = clock64();)
                 asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
                 TCP(t_bar += clock64() - c4;)
-                mx = fmaxf(mx, xch[g & 1][half ^ 1][R]);
+                mx = fmaxf(mx, xch[gc & 1][half ^ 1][R]);
                 // the running maximum only moves (and O is only rescaled) when it would grow by more than 2^8
                 float alpha = 1.0f;
                 bool moved = false;
-                if (!failed && mx > m_run && (m_run == -INFINITY || (mx - m_run) * c > kRescaleLog2)) {
-                    alpha = fast_exp2((m_run - mx) * c);                  // 0 when nothing was visible before
+                if (!failed && mx > m_run && (m_run == -INFINITY || (mx - m_run) * cs > kRescaleLog2)) {
+                    alpha = fast_exp2((m_run - mx) * cs);                 // 0 when nothing was visible before
                     m_run = mx;
                     l_run *= alpha;
                     moved = g > 0;
                 }
                 if (g > 0 && __any_sync(0xffffffffu, moved)) {
                     // O is being updated by the previous group's MMAs: wait for them, then scale this thread's half row
-                    if (!mbar_wait(pv_done + 8 * ((g - 1) % kTcSBufs), ((g - 1) / kTcSBufs) & 1, &abort_s)) failed = true;
+                    if (!mbar_wait(pv_done + 8 * ((gc - 1) % kTcSBufs), ((gc - 1) / kTcSBufs) & 1, &c->abort)) failed = true;
                     failed = __any_sync(0xffffffffu, failed);
                     if (!failed) {
                         tc_fence_after();
@@ -989,13 +1136,13 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
                     }
                 }
                 if (!failed) {
-                    const float mc = (m_run == -INFINITY ? 0.0f : m_run) * c;
+                    const float mc = (m_run == -INFINITY ? 0.0f : m_run) * cs;
                     float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                     uint32_t pw[16];
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), c, -mc));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), c, -mc));
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), cs, -mc));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), cs, -mc));
                         sum4[e & 3] += p0 + p1;
                         pw[e] = pack_bf16(p0, p1);
                     }
@@ -1009,84 +1156,139 @@ __device__ __forceinline__ void tc_item(const CUtensorMap& k2_map, const CUtenso
             }
             TCP(if (blockIdx.x == 0 && R == 0) printf("softmax half %d: wait_s %lld work %lld (pair barrier %lld)\n", half, t_ws, t_wk, t_bar);)
             // epilogue: the item's O row, normalised; this thread writes columns [64 * half, 64 * half + 64)
-            if (!failed && !mbar_wait(pv_done + 8 * ((n_groups - 1) % kTcSBufs), ((n_groups - 1) / kTcSBufs) & 1, &abort_s)) failed = true;
+            const int gl = G0 + n_groups - 1;
+            if (!failed && !mbar_wait(pv_done + 8 * (gl % kTcSBufs), (gl / kTcSBufs) & 1, &c->abort)) failed = true;
             failed = __any_sync(0xffffffffu, failed);
             tc_fence_after();
-            asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");   // every exchange read of the last group is done
-            xch[0][half][R] = l_run;
-            asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
-            l_run += xch[0][half ^ 1][R];
-            if (!failed) {
-                const float inv = l_run > 0.0f ? 1.0f / l_run : 0.0f;
-                const float lse_nat = l_run > 0.0f ? (m_run * c + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
-                const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
-                const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
-#pragma unroll 1
-                for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
-                    uint32_t o[32];
-                    tc_ld32(t_lane + cc, o);
-                    tc_wait_ld();
-                    if (R < M) {
-                        if (item.n_chunks == 1) {
+            xl[half][R] = l_run;
+            if (failed) c->abort = 1;
+            if (bar_any(2 + quarter, 64, failed)) {
+                failed = true;
+                break;
+            }
+            l_run += xl[half ^ 1][R];
+            const float inv = l_run > 0.0f ? 1.0f / l_run : 0.0f;
+            const float lse_nat = l_run > 0.0f ? (m_run * cs + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
+            const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+            uint32_t o0[32], o1[32];
+            tc_ld32(t_lane + 64 * half, o0);
+            tc_ld32(t_lane + 64 * half + 32, o1);
+            tc_wait_ld();
+            tc_fence_before();
+            mbar_arrive(o_free);                                            // O may be overwritten by the next item
 #pragma unroll
-                            for (int e = 0; e < 32; e += 8) {
-                                uint32_t w[4];
-#pragma unroll
-                                for (int j = 0; j < 4; ++j)
-                                    w[j] = pack_bf16(__uint_as_float(o[e + 2 * j]) * inv, __uint_as_float(o[e + 2 * j + 1]) * inv);
-                                *reinterpret_cast<uint4*>(a.out + orow * 128 + cc + e) = make_uint4(w[0], w[1], w[2], w[3]);
-                            }
-                        } else {
-                            float* po = a.part_o + ((size_t)item.part_row + R) * 128 + cc;
-#pragma unroll
-                            for (int e = 0; e < 32; e += 4)
-                                *reinterpret_cast<float4*>(po + e) =
-                                    make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
-                                                __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-                        }
-                    }
-                }
-                if (R < M && half == 0) {
+            for (int hh = 0; hh < 2; ++hh) {
+                const uint32_t* o = hh ? o1 : o0;
+                const int cc = 64 * half + 32 * hh;
+                if (R < M) {
                     if (item.n_chunks == 1) {
-                        if (a.lse) a.lse[orow] = lse_nat;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                w[j] = pack_bf16(__uint_as_float(o[e + 2 * j]) * inv, __uint_as_float(o[e + 2 * j + 1]) * inv);
+                            *reinterpret_cast<uint4*>(a.out + orow * 128 + cc + e) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
                     } else {
-                        a.part_lse[(size_t)item.part_row + R] = lse_nat;
+                        float* po = a.part_o + ((size_t)item.part_row + R) * 128 + cc;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<float4*>(po + e) =
+                                make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
+                                            __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
                     }
                 }
             }
+            if (R < M && half == 0) {
+                if (item.n_chunks == 1) {
+                    if (a.lse) a.lse[orow] = lse_nat;
+                } else {
+                    a.part_lse[(size_t)item.part_row + R] = lse_nat;
+                }
+            }
+            sched_release(c, kPhase, n);
+            G0 += n_groups;
         }
     }
     if (failed) {
         atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
-        *(volatile int*)&abort_s = 1;
-    }
-    tc_fence_before();
-    asm volatile("bar.sync 0, %0;" ::"n"(kTcThreads) : "memory");
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_o), "n"(kTcCols) : "memory");
+        c->abort = 1;
     }
 }
 
-// One CTA per work item; the item says which of the two paths takes it.
+
+template <int DH>
+constexpr int kDataBytes = (DH == 128 && kTcRingBytes > MmaSmem<DH>::kTotal) ? kTcRingBytes : MmaSmem<DH>::kTotal;
+template <int DH>
+constexpr int kSmemBytes = kDataBytes<DH> + 1024 /* alignment slack */ + 1024 /* control block */;
+static_assert(sizeof(Ctrl) <= 1024, "control block");
+
+// Persistent kernel: one CTA per SM takes work items from two queues, first the tcgen05-path items, then the
+// warp-level-MMA items (each queue longest first, so the items that start last are the short ones).
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
                  const __grid_constant__ CUtensorMap k2_map, AttnArgs a) {
-    // launched with programmatic stream serialization: the CTAs may become resident while the plan kernel still
-    // runs, so nothing it writes is read before this wait
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Ctrl* c = reinterpret_cast<Ctrl*>(smem + kDataBytes<DH>);
+    __shared__ float xch[2][2][128];   // [group parity][column half][row]: partial row maxima of the tcgen05 phase
+    __shared__ float xl[2][128];       // [column half][row]: partial row sums at the end of an item
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMmaStages; ++s) {
+            mbar_init(smem_u32(&c->ring_full[s]), 1);    // tcgen05 phase: one arrival (with the group's byte count)
+            mbar_init(smem_u32(&c->ring_empty[s]), 1);
+        }
+        for (int b = 0; b < kTcSBufs; ++b) {
+            mbar_init(smem_u32(&c->s_full[b]), 1);
+            mbar_init(smem_u32(&c->p_full[b]), kTcSoftmaxThreads);
+            mbar_init(smem_u32(&c->pv_done[b]), 1);
+        }
+        mbar_init(smem_u32(&c->q_ready), kTcSoftmaxThreads);
+        mbar_init(smem_u32(&c->o_free), kTcSoftmaxThreads);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&c->sched_full[0][s]), 1);
+            mbar_init(smem_u32(&c->sched_full[1][s]), 1);
+            mbar_init(smem_u32(&c->sched_empty[0][s]), 1 + kTcSoftmaxThreads / 32);   // MMA warp + softmax warps
+            mbar_init(smem_u32(&c->sched_empty[1][s]), kMmaWarps);
+        }
+        mbar_init(smem_u32(&c->geom_a), kMmaWarps + 1);
+        mbar_init(smem_u32(&c->geom_b), 1);
+        c->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (DH == 128 && warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c->tmem_base)), "n"(kTcCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // launched with programmatic stream serialization: everything above overlaps the plan kernel; nothing it writes
+    // is read before this wait
     STAMP_MIN(2);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     STAMP_MIN(6);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if ((int)blockIdx.x >= a.plan[0]) return;
-    extern __shared__ unsigned char smem_raw[];
-    const AttnItem item = a.items[blockIdx.x];
-    if (DH == 128 && item.pad[0])
-        tc_item(k2_map, v_map, a, item, smem_raw);
-    else
-        split_item<DH>(k_map, v_map, a, item, smem_raw);
+    const int n_items = a.plan[0], n_tc = a.plan[5];
+    if (DH == 128 && n_tc > 0) {
+        tc_phase(k2_map, v_map, a, smem, c, xch, xl, a.plan + 8, n_tc);
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+    if (n_items > n_tc && !ABORTED(c)) mma_phase<DH>(k_map, v_map, a, smem, c, a.plan + 9, n_items);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may take this SM
+    tc_fence_before();
+    __syncthreads();
     STAMP_MAX(3);
+    if (DH == 128 && warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c->tmem_base), "n"(kTcCols) : "memory");
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1174,16 +1376,15 @@ dcut_status make_cache_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, lo
 template <int DH>
 dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm, const CUtensorMap& k2m, const AttnArgs& aa,
                      const CombineArgs& ca, int T_cap, cudaStream_t stream) {
-    constexpr int kSmem = (DH == 128 && kTcSmem > SmemLayout<DH>::kTotal) ? kTcSmem : SmemLayout<DH>::kTotal;
     // Both kernels may be scheduled before their predecessor has finished (they wait on the device before reading
     // its results), which hides the launch latency between the three kernels of the call.
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(ctx->max_items);
+    lc.gridDim = dim3(ctx->sm_count);   // persistent: one CTA per SM
     lc.blockDim = dim3(kThreads);
-    lc.dynamicSmemBytes = kSmem;
+    lc.dynamicSmemBytes = kSmemBytes<DH>;
     lc.stream = stream;
     lc.attrs = attr;
     lc.numAttrs = 1;
@@ -1200,10 +1401,9 @@ dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm
 }  // namespace
 
 dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
-    constexpr int kSmem128 = kTcSmem > SmemLayout<128>::kTotal ? kTcSmem : SmemLayout<128>::kTotal;
-    cudaError_t e = cudaFuncSetAttribute(attn_item_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem128);
+    cudaError_t e = cudaFuncSetAttribute(attn_item_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes<128>);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 128)");
-    e = cudaFuncSetAttribute(attn_item_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemLayout<64>::kTotal);
+    e = cudaFuncSetAttribute(attn_item_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes<64>);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn 64)");
     {
         const char* env = getenv("DCUT_ATTN_TC_MIN_ROWS");   // query rows from which an item goes to the tcgen05 kernel
@@ -1255,7 +1455,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     while (pa.npad < B) pa.npad <<= 1;
     pa.status = ctx->d_status;
     pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
-    pa.max_item_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? 128 : 144;
+    pa.max_item_rows = 128;
     pa.max_items = ctx->max_items;
     pa.part_rows_cap = ctx->part_rows_cap;
     pa.items = ctx->d_items;
