@@ -429,6 +429,40 @@ def run_dcut(args):
             tot_ms = sum(r["ms"] for r in rows.values())
             rows["all"] = {"ms": round(tot_ms, 4), "tflops": round(layer_flops(cfg, T) / tot_ms / 1e9, 1)}
             gemm[arm] = rows
+        # LM head fused with acceptance (logits never stored) beside the unfused pair, full-gamma packing
+        try:
+            V = cfg.vocab
+            Vp = (V + 255) // 256 * 256
+            T = res["full_gamma"]["T"]
+            cu_full = torch.arange(0, cfg.B + 1, dtype=torch.int32, device=dev) * (cfg.gamma + 1)
+            w_lm = torch.zeros((Vp, cfg.hidden), dtype=torch.bfloat16, device=dev)
+            w_lm[:V] = wl.lm_head_weight(cfg).to(dev)
+            xh = torch.randn((cap, cfg.hidden), device=dev, dtype=torch.float32).to(torch.bfloat16)
+            logits_buf = torch.empty((cap, Vp), dtype=torch.bfloat16, device=dev)
+
+            def timed(fn, n=10):
+                for _ in range(2):
+                    fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(n):
+                    fn()
+                e1.record()
+                e1.synchronize()
+                return e0.elapsed_time(e1) / n
+
+            fused_ms = timed(lambda: ctx.lm_head_accept(xh, w_lm[:V], d_draft, cu_full, cap, out_tokens=False))
+            gemm_ms = timed(lambda: ctx.gemm_bf16(xh, w_lm, cu_full, cap, logits_buf))
+            ctx_v = binding.Context(max_B=cfg.B, max_gamma=cfg.gamma, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                                    head_dim=cfg.head_dim, page_size=cfg.page_size, max_pages_per_req=1, vocab=Vp)
+            acc_ms = timed(lambda: ctx_v.accept(logits_buf, d_draft, cu_full, cap, out_tokens=False))
+            fl = 2.0 * T * cfg.hidden * V
+            gemm["lm_head"] = {"T": T, "V": V, "fused_ms": round(fused_ms, 4), "fused_tflops": round(fl / fused_ms / 1e9, 1),
+                               "unfused_gemm_ms": round(gemm_ms, 4), "unfused_accept_ms": round(acc_ms, 4),
+                               "logits_bytes_not_moved": 2 * T * V * 2}
+            del w_lm, logits_buf, ctx_v
+        except Exception as exc:   # the extra measurement must not take the bench line down
+            gemm["lm_head"] = {"error": repr(exc)[:200]}
 
     if rank != 0:
         return

@@ -193,6 +193,22 @@ dcut_status dcut_layer_forward(dcut_ctx* ctx, const dcut_layer_weights* weights,
                                int T_cap, void* stream);
 
 /*
+ * LM head fused with acceptance (the step between the last layer and dcut_accept, Section 3.1: the target's next-token
+ * prediction at every retained position): logits[T, V] = x[T, hidden] . w_lm[V, hidden]^T (bf16 in, fp32 accumulate,
+ * rounded to bf16 exactly as if the logits were stored), reduced inside the GEMM's epilogue to the row's argmax
+ * (largest bf16 value, lowest index among equal values, NaN never selected, a row without any selectable value gives
+ * 0), followed by the prefix match of dcut_accept.  The T * V * 2 bytes of logits are never written or read.
+ * The outputs equal those of dcut_gemm_bf16 (mode 0, N = V) followed by dcut_accept on the same inputs.
+ * DEVICE in: x bf16 [T_cap rows readable, hidden], w_lm bf16 [V, hidden] (both 128-byte aligned), draft_ids, cu_q as
+ * in dcut_accept.  DEVICE out: as dcut_accept, plus row_argmax int32 [T] (optional, may be null): the argmax of
+ * every packed row.  Requirements: context created with layer shapes (hidden > 0); 1 <= V (any value: the ragged
+ * last tile is masked).  Uses the context's per-row words (not concurrently with dcut_accept on the same context).
+ */
+dcut_status dcut_lm_head_accept(dcut_ctx* ctx, const void* x, const void* w_lm, int V, const int* draft_ids,
+                                const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
+                                int* out_tokens, int* n_accepted_total, int* row_argmax, void* stream);
+
+/*
  * dcut_accept without any allocation.  (The paper has no counterpart: this entry point exists for
  * the way the library gets embedded, not for the method.)
  *

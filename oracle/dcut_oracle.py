@@ -236,6 +236,15 @@ def linear(a, w) -> np.ndarray:
     return c
 
 
+def lm_head_accept(x, w_lm, draft_ids, cu_q, gamma: int):
+    """The LM head followed by greedy acceptance (Section 3.1: the target's prediction at every retained position):
+    logits = x . w_lm^T in fp64 from the bf16 inputs, rounded to bf16 (the tensor a target model hands to the
+    acceptance step), then `accept`.  Returns (AcceptResult, logits fp64 [T, V])."""
+    logits64 = linear(x, w_lm)
+    res = accept(_as_bf16_tensor(round_bf16(logits64)), draft_ids, cu_q, gamma)
+    return res, logits64
+
+
 def rope(x, pos, theta: float) -> np.ndarray:
     xb = _bf16_bits(x)
     rows, heads, dh = xb.shape

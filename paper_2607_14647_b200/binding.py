@@ -28,7 +28,8 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
-           "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_poll_device_status"]
+           "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_lm_head_accept",
+           "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -76,6 +77,7 @@ class LayerWeights(C.Structure):
 
 
 _lib.dcut_gemm_bf16.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _vp, _vp]
+_lib.dcut_lm_head_accept.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.dcut_layer_forward.argtypes = [_vp, C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _vp, _vp,
                                     _i, _i, _vp]
 
@@ -273,6 +275,20 @@ class Context:
                                         _ptr(w2, torch.bfloat16), mode, N, K, _ptr(cu_q, torch.int32), B, T_cap,
                                         _ptr(out, torch.bfloat16), _ptr(residual, torch.bfloat16), _stream()))
         return out
+
+    def lm_head_accept(self, x, w_lm, draft_ids, cu_q, T_cap: int, out_tokens: bool = True, row_argmax: bool = False):
+        """dcut_lm_head_accept: acceptance straight from the last hidden states x[T, hidden] and the LM head w_lm[V, hidden]."""
+        B, gamma = draft_ids.shape
+        V = w_lm.shape[0]
+        i32 = dict(dtype=torch.int32, device=x.device)
+        accept_len, bonus = torch.empty(B, **i32), torch.empty(B, **i32)
+        toks = torch.empty((B, gamma + 1), **i32) if out_tokens else None
+        total = torch.empty(1, **i32)
+        am = torch.full((T_cap,), -1, **i32) if row_argmax else None
+        self._check(_lib.dcut_lm_head_accept(self._h, _ptr(x, torch.bfloat16), _ptr(w_lm, torch.bfloat16), V,
+                                             _ptr(draft_ids, torch.int32), _ptr(cu_q, torch.int32), B, gamma, T_cap,
+                                             _ptr(accept_len), _ptr(bonus), _ptr(toks), _ptr(total), _ptr(am), _stream()))
+        return accept_len, bonus, toks, total, am
 
     def layer_forward(self, weights: dict, x, y, k_cache, v_cache, block_table, ctx_lens, cu_q, tok_req, tok_pos,
                       T_cap: int, rms_eps: float = 1e-6, rope_theta: float = 1e6):

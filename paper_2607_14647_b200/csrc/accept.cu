@@ -24,12 +24,7 @@ __device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
     return r;
 }
 
-// value order as an unsigned integer: larger float <=> larger code; every non-NaN code is > 0
-__device__ __forceinline__ unsigned int ordered_bits(float f) {
-    if (f == 0.0f) f = 0.0f;   // -0 and +0 are the same value
-    const unsigned int b = __float_as_uint(f);
-    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
+__device__ __forceinline__ unsigned int ordered_bits(float f) { return dcut_ordered_bits(f); }
 
 __device__ __forceinline__ void take(float f, int idx, float& best, int& bidx) {
     if (f > best) {   // strict: the first of equal values stays; NaN never passes
@@ -114,7 +109,7 @@ __global__ void __launch_bounds__(1024) accept_match_kernel(
     const unsigned short* __restrict__ logits, int V, const int* __restrict__ draft_ids,
     const int* __restrict__ cu_q, int B, int gamma, unsigned long long* __restrict__ row_key,
     int* __restrict__ accept_len, int* __restrict__ bonus, int* __restrict__ out_tokens,
-    int* __restrict__ n_accepted_total) {
+    int* __restrict__ n_accepted_total, int* __restrict__ row_argmax) {
     __shared__ int total_s;
     if (threadIdx.x == 0) total_s = 0;
     __syncthreads();
@@ -130,7 +125,9 @@ __global__ void __launch_bounds__(1024) accept_match_kernel(
             if (t <= d) {
                 const unsigned long long key = row_key[a + t];
                 row_key[a + t] = 0;
-                am = key ? (int)(0xffffffffu - (unsigned int)key) : slow_first_valid(logits + (size_t)(a + t) * V, V);
+                am = key ? (int)(0xffffffffu - (unsigned int)key)
+                         : (logits ? slow_first_valid(logits + (size_t)(a + t) * V, V) : 0);
+                if (row_argmax) row_argmax[a + t] = am;
                 stop = (t == d) || am != draft_ids[(size_t)i * gamma + t];
             }
             const unsigned int mask = __ballot_sync(0xffffffffu, stop);
@@ -181,7 +178,16 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
     dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_argmax_kernel");
     if (st != DCUT_OK) return st;
     accept_match_kernel<<<1, 1024, 0, stream>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B,
-                                               gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total);
+                                               gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total, nullptr);
+    return dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_match_kernel");
+}
+
+dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
+                                     int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
+                                     int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
+                                     cudaStream_t stream) {
+    accept_match_kernel<<<1, 1024, 0, stream>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B,
+                                               gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total, row_argmax);
     return dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_match_kernel");
 }
 
@@ -275,7 +281,7 @@ extern "C" dcut_status dcut_accept_static(const void* logits, int V, const int* 
     accept_argmax_kernel<<<grid, kArgmaxThreads, 0, cs>>>(static_cast<const unsigned short*>(logits), V, cu_q, B, seg, keys);
     if ((e = cudaGetLastError()) == cudaSuccess) {
         accept_match_kernel<<<1, 1024, 0, cs>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma,
-                                               keys, accept_len, bonus, out_tokens, n_accepted_total);
+                                               keys, accept_len, bonus, out_tokens, n_accepted_total, nullptr);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) {

@@ -292,6 +292,25 @@ dcut_status dcut_gemm_bf16(dcut_ctx* c, const void* a, const void* w, const void
     return dcut_launch_gemm(c, a, w, w2, mode, N, K, cu_q, B, T_cap, out, residual, static_cast<cudaStream_t>(stream));
 }
 
+dcut_status dcut_lm_head_accept(dcut_ctx* c, const void* x, const void* w_lm, int V, const int* draft_ids,
+                                const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
+                                int* out_tokens, int* n_accepted_total, int* row_argmax, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (c->lim.hidden <= 0 || !c->layer_maps) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
+    if (!x || !w_lm || !draft_ids || !cu_q || !accept_len || !bonus) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (V < 1 || c->lim.hidden % 64) return dcut_fail(c, DCUT_EINVAL, "need V >= 1 and hidden %% 64 == 0");
+    if (B < 1 || B > c->lim.max_B || gamma < 1 || gamma > c->lim.max_gamma || T_cap < B ||
+        T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
+        return dcut_fail(c, DCUT_ECAPACITY, "B = %d, gamma = %d, T_cap = %d outside the limits", B, gamma, T_cap);
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(w_lm)) & 127)
+        return dcut_fail(c, DCUT_EINVAL, "x and w_lm must be 128-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    dcut_status st = dcut_launch_lm_head_argmax(c, x, w_lm, V, c->lim.hidden, cu_q, B, T_cap, c->d_row_key, s);
+    if (st != DCUT_OK) return st;
+    return dcut_launch_accept_match(c, nullptr, V, draft_ids, cu_q, B, gamma, accept_len, bonus, out_tokens,
+                                    n_accepted_total, row_argmax, c->d_row_key, s);
+}
+
 dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                                void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                                const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,

@@ -80,6 +80,15 @@ struct dcut_ctx {
     int* hs_host_cu_q;      // pinned
 };
 
+#ifdef __CUDACC__
+// value order as an unsigned integer: larger float <=> larger code; every non-NaN code is > 0
+__device__ __forceinline__ unsigned int dcut_ordered_bits(float f) {
+    if (f == 0.0f) f = 0.0f;   // -0 and +0 are the same value
+    const unsigned int b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+#endif
+
 dcut_status dcut_fail(dcut_ctx* ctx, dcut_status st, const char* fmt, ...);
 dcut_status dcut_check_cuda(dcut_ctx* ctx, cudaError_t e, const char* what);
 
@@ -105,6 +114,13 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
                                     void* out, float* lse, cudaStream_t stream);
 dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
                              const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream);
+dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void* w_lm, int V, int K, const int* cu_q, int B,
+                                       int T_cap, unsigned long long* row_key, cudaStream_t stream);
+// second half of dcut_accept on per-row words that are already filled (logits may be null: rows without a word give 0)
+dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
+                                     int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
+                                     int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
+                                     cudaStream_t stream);
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,

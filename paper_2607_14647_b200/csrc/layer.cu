@@ -32,7 +32,7 @@ constexpr int kTmemCols = 512;              // two 128 x 256 fp32 accumulators
 constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256 /* barriers, tmem ptr */;
 constexpr int kWaitLimit = 1 << 22;
 
-enum GemmMode { kPlain = 0, kResidual = 1, kSwiGLU = 2 };
+enum GemmMode { kPlain = 0, kResidual = 1, kSwiGLU = 2, kArgmax = 3 };
 
 // ------------------------------------------------------------------------------------------------ PTX
 
@@ -128,6 +128,8 @@ struct GemmArgs {
     int n_tiles;       // output tiles along N
     __nv_bfloat16* out;
     const __nv_bfloat16* residual;   // [T, N_out] or null
+    unsigned long long* row_key;     // kArgmax: one packed (ordered maximum, ~column) word per row
+    int V;                           // kArgmax: live columns (rows of the weight)
     int* status;
 };
 
@@ -269,6 +271,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                         }
                     }
                 }
+            } else if (MODE == kArgmax) {
+                // The bf16 logits an unfused path would store are formed in registers and reduced to the row's
+                // (maximum, first column) over this tile; rows merge across tiles with a 64-bit atomicMax on
+                // (ordered value << 32 | ~column): largest value, lowest column, whatever order the tiles finish in.
+                float best = -INFINITY;
+                int bidx = -1;
+                const int col0 = n_tile * BN;
+#pragma unroll 1
+                for (int c = 0; c < BN; c += 32) {
+                    uint32_t av[32];
+                    tc_ld32(t_row + c, av);
+                    tc_wait_ld();
+                    if (col0 + c < g.V) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2) {
+                            const uint32_t pk = pack_bf16(__uint_as_float(av[e]), __uint_as_float(av[e + 1]));
+                            const float f0 = bf_lo(pk), f1 = bf_hi(pk);
+                            const int col = col0 + c + e;
+                            if (col < g.V && f0 > best) {        // strict: the first of equal values stays; NaN never passes
+                                best = f0;
+                                bidx = col;
+                            }
+                            if (col + 1 < g.V && f1 > best) {
+                                best = f1;
+                                bidx = col + 1;
+                            }
+                        }
+                    }
+                }
+                if (row < T && bidx >= 0)
+                    atomicMax(g.row_key + row, ((unsigned long long)dcut_ordered_bits(best) << 32) | (0xffffffffu - (unsigned int)bidx));
             } else {
                 __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + (size_t)n_tile * BN;
                 const __nv_bfloat16* rrow = MODE == kResidual ? g.residual + (size_t)row * g.N_out + (size_t)n_tile * BN : nullptr;
@@ -443,12 +476,33 @@ dcut_status dcut_init_layer(dcut_ctx* ctx) {
     cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(gemm)");
     ctx->layer_maps = calloc(1, sizeof(LayerMaps));
     return ctx->layer_maps ? DCUT_OK : dcut_fail(ctx, DCUT_EINVAL, "out of host memory");
 }
 
 void dcut_free_layer(dcut_ctx* ctx) { free(ctx->layer_maps); }
+
+// logits = x . w_lm^T reduced on the fly to one (maximum, first column) word per row: the [T, V] logits never exist
+dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void* w_lm, int V, int K, const int* cu_q, int B,
+                                       int T_cap, unsigned long long* row_key, cudaStream_t stream) {
+    CUtensorMap am, bm;
+    dcut_status st = make_kmajor_map(ctx, &am, x, T_cap, K, BM);
+    if (st != DCUT_OK) return st;
+    if ((st = make_kmajor_map(ctx, &bm, w_lm, V, K, BN / 2)) != DCUT_OK) return st;   // rows past V read as zeros
+    GemmArgs g;
+    g.cu_q = cu_q;
+    g.B = B;
+    g.N_out = V;
+    g.K = K;
+    g.out = nullptr;
+    g.residual = nullptr;
+    g.row_key = row_key;
+    g.V = V;
+    g.status = ctx->d_status;
+    return launch_gemm<kArgmax>(ctx, am, bm, bm, (V + BN - 1) / BN, T_cap, g, stream);
+}
 
 dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
                              const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream) {
@@ -467,6 +521,8 @@ dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const 
     g.K = K;
     g.out = static_cast<__nv_bfloat16*>(out);
     g.residual = static_cast<const __nv_bfloat16*>(residual);
+    g.row_key = nullptr;
+    g.V = 0;
     g.status = ctx->d_status;
     if (mode == kSwiGLU) return launch_gemm<kSwiGLU>(ctx, am, bm, b2m, N / (BN / 2), T_cap, g, stream);
     if (mode == kResidual) return launch_gemm<kResidual>(ctx, am, bm, b2m, N / BN, T_cap, g, stream);
@@ -500,6 +556,8 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     GemmArgs g;
     g.cu_q = cu_q;
     g.B = B;
+    g.row_key = nullptr;
+    g.V = 0;
     g.status = ctx->d_status;
 
     // 1. n = RMSNorm(x)

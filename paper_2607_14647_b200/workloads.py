@@ -30,6 +30,7 @@ import torch
 # stream tags
 _TAG_CONF, _TAG_IDS, _TAG_CTX, _TAG_REJECT, _TAG_PAGES, _TAG_KV, _TAG_Q, _TAG_LOGITS = range(1, 9)
 _TAG_LAYER_X, _TAG_LAYER_W = 9, 10
+_TAG_LM_W, _TAG_LM_X = 11, 12
 
 
 @dataclass(frozen=True)
@@ -288,4 +289,31 @@ def layer_x_rows(cfg: WorkloadConfig, depths: np.ndarray, hidden: Optional[int] 
         for t in range(int(d) + 1):
             rng = np.random.default_rng([cfg.seed, _TAG_LAYER_X, i, t])
             out[cu[i] + t] = torch.from_numpy(rng.standard_normal(H, dtype=np.float32)).to(torch.bfloat16)
+    return out
+
+
+# --------------------------------------------------------------------------- LM head inputs
+
+def lm_head_weight(cfg: WorkloadConfig, vocab: Optional[int] = None, hidden: Optional[int] = None) -> torch.Tensor:
+    """LM-head weight bf16 [V, hidden] ~ N(0, 0.02^2)."""
+    V = cfg.vocab if vocab is None else vocab
+    H = cfg.hidden if hidden is None else hidden
+    rng = np.random.default_rng([cfg.seed, _TAG_LM_W])
+    return (_randn_bf16(rng, V * H).float().mul_(0.02)).to(torch.bfloat16).view(V, H)
+
+
+def lm_head_x_rows(cfg: WorkloadConfig, sel: SelectInputs, depths: np.ndarray, w_lm: torch.Tensor) -> torch.Tensor:
+    """Last hidden states bf16 [T, hidden], packed like `q_rows`.  Rows t < reject_index[i] are 5 x the LM-head row of
+    the next draft token z_{i,t+1}, which makes that token the maximum by a wide margin (the target 'accepts' exactly
+    reject_index[i] drafts); every other row is ~ N(0,1), one counter-seeded draw per (i, t)."""
+    V, H = w_lm.shape
+    cu = cu_q_from_depths(depths)
+    out = torch.empty((int(cu[-1]), H), dtype=torch.bfloat16)
+    for i, d in enumerate(depths):
+        for t in range(int(d) + 1):
+            if t < int(sel.reject_index[i]) and t < cfg.gamma:
+                out[cu[i] + t] = (w_lm[int(sel.draft_ids[i, t]) % V].float() * 5.0).to(torch.bfloat16)
+            else:
+                rng = np.random.default_rng([cfg.seed, _TAG_LM_X, i, t])
+                out[cu[i] + t] = torch.from_numpy(rng.standard_normal(H, dtype=np.float32)).to(torch.bfloat16)
     return out

@@ -1,0 +1,141 @@
+"""dcut_lm_head_accept (LM-head GEMM whose epilogue keeps only the row argmax, then the prefix match) against the
+oracle and against the unfused CUDA path (dcut_gemm_bf16 followed by dcut_accept).
+
+The argmax is taken on bf16-rounded logits.  The kernel accumulates in fp32 and the oracle in fp64, so a logit that
+sits on a rounding boundary can land one bf16 step apart; where that changes the winner both answers are correct.
+The tests therefore require: the same index as the oracle, or an index whose fp64 logit is within two bf16 steps of
+the oracle's maximum (and the same index on at least 97 % of the rows); acceptance outputs that follow exactly from
+the kernel's own row argmax; and outputs identical to the unfused CUDA path, which rounds the same fp32 sums."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dcut_oracle as orc
+from paper_2607_14647_b200 import workloads as wl
+from tests.gpu_helpers import dev, make_ctx
+
+pytestmark = pytest.mark.gpu
+
+
+def _accept_from_argmax(am, draft_ids, cu, gamma):
+    B = len(cu) - 1
+    al, bo, ot = np.zeros(B, np.int32), np.zeros(B, np.int32), np.full((B, gamma + 1), -1, np.int32)
+    for i in range(B):
+        d = cu[i + 1] - cu[i] - 1
+        m = 0
+        while m < d and am[cu[i] + m] == draft_ids[i, m]:
+            m += 1
+        al[i], bo[i] = m, am[cu[i] + m]
+        ot[i, :m] = draft_ids[i, :m]
+        ot[i, m] = bo[i]
+    return al, bo, ot
+
+
+def _check_rows(am_gpu, ref_am, logits64, rows=None):
+    rows = range(len(ref_am)) if rows is None else rows
+    same = 0
+    for k, r in enumerate(rows):
+        g, o = int(am_gpu[r]), int(ref_am[k])
+        if g == o:
+            same += 1
+            continue
+        top = logits64[k, o]
+        assert abs(logits64[k, g] - top) <= 2.0 ** -7 * max(abs(top), 1e-30), (r, g, o, logits64[k, g], top)
+    return same
+
+
+def _case(B, gamma, V, H, depths, seed=0):
+    cfg = wl.custom_config(B=B, gamma=gamma, n_q_heads=4, n_kv_heads=2, head_dim=128, vocab=V, index=100 + seed)
+    sel = wl.select_inputs(cfg)
+    w = wl.lm_head_weight(cfg, vocab=V, hidden=H)
+    x = wl.lm_head_x_rows(cfg, sel, depths, w)
+    cu = wl.cu_q_from_depths(depths)
+    return cfg, sel, w, x, cu
+
+
+@pytest.mark.parametrize("B,V,H", [(5, 1000, 256), (8, 256, 512), (16, 700, 256), (3, 1, 256), (12, 2049, 1024)])
+def test_small_shapes_every_row(B, V, H):
+    gamma = 8
+    rng = np.random.default_rng(V + H)
+    depths = rng.integers(0, gamma + 1, B).astype(np.int32)
+    depths[0], depths[-1] = gamma, 0
+    cfg, sel, w, x, cu = _case(B, gamma, V, H, depths, seed=V)
+    draft = (sel.draft_ids % V).astype(np.int32)
+    ctx = make_ctx(cfg, max_pages=1, hidden=H, intermediate=H, vocab=0)
+    T = int(cu[-1])
+    xd = torch.zeros((cfg.t_cap, H), dtype=torch.bfloat16, device="cuda")
+    xd[:T] = dev(x)
+    al, bo, toks, total, am = ctx.lm_head_accept(xd, dev(w), dev(draft), dev(cu), cfg.t_cap, row_argmax=True)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    ref, logits64 = orc.lm_head_accept(x, w, draft, cu, gamma)
+    am = am.cpu().numpy()
+    same = _check_rows(am[:T], ref.argmax, logits64)
+    assert same >= int(0.97 * T)
+    assert np.all(am[T:] == -1)
+    want_al, want_bo, want_ot = _accept_from_argmax(am, draft, cu, gamma)
+    assert np.array_equal(al.cpu().numpy(), want_al) and np.array_equal(bo.cpu().numpy(), want_bo)
+    assert np.array_equal(toks.cpu().numpy(), want_ot) and int(total.item()) == int((want_al + 1).sum())
+    if same == T:
+        assert np.array_equal(al.cpu().numpy(), ref.accept_len) and np.array_equal(bo.cpu().numpy(), ref.bonus)
+        assert np.array_equal(toks.cpu().numpy(), ref.out_tokens) and int(total.item()) == ref.n_accepted_total
+    # a second call on the same context starts from clean per-row words
+    al2, bo2, *_ = ctx.lm_head_accept(xd, dev(w), dev(draft), dev(cu), cfg.t_cap)
+    assert torch.equal(al, al2) and torch.equal(bo, bo2)
+
+
+@pytest.mark.parametrize("B,V,H", [(16, 1024, 512), (40, 8192, 4096)])
+def test_equals_unfused_cuda_path(B, V, H):
+    gamma = 16
+    rng = np.random.default_rng(B)
+    depths = rng.integers(0, gamma + 1, B).astype(np.int32)
+    cfg, sel, w, x, cu = _case(B, gamma, V, H, depths, seed=B)
+    draft = (sel.draft_ids % V).astype(np.int32)
+    ctx = make_ctx(cfg, max_pages=1, hidden=H, intermediate=H, vocab=V)
+    T = int(cu[-1])
+    xd = torch.zeros((cfg.t_cap, H), dtype=torch.bfloat16, device="cuda")
+    xd[:T] = dev(x)
+    wd, dd, cd = dev(w), dev(draft), dev(cu)
+    fused = ctx.lm_head_accept(xd, wd, dd, cd, cfg.t_cap, row_argmax=True)
+    logits = torch.empty((cfg.t_cap, V), dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(xd, wd, cd, cfg.t_cap, logits)
+    unfused = ctx.accept(logits, dd, cd, cfg.t_cap)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    for a, b in zip(fused[:4], unfused):
+        assert torch.equal(a, b)
+    lf = logits[:T].float()
+    lf[lf.isnan()] = -float("inf")
+    assert torch.equal(fused[4][:T].long(), lf.argmax(dim=1))   # (ties: both take the first index)
+
+
+def test_config4_sampled_rows():
+    cfg = wl.config(4)
+    sel = wl.select_inputs(cfg)
+    rng = np.random.default_rng(4)
+    depths = np.minimum(rng.integers(0, cfg.gamma + 1, cfg.B), cfg.gamma).astype(np.int32)
+    w = wl.lm_head_weight(cfg)                 # [151 936, 4096]
+    x = wl.lm_head_x_rows(cfg, sel, depths, w)
+    cu = wl.cu_q_from_depths(depths)
+    T = int(cu[-1])
+    draft = (sel.draft_ids % cfg.vocab).astype(np.int32)
+    ctx = make_ctx(cfg, max_pages=1, hidden=cfg.hidden, intermediate=cfg.intermediate, vocab=0)
+    xd = torch.zeros((cfg.t_cap, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+    xd[:T] = dev(x)
+    al, bo, toks, total, am = ctx.lm_head_accept(xd, dev(w), dev(draft), dev(cu), cfg.t_cap, row_argmax=True)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    am = am.cpu().numpy()
+    want_al, want_bo, want_ot = _accept_from_argmax(am, draft, cu, cfg.gamma)
+    assert np.array_equal(al.cpu().numpy(), want_al) and np.array_equal(bo.cpu().numpy(), want_bo)
+    assert np.array_equal(toks.cpu().numpy(), want_ot) and int(total.item()) == int((want_al + 1).sum())
+    # planted rows: the draft token must win
+    for i, d in enumerate(depths):
+        for t in range(min(int(sel.reject_index[i]), int(d))):
+            assert am[cu[i] + t] == draft[i, t]
+    # sampled rows against the oracle (first, last, and a few in between; planted and random ones)
+    rows = sorted(set([0, 1, T // 3, T // 2, T - 2, T - 1]))
+    logits64 = orc.linear(x[rows], w)
+    ref_am = orc.accept(orc._as_bf16_tensor(orc.round_bf16(logits64)), np.zeros((len(rows), 1), np.int32),
+                        np.arange(len(rows) + 1, dtype=np.int32), 1).argmax
+    _check_rows(am, ref_am, logits64, rows)
