@@ -17,6 +17,10 @@
  *                       bonus token)
  *   oracle_layer_*      the decoder-layer pieces of the full-layer workload (textbook RMSNorm,
  *                       rotary embedding, SwiGLU, matrix product; not from the paper)
+ *   oracle_scores_shifted, oracle_select_causal, oracle_accept_rs
+ *                       Appendix B "Causality under Rejection Sampling": Eq. 7 (shifted score), the
+ *                       causal early-stopping frontier scan, standard rejection sampling with the
+ *                       residual distribution
  *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py against closed forms,
  * brute force, hand-derived examples or numpy float64 formulas, except the comparison of the
@@ -459,4 +463,188 @@ int oracle_swiglu_f64(const double* g, const double* u, long n, double* y) {
     if (!g || !u || !y) return ORACLE_EINVAL;
     for (long i = 0; i < n; ++i) y[i] = g[i] / (1.0 + exp(-g[i])) * u[i];
     return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Stochastic variant (Appendix B "Causality under Rejection Sampling").                       */
+/*                                                                                              */
+/* Shifted score (Eq. 7): s~_{i,1} = 1 and s~_{i,k} = prod_{t=1}^{k-1} c_{i,t}: the admission    */
+/* score of depth k uses only the confidences before k, fp32 left to right like Eq. 3.           */
+int oracle_scores_shifted(const float* conf, int B, int gamma, float* scores) {
+    if (!conf || !scores || B < 0 || gamma < 0) return ORACLE_EINVAL;
+    for (int i = 0; i < B; ++i) {
+        float s = 1.0f;
+        for (int k = 1; k <= gamma; ++k) {
+            scores[(size_t)i * gamma + (k - 1)] = s;   /* before the k-th confidence is applied */
+            s = s * clamp_conf(conf[(size_t)i * gamma + (k - 1)]);
+            if (s == 0.0f) s = 0.0f;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Causal early-stopping scan ("maintains one frontier position per request and repeatedly considers
+ * the frontier with the largest shifted score ... if the objective improves, the position is
+ * irrevocably admitted and the next position from that request is exposed, otherwise the scan
+ * stops").  Written as that loop, one admission per iteration.
+ * Readings: ties between frontiers by shallower depth, then request index (same paragraph); the
+ * utility is B + the sum of the admitted SHIFTED scores (the only quantity the scan may consult),
+ * summed exactly in units of 2^-40 like oracle_select; "improves" is a strict '>' between two fp64
+ * quotients by (double)cost_fp32; the cost table is dense in the packed length T = B + N.
+ * Outputs as oracle_select (depths, cu_q, packed metadata, info; candidate = n_star).
+ */
+int oracle_select_causal(const float* conf, int B, int gamma, const int32_t* draft_ids,
+                         const int32_t* bonus_ids, const int32_t* ctx_lens, const float* cost_ms, int n_cost,
+                         int32_t* depths, int32_t* cu_q, int32_t* tok_req, int32_t* tok_pos, int32_t* tok_id,
+                         float* scores_out, oracle_select_info* info) {
+    if (!conf || !depths || !cu_q || !info || !cost_ms || B < 0 || gamma < 0) return ORACLE_EINVAL;
+    const int n = B * gamma;
+    if (n_cost < B + n + 1) return ORACLE_ECOST;
+    for (int t = B; t <= B + n; ++t)
+        if (!(cost_ms[t] > 0.0f) || isinf(cost_ms[t])) return ORACLE_ECOST;
+    const int64_t ONE = (int64_t)1 << 40;
+    float* s = (float*)malloc(sizeof(float) * (size_t)(n > 0 ? n : 1));
+    oracle_scores_shifted(conf, B, gamma, s);
+    if (scores_out) memcpy(scores_out, s, sizeof(float) * (size_t)n);
+    int* frontier = (int*)malloc(sizeof(int) * (size_t)(B > 0 ? B : 1));   /* next depth to expose, 1-based */
+    for (int i = 0; i < B; ++i) frontier[i] = 1;
+    int N = 0;
+    int64_t Q = 0;
+    double S = 0.0;
+    double cur = (double)((int64_t)B * ONE) / (double)cost_ms[B];
+    for (;;) {
+        int bi = -1;
+        for (int i = 0; i < B; ++i) {
+            if (frontier[i] > gamma) continue;
+            if (bi < 0) { bi = i; continue; }
+            const float a = s[i * gamma + frontier[i] - 1], b = s[bi * gamma + frontier[bi] - 1];
+            if (a > b || (a == b && frontier[i] < frontier[bi])) bi = i;   /* equal depth: the lower request stays */
+        }
+        if (bi < 0) break;
+        const float sc = s[bi * gamma + frontier[bi] - 1];
+        const int64_t q = (int64_t)floor((double)sc * 1099511627776.0);
+        const double obj = (double)((int64_t)B * ONE + Q + q) / (double)cost_ms[B + N + 1];
+        if (!(obj > cur)) break;
+        cur = obj;
+        Q += q;
+        S += (double)sc;
+        N += 1;
+        frontier[bi] += 1;
+    }
+    info->n_star = N;
+    info->t_total = B + N;
+    info->candidate = N;
+    info->closure_ok = 1;   /* by construction: a request's positions are admitted in depth order */
+    info->sum_fixed = (int64_t)B * ONE + Q;
+    info->objective = cur;
+    info->sum_f64 = (double)B + S;
+    cu_q[0] = 0;
+    for (int i = 0; i < B; ++i) {
+        depths[i] = frontier[i] - 1;
+        cu_q[i + 1] = cu_q[i] + 1 + depths[i];
+    }
+    for (int i = 0; i < B; ++i)
+        for (int t = 0; t <= depths[i]; ++t) {
+            const int r = cu_q[i] + t;
+            if (tok_req) tok_req[r] = i;
+            if (tok_pos) tok_pos[r] = (ctx_lens ? ctx_lens[i] : 0) + t;
+            if (tok_id) tok_id[r] = t == 0 ? (bonus_ids ? bonus_ids[i] : -1) : (draft_ids ? draft_ids[i * gamma + (t - 1)] : -1);
+        }
+    free(frontier);
+    free(s);
+    return ORACLE_OK;
+}
+
+/*
+ * Rejection-sampling acceptance ("Standard RS then accepts with probability min(1, p(z)/q(z)) and,
+ * upon rejection, samples from the residual distribution proportional to (p - q)+; if the retained
+ * block is fully accepted, the bonus token is sampled directly from the next target distribution").
+ * p = softmax of the target logits row (cu_q[i] + t), q = softmax of the draft logits row (i, t),
+ * both at temperature 1, in double.  The random numbers are inputs: u_accept[i, t] decides draft
+ * t + 1 of request i (accepted iff u * q(z) < p(z)), u_sample[i] draws the one token that ends the
+ * request's step by inversion over ascending token index (the smallest v whose cumulative weight
+ * exceeds u * total; all weights zero -> the same draw from p).
+ * Outputs as oracle_accept; out_prob (optional) = the probabilities the decisions used:
+ * [i][0] = p(z) / q(z) of the first rejected draft (or of the last accepted one), [i][1] = total
+ * residual mass (0 when the block was fully accepted).
+ */
+static void softmax_row(const uint16_t* row, int V, double* out) {
+    double m = -INFINITY;
+    for (int v = 0; v < V; ++v) {
+        const double x = (double)bf16_to_float(row[v]);
+        if (x > m) m = x;
+    }
+    double z = 0.0;
+    for (int v = 0; v < V; ++v) {
+        out[v] = exp((double)bf16_to_float(row[v]) - m);
+        z += out[v];
+    }
+    for (int v = 0; v < V; ++v) out[v] /= z;
+}
+
+static int inverse_cdf(const double* w, int V, double u) {
+    double total = 0.0;
+    for (int v = 0; v < V; ++v) total += w[v];
+    if (!(total > 0.0)) return -1;
+    const double target = u * total;
+    double run = 0.0;
+    int last = 0;
+    for (int v = 0; v < V; ++v) {
+        if (w[v] > 0.0) last = v;
+        run += w[v];
+        if (run > target) return v;
+    }
+    return last;   /* rounding left run == target at the end */
+}
+
+int oracle_accept_rs(const uint16_t* target_logits, const uint16_t* draft_logits, int V, const int32_t* draft_ids,
+                     const int32_t* cu_q, int B, int gamma, const float* u_accept, const float* u_sample,
+                     int32_t* accept_len, int32_t* bonus, int32_t* out_tokens, int32_t* n_accepted_total,
+                     double* out_prob) {
+    if (!target_logits || !draft_logits || !draft_ids || !cu_q || !u_accept || !u_sample || !accept_len || !bonus || V < 1)
+        return ORACLE_EINVAL;
+    double* p = (double*)malloc(sizeof(double) * (size_t)V);
+    double* q = (double*)malloc(sizeof(double) * (size_t)V);
+    int total = 0, rc = ORACLE_OK;
+    for (int i = 0; i < B && rc == ORACLE_OK; ++i) {
+        const int d = cu_q[i + 1] - cu_q[i] - 1;
+        int m = 0, tok = -1;
+        double ratio = 0.0, mass = 0.0;
+        for (; m < d; ++m) {
+            const int z = draft_ids[i * gamma + m];
+            if (z < 0 || z >= V) { rc = ORACLE_EINVAL; break; }
+            softmax_row(target_logits + (size_t)(cu_q[i] + m) * V, V, p);
+            softmax_row(draft_logits + ((size_t)i * gamma + m) * V, V, q);
+            ratio = p[z] / q[z];
+            if ((double)u_accept[i * gamma + m] * q[z] < p[z]) continue;   /* accepted */
+            for (int v = 0; v < V; ++v) {
+                q[v] = p[v] > q[v] ? p[v] - q[v] : 0.0;                    /* residual (p - q)+ */
+                mass += q[v];
+            }
+            tok = inverse_cdf(q, V, (double)u_sample[i]);
+            if (tok < 0) tok = inverse_cdf(p, V, (double)u_sample[i]);
+            break;
+        }
+        if (rc != ORACLE_OK) break;
+        if (tok < 0) {   /* every retained draft accepted: the bonus comes from the next target distribution */
+            softmax_row(target_logits + (size_t)(cu_q[i] + d) * V, V, p);
+            tok = inverse_cdf(p, V, (double)u_sample[i]);
+            m = d;
+        }
+        accept_len[i] = m;
+        bonus[i] = tok;
+        total += m + 1;
+        if (out_tokens)
+            for (int t = 0; t <= gamma; ++t)
+                out_tokens[i * (gamma + 1) + t] = t < m ? draft_ids[i * gamma + t] : (t == m ? tok : -1);
+        if (out_prob) {
+            out_prob[2 * i] = ratio;
+            out_prob[2 * i + 1] = mass;
+        }
+    }
+    if (n_accepted_total) *n_accepted_total = total;
+    free(p);
+    free(q);
+    return rc;
 }

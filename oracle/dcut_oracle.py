@@ -140,6 +140,74 @@ def select(conf, draft_ids, bonus_ids, ctx_lens, cost_ms, bucket_K: Optional[Seq
                         info.candidate, bool(info.closure_ok), info.sum_fixed, info.objective, info.sum_f64)
 
 
+def scores_shifted(conf: np.ndarray) -> np.ndarray:
+    """Eq. 7: the admission score of depth k is the product of the confidences before k."""
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    B, g = conf.shape
+    out = np.empty((B, g), dtype=np.float32)
+    rc = lib().oracle_scores_shifted(_p(conf, C.c_float), B, g, _p(out, C.c_float))
+    assert rc == 0, rc
+    return out
+
+
+def select_causal(conf, draft_ids, bonus_ids, ctx_lens, cost_ms) -> SelectResult:
+    """Causal early-stopping frontier scan on the shifted scores (dense cost table); `ranks` is not filled."""
+    conf = np.ascontiguousarray(conf, dtype=np.float32)
+    B, g = conf.shape
+    draft_ids, bonus_ids, ctx_lens = _i32(draft_ids).reshape(B, g), _i32(bonus_ids), _i32(ctx_lens)
+    cost_ms = np.ascontiguousarray(cost_ms, dtype=np.float32)
+    cap = B * (g + 1)
+    depths = np.zeros(B, np.int32)
+    cu_q = np.zeros(B + 1, np.int32)
+    tok_req = np.full(max(cap, 1), -1, np.int32)
+    tok_pos = np.full(max(cap, 1), -1, np.int32)
+    tok_id = np.full(max(cap, 1), -1, np.int32)
+    sc = np.zeros((B, g), np.float32)
+    info = _Info()
+    rc = lib().oracle_select_causal(_p(conf, C.c_float), B, g, _p(draft_ids, C.c_int32), _p(bonus_ids, C.c_int32),
+                                    _p(ctx_lens, C.c_int32), _p(cost_ms, C.c_float), len(cost_ms),
+                                    _p(depths, C.c_int32), _p(cu_q, C.c_int32), _p(tok_req, C.c_int32),
+                                    _p(tok_pos, C.c_int32), _p(tok_id, C.c_int32), _p(sc, C.c_float), C.byref(info))
+    if rc != 0:
+        raise OracleError(rc)
+    T = info.t_total
+    return SelectResult(depths, cu_q, tok_req[:T], tok_pos[:T], tok_id[:T], np.zeros((B, g), np.int32), sc, info.n_star,
+                        T, info.candidate, bool(info.closure_ok), info.sum_fixed, info.objective, info.sum_f64)
+
+
+@dataclass
+class AcceptRsResult:
+    accept_len: np.ndarray
+    bonus: np.ndarray
+    out_tokens: np.ndarray
+    n_accepted_total: int
+    prob: np.ndarray       # [B, 2]: p(z)/q(z) of the deciding draft, residual mass (0 if fully accepted)
+
+
+def accept_rs(target_logits, draft_logits, draft_ids, cu_q, gamma: int, u_accept, u_sample) -> AcceptRsResult:
+    """Rejection-sampling acceptance; target_logits bf16 [T, V], draft_logits bf16 [B, gamma, V], u_accept fp32
+    [B, gamma], u_sample fp32 [B]."""
+    tb, db = _bf16_bits(target_logits), _bf16_bits(draft_logits)
+    T, V = tb.shape
+    cu_q = _i32(cu_q)
+    B = len(cu_q) - 1
+    assert int(cu_q[B]) <= T and db.size == B * gamma * V
+    draft_ids = _i32(draft_ids).reshape(B, gamma)
+    ua = np.ascontiguousarray(u_accept, dtype=np.float32).reshape(B, gamma)
+    us = np.ascontiguousarray(u_sample, dtype=np.float32).reshape(B)
+    al, bo = np.zeros(B, np.int32), np.zeros(B, np.int32)
+    ot = np.zeros((B, gamma + 1), np.int32)
+    tot = C.c_int32(0)
+    prob = np.zeros((B, 2), np.float64)
+    f = lib().oracle_accept_rs
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 7
+    rc = f(tb.ctypes.data, db.ctypes.data, V, draft_ids.ctypes.data, cu_q.ctypes.data, B, gamma, ua.ctypes.data,
+           us.ctypes.data, al.ctypes.data, bo.ctypes.data, ot.ctypes.data, C.addressof(tot), prob.ctypes.data)
+    if rc != 0:
+        raise OracleError(rc)
+    return AcceptRsResult(al, bo, ot, tot.value, prob)
+
+
 def verify_attn(q, k_cache, v_cache, block_table, ctx_lens, cu_q, n_q_heads, n_kv_heads, head_dim,
                 page_size, scale=None, sample_tok=None, sample_head=None):
     """Returns (out, lse) in float64: [T, Hq, Dh], [T, Hq], or [n, Dh], [n] for sampled rows."""
