@@ -193,6 +193,46 @@ dcut_status dcut_layer_forward(dcut_ctx* ctx, const dcut_layer_weights* weights,
                                int T_cap, void* stream);
 
 /*
+ * Stochastic variant, selection (Appendix B "Causality under Rejection Sampling").  Same arguments and outputs as
+ * dcut_select, with two differences.  (1) The ranking score of draft depth k is the SHIFTED score of Eq. 7,
+ * s~_{i,1} = 1, s~_{i,k} = prod_{t<k} c_{i,t}: it does not depend on the proposal at depth k itself (scores_out
+ * returns these).  (2) With a dense cost table the budget comes from the causal early-stopping scan: positions are
+ * admitted in ranked order (the order in which the per-request frontiers would be exposed; ties by shallower depth,
+ * then request index) while the objective (B + sum of admitted shifted scores) / cost(B + N) strictly improves, and
+ * the scan stops at the first position that does not improve it - it may miss a later optimum of a curve that is not
+ * unimodal, as the appendix says.  With exactly one bucket (set through dcut_set_cost_buckets) the budget is that
+ * bucket's K, fixed before the block is seen (the appendix's history-determined K); more buckets -> DCUT_ECOST.
+ * info.candidate = N*.  Same fixed-point sum and fp64 objective as dcut_select.
+ */
+dcut_status dcut_select_causal(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
+                               const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q, int* tok_req,
+                               int* tok_pos, int* tok_id, dcut_select_info* info, float* scores_out, int* ranks_out,
+                               void* stream);
+
+/*
+ * Stochastic variant, acceptance by rejection sampling (Appendix B: accept draft z with probability
+ * min(1, p(z)/q(z)); upon the first rejection sample from the residual distribution proportional to (p - q)+; if the
+ * retained block is fully accepted, sample the bonus token from the next target distribution).
+ *   p = softmax(target_logits[cu_q[i] + t, :]), q = softmax(draft_logits[i, t, :]), temperature 1, fp32.
+ *   Draft t + 1 of request i (token draft_ids[i, t]) is accepted iff u_accept[i, t] * q(z) < p(z).
+ *   The token that ends the request's step is drawn with u_sample[i] by inversion over ascending token index: the
+ *   smallest v whose cumulative weight exceeds u * total (weights (p - q)+ of the rejected position, or p of row
+ *   cu_q[i] + d_i when every retained draft was accepted; if (p - q)+ vanishes, p).
+ * The random numbers are inputs (uniform in [0, 1)); the library draws none.
+ * DEVICE in: target_logits bf16 [T, V]; draft_logits bf16 [B, gamma, V] (rows (i, t) with t >= d_i are not read);
+ * draft_ids int32 [B, gamma] in [0, V); cu_q; u_accept fp32 [B, gamma]; u_sample fp32 [B].
+ * DEVICE out: accept_len, bonus (the sampled token), out_tokens, n_accepted_total as in dcut_accept; prob fp32
+ * [B, 2] (optional, may be null): p(z)/q(z) of the deciding draft and the residual mass.
+ * Requirements: context created with vocab >= V.  Sums run in a fixed order, so results are reproducible; they are
+ * fp32 (double for the inversion), so a draw that falls within rounding of a boundary may differ from an fp64
+ * evaluation by one token.
+ */
+dcut_status dcut_accept_rs(dcut_ctx* ctx, const void* target_logits, const void* draft_logits, int V,
+                           const int* draft_ids, const int* cu_q, int B, int gamma, int T_cap, const float* u_accept,
+                           const float* u_sample, int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total,
+                           float* prob, void* stream);
+
+/*
  * LM head fused with acceptance (the step between the last layer and dcut_accept, Section 3.1: the target's next-token
  * prediction at every retained position): logits[T, V] = x[T, hidden] . w_lm[V, hidden]^T (bf16 in, fp32 accumulate,
  * rounded to bf16 exactly as if the logits were stored), reduced inside the GEMM's epilogue to the row's argmax

@@ -29,7 +29,7 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
            "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_lm_head_accept",
-           "dcut_poll_device_status"]
+           "dcut_select_causal", "dcut_accept_rs", "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -62,6 +62,8 @@ _lib.dcut_set_cost_dense.argtypes = [_vp, _vp, _i]
 _lib.dcut_set_cost_buckets.argtypes = [_vp, _i, _i, _vp, _vp, _i]
 _lib.dcut_budget_from_ratio.argtypes = [_i, _i, _i, _i, C.POINTER(_i)]
 _lib.dcut_select.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
+_lib.dcut_select_causal.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
+_lib.dcut_accept_rs.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i] + [_vp] * 8
 _lib.dcut_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _i, _i, _f, _vp, _vp, _vp]
 _lib.dcut_accept.argtypes = [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.dcut_poll_device_status.argtypes = [_vp, C.POINTER(_i), _vp]
@@ -186,7 +188,8 @@ class Context:
 
     # -- hot path ------------------------------------------------------------------------------
     def select(self, conf, draft_ids, bonus_ids, ctx_lens, out: Optional[SelectOut] = None,
-               want_scores: bool = False, want_ranks: bool = False) -> SelectOut:
+               want_scores: bool = False, want_ranks: bool = False, causal: bool = False) -> SelectOut:
+        """dcut_select, or dcut_select_causal (shifted scores + early-stopping scan) with causal=True."""
         B, gamma = conf.shape
         dev = conf.device
         if out is None:
@@ -197,7 +200,8 @@ class Context:
                             torch.zeros(4, dtype=torch.int64, device=dev),
                             torch.empty((B, gamma), dtype=torch.float32, device=dev) if want_scores else None,
                             torch.empty((B, gamma), **i32) if want_ranks else None)
-        self._check(_lib.dcut_select(self._h, _ptr(conf, torch.float32), B, gamma, _ptr(draft_ids, torch.int32),
+        fn = _lib.dcut_select_causal if causal else _lib.dcut_select
+        self._check(fn(self._h, _ptr(conf, torch.float32), B, gamma, _ptr(draft_ids, torch.int32),
                                      _ptr(bonus_ids, torch.int32), _ptr(ctx_lens, torch.int32),
                                      _ptr(out.depths), _ptr(out.cu_q), _ptr(out.tok_req), _ptr(out.tok_pos),
                                      _ptr(out.tok_id), _ptr(out.info), _ptr(out.scores), _ptr(out.ranks), _stream()))
@@ -217,6 +221,22 @@ class Context:
                                           float(scale), _ptr(out, torch.bfloat16), _ptr(lse, torch.float32),
                                           _stream()))
         return out
+
+    def accept_rs(self, target_logits, draft_logits, draft_ids, cu_q, T_cap: int, u_accept, u_sample,
+                  want_prob: bool = False):
+        """dcut_accept_rs: rejection-sampling acceptance; returns (accept_len, sampled token, out_tokens, total, prob)."""
+        B, gamma = draft_ids.shape
+        V = target_logits.shape[1]
+        dev_ = target_logits.device
+        i32 = dict(dtype=torch.int32, device=dev_)
+        accept_len, bonus = torch.empty(B, **i32), torch.empty(B, **i32)
+        toks, total = torch.empty((B, gamma + 1), **i32), torch.empty(1, **i32)
+        prob = torch.zeros((B, 2), dtype=torch.float32, device=dev_) if want_prob else None
+        self._check(_lib.dcut_accept_rs(self._h, _ptr(target_logits, torch.bfloat16), _ptr(draft_logits, torch.bfloat16), V,
+                                        _ptr(draft_ids, torch.int32), _ptr(cu_q, torch.int32), B, gamma, T_cap,
+                                        _ptr(u_accept, torch.float32), _ptr(u_sample, torch.float32), _ptr(accept_len),
+                                        _ptr(bonus), _ptr(toks), _ptr(total), _ptr(prob), _stream()))
+        return accept_len, bonus, toks, total, prob
 
     def accept(self, logits, draft_ids, cu_q, T_cap: int, out_tokens: bool = True):
         B, gamma = draft_ids.shape

@@ -52,6 +52,7 @@ void free_all(dcut_ctx* c) {
     cudaFree(c->d_part_o);
     cudaFree(c->d_part_lse);
     cudaFree(c->d_row_key);
+    cudaFree(c->d_rs_scratch);
     cudaFree(c->d_status);
     cudaFree(c->ly_norm);
     cudaFree(c->ly_qkv);
@@ -118,6 +119,13 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
     if ((st = dmalloc(c, &c->d_bucket_K, DCUT_MAX_BUCKETS, "cudaMalloc(bucket_K)")) != DCUT_OK) return st;
     if ((st = dmalloc(c, &c->d_row_key, max_T, "cudaMalloc(row_key)")) != DCUT_OK) return st;
     if ((st = dmalloc(c, &c->d_status, 4, "cudaMalloc(status)")) != DCUT_OK) return st;
+    if (lim->vocab > 0) {   // rejection-sampling acceptance: per-row softmax statistics of vocabulary segments of ~8k tokens
+        c->rs_n_seg = (lim->vocab + 8191) / 8192;
+        if (c->rs_n_seg > 32) c->rs_n_seg = 32;
+        unsigned char* p = nullptr;
+        if ((st = dmalloc(c, &p, dcut_accept_rs_scratch_bytes(c, c->rs_n_seg), "cudaMalloc(rs scratch)")) != DCUT_OK) return st;
+        c->d_rs_scratch = p;
+    }
     if ((st = dcut_init_select(c)) != DCUT_OK) return st;
     if ((st = dcut_init_accept(c)) != DCUT_OK) return st;
     if (has_attn) {
@@ -222,10 +230,12 @@ dcut_status dcut_budget_from_ratio(int B, int gamma, int num, int den, int* K) {
     return DCUT_OK;
 }
 
-dcut_status dcut_select(dcut_ctx* c, const float* conf, int B, int gamma, const int* draft_ids, const int* bonus_ids,
-                        const int* ctx_lens, int* depths, int* cu_q, int* tok_req, int* tok_pos, int* tok_id,
-                        dcut_select_info* info, float* scores_out, int* ranks_out, void* stream) {
+static dcut_status select_common(dcut_ctx* c, const float* conf, int B, int gamma, const int* draft_ids, const int* bonus_ids,
+                                 const int* ctx_lens, int* depths, int* cu_q, int* tok_req, int* tok_pos, int* tok_id,
+                                 dcut_select_info* info, float* scores_out, int* ranks_out, int causal, void* stream) {
     if (!c) return DCUT_EINVAL;
+    if (causal && c->n_buckets > 1)
+        return dcut_fail(c, DCUT_ECOST, "the causal selector takes a dense cost table or exactly one bucket (a budget fixed beforehand)");
     if (!conf || !depths || !cu_q) return dcut_fail(c, DCUT_EINVAL, "conf, depths and cu_q must not be null");
     if (B < 1 || gamma < 1) return dcut_fail(c, DCUT_EINVAL, "B and gamma must be >= 1");
     if (B > c->lim.max_B || gamma > c->lim.max_gamma) return dcut_fail(c, DCUT_ECAPACITY, "B = %d, gamma = %d exceed the limits (%d, %d)", B, gamma, c->lim.max_B, c->lim.max_gamma);
@@ -240,7 +250,22 @@ dcut_status dcut_select(dcut_ctx* c, const float* conf, int B, int gamma, const 
         return dcut_fail(c, DCUT_ECOST, "dense cost table has %d entries, need %d", c->cost_n, B * (gamma + 1) + 1);
     }
     return dcut_launch_select(c, conf, B, gamma, draft_ids, bonus_ids, ctx_lens, depths, cu_q, tok_req, tok_pos, tok_id,
-                              info, scores_out, ranks_out, static_cast<cudaStream_t>(stream));
+                              info, scores_out, ranks_out, causal, static_cast<cudaStream_t>(stream));
+}
+
+dcut_status dcut_select(dcut_ctx* c, const float* conf, int B, int gamma, const int* draft_ids, const int* bonus_ids,
+                        const int* ctx_lens, int* depths, int* cu_q, int* tok_req, int* tok_pos, int* tok_id,
+                        dcut_select_info* info, float* scores_out, int* ranks_out, void* stream) {
+    return select_common(c, conf, B, gamma, draft_ids, bonus_ids, ctx_lens, depths, cu_q, tok_req, tok_pos, tok_id, info,
+                         scores_out, ranks_out, 0, stream);
+}
+
+dcut_status dcut_select_causal(dcut_ctx* c, const float* conf, int B, int gamma, const int* draft_ids,
+                               const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q, int* tok_req,
+                               int* tok_pos, int* tok_id, dcut_select_info* info, float* scores_out, int* ranks_out,
+                               void* stream) {
+    return select_common(c, conf, B, gamma, draft_ids, bonus_ids, ctx_lens, depths, cu_q, tok_req, tok_pos, tok_id, info,
+                         scores_out, ranks_out, 1, stream);
 }
 
 dcut_status dcut_verify_attn(dcut_ctx* c, const void* q, const void* k_cache, const void* v_cache, long long num_pages,
@@ -276,6 +301,21 @@ dcut_status dcut_accept(dcut_ctx* c, const void* logits, int V, const int* draft
     if (reinterpret_cast<uintptr_t>(logits) & 1) return dcut_fail(c, DCUT_EINVAL, "logits must be 2-byte aligned");
     return dcut_launch_accept(c, logits, V, draft_ids, cu_q, B, gamma, T_cap, accept_len, bonus, out_tokens,
                               n_accepted_total, c->d_row_key, static_cast<cudaStream_t>(stream));
+}
+
+dcut_status dcut_accept_rs(dcut_ctx* c, const void* target_logits, const void* draft_logits, int V, const int* draft_ids,
+                           const int* cu_q, int B, int gamma, int T_cap, const float* u_accept, const float* u_sample,
+                           int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, float* prob, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (!c->d_rs_scratch) return dcut_fail(c, DCUT_EINVAL, "context was created with vocab = 0");
+    if (!target_logits || !draft_logits || !draft_ids || !cu_q || !u_accept || !u_sample || !accept_len || !bonus)
+        return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (B < 1 || gamma < 1 || V < 1 || T_cap < B) return dcut_fail(c, DCUT_EINVAL, "need B, gamma, V >= 1 and T_cap >= B");
+    if (B > c->lim.max_B || gamma > c->lim.max_gamma || T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
+        return dcut_fail(c, DCUT_ECAPACITY, "B = %d, gamma = %d, T_cap = %d exceed the limits", B, gamma, T_cap);
+    if (V > c->lim.vocab) return dcut_fail(c, DCUT_ECAPACITY, "V = %d exceeds the limit %d", V, c->lim.vocab);
+    return dcut_launch_accept_rs(c, target_logits, draft_logits, V, draft_ids, cu_q, B, gamma, T_cap, u_accept, u_sample,
+                                 accept_len, bonus, out_tokens, n_accepted_total, prob, static_cast<cudaStream_t>(stream));
 }
 
 dcut_status dcut_gemm_bf16(dcut_ctx* c, const void* a, const void* w, const void* w2, int mode, int N, int K,

@@ -61,6 +61,10 @@ struct dcut_ctx {
     // accept scratch
     unsigned long long* d_row_key;   // [max_T] packed (ordered max, ~index); zero between calls
 
+    // rejection-sampling acceptance scratch (vocab > 0 only)
+    void* d_rs_scratch;
+    int rs_n_seg;
+
     int* d_status;          // device status word
 
     // tensor-map encoder (driver entry point fetched through the runtime)
@@ -103,11 +107,16 @@ void dcut_free_layer(dcut_ctx* ctx);
 dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
                                const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q,
                                int* tok_req, int* tok_pos, int* tok_id, dcut_select_info* info,
-                               float* scores_out, int* ranks_out, cudaStream_t stream);
+                               float* scores_out, int* ranks_out, int causal, cudaStream_t stream);
 dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids,
                                const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
                                int* out_tokens, int* n_accepted_total, unsigned long long* row_key,
                                cudaStream_t stream);
+size_t dcut_accept_rs_scratch_bytes(const dcut_ctx* ctx, int n_seg);
+dcut_status dcut_launch_accept_rs(dcut_ctx* ctx, const void* target_logits, const void* draft_logits, int V,
+                                  const int* draft_ids, const int* cu_q, int B, int gamma, int T_cap,
+                                  const float* u_accept, const float* u_sample, int* accept_len, int* bonus,
+                                  int* out_tokens, int* n_accepted_total, float* prob, cudaStream_t stream);
 dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                     long long num_pages, const int* block_table, int block_table_stride,
                                     const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,

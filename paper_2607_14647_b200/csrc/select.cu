@@ -34,6 +34,7 @@ struct SelectArgs {
     const float* cost;      // dense: cost[T]; bucket: cost[c]
     const int* bucket_K;    // bucket mode only
     int n_buckets;          // 0 = dense
+    int causal;             // 1: shifted scores (Eq. 7); dense table: early-stopping scan instead of the argmax
     int B, gamma, npad;
     int* depths;
     int* cu_q;
@@ -185,10 +186,13 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     for (int e = tid; e < n; e += kThreads) conf_s[e] = a.conf[e];
     __syncthreads();
     for (int i = tid; i < B; i += kThreads) {
-        float p = 1.0f;
+        float prev = 1.0f;
         for (int k = 0; k < gamma; ++k) {
-            p = __fmul_rn(p, clamp_conf(conf_s[i * gamma + k]));
-            if (p == 0.0f) p = 0.0f;   // -0 -> +0
+            float nxt = __fmul_rn(prev, clamp_conf(conf_s[i * gamma + k]));
+            if (nxt == 0.0f) nxt = 0.0f;   // -0 -> +0
+            // Eq. 3: the score of depth k + 1 includes its own confidence; Eq. 7 (causal mode): only those before it
+            const float p = a.causal ? prev : nxt;
+            prev = nxt;
             if (a.scores_out) a.scores_out[(size_t)i * gamma + k] = p;
             const unsigned int bits = __float_as_uint(p);
             keys[i * gamma + k] = ((unsigned long long)(0xffffffffu - bits) << 32) |
@@ -238,7 +242,35 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
 
     SELP(long long t3 = clock64();)
     // 4. objective over the candidates
-    {
+    if (a.causal && a.n_buckets == 0) {
+        // Causal early-stopping scan (Appendix B): positions are admitted in ranked order while the objective strictly
+        // improves, so N* is the first N whose successor is not better.  A request's shifted scores never increase
+        // with depth, so the ranked order is the order in which the frontiers would be exposed.
+        const long long bfix = (long long)B << 40;
+        int first = n;
+        for (int c = tid; c < n; c += kThreads) {
+            const double o0 = __ddiv_rn(__ll2double_rn(bfix + qs[c]), (double)a.cost[B + c]);
+            const double o1 = __ddiv_rn(__ll2double_rn(bfix + qs[c + 1]), (double)a.cost[B + c + 1]);
+            if (!(o1 > o0)) {
+                first = c;
+                break;          // this thread's later candidates are larger
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
+        if (lane == 0) ws32[warp] = first;
+        __syncthreads();
+        if (warp == 0) {
+            first = ws32[lane];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
+            if (lane == 0) {
+                Best b = {__ddiv_rn(__ll2double_rn(bfix + qs[first]), (double)a.cost[B + first]), first, first};
+                best_s = b;
+            }
+        }
+        __syncthreads();
+    } else {
         const long long bfix = (long long)B << 40;
         Best b = {-1.0, INT_MAX, -1};
         const int n_cand = a.n_buckets > 0 ? a.n_buckets : n + 1;
@@ -354,7 +386,7 @@ dcut_status dcut_init_select(dcut_ctx* ctx) {
 dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
                                const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q,
                                int* tok_req, int* tok_pos, int* tok_id, dcut_select_info* info,
-                               float* scores_out, int* ranks_out, cudaStream_t stream) {
+                               float* scores_out, int* ranks_out, int causal, cudaStream_t stream) {
     const int n = B * gamma;
     int npad = 32;
     while (npad < n) npad <<= 1;
@@ -366,6 +398,7 @@ dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamm
     a.cost = ctx->d_cost;
     a.bucket_K = ctx->d_bucket_K;
     a.n_buckets = ctx->n_buckets;
+    a.causal = causal;
     a.B = B;
     a.gamma = gamma;
     a.npad = npad;

@@ -31,6 +31,7 @@ import torch
 _TAG_CONF, _TAG_IDS, _TAG_CTX, _TAG_REJECT, _TAG_PAGES, _TAG_KV, _TAG_Q, _TAG_LOGITS = range(1, 9)
 _TAG_LAYER_X, _TAG_LAYER_W = 9, 10
 _TAG_LM_W, _TAG_LM_X = 11, 12
+_TAG_DRAFT_LOGITS, _TAG_UNIFORM = 13, 14
 
 
 @dataclass(frozen=True)
@@ -317,3 +318,29 @@ def lm_head_x_rows(cfg: WorkloadConfig, sel: SelectInputs, depths: np.ndarray, w
                 rng = np.random.default_rng([cfg.seed, _TAG_LM_X, i, t])
                 out[cu[i] + t] = torch.from_numpy(rng.standard_normal(H, dtype=np.float32)).to(torch.bfloat16)
     return out
+
+
+# --------------------------------------------------------------------------- stochastic variant inputs
+
+def draft_logits_rows(cfg: WorkloadConfig, target_rows: torch.Tensor, depths: np.ndarray, noise: float = 0.7,
+                      vocab: Optional[int] = None) -> torch.Tensor:
+    """Drafter logits bf16 [B, gamma, V]: row (i, t) = the target row that verifies draft t + 1 of request i plus
+    N(0, noise^2) per token (a drafter that tracks the target imperfectly, so p(z)/q(z) scatters around 1); rows
+    t >= d_i have no target row and are ~ N(0, 1).  One counter-seeded draw per (i, t)."""
+    V = cfg.vocab if vocab is None else vocab
+    cu = cu_q_from_depths(depths)
+    out = torch.empty((cfg.B, cfg.gamma, V), dtype=torch.bfloat16)
+    for i, d in enumerate(depths):
+        for t in range(cfg.gamma):
+            rng = np.random.default_rng([cfg.seed, _TAG_DRAFT_LOGITS, i, t])
+            r = torch.from_numpy(rng.standard_normal(V, dtype=np.float32))
+            if t < int(d):
+                r = target_rows[cu[i] + t].float() + noise * r
+            out[i, t] = r.to(torch.bfloat16)
+    return out
+
+
+def uniforms(cfg: WorkloadConfig):
+    """The random numbers of rejection-sampling acceptance: u_accept fp32 [B, gamma], u_sample fp32 [B], in [0, 1)."""
+    rng = np.random.default_rng([cfg.seed, _TAG_UNIFORM])
+    return rng.random((cfg.B, cfg.gamma), dtype=np.float32), rng.random(cfg.B, dtype=np.float32)
