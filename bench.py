@@ -464,6 +464,42 @@ def run_dcut(args):
         except Exception as exc:   # the extra measurement must not take the bench line down
             gemm["lm_head"] = {"error": repr(exc)[:200]}
 
+    # ---- stochastic variant (causal selector + rejection-sampling acceptance), timed alone at full depth ----------
+    stochastic = None
+    if not is_layer and rank == 0:
+        try:
+            def timed_us(fn, n=20):
+                for _ in range(3):
+                    fn()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(n):
+                    fn()
+                e1.record()
+                e1.synchronize()
+                return e0.elapsed_time(e1) / n * 1e3
+
+            ctx.set_cost_dense(cost)
+            t_sel = timed_us(lambda: ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=sel_out))
+            t_selc = timed_us(lambda: ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=sel_out, causal=True))
+            full = np.full(cfg.B, cfg.gamma, np.int32)
+            cu_full = torch.from_numpy(wl.cu_q_from_depths(full)).to(dev)
+            # drafter logits: the target rows plus noise (generated on the device; the values do not change the traffic)
+            idx = torch.from_numpy(np.concatenate([i * (cfg.gamma + 1) + np.arange(cfg.gamma) for i in range(cfg.B)])).to(dev)
+            d_dl = d_logits_all.index_select(0, idx).view(cfg.B, cfg.gamma, cfg.vocab).contiguous()
+            d_dl += (0.3 * torch.randn(d_dl.shape, device=dev, dtype=torch.float32)).to(torch.bfloat16)
+            ua_np, us_np = wl.uniforms(cfg)
+            d_ua, d_us = torch.from_numpy(ua_np).to(dev), torch.from_numpy(us_np).to(dev)
+            dr = (d_draft % cfg.vocab).contiguous()
+            t_rs = timed_us(lambda: ctx.accept_rs(d_logits_all, d_dl, dr, cu_full, cap, d_ua, d_us), n=10)
+            rs_bytes = 2 * cfg.vocab * (cfg.t_cap + cfg.B * cfg.gamma)
+            stochastic = {"select_us": round(t_sel, 2), "select_causal_us": round(t_selc, 2),
+                          "accept_rs_us": round(t_rs, 1), "accept_rs_scan_bytes": rs_bytes,
+                          "accept_rs_gbs": round(rs_bytes / (t_rs * 1e-6) / 1e9, 1)}
+            del d_dl
+        except Exception as exc:   # the extra measurement must not take the bench line down
+            stochastic = {"error": repr(exc)[:200]}
+
     if rank != 0:
         return
     pk = peaks()
@@ -496,6 +532,8 @@ def run_dcut(args):
         "cost_table_ms": {str(t): round(c, 4) for t, c in zip(grid, prof)},
         "clocks": clocks,
     }
+    if stochastic is not None:
+        line["stochastic"] = stochastic
     if is_layer:
         pkj = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
         tf_peak = float(pkj.get("bf16_tflops", 1590.0))

@@ -223,7 +223,7 @@ dcut_status dcut_select_causal(dcut_ctx* ctx, const float* conf, int B, int gamm
  * draft_ids int32 [B, gamma] in [0, V); cu_q; u_accept fp32 [B, gamma]; u_sample fp32 [B].
  * DEVICE out: accept_len, bonus (the sampled token), out_tokens, n_accepted_total as in dcut_accept; prob fp32
  * [B, 2] (optional, may be null): p(z)/q(z) of the deciding draft and the residual mass.
- * Requirements: context created with vocab >= V.  Sums run in a fixed order, so results are reproducible; they are
+ * Requirements: context created with vocab >= V; V <= 262 144.  Sums run in a fixed order, so results are reproducible; they are
  * fp32 (double for the inversion), so a draw that falls within rounding of a boundary may differ from an fp64
  * evaluation by one token.
  */

@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kStatThreads) rs_stats_kernel(RsArgs a) {
     }
     const int start = seg * a.seg_elems, end = min(a.V, start + a.seg_elems);
     float m = -INFINITY, s = 0.0f;
-    auto take = [&](float x) {
+    auto take = [&](float x) {           // scalar head / tail elements
         if (x > m) {
             s = s * __expf(m - x) + 1.0f;   // m = -inf: s is 0, the product is 0 * 0
             m = x;
@@ -78,12 +78,27 @@ __global__ void __launch_bounds__(kStatThreads) rs_stats_kernel(RsArgs a) {
         const int nvec = (end - start - head) >> 3;
         const uint4* vp = reinterpret_cast<const uint4*>(rp + start + head);
         for (int k = threadIdx.x; k < nvec; k += kStatThreads) {
+            // eight values at a time: one rescale of the running sum per vector, no data-dependent branch
             const uint4 w = ld_stream_v4(vp + k);
             const unsigned int ws[4] = {w.x, w.y, w.z, w.w};
+            float x[8];
+            float vmax = -INFINITY;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                take(__uint_as_float(ws[e] << 16));
-                take(__uint_as_float(ws[e] & 0xffff0000u));
+                x[2 * e] = __uint_as_float(ws[e] << 16);
+                x[2 * e + 1] = __uint_as_float(ws[e] & 0xffff0000u);
+                vmax = fmaxf(vmax, fmaxf(x[2 * e], x[2 * e + 1]));   // fmaxf drops NaN
+            }
+            const float mn = fmaxf(m, vmax);
+            if (mn > -INFINITY) {
+                float add = 0.0f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float t = __expf(x[e] - mn);                // -inf -> 0; NaN -> NaN
+                    add += (t == t) ? t : 0.0f;
+                }
+                s = s * __expf(m - mn) + add;
+                m = mn;
             }
         }
         for (int v = start + head + nvec * 8 + threadIdx.x; v < end; v += kStatThreads) take(bf_at(rp, v));
@@ -202,7 +217,12 @@ __device__ __forceinline__ T block_exclusive_scan_d(T v, T* ws, T* total) {
     return res;
 }
 
-// One CTA per request: the token that ends the request's step.
+// One CTA per request: the token that ends the request's step.  The vocabulary is cut into chunks of 256 tokens;
+// warp w sums the chunks w, w + 32, ... (16-byte loads, lane l holds tokens 8l .. 8l+7 of the chunk), the chunk sums
+// are scanned in double, and one warp rescans the chunk that holds u * total.
+constexpr int kChunk = 256;
+constexpr int kMaxChunks = 1024;   // vocabularies up to 262 144 tokens
+
 __global__ void __launch_bounds__(kSampleThreads) rs_sample_kernel(RsArgs a) {
     const int i = blockIdx.x;
     const int4 job = a.job[i];
@@ -210,11 +230,14 @@ __global__ void __launch_bounds__(kSampleThreads) rs_sample_kernel(RsArgs a) {
     const unsigned short* tp = a.target + (size_t)job.x * a.V;
     const unsigned short* dp = job.y >= 0 ? a.draft + (size_t)job.y * a.V : nullptr;
     __shared__ double ws[33];
+    __shared__ double csum[kMaxChunks];
     __shared__ int found_s, last_s;
-    const int per = (a.V + kSampleThreads - 1) / kSampleThreads;
-    const int v0 = min(a.V, (int)threadIdx.x * per), v1 = min(a.V, v0 + per);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_chunks = (a.V + kChunk - 1) / kChunk;
     const float inv_p = 1.0f / st.y, inv_q = dp ? 1.0f / st.w : 0.0f;
     bool use_p = dp == nullptr;
+    int tok = 0;
+    double mass = 0.0;
     for (int round = 0; round < 2; ++round) {
         auto weight = [&](int v) -> float {
             const float p = __expf(bf_at(tp, v) - st.x) * inv_p;
@@ -223,60 +246,90 @@ __global__ void __launch_bounds__(kSampleThreads) rs_sample_kernel(RsArgs a) {
             const float r = p - q;
             return r > 0.0f ? r : 0.0f;
         };
+        // the eight weights of this lane in chunk c, in token order (scalar loads: rows need not be 16-byte aligned)
+        auto lane_weights = [&](int c, float (&w)[8]) {
+            const int v0 = c * kChunk + lane * 8;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) w[e] = v0 + e < a.V ? weight(v0 + e) : 0.0f;
+        };
         if (threadIdx.x == 0) {
-            found_s = a.V;
+            found_s = n_chunks;
             last_s = -1;
         }
-        double local = 0.0;
         int my_last = -1;
-        for (int v = v0; v < v1; ++v) {
-            const float w = weight(v);
-            local += (double)w;
-            if (w > 0.0f) my_last = v;
+        for (int c = warp; c < n_chunks; c += kSampleThreads / 32) {
+            float w[8];
+            lane_weights(c, w);
+            double part = 0.0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                part += (double)w[e];
+                if (w[e] > 0.0f) my_last = c * kChunk + lane * 8 + e;
+            }
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {   // inclusive scan over the lanes (fixed order), lane 31 ends with the chunk sum
+                const double u = __shfl_up_sync(0xffffffffu, part, o);
+                if (lane >= o) part += u;
+            }
+            if (lane == 31) csum[c] = part;
         }
+        __syncthreads();
         double total;
-        const double before = block_exclusive_scan_d<double>(local, ws, &total);   // also orders the writes above
+        const double mine = (int)threadIdx.x < n_chunks ? csum[threadIdx.x] : 0.0;
+        const double before = block_exclusive_scan_d<double>(mine, ws, &total);
         if (my_last >= 0) atomicMax(&last_s, my_last);
         if (!(total > 0.0)) {
-            // (p - q)+ vanished in this precision: the same draw from p (once)
-            if (use_p) break;
-            use_p = true;
+            if (use_p) break;        // no positive weight at all (a row of NaN): token 0
+            use_p = true;            // (p - q)+ vanished in this precision: the same draw from p
+            __syncthreads();
             continue;
         }
         const double target = (double)a.u_sample[i] * total;
-        if (target >= before && target < before + local) {
-            double run = before;
-            for (int v = v0; v < v1; ++v) {
-                run += (double)weight(v);
-                if (run > target) {
-                    atomicMin(&found_s, v);
-                    break;
-                }
-            }
-        }
+        if ((int)threadIdx.x < n_chunks && target >= before && target < before + mine) atomicMin(&found_s, (int)threadIdx.x);
         __syncthreads();
-        if (threadIdx.x == 0) {
-            const int tok = found_s < a.V ? found_s : max(last_s, 0);   // rounding left the running sum at the target
-            const int m = job.z;
-            a.bonus[i] = tok;
-            if (a.prob) a.prob[2 * i + 1] = (dp && !use_p) ? (float)total : 0.0f;   // residual mass
-            if (a.out_tokens) {
-                int* o = a.out_tokens + (size_t)i * (a.gamma + 1);
-                for (int t = 0; t <= a.gamma; ++t) o[t] = t < m ? a.draft_ids[(size_t)i * a.gamma + t] : (t == m ? tok : -1);
+        mass = (dp && !use_p) ? total : 0.0;
+        const int c = found_s;
+        tok = max(last_s, 0);        // if rounding left the running sum at the target: the last token with weight
+        if (c < n_chunks) {
+            // every warp resolves the chunk the same way (cheaper than electing one and broadcasting)
+            double base;
+            float w[8];
+            lane_weights(c, w);
+            double part = 0.0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) part += (double)w[e];
+            double inc = part;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double u = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += u;
             }
-            if (a.n_accepted_total) atomicAdd(a.n_accepted_total, m + 1);
+            // prefix of the chunk = scan value of thread c; recompute it the same way: sum of csum[0..c) in scan order
+            // is what thread c holds in `before`; fetch it through shared memory
+            if ((int)threadIdx.x == c) ws[0] = before;
+            __syncthreads();
+            base = ws[0];
+            double run = base + inc - part;     // weight before this lane's first token
+            int hit = -1;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                run += (double)w[e];
+                if (hit < 0 && run > target) hit = c * kChunk + lane * 8 + e;
+            }
+            const unsigned int mask = __ballot_sync(0xffffffffu, hit >= 0);
+            if (mask) tok = __shfl_sync(0xffffffffu, hit, __ffs(mask) - 1);
         }
-        return;
+        break;
     }
-    // no positive weight at all (a row of NaN): token 0
     if (threadIdx.x == 0) {
-        a.bonus[i] = 0;
-        if (a.prob) a.prob[2 * i + 1] = 0.0f;
+        const int m = job.z;
+        a.bonus[i] = tok;
+        if (a.prob) a.prob[2 * i + 1] = (float)mass;   // residual mass (0 when the draw came from p)
         if (a.out_tokens) {
             int* o = a.out_tokens + (size_t)i * (a.gamma + 1);
-            for (int t = 0; t <= a.gamma; ++t) o[t] = t < job.z ? a.draft_ids[(size_t)i * a.gamma + t] : (t == job.z ? 0 : -1);
+            for (int t = 0; t <= a.gamma; ++t) o[t] = t < m ? a.draft_ids[(size_t)i * a.gamma + t] : (t == m ? tok : -1);
         }
-        if (a.n_accepted_total) atomicAdd(a.n_accepted_total, job.z + 1);
+        if (a.n_accepted_total) atomicAdd(a.n_accepted_total, m + 1);
     }
 }
 
@@ -307,8 +360,15 @@ dcut_status dcut_launch_accept_rs(dcut_ctx* ctx, const void* target_logits, cons
     a.V = V;
     a.B = B;
     a.gamma = gamma;
-    a.n_seg = ctx->rs_n_seg;
-    a.seg_elems = ((V + a.n_seg - 1) / a.n_seg + 7) & ~7;
+    // segments: enough CTAs for a few waves over the SMs, at least ~16 KB each, at most what the scratch was sized for
+    const int n_rows = T_cap + B * gamma;
+    int n_seg = (ctx->sm_count * 16 + n_rows - 1) / n_rows;
+    const int max_seg = (V + 8191) / 8192;
+    if (n_seg > max_seg) n_seg = max_seg;
+    if (n_seg > ctx->rs_n_seg) n_seg = ctx->rs_n_seg;
+    if (n_seg < 1) n_seg = 1;
+    a.seg_elems = ((V + n_seg - 1) / n_seg + 7) & ~7;
+    a.n_seg = (V + a.seg_elems - 1) / a.seg_elems;
     a.T_cap = T_cap;
     unsigned char* base = static_cast<unsigned char*>(ctx->d_rs_scratch);
     a.stats = reinterpret_cast<float2*>(base);

@@ -313,7 +313,7 @@ dcut_status dcut_accept_rs(dcut_ctx* c, const void* target_logits, const void* d
     if (B < 1 || gamma < 1 || V < 1 || T_cap < B) return dcut_fail(c, DCUT_EINVAL, "need B, gamma, V >= 1 and T_cap >= B");
     if (B > c->lim.max_B || gamma > c->lim.max_gamma || T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
         return dcut_fail(c, DCUT_ECAPACITY, "B = %d, gamma = %d, T_cap = %d exceed the limits", B, gamma, T_cap);
-    if (V > c->lim.vocab) return dcut_fail(c, DCUT_ECAPACITY, "V = %d exceeds the limit %d", V, c->lim.vocab);
+    if (V > c->lim.vocab || V > 262144) return dcut_fail(c, DCUT_ECAPACITY, "V = %d exceeds the limit %d", V, c->lim.vocab < 262144 ? c->lim.vocab : 262144);
     return dcut_launch_accept_rs(c, target_logits, draft_logits, V, draft_ids, cu_q, B, gamma, T_cap, u_accept, u_sample,
                                  accept_len, bonus, out_tokens, n_accepted_total, prob, static_cast<cudaStream_t>(stream));
 }
