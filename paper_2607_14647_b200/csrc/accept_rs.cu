@@ -4,19 +4,20 @@
 // target distribution).  p = softmax of a target logits row, q = softmax of the matching draft logits row, both at
 // temperature 1.  The random numbers are inputs.
 //
-// Three launches.
+// Two launches.
 //   rs_stats_kernel    HBM-bound scan of the bf16 target rows [T, V] and of the draft rows that are in use
 //       ((i, t) with t < d_i): every (segment, row) CTA produces the segment's (maximum, sum of exp(x - maximum)).
-//   rs_decide_kernel   one warp per request: merges the segments of its rows, walks the drafts in order
-//       (u * q(z) < p(z) accepts) and records which distribution ends the request's step.
-//   rs_sample_kernel   one CTA per request: inversion sampling over ascending token index from (p - q)+ of the
-//       rejected position, or from p of the row after the last accepted draft.  Thread t owns the t-th contiguous
-//       slice of the vocabulary; slice sums are scanned in double, the slice that holds u * total is rescanned.
+//   rs_sample_kernel   one CTA per request.  Its first warp merges the segments of the request's rows, walks the
+//       drafts in order (u * q(z) < p(z) accepts) and finds which distribution ends the request's step; the CTA then
+//       draws from it by inversion over ascending token index: (p - q)+ of the rejected position, or p of the row
+//       after the last accepted draft.  The vocabulary is cut into chunks of 256 tokens; chunk sums are scanned in
+//       double, the chunk that holds u * total is rescanned.
 #include "dcut_internal.h"
 
 namespace {
 
 constexpr int kStatThreads = 256;
+constexpr int kUnroll = 4;
 constexpr int kSampleThreads = 1024;
 
 __device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
@@ -38,8 +39,6 @@ struct RsArgs {
     int V, B, gamma, n_seg, seg_elems;
     float2* stats;                  // [(T_cap + B * gamma) * n_seg]: (max, sum) per segment; draft rows after the target rows
     int T_cap;
-    int4* job;                      // [B]: x = target row, y = draft row (-1: sample from p), z = accept_len
-    float4* job_stats;              // [B]: (max_p, sum_p, max_q, sum_q) of the job's rows
     int* accept_len;
     int* bonus;
     int* out_tokens;
@@ -77,23 +76,32 @@ __global__ void __launch_bounds__(kStatThreads) rs_stats_kernel(RsArgs a) {
         for (int v = start + threadIdx.x; v < start + head; v += kStatThreads) take(bf_at(rp, v));
         const int nvec = (end - start - head) >> 3;
         const uint4* vp = reinterpret_cast<const uint4*>(rp + start + head);
-        for (int k = threadIdx.x; k < nvec; k += kStatThreads) {
-            // eight values at a time: one rescale of the running sum per vector, no data-dependent branch
-            const uint4 w = ld_stream_v4(vp + k);
-            const unsigned int ws[4] = {w.x, w.y, w.z, w.w};
-            float x[8];
+        for (int k0 = 0; k0 < nvec; k0 += kUnroll * kStatThreads) {
+            // up to four 16-byte vectors in flight per thread, one rescale of the running sum per batch, no
+            // data-dependent branch (vectors past the end repeat -inf, which adds nothing)
+            uint4 w[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const int k = k0 + u * kStatThreads + threadIdx.x;
+                w[u] = k < nvec ? ld_stream_v4(vp + k) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            }
+            float x[8 * kUnroll];
             float vmax = -INFINITY;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                x[2 * e] = __uint_as_float(ws[e] << 16);
-                x[2 * e + 1] = __uint_as_float(ws[e] & 0xffff0000u);
-                vmax = fmaxf(vmax, fmaxf(x[2 * e], x[2 * e + 1]));   // fmaxf drops NaN
+            for (int u = 0; u < kUnroll; ++u) {
+                const unsigned int ws[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    x[8 * u + 2 * e] = __uint_as_float(ws[e] << 16);
+                    x[8 * u + 2 * e + 1] = __uint_as_float(ws[e] & 0xffff0000u);
+                    vmax = fmaxf(vmax, fmaxf(x[8 * u + 2 * e], x[8 * u + 2 * e + 1]));   // fmaxf drops NaN
+                }
             }
             const float mn = fmaxf(m, vmax);
             if (mn > -INFINITY) {
                 float add = 0.0f;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
+                for (int e = 0; e < 8 * kUnroll; ++e) {
                     const float t = __expf(x[e] - mn);                // -inf -> 0; NaN -> NaN
                     add += (t == t) ? t : 0.0f;
                 }
@@ -136,56 +144,50 @@ __device__ __forceinline__ float2 row_stats(const RsArgs& a, int row) {
     return make_float2(m, s);
 }
 
-// One warp per request; lane t looks at draft t + 1, a ballot finds the first rejection.
-__global__ void __launch_bounds__(1024) rs_decide_kernel(RsArgs a) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    for (int i = warp; i < a.B; i += n_warps) {
-        const int r0 = a.cu_q[i], d = a.cu_q[i + 1] - r0 - 1;
-        int m = d;
-        float ratio = 0.0f;
-        float4 st = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int t0 = 0; t0 < d && m == d; t0 += 32) {
-            const int t = t0 + lane;
-            bool reject = false;
-            float my_ratio = 0.0f;
-            float4 my_st = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (t < d) {
-                const float2 sp = row_stats(a, r0 + t), sq = row_stats(a, a.T_cap + i * a.gamma + t);
-                const int z = min(max(a.draft_ids[(size_t)i * a.gamma + t], 0), a.V - 1);
-                const float pz = __expf(bf_at(a.target + (size_t)(r0 + t) * a.V, z) - sp.x) / sp.y;
-                const float qz = __expf(bf_at(a.draft + ((size_t)i * a.gamma + t) * a.V, z) - sq.x) / sq.y;
-                reject = !(a.u_accept[(size_t)i * a.gamma + t] * qz < pz);
-                my_ratio = pz / qz;
-                my_st = make_float4(sp.x, sp.y, sq.x, sq.y);
-            }
-            const unsigned int mask = __ballot_sync(0xffffffffu, reject);
-            const int src = mask ? __ffs(mask) - 1 : min(31, d - 1 - t0);   // first rejection, else the last draft seen
-            ratio = __shfl_sync(0xffffffffu, my_ratio, src);
-            st.x = __shfl_sync(0xffffffffu, my_st.x, src);
-            st.y = __shfl_sync(0xffffffffu, my_st.y, src);
-            st.z = __shfl_sync(0xffffffffu, my_st.z, src);
-            st.w = __shfl_sync(0xffffffffu, my_st.w, src);
-            if (mask) m = t0 + src;
+// Decision for request i by one warp: lane t looks at draft t + 1, a ballot finds the first rejection.  Returns (in every
+// lane) the job: x = target row, y = draft row (-1: the draw comes from p), z = accept_len; st = (max_p, sum_p, max_q, sum_q).
+__device__ __forceinline__ int4 rs_decide(const RsArgs& a, int i, float4& st, float& ratio) {
+    const int lane = threadIdx.x & 31;
+    const int r0 = a.cu_q[i], d = a.cu_q[i + 1] - r0 - 1;
+    int m = d;
+    ratio = 0.0f;
+    st = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int t0 = 0; t0 < d && m == d; t0 += 32) {
+        const int t = t0 + lane;
+        bool reject = false;
+        float my_ratio = 0.0f;
+        float4 my_st = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (t < d) {
+            const float2 sp = row_stats(a, r0 + t), sq = row_stats(a, a.T_cap + i * a.gamma + t);
+            const int z = min(max(a.draft_ids[(size_t)i * a.gamma + t], 0), a.V - 1);
+            const float pz = __expf(bf_at(a.target + (size_t)(r0 + t) * a.V, z) - sp.x) / sp.y;
+            const float qz = __expf(bf_at(a.draft + ((size_t)i * a.gamma + t) * a.V, z) - sq.x) / sq.y;
+            reject = !(a.u_accept[(size_t)i * a.gamma + t] * qz < pz);
+            my_ratio = pz / qz;
+            my_st = make_float4(sp.x, sp.y, sq.x, sq.y);
         }
-        if (lane == 0) {
-            int4 job;
-            job.z = m;
-            job.w = 0;
-            if (m < d) {           // rejected at draft m + 1: residual of target row r0 + m and draft row (i, m)
-                job.x = r0 + m;
-                job.y = i * a.gamma + m;
-            } else {               // all accepted (or d = 0): bonus from the target row after the last draft
-                job.x = r0 + d;
-                job.y = -1;
-                const float2 sp = row_stats(a, r0 + d);
-                st = make_float4(sp.x, sp.y, 0.f, 0.f);
-            }
-            a.job[i] = job;
-            a.job_stats[i] = st;
-            a.accept_len[i] = m;
-            if (a.prob) a.prob[2 * i] = ratio;
-        }
+        const unsigned int mask = __ballot_sync(0xffffffffu, reject);
+        const int src = mask ? __ffs(mask) - 1 : min(31, d - 1 - t0);   // first rejection, else the last draft seen
+        ratio = __shfl_sync(0xffffffffu, my_ratio, src);
+        st.x = __shfl_sync(0xffffffffu, my_st.x, src);
+        st.y = __shfl_sync(0xffffffffu, my_st.y, src);
+        st.z = __shfl_sync(0xffffffffu, my_st.z, src);
+        st.w = __shfl_sync(0xffffffffu, my_st.w, src);
+        if (mask) m = t0 + src;
     }
+    int4 job;
+    job.z = m;
+    job.w = 0;
+    if (m < d) {           // rejected at draft m + 1: residual of target row r0 + m and draft row (i, m)
+        job.x = r0 + m;
+        job.y = i * a.gamma + m;
+    } else {               // all accepted (or d = 0): bonus from the target row after the last draft
+        job.x = r0 + d;
+        job.y = -1;
+        const float2 sp = row_stats(a, r0 + d);
+        st = make_float4(sp.x, sp.y, 0.f, 0.f);
+    }
+    return job;
 }
 
 template <typename T>
@@ -225,8 +227,22 @@ constexpr int kMaxChunks = 1024;   // vocabularies up to 262 144 tokens
 
 __global__ void __launch_bounds__(kSampleThreads) rs_sample_kernel(RsArgs a) {
     const int i = blockIdx.x;
-    const int4 job = a.job[i];
-    const float4 st = a.job_stats[i];
+    __shared__ int4 job_s;
+    __shared__ float4 st_s;
+    if (threadIdx.x < 32) {
+        float4 st0;
+        float ratio;
+        const int4 job0 = rs_decide(a, i, st0, ratio);
+        if (threadIdx.x == 0) {
+            job_s = job0;
+            st_s = st0;
+            a.accept_len[i] = job0.z;
+            if (a.prob) a.prob[2 * i] = ratio;
+        }
+    }
+    __syncthreads();
+    const int4 job = job_s;
+    const float4 st = st_s;
     const unsigned short* tp = a.target + (size_t)job.x * a.V;
     const unsigned short* dp = job.y >= 0 ? a.draft + (size_t)job.y * a.V : nullptr;
     __shared__ double ws[33];
@@ -236,6 +252,8 @@ __global__ void __launch_bounds__(kSampleThreads) rs_sample_kernel(RsArgs a) {
     const int n_chunks = (a.V + kChunk - 1) / kChunk;
     const float inv_p = 1.0f / st.y, inv_q = dp ? 1.0f / st.w : 0.0f;
     bool use_p = dp == nullptr;
+    const bool vec_ok = (a.V & 7) == 0 && (reinterpret_cast<uintptr_t>(a.target) & 15) == 0 &&
+                        (reinterpret_cast<uintptr_t>(a.draft) & 15) == 0;   // every row then starts on 16 bytes
     int tok = 0;
     double mass = 0.0;
     for (int round = 0; round < 2; ++round) {
@@ -249,6 +267,25 @@ __global__ void __launch_bounds__(kSampleThreads) rs_sample_kernel(RsArgs a) {
         // the eight weights of this lane in chunk c, in token order (scalar loads: rows need not be 16-byte aligned)
         auto lane_weights = [&](int c, float (&w)[8]) {
             const int v0 = c * kChunk + lane * 8;
+            if (vec_ok && v0 + 8 <= a.V) {
+                const uint4 tv = *reinterpret_cast<const uint4*>(tp + v0);
+                uint4 dv = make_uint4(0, 0, 0, 0);
+                if (!use_p) dv = *reinterpret_cast<const uint4*>(dp + v0);
+                const unsigned int tw[4] = {tv.x, tv.y, tv.z, tv.w}, dw[4] = {dv.x, dv.y, dv.z, dv.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float xt = __uint_as_float((e & 1) ? (tw[e >> 1] & 0xffff0000u) : (tw[e >> 1] << 16));
+                    const float p = __expf(xt - st.x) * inv_p;
+                    if (use_p) {
+                        w[e] = p == p ? p : 0.0f;
+                    } else {
+                        const float xd = __uint_as_float((e & 1) ? (dw[e >> 1] & 0xffff0000u) : (dw[e >> 1] << 16));
+                        const float r = p - __expf(xd - st.z) * inv_q;
+                        w[e] = r > 0.0f ? r : 0.0f;
+                    }
+                }
+                return;
+            }
 #pragma unroll
             for (int e = 0; e < 8; ++e) w[e] = v0 + e < a.V ? weight(v0 + e) : 0.0f;
         };
@@ -372,8 +409,6 @@ dcut_status dcut_launch_accept_rs(dcut_ctx* ctx, const void* target_logits, cons
     a.T_cap = T_cap;
     unsigned char* base = static_cast<unsigned char*>(ctx->d_rs_scratch);
     a.stats = reinterpret_cast<float2*>(base);
-    a.job = reinterpret_cast<int4*>(base + rs_stats_bytes(ctx, a.n_seg));
-    a.job_stats = reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(a.job) + (size_t)ctx->lim.max_B * sizeof(int4));
     a.accept_len = accept_len;
     a.bonus = bonus;
     a.out_tokens = out_tokens;
@@ -387,8 +422,6 @@ dcut_status dcut_launch_accept_rs(dcut_ctx* ctx, const void* target_logits, cons
     rs_stats_kernel<<<grid, kStatThreads, 0, stream>>>(a);
     dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch rs_stats_kernel");
     if (st != DCUT_OK) return st;
-    rs_decide_kernel<<<1, 1024, 0, stream>>>(a);
-    if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch rs_decide_kernel")) != DCUT_OK) return st;
     rs_sample_kernel<<<B, kSampleThreads, 0, stream>>>(a);
     return dcut_check_cuda(ctx, cudaGetLastError(), "launch rs_sample_kernel");
 }
