@@ -233,6 +233,24 @@ dcut_status dcut_accept_rs(dcut_ctx* ctx, const void* target_logits, const void*
                            float* prob, void* stream);
 
 /*
+ * End of a step / start of the next (Section 3.1: a request commits its accepted drafts plus one more token;
+ * Appendix A: every request advances by at least one token per step).  For every request i, with m_i = accept_len[i]
+ * and the emitted tokens out_tokens[i, 0..m_i] (as written by dcut_accept / dcut_accept_rs / dcut_lm_head_accept):
+ *   ctx_lens[i] += m_i + 1   the cache now holds the old bonus token and the m_i accepted drafts; the slots of the
+ *                            rejected drafts are simply written over by the next step (that is the whole roll-back);
+ *   bonus_ids[i] = out_tokens[i, m_i]   the closing token of this step is z_{i,0} of the next one;
+ *   stream_tokens[i, stream_len[i] ..] gets the m_i + 1 emitted tokens and stream_len[i] grows by as much (optional:
+ *   pass null for both).
+ * DEVICE pointers; ctx_lens and stream_len are read and written.  max_ctx = tokens a request's pages can hold: a
+ * request left with less than gamma + 1 free positions, or a stream without room, sets the device status word
+ * (dcut_poll_device_status: code 5) - the stream is then left as it was, the context length is still advanced.
+ * The paper keeps this bookkeeping in the serving engine; it is here so that consecutive steps can run without a
+ * host round trip.
+ */
+dcut_status dcut_commit(dcut_ctx* ctx, const int* accept_len, const int* out_tokens, int B, int gamma, int max_ctx,
+                        int* ctx_lens, int* bonus_ids, int* stream_tokens, int* stream_len, int stream_cap, void* stream);
+
+/*
  * LM head fused with acceptance (the step between the last layer and dcut_accept, Section 3.1: the target's next-token
  * prediction at every retained position): logits[T, V] = x[T, hidden] . w_lm[V, hidden]^T (bf16 in, fp32 accumulate,
  * rounded to bf16 exactly as if the logits were stored), reduced inside the GEMM's epilogue to the row's argmax

@@ -140,6 +140,20 @@ def select(conf, draft_ids, bonus_ids, ctx_lens, cost_ms, bucket_K: Optional[Seq
                         info.candidate, bool(info.closure_ok), info.sum_fixed, info.objective, info.sum_f64)
 
 
+def commit(accept_len, out_tokens, ctx_lens, streams):
+    """End of a step (Section 3.1): request i has emitted out_tokens[i, 0..m_i]; its context grows by m_i + 1 (the old
+    bonus token and the m_i accepted drafts are now part of it), the closing token becomes the next bonus token, and the
+    emitted tokens are appended to the request's stream (a list of lists, changed in place).
+    Returns (new ctx_lens, next bonus_ids)."""
+    accept_len, out_tokens, ctx_lens = _i32(accept_len), _i32(out_tokens), _i32(ctx_lens)
+    new_ctx, nxt = ctx_lens.copy(), np.zeros(len(ctx_lens), np.int32)
+    for i, m in enumerate(accept_len):
+        new_ctx[i] = ctx_lens[i] + m + 1
+        nxt[i] = out_tokens[i, m]
+        streams[i].extend(int(t) for t in out_tokens[i, : m + 1])
+    return new_ctx, nxt
+
+
 def scores_shifted(conf: np.ndarray) -> np.ndarray:
     """Eq. 7: the admission score of depth k is the product of the confidences before k."""
     conf = np.ascontiguousarray(conf, dtype=np.float32)

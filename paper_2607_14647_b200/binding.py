@@ -29,7 +29,7 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
            "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_lm_head_accept",
-           "dcut_select_causal", "dcut_accept_rs", "dcut_poll_device_status"]
+           "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -64,6 +64,7 @@ _lib.dcut_budget_from_ratio.argtypes = [_i, _i, _i, _i, C.POINTER(_i)]
 _lib.dcut_select.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
 _lib.dcut_select_causal.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
 _lib.dcut_accept_rs.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i] + [_vp] * 8
+_lib.dcut_commit.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.dcut_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _i, _i, _f, _vp, _vp, _vp]
 _lib.dcut_accept.argtypes = [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp]
 _lib.dcut_poll_device_status.argtypes = [_vp, C.POINTER(_i), _vp]
@@ -221,6 +222,14 @@ class Context:
                                           float(scale), _ptr(out, torch.bfloat16), _ptr(lse, torch.float32),
                                           _stream()))
         return out
+
+    def commit(self, accept_len, out_tokens, ctx_lens, bonus_ids, max_ctx: int, stream_tokens=None, stream_len=None):
+        """dcut_commit: advances ctx_lens in place, writes the next step's bonus_ids, appends to the token streams."""
+        B, g1 = out_tokens.shape
+        cap = stream_tokens.shape[1] if stream_tokens is not None else 0
+        self._check(_lib.dcut_commit(self._h, _ptr(accept_len, torch.int32), _ptr(out_tokens, torch.int32), B, g1 - 1,
+                                     max_ctx, _ptr(ctx_lens, torch.int32), _ptr(bonus_ids, torch.int32),
+                                     _ptr(stream_tokens, torch.int32), _ptr(stream_len, torch.int32), cap, _stream()))
 
     def accept_rs(self, target_logits, draft_logits, draft_ids, cu_q, T_cap: int, u_accept, u_sample,
                   want_prob: bool = False):

@@ -318,6 +318,18 @@ dcut_status dcut_accept_rs(dcut_ctx* c, const void* target_logits, const void* d
                                  accept_len, bonus, out_tokens, n_accepted_total, prob, static_cast<cudaStream_t>(stream));
 }
 
+dcut_status dcut_commit(dcut_ctx* c, const int* accept_len, const int* out_tokens, int B, int gamma, int max_ctx,
+                        int* ctx_lens, int* bonus_ids, int* stream_tokens, int* stream_len, int stream_cap, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (!accept_len || !out_tokens || !ctx_lens || !bonus_ids) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if ((stream_tokens != nullptr) != (stream_len != nullptr) || (stream_tokens && stream_cap < 1))
+        return dcut_fail(c, DCUT_EINVAL, "stream_tokens, stream_len and stream_cap go together");
+    if (B < 1 || gamma < 1 || max_ctx < gamma + 1) return dcut_fail(c, DCUT_EINVAL, "need B, gamma >= 1 and max_ctx > gamma");
+    if (B > c->lim.max_B || gamma > c->lim.max_gamma) return dcut_fail(c, DCUT_ECAPACITY, "B = %d, gamma = %d exceed the limits", B, gamma);
+    return dcut_launch_commit(c, accept_len, out_tokens, B, gamma, max_ctx, ctx_lens, bonus_ids, stream_tokens, stream_len,
+                              stream_cap, static_cast<cudaStream_t>(stream));
+}
+
 dcut_status dcut_gemm_bf16(dcut_ctx* c, const void* a, const void* w, const void* w2, int mode, int N, int K,
                            const int* cu_q, int B, int T_cap, void* out, const void* residual, void* stream) {
     if (!c) return DCUT_EINVAL;

@@ -16,6 +16,7 @@
 #define DCUT_DEV_BAD_PAGE 2            // a block-table entry outside [0, num_pages)
 #define DCUT_DEV_PLAN_OVERFLOW 3       // the attention work list did not fit the context's scratch
 #define DCUT_DEV_GEMM_WAIT_TIMEOUT 4    // a bounded mbarrier wait in the GEMM kernel gave up
+#define DCUT_DEV_COMMIT_OVERFLOW 5      // dcut_commit: a context or a token stream ran out of room
 
 // One split-KV work item of the attention kernel: one (request, kv head, page range).
 struct __align__(16) AttnItem {
@@ -130,6 +131,9 @@ dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, c
                                      int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
                                      int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
                                      cudaStream_t stream);
+dcut_status dcut_launch_commit(dcut_ctx* ctx, const int* accept_len, const int* out_tokens, int B, int gamma, int max_ctx,
+                               int* ctx_lens, int* bonus_ids, int* stream_tokens, int* stream_len, int stream_cap,
+                               cudaStream_t stream);
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
