@@ -1072,7 +1072,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             }
             const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
             float m_run = -INFINITY, l_run = 0.0f;
-            TCP(long long t_ws = 0, t_wk = 0, t_bar = 0;)
+            TCP(long long t_ws = 0, t_wk = 0, t_bar = 0, t_ld = 0, t_exp = 0, t_st = 0;)
             for (int g = 0; g < n_groups; ++g) {
                 const int gc = G0 + g, b = gc % kTcSBufs;
                 TCP(long long c0 = clock64();)
@@ -1084,8 +1084,10 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                 if (!failed) {
                     tc_fence_after();
+                    TCP(long long c2 = clock64();)
                     tc_ld32(t_s + 32 * half, sr);
                     tc_wait_ld();
+                    TCP(t_ld += clock64() - c2;)
                     const int ncols = min(4, n_pages - 4 * g) * kPage;
                     const int j0 = (item.page_begin + 4 * g) * kPage + 32 * half;
                     if (ncols < 64 || j0 + 31 > ctx_len) {                  // a partial group or one that holds hidden keys
@@ -1136,6 +1138,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                     }
                 }
                 if (!failed) {
+                    TCP(long long c5 = clock64();)
                     const float mc = (m_run == -INFINITY ? 0.0f : m_run) * cs;
                     float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                     uint32_t pw[16];
@@ -1147,14 +1150,16 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                         pw[e] = pack_bf16(p0, p1);
                     }
                     l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                    TCP(long long c6 = clock64(); t_exp += c6 - c5;)
                     tc_st16(t_s + 16 * half, pw);                           // P over the columns S occupied
                     tc_wait_st();
                     tc_fence_before();
                     mbar_arrive(p_full + 8 * b);
+                    TCP(t_st += clock64() - c6;)
                 }
                 TCP(t_wk += clock64() - c1;)
             }
-            TCP(if (blockIdx.x == 0 && R == 0) printf("softmax half %d: wait_s %lld work %lld (pair barrier %lld)\n", half, t_ws, t_wk, t_bar);)
+            TCP(if (blockIdx.x == 0 && R == 0) printf("softmax half %d: wait_s %lld work %lld (ld %lld, pair barrier %lld, exp %lld, st %lld) groups %d\n", half, t_ws, t_wk, t_ld, t_bar, t_exp, t_st, n_groups);)
             // epilogue: the item's O row, normalised; this thread writes columns [64 * half, 64 * half + 64)
             const int gl = G0 + n_groups - 1;
             if (!failed && !mbar_wait(pv_done + 8 * (gl % kTcSBufs), (gl / kTcSBufs) & 1, &c->abort)) failed = true;
