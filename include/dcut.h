@@ -23,6 +23,13 @@
  *   - KV cache layout, for K and for V: [num_pages, n_kv_heads, page_size, head_dim] bf16, so the
  *     (page, kv head) tile is one contiguous block.  The cache base must be 128-byte aligned.
  *     Position j of request i lives in page block_table[i][j / page_size], slot j % page_size.
+ *
+ * Environment variables read once, in dcut_create (measurement knobs; the defaults are the measured best):
+ *   DCUT_ATTN_TC_MIN_ROWS     query rows from which a work item goes to the tcgen05 phase (17; above 128: never)
+ *   DCUT_ATTN_TARGET_ITEMS    requests are cut along the context only below this many (request, kv head) pairs (2 x SMs)
+ *   DCUT_ATTN_TAIL_REQ_DIV    cut the shortest B / n requests finer (0 = off)
+ *   DCUT_ATTN_TAIL_MIN_PAGES  smallest such piece, in pages (32)
+ *   DCUT_GEMM_2CTA            1 = run the GEMMs on pairs of SMs (tcgen05 cta_group::2); 0 (default) = one SM per tile
  */
 #ifndef DCUT_H_
 #define DCUT_H_
@@ -337,7 +344,10 @@ typedef struct {
 dcut_status dcut_verify_step_host(dcut_ctx* ctx, const dcut_host_step* step, void* stream);
 
 /* Reads the device status word (0 = no kernel reported an error) after synchronising `stream`,
- * and clears it.  A non-zero code also makes this call return DCUT_EDEVICE. */
+ * and clears it.  A non-zero code also makes this call return DCUT_EDEVICE.  Codes: 1 = a bounded
+ * wait in the attention kernel gave up, 2 = a block-table entry outside [0, num_pages) (page 0 was
+ * read instead), 3 = the attention work list did not fit the scratch, 4 = a bounded wait in the GEMM
+ * kernel gave up, 5 = dcut_commit ran out of room. */
 dcut_status dcut_poll_device_status(dcut_ctx* ctx, int* code, void* stream);
 
 #ifdef __cplusplus
