@@ -45,6 +45,8 @@ __device__ __forceinline__ void take8(const uint4& v, int base, float& best, int
 __global__ void __launch_bounds__(kArgmaxThreads) accept_argmax_kernel(
     const unsigned short* __restrict__ logits, int V, const int* __restrict__ cu_q, int B, int seg_elems,
     unsigned long long* __restrict__ row_key) {
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
     const int row = blockIdx.y;
     if (row >= cu_q[B]) return;
     const int start = blockIdx.x * seg_elems;
@@ -113,6 +115,8 @@ __global__ void __launch_bounds__(1024) accept_match_kernel(
     __shared__ int total_s;
     if (threadIdx.x == 0) total_s = 0;
     __syncthreads();
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     int local = 0;
     for (int i = warp; i < B; i += n_warps) {
@@ -173,22 +177,24 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
     seg = (seg + 7) & ~7;
     splits = (V + seg - 1) / seg;
     dim3 grid(splits, T_cap);
-    accept_argmax_kernel<<<grid, kArgmaxThreads, 0, stream>>>(static_cast<const unsigned short*>(logits), V, cu_q,
-                                                            B, seg, row_key);
-    dcut_status st = dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_argmax_kernel");
+    dcut_status st = dcut_check_cuda(ctx, dcut_launch_pdl(accept_argmax_kernel, grid, dim3(kArgmaxThreads), 0, stream,
+                                                          static_cast<const unsigned short*>(logits), V, cu_q, B, seg, row_key),
+                                     "launch accept_argmax_kernel");
     if (st != DCUT_OK) return st;
-    accept_match_kernel<<<1, 1024, 0, stream>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B,
-                                               gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total, nullptr);
-    return dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_match_kernel");
+    return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
+                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, row_key,
+                                                accept_len, bonus, out_tokens, n_accepted_total, static_cast<int*>(nullptr)),
+                           "launch accept_match_kernel");
 }
 
 dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
                                      int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
                                      int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
                                      cudaStream_t stream) {
-    accept_match_kernel<<<1, 1024, 0, stream>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B,
-                                               gamma, row_key, accept_len, bonus, out_tokens, n_accepted_total, row_argmax);
-    return dcut_check_cuda(ctx, cudaGetLastError(), "launch accept_match_kernel");
+    return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
+                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, row_key,
+                                                accept_len, bonus, out_tokens, n_accepted_total, row_argmax),
+                           "launch accept_match_kernel");
 }
 
 // ---------------------------------------------------------------------------------------------

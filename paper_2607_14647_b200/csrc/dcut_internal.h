@@ -87,6 +87,29 @@ struct dcut_ctx {
 };
 
 #ifdef __CUDACC__
+#include <utility>
+// Programmatic dependent launch: the kernel may be scheduled while its predecessor in the stream is still running
+// (its CTAs take SMs as the predecessor's CTAs leave), which hides launch latency and the kernel's own set-up.  Every
+// kernel launched this way calls dcut_pdl_wait() before it touches global memory: the wait returns when the
+// predecessor grid has completed, and since the predecessor did the same, everything earlier has completed too.
+template <typename... KArgs, typename... Args>
+inline cudaError_t dcut_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                   Args&&... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
+__device__ __forceinline__ void dcut_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dcut_pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // value order as an unsigned integer: larger float <=> larger code; every non-NaN code is > 0
 __device__ __forceinline__ unsigned int dcut_ordered_bits(float f) {
     if (f == 0.0f) f = 0.0f;   // -0 and +0 are the same value

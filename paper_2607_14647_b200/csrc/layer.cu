@@ -223,10 +223,6 @@ template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                     const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
-    const int T = g.cu_q[g.B];
-    const int m_tiles = (T + BM - 1) / BM;
-    const int n_work = m_tiles * g.n_tiles;
-    if ((int)blockIdx.x >= n_work) return;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
@@ -257,6 +253,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    // everything above overlaps the previous kernel of the stream; nothing it wrote is read before this wait
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
+    const int T = g.cu_q[g.B];
+    const int m_tiles = (T + BM - 1) / BM;
+    const int n_work = m_tiles * g.n_tiles;   // (a CTA without work falls through the loops below)
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
@@ -406,9 +408,6 @@ template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                      const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
-    const int T = g.cu_q[g.B];
-    const int m_tiles = (T + 2 * BM - 1) / (2 * BM);          // 256-row tiles of the pair
-    const int n_work = m_tiles * g.n_tiles;
     const uint32_t rank = cluster_ctarank();                   // 0: leader
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     // (no early exit: both CTAs of every pair take part in the cluster barriers below)
@@ -443,6 +442,11 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
+    const int T = g.cu_q[g.B];
+    const int m_tiles = (T + 2 * BM - 1) / (2 * BM);          // 256-row tiles of the pair
+    const int n_work = m_tiles * g.n_tiles;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (both CTAs)
@@ -539,6 +543,8 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_con
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ gain,
                                                       const int* __restrict__ cu_q, int B, int hidden, float eps,
                                                       __nv_bfloat16* __restrict__ y) {
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
     const int row = blockIdx.x;
     if (row >= cu_q[B]) return;
     const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * hidden);
@@ -590,6 +596,8 @@ struct RopeArgs {
 };
 
 __global__ void __launch_bounds__(256) rope_append_kernel(RopeArgs a) {
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
     const int tok = blockIdx.x;
     if (tok >= a.cu_q[a.B]) return;
     const int Dh = a.head_dim, half = Dh >> 1;
@@ -655,24 +663,26 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& 
         // pairs of CTAs (clusters of two SMs), 256-row tiles
         const int n_work2 = ((T_cap + 2 * BM - 1) / (2 * BM)) * n_tiles;
         const int pairs = n_work2 < ctx->ly_gemm_pairs ? n_work2 : ctx->ly_gemm_pairs;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t lc = {};
         lc.gridDim = dim3(2 * pairs);
         lc.blockDim = dim3(kGemmThreads);
         lc.dynamicSmemBytes = kG2Smem;
         lc.stream = stream;
         lc.attrs = attr;
-        lc.numAttrs = 1;
+        lc.numAttrs = 2;
         return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm2_tcgen05_kernel<MODE>, a, b, b2, ga), "launch gemm2_tcgen05_kernel");
     }
     const int n_work = ((T_cap + BM - 1) / BM) * n_tiles;
     const int grid = n_work < ctx->sm_count ? n_work : ctx->sm_count;   // persistent: at most one CTA per SM
-    gemm_tcgen05_kernel<MODE><<<grid, kGemmThreads, kGemmSmem, stream>>>(a, b, b2, ga);
-    return dcut_check_cuda(ctx, cudaGetLastError(), "launch gemm_tcgen05_kernel");
+    return dcut_check_cuda(ctx, dcut_launch_pdl(gemm_tcgen05_kernel<MODE>, dim3(grid), dim3(kGemmThreads), kGemmSmem, stream, a, b, b2, ga),
+                           "launch gemm_tcgen05_kernel");
 }
 
 struct LayerMaps {
@@ -802,8 +812,9 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     g.status = ctx->d_status;
 
     // 1. n = RMSNorm(x)
-    rmsnorm_kernel<<<T_cap, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w->g_attn),
-                                              cu_q, B, H, w->rms_eps, ctx->ly_norm);
+    if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(x),
+                                                   static_cast<const __nv_bfloat16*>(w->g_attn), cu_q, B, H, w->rms_eps, ctx->ly_norm),
+                              "launch rmsnorm_kernel")) != DCUT_OK) return st;
     // 2. qkv = n . Wqkv^T
     g.N_out = qkv_w; g.K = H; g.out = ctx->ly_qkv; g.residual = nullptr;
     if ((st = launch_gemm<kPlain>(ctx, lm->act[0], lm->m[0], lm->m[0], qkv_w / BN, T_cap, g, stream)) != DCUT_OK) return st;
@@ -813,8 +824,7 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     r.block_table_stride = block_table_stride; r.inv_freq = ctx->ly_inv_freq; r.B = B; r.n_q_heads = l.n_q_heads;
     r.n_kv_heads = l.n_kv_heads; r.head_dim = Dh; r.num_pages = num_pages; r.q_out = ctx->ly_q;
     r.k_cache = static_cast<__nv_bfloat16*>(k_cache); r.v_cache = static_cast<__nv_bfloat16*>(v_cache); r.status = ctx->d_status;
-    rope_append_kernel<<<T_cap, 256, 0, stream>>>(r);
-    if ((st = dcut_check_cuda(ctx, cudaGetLastError(), "launch rope_append_kernel")) != DCUT_OK) return st;
+    if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rope_append_kernel, dim3(T_cap), dim3(256), 0, stream, r), "launch rope_append_kernel")) != DCUT_OK) return st;
     // 4. attention
     st = dcut_launch_verify_attn(ctx, ctx->ly_q, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens,
                                  cu_q, B, T_cap, 1.0f / sqrtf((float)Dh), ctx->ly_attn, nullptr, stream);
@@ -823,7 +833,9 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     g.N_out = H; g.K = q_w; g.out = ctx->ly_h1; g.residual = static_cast<const __nv_bfloat16*>(x);
     if ((st = launch_gemm<kResidual>(ctx, lm->act[1], lm->m[1], lm->m[1], H / BN, T_cap, g, stream)) != DCUT_OK) return st;
     // 6. n2 = RMSNorm(h1)
-    rmsnorm_kernel<<<T_cap, 256, 0, stream>>>(ctx->ly_h1, static_cast<const __nv_bfloat16*>(w->g_mlp), cu_q, B, H, w->rms_eps, ctx->ly_norm2);
+    if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(ctx->ly_h1),
+                                                   static_cast<const __nv_bfloat16*>(w->g_mlp), cu_q, B, H, w->rms_eps, ctx->ly_norm2),
+                              "launch rmsnorm_kernel")) != DCUT_OK) return st;
     // 7. act = SiLU(n2 . Wg^T) * (n2 . Wu^T)
     g.N_out = I; g.K = H; g.out = ctx->ly_act; g.residual = nullptr;
     if ((st = launch_gemm<kSwiGLU>(ctx, lm->act[2], lm->m[2], lm->m[3], I / (BN / 2), T_cap, g, stream)) != DCUT_OK) return st;

@@ -179,6 +179,8 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     __shared__ Best best_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
     SELP(long long t0 = clock64();)
     // 1. prefix scores and sort keys.  The confidences come in through shared memory with coalesced loads
     // (the later prefix-sum array is free at this point), so the per-request product chain reads no global memory.
@@ -411,6 +413,5 @@ dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamm
     a.scores_out = scores_out;
     a.ranks_out = ranks_out;
     const size_t smem = select_smem_bytes(B, npad);
-    dcut_select_kernel<<<1, kThreads, smem, stream>>>(a);
-    return dcut_check_cuda(ctx, cudaGetLastError(), "launch dcut_select_kernel");
+    return dcut_check_cuda(ctx, dcut_launch_pdl(dcut_select_kernel, dim3(1), dim3(kThreads), smem, stream, a), "launch dcut_select_kernel");
 }

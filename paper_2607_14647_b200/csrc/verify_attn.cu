@@ -198,6 +198,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     __shared__ int ws[33];
     __shared__ int total_s, tail_s;
     const int tid = threadIdx.x, nthr = blockDim.x;   // 256 threads for small batches: cheaper barriers
+    dcut_pdl_wait();
     STAMP_MIN(0);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the item kernel's CTAs may take their SMs now
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -1316,6 +1317,7 @@ __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
     // Launched with programmatic stream serialization (see attn_item_kernel).
     STAMP_MIN(4);
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     STAMP_MAX(5);
     if (a.plan[4]) return;
     const int req = blockIdx.x / a.tokens_per_req, t = blockIdx.x - req * a.tokens_per_req;
@@ -1466,8 +1468,8 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.items = ctx->d_items;
     pa.plan = ctx->d_plan;
     pa.req_part = ctx->d_req_part;
-    attn_plan_kernel<<<1, B <= 256 ? 256 : kPlanThreads, sizeof(unsigned long long) * pa.npad, stream>>>(pa);
-    st = dcut_check_cuda(ctx, cudaGetLastError(), "launch attn_plan_kernel");
+    st = dcut_check_cuda(ctx, dcut_launch_pdl(attn_plan_kernel, dim3(1), dim3(B <= 256 ? 256 : kPlanThreads),
+                                              sizeof(unsigned long long) * pa.npad, stream, pa), "launch attn_plan_kernel");
     if (st != DCUT_OK) return st;
 
     AttnArgs aa;
