@@ -29,7 +29,7 @@
  *   DCUT_ATTN_TARGET_ITEMS    requests are cut along the context only below this many (request, kv head) pairs (2 x SMs)
  *   DCUT_ATTN_TAIL_REQ_DIV    cut the shortest B / n requests finer (0 = off)
  *   DCUT_ATTN_TAIL_MIN_PAGES  smallest such piece, in pages (32)
- *   DCUT_GEMM_2CTA            1 = run the GEMMs on pairs of SMs (tcgen05 cta_group::2); 0 (default) = one SM per tile
+ *   DCUT_GEMM_2CTA            0 = never run GEMM tiles on pairs of SMs (tcgen05 cta_group::2); default: where it pays
  */
 #ifndef DCUT_H_
 #define DCUT_H_

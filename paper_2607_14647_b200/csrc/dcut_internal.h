@@ -73,7 +73,8 @@ struct dcut_ctx {
 
     // decoder-layer workspace (hidden > 0 only), all [max_T, width] bf16
     __nv_bfloat16 *ly_norm, *ly_qkv, *ly_q, *ly_attn, *ly_h1, *ly_norm2, *ly_act;
-    int ly_gemm_pairs;      // clusters of two CTAs the GEMM runs on (0: one-CTA kernel)
+    int ly_gemm_pairs;      // clusters of two CTAs the device runs at once
+    int ly_gemm_pair_mode;  // 0: the GEMM never runs tiles on pairs of SMs
     float* ly_inv_freq;     // [head_dim / 2]
     float ly_theta;         // theta the table was built for (0 = none yet)
     void* layer_maps;       // cached tensor maps (layer.cu)

@@ -30,7 +30,7 @@ constexpr int kBTile = BN * BK * 2;            // 32 KB
 constexpr int kGemmStageBytes = kATile + kBTile;
 constexpr int kGemmThreads = 192;              // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int kTmemCols = 512;              // two 128 x 256 fp32 accumulators
-constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256 /* barriers, tmem ptr */;
+constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256 /* two sets of barriers, tmem ptr */;
 constexpr int kWaitLimit = 1 << 22;
 
 enum GemmMode { kPlain = 0, kResidual = 1, kSwiGLU = 2, kArgmax = 3 };
@@ -131,6 +131,7 @@ struct GemmArgs {
     const __nv_bfloat16* residual;   // [T, N_out] or null
     unsigned long long* row_key;     // kArgmax: one packed (ordered maximum, ~column) word per row
     int V;                           // kArgmax: live columns (rows of the weight)
+    int pairs;                       // launched as clusters of two CTAs: the pair mode may be chosen
     int* status;
 };
 
@@ -216,139 +217,6 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
     }
 }
 
-// Persistent: a CTA walks the output tiles b, b + gridDim.x, ... (m fastest, so the CTAs running together share
-// weight tiles in L2).  The operand ring and its barriers simply continue across tiles; the accumulator is
-// double-buffered in tensor memory (2 x 256 columns), so the epilogue of one tile overlaps the main loop of the next.
-template <int MODE>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
-                    const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGemmStages + 4);
-    const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
-    const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages), acc_empty = acc_full + 16;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_kb = g.K / BK;
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kGemmStages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(acc_full + 8 * b, 1);
-            mbar_init(acc_empty + 8 * b, 128);   // the four epilogue warps
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 1) {   // tensor memory: two 128 x 256 fp32 accumulators
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    bool failed = false;
-    // everything above overlaps the previous kernel of the stream; nothing it wrote is read before this wait
-    dcut_pdl_wait();
-    dcut_pdl_launch_dependents();
-    const int T = g.cu_q[g.B];
-    const int m_tiles = (T + BM - 1) / BM;
-    const int n_work = m_tiles * g.n_tiles;   // (a CTA without work falls through the loops below)
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
-        int kc = 0;   // k-blocks issued so far, over all tiles
-        for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x) {
-            const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
-            for (int kb = 0; kb < n_kb; ++kb, ++kc) {
-                const int s = kc % kGemmStages;
-                if (kc >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kGemmStages) - 1) & 1))) {
-                    failed = true;
-                    break;
-                }
-                if (elect_one()) {
-                    const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
-                    const uint32_t bar = full_bar + 8 * s;
-                    mbar_arrive_expect_tx(bar, kGemmStageBytes);
-                    tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
-                    if (MODE == kSwiGLU) {   // 128 gate rows, then the 128 up rows of the same features
-                        tma_load_2d(b_dst, &b_map, kb * BK, n_tile * (BN / 2), bar);
-                        tma_load_2d(b_dst + kBTile / 2, &b2_map, kb * BK, n_tile * (BN / 2), bar);
-                    } else {
-                        tma_load_2d(b_dst, &b_map, kb * BK, n_tile * BN, bar);
-                        tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
-                    }
-                }
-                __syncwarp();
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
-        int kc = 0, it = 0;
-        for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
-            const int acc = it & 1;
-            // the epilogue must have drained this accumulator (used by tile it - 2)
-            if (it >= 2 && !__all_sync(0xffffffffu, mbar_wait(acc_empty + 8 * acc, ((it >> 1) - 1) & 1))) {
-                failed = true;
-                break;
-            }
-            tc_fence_after();
-            const uint32_t tmem_d = tmem_base + acc * BN;
-            for (int kb = 0; kb < n_kb; ++kb, ++kc) {
-                const int s = kc % kGemmStages;
-                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kGemmStages) & 1))) {
-                    failed = true;
-                    break;
-                }
-                tc_fence_after();
-                if (elect_one()) {
-                    const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
-                    const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
-#pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
-                        tc_mma(tmem_d, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
-                    tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
-                }
-                __syncwarp();
-            }
-            if (failed) break;
-            if (elect_one()) tc_commit(acc_full + 8 * acc);   // accumulator complete
-            __syncwarp();
-        }
-    } else {
-        // ---------------------------------------------------------------- epilogue warps
-        const int quarter = warp & 3;               // tensor-memory lanes 32 * quarter .. + 31
-        int it = 0;
-        for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
-            const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
-            const int acc = it & 1;
-            const int row = m0 + quarter * 32 + lane;
-            if (!mbar_wait(acc_full + 8 * acc, (it >> 1) & 1)) {
-                failed = true;
-                break;
-            }
-            tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-            gemm_epilogue<MODE>(g, T, row, n_tile, t_row);
-            // this accumulator may be overwritten once all four epilogue warps have read it
-            tc_fence_before();
-            mbar_arrive(acc_empty + 8 * acc);
-        }
-    }
-    if (failed) atomicExch(g.status, DCUT_DEV_GEMM_WAIT_TIMEOUT);
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
-    }
-}
-
 // ------------------------------------------------------------------------------------------------ 2-CTA GEMM
 //
 // The same GEMM on pairs of CTAs (a cluster of two SMs, tcgen05 cta_group::2): a pair owns a 256 x 256 output tile,
@@ -404,82 +272,117 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
                  ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
 
+// One persistent kernel, two ways of running a GEMM, chosen on the device from the packed length (the same answer in
+// every CTA).
+//   One SM per tile: a CTA walks the 128 x 256 output tiles b, b + gridDim.x, ... (m fastest, so the CTAs running
+//   together share weight tiles in L2); four 48 KB operand stages.
+//   A pair of SMs per tile (see above): 256 x 256 tiles, six 32 KB stages.  It needs ~7 % fewer cycles per flop but
+//   pads the rows to 256 and has half as many, larger work items, so it is taken when it does not add a wave
+//   (gemm_use_pairs).
+// In both the operand ring and its barriers continue across tiles and the accumulator is double-buffered in tensor
+// memory (2 x 256 columns), so the epilogue of one tile overlaps the main loop of the next.
+__device__ __forceinline__ bool gemm_use_pairs(int T, int n_tiles, int K, int grid) {
+    const int tiles1 = ((T + BM - 1) / BM) * n_tiles, tiles2 = ((T + 2 * BM - 1) / (2 * BM)) * n_tiles;
+    const int pairs = grid >> 1;
+    if (tiles1 == 0 || pairs == 0) return false;
+    const int w1 = (tiles1 + grid - 1) / grid, w2 = (tiles2 + pairs - 1) / pairs;   // waves either way
+    // measured: a pair tile takes ~0.93 of two single tiles, and a single short wave (K = 4096) is faster on single SMs
+    return w2 * 15 < w1 * 16 && (w1 >= 2 || K >= 8192);
+}
+
+static_assert(kGemmStages * kGemmStageBytes == kG2Stages * kG2StageBytes, "both modes use the same operand area");
+
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
-                     const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
-    const uint32_t rank = cluster_ctarank();                   // 0: leader
-    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    // (no early exit: both CTAs of every pair take part in the cluster barriers below)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
+                    const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kG2Stages * kG2StageBytes);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kG2Stages + 4);
-    const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kG2Stages);
-    const uint32_t acc_full = smem_u32(bars + 2 * kG2Stages), acc_empty = acc_full + 16;
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
+    unsigned long long* bars2 = bars + 2 * kGemmStages + 4;                 // the pair mode's set
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars2 + 2 * kG2Stages + 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_kb = g.K / BK;
 
     if (threadIdx.x == 0) {
+        for (int s = 0; s < kGemmStages; ++s) {
+            mbar_init(smem_u32(bars + s), 1);
+            mbar_init(smem_u32(bars + kGemmStages + s), 1);
+        }
         for (int s = 0; s < kG2Stages; ++s) {
-            mbar_init(full_bar + 8 * s, 1);      // the leader's expect_tx arrival (bytes of both CTAs)
-            mbar_init(empty_bar + 8 * s, 1);     // the leader's multicast commit
+            mbar_init(smem_u32(bars2 + s), 1);                 // the leader's expect_tx arrival (bytes of both CTAs)
+            mbar_init(smem_u32(bars2 + kG2Stages + s), 1);     // the leader's multicast commit
         }
         for (int k = 0; k < 2; ++k) {
-            mbar_init(acc_full + 8 * k, 1);      // the leader's multicast commit
-            mbar_init(acc_empty + 8 * k, 256);   // (leader's copy) the epilogue threads of both CTAs
+            mbar_init(smem_u32(bars + 2 * kGemmStages + k), 1);
+            mbar_init(smem_u32(bars + 2 * kGemmStages + 2 + k), 128);   // the four epilogue warps
+            mbar_init(smem_u32(bars2 + 2 * kG2Stages + k), 1);          // the leader's multicast commit
+            mbar_init(smem_u32(bars2 + 2 * kG2Stages + 2 + k), 256);    // (leader's copy) the epilogue threads of both CTAs
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {   // tensor memory: two 128 x 256 fp32 accumulators per CTA, allocated for the pair
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
     __syncthreads();
     cluster_sync_all();                          // the peer's barriers exist before anything is signalled on them
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    bool failed = false;
+    // everything above overlaps the previous kernel of the stream; nothing it wrote is read before this wait
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
     const int T = g.cu_q[g.B];
-    const int m_tiles = (T + 2 * BM - 1) / (2 * BM);          // 256-row tiles of the pair
-    const int n_work = m_tiles * g.n_tiles;
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer (both CTAs)
-        const uint32_t lead_full = mapa_rank(full_bar, 0);
-        int kc = 0;
-        for (int w = pair; w < n_work && !failed; w += n_pairs) {
-            const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * (2 * BM) + (int)rank * BM;
-            for (int kb = 0; kb < n_kb; ++kb, ++kc) {
-                const int s = kc % kG2Stages;
-                if (kc >= kG2Stages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kG2Stages) - 1) & 1))) {
-                    failed = true;
-                    break;
-                }
-                if (elect_one()) {
-                    const uint32_t a_dst = smem_u32(smem + s * kG2StageBytes), b_dst = a_dst + kATile;
-                    if (rank == 0) mbar_arrive_expect_tx(full_bar + 8 * s, 2 * kG2StageBytes);
-                    const uint32_t bar = lead_full + 8 * s;
-                    tma_load_2d_pair(a_dst, &a_map, kb * BK, m0, bar);
-                    if (MODE == kSwiGLU)      // the leader's half: 128 gate rows; the peer's: the 128 up rows of the same features
-                        tma_load_2d_pair(b_dst, rank == 0 ? &b_map : &b2_map, kb * BK, n_tile * (BN / 2), bar);
-                    else
-                        tma_load_2d_pair(b_dst, &b_map, kb * BK, n_tile * BN + (int)rank * (BN / 2), bar);
-                }
-                __syncwarp();
-            }
+    const bool pairs = g.pairs && gemm_use_pairs(T, g.n_tiles, g.K, (int)gridDim.x);
+    if (warp == 1) {   // tensor memory: two 128 x 256 fp32 accumulators (per CTA; allocated for the pair in pair mode)
+        if (pairs) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer (leader CTA only)
-        if (rank == 0) {
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (pairs) cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool failed = false;
+
+    if (!pairs) {
+        const int m_tiles = (T + BM - 1) / BM;
+        const int n_work = m_tiles * g.n_tiles;   // (a CTA without work falls through the loops below)
+        const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
+        const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages), acc_empty = acc_full + 16;
+        if (warp == 0) {
+            // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
+            int kc = 0;   // k-blocks issued so far, over all tiles
+            for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x) {
+                const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
+                for (int kb = 0; kb < n_kb; ++kb, ++kc) {
+                    const int s = kc % kGemmStages;
+                    if (kc >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kGemmStages) - 1) & 1))) {
+                        failed = true;
+                        break;
+                    }
+                    if (elect_one()) {
+                        const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
+                        const uint32_t bar = full_bar + 8 * s;
+                        mbar_arrive_expect_tx(bar, kGemmStageBytes);
+                        tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
+                        if (MODE == kSwiGLU) {   // 128 gate rows, then the 128 up rows of the same features
+                            tma_load_2d(b_dst, &b_map, kb * BK, n_tile * (BN / 2), bar);
+                            tma_load_2d(b_dst + kBTile / 2, &b2_map, kb * BK, n_tile * (BN / 2), bar);
+                        } else {
+                            tma_load_2d(b_dst, &b_map, kb * BK, n_tile * BN, bar);
+                            tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+        } else if (warp == 1) {
+            // ---------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
             int kc = 0, it = 0;
-            for (int w = pair; w < n_work && !failed; w += n_pairs, ++it) {
+            for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
                 const int acc = it & 1;
-                // the epilogues of both CTAs must have drained this accumulator (used by tile it - 2)
+                // the epilogue must have drained this accumulator (used by tile it - 2)
                 if (it >= 2 && !__all_sync(0xffffffffu, mbar_wait(acc_empty + 8 * acc, ((it >> 1) - 1) & 1))) {
                     failed = true;
                     break;
@@ -487,45 +390,132 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_con
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + acc * BN;
                 for (int kb = 0; kb < n_kb; ++kb, ++kc) {
-                    const int s = kc % kG2Stages;
-                    if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kG2Stages) & 1))) {
+                    const int s = kc % kGemmStages;
+                    if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kGemmStages) & 1))) {
                         failed = true;
                         break;
                     }
                     tc_fence_after();
                     if (elect_one()) {
-                        const uint32_t a_addr = smem_u32(smem + s * kG2StageBytes);
+                        const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
                         const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
-#pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            tc_mma2(tmem_d, da + 2 * k, db + 2 * k, kIdesc2, (kb | k) ? 1u : 0u);
-                        tc_commit_pair(empty_bar + 8 * s);     // the stage is free in both CTAs once these MMAs have read it
+    #pragma unroll
+                        for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
+                            tc_mma(tmem_d, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+                        tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
                     }
                     __syncwarp();
                 }
                 if (failed) break;
-                if (elect_one()) tc_commit_pair(acc_full + 8 * acc);   // accumulator complete, in both CTAs
+                if (elect_one()) tc_commit(acc_full + 8 * acc);   // accumulator complete
                 __syncwarp();
+            }
+        } else {
+            // ---------------------------------------------------------------- epilogue warps
+            const int quarter = warp & 3;               // tensor-memory lanes 32 * quarter .. + 31
+            int it = 0;
+            for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
+                const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
+                const int acc = it & 1;
+                const int row = m0 + quarter * 32 + lane;
+                if (!mbar_wait(acc_full + 8 * acc, (it >> 1) & 1)) {
+                    failed = true;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+                gemm_epilogue<MODE>(g, T, row, n_tile, t_row);
+                // this accumulator may be overwritten once all four epilogue warps have read it
+                tc_fence_before();
+                mbar_arrive(acc_empty + 8 * acc);
             }
         }
     } else {
-        // ---------------------------------------------------------------- epilogue warps (both CTAs)
-        const int quarter = warp & 3;
-        const uint32_t lead_acc_empty = mapa_rank(acc_empty, 0);
-        int it = 0;
-        for (int w = pair; w < n_work && !failed; w += n_pairs, ++it) {
-            const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * (2 * BM) + (int)rank * BM;
-            const int acc = it & 1;
-            const int row = m0 + quarter * 32 + lane;
-            if (!mbar_wait(acc_full + 8 * acc, (it >> 1) & 1)) {
-                failed = true;
-                break;
+        const int m_tiles = (T + 2 * BM - 1) / (2 * BM);          // 256-row tiles of the pair
+        const int n_work = m_tiles * g.n_tiles;
+        const uint32_t rank = cluster_ctarank();                   // 0: leader
+        const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+        const uint32_t full_bar = smem_u32(bars2), empty_bar = smem_u32(bars2 + kG2Stages);
+        const uint32_t acc_full = smem_u32(bars2 + 2 * kG2Stages), acc_empty = acc_full + 16;
+        if (warp == 0) {
+            // ---------------------------------------------------------------- TMA producer (both CTAs)
+            const uint32_t lead_full = mapa_rank(full_bar, 0);
+            int kc = 0;
+            for (int w = pair; w < n_work && !failed; w += n_pairs) {
+                const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * (2 * BM) + (int)rank * BM;
+                for (int kb = 0; kb < n_kb; ++kb, ++kc) {
+                    const int s = kc % kG2Stages;
+                    if (kc >= kG2Stages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kG2Stages) - 1) & 1))) {
+                        failed = true;
+                        break;
+                    }
+                    if (elect_one()) {
+                        const uint32_t a_dst = smem_u32(smem + s * kG2StageBytes), b_dst = a_dst + kATile;
+                        if (rank == 0) mbar_arrive_expect_tx(full_bar + 8 * s, 2 * kG2StageBytes);
+                        const uint32_t bar = lead_full + 8 * s;
+                        tma_load_2d_pair(a_dst, &a_map, kb * BK, m0, bar);
+                        if (MODE == kSwiGLU)      // the leader's half: 128 gate rows; the peer's: the 128 up rows of the same features
+                            tma_load_2d_pair(b_dst, rank == 0 ? &b_map : &b2_map, kb * BK, n_tile * (BN / 2), bar);
+                        else
+                            tma_load_2d_pair(b_dst, &b_map, kb * BK, n_tile * BN + (int)rank * (BN / 2), bar);
+                    }
+                    __syncwarp();
+                }
             }
-            tc_fence_after();
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-            gemm_epilogue<MODE>(g, T, row, n_tile, t_row);
-            tc_fence_before();
-            mbar_arrive_remote(lead_acc_empty + 8 * acc);
+        } else if (warp == 1) {
+            // ---------------------------------------------------------------- MMA issuer (leader CTA only)
+            if (rank == 0) {
+                int kc = 0, it = 0;
+                for (int w = pair; w < n_work && !failed; w += n_pairs, ++it) {
+                    const int acc = it & 1;
+                    // the epilogues of both CTAs must have drained this accumulator (used by tile it - 2)
+                    if (it >= 2 && !__all_sync(0xffffffffu, mbar_wait(acc_empty + 8 * acc, ((it >> 1) - 1) & 1))) {
+                        failed = true;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t tmem_d = tmem_base + acc * BN;
+                    for (int kb = 0; kb < n_kb; ++kb, ++kc) {
+                        const int s = kc % kG2Stages;
+                        if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kG2Stages) & 1))) {
+                            failed = true;
+                            break;
+                        }
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint32_t a_addr = smem_u32(smem + s * kG2StageBytes);
+                            const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
+    #pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                tc_mma2(tmem_d, da + 2 * k, db + 2 * k, kIdesc2, (kb | k) ? 1u : 0u);
+                            tc_commit_pair(empty_bar + 8 * s);     // the stage is free in both CTAs once these MMAs have read it
+                        }
+                        __syncwarp();
+                    }
+                    if (failed) break;
+                    if (elect_one()) tc_commit_pair(acc_full + 8 * acc);   // accumulator complete, in both CTAs
+                    __syncwarp();
+                }
+            }
+        } else {
+            // ---------------------------------------------------------------- epilogue warps (both CTAs)
+            const int quarter = warp & 3;
+            const uint32_t lead_acc_empty = mapa_rank(acc_empty, 0);
+            int it = 0;
+            for (int w = pair; w < n_work && !failed; w += n_pairs, ++it) {
+                const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * (2 * BM) + (int)rank * BM;
+                const int acc = it & 1;
+                const int row = m0 + quarter * 32 + lane;
+                if (!mbar_wait(acc_full + 8 * acc, (it >> 1) & 1)) {
+                    failed = true;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+                gemm_epilogue<MODE>(g, T, row, n_tile, t_row);
+                tc_fence_before();
+                mbar_arrive_remote(lead_acc_empty + 8 * acc);
+            }
         }
     }
     if (failed) atomicExch(g.status, DCUT_DEV_GEMM_WAIT_TIMEOUT);
@@ -534,7 +524,10 @@ gemm2_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_con
     cluster_sync_all();                          // nobody leaves while the other CTA may still signal its barriers
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
+        if (pairs)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
     }
 }
 
@@ -659,10 +652,14 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& 
                         int T_cap, const GemmArgs& g, cudaStream_t stream) {
     GemmArgs ga = g;
     ga.n_tiles = n_tiles;
+    const int n_work = ((T_cap + BM - 1) / BM) * n_tiles;
+    int grid = n_work < ctx->sm_count ? n_work : ctx->sm_count;   // persistent: at most one CTA per SM
+    ga.pairs = 0;
     if (ctx->ly_gemm_pairs > 0) {
-        // pairs of CTAs (clusters of two SMs), 256-row tiles
-        const int n_work2 = ((T_cap + 2 * BM - 1) / (2 * BM)) * n_tiles;
-        const int pairs = n_work2 < ctx->ly_gemm_pairs ? n_work2 : ctx->ly_gemm_pairs;
+        // always launched as clusters of two CTAs (the kernel holds cta_group::2 instructions); the pair mode itself
+        // can be switched off
+        grid = 2 * (n_work < ctx->ly_gemm_pairs ? n_work : ctx->ly_gemm_pairs);   // room for either mode
+        ga.pairs = ctx->ly_gemm_pair_mode;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
@@ -671,16 +668,14 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& 
         attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t lc = {};
-        lc.gridDim = dim3(2 * pairs);
+        lc.gridDim = dim3(grid);
         lc.blockDim = dim3(kGemmThreads);
-        lc.dynamicSmemBytes = kG2Smem;
+        lc.dynamicSmemBytes = kGemmSmem;
         lc.stream = stream;
         lc.attrs = attr;
         lc.numAttrs = 2;
-        return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm2_tcgen05_kernel<MODE>, a, b, b2, ga), "launch gemm2_tcgen05_kernel");
+        return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_tcgen05_kernel<MODE>, a, b, b2, ga), "launch gemm_tcgen05_kernel");
     }
-    const int n_work = ((T_cap + BM - 1) / BM) * n_tiles;
-    const int grid = n_work < ctx->sm_count ? n_work : ctx->sm_count;   // persistent: at most one CTA per SM
     return dcut_check_cuda(ctx, dcut_launch_pdl(gemm_tcgen05_kernel<MODE>, dim3(grid), dim3(kGemmThreads), kGemmSmem, stream, a, b, b2, ga),
                            "launch gemm_tcgen05_kernel");
 }
@@ -699,18 +694,14 @@ dcut_status dcut_init_layer(dcut_ctx* ctx) {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tcgen05_kernel<kArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemmSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<kPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kG2Smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<kResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, kG2Smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<kSwiGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kG2Smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm2_tcgen05_kernel<kArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, kG2Smem);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(gemm)");
     {
-        // DCUT_GEMM_2CTA=1 selects the pair kernel (off by default: its 256-row tiles pay for the faster MMA with
-        // padding and coarser waves at most packed lengths; see gemm2_tcgen05_kernel).  ly_gemm_pairs = how many
-        // clusters of two CTAs the device runs at once.
+        // The GEMM is launched as clusters of two CTAs so that it can run tiles on pairs of SMs where that pays
+        // (DCUT_GEMM_2CTA=0: never).  ly_gemm_pairs = how many such clusters the device runs at once.
         const char* env = getenv("DCUT_GEMM_2CTA");
+        ctx->ly_gemm_pair_mode = (!env || atoi(env) != 0) ? 1 : 0;
         ctx->ly_gemm_pairs = 0;
-        if (env && atoi(env) != 0) {
+        {
             cudaLaunchAttribute attr[1];
             attr[0].id = cudaLaunchAttributeClusterDimension;
             attr[0].val.clusterDim.x = 2;
@@ -719,11 +710,11 @@ dcut_status dcut_init_layer(dcut_ctx* ctx) {
             cudaLaunchConfig_t lc = {};
             lc.gridDim = dim3(2 * ctx->sm_count);
             lc.blockDim = dim3(kGemmThreads);
-            lc.dynamicSmemBytes = kG2Smem;
+            lc.dynamicSmemBytes = kGemmSmem;
             lc.attrs = attr;
             lc.numAttrs = 1;
             int n_clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&n_clusters, gemm2_tcgen05_kernel<kPlain>, &lc) == cudaSuccess && n_clusters > 0)
+            if (cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tcgen05_kernel<kPlain>, &lc) == cudaSuccess && n_clusters > 0)
                 ctx->ly_gemm_pairs = n_clusters;
             else
                 (void)cudaGetLastError();

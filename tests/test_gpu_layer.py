@@ -115,9 +115,10 @@ def test_full_layer_workload_on_sampled_requests():
 
 
 @pytest.mark.parametrize("T,N,K,mode", [(300, 512, 1024, 0), (257, 256, 4096, 1), (640, 1024, 512, 2), (100, 256, 128, 0)])
-def test_pair_kernel_matches_the_oracle(T, N, K, mode, monkeypatch):
-    """The cta_group::2 variant of the GEMM (selected with DCUT_GEMM_2CTA=1 when the context is created)."""
-    monkeypatch.setenv("DCUT_GEMM_2CTA", "1")
+def test_single_sm_mode_matches_the_oracle(T, N, K, mode, monkeypatch):
+    """The GEMM with its pair mode (cta_group::2) switched off when the context is created: single-SM tiles only.
+    (The default build picks the mode per launch; the other GEMM tests cover that.)"""
+    monkeypatch.setenv("DCUT_GEMM_2CTA", "0")
     rng = np.random.default_rng(T + N + K + mode)
     cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
     ctx = make_ctx(cfg, max_pages=1, vocab=0)
@@ -135,5 +136,29 @@ def test_pair_kernel_matches_the_oracle(T, N, K, mode, monkeypatch):
         want = orc.swiglu_f64(orc.linear(a[:T], w), orc.linear(a[:T], w2))
     else:
         want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
-    _close(out[:T], want, f"pair kernel mode {mode}")
+    _close(out[:T], want, f"single-SM mode, epilogue {mode}")
+    assert (out[T:].float() == 7.0).all()       # rows past T are never written
+
+
+@pytest.mark.parametrize("T,N,K,mode", [(300, 512, 8192, 0), (257, 256, 8192, 1), (640, 1024, 8192, 2), (40, 256, 8192, 0)])
+def test_pair_mode_matches_the_oracle(T, N, K, mode):
+    """Shapes for which the kernel picks its pair mode (one wave either way and K >= 8192), every stored epilogue."""
+    rng = np.random.default_rng(T + N + K + mode)
+    cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
+    ctx = make_ctx(cfg, max_pages=1, vocab=0)
+    T_cap = T + 5
+    a, w = _bf(rng, (T_cap, K)), _bf(rng, (N, K), 0.05)
+    w2 = _bf(rng, (N, K), 0.05) if mode == 2 else None
+    res = _bf(rng, (T_cap, N)) if mode == 1 else None
+    cu = dev(np.array([0, T], np.int32))
+    out = torch.full((T_cap, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(w), cu, T_cap, out, mode=mode, w2=None if w2 is None else dev(w2),
+                  residual=None if res is None else dev(res))
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    if mode == 2:
+        want = orc.swiglu_f64(orc.linear(a[:T], w), orc.linear(a[:T], w2))
+    else:
+        want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
+    _close(out[:T], want, f"pair mode, epilogue {mode}")
     assert (out[T:].float() == 7.0).all()       # rows past T are never written

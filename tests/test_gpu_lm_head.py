@@ -53,7 +53,7 @@ def _case(B, gamma, V, H, depths, seed=0):
     return cfg, sel, w, x, cu
 
 
-@pytest.mark.parametrize("B,V,H", [(5, 1000, 256), (8, 256, 512), (16, 700, 256), (3, 1, 256), (12, 2049, 1024)])
+@pytest.mark.parametrize("B,V,H", [(5, 1000, 256), (8, 256, 512), (16, 700, 256), (3, 1, 256), (12, 2049, 1024), (20, 700, 8192)])
 def test_small_shapes_every_row(B, V, H):
     gamma = 8
     rng = np.random.default_rng(V + H)
