@@ -233,7 +233,6 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
 
 constexpr int kG2Stages = 6;
 constexpr int kG2StageBytes = kATile + kBTile / 2;     // 32 KB
-constexpr int kG2Smem = kG2Stages * kG2StageBytes + 1024 /* align */ + 256 /* barriers, tmem ptr */;
 constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
