@@ -217,9 +217,9 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
     }
 }
 
-// ------------------------------------------------------------------------------------------------ 2-CTA GEMM
+// ------------------------------------------------------------------------------------------------ GEMM, pair mode
 //
-// The same GEMM on pairs of CTAs (a cluster of two SMs, tcgen05 cta_group::2): a pair owns a 256 x 256 output tile,
+// Pair mode of the GEMM kernel (a cluster of two SMs, tcgen05 cta_group::2): a pair owns a 256 x 256 output tile,
 // each CTA its 128 rows.  Each CTA loads its own A tile and HALF of the B tile (128 of the 256 weight rows; for
 // SwiGLU the leader's half is the gate rows, the peer's the up rows); the leader's MMA warp issues M256 N256 K16 MMAs
 // that read both halves, so an MMA streams 8 KB per SM from shared memory instead of 12 KB and a stage is 32 KB
@@ -228,8 +228,8 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
 // on the leader's accumulator-empty barrier through distributed shared memory.
 // Measured against the one-CTA kernel: 74 us against 86 us for the down projection at T = 512-640 (K = 12288), 81 against
 // 90 us for gate/up + SwiGLU at T = 512, but 135 against 92 us for the down projection at T = 1088, where 5 x 16 = 80
-// pair tiles need two waves on 74 pairs (and 1280 padded rows are computed instead of 1152): the one-CTA kernel stays
-// the default.
+// pair tiles need two waves on 74 pairs (and 1280 padded rows are computed instead of 1152): the kernel therefore
+// picks the mode per launch (gemm_use_pairs).
 
 constexpr int kG2Stages = 6;
 constexpr int kG2StageBytes = kATile + kBTile / 2;     // 32 KB
