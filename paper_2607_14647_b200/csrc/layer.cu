@@ -6,15 +6,19 @@
 //   rmsnorm_kernel        one CTA per packed token, fp32 sum of squares, bf16 out
 //   rope_append_kernel    rotate-half RoPE on q and k heads, K/V of the new tokens written into the paged cache at
 //                         position L_i + t, q written as the attention kernel's [T, Hq, Dh] input
-//   gemm_tcgen05_kernel   C[M, N] = A[M, K] . B[N, K]^T on the 5th-generation tensor cores: 128 x 256 output tile
-//                         per CTA, accumulator in tensor memory (256 fp32 columns), operands staged by TMA into a
-//                         4-stage ring of 128-byte-swizzled K-major tiles (BK = 64), one elected lane issuing
-//                         tcgen05.mma (M128 N256 K16) and releasing stages with tcgen05.commit, four epilogue warps
-//                         reading the accumulator with tcgen05.ld.  Epilogues: plain bf16, + residual, or SwiGLU
-//                         (the B tile is 128 gate rows followed by the 128 matching up rows, so silu(g) * u is
-//                         formed in registers and the [T, 2I] intermediate never exists).
-// M is ragged and known only on the device (T = cu_q[B]): grids are sized for T_cap, CTAs past T leave at once,
-// rows past T are computed on whatever the buffers hold and never stored.
+//   gemm_tcgen05_kernel   C[M, N] = A[M, K] . B[N, K]^T on the 5th-generation tensor cores.  Persistent; launched as
+//                         clusters of two CTAs.  After reading the packed length it runs either 128 x 256 tiles on
+//                         single SMs (tcgen05.mma M128 N256 K16, four 48 KB operand stages) or 256 x 256 tiles on
+//                         pairs of SMs (cta_group::2, M256, each CTA loading half of B, six 32 KB stages).  Operands
+//                         are staged by TMA as 128-byte-swizzled K-major tiles (BK = 64); one elected lane issues the
+//                         MMAs and releases stages with tcgen05.commit; two accumulators in tensor memory let the four
+//                         epilogue warps (tcgen05.ld) work on one tile while the next is being multiplied.
+//                         Epilogues: plain bf16, + residual, SwiGLU (the B tile is 128 gate rows and the 128 matching
+//                         up rows, so silu(g) * u is formed in registers and the [T, 2I] intermediate never exists),
+//                         or row argmax (the LM head fused with acceptance: the logits are never stored).
+// M is ragged and known only on the device (T = cu_q[B]): grids are sized for T_cap, CTAs without work fall through,
+// rows past T are computed on whatever the buffers hold and never stored.  Every kernel is launched with programmatic
+// dependent launch and waits for its predecessor before touching global memory.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <math.h>
