@@ -27,6 +27,11 @@ __device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
                  : "l"(p));
     return r;
 }
+__device__ __forceinline__ float exp2f_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float bf_at(const unsigned short* p, int v) { return __uint_as_float((unsigned int)p[v] << 16); }
 
 struct RsArgs {
@@ -99,13 +104,16 @@ __global__ void __launch_bounds__(kStatThreads) rs_stats_kernel(RsArgs a) {
             }
             const float mn = fmaxf(m, vmax);
             if (mn > -INFINITY) {
-                float add = 0.0f;
+                // exp(x - mn) = 2^(x * log2(e) - mn * log2(e)): one FMA, one clamp that turns NaN into -inf (weight 0),
+                // one special-function operation, one add per value; two partial sums for instruction-level parallelism
+                const float kL2e = 1.4426950408889634f, off = -mn * kL2e;
+                float add0 = 0.0f, add1 = 0.0f;
 #pragma unroll
-                for (int e = 0; e < 8 * kUnroll; ++e) {
-                    const float t = __expf(x[e] - mn);                // -inf -> 0; NaN -> NaN
-                    add += (t == t) ? t : 0.0f;
+                for (int e = 0; e < 8 * kUnroll; e += 2) {
+                    add0 += exp2f_fast(fmaxf(fmaf(x[e], kL2e, off), -INFINITY));
+                    add1 += exp2f_fast(fmaxf(fmaf(x[e + 1], kL2e, off), -INFINITY));
                 }
-                s = s * __expf(m - mn) + add;
+                s = s * __expf(m - mn) + (add0 + add1);
                 m = mn;
             }
         }
