@@ -15,6 +15,7 @@ sample of the same workload.  With N > 1 every rank runs an independent replica 
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -49,6 +50,8 @@ def parse_args():
     ap.add_argument("--cost-points", type=int, default=18)
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--gamma", type=int, default=0,
+                    help="draft tokens per request, if not the config's (7 = the paper's block-8 setting)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the step's kernels one by one instead of replaying a CUDA graph")
     return ap.parse_args()
@@ -207,6 +210,8 @@ def run_reference(args):
     if rank != 0:
         return
     cfg = wl.config(args.config)
+    if args.gamma > 0:
+        cfg = dataclasses.replace(cfg, gamma=args.gamma, name=f"{cfg.name}_gamma{args.gamma}")
     sel, kv, q_all, logits_all = host_inputs(cfg)
     cost = wl.cost_table_for(cfg)
     per_step = max(2.0, min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup)))
@@ -241,6 +246,8 @@ def run_dcut(args):
     from paper_2607_14647_b200 import binding
 
     cfg = wl.config(args.config)
+    if args.gamma > 0:
+        cfg = dataclasses.replace(cfg, gamma=args.gamma, name=f"{cfg.name}_gamma{args.gamma}")
     sel, kv, q_all, logits_all = host_inputs(cfg)
     dev = torch.device("cuda", local)
     d_conf = torch.from_numpy(sel.conf).to(dev)
