@@ -1319,13 +1319,16 @@ __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     STAMP_MAX(5);
-    if (a.plan[4]) return;
-    const int req = blockIdx.x / a.tokens_per_req, t = blockIdx.x - req * a.tokens_per_req;
-    const int nc = a.req_part[2 * req + 1];
-    if (nc <= 1) return;
+    if (a.plan[4] || a.plan[3] == 0) return;   // overflow, or no request was cut: nothing to merge
     const int lane = threadIdx.x & 31;
     const int h = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (h >= a.n_q_heads || t >= a.cu_q[req + 1] - a.cu_q[req]) return;
+    if (h >= a.n_q_heads) return;
+    // grid-stride over (request, block position): the grid is capped at two CTAs per SM so that the usual case of an
+    // uncut batch costs a few hundred CTA launches, not B * (gamma + 1)
+    for (int k = blockIdx.x; k < a.B * a.tokens_per_req; k += gridDim.x) {
+    const int req = k / a.tokens_per_req, t = k - req * a.tokens_per_req;
+    const int nc = a.req_part[2 * req + 1];
+    if (nc <= 1 || t >= a.cu_q[req + 1] - a.cu_q[req]) continue;
     const int tok = a.cu_q[req] + t;
     const int group = a.n_q_heads / a.n_kv_heads;
     const int q0 = a.cu_q[req];
@@ -1354,6 +1357,7 @@ __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
 #pragma unroll
     for (int e = 0; e < kPer; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
     if (a.lse && lane == 0) a.lse[(size_t)tok * a.n_q_heads + h] = wsum > 0.0f ? m_all + logf(wsum) : -INFINITY;
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1399,7 +1403,8 @@ dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm
     if (st != DCUT_OK) return st;
     (void)T_cap;
     const int heads_per_cta = ctx->lim.n_q_heads < 32 ? ((ctx->lim.n_q_heads + 7) / 8) * 8 : 32;
-    lc.gridDim = dim3(ca.B * ca.tokens_per_req, (ctx->lim.n_q_heads + heads_per_cta - 1) / heads_per_cta);
+    const int cgrid = ca.B * ca.tokens_per_req < 2 * ctx->sm_count ? ca.B * ca.tokens_per_req : 2 * ctx->sm_count;
+    lc.gridDim = dim3(cgrid, (ctx->lim.n_q_heads + heads_per_cta - 1) / heads_per_cta);
     lc.blockDim = dim3(32 * heads_per_cta);
     lc.dynamicSmemBytes = 0;
     return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, attn_combine_kernel<DH>, ca), "launch attn_combine_kernel");
