@@ -371,8 +371,9 @@ static_assert(kThreads == 64 + kTcSoftmaxThreads, "roles of the tcgen05 phase");
 constexpr int kTcPageBytes = kPage * 128 * 2;      // 4 KB: one K or V page tile
 constexpr int kTcGroupBytes = 8 * kTcPageBytes;    // K of 4 pages (16 KB, [half][64 rows][64]) + V of 4 pages
 constexpr int kTcRingBytes = kTcGroupStages * kTcGroupBytes;
-constexpr int kTcCols = 512;                       // O: 0..127, S/P buffers: 128..319, Q: 320..383
-constexpr int kTcColS = 128, kTcColQ = kTcColS + 64 * kTcSBufs;
+constexpr int kTcCols = 512;                       // O of team 0: 0..127, of team 1: 128..255, S/P buffers: 256..447, Q: 448..511
+constexpr int kTcColOB = 128, kTcColS = 256, kTcColQ = kTcColS + 64 * kTcSBufs;
+static_assert(kTcColQ + 64 <= kTcCols, "tensor-memory columns");
 constexpr float kRescaleLog2 = 8.0f;
 
 // One lane of a converged warp.  Issuing tcgen05.mma / tcgen05.commit under this predicate (not under `lane == 0`)
@@ -883,7 +884,7 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
 // current item is still being finished; only Q and O (single-buffered in tensor memory) serialise at an item boundary,
 // through the q_ready and o_free barriers.
 __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtensorMap& v_map, const AttnArgs& a,
-                                         unsigned char* ring, Ctrl* c, float (*xch)[2][128], float (*xl)[128],
+                                         unsigned char* ring, Ctrl* c, float (*xm)[128], float (*xl)[128],
                                          int* counter, int end) {
     constexpr int kPhase = 0;
     const uint32_t full_bar = smem_u32(c->ring_full), empty_bar = smem_u32(c->ring_empty);
@@ -1007,14 +1008,15 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                 if (elect_one()) {
                     const int np = min(4, n_pages - 4 * g), gs = gc % kTcGroupStages;
                     const uint32_t tmem_p = tmem_o + kTcColS + 64 * b;
+                    const uint32_t tmem_ov = tmem_o + kTcColOB * (g & 1);   // the O accumulator of the team that owns group g
                     const uint64_t dv = desc_mnmajor(smem_u32(ring + gs * kTcGroupBytes) + 4 * kTcPageBytes);
                     if (np == 4) {
 #pragma unroll
                         for (int j = 0; j < 4; ++j)        // 16 keys = 8 words of P; the next V tile is 4 KB = 256 units on
-                            tc_mma_ts(tmem_o, tmem_p + 8 * j, dv + 256 * j, kIdescPV, (g | j) ? 1u : 0u);
+                            tc_mma_ts(tmem_ov, tmem_p + 8 * j, dv + 256 * j, kIdescPV, ((g >> 1) | j) ? 1u : 0u);
                     } else {
                         for (int j = 0; j < np; ++j)
-                            tc_mma_ts(tmem_o, tmem_p + 8 * j, dv + 256 * j, kIdescPV, (g | j) ? 1u : 0u);
+                            tc_mma_ts(tmem_ov, tmem_p + 8 * j, dv + 256 * j, kIdescPV, ((g >> 1) | j) ? 1u : 0u);
                     }
                     tc_commit(empty_bar + 8 * gs);         // the group's K and V tiles are free again
                     tc_commit(pv_done + 8 * b);
@@ -1030,13 +1032,16 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
         }
     } else if (warp < 2 + kTcSoftmaxThreads / 32) {
         // ---------------------------------------------------------------- softmax + epilogue
-        // row R = tensor-memory lane; this thread owns columns [32 * half, 32 * half + 32) of every S tile.
-        // The two threads of a row meet at a named barrier every group, so a thread whose wait has given up keeps
-        // walking (skipping the tensor-memory work) until a point where both leave together.
+        // Two teams of 128 threads (warps 2-5 and 6-9) take the page groups of an item alternately; each has its own
+        // running (maximum, sum) per row and its own O accumulator, so while one team works through the latency chain
+        // of its group (tcgen05.ld, maximum, exponentials, tcgen05.st) the other team's group is in flight too.
+        // Row R = tensor-memory lane; a thread owns the whole row (64 columns) of its team's S tiles.  The two threads
+        // of a row (one per team) meet at a named barrier at the top and at the end of an item only.
         const uint32_t tmem_q = tmem_o + kTcColQ;
-        const int quarter = warp & 3, half = (warp - 2) >> 2;     // lane quarter of tensor memory, column half
+        const int quarter = warp & 3, team = (warp - 2) >> 2;     // lane quarter of tensor memory; team 0 / 1
         const int R = quarter * 32 + lane;
         const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t t_mine = t_lane + kTcColOB * team, t_other = t_lane + kTcColOB * (team ^ 1);
         const float cs = a.scale_log2;
         for (int n = 0;; ++n) {
             const int idx = sched_wait(c, kPhase, n, item);
@@ -1051,12 +1056,12 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             const int n_pages = item.page_end - item.page_begin;
             const int n_groups = (n_pages + 3) >> 2;
             {
-                // the query tile goes to tensor memory (every QK^T of the previous item has completed: its last
-                // s_full was seen): row R = lane of tensor memory, 128 bf16 = 64 words, 32 per thread
+                // the query tile goes to tensor memory (every MMA of the previous item has completed: both teams
+                // waited for its last PV): row R = lane of tensor memory, 128 bf16 = 64 words, 32 per team
                 uint32_t qw[32];
                 if (R < M) {
                     const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
-                    const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * half;
+                    const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * team;
 #pragma unroll
                     for (int cc = 0; cc < 8; ++cc) {
                         const uint4 v = src[cc];
@@ -1066,148 +1071,137 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
 #pragma unroll
                     for (int cc = 0; cc < 32; ++cc) qw[cc] = 0;
                 }
-                tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * half, qw);
+                tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * team, qw);
                 tc_wait_st();
                 tc_fence_before();
                 mbar_arrive(q_ready);
             }
             const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
             float m_run = -INFINITY, l_run = 0.0f;
-            TCP(long long t_ws = 0, t_wk = 0, t_bar = 0, t_ld = 0, t_exp = 0, t_st = 0;)
-            for (int g = 0; g < n_groups; ++g) {
+            for (int g = team; g < n_groups; g += 2) {
                 const int gc = G0 + g, b = gc % kTcSBufs;
-                TCP(long long c0 = clock64();)
                 if (!failed && !mbar_wait(s_full + 8 * b, (gc / kTcSBufs) & 1, &c->abort)) failed = true;
                 failed = __any_sync(0xffffffffu, failed);
-                TCP(long long c1 = clock64(); t_ws += c1 - c0;)
+                if (failed) break;
                 const uint32_t t_s = t_lane + kTcColS + 64 * b;
-                uint32_t sr[32];
+                uint32_t sr[64];
+                tc_fence_after();
+                tc_ld32(t_s, sr);
+                tc_ld32(t_s + 32, sr + 32);
+                tc_wait_ld();
                 float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                if (!failed) {
-                    tc_fence_after();
-                    TCP(long long c2 = clock64();)
-                    tc_ld32(t_s + 32 * half, sr);
-                    tc_wait_ld();
-                    TCP(t_ld += clock64() - c2;)
-                    const int ncols = min(4, n_pages - 4 * g) * kPage;
-                    const int j0 = (item.page_begin + 4 * g) * kPage + 32 * half;
-                    if (ncols < 64 || j0 + 31 > ctx_len) {                  // a partial group or one that holds hidden keys
-                        const int lim = min(ncols - 32 * half - 1, jmax - j0);   // own columns 0..lim are visible
+                const int ncols = min(4, n_pages - 4 * g) * kPage;
+                const int j0 = (item.page_begin + 4 * g) * kPage;
+                if (ncols < 64 || j0 + 63 > ctx_len) {                  // a partial group or one that holds hidden keys
+                    const int lim = min(ncols - 1, jmax - j0);          // columns 0..lim are visible
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const float v = e <= lim ? __uint_as_float(sr[e]) : -INFINITY;
-                            sr[e] = __float_as_uint(v);
-                            mx4[e & 3] = fmaxf(mx4[e & 3], v);
-                        }
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sr[e]));
+                    for (int e = 0; e < 64; ++e) {
+                        const float v = e <= lim ? __uint_as_float(sr[e]) : -INFINITY;
+                        sr[e] = __float_as_uint(v);
+                        mx4[e & 3] = fmaxf(mx4[e & 3], v);
                     }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 64; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sr[e]));
                 }
-                // the two threads of a row exchange their partial maxima
-                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                xch[gc & 1][half][R] = mx;
-                TCP(long long c4 = clock64();)
-                asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
-                TCP(t_bar += clock64() - c4;)
-                mx = fmaxf(mx, xch[gc & 1][half ^ 1][R]);
+                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // the running maximum only moves (and O is only rescaled) when it would grow by more than 2^8
                 float alpha = 1.0f;
                 bool moved = false;
-                if (!failed && mx > m_run && (m_run == -INFINITY || (mx - m_run) * cs > kRescaleLog2)) {
+                if (mx > m_run && (m_run == -INFINITY || (mx - m_run) * cs > kRescaleLog2)) {
                     alpha = fast_exp2((m_run - mx) * cs);                 // 0 when nothing was visible before
                     m_run = mx;
                     l_run *= alpha;
-                    moved = g > 0;
+                    moved = g >= 2;                                       // this team's O holds its earlier groups
                 }
-                if (g > 0 && __any_sync(0xffffffffu, moved)) {
-                    // O is being updated by the previous group's MMAs: wait for them, then scale this thread's half row
-                    if (!mbar_wait(pv_done + 8 * ((gc - 1) % kTcSBufs), ((gc - 1) / kTcSBufs) & 1, &c->abort)) failed = true;
+                if (g >= 2 && __any_sync(0xffffffffu, moved)) {
+                    // this team's O is being updated by its previous group's MMAs: wait for them, then scale the row
+                    if (!mbar_wait(pv_done + 8 * ((gc - 2) % kTcSBufs), ((gc - 2) / kTcSBufs) & 1, &c->abort)) failed = true;
                     failed = __any_sync(0xffffffffu, failed);
-                    if (!failed) {
-                        tc_fence_after();
+                    if (failed) break;
+                    tc_fence_after();
 #pragma unroll 1
-                        for (int cc = 64 * half; cc < 64 * half + 64; cc += 32) {
-                            uint32_t o[32];
-                            tc_ld32(t_lane + cc, o);
-                            tc_wait_ld();
+                    for (int cc = 0; cc < 128; cc += 32) {
+                        uint32_t o[32];
+                        tc_ld32(t_mine + cc, o);
+                        tc_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                            tc_st32(t_lane + cc, o);
-                        }
-                        tc_wait_st();
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tc_st32(t_mine + cc, o);
                     }
-                }
-                if (!failed) {
-                    TCP(long long c5 = clock64();)
-                    const float mc = (m_run == -INFINITY ? 0.0f : m_run) * cs;
-                    float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                    uint32_t pw[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), cs, -mc));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), cs, -mc));
-                        sum4[e & 3] += p0 + p1;
-                        pw[e] = pack_bf16(p0, p1);
-                    }
-                    l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-                    TCP(long long c6 = clock64(); t_exp += c6 - c5;)
-                    tc_st16(t_s + 16 * half, pw);                           // P over the columns S occupied
                     tc_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(p_full + 8 * b);
-                    TCP(t_st += clock64() - c6;)
                 }
-                TCP(t_wk += clock64() - c1;)
+                const float mc = (m_run == -INFINITY ? 0.0f : m_run) * cs;
+                float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                uint32_t pw[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), cs, -mc));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), cs, -mc));
+                    sum4[e & 3] += p0 + p1;
+                    pw[e] = pack_bf16(p0, p1);
+                }
+                l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                tc_st32(t_s, pw);                                         // P over the columns S occupied
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(p_full + 8 * b);
             }
-            TCP(if (blockIdx.x == 0 && R == 0) printf("softmax half %d: wait_s %lld work %lld (ld %lld, pair barrier %lld, exp %lld, st %lld) groups %d\n", half, t_ws, t_wk, t_ld, t_bar, t_exp, t_st, n_groups);)
-            // epilogue: the item's O row, normalised; this thread writes columns [64 * half, 64 * half + 64)
+            // epilogue: every MMA of the item has completed once its last PV has; the two teams' (m, l, O) are merged
+            // and normalised; this thread writes columns [64 * team, 64 * team + 64) of its row
             const int gl = G0 + n_groups - 1;
             if (!failed && !mbar_wait(pv_done + 8 * (gl % kTcSBufs), (gl / kTcSBufs) & 1, &c->abort)) failed = true;
             failed = __any_sync(0xffffffffu, failed);
             tc_fence_after();
-            xl[half][R] = l_run;
+            xm[team][R] = m_run;
+            xl[team][R] = l_run;
             if (failed) c->abort = 1;
             if (bar_any(2 + quarter, 64, failed)) {
                 failed = true;
                 break;
             }
-            l_run += xl[half ^ 1][R];
-            const float inv = l_run > 0.0f ? 1.0f / l_run : 0.0f;
-            const float lse_nat = l_run > 0.0f ? (m_run * cs + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
+            const float m_o = xm[team ^ 1][R], l_o = xl[team ^ 1][R];
+            const float m_all = fmaxf(m_run, m_o);
+            const float w_s = m_run == -INFINITY ? 0.0f : fast_exp2((m_run - m_all) * cs);
+            const float w_o = m_o == -INFINITY ? 0.0f : fast_exp2((m_o - m_all) * cs);
+            const float l_all = l_run * w_s + l_o * w_o;
+            const float inv = l_all > 0.0f ? 1.0f / l_all : 0.0f;
+            const float lse_nat = l_all > 0.0f ? (m_all * cs + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+            const float f_s = w_s * inv, f_o = w_o * inv;
             const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
             const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
-            uint32_t o0[32], o1[32];
-            tc_ld32(t_lane + 64 * half, o0);
-            tc_ld32(t_lane + 64 * half + 32, o1);
-            tc_wait_ld();
-            tc_fence_before();
-            mbar_arrive(o_free);                                            // O may be overwritten by the next item
-#pragma unroll
+#pragma unroll 1
             for (int hh = 0; hh < 2; ++hh) {
-                const uint32_t* o = hh ? o1 : o0;
-                const int cc = 64 * half + 32 * hh;
+                const int cc = 64 * team + 32 * hh;
+                uint32_t os[32], oo[32];
+                tc_ld32(t_mine + cc, os);
+                tc_ld32(t_other + cc, oo);
+                tc_wait_ld();
+                if (hh == 1) {
+                    tc_fence_before();
+                    mbar_arrive(o_free);                                  // both O accumulators may be overwritten by the next item
+                }
+                float v[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e)   // a team without groups (or without visible keys) has weight 0: its O is not read as a number
+                    v[e] = (w_s > 0.0f ? __uint_as_float(os[e]) * f_s : 0.0f) + (w_o > 0.0f ? __uint_as_float(oo[e]) * f_o : 0.0f);
                 if (R < M) {
                     if (item.n_chunks == 1) {
 #pragma unroll
                         for (int e = 0; e < 32; e += 8) {
                             uint32_t w[4];
 #pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                w[j] = pack_bf16(__uint_as_float(o[e + 2 * j]) * inv, __uint_as_float(o[e + 2 * j + 1]) * inv);
+                            for (int j = 0; j < 4; ++j) w[j] = pack_bf16(v[e + 2 * j], v[e + 2 * j + 1]);
                             *reinterpret_cast<uint4*>(a.out + orow * 128 + cc + e) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
                     } else {
                         float* po = a.part_o + ((size_t)item.part_row + R) * 128 + cc;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            *reinterpret_cast<float4*>(po + e) =
-                                make_float4(__uint_as_float(o[e]) * inv, __uint_as_float(o[e + 1]) * inv,
-                                            __uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+                        for (int e = 0; e < 32; e += 4) *reinterpret_cast<float4*>(po + e) = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
                     }
                 }
             }
-            if (R < M && half == 0) {
+            if (R < M && team == 0) {
                 if (item.n_chunks == 1) {
                     if (a.lse) a.lse[orow] = lse_nat;
                 } else {
@@ -1240,8 +1234,8 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Ctrl* c = reinterpret_cast<Ctrl*>(smem + kDataBytes<DH>);
-    __shared__ float xch[2][2][128];   // [group parity][column half][row]: partial row maxima of the tcgen05 phase
-    __shared__ float xl[2][128];       // [column half][row]: partial row sums at the end of an item
+    __shared__ float xm[2][128];       // [team][row]: the teams' running maxima at the end of an item (tcgen05 phase)
+    __shared__ float xl[2][128];       // [team][row]: their running sums
     const int warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) {
@@ -1250,7 +1244,7 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
         }
         for (int b = 0; b < kTcSBufs; ++b) {
             mbar_init(smem_u32(&c->s_full[b]), 1);
-            mbar_init(smem_u32(&c->p_full[b]), kTcSoftmaxThreads);
+            mbar_init(smem_u32(&c->p_full[b]), kTcSoftmaxThreads / 2);   // the team that owns the group
             mbar_init(smem_u32(&c->pv_done[b]), 1);
         }
         mbar_init(smem_u32(&c->q_ready), kTcSoftmaxThreads);
@@ -1281,7 +1275,7 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
     STAMP_MIN(6);
     const int n_items = a.plan[0], n_tc = a.plan[5];
     if (DH == 128 && n_tc > 0) {
-        tc_phase(k2_map, v_map, a, smem, c, xch, xl, a.plan + 8, n_tc);
+        tc_phase(k2_map, v_map, a, smem, c, xm, xl, a.plan + 8, n_tc);
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
