@@ -349,24 +349,26 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// tcgen05 variant of the split kernel for items with many query rows (head_dim 128, rows <= 128).
+// tcgen05 phase: items with many query rows (head_dim 128, 17 <= rows <= 128).
 //
 // With 3+ m-tiles the warp-level MMA path is bound by the tensor pipe and by operand traffic through
 // registers, not by HBM.  Here the query tile is padded to 128 rows (row = tensor-memory lane) and lives in
 // tensor memory for the whole item; pages are handled in groups of four (64 keys):
 //   S[128, 64]  = Q . K_group^T     8 MMAs (M128 N64 K16): A = Q from tensor memory, B = the group's K tiles,
 //                 which TMA lays out contiguously so the 64 key rows form one K-major operand;
-//                 accumulator in tensor memory, double-buffered;
-//   softmax     128 threads, one per row: tcgen05.ld of the row, mask, running max and sum without any
-//                 shuffle; P goes back as bf16 into the columns S occupied (tcgen05.st), so it never
-//                 touches shared memory; O is only rescaled when a row's maximum grows by more than 2^8;
-//   O[128, 128] += P . V_page       one MMA (M128 N128 K16) per page: A = P from tensor memory, B = the V tile
-//                 read MN-major (transposed by its descriptor); accumulator in tensor memory for the item.
-// Both MMAs therefore stream only K and V from shared memory.  Warp 0: TMA producer (4 lanes, one page of
-// every group each), warp 1: MMA issuer and tensor-memory owner, warps 2-5: softmax + epilogue.
+//                 accumulator in tensor memory, three buffers;
+//   softmax     two teams of 128 threads take the groups alternately; a thread owns a row: tcgen05.ld of the
+//                 row, mask, running max and sum without any shuffle; P goes back as bf16 into the columns S
+//                 occupied (tcgen05.st), so it never touches shared memory; the team's O is only rescaled when
+//                 a row's maximum grows by more than 2^8; the teams' (m, l, O) are merged in the item's epilogue;
+//   O_team[128, 128] += P . V_page  one MMA (M128 N128 K16) per page: A = P from tensor memory, B = the V tile
+//                 read MN-major (transposed by its descriptor); one accumulator per team in tensor memory.
+// Both MMAs therefore stream only K and V from shared memory.  Warp 0: TMA producer (lanes 0-3 look up the
+// group's pages, one elected lane issues its loads), warp 1: MMA issuer and tensor-memory owner, warps 2-5 and
+// 6-9: the two softmax teams, which also write the output.
 constexpr int kTcGroupStages = 6;                  // ring of page groups (192 KB in flight)
 constexpr int kTcSBufs = 3;                        // S/P buffers in tensor memory: groups in flight between QK^T and PV
-constexpr int kTcSoftmaxThreads = 256;             // two threads per row, 32 columns each
+constexpr int kTcSoftmaxThreads = 256;             // two teams of 128: one thread per row and team
 static_assert(kThreads == 64 + kTcSoftmaxThreads, "roles of the tcgen05 phase");
 constexpr int kTcPageBytes = kPage * 128 * 2;      // 4 KB: one K or V page tile
 constexpr int kTcGroupBytes = 8 * kTcPageBytes;    // K of 4 pages (16 KB, [half][64 rows][64]) + V of 4 pages
