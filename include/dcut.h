@@ -274,6 +274,41 @@ dcut_status dcut_lm_head_accept(dcut_ctx* ctx, const void* x, const void* w_lm, 
                                 int* out_tokens, int* n_accepted_total, int* row_argmax, void* stream);
 
 /*
+ * The whole verification forward of a model on the retained tokens (Section 3.1: the target verifies the first d_i
+ * draft tokens of every request in one packed forward; the full-layer workload repeated): token embedding,
+ * n_layers decoder layers as in dcut_layer_forward (layer l appends to and reads its own paged cache k_caches[l],
+ * v_caches[l]; all layers share block_table, ctx_lens and the packing metadata), the final RMSNorm with gain
+ * g_final, then dcut_lm_head_accept.  Every step runs in this library's kernels; the hidden states between layers
+ * live in the context.
+ * The dcut_model struct and its three arrays (layers, k_caches, v_caches: n_layers entries each) are HOST memory,
+ * read during the call only; every pointer inside them is a DEVICE pointer: embed bf16 [vocab, hidden], g_final bf16
+ * [hidden], w_lm bf16 [vocab, hidden] (may equal embed: tied weights).  rope_theta must be the same in all layers;
+ * layers[0].rms_eps is used for the final norm (1e-6 when n_layers = 0).
+ * DEVICE in: tok_id i32 [T] = the packed input tokens (request i contributes its bonus token of the previous step
+ * followed by its first d_i draft tokens: the layout dcut_select's packing metadata describes); draft_ids
+ * i32 [B, gamma]; the other arguments as in dcut_layer_forward / dcut_lm_head_accept.  A token id outside [0, vocab)
+ * is read as id 0 and sets device status 6.
+ * DEVICE out: as dcut_lm_head_accept, plus hidden_out bf16 [T_cap, hidden] (optional, may be NULL; 16-byte aligned):
+ * the last layer's output before the final norm (what a feature-level drafter takes from the target).
+ * Alignment: weights, embedding and caches 128 bytes, gains 16 bytes.
+ */
+typedef struct {
+    int n_layers;
+    const dcut_layer_weights* layers;
+    void* const* k_caches;
+    void* const* v_caches;
+    const void* embed;
+    const void* g_final;
+    const void* w_lm;
+    int vocab;
+} dcut_model;
+dcut_status dcut_model_verify(dcut_ctx* ctx, const dcut_model* model, long long num_pages, const int* block_table,
+                              int block_table_stride, const int* ctx_lens, const int* cu_q, const int* tok_req,
+                              const int* tok_pos, const int* tok_id, const int* draft_ids, int B, int gamma, int T_cap,
+                              int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, int* row_argmax,
+                              void* hidden_out, void* stream);
+
+/*
  * dcut_accept without any allocation.  (The paper has no counterpart: this entry point exists for
  * the way the library gets embedded, not for the method.)
  *
@@ -347,7 +382,7 @@ dcut_status dcut_verify_step_host(dcut_ctx* ctx, const dcut_host_step* step, voi
  * and clears it.  A non-zero code also makes this call return DCUT_EDEVICE.  Codes: 1 = a bounded
  * wait in the attention kernel gave up, 2 = a block-table entry outside [0, num_pages) (page 0 was
  * read instead), 3 = the attention work list did not fit the scratch, 4 = a bounded wait in the GEMM
- * kernel gave up, 5 = dcut_commit ran out of room. */
+ * kernel gave up, 5 = dcut_commit ran out of room, 6 = dcut_model_verify met a token id outside [0, vocab). */
 dcut_status dcut_poll_device_status(dcut_ctx* ctx, int* code, void* stream);
 
 #ifdef __cplusplus

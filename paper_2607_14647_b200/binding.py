@@ -29,7 +29,7 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
            "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_lm_head_accept",
-           "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_poll_device_status"]
+           "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_model_verify", "dcut_poll_device_status"]
 
 
 class Limits(C.Structure):
@@ -79,6 +79,13 @@ class LayerWeights(C.Structure):
                [("rms_eps", _f), ("rope_theta", _f)]
 
 
+class Model(C.Structure):
+    _fields_ = [("n_layers", _i), ("layers", C.POINTER(LayerWeights)), ("k_caches", C.POINTER(_vp)),
+                ("v_caches", C.POINTER(_vp)), ("embed", _vp), ("g_final", _vp), ("w_lm", _vp), ("vocab", _i)]
+
+
+_lib.dcut_model_verify.argtypes = [_vp, C.POINTER(Model), _ll, _vp, _i, _vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i,
+                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.dcut_gemm_bf16.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp, _vp, _vp]
 _lib.dcut_lm_head_accept.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.dcut_layer_forward.argtypes = [_vp, C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _vp, _vp,
@@ -331,6 +338,34 @@ class Context:
                                             _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32),
                                             _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32), B, T_cap, _stream()))
         return y
+
+    def model_verify(self, layers: list, embed, g_final, w_lm, k_caches: list, v_caches: list, block_table, ctx_lens,
+                     cu_q, tok_req, tok_pos, tok_id, draft_ids, T_cap: int, rms_eps: float = 1e-6,
+                     rope_theta: float = 1e6, out_tokens: bool = True, row_argmax: bool = False, hidden_out=None):
+        """dcut_model_verify: embedding, len(layers) decoder layers (dicts as in layer_forward, one paged cache pair
+        per layer), final norm, LM head and acceptance in one call."""
+        L = len(layers)
+        names = ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")
+        lw = (LayerWeights * max(L, 1))(*[LayerWeights(*[_ptr(w[n], torch.bfloat16) for n in names], rms_eps, rope_theta)
+                                          for w in layers])
+        kc = (_vp * max(L, 1))(*[_ptr(k, torch.bfloat16) for k in k_caches])
+        vc = (_vp * max(L, 1))(*[_ptr(v, torch.bfloat16) for v in v_caches])
+        m = Model(L, lw, kc, vc, _ptr(embed, torch.bfloat16), _ptr(g_final, torch.bfloat16), _ptr(w_lm, torch.bfloat16),
+                  w_lm.shape[0])
+        B, gamma = draft_ids.shape
+        i32 = dict(dtype=torch.int32, device=embed.device)
+        accept_len, bonus = torch.empty(B, **i32), torch.empty(B, **i32)
+        toks = torch.empty((B, gamma + 1), **i32) if out_tokens else None
+        total = torch.empty(1, **i32)
+        am = torch.full((T_cap,), -1, **i32) if row_argmax else None
+        num_pages = k_caches[0].shape[0] if L else 0
+        self._check(_lib.dcut_model_verify(self._h, C.byref(m), num_pages, _ptr(block_table, torch.int32),
+                                           block_table.shape[1], _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32),
+                                           _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32),
+                                           _ptr(tok_id, torch.int32), _ptr(draft_ids, torch.int32), B, gamma, T_cap,
+                                           _ptr(accept_len), _ptr(bonus), _ptr(toks), _ptr(total), _ptr(am),
+                                           _ptr(hidden_out, torch.bfloat16), _stream()))
+        return accept_len, bonus, toks, total, am
 
     def poll_device_status(self) -> int:
         code = _i(0)

@@ -61,6 +61,8 @@ void free_all(dcut_ctx* c) {
     cudaFree(c->ly_h1);
     cudaFree(c->ly_norm2);
     cudaFree(c->ly_act);
+    cudaFree(c->ly_x[0]);
+    cudaFree(c->ly_x[1]);
     cudaFree(c->ly_inv_freq);
     dcut_free_layer(c);
     cudaFree(c->hs_conf);
@@ -162,6 +164,8 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
         if ((st = dmalloc(c, &c->ly_h1, mt * lim->hidden, "cudaMalloc(layer h1)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->ly_norm2, mt * lim->hidden, "cudaMalloc(layer norm2)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->ly_act, mt * lim->intermediate, "cudaMalloc(layer act)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_x[0], mt * lim->hidden, "cudaMalloc(model x0)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->ly_x[1], mt * lim->hidden, "cudaMalloc(model x1)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->ly_inv_freq, (size_t)lim->head_dim / 2, "cudaMalloc(inv_freq)")) != DCUT_OK) return st;
     }
     if (has_attn && (st = dcut_init_layer(c)) != DCUT_OK) return st;
@@ -318,6 +322,51 @@ dcut_status dcut_accept_rs(dcut_ctx* c, const void* target_logits, const void* d
                                  accept_len, bonus, out_tokens, n_accepted_total, prob, static_cast<cudaStream_t>(stream));
 }
 
+static dcut_status dcut_prepare_rope(dcut_ctx* c, float rope_theta, cudaStream_t stream);
+
+dcut_status dcut_model_verify(dcut_ctx* c, const dcut_model* m, long long num_pages, const int* block_table,
+                              int block_table_stride, const int* ctx_lens, const int* cu_q, const int* tok_req,
+                              const int* tok_pos, const int* tok_id, const int* draft_ids, int B, int gamma, int T_cap,
+                              int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, int* row_argmax,
+                              void* hidden_out, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    if (c->lim.hidden <= 0 || !c->ly_x[0]) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
+    if (!m || !m->embed || !m->g_final || !m->w_lm || m->n_layers < 0 || (m->n_layers > 0 && (!m->layers || !m->k_caches || !m->v_caches)))
+        return dcut_fail(c, DCUT_EINVAL, "incomplete model description");
+    if (!block_table || !ctx_lens || !cu_q || !tok_req || !tok_pos || !tok_id || !draft_ids || !accept_len || !bonus)
+        return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (m->vocab < 1) return dcut_fail(c, DCUT_EINVAL, "vocab must be >= 1");
+    if (B < 1 || B > c->lim.max_B || gamma < 1 || gamma > c->lim.max_gamma || T_cap < B ||
+        T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
+        return dcut_fail(c, DCUT_ECAPACITY, "B = %d, gamma = %d, T_cap = %d outside the limits", B, gamma, T_cap);
+    if (block_table_stride < 1 || block_table_stride > c->lim.max_pages_per_req)
+        return dcut_fail(c, DCUT_ECAPACITY, "block_table_stride = %d outside [1, %d]", block_table_stride, c->lim.max_pages_per_req);
+    uintptr_t al = reinterpret_cast<uintptr_t>(m->w_lm) | reinterpret_cast<uintptr_t>(m->embed);
+    for (int l = 0; l < m->n_layers; ++l) {
+        const dcut_layer_weights& w = m->layers[l];
+        if (!w.w_qkv || !w.w_o || !w.w_gate || !w.w_up || !w.w_down || !w.g_attn || !w.g_mlp || !m->k_caches[l] || !m->v_caches[l])
+            return dcut_fail(c, DCUT_EINVAL, "layer %d: null pointer", l);
+        if (!(w.rope_theta > 1.0f) || !(w.rms_eps >= 0.0f) || w.rope_theta != m->layers[0].rope_theta)
+            return dcut_fail(c, DCUT_EINVAL, "layer %d: rope_theta must exceed 1 and be the same in every layer, rms_eps >= 0", l);
+        if ((reinterpret_cast<uintptr_t>(w.g_attn) | reinterpret_cast<uintptr_t>(w.g_mlp)) & 15)
+            return dcut_fail(c, DCUT_EINVAL, "layer %d: gains must be 16-byte aligned", l);
+        al |= reinterpret_cast<uintptr_t>(w.w_qkv) | reinterpret_cast<uintptr_t>(w.w_o) | reinterpret_cast<uintptr_t>(w.w_gate) |
+              reinterpret_cast<uintptr_t>(w.w_up) | reinterpret_cast<uintptr_t>(w.w_down) |
+              reinterpret_cast<uintptr_t>(m->k_caches[l]) | reinterpret_cast<uintptr_t>(m->v_caches[l]);
+    }
+    if (al & 127) return dcut_fail(c, DCUT_EINVAL, "weights, embedding and caches must be 128-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(m->g_final) | reinterpret_cast<uintptr_t>(hidden_out)) & 15)
+        return dcut_fail(c, DCUT_EINVAL, "g_final and hidden_out must be 16-byte aligned");
+    if (c->lim.vocab > 0 && m->vocab > c->lim.vocab) return dcut_fail(c, DCUT_ECAPACITY, "vocab = %d exceeds the limit %d", m->vocab, c->lim.vocab);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (m->n_layers > 0) {
+        dcut_status st = dcut_prepare_rope(c, m->layers[0].rope_theta, s);
+        if (st != DCUT_OK) return st;
+    }
+    return dcut_launch_model(c, m, num_pages, block_table, block_table_stride, ctx_lens, cu_q, tok_req, tok_pos, tok_id, draft_ids,
+                             B, gamma, T_cap, accept_len, bonus, out_tokens, n_accepted_total, row_argmax, hidden_out, s);
+}
+
 dcut_status dcut_commit(dcut_ctx* c, const int* accept_len, const int* out_tokens, int B, int gamma, int max_ctx,
                         int* ctx_lens, int* bonus_ids, int* stream_tokens, int* stream_len, int stream_cap, void* stream) {
     if (!c) return DCUT_EINVAL;
@@ -363,6 +412,20 @@ dcut_status dcut_lm_head_accept(dcut_ctx* c, const void* x, const void* w_lm, in
                                     n_accepted_total, row_argmax, c->d_row_key, s);
 }
 
+// first call (or a new theta): build the RoPE inverse-frequency table in fp64, round once to fp32
+static dcut_status dcut_prepare_rope(dcut_ctx* c, float rope_theta, cudaStream_t stream) {
+    if (c->ly_theta == rope_theta) return DCUT_OK;
+    const int half = c->lim.head_dim / 2;
+    float tab[128];
+    for (int e = 0; e < half; ++e) tab[e] = (float)pow((double)rope_theta, -2.0 * e / c->lim.head_dim);
+    // the table is read by kernels of this stream only; a pageable source is copied before the call returns
+    dcut_status st = dcut_check_cuda(c, cudaMemcpyAsync(c->ly_inv_freq, tab, sizeof(float) * half, cudaMemcpyHostToDevice, stream),
+                                     "cudaMemcpyAsync(inv_freq)");
+    if (st != DCUT_OK) return st;
+    c->ly_theta = rope_theta;
+    return DCUT_OK;
+}
+
 dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                                void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                                const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
@@ -384,14 +447,9 @@ dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const v
     if ((al & 127) || ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) |
                         reinterpret_cast<uintptr_t>(w->g_attn) | reinterpret_cast<uintptr_t>(w->g_mlp)) & 15))
         return dcut_fail(c, DCUT_EINVAL, "weights and caches must be 128-byte aligned, x / y / gains 16-byte aligned");
-    if (c->ly_theta != w->rope_theta) {   // first call (or a new theta): build the inverse-frequency table in fp64
-        const int half = c->lim.head_dim / 2;
-        float tab[128];
-        for (int e = 0; e < half; ++e) tab[e] = (float)pow((double)w->rope_theta, -2.0 * e / c->lim.head_dim);
-        dcut_status st = dcut_check_cuda(c, cudaMemcpyAsync(c->ly_inv_freq, tab, sizeof(float) * half, cudaMemcpyHostToDevice,
-                                                            static_cast<cudaStream_t>(stream)), "cudaMemcpyAsync(inv_freq)");
+    {
+        dcut_status st = dcut_prepare_rope(c, w->rope_theta, static_cast<cudaStream_t>(stream));
         if (st != DCUT_OK) return st;
-        c->ly_theta = w->rope_theta;
     }
     return dcut_launch_layer(c, w, x, y, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q,
                              tok_req, tok_pos, B, T_cap, static_cast<cudaStream_t>(stream));

@@ -17,6 +17,7 @@
 #define DCUT_DEV_PLAN_OVERFLOW 3       // the attention work list did not fit the context's scratch
 #define DCUT_DEV_GEMM_WAIT_TIMEOUT 4    // a bounded mbarrier wait in the GEMM kernel gave up
 #define DCUT_DEV_COMMIT_OVERFLOW 5      // dcut_commit: a context or a token stream ran out of room
+#define DCUT_DEV_BAD_TOKEN 6            // dcut_model_verify: a token id outside [0, vocab)
 
 // One split-KV work item of the attention kernel: one (request, kv head, page range).
 struct __align__(16) AttnItem {
@@ -73,6 +74,7 @@ struct dcut_ctx {
 
     // decoder-layer workspace (hidden > 0 only), all [max_T, width] bf16
     __nv_bfloat16 *ly_norm, *ly_qkv, *ly_q, *ly_attn, *ly_h1, *ly_norm2, *ly_act;
+    __nv_bfloat16* ly_x[2];   // hidden states between the layers of dcut_model_verify (ping-pong)
     int ly_gemm_pairs;      // clusters of two CTAs the device runs at once
     int ly_gemm_pair_mode;  // 0: the GEMM never runs tiles on pairs of SMs
     float* ly_inv_freq;     // [head_dim / 2]
@@ -156,6 +158,11 @@ dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, c
                                      int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
                                      int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
                                      cudaStream_t stream);
+dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_pages, const int* block_table,
+                              int block_table_stride, const int* ctx_lens, const int* cu_q, const int* tok_req,
+                              const int* tok_pos, const int* tok_id, const int* draft_ids, int B, int gamma, int T_cap,
+                              int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, int* row_argmax,
+                              void* hidden_out, cudaStream_t stream);
 dcut_status dcut_launch_commit(dcut_ctx* ctx, const int* accept_len, const int* out_tokens, int B, int gamma, int max_ctx,
                                int* ctx_lens, int* bonus_ids, int* stream_tokens, int* stream_len, int stream_cap,
                                cudaStream_t stream);

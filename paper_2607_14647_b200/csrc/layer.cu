@@ -729,6 +729,56 @@ dcut_status dcut_init_layer(dcut_ctx* ctx) {
 
 void dcut_free_layer(dcut_ctx* ctx) { free(ctx->layer_maps); }
 
+// x[t, :] = embed[tok_id[t], :] for the packed tokens (ids outside [0, V) read row 0 and set the status word)
+__global__ void __launch_bounds__(128) embed_kernel(const __nv_bfloat16* __restrict__ embed, const int* __restrict__ tok_id,
+                                                    const int* __restrict__ cu_q, int B, int hidden, int V,
+                                                    __nv_bfloat16* __restrict__ x, int* __restrict__ status) {
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
+    const int row = blockIdx.x;
+    if (row >= cu_q[B]) return;
+    int id = tok_id[row];
+    if (id < 0 || id >= V) {
+        if (threadIdx.x == 0) atomicExch(status, DCUT_DEV_BAD_TOKEN);
+        id = 0;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(embed + (size_t)id * hidden);
+    uint4* dst = reinterpret_cast<uint4*>(x + (size_t)row * hidden);
+    for (int v = threadIdx.x; v < hidden / 8; v += 128) dst[v] = src[v];
+}
+
+// The whole verification forward of a small model: embedding, n_layers decoder layers (each with its own paged
+// cache), final RMSNorm, LM head fused with acceptance.
+dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_pages, const int* block_table,
+                              int block_table_stride, const int* ctx_lens, const int* cu_q, const int* tok_req,
+                              const int* tok_pos, const int* tok_id, const int* draft_ids, int B, int gamma, int T_cap,
+                              int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, int* row_argmax,
+                              void* hidden_out, cudaStream_t stream) {
+    const int H = ctx->lim.hidden;
+    __nv_bfloat16* user = static_cast<__nv_bfloat16*>(hidden_out);
+    dcut_status st = dcut_check_cuda(ctx, dcut_launch_pdl(embed_kernel, dim3(T_cap), dim3(128), 0, stream,
+                                                          static_cast<const __nv_bfloat16*>(m->embed), tok_id, cu_q, B, H, m->vocab,
+                                                          (m->n_layers == 0 && user) ? user : ctx->ly_x[0], ctx->d_status),
+                                     "launch embed_kernel");
+    if (st != DCUT_OK) return st;
+    __nv_bfloat16* x = (m->n_layers == 0 && user) ? user : ctx->ly_x[0];
+    for (int l = 0; l < m->n_layers; ++l) {   // ping-pong between the context's two buffers; the last layer may write to the caller
+        __nv_bfloat16* y = (l == m->n_layers - 1 && user) ? user : ctx->ly_x[(l + 1) & 1];
+        st = dcut_launch_layer(ctx, &m->layers[l], x, y, m->k_caches[l], m->v_caches[l], num_pages,
+                               block_table, block_table_stride, ctx_lens, cu_q, tok_req, tok_pos, B, T_cap, stream);
+        if (st != DCUT_OK) return st;
+        x = y;
+    }
+    const float eps = m->n_layers > 0 ? m->layers[0].rms_eps : 1e-6f;
+    if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream,
+                                                   static_cast<const __nv_bfloat16*>(x),
+                                                   static_cast<const __nv_bfloat16*>(m->g_final), cu_q, B, H, eps, ctx->ly_norm),
+                              "launch rmsnorm_kernel")) != DCUT_OK) return st;
+    if ((st = dcut_launch_lm_head_argmax(ctx, ctx->ly_norm, m->w_lm, m->vocab, H, cu_q, B, T_cap, ctx->d_row_key, stream)) != DCUT_OK) return st;
+    return dcut_launch_accept_match(ctx, nullptr, m->vocab, draft_ids, cu_q, B, gamma, accept_len, bonus, out_tokens,
+                                    n_accepted_total, row_argmax, ctx->d_row_key, stream);
+}
+
 // logits = x . w_lm^T reduced on the fly to one (maximum, first column) word per row: the [T, V] logits never exist
 dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void* w_lm, int V, int K, const int* cu_q, int B,
                                        int T_cap, unsigned long long* row_key, cudaStream_t stream) {

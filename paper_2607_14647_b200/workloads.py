@@ -32,6 +32,7 @@ _TAG_CONF, _TAG_IDS, _TAG_CTX, _TAG_REJECT, _TAG_PAGES, _TAG_KV, _TAG_Q, _TAG_LO
 _TAG_LAYER_X, _TAG_LAYER_W = 9, 10
 _TAG_LM_W, _TAG_LM_X = 11, 12
 _TAG_DRAFT_LOGITS, _TAG_UNIFORM = 13, 14
+_TAG_EMBED, _TAG_G_FINAL = 15, 16
 
 
 @dataclass(frozen=True)
@@ -181,11 +182,12 @@ def _randn_bf16(rng: np.random.Generator, n: int, chunk: int = 1 << 24) -> torch
     return out
 
 
-def paged_kv(cfg: WorkloadConfig, ctx_lens: np.ndarray, extra_pages: int = 3) -> PagedKV:
+def paged_kv(cfg: WorkloadConfig, ctx_lens: np.ndarray, extra_pages: int = 3, layer: int = 0) -> PagedKV:
     """KV cache holding, per request, L_i cached tokens plus the gamma+1 block positions
     (bonus and all drafts: the caller appends them before verification, whatever depth
     is later kept).  Physical pages are assigned by a seeded permutation; the last page
-    of a request is partially filled and its unused slots hold ordinary random values."""
+    of a request is partially filled and its unused slots hold ordinary random values.
+    `layer` > 0 gives another layer's cache: same block table, different contents."""
     B, ps = len(ctx_lens), cfg.page_size
     n_tok = ctx_lens.astype(np.int64) + cfg.gamma + 1
     n_pg = (n_tok + ps - 1) // ps
@@ -198,7 +200,7 @@ def paged_kv(cfg: WorkloadConfig, ctx_lens: np.ndarray, extra_pages: int = 3) ->
     for i in range(B):
         bt[i, : n_pg[i]] = perm[o : o + n_pg[i]]
         o += int(n_pg[i])
-    rng = np.random.default_rng([cfg.seed, _TAG_KV])
+    rng = np.random.default_rng([cfg.seed, _TAG_KV] + ([layer] if layer else []))
     shape = (total, cfg.n_kv_heads, ps, cfg.head_dim)
     n = int(np.prod(shape))
     k = _randn_bf16(rng, n).view(shape)
@@ -261,11 +263,11 @@ class LayerWeights:
 
 
 def layer_weights(cfg: WorkloadConfig, hidden: Optional[int] = None,
-                  intermediate: Optional[int] = None) -> LayerWeights:
-    """Random-init weights ~ N(0, 0.02^2), gains ~ 1 + N(0, 0.02^2), bf16."""
+                  intermediate: Optional[int] = None, layer: int = 0) -> LayerWeights:
+    """Random-init weights ~ N(0, 0.02^2), gains ~ 1 + N(0, 0.02^2), bf16; `layer` > 0 draws another layer's set."""
     H = cfg.hidden if hidden is None else hidden
     I = cfg.intermediate if intermediate is None else intermediate
-    rng = np.random.default_rng([cfg.seed, _TAG_LAYER_W])
+    rng = np.random.default_rng([cfg.seed, _TAG_LAYER_W] + ([layer] if layer else []))
 
     def w(r, c):
         return (_randn_bf16(rng, r * c).float() * 0.02).to(torch.bfloat16).view(r, c)
@@ -318,6 +320,34 @@ def lm_head_x_rows(cfg: WorkloadConfig, sel: SelectInputs, depths: np.ndarray, w
                 rng = np.random.default_rng([cfg.seed, _TAG_LM_X, i, t])
                 out[cu[i] + t] = torch.from_numpy(rng.standard_normal(H, dtype=np.float32)).to(torch.bfloat16)
     return out
+
+
+# --------------------------------------------------------------------------- whole-model inputs
+
+@dataclass
+class ModelWeights:
+    embed: torch.Tensor        # bf16 [V, hidden] ~ N(0, 1): the hidden states enter the first layer at unit scale
+    layers: list               # LayerWeights per layer
+    g_final: torch.Tensor      # bf16 [hidden]
+    w_lm: torch.Tensor         # bf16 [V, hidden]
+
+
+def model_weights(cfg: WorkloadConfig, n_layers: int, vocab: Optional[int] = None, hidden: Optional[int] = None,
+                  intermediate: Optional[int] = None) -> ModelWeights:
+    """Random-init weights of a small decoder-only model (untied embedding and LM head)."""
+    V = cfg.vocab if vocab is None else vocab
+    H = cfg.hidden if hidden is None else hidden
+    embed = _randn_bf16(np.random.default_rng([cfg.seed, _TAG_EMBED]), V * H).view(V, H)
+    g = (1.0 + 0.02 * _randn_bf16(np.random.default_rng([cfg.seed, _TAG_G_FINAL]), H).float()).to(torch.bfloat16)
+    return ModelWeights(embed, [layer_weights(cfg, H, intermediate, layer=l) for l in range(n_layers)], g,
+                        lm_head_weight(cfg, V, H))
+
+
+def model_tok_ids(sel: SelectInputs, depths: np.ndarray, vocab: int) -> np.ndarray:
+    """The packed input tokens of the verification forward: per request the previous step's bonus token, then its
+    first d_i draft tokens (ids folded into [0, vocab))."""
+    return np.concatenate([np.concatenate([[sel.bonus_ids[i]], sel.draft_ids[i, : int(d)]])
+                           for i, d in enumerate(depths)]).astype(np.int64) % vocab
 
 
 # --------------------------------------------------------------------------- stochastic variant inputs

@@ -1,0 +1,206 @@
+"""dcut_model_verify (embedding, L decoder layers, final norm, LM head + acceptance in one call) against the oracle and
+against the chain of separately tested calls.
+
+Floating point decides integers here (the argmax of every row), and three layers of bf16 tensors lie between the inputs
+and that decision, so the comparison is split the way the arithmetic allows:
+  * the hidden states after the last layer and every layer's appended K/V: element by element against the oracle,
+    tolerance 3e-2 + 3e-2 |ref| (the one-layer bound 2e-2 + 2e-2 |ref| widened for the depth);
+  * the last stage (final norm, head, argmax) against the oracle run on the GPU's own hidden states: a row's token
+    must be the oracle's whenever the oracle's first and second logits differ by more than the head's tolerance, and
+    must always be a token whose oracle logit is within that tolerance of the maximum;
+  * accepted lengths, bonus tokens and emitted tokens: exactly the prefix match of the row tokens the call reports;
+  * the same outputs and caches, bit for bit, as dcut_layer_forward called layer by layer.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dcut_oracle as orc
+from paper_2607_14647_b200 import workloads as wl
+from tests.gpu_helpers import dev, make_ctx
+
+pytestmark = pytest.mark.gpu
+
+NAMES = ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")
+
+
+def _case(n_layers, depths, vocab=1000, hidden=512, inter=1024, B=6):
+    cfg = wl.custom_config(B=B, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128, ctx_lo=5, ctx_hi=400,
+                           conf_kind="skew_halves", vocab=vocab)
+    sel = wl.select_inputs(cfg)
+    mw = wl.model_weights(cfg, n_layers, vocab, hidden, inter)
+    layers = []
+    for w in mw.layers:          # 2 x the 0.02 init: both branches about half the size of the residual stream, so a
+        d = {n: getattr(w, n) for n in NAMES}   # wiring mistake shows, while no element is a difference of large terms
+        for k in NAMES[:5]:
+            d[k] = (d[k].float() * 2.0).to(torch.bfloat16)
+        layers.append(d)
+    kvs = [wl.paged_kv(cfg, sel.ctx_lens, layer=l) for l in range(n_layers)]
+    if not kvs:
+        kvs_bt = wl.paged_kv(cfg, sel.ctx_lens).block_table
+    else:
+        kvs_bt = kvs[0].block_table
+    drafts = (sel.draft_ids % vocab).astype(np.int32)
+    return cfg, sel, mw, layers, kvs, kvs_bt, drafts
+
+
+def _meta(sel, depths):
+    cu = wl.cu_q_from_depths(depths)
+    tok_req = np.concatenate([np.full(d + 1, i) for i, d in enumerate(depths)]).astype(np.int32)
+    tok_pos = np.concatenate([sel.ctx_lens[i] + np.arange(d + 1) for i, d in enumerate(depths)]).astype(np.int32)
+    return cu, tok_req, tok_pos
+
+
+def _close(got, want, what, tol=3e-2):
+    got = got.float().cpu().numpy().astype(np.float64)
+    want = want.float().numpy().astype(np.float64) if isinstance(want, torch.Tensor) else np.asarray(want, np.float64)
+    err, lim = np.abs(got - want), tol + tol * np.abs(want)
+    assert (err <= lim).all(), f"{what}: worst err/limit {(err / lim).max():.2f}"
+
+
+def _prefix_match(row_tok, drafts, cu, depths):
+    acc, bonus = [], []
+    for i, d in enumerate(depths):
+        m = 0
+        while m < d and row_tok[cu[i] + m] == drafts[i, m]:
+            m += 1
+        acc.append(m)
+        bonus.append(row_tok[cu[i] + m])
+    return np.array(acc), np.array(bonus)
+
+
+def _run_gpu(cfg, sel, mw, layers, kvs, bt, drafts, depths, tok):
+    cu, tok_req, tok_pos = _meta(sel, depths)
+    T = int(cu[-1])
+    ctx = make_ctx(cfg, max_pages=bt.shape[1], hidden=mw.embed.shape[1], intermediate=layers[0]["w_gate"].shape[0] if layers else 1024,
+                   vocab=mw.w_lm.shape[0])
+    d_layers = [{k: dev(v) for k, v in w.items()} for w in layers]
+    d_k, d_v = [dev(k.k_cache) for k in kvs], [dev(k.v_cache) for k in kvs]
+    hid = torch.zeros((cfg.t_cap, mw.embed.shape[1]), dtype=torch.bfloat16, device="cuda")
+    out = ctx.model_verify(d_layers, dev(mw.embed), dev(mw.g_final), dev(mw.w_lm), d_k, d_v, dev(bt), dev(sel.ctx_lens),
+                           dev(cu), dev(tok_req), dev(tok_pos), dev(tok.astype(np.int32)), dev(drafts), cfg.t_cap,
+                           cfg.rms_eps, cfg.rope_theta, row_argmax=True, hidden_out=hid)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    return ctx, out, hid[:T].cpu(), d_layers, d_k, d_v
+
+
+def _check_last_stage(hid_gpu, mw, row_tok, eps):
+    """Final norm + head + argmax, given the GPU's own last hidden states."""
+    n = orc._as_bf16_tensor(orc.round_bf16(orc.rmsnorm(hid_gpu, mw.g_final, eps)))
+    logits = orc.linear(n, mw.w_lm)
+    top = np.sort(logits, 1)[:, ::-1]
+    tol = 1e-2 + 1e-2 * np.abs(top[:, 0])        # one bf16 rounding of n (shared) + fp32 accumulation + bf16 logits
+    chosen = logits[np.arange(len(row_tok)), row_tok]
+    assert (chosen >= top[:, 0] - tol).all(), "a row token is not within tolerance of the maximum logit"
+    clear = top[:, 0] - top[:, 1] > tol
+    assert clear.sum() > 0.5 * len(row_tok)
+    assert np.array_equal(row_tok[clear], logits.argmax(1)[clear])
+
+
+@pytest.mark.parametrize("n_layers", [1, 3])
+def test_model_against_the_oracle(n_layers):
+    depths = np.array([16, 0, 3, 9, 1, 16], np.int32)
+    cfg, sel, mw, layers, kvs, bt, drafts = _case(n_layers, depths)
+    tok = wl.model_tok_ids(sel, depths, mw.w_lm.shape[0])
+    ref, ref_logits, ref_hidden, ref_caches = orc.model_verify(
+        tok, mw.embed, layers, mw.g_final, mw.w_lm, [k.k_cache for k in kvs], [k.v_cache for k in kvs], bt, sel.ctx_lens,
+        depths, drafts, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.page_size, cfg.rms_eps, cfg.rope_theta)
+    ctx, (acc, bonus, toks, total, am), hid, _, d_k, d_v = _run_gpu(cfg, sel, mw, layers, kvs, bt, drafts, depths, tok)
+    cu = wl.cu_q_from_depths(depths)
+    T = int(cu[-1])
+    _close(hid, ref_hidden[n_layers - 1], "hidden states after the last layer")
+    for l in range(n_layers):
+        kc, vc = d_k[l].cpu(), d_v[l].cpu()
+        touched = torch.zeros(kc.shape[0], dtype=torch.bool)
+        for i, d in enumerate(depths):
+            for t in range(d + 1):
+                pos = int(sel.ctx_lens[i]) + t
+                page = bt[i, pos // 16]
+                touched[page] = True
+                _close(kc[page, :, pos % 16], ref_caches[l][0][page, :, pos % 16], f"layer {l} appended K")
+                _close(vc[page, :, pos % 16], ref_caches[l][1][page, :, pos % 16], f"layer {l} appended V")
+        assert torch.equal(kc[~touched], kvs[l].k_cache[~touched]) and torch.equal(vc[~touched], kvs[l].v_cache[~touched])
+    row_tok = am[:T].cpu().numpy()
+    assert (am[T:] == -1).all()
+    _check_last_stage(hid, mw, row_tok, cfg.rms_eps)
+    # end to end: wherever the oracle's own decision is clear of the accumulated tolerance, the token is the oracle's
+    top = np.sort(ref_logits, 1)[:, ::-1]
+    clear = top[:, 0] - top[:, 1] > 3e-2 + 3e-2 * np.abs(top[:, 0])
+    assert clear.sum() > 0.4 * T
+    assert np.array_equal(row_tok[clear], ref_logits.argmax(1)[clear])
+    want_acc, want_bonus = _prefix_match(row_tok, drafts, cu, depths)
+    assert np.array_equal(acc.cpu().numpy(), want_acc) and np.array_equal(bonus.cpu().numpy(), want_bonus)
+    assert int(total.item()) == int(want_acc.sum()) + cfg.B
+    toks = toks.cpu().numpy()
+    for i in range(cfg.B):
+        m = want_acc[i]
+        assert np.array_equal(toks[i, :m], drafts[i, :m]) and toks[i, m] == want_bonus[i] and (toks[i, m + 1:] == -1).all()
+    ctx.close()
+
+
+def test_model_equals_the_chain_of_layer_calls_and_accepts_its_own_greedy_drafts():
+    """Drafts produced by the model itself (greedy, through dcut_model_verify position by position on scratch caches)
+    are all accepted; the spoiled position ends the accepted prefix; the call is bit-identical to the layer-by-layer chain."""
+    n_layers = 2
+    depths = np.array([5, 5, 5, 5], np.int32)
+    cfg, sel, mw, layers, kvs, bt, drafts = _case(n_layers, depths, B=4)
+    V = mw.w_lm.shape[0]
+    drafts = drafts.copy()
+    cu = wl.cu_q_from_depths(depths)
+    bonus0 = (sel.bonus_ids % V).astype(np.int64)
+
+    def tok_of():
+        return np.concatenate([np.concatenate([[bonus0[i]], drafts[i, : int(d)]]) for i, d in enumerate(depths)])
+
+    for t in range(5):                          # greedy decoding: position t's prediction becomes draft t + 1
+        ctx, (_, _, _, _, am), _, _, _, _ = _run_gpu(cfg, sel, mw, layers, kvs, bt, drafts, depths, tok_of())
+        drafts[:, t] = am.cpu().numpy()[cu[:-1] + t]
+        ctx.close()
+    spoil = {1: 2, 3: 0}
+    for i, t in spoil.items():
+        drafts[i, t] = (drafts[i, t] + 1) % V
+    tok = tok_of()
+    ctx, (acc, bonus, toks, total, am), hid, d_layers, d_k, d_v = _run_gpu(cfg, sel, mw, layers, kvs, bt, drafts, depths, tok)
+    assert acc.cpu().tolist() == [5, 2, 5, 0]
+    # the chain of public calls: embedding gather by torch, dcut_layer_forward per layer on fresh caches
+    _, tok_req, tok_pos = _meta(sel, depths)
+    x = dev(mw.embed)[torch.from_numpy(tok).cuda()].contiguous()
+    k2, v2 = [dev(k.k_cache) for k in kvs], [dev(k.v_cache) for k in kvs]
+    for l in range(n_layers):
+        y = torch.empty_like(x)
+        ctx.layer_forward(d_layers[l], x, y, k2[l], v2[l], dev(bt), dev(sel.ctx_lens), dev(cu), dev(tok_req), dev(tok_pos),
+                          cfg.t_cap, cfg.rms_eps, cfg.rope_theta)
+        x = y
+    torch.cuda.synchronize()
+    assert torch.equal(x.cpu(), hid)
+    for l in range(n_layers):
+        assert torch.equal(k2[l], d_k[l]) and torch.equal(v2[l], d_v[l])
+    ctx.close()
+
+
+def test_zero_layers_bad_token_and_argument_checks():
+    from paper_2607_14647_b200 import binding
+    depths = np.array([2, 0, 1, 3, 0, 2], np.int32)
+    cfg, sel, mw, layers, kvs, bt, drafts = _case(0, depths, vocab=300)
+    tok = wl.model_tok_ids(sel, depths, 300)
+    ctx, (acc, bonus, toks, total, am), hid, _, _, _ = _run_gpu(cfg, sel, mw, [], [], bt, drafts, depths, tok)
+    T = len(tok)
+    assert torch.equal(hid, mw.embed[torch.from_numpy(tok)])                       # embedding rows, bit for bit
+    _check_last_stage(hid, mw, am[:T].cpu().numpy(), cfg.rms_eps)
+    # a token id outside the vocabulary: read as id 0, reported through the status word
+    cu, tok_req, tok_pos = _meta(sel, depths)
+    bad = tok.astype(np.int32).copy()
+    bad[1] = 300
+    args = ([], dev(mw.embed), dev(mw.g_final), dev(mw.w_lm), [], [], dev(bt), dev(sel.ctx_lens), dev(cu), dev(tok_req),
+            dev(tok_pos))
+    ctx.model_verify(*args, dev(bad), dev(drafts), cfg.t_cap, hidden_out=None)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 6 and ctx.poll_device_status() == 0
+    with pytest.raises(binding.DcutError):                                        # T_cap beyond the context's limit
+        ctx.model_verify(*args, dev(bad), dev(drafts), cfg.t_cap + 1)
+    ctx.close()
+    plain = make_ctx(cfg, max_pages=1, vocab=300)                                  # a context without layer shapes
+    with pytest.raises(binding.DcutError):
+        plain.model_verify(*args, dev(bad), dev(drafts), cfg.t_cap)
+    plain.close()
