@@ -52,6 +52,9 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--gamma", type=int, default=0,
                     help="draft tokens per request, if not the config's (7 = the paper's block-8 setting)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="with a layer config (4): time the whole verification forward of a model of this many decoder "
+                         "layers (dcut_model_verify) instead of one layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the step's kernels one by one instead of replaying a CUDA graph")
     return ap.parse_args()
@@ -560,10 +563,135 @@ def run_dcut(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------------------------ whole-model arm
+
+def run_model(args):
+    """select -> dcut_model_verify (embedding, L layers, final norm, LM head + acceptance) per step, for a random-init
+    model of the layer config's shapes.  Weights and the per-layer KV caches are drawn on the device (seeded)."""
+    world, rank, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    from paper_2607_14647_b200 import binding
+    cfg = wl.config(args.config)
+    if cfg.hidden <= 0:
+        raise SystemExit("--layers needs a layer config (--config 4)")
+    L, H, I, V = args.layers, cfg.hidden, cfg.intermediate, cfg.vocab
+    dev = torch.device("cuda", local)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed)
+
+    def w(r, c, scale=0.02):
+        return (torch.randn((r, c), generator=gen, device=dev, dtype=torch.float32) * scale).to(torch.bfloat16)
+
+    qkv_rows, q_w = (cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim, cfg.n_q_heads * cfg.head_dim
+    ones = torch.ones(H, dtype=torch.bfloat16, device=dev)
+    layers = [dict(w_qkv=w(qkv_rows, H), w_o=w(H, q_w), w_gate=w(I, H), w_up=w(I, H), w_down=w(H, I), g_attn=ones, g_mlp=ones)
+              for _ in range(L)]
+    k0, v0 = kv.k_cache.to(dev), kv.v_cache.to(dev)
+    k_caches = [k0] + [k0.clone() for _ in range(L - 1)]       # own memory per layer; the contents do not matter for time
+    v_caches = [v0] + [v0.clone() for _ in range(L - 1)]
+    embed, w_lm = w(V, H, 1.0), w(V, H)
+    d_conf, d_draft = torch.from_numpy(sel.conf).to(dev), torch.from_numpy(sel.draft_ids % V).to(dev)
+    d_bonus, d_ctx = torch.from_numpy(sel.bonus_ids % V).to(dev), torch.from_numpy(sel.ctx_lens).to(dev)
+    d_bt = torch.from_numpy(kv.block_table).to(dev)
+    ctx = binding.Context(max_B=cfg.B, max_gamma=cfg.gamma, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                          head_dim=cfg.head_dim, page_size=cfg.page_size, max_pages_per_req=kv.max_pages_per_req,
+                          vocab=V, hidden=H, intermediate=I)
+    model = ctx.make_model(layers, embed, ones, w_lm, k_caches, v_caches, cfg.rms_eps, cfg.rope_theta)
+    cap = cfg.t_cap
+    state = {"sel": None, "out": None}
+
+    def step(ev=None):
+        so = state["sel"] = ctx.select(d_conf, d_draft, d_bonus, d_ctx, out=state["sel"])
+        if ev:
+            ev[0].record()
+        state["out"] = ctx.model_verify(model, d_bt, d_ctx, so.cu_q, so.tok_req, so.tok_pos, so.tok_id, d_draft, cap,
+                                        out=state["out"])
+        if ev:
+            ev[1].record()
+
+    def timed(n):
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        barrier(world)
+        start.record()
+        for k in range(n):
+            step(evs[k])
+        end.record()
+        barrier(world)
+        return max_over_ranks(start.elapsed_time(end), world) / n, statistics.mean(a.elapsed_time(b) for a, b in evs)
+
+    def depths_now():
+        so = ctx.select(d_conf, d_draft, d_bonus, d_ctx)
+        torch.cuda.synchronize()
+        return so.depths.cpu().numpy()
+
+    grid = sorted(set(int(round(x)) for x in np.linspace(cfg.B, cap, args.cost_points)))
+    prof = []
+    for T in grid:                                   # step latency against the packed length, profiled on this GPU
+        ctx.set_cost_buckets(cfg.B, cfg.gamma, [T], [1.0])
+        step()
+        prof.append(timed(3)[0])
+    cost = np.maximum.accumulate(np.interp(np.arange(cap + 1), grid, prof)).astype(np.float32)
+    arms = {"pruned": cost, "full_gamma": np.ones(cap + 1, np.float32),
+            "gamma0": (1.0 + 10.0 * np.maximum(0, np.arange(cap + 1) - cfg.B)).astype(np.float32)}
+    flops_tok = L * layer_flops(cfg, 1) + 2.0 * H * V
+    res = {}
+    sampler = ClockSampler(local) if rank == 0 else None
+    for name, table in arms.items():
+        ctx.set_cost_dense(table)
+        d = depths_now()
+        T = int(d.sum()) + cfg.B
+        for _ in range(max(3, args.warmup)):
+            step()
+        ms, fwd_ms = timed(args.steps)
+        assert ctx.poll_device_status() == 0
+        planted = int((np.minimum(d, sel.reject_index) + 1).sum())
+        res[name] = {"T": T, "ms_per_step": round(ms, 4), "forward_ms": round(fwd_ms, 4),
+                     "accepted_tokens_planted": planted, "accepted_tokens_by_the_random_init_model": int(state["out"][3].item()),
+                     "tokens_per_s": round(world * planted / (ms * 1e-3), 1),
+                     "verified_tokens_per_s": round(world * T / (ms * 1e-3), 1),
+                     "forward_tflops": round(flops_tok * T / fwd_ms / 1e9, 1),
+                     "kv_streamed_gb": round(L * attn_algorithmic_bytes(cfg, sel.ctx_lens, d) / 1e9, 2)}
+    clocks = sampler.stop() if sampler else {}
+    if rank != 0:
+        return
+    pkj = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    tf_peak = float(pkj.get("bf16_tflops_sustained", pkj.get("bf16_tflops", 1400.0)))
+    p = res["pruned"]
+    weights_gb = (L * (qkv_rows * H + H * q_w + 3 * H * I) + 2 * V * H) * 2 / 1e9
+    line = {
+        "metric": METRIC, "value": p["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": p["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"configs[{cfg.index}] {cfg.name} as a {L}-layer model: B={cfg.B} gamma={cfg.gamma} {cfg.n_q_heads}q/"
+                               f"{cfg.n_kv_heads}kv Dh={cfg.head_dim} hidden={H} intermediate={I} V={V} ctx {cfg.ctx_lo}-{cfg.ctx_hi}",
+                   "arm": "D-cut pruned (cost table profiled on this GPU); step = dcut_select + dcut_model_verify",
+                   "accepted_tokens": "random-init weights accept no draft, so the numerator is the workload's planted acceptance "
+                                      "min(d_i, reject_index_i) + 1 per request; the LM head, argmax and prefix match run in the timed region",
+                   "launch": "kernel by kernel (programmatic dependent launch)",
+                   "l2": f"each step streams {weights_gb:.1f} GB of weights and {p['kv_streamed_gb']:.1f} GB of KV once (L2 is 126 MB)",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "arms": res,
+        "roofline": {"kernel": "all kernels of dcut_model_verify (projections, attention, norms, LM head), pruned arm",
+                     "bound": "tensor", "achieved": p["forward_tflops"], "peak": tf_peak, "unit": "TFLOP/s",
+                     "frac": round(p["forward_tflops"] / tf_peak, 4),
+                     "peak_source": "of measured (sustained)" if "bf16_tflops_sustained" in pkj else "of fallback", "traffic": None},
+        "e2e": None, "gpu_launches": (5 + 10 * L) * args.steps,   # select, embed, 10 per layer, norm, LM head, match
+        "cost_table_ms": {str(t): round(c, 4) for t, c in zip(grid, prof)}, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.layers > 0:
+        run_model(args)
     else:
         run_dcut(args)
 

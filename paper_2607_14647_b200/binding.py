@@ -92,6 +92,14 @@ _lib.dcut_layer_forward.argtypes = [_vp, C.POINTER(LayerWeights), _vp, _vp, _vp,
                                     _i, _i, _vp]
 
 
+@dataclass
+class PreparedModel:
+    rec: "Model"
+    keep: tuple              # the ctypes arrays and tensors `rec` points into
+    num_pages: int
+    device: torch.device
+
+
 class DcutError(RuntimeError):
     def __init__(self, status: int, msg: str):
         super().__init__(f"{STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else status}: {msg}")
@@ -339,33 +347,39 @@ class Context:
                                             _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32), B, T_cap, _stream()))
         return y
 
-    def model_verify(self, layers: list, embed, g_final, w_lm, k_caches: list, v_caches: list, block_table, ctx_lens,
-                     cu_q, tok_req, tok_pos, tok_id, draft_ids, T_cap: int, rms_eps: float = 1e-6,
-                     rope_theta: float = 1e6, out_tokens: bool = True, row_argmax: bool = False, hidden_out=None):
-        """dcut_model_verify: embedding, len(layers) decoder layers (dicts as in layer_forward, one paged cache pair
-        per layer), final norm, LM head and acceptance in one call."""
+    def make_model(self, layers: list, embed, g_final, w_lm, k_caches: list, v_caches: list, rms_eps: float = 1e-6,
+                   rope_theta: float = 1e6) -> "PreparedModel":
+        """The dcut_model record for model_verify: `layers` are dicts as in layer_forward, one paged cache pair per
+        layer.  The returned object keeps the tensors alive."""
         L = len(layers)
+        assert len(k_caches) == L and len(v_caches) == L
         names = ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")
         lw = (LayerWeights * max(L, 1))(*[LayerWeights(*[_ptr(w[n], torch.bfloat16) for n in names], rms_eps, rope_theta)
                                           for w in layers])
         kc = (_vp * max(L, 1))(*[_ptr(k, torch.bfloat16) for k in k_caches])
         vc = (_vp * max(L, 1))(*[_ptr(v, torch.bfloat16) for v in v_caches])
-        m = Model(L, lw, kc, vc, _ptr(embed, torch.bfloat16), _ptr(g_final, torch.bfloat16), _ptr(w_lm, torch.bfloat16),
-                  w_lm.shape[0])
+        rec = Model(L, lw, kc, vc, _ptr(embed, torch.bfloat16), _ptr(g_final, torch.bfloat16), _ptr(w_lm, torch.bfloat16),
+                    w_lm.shape[0])
+        return PreparedModel(rec, (lw, kc, vc, layers, embed, g_final, w_lm, k_caches, v_caches),
+                             k_caches[0].shape[0] if L else 0, embed.device)
+
+    def model_verify(self, model: "PreparedModel", block_table, ctx_lens, cu_q, tok_req, tok_pos, tok_id, draft_ids,
+                     T_cap: int, out_tokens: bool = True, row_argmax: bool = False, hidden_out=None, out=None):
+        """dcut_model_verify: embedding, the model's decoder layers, final norm, LM head and acceptance in one call.
+        `out` = (accept_len, bonus, out_tokens, total, row_argmax) of an earlier call is written in place."""
         B, gamma = draft_ids.shape
-        i32 = dict(dtype=torch.int32, device=embed.device)
-        accept_len, bonus = torch.empty(B, **i32), torch.empty(B, **i32)
-        toks = torch.empty((B, gamma + 1), **i32) if out_tokens else None
-        total = torch.empty(1, **i32)
-        am = torch.full((T_cap,), -1, **i32) if row_argmax else None
-        num_pages = k_caches[0].shape[0] if L else 0
-        self._check(_lib.dcut_model_verify(self._h, C.byref(m), num_pages, _ptr(block_table, torch.int32),
+        if out is None:
+            i32 = dict(dtype=torch.int32, device=model.device)
+            out = (torch.empty(B, **i32), torch.empty(B, **i32), torch.empty((B, gamma + 1), **i32) if out_tokens else None,
+                   torch.empty(1, **i32), torch.full((T_cap,), -1, **i32) if row_argmax else None)
+        accept_len, bonus, toks, total, am = out
+        self._check(_lib.dcut_model_verify(self._h, C.byref(model.rec), model.num_pages, _ptr(block_table, torch.int32),
                                            block_table.shape[1], _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32),
                                            _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32),
                                            _ptr(tok_id, torch.int32), _ptr(draft_ids, torch.int32), B, gamma, T_cap,
                                            _ptr(accept_len), _ptr(bonus), _ptr(toks), _ptr(total), _ptr(am),
                                            _ptr(hidden_out, torch.bfloat16), _stream()))
-        return accept_len, bonus, toks, total, am
+        return out
 
     def poll_device_status(self) -> int:
         code = _i(0)

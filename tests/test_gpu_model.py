@@ -77,9 +77,9 @@ def _run_gpu(cfg, sel, mw, layers, kvs, bt, drafts, depths, tok):
     d_layers = [{k: dev(v) for k, v in w.items()} for w in layers]
     d_k, d_v = [dev(k.k_cache) for k in kvs], [dev(k.v_cache) for k in kvs]
     hid = torch.zeros((cfg.t_cap, mw.embed.shape[1]), dtype=torch.bfloat16, device="cuda")
-    out = ctx.model_verify(d_layers, dev(mw.embed), dev(mw.g_final), dev(mw.w_lm), d_k, d_v, dev(bt), dev(sel.ctx_lens),
-                           dev(cu), dev(tok_req), dev(tok_pos), dev(tok.astype(np.int32)), dev(drafts), cfg.t_cap,
-                           cfg.rms_eps, cfg.rope_theta, row_argmax=True, hidden_out=hid)
+    model = ctx.make_model(d_layers, dev(mw.embed), dev(mw.g_final), dev(mw.w_lm), d_k, d_v, cfg.rms_eps, cfg.rope_theta)
+    out = ctx.model_verify(model, dev(bt), dev(sel.ctx_lens), dev(cu), dev(tok_req), dev(tok_pos),
+                           dev(tok.astype(np.int32)), dev(drafts), cfg.t_cap, row_argmax=True, hidden_out=hid)
     torch.cuda.synchronize()
     assert ctx.poll_device_status() == 0
     return ctx, out, hid[:T].cpu(), d_layers, d_k, d_v
@@ -192,8 +192,8 @@ def test_zero_layers_bad_token_and_argument_checks():
     cu, tok_req, tok_pos = _meta(sel, depths)
     bad = tok.astype(np.int32).copy()
     bad[1] = 300
-    args = ([], dev(mw.embed), dev(mw.g_final), dev(mw.w_lm), [], [], dev(bt), dev(sel.ctx_lens), dev(cu), dev(tok_req),
-            dev(tok_pos))
+    model = ctx.make_model([], dev(mw.embed), dev(mw.g_final), dev(mw.w_lm), [], [])
+    args = (model, dev(bt), dev(sel.ctx_lens), dev(cu), dev(tok_req), dev(tok_pos))
     ctx.model_verify(*args, dev(bad), dev(drafts), cfg.t_cap, hidden_out=None)
     torch.cuda.synchronize()
     assert ctx.poll_device_status() == 6 and ctx.poll_device_status() == 0
