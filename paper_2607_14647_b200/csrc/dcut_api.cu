@@ -127,6 +127,7 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
         unsigned char* p = nullptr;
         if ((st = dmalloc(c, &p, dcut_accept_rs_scratch_bytes(c, c->rs_n_seg), "cudaMalloc(rs scratch)")) != DCUT_OK) return st;
         c->d_rs_scratch = p;
+        if ((st = dcut_init_accept_rs(c)) != DCUT_OK) return st;
     }
     if ((st = dcut_init_select(c)) != DCUT_OK) return st;
     if ((st = dcut_init_accept(c)) != DCUT_OK) return st;

@@ -141,6 +141,7 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
                                int* out_tokens, int* n_accepted_total, unsigned long long* row_key,
                                cudaStream_t stream);
 size_t dcut_accept_rs_scratch_bytes(const dcut_ctx* ctx, int n_seg);
+dcut_status dcut_init_accept_rs(dcut_ctx* ctx);
 dcut_status dcut_launch_accept_rs(dcut_ctx* ctx, const void* target_logits, const void* draft_logits, int V,
                                   const int* draft_ids, const int* cu_q, int B, int gamma, int T_cap,
                                   const float* u_accept, const float* u_sample, int* accept_len, int* bonus,
