@@ -292,7 +292,7 @@ dcut_status dcut_verify_attn(dcut_ctx* c, const void* q, const void* k_cache, co
         return dcut_fail(c, DCUT_ECAPACITY, "cache has too many token rows for 32-bit tile coordinates");
     if (!(scale > 0.0f) || isinf(scale)) return dcut_fail(c, DCUT_EINVAL, "scale must be positive and finite");
     return dcut_launch_verify_attn(c, q, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q, B,
-                                   T_cap, scale, out, lse, static_cast<cudaStream_t>(stream));
+                                   T_cap, scale, out, lse, 0, static_cast<cudaStream_t>(stream));
 }
 
 dcut_status dcut_accept(dcut_ctx* c, const void* logits, int V, const int* draft_ids, const int* cu_q, int B, int gamma,
@@ -453,7 +453,7 @@ dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const v
         if (st != DCUT_OK) return st;
     }
     return dcut_launch_layer(c, w, x, y, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q,
-                             tok_req, tok_pos, B, T_cap, static_cast<cudaStream_t>(stream));
+                             tok_req, tok_pos, B, T_cap, 0, static_cast<cudaStream_t>(stream));
 }
 
 dcut_status dcut_poll_device_status(dcut_ctx* c, int* code, void* stream) {

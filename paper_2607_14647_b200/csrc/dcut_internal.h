@@ -149,7 +149,7 @@ dcut_status dcut_launch_accept_rs(dcut_ctx* ctx, const void* target_logits, cons
 dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                     long long num_pages, const int* block_table, int block_table_stride,
                                     const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
-                                    void* out, float* lse, cudaStream_t stream);
+                                    void* out, float* lse, int reuse_plan, cudaStream_t stream);
 dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
                              const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream);
 dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void* w_lm, int V, int K, const int* cu_q, int B,
@@ -170,4 +170,4 @@ dcut_status dcut_launch_commit(dcut_ctx* ctx, const int* accept_len, const int* 
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
-                              int T_cap, cudaStream_t stream);
+                              int T_cap, int reuse_plan, cudaStream_t stream);

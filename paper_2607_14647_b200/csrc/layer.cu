@@ -606,27 +606,33 @@ __global__ void __launch_bounds__(256) rope_append_kernel(RopeArgs a) {
     const int slot = pos & 15;
     const int row_w = (a.n_q_heads + 2 * a.n_kv_heads) * Dh;
     const __nv_bfloat16* row = a.qkv + (size_t)tok * row_w;
-    const int n_rot = (a.n_q_heads + a.n_kv_heads) * half;   // rotated pairs of the q and k heads
-    for (int idx = threadIdx.x; idx < n_rot; idx += blockDim.x) {
-        const int h = idx / half, e = idx - h * half;
-        float sn, cs;
-        sincosf((float)pos * a.inv_freq[e], &sn, &cs);
-        const float x0 = __bfloat162float(row[h * Dh + e]), x1 = __bfloat162float(row[h * Dh + e + half]);
-        const __nv_bfloat16 y0 = __float2bfloat16_rn(x0 * cs - x1 * sn), y1 = __float2bfloat16_rn(x1 * cs + x0 * sn);
-        if (h < a.n_q_heads) {
-            __nv_bfloat16* q = a.q_out + ((size_t)tok * a.n_q_heads + h) * Dh;
-            q[e] = y0;
-            q[e + half] = y1;
-        } else {
-            __nv_bfloat16* k = a.k_cache + (((size_t)page * a.n_kv_heads + (h - a.n_q_heads)) * 16 + slot) * Dh;
-            k[e] = y0;
-            k[e + half] = y1;
+    // A thread keeps its two rotation pairs (e, e + 1) and walks the heads: one sincos pair per thread, 4-byte accesses.
+    // (head_dim is a multiple of 16, so half is even and rows are 4-byte aligned.)
+    const int lanes_per_head = half >> 1;                      // threads that cover one head
+    const int heads_per_pass = blockDim.x / lanes_per_head;
+    const int e = (threadIdx.x % lanes_per_head) * 2;
+    float sn0, cs0, sn1, cs1;
+    sincosf((float)pos * a.inv_freq[e], &sn0, &cs0);
+    sincosf((float)pos * a.inv_freq[e + 1], &sn1, &cs1);
+    if ((int)threadIdx.x < heads_per_pass * lanes_per_head) {
+        for (int h = threadIdx.x / lanes_per_head; h < a.n_q_heads + a.n_kv_heads; h += heads_per_pass) {
+            const uint32_t lo = *reinterpret_cast<const uint32_t*>(row + h * Dh + e);
+            const uint32_t hi = *reinterpret_cast<const uint32_t*>(row + h * Dh + e + half);
+            const float a0 = bf_lo(lo), a1 = bf_hi(lo), b0 = bf_lo(hi), b1 = bf_hi(hi);
+            const uint32_t y_lo = pack_bf16(a0 * cs0 - b0 * sn0, a1 * cs1 - b1 * sn1);
+            const uint32_t y_hi = pack_bf16(b0 * cs0 + a0 * sn0, b1 * cs1 + a1 * sn1);
+            __nv_bfloat16* dst = h < a.n_q_heads
+                                     ? a.q_out + ((size_t)tok * a.n_q_heads + h) * Dh
+                                     : a.k_cache + (((size_t)page * a.n_kv_heads + (h - a.n_q_heads)) * 16 + slot) * Dh;
+            *reinterpret_cast<uint32_t*>(dst + e) = y_lo;
+            *reinterpret_cast<uint32_t*>(dst + e + half) = y_hi;
         }
     }
-    const __nv_bfloat16* vrow = row + (a.n_q_heads + a.n_kv_heads) * Dh;
-    for (int idx = threadIdx.x; idx < a.n_kv_heads * Dh; idx += blockDim.x) {
-        const int h = idx / Dh, e = idx - h * Dh;
-        a.v_cache[(((size_t)page * a.n_kv_heads + h) * 16 + slot) * Dh + e] = vrow[idx];
+    const uint4* vrow = reinterpret_cast<const uint4*>(row + (a.n_q_heads + a.n_kv_heads) * Dh);   // 16-byte aligned: Dh % 8 == 0
+    const int vec_per_head = Dh >> 3;
+    for (int idx = threadIdx.x; idx < a.n_kv_heads * vec_per_head; idx += blockDim.x) {
+        const int h = idx / vec_per_head, v = idx - h * vec_per_head;
+        reinterpret_cast<uint4*>(a.v_cache + (((size_t)page * a.n_kv_heads + h) * 16 + slot) * Dh)[v] = vrow[idx];
     }
 }
 
@@ -765,7 +771,8 @@ dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_
     for (int l = 0; l < m->n_layers; ++l) {   // ping-pong between the context's two buffers; the last layer may write to the caller
         __nv_bfloat16* y = (l == m->n_layers - 1 && user) ? user : ctx->ly_x[(l + 1) & 1];
         st = dcut_launch_layer(ctx, &m->layers[l], x, y, m->k_caches[l], m->v_caches[l], num_pages,
-                               block_table, block_table_stride, ctx_lens, cu_q, tok_req, tok_pos, B, T_cap, stream);
+                               block_table, block_table_stride, ctx_lens, cu_q, tok_req, tok_pos, B, T_cap,
+                               l > 0 /* the attention work list of layer 0 serves every layer */, stream);
         if (st != DCUT_OK) return st;
         x = y;
     }
@@ -827,7 +834,7 @@ dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const 
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
-                              int T_cap, cudaStream_t stream) {
+                              int T_cap, int reuse_plan, cudaStream_t stream) {
     const dcut_limits& l = ctx->lim;
     const int H = l.hidden, I = l.intermediate, Dh = l.head_dim;
     const int qkv_w = (l.n_q_heads + 2 * l.n_kv_heads) * Dh, q_w = l.n_q_heads * Dh;
@@ -871,7 +878,7 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rope_append_kernel, dim3(T_cap), dim3(256), 0, stream, r), "launch rope_append_kernel")) != DCUT_OK) return st;
     // 4. attention
     st = dcut_launch_verify_attn(ctx, ctx->ly_q, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens,
-                                 cu_q, B, T_cap, 1.0f / sqrtf((float)Dh), ctx->ly_attn, nullptr, stream);
+                                 cu_q, B, T_cap, 1.0f / sqrtf((float)Dh), ctx->ly_attn, nullptr, reuse_plan, stream);
     if (st != DCUT_OK) return st;
     // 5. h1 = x + attn . Wo^T
     g.N_out = H; g.K = q_w; g.out = ctx->ly_h1; g.residual = static_cast<const __nv_bfloat16*>(x);

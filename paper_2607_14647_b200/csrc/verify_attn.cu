@@ -1301,7 +1301,7 @@ struct CombineArgs {
     const int* req_part;
     const float* part_o;
     const float* part_lse;
-    const int* plan;
+    int* plan;   // read; the two queue heads are rewound
     int B, n_q_heads, n_kv_heads, tokens_per_req;
     __nv_bfloat16* out;
     float* lse;
@@ -1315,6 +1315,12 @@ __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     STAMP_MAX(5);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        // the item kernel has drained both queues: rewind them, so that the same plan can serve another launch over
+        // the same batch (the layers of one model forward)
+        a.plan[8] = 0;
+        a.plan[9] = a.plan[5];
+    }
     if (a.plan[4] || a.plan[3] == 0) return;   // overflow, or no request was cut: nothing to merge
     const int lane = threadIdx.x & 31;
     const int h = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -1431,7 +1437,7 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
 dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                     long long num_pages, const int* block_table, int block_table_stride,
                                     const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
-                                    void* out, float* lse, cudaStream_t stream) {
+                                    void* out, float* lse, int reuse_plan, cudaStream_t stream) {
     CUtensorMap km, vm, k2m;
     dcut_status st = make_cache_map(ctx, &km, k_cache, num_pages);
     if (st != DCUT_OK) return st;
@@ -1469,9 +1475,11 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.items = ctx->d_items;
     pa.plan = ctx->d_plan;
     pa.req_part = ctx->d_req_part;
-    st = dcut_check_cuda(ctx, dcut_launch_pdl(attn_plan_kernel, dim3(1), dim3(B <= 256 ? 256 : kPlanThreads),
-                                              sizeof(unsigned long long) * pa.npad, stream, pa), "launch attn_plan_kernel");
-    if (st != DCUT_OK) return st;
+    if (!reuse_plan) {   // reuse_plan: the previous launch on this stream had the same ctx_lens, cu_q and B (its work list stands)
+        st = dcut_check_cuda(ctx, dcut_launch_pdl(attn_plan_kernel, dim3(1), dim3(B <= 256 ? 256 : kPlanThreads),
+                                                  sizeof(unsigned long long) * pa.npad, stream, pa), "launch attn_plan_kernel");
+        if (st != DCUT_OK) return st;
+    }
 
     AttnArgs aa;
     aa.q = static_cast<const __nv_bfloat16*>(q);
