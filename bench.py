@@ -159,6 +159,21 @@ def attn_algorithmic_bytes(cfg, ctx_lens: np.ndarray, depths: np.ndarray) -> int
             + pages * 4 * cfg.n_kv_heads)
 
 
+def cost_grid(cfg, points: int, tiled: bool) -> list:
+    """Packed lengths at which the step is timed for the cost table.  Evenly spaced; where the forward holds GEMMs
+    (`tiled`), whose cost moves in steps of their 128-row tiles, the points are the last length of a row block and the
+    first of the next, thinned to about `points`, so that the table shows the steps and the selector can stop at them."""
+    cap = cfg.t_cap
+    if not tiled:
+        return sorted(set(int(round(x)) for x in np.linspace(cfg.B, cap, points)))
+    edges = [k * 128 for k in range(1, cap // 128 + 1) if cfg.B < k * 128 < cap]
+    stride = max(1, int(np.ceil(2 * len(edges) / max(points - 2, 1))))
+    pts = {cfg.B, cap}
+    for e in edges[::stride]:
+        pts.update((e, e + 1))
+    return sorted(pts)
+
+
 def peaks() -> dict:
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -309,7 +324,7 @@ def run_dcut(args):
         return step_sel.depths.cpu().numpy()
 
     # ---- cost table: step latency against the packed length T, profiled on this GPU ---------------
-    grid = sorted(set(int(round(x)) for x in np.linspace(cfg.B, cap, args.cost_points)))
+    grid = cost_grid(cfg, args.cost_points, is_layer)
     prof = []
     for T in grid:
         ctx.set_cost_buckets(cfg.B, cfg.gamma, [T], [1.0])
@@ -629,7 +644,7 @@ def run_model(args):
         torch.cuda.synchronize()
         return so.depths.cpu().numpy()
 
-    grid = sorted(set(int(round(x)) for x in np.linspace(cfg.B, cap, args.cost_points)))
+    grid = cost_grid(cfg, args.cost_points, True)
     prof = []
     for T in grid:                                   # step latency against the packed length, profiled on this GPU
         ctx.set_cost_buckets(cfg.B, cfg.gamma, [T], [1.0])

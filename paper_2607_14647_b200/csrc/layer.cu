@@ -21,6 +21,7 @@
 // dependent launch and waits for its predecessor before touching global memory.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <limits.h>
 #include <math.h>
 #include <stdlib.h>
 
@@ -38,6 +39,18 @@ constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256
 constexpr int kWaitLimit = 1 << 22;
 
 enum GemmMode { kPlain = 0, kResidual = 1, kSwiGLU = 2, kArgmax = 3 };
+
+// Widths of the output tile that the one-SM mode may use: 256, 224, ..., 64 columns.  A narrower tile costs a little
+// efficiency per flop and buys more tiles, which is what a GEMM with fewer than one wave of 128 x 256 tiles needs
+// (T = 600, N = 4096: 80 tiles for 148 SMs at width 256, 130 at width 160).  One tensor map of the weight per width
+// (box = half the width in rows: a B tile is loaded as two halves, which is also how the SwiGLU tile is put together).
+constexpr int kNumBn = 7;
+__host__ __device__ constexpr int bn_of(int i) { return BN - 32 * i; }
+struct BMaps {
+    CUtensorMap m[kNumBn];
+};
+constexpr unsigned kBnMaskAll = (1u << kNumBn) - 1;
+constexpr unsigned kBnMaskSwiGLU = 0x55;   // widths whose halves are whole 32-column epilogue steps: 256, 192, 128, 64
 
 // ------------------------------------------------------------------------------------------------ PTX
 
@@ -114,7 +127,7 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
     return d;
 }
 // Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N = 256, M = 128.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+constexpr uint32_t kIdescNoN = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);   // N >> 3 goes to bits 17..22
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -136,23 +149,41 @@ struct GemmArgs {
     unsigned long long* row_key;     // kArgmax: one packed (ordered maximum, ~column) word per row
     int V;                           // kArgmax: live columns (rows of the weight)
     int pairs;                       // launched as clusters of two CTAs: the pair mode may be chosen
+    unsigned bn_mask;                // tile widths whose tensor maps were supplied (bit i: bn_of(i)); bit 0 always
+    int force;                       // experiments: -1 = let gemm_plan choose, 0..6 = that width on one SM, 8..14 = on a pair
     int* status;
 };
 
-// Epilogue of one 128 x 256 accumulator (this thread: tensor-memory lane = output row `row`), for every mode.
+// the map of width index i; every address is formed statically (kernel parameter space)
+__device__ __forceinline__ const CUtensorMap* pick_map(const BMaps& s, int i) {
+    switch (i) {
+        case 1: return &s.m[1];
+        case 2: return &s.m[2];
+        case 3: return &s.m[3];
+        case 4: return &s.m[4];
+        case 5: return &s.m[5];
+        case 6: return &s.m[6];
+        default: return &s.m[0];
+    }
+}
+
+// Epilogue of one 128 x bn accumulator (this thread: tensor-memory lane = output row `row`), for every mode.  Columns
+// past N_out (a ragged last tile of a narrow width) were computed on zero weight rows and are not stored.
 template <int MODE>
-__device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row, int n_tile, uint32_t t_row) {
+__device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row, int n_tile, uint32_t t_row, int bn) {
     if (MODE == kSwiGLU) {
-        __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + (size_t)n_tile * (BN / 2);
+        const int half = bn >> 1, col0 = n_tile * half;
+        __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + col0;
 #pragma unroll 1
-        for (int c = 0; c < BN / 2; c += 32) {
+        for (int c = 0; c < half; c += 32) {
             uint32_t gt[32], up[32];
             tc_ld32(t_row + c, gt);
-            tc_ld32(t_row + BN / 2 + c, up);
+            tc_ld32(t_row + half + c, up);
             tc_wait_ld();
             if (row < T) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
+                    if (col0 + c + e >= g.N_out) break;
                     uint32_t o[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -170,9 +201,9 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
         // (ordered value << 32 | ~column): largest value, lowest column, whatever order the tiles finish in.
         float best = -INFINITY;
         int bidx = -1;
-        const int col0 = n_tile * BN;
+        const int col0 = n_tile * bn;
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = 0; c < bn; c += 32) {
             uint32_t av[32];
             tc_ld32(t_row + c, av);
             tc_wait_ld();
@@ -196,16 +227,18 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
         if (row < T && bidx >= 0)
             atomicMax(g.row_key + row, ((unsigned long long)dcut_ordered_bits(best) << 32) | (0xffffffffu - (unsigned int)bidx));
     } else {
-        __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + (size_t)n_tile * BN;
-        const __nv_bfloat16* rrow = MODE == kResidual ? g.residual + (size_t)row * g.N_out + (size_t)n_tile * BN : nullptr;
+        const int col0 = n_tile * bn;
+        __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + col0;
+        const __nv_bfloat16* rrow = MODE == kResidual ? g.residual + (size_t)row * g.N_out + col0 : nullptr;
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = 0; c < bn; c += 32) {
             uint32_t av[32];
             tc_ld32(t_row + c, av);
             tc_wait_ld();
             if (row < T) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
+                    if (col0 + c + e >= g.N_out) break;
                     uint4 res = make_uint4(0, 0, 0, 0);
                     if (MODE == kResidual) res = *reinterpret_cast<const uint4*>(rrow + c + e);
                     const uint32_t rw[4] = {res.x, res.y, res.z, res.w};
@@ -237,7 +270,7 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
 
 constexpr int kG2Stages = 6;
 constexpr int kG2StageBytes = kATile + kBTile / 2;     // 32 KB
-constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
+constexpr uint32_t kIdesc2NoN = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * BM) >> 4) << 24);
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -284,21 +317,44 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
 //   (gemm_use_pairs).
 // In both the operand ring and its barriers continue across tiles and the accumulator is double-buffered in tensor
 // memory (2 x 256 columns), so the epilogue of one tile overlaps the main loop of the next.
-__device__ __forceinline__ bool gemm_use_pairs(int T, int n_tiles, int K, int grid) {
-    const int tiles1 = ((T + BM - 1) / BM) * n_tiles, tiles2 = ((T + 2 * BM - 1) / (2 * BM)) * n_tiles;
-    const int pairs = grid >> 1;
-    if (tiles1 == 0 || pairs == 0) return false;
-    const int w1 = (tiles1 + grid - 1) / grid, w2 = (tiles2 + pairs - 1) / pairs;   // waves either way
-    // measured: a pair tile takes ~0.93 of two single tiles, and a single short wave (K = 4096) is faster on single SMs
-    return w2 * 15 < w1 * 16 && (w1 >= 2 || K >= 8192);
+// The cheapest way to run this launch under a model fitted to measurements on the four projections of an 8B-class
+// layer at 17 packed lengths from 64 to 1088 (every width, both modes): time = waves x (4 bn + 1664) on one SM per
+// tile, waves x (7 bn + 800) on a pair.  (A pair tile moves two thirds of the bytes per flop from L2 and its MMAs are
+// issued at about 0.57 of the one-SM rate per column; the constants stand for what a tile costs whatever its width.)
+// Over those 68 cases the pick is within 0.3 % (geometric mean; worst case 7 %) of the best measured choice.  Returns
+// the width index, + kPlanPair for the pair mode; the wider tile wins ties.
+constexpr int kPlanPair = 8;
+__device__ __forceinline__ int gemm_plan(int T, const GemmArgs& g, bool swiglu, int grid) {
+    const int m1 = (T + BM - 1) / BM, m2 = (T + 2 * BM - 1) / (2 * BM);
+    if (m1 == 0) return 0;
+    if (g.force >= 0) return g.force;
+    const int n_pairs = g.pairs ? grid >> 1 : 0;
+    int best = 0, best_cost = INT_MAX;
+    for (int i = 0; i < kNumBn; ++i) {
+        if (!((g.bn_mask >> i) & 1)) continue;
+        const int bn = bn_of(i), per = swiglu ? bn >> 1 : bn, n_tiles = (g.N_out + per - 1) / per;
+        const int cost1 = ((m1 * n_tiles + grid - 1) / grid) * (4 * bn + 1664);
+        if (cost1 < best_cost) {
+            best_cost = cost1;
+            best = i;
+        }
+        if (n_pairs > 0) {
+            const int cost2 = ((m2 * n_tiles + n_pairs - 1) / n_pairs) * (7 * bn + 800);
+            if (cost2 < best_cost) {
+                best_cost = cost2;
+                best = kPlanPair + i;
+            }
+        }
+    }
+    return best;
 }
 
 static_assert(kGemmStages * kGemmStageBytes == kG2Stages * kG2StageBytes, "both modes use the same operand area");
 
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
-                    const __grid_constant__ CUtensorMap b2_map, GemmArgs g) {
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ BMaps b_maps,
+                    const __grid_constant__ BMaps b2_maps, GemmArgs g) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
@@ -331,7 +387,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
     const int T = g.cu_q[g.B];
-    const bool pairs = g.pairs && gemm_use_pairs(T, g.n_tiles, g.K, (int)gridDim.x);
+    const int plan_all = gemm_plan(T, g, MODE == kSwiGLU, (int)gridDim.x);
+    const bool pairs = plan_all >= kPlanPair;
+    const int plan = plan_all & 7;                                  // width index
+    const int bn = bn_of(plan), half_rows = bn >> 1;                // tile width; a B tile is loaded as two halves
+    const int per = MODE == kSwiGLU ? half_rows : bn;               // output columns per tile
+    const int n_tiles = (g.N_out + per - 1) / per;
     if (warp == 1) {   // tensor memory: two 128 x 256 fp32 accumulators (per CTA; allocated for the pair in pair mode)
         if (pairs) {
             asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
@@ -350,11 +411,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
 
     if (!pairs) {
         const int m_tiles = (T + BM - 1) / BM;
-        const int n_work = m_tiles * g.n_tiles;   // (a CTA without work falls through the loops below)
+        const int n_work = m_tiles * n_tiles;                      // (a CTA without work falls through the loops below)
         const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
         const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages), acc_empty = acc_full + 16;
         if (warp == 0) {
             // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
+            const CUtensorMap* b_map = pick_map(b_maps, plan);
+            const CUtensorMap* b2_map = pick_map(b2_maps, plan);
+            const uint32_t stage_tx = kATile + bn * BK * 2;
             int kc = 0;   // k-blocks issued so far, over all tiles
             for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x) {
                 const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
@@ -367,14 +431,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                     if (elect_one()) {
                         const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
                         const uint32_t bar = full_bar + 8 * s;
-                        mbar_arrive_expect_tx(bar, kGemmStageBytes);
+                        mbar_arrive_expect_tx(bar, stage_tx);
                         tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
-                        if (MODE == kSwiGLU) {   // 128 gate rows, then the 128 up rows of the same features
-                            tma_load_2d(b_dst, &b_map, kb * BK, n_tile * (BN / 2), bar);
-                            tma_load_2d(b_dst + kBTile / 2, &b2_map, kb * BK, n_tile * (BN / 2), bar);
-                        } else {
-                            tma_load_2d(b_dst, &b_map, kb * BK, n_tile * BN, bar);
-                            tma_load_2d(b_dst + kBTile / 2, &b_map, kb * BK, n_tile * BN + BN / 2, bar);
+                        if (MODE == kSwiGLU) {   // the gate rows, then the up rows of the same features
+                            tma_load_2d(b_dst, b_map, kb * BK, n_tile * half_rows, bar);
+                            tma_load_2d(b_dst + half_rows * BK * 2, b2_map, kb * BK, n_tile * half_rows, bar);
+                        } else {                 // (weight rows past N read as zeros)
+                            tma_load_2d(b_dst, b_map, kb * BK, n_tile * bn, bar);
+                            tma_load_2d(b_dst + half_rows * BK * 2, b_map, kb * BK, n_tile * bn + half_rows, bar);
                         }
                     }
                     __syncwarp();
@@ -382,6 +446,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
             }
         } else if (warp == 1) {
             // ---------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
+            const uint32_t idesc = kIdescNoN | ((uint32_t)(bn >> 3) << 17);
             int kc = 0, it = 0;
             for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
                 const int acc = it & 1;
@@ -404,7 +469,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                         const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
     #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
-                            tc_mma(tmem_d, da + 2 * k, db + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+                            tc_mma(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
                         tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
                     }
                     __syncwarp();
@@ -427,7 +492,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                 }
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-                gemm_epilogue<MODE>(g, T, row, n_tile, t_row);
+                gemm_epilogue<MODE>(g, T, row, n_tile, t_row, bn);
                 // this accumulator may be overwritten once all four epilogue warps have read it
                 tc_fence_before();
                 mbar_arrive(acc_empty + 8 * acc);
@@ -435,7 +500,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
         }
     } else {
         const int m_tiles = (T + 2 * BM - 1) / (2 * BM);          // 256-row tiles of the pair
-        const int n_work = m_tiles * g.n_tiles;
+        const int n_work = m_tiles * n_tiles;
         const uint32_t rank = cluster_ctarank();                   // 0: leader
         const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
         const uint32_t full_bar = smem_u32(bars2), empty_bar = smem_u32(bars2 + kG2Stages);
@@ -443,6 +508,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
         if (warp == 0) {
             // ---------------------------------------------------------------- TMA producer (both CTAs)
             const uint32_t lead_full = mapa_rank(full_bar, 0);
+            const CUtensorMap* b_map = pick_map(b_maps, plan);
+            const CUtensorMap* b2_map = pick_map(b2_maps, plan);
+            const uint32_t pair_tx = 2 * (kATile + half_rows * BK * 2);   // both CTAs' A tile and half of the B tile
             int kc = 0;
             for (int w = pair; w < n_work && !failed; w += n_pairs) {
                 const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * (2 * BM) + (int)rank * BM;
@@ -454,13 +522,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                     }
                     if (elect_one()) {
                         const uint32_t a_dst = smem_u32(smem + s * kG2StageBytes), b_dst = a_dst + kATile;
-                        if (rank == 0) mbar_arrive_expect_tx(full_bar + 8 * s, 2 * kG2StageBytes);
+                        if (rank == 0) mbar_arrive_expect_tx(full_bar + 8 * s, pair_tx);
                         const uint32_t bar = lead_full + 8 * s;
                         tma_load_2d_pair(a_dst, &a_map, kb * BK, m0, bar);
                         if (MODE == kSwiGLU)      // the leader's half: 128 gate rows; the peer's: the 128 up rows of the same features
-                            tma_load_2d_pair(b_dst, rank == 0 ? &b_map : &b2_map, kb * BK, n_tile * (BN / 2), bar);
+                            tma_load_2d_pair(b_dst, rank == 0 ? b_map : b2_map, kb * BK, n_tile * half_rows, bar);
                         else
-                            tma_load_2d_pair(b_dst, &b_map, kb * BK, n_tile * BN + (int)rank * (BN / 2), bar);
+                            tma_load_2d_pair(b_dst, b_map, kb * BK, n_tile * bn + (int)rank * half_rows, bar);
                     }
                     __syncwarp();
                 }
@@ -468,6 +536,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
         } else if (warp == 1) {
             // ---------------------------------------------------------------- MMA issuer (leader CTA only)
             if (rank == 0) {
+                const uint32_t idesc2 = kIdesc2NoN | ((uint32_t)(bn >> 3) << 17);
                 int kc = 0, it = 0;
                 for (int w = pair; w < n_work && !failed; w += n_pairs, ++it) {
                     const int acc = it & 1;
@@ -490,7 +559,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                             const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
     #pragma unroll
                             for (int k = 0; k < BK / 16; ++k)
-                                tc_mma2(tmem_d, da + 2 * k, db + 2 * k, kIdesc2, (kb | k) ? 1u : 0u);
+                                tc_mma2(tmem_d, da + 2 * k, db + 2 * k, idesc2, (kb | k) ? 1u : 0u);
                             tc_commit_pair(empty_bar + 8 * s);     // the stage is free in both CTAs once these MMAs have read it
                         }
                         __syncwarp();
@@ -515,7 +584,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                 }
                 tc_fence_after();
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-                gemm_epilogue<MODE>(g, T, row, n_tile, t_row);
+                gemm_epilogue<MODE>(g, T, row, n_tile, t_row, bn);
                 tc_fence_before();
                 mbar_arrive_remote(lead_acc_empty + 8 * acc);
             }
@@ -656,12 +725,32 @@ dcut_status make_kmajor_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, l
     return DCUT_OK;
 }
 
+// The weight's tensor maps for the tile widths in `mask` (box = half the width in rows)
+dcut_status make_weight_maps(dcut_ctx* ctx, BMaps* maps, const void* w, long long rows, long long cols, unsigned mask) {
+    for (int i = 0; i < kNumBn; ++i) {
+        if (!((mask >> i) & 1)) continue;
+        dcut_status st = make_kmajor_map(ctx, &maps->m[i], w, rows, cols, bn_of(i) / 2);
+        if (st != DCUT_OK) return st;
+    }
+    return DCUT_OK;
+}
+
 template <int MODE>
-dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& b2, int n_tiles,
-                        int T_cap, const GemmArgs& g, cudaStream_t stream) {
+dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, const BMaps& b2, int n_tiles,
+                        int T_cap, unsigned bn_mask, const GemmArgs& g, cudaStream_t stream) {
     GemmArgs ga = g;
     ga.n_tiles = n_tiles;
-    const int n_work = ((T_cap + BM - 1) / BM) * n_tiles;
+    ga.bn_mask = bn_mask | 1u;
+    {
+        const char* envf = getenv("DCUT_GEMM_FORCE");
+        ga.force = envf ? atoi(envf) : -1;
+        if (ga.force >= 0 && (!((ga.bn_mask >> (ga.force & 7)) & 1) || (ga.force >= 8 && !ga.pairs))) ga.force = -1;
+    }
+    // work items at the narrowest width that may be chosen (the widest has n_tiles per row block)
+    int narrow = 0;
+    for (int i = 0; i < kNumBn; ++i)
+        if ((ga.bn_mask >> i) & 1) narrow = i;
+    const int n_work = ((T_cap + BM - 1) / BM) * ((n_tiles * BN + bn_of(narrow) - 1) / bn_of(narrow));
     int grid = n_work < ctx->sm_count ? n_work : ctx->sm_count;   // persistent: at most one CTA per SM
     ga.pairs = 0;
     if (ctx->ly_gemm_pairs > 0) {
@@ -689,11 +778,17 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const CUtensorMap& 
                            "launch gemm_tcgen05_kernel");
 }
 
-struct LayerMaps {
+// Tensor maps of the layers seen so far: the weights' (for every tile width) in a small direct-mapped cache keyed by the
+// layer's w_qkv pointer, so that a model forward does not encode 36 x 31 maps on every call
+struct WeightMaps {
     const void* w[5];
-    CUtensorMap m[5];   // w_qkv, w_o, w_gate, w_up, w_down
+    BMaps m[5];         // w_qkv, w_o, w_gate, w_up, w_down
+};
+constexpr int kLayerCache = 64;
+struct LayerMaps {
     CUtensorMap act[4]; // norm out, attention out, norm-2 out, mlp activation
     bool act_ready;
+    WeightMaps cache[kLayerCache];
 };
 
 }  // namespace
@@ -709,6 +804,8 @@ dcut_status dcut_init_layer(dcut_ctx* ctx) {
         // (DCUT_GEMM_2CTA=0: never).  ly_gemm_pairs = how many such clusters the device runs at once.
         const char* env = getenv("DCUT_GEMM_2CTA");
         ctx->ly_gemm_pair_mode = (!env || atoi(env) != 0) ? 1 : 0;
+        const char* envw = getenv("DCUT_GEMM_WIDTHS");   // bit i allows tile width 256 - 32 i in the one-SM mode
+        ctx->ly_gemm_bn_mask = ((envw ? (unsigned)strtoul(envw, nullptr, 0) : kBnMaskAll) & kBnMaskAll) | 1u;
         ctx->ly_gemm_pairs = 0;
         {
             cudaLaunchAttribute attr[1];
@@ -789,10 +886,13 @@ dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_
 // logits = x . w_lm^T reduced on the fly to one (maximum, first column) word per row: the [T, V] logits never exist
 dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void* w_lm, int V, int K, const int* cu_q, int B,
                                        int T_cap, unsigned long long* row_key, cudaStream_t stream) {
-    CUtensorMap am, bm;
+    CUtensorMap am;
+    BMaps bm;
     dcut_status st = make_kmajor_map(ctx, &am, x, T_cap, K, BM);
     if (st != DCUT_OK) return st;
-    if ((st = make_kmajor_map(ctx, &bm, w_lm, V, K, BN / 2)) != DCUT_OK) return st;   // rows past V read as zeros
+    // rows past V read as zeros; hundreds of tiles per row block: only the full width is offered
+    if ((st = make_weight_maps(ctx, &bm, w_lm, V, K, 1u)) != DCUT_OK) return st;
+    for (int i = 1; i < kNumBn; ++i) bm.m[i] = bm.m[0];
     GemmArgs g;
     g.cu_q = cu_q;
     g.B = B;
@@ -803,19 +903,21 @@ dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void*
     g.row_key = row_key;
     g.V = V;
     g.status = ctx->d_status;
-    return launch_gemm<kArgmax>(ctx, am, bm, bm, (V + BN - 1) / BN, T_cap, g, stream);
+    return launch_gemm<kArgmax>(ctx, am, bm, bm, (V + BN - 1) / BN, T_cap, 1u, g, stream);
 }
 
 dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
                              const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream) {
     // generic entry used by dcut_gemm_bf16 (tests, benchmarks): encodes its maps on every call
-    CUtensorMap am, bm, b2m;
+    CUtensorMap am;
+    BMaps bm, b2m;
     dcut_status st = make_kmajor_map(ctx, &am, a, T_cap, K, BM);
     if (st != DCUT_OK) return st;
-    const int rows_w = mode == kSwiGLU ? N : N;
-    if ((st = make_kmajor_map(ctx, &bm, w, rows_w, K, BN / 2)) != DCUT_OK) return st;
+    const unsigned mask = (mode == kSwiGLU ? ctx->ly_gemm_bn_mask & kBnMaskSwiGLU : ctx->ly_gemm_bn_mask) | 1u;
+    for (int i = 0; i < kNumBn; ++i) bm.m[i] = am;     // entries outside the mask are never used; keep them defined
+    if ((st = make_weight_maps(ctx, &bm, w, N, K, mask)) != DCUT_OK) return st;
     b2m = bm;
-    if (mode == kSwiGLU && (st = make_kmajor_map(ctx, &b2m, w2, rows_w, K, BN / 2)) != DCUT_OK) return st;
+    if (mode == kSwiGLU && (st = make_weight_maps(ctx, &b2m, w2, N, K, mask)) != DCUT_OK) return st;
     GemmArgs g;
     g.cu_q = cu_q;
     g.B = B;
@@ -826,9 +928,9 @@ dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const 
     g.row_key = nullptr;
     g.V = 0;
     g.status = ctx->d_status;
-    if (mode == kSwiGLU) return launch_gemm<kSwiGLU>(ctx, am, bm, b2m, N / (BN / 2), T_cap, g, stream);
-    if (mode == kResidual) return launch_gemm<kResidual>(ctx, am, bm, b2m, N / BN, T_cap, g, stream);
-    return launch_gemm<kPlain>(ctx, am, bm, b2m, N / BN, T_cap, g, stream);
+    if (mode == kSwiGLU) return launch_gemm<kSwiGLU>(ctx, am, bm, b2m, N / (BN / 2), T_cap, mask, g, stream);
+    if (mode == kResidual) return launch_gemm<kResidual>(ctx, am, bm, b2m, N / BN, T_cap, mask, g, stream);
+    return launch_gemm<kPlain>(ctx, am, bm, b2m, N / BN, T_cap, mask, g, stream);
 }
 
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
@@ -850,10 +952,12 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     }
     const void* wp[5] = {w->w_qkv, w->w_o, w->w_gate, w->w_up, w->w_down};
     const long long wr[5] = {qkv_w, H, I, I, H}, wc[5] = {H, q_w, H, H, I};
+    const unsigned mask = ctx->ly_gemm_bn_mask, wmask[5] = {mask, mask, mask & kBnMaskSwiGLU, mask & kBnMaskSwiGLU, mask};
+    WeightMaps* wm = &lm->cache[(reinterpret_cast<uintptr_t>(w->w_qkv) >> 8) % kLayerCache];
     for (int i = 0; i < 5; ++i)
-        if (lm->w[i] != wp[i]) {
-            if ((st = make_kmajor_map(ctx, &lm->m[i], wp[i], wr[i], wc[i], BN / 2)) != DCUT_OK) return st;
-            lm->w[i] = wp[i];
+        if (wm->w[i] != wp[i]) {
+            if ((st = make_weight_maps(ctx, &wm->m[i], wp[i], wr[i], wc[i], wmask[i] | 1u)) != DCUT_OK) return st;
+            wm->w[i] = wp[i];
         }
     GemmArgs g;
     g.cu_q = cu_q;
@@ -868,7 +972,7 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
                               "launch rmsnorm_kernel")) != DCUT_OK) return st;
     // 2. qkv = n . Wqkv^T
     g.N_out = qkv_w; g.K = H; g.out = ctx->ly_qkv; g.residual = nullptr;
-    if ((st = launch_gemm<kPlain>(ctx, lm->act[0], lm->m[0], lm->m[0], qkv_w / BN, T_cap, g, stream)) != DCUT_OK) return st;
+    if ((st = launch_gemm<kPlain>(ctx, lm->act[0], wm->m[0], wm->m[0], qkv_w / BN, T_cap, wmask[0], g, stream)) != DCUT_OK) return st;
     // 3. RoPE, append the new K/V to the paged cache
     RopeArgs r;
     r.qkv = ctx->ly_qkv; r.cu_q = cu_q; r.tok_req = tok_req; r.tok_pos = tok_pos; r.block_table = block_table;
@@ -882,15 +986,15 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     if (st != DCUT_OK) return st;
     // 5. h1 = x + attn . Wo^T
     g.N_out = H; g.K = q_w; g.out = ctx->ly_h1; g.residual = static_cast<const __nv_bfloat16*>(x);
-    if ((st = launch_gemm<kResidual>(ctx, lm->act[1], lm->m[1], lm->m[1], H / BN, T_cap, g, stream)) != DCUT_OK) return st;
+    if ((st = launch_gemm<kResidual>(ctx, lm->act[1], wm->m[1], wm->m[1], H / BN, T_cap, wmask[1], g, stream)) != DCUT_OK) return st;
     // 6. n2 = RMSNorm(h1)
     if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(ctx->ly_h1),
                                                    static_cast<const __nv_bfloat16*>(w->g_mlp), cu_q, B, H, w->rms_eps, ctx->ly_norm2),
                               "launch rmsnorm_kernel")) != DCUT_OK) return st;
     // 7. act = SiLU(n2 . Wg^T) * (n2 . Wu^T)
     g.N_out = I; g.K = H; g.out = ctx->ly_act; g.residual = nullptr;
-    if ((st = launch_gemm<kSwiGLU>(ctx, lm->act[2], lm->m[2], lm->m[3], I / (BN / 2), T_cap, g, stream)) != DCUT_OK) return st;
+    if ((st = launch_gemm<kSwiGLU>(ctx, lm->act[2], wm->m[2], wm->m[3], I / (BN / 2), T_cap, wmask[2], g, stream)) != DCUT_OK) return st;
     // 8. y = h1 + act . Wd^T
     g.N_out = H; g.K = I; g.out = static_cast<__nv_bfloat16*>(y); g.residual = ctx->ly_h1;
-    return launch_gemm<kResidual>(ctx, lm->act[3], lm->m[4], lm->m[4], H / BN, T_cap, g, stream);
+    return launch_gemm<kResidual>(ctx, lm->act[3], wm->m[4], wm->m[4], H / BN, T_cap, wmask[4], g, stream);
 }

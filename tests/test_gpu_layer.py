@@ -162,3 +162,62 @@ def test_pair_mode_matches_the_oracle(T, N, K, mode):
         want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
     _close(out[:T], want, f"pair mode, epilogue {mode}")
     assert (out[T:].float() == 7.0).all()       # rows past T are never written
+
+
+@pytest.mark.parametrize("width_bit", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_every_tile_width_matches_the_oracle(width_bit, mode, monkeypatch):
+    """The one-SM mode picks its tile width (256, 224, ..., 64 columns) per launch; with only one narrower width allowed
+    and less than a wave of tiles the narrower one is always the cheaper.  N = 768 is not a multiple of most widths
+    (ragged last tile: zero-filled weight rows, masked stores); T spans three row blocks with a ragged last one."""
+    if mode == 2 and width_bit % 2:
+        pytest.skip("the SwiGLU tile uses the widths whose halves are multiples of 32 columns")
+    monkeypatch.setenv("DCUT_GEMM_WIDTHS", str(1 | (1 << width_bit)))
+    T, N, K = 300, 768, 512
+    rng = np.random.default_rng(100 * width_bit + mode)
+    cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
+    ctx = make_ctx(cfg, max_pages=1, vocab=0)
+    T_cap = T + 3
+    a, w = _bf(rng, (T_cap, K)), _bf(rng, (N, K), 0.05)
+    w2 = _bf(rng, (N, K), 0.05) if mode == 2 else None
+    res = _bf(rng, (T_cap, N)) if mode == 1 else None
+    out = torch.full((T_cap, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(w), dev(np.array([0, T], np.int32)), T_cap, out, mode=mode, w2=None if w2 is None else dev(w2),
+                  residual=None if res is None else dev(res))
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    if mode == 2:
+        want = orc.swiglu_f64(orc.linear(a[:T], w), orc.linear(a[:T], w2))
+    else:
+        want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
+    _close(out[:T], want, f"width bit {width_bit}, epilogue {mode}")
+    assert (out[T:].float() == 7.0).all()
+    ctx.close()
+
+
+@pytest.mark.parametrize("width_bit", [1, 2, 4, 6])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_pair_mode_at_every_tile_width(width_bit, mode, monkeypatch):
+    """The pair mode (two SMs per 256-row tile) with a narrower tile, forced through the experiment knob; ragged last
+    column tile and ragged last row block as above."""
+    monkeypatch.setenv("DCUT_GEMM_FORCE", str(8 + width_bit))
+    T, N, K = 300, 768, 8192
+    rng = np.random.default_rng(1000 + 100 * width_bit + mode)
+    cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
+    ctx = make_ctx(cfg, max_pages=1, vocab=0)
+    T_cap = T + 3
+    a, w = _bf(rng, (T_cap, K), 0.5), _bf(rng, (N, K), 0.05)
+    w2 = _bf(rng, (N, K), 0.05) if mode == 2 else None
+    res = _bf(rng, (T_cap, N)) if mode == 1 else None
+    out = torch.full((T_cap, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(w), dev(np.array([0, T], np.int32)), T_cap, out, mode=mode, w2=None if w2 is None else dev(w2),
+                  residual=None if res is None else dev(res))
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    if mode == 2:
+        want = orc.swiglu_f64(orc.linear(a[:T], w), orc.linear(a[:T], w2))
+    else:
+        want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
+    _close(out[:T], want, f"pair mode, width bit {width_bit}, epilogue {mode}")
+    assert (out[T:].float() == 7.0).all()
+    ctx.close()
