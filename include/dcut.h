@@ -30,6 +30,8 @@
  *   DCUT_ATTN_TAIL_REQ_DIV    cut the shortest B / n requests finer (0 = off)
  *   DCUT_ATTN_TAIL_MIN_PAGES  smallest such piece, in pages (32)
  *   DCUT_GEMM_2CTA            0 = never run GEMM tiles on pairs of SMs (tcgen05 cta_group::2); default: where it pays
+ *   DCUT_GEMM_WIDTHS          bit mask of the GEMM tile widths that may be chosen (bit i: 256 - 32 i columns; default 0x7f)
+ *   DCUT_GEMM_FORCE           experiments: 0..6 = that width on one SM per tile, 8..14 = on a pair, whatever the packed length
  */
 #ifndef DCUT_H_
 #define DCUT_H_

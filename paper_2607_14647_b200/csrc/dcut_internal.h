@@ -77,6 +77,7 @@ struct dcut_ctx {
     __nv_bfloat16* ly_x[2];   // hidden states between the layers of dcut_model_verify (ping-pong)
     int ly_gemm_pairs;      // clusters of two CTAs the device runs at once
     int ly_gemm_pair_mode;  // 0: the GEMM never runs tiles on pairs of SMs
+    int ly_gemm_force;      // experiments: -1 = gemm_plan chooses; 0..6 a width on one SM; 8..14 on a pair
     unsigned ly_gemm_bn_mask;   // tile widths the one-SM mode may choose from (bit i: 256 - 32 i columns)
     float* ly_inv_freq;     // [head_dim / 2]
     float ly_theta;         // theta the table was built for (0 = none yet)

@@ -50,6 +50,7 @@ struct BMaps {
     CUtensorMap m[kNumBn];
 };
 constexpr unsigned kBnMaskAll = (1u << kNumBn) - 1;
+constexpr int kPlanRows = 72;
 constexpr unsigned kBnMaskSwiGLU = 0x55;   // widths whose halves are whole 32-column epilogue steps: 256, 192, 128, 64
 
 // ------------------------------------------------------------------------------------------------ PTX
@@ -151,6 +152,7 @@ struct GemmArgs {
     int pairs;                       // launched as clusters of two CTAs: the pair mode may be chosen
     unsigned bn_mask;                // tile widths whose tensor maps were supplied (bit i: bn_of(i)); bit 0 always
     int force;                       // experiments: -1 = let gemm_plan choose, 0..6 = that width on one SM, 8..14 = on a pair
+    unsigned char plan_by_m[kPlanRows];   // gemm_plan for 1, 2, ... row blocks of 128 (the last entry serves all larger counts)
     int* status;
 };
 
@@ -323,16 +325,17 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
 // issued at about 0.57 of the one-SM rate per column; the constants stand for what a tile costs whatever its width.)
 // Over those 68 cases the pick is within 0.3 % (geometric mean; worst case 7 %) of the best measured choice.  Returns
 // the width index, + kPlanPair for the pair mode; the wider tile wins ties.
+// The choice depends on T only through the number of 128-row blocks, so the host tabulates it per launch
+// (GemmArgs::plan_by_m) and the kernel looks it up after reading T.
 constexpr int kPlanPair = 8;
-__device__ __forceinline__ int gemm_plan(int T, const GemmArgs& g, bool swiglu, int grid) {
-    const int m1 = (T + BM - 1) / BM, m2 = (T + 2 * BM - 1) / (2 * BM);
-    if (m1 == 0) return 0;
-    if (g.force >= 0) return g.force;
-    const int n_pairs = g.pairs ? grid >> 1 : 0;
+inline int gemm_plan(int m1, int N_out, unsigned bn_mask, bool pairs, int force, bool swiglu, int grid) {
+    if (force >= 0) return force;
+    const int m2 = (m1 + 1) / 2;
+    const int n_pairs = pairs ? grid >> 1 : 0;
     int best = 0, best_cost = INT_MAX;
     for (int i = 0; i < kNumBn; ++i) {
-        if (!((g.bn_mask >> i) & 1)) continue;
-        const int bn = bn_of(i), per = swiglu ? bn >> 1 : bn, n_tiles = (g.N_out + per - 1) / per;
+        if (!((bn_mask >> i) & 1)) continue;
+        const int bn = bn_of(i), per = swiglu ? bn >> 1 : bn, n_tiles = (N_out + per - 1) / per;
         const int cost1 = ((m1 * n_tiles + grid - 1) / grid) * (4 * bn + 1664);
         if (cost1 < best_cost) {
             best_cost = cost1;
@@ -387,7 +390,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
     const int T = g.cu_q[g.B];
-    const int plan_all = gemm_plan(T, g, MODE == kSwiGLU, (int)gridDim.x);
+    const int m_blocks = (T + BM - 1) / BM;
+    const int plan_all = m_blocks > 0 ? g.plan_by_m[(m_blocks < kPlanRows ? m_blocks : kPlanRows) - 1] : 0;
     const bool pairs = plan_all >= kPlanPair;
     const int plan = plan_all & 7;                                  // width index
     const int bn = bn_of(plan), half_rows = bn >> 1;                // tile width; a B tile is loaded as two halves
@@ -741,11 +745,7 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
     GemmArgs ga = g;
     ga.n_tiles = n_tiles;
     ga.bn_mask = bn_mask | 1u;
-    {
-        const char* envf = getenv("DCUT_GEMM_FORCE");
-        ga.force = envf ? atoi(envf) : -1;
-        if (ga.force >= 0 && (!((ga.bn_mask >> (ga.force & 7)) & 1) || (ga.force >= 8 && !ga.pairs))) ga.force = -1;
-    }
+
     // work items at the narrowest width that may be chosen (the widest has n_tiles per row block)
     int narrow = 0;
     for (int i = 0; i < kNumBn; ++i)
@@ -753,11 +753,16 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
     const int n_work = ((T_cap + BM - 1) / BM) * ((n_tiles * BN + bn_of(narrow) - 1) / bn_of(narrow));
     int grid = n_work < ctx->sm_count ? n_work : ctx->sm_count;   // persistent: at most one CTA per SM
     ga.pairs = 0;
+    ga.force = ctx->ly_gemm_force >= 0 && ctx->ly_gemm_force < kNumBn && ((ga.bn_mask >> ctx->ly_gemm_force) & 1) ? ctx->ly_gemm_force : -1;
     if (ctx->ly_gemm_pairs > 0) {
         // always launched as clusters of two CTAs (the kernel holds cta_group::2 instructions); the pair mode itself
         // can be switched off
         grid = 2 * (n_work < ctx->ly_gemm_pairs ? n_work : ctx->ly_gemm_pairs);   // room for either mode
         ga.pairs = ctx->ly_gemm_pair_mode;
+        ga.force = ctx->ly_gemm_force;
+        if (ga.force >= 0 && (ga.force > 14 || !((ga.bn_mask >> (ga.force & 7)) & 1) || (ga.force >= 8 && !ga.pairs))) ga.force = -1;
+        for (int m = 1; m <= kPlanRows; ++m)
+            ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, ga.pairs != 0, ga.force, MODE == kSwiGLU, grid);
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
@@ -774,6 +779,8 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
         lc.numAttrs = 2;
         return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_tcgen05_kernel<MODE>, a, b, b2, ga), "launch gemm_tcgen05_kernel");
     }
+    for (int m = 1; m <= kPlanRows; ++m)
+        ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, false, ga.force, MODE == kSwiGLU, grid);
     return dcut_check_cuda(ctx, dcut_launch_pdl(gemm_tcgen05_kernel<MODE>, dim3(grid), dim3(kGemmThreads), kGemmSmem, stream, a, b, b2, ga),
                            "launch gemm_tcgen05_kernel");
 }
@@ -804,6 +811,8 @@ dcut_status dcut_init_layer(dcut_ctx* ctx) {
         // (DCUT_GEMM_2CTA=0: never).  ly_gemm_pairs = how many such clusters the device runs at once.
         const char* env = getenv("DCUT_GEMM_2CTA");
         ctx->ly_gemm_pair_mode = (!env || atoi(env) != 0) ? 1 : 0;
+        const char* envf = getenv("DCUT_GEMM_FORCE");
+        ctx->ly_gemm_force = envf ? atoi(envf) : -1;
         const char* envw = getenv("DCUT_GEMM_WIDTHS");   // bit i allows tile width 256 - 32 i in the one-SM mode
         ctx->ly_gemm_bn_mask = ((envw ? (unsigned)strtoul(envw, nullptr, 0) : kBnMaskAll) & kBnMaskAll) | 1u;
         ctx->ly_gemm_pairs = 0;
