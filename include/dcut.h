@@ -31,7 +31,8 @@
  *   DCUT_ATTN_TAIL_MIN_PAGES  smallest such piece, in pages (32)
  *   DCUT_GEMM_2CTA            0 = never run GEMM tiles on pairs of SMs (tcgen05 cta_group::2); default: where it pays
  *   DCUT_GEMM_WIDTHS          bit mask of the GEMM tile widths that may be chosen (bit i: 256 - 32 i columns; default 0x7f)
- *   DCUT_GEMM_FORCE           experiments: 0..6 = that width on one SM per tile, 8..14 = on a pair, whatever the packed length
+ *   DCUT_GEMM_FORCE           experiments: 0..6 = that width on one SM per tile, 8..14 = on a pair, 16..22 = a pair splitting K,
+ *                             whatever the packed length (a split needs every tile to fit one wave of pairs)
  */
 #ifndef DCUT_H_
 #define DCUT_H_

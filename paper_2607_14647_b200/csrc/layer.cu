@@ -51,6 +51,7 @@ struct BMaps {
 };
 constexpr unsigned kBnMaskAll = (1u << kNumBn) - 1;
 constexpr int kPlanRows = 72;
+constexpr int kSplitCost = 50;             // gemm_plan: what the exchange of partial sums between the two SMs costs
 constexpr unsigned kBnMaskSwiGLU = 0x55;   // widths whose halves are whole 32-column epilogue steps: 256, 192, 128, 64
 
 // ------------------------------------------------------------------------------------------------ PTX
@@ -327,8 +328,8 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
 // the width index, + kPlanPair for the pair mode; the wider tile wins ties.
 // The choice depends on T only through the number of 128-row blocks, so the host tabulates it per launch
 // (GemmArgs::plan_by_m) and the kernel looks it up after reading T.
-constexpr int kPlanPair = 8;
-inline int gemm_plan(int m1, int N_out, unsigned bn_mask, bool pairs, int force, bool swiglu, int grid) {
+constexpr int kPlanPair = 8, kPlanSplit = 16;
+inline int gemm_plan(int m1, int N_out, unsigned bn_mask, bool pairs, bool may_split, int force, bool swiglu, int grid) {
     if (force >= 0) return force;
     const int m2 = (m1 + 1) / 2;
     const int n_pairs = pairs ? grid >> 1 : 0;
@@ -346,6 +347,14 @@ inline int gemm_plan(int m1, int N_out, unsigned bn_mask, bool pairs, int force,
             if (cost2 < best_cost) {
                 best_cost = cost2;
                 best = kPlanPair + i;
+            }
+            // both SMs of a pair on one 128-row tile, half of K each (only as a single wave: a tile per pair)
+            if (may_split && m1 * n_tiles <= n_pairs) {
+                const int cost3 = (4 * bn + 1664) / 2 + kSplitCost;
+                if (cost3 < best_cost) {
+                    best_cost = cost3;
+                    best = kPlanSplit + i;
+                }
             }
         }
     }
@@ -392,7 +401,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     const int T = g.cu_q[g.B];
     const int m_blocks = (T + BM - 1) / BM;
     const int plan_all = m_blocks > 0 ? g.plan_by_m[(m_blocks < kPlanRows ? m_blocks : kPlanRows) - 1] : 0;
-    const bool pairs = plan_all >= kPlanPair;
+    const bool split = plan_all >= kPlanSplit;                      // the pair shares one 128-row tile, half of K each
+    const bool pairs = plan_all >= kPlanPair && !split;
     const int plan = plan_all & 7;                                  // width index
     const int bn = bn_of(plan), half_rows = bn >> 1;                // tile width; a B tile is loaded as two halves
     const int per = MODE == kSwiGLU ? half_rows : bn;               // output columns per tile
@@ -413,7 +423,126 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
 
-    if (!pairs) {
+    if (split) {
+        // ------------------------------------------------------------------ one tile per pair of SMs, K cut in two
+        // Each CTA runs the one-SM main loop over its half of the k-blocks into its own accumulator.  Then the two
+        // exchange: a CTA sends the columns the other one will finish (fp32, through distributed shared memory into
+        // the other's idle operand ring) and finishes its own columns with what it received.  Every thread of both
+        // CTAs passes the same two cluster barriers whatever happened before, so a wait that gave up cannot strand
+        // the peer.
+        const int m_tiles = (T + BM - 1) / BM;
+        const int w = blockIdx.x >> 1;                              // the pair's tile
+        const bool has_tile = w < m_tiles * n_tiles;
+        const uint32_t rank = cluster_ctarank();
+        const int n_tile = has_tile ? w / m_tiles : 0, m0 = has_tile ? (w - n_tile * m_tiles) * BM : 0;
+        const int kb_mid = (n_kb + 1) >> 1, kb0 = rank ? kb_mid : 0, kb1 = rank ? n_kb : kb_mid;
+        const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
+        const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages);
+        if (has_tile && warp == 0) {
+            const CUtensorMap* b_map = pick_map(b_maps, plan);
+            const uint32_t stage_tx = kATile + bn * BK * 2;
+            for (int kb = kb0, kc = 0; kb < kb1; ++kb, ++kc) {
+                const int s = kc % kGemmStages;
+                if (kc >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kGemmStages) - 1) & 1))) {
+                    failed = true;
+                    break;
+                }
+                if (elect_one()) {
+                    const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
+                    const uint32_t bar = full_bar + 8 * s;
+                    mbar_arrive_expect_tx(bar, stage_tx);
+                    tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
+                    tma_load_2d(b_dst, b_map, kb * BK, n_tile * bn, bar);
+                    tma_load_2d(b_dst + half_rows * BK * 2, b_map, kb * BK, n_tile * bn + half_rows, bar);
+                }
+                __syncwarp();
+            }
+        } else if (has_tile && warp == 1) {
+            const uint32_t idesc = kIdescNoN | ((uint32_t)(bn >> 3) << 17);
+            for (int kb = kb0, kc = 0; kb < kb1; ++kb, ++kc) {
+                const int s = kc % kGemmStages;
+                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kGemmStages) & 1))) {
+                    failed = true;
+                    break;
+                }
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
+                    const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) tc_mma(tmem_base, da + 2 * k, db + 2 * k, idesc, (kc | k) ? 1u : 0u);
+                    tc_commit(empty_bar + 8 * s);
+                }
+                __syncwarp();
+            }
+            if (!failed && elect_one()) tc_commit(acc_full);    // this CTA's partial sums are complete
+            __syncwarp();
+        } else if (has_tile) {
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_full, 0))) failed = true;   // ... and its operand ring is idle
+            tc_fence_after();
+        }
+        // columns [0, cut) are finished by rank 0, [cut, bn) by rank 1
+        const int cut = (bn >> 6) << 5;
+        const int own0 = rank ? cut : 0, own1 = rank ? bn : cut, send0 = rank ? 0 : cut, send1 = rank ? cut : bn;
+        const int quarter = warp & 3, row_in_tile = quarter * 32 + lane;
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t stage_local = smem_u32(smem);              // [column / 4][row] vectors of four fp32: 64 KB at most
+        tc_fence_before();
+        cluster_sync_all();                                       // both accumulators complete, both rings idle
+        tc_fence_after();
+        if (has_tile && warp >= 2 && !failed) {
+            asm volatile("fence.proxy.async;" ::: "memory");      // the ring was last written and read through the async proxy
+            const uint32_t stage_peer = mapa_rank(stage_local, rank ^ 1);
+#pragma unroll 1
+            for (int c = send0; c < send1; c += 32) {
+                uint32_t av[32];
+                tc_ld32(t_row + c, av);
+                tc_wait_ld();
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const uint32_t dst = stage_peer + (uint32_t)((((c - send0) >> 2) + v) * BM + row_in_tile) * 16;
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(av[4 * v]), "r"(av[4 * v + 1]),
+                                 "r"(av[4 * v + 2]), "r"(av[4 * v + 3]) : "memory");
+                }
+            }
+        }
+        tc_fence_before();
+        cluster_sync_all();                                       // the peer's partial sums have arrived
+        tc_fence_after();
+        if (has_tile && warp >= 2 && !failed) {
+            const int row = m0 + row_in_tile, col0 = n_tile * bn;
+            __nv_bfloat16* orow = g.out + (size_t)row * g.N_out + col0;
+            const __nv_bfloat16* rrow = MODE == kResidual ? g.residual + (size_t)row * g.N_out + col0 : nullptr;
+#pragma unroll 1
+            for (int c = own0; c < own1; c += 32) {
+                uint32_t av[32];
+                tc_ld32(t_row + c, av);
+                tc_wait_ld();
+                if (row < T) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        if (col0 + c + e >= g.N_out) break;
+                        float add[8];
+#pragma unroll
+                        for (int v = 0; v < 2; ++v) {
+                            const uint32_t src = stage_local + (uint32_t)((((c - own0 + e) >> 2) + v) * BM + row_in_tile) * 16;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                         : "=f"(add[4 * v]), "=f"(add[4 * v + 1]), "=f"(add[4 * v + 2]), "=f"(add[4 * v + 3]) : "r"(src));
+                        }
+                        uint4 res = make_uint4(0, 0, 0, 0);
+                        if (MODE == kResidual) res = *reinterpret_cast<const uint4*>(rrow + c + e);
+                        const uint32_t rw[4] = {res.x, res.y, res.z, res.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)   // (rank 0's half of K) + (rank 1's), then the residual
+                            o[j] = pack_bf16((rank ? add[2 * j] + __uint_as_float(av[e + 2 * j]) : __uint_as_float(av[e + 2 * j]) + add[2 * j]) + bf_lo(rw[j]),
+                                             (rank ? add[2 * j + 1] + __uint_as_float(av[e + 2 * j + 1]) : __uint_as_float(av[e + 2 * j + 1]) + add[2 * j + 1]) + bf_hi(rw[j]));
+                        *reinterpret_cast<uint4*>(orow + c + e) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+            }
+        }
+    } else if (!pairs) {
         const int m_tiles = (T + BM - 1) / BM;
         const int n_work = m_tiles * n_tiles;                      // (a CTA without work falls through the loops below)
         const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
@@ -760,9 +889,13 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
         grid = 2 * (n_work < ctx->ly_gemm_pairs ? n_work : ctx->ly_gemm_pairs);   // room for either mode
         ga.pairs = ctx->ly_gemm_pair_mode;
         ga.force = ctx->ly_gemm_force;
-        if (ga.force >= 0 && (ga.force > 14 || !((ga.bn_mask >> (ga.force & 7)) & 1) || (ga.force >= 8 && !ga.pairs))) ga.force = -1;
+        if (ga.force >= 0 && (ga.force > 22 || (ga.force & 7) == 7 || !((ga.bn_mask >> (ga.force & 7)) & 1) || (ga.force >= 8 && !ga.pairs) ||
+                              (ga.force >= 16 && !((MODE == kPlain || MODE == kResidual) && ga.K >= 2 * BK))))
+            ga.force = -1;
         for (int m = 1; m <= kPlanRows; ++m)
-            ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, ga.pairs != 0, ga.force, MODE == kSwiGLU, grid);
+            ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, ga.pairs != 0,
+                                                           ga.pairs != 0 && (MODE == kPlain || MODE == kResidual) && ga.K >= 2 * BK,
+                                                           ga.force, MODE == kSwiGLU, grid);
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
@@ -780,7 +913,7 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
         return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_tcgen05_kernel<MODE>, a, b, b2, ga), "launch gemm_tcgen05_kernel");
     }
     for (int m = 1; m <= kPlanRows; ++m)
-        ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, false, ga.force, MODE == kSwiGLU, grid);
+        ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, false, false, ga.force, MODE == kSwiGLU, grid);
     return dcut_check_cuda(ctx, dcut_launch_pdl(gemm_tcgen05_kernel<MODE>, dim3(grid), dim3(kGemmThreads), kGemmSmem, stream, a, b, b2, ga),
                            "launch gemm_tcgen05_kernel");
 }

@@ -221,3 +221,29 @@ def test_pair_mode_at_every_tile_width(width_bit, mode, monkeypatch):
     _close(out[:T], want, f"pair mode, width bit {width_bit}, epilogue {mode}")
     assert (out[T:].float() == 7.0).all()
     ctx.close()
+
+
+@pytest.mark.parametrize("width_bit", [0, 1, 3, 4, 6])
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("T,K", [(300, 1024), (120, 192), (257, 12288)])
+def test_split_k_mode_at_every_tile_width(width_bit, mode, T, K, monkeypatch):
+    """Both SMs of a pair on one 128-row tile, half of the k-blocks each (an odd count too: K = 192 is three), partial
+    sums exchanged through distributed shared memory; forced through the experiment knob.  N = 768 keeps the tiles
+    within one wave of pairs and leaves a ragged last column tile for most widths."""
+    monkeypatch.setenv("DCUT_GEMM_FORCE", str(16 + width_bit))
+    N = 768
+    rng = np.random.default_rng(2000 + 100 * width_bit + mode + T)
+    cfg = wl.custom_config(B=1, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128)
+    ctx = make_ctx(cfg, max_pages=1, vocab=0)
+    T_cap = T + 3
+    a, w = _bf(rng, (T_cap, K), 0.5), _bf(rng, (N, K), 0.05)
+    res = _bf(rng, (T_cap, N)) if mode == 1 else None
+    out = torch.full((T_cap, N), 7.0, dtype=torch.bfloat16, device="cuda")
+    ctx.gemm_bf16(dev(a), dev(w), dev(np.array([0, T], np.int32)), T_cap, out, mode=mode,
+                  residual=None if res is None else dev(res))
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
+    _close(out[:T], want, f"split-K, width bit {width_bit}, epilogue {mode}")
+    assert (out[T:].float() == 7.0).all()
+    ctx.close()
