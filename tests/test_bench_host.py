@@ -74,3 +74,23 @@ def test_reference_arm_runs_without_gpu():
     line = json.loads(out.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_cost_grid_marks_the_row_block_steps():
+    """Cost-table sample points: evenly spaced for the attention workloads; for the layer workloads the last length
+    of a 128-row block and the first of the next, always with both ends."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2607_14647_b200 import workloads as wl
+    cfg2, cfg4 = wl.config(2), wl.config(4)
+    even = bench.cost_grid(cfg2, 18, False)
+    assert even[0] == cfg2.B and even[-1] == cfg2.t_cap and len(even) == 18 and even == sorted(even)
+    steps = np.diff(even)
+    assert steps.max() - steps.min() <= 1
+    tiled = bench.cost_grid(cfg4, 18, True)
+    assert tiled[0] == cfg4.B and tiled[-1] == cfg4.t_cap and tiled == sorted(set(tiled))
+    inner = tiled[1:-1]
+    assert len(inner) % 2 == 0 and all(a % 128 == 0 and b == a + 1 for a, b in zip(inner[::2], inner[1::2]))
+    assert [a for a in inner[::2]] == list(range(128, cfg4.t_cap, 128))          # every block edge at 18 points
+    few = bench.cost_grid(cfg4, 6, True)
+    assert few[0] == cfg4.B and few[-1] == cfg4.t_cap and 4 <= len(few) <= 8
