@@ -399,16 +399,17 @@ def layer_forward(x, w, k_cache, v_cache, block_table, ctx_lens, depths, n_q_hea
 
 
 def model_verify(tok_id, embed, layers, g_final, w_lm, k_caches, v_caches, block_table, ctx_lens, depths, draft_ids,
-                 n_q_heads, n_kv_heads, head_dim, page_size, rms_eps, rope_theta):
+                 n_q_heads, n_kv_heads, head_dim, page_size, rms_eps, rope_theta, return_stages=False):
     """The verification forward of a whole model on the retained tokens (Section 3.1: one packed target forward
     over each request's first d_i draft tokens, then acceptance): embedding lookup, `layer_forward` for every
     layer in turn (layer l with its own cache pair), final RMSNorm rounded to bf16, `lm_head_accept`.
     Returns (AcceptResult, logits fp64 [T, V], hidden: list of the bf16 hidden states after each layer, final
-    normed states last, updated cache copies per layer)."""
+    normed states last, updated cache copies per layer); with `return_stages` also the list of `layer_forward`'s stage
+    dicts, one per layer."""
     import torch
     tok_id = np.asarray(tok_id, np.int64)
     x = embed[torch.from_numpy(tok_id)]
-    hidden, caches = [], []
+    hidden, caches, stages = [], [], []
     cu = None
     for l, w in enumerate(layers):
         st = layer_forward(x, w, k_caches[l], v_caches[l], block_table, ctx_lens, depths, n_q_heads, n_kv_heads,
@@ -416,6 +417,7 @@ def model_verify(tok_id, embed, layers, g_final, w_lm, k_caches, v_caches, block
         x, cu = st["y"], st["cu_q"]
         hidden.append(x)
         caches.append((st["k_cache"], st["v_cache"]))
+        stages.append(st)
     if cu is None:
         d = np.asarray(depths, np.int32)
         cu = np.zeros(len(d) + 1, np.int32)
@@ -424,4 +426,6 @@ def model_verify(tok_id, embed, layers, g_final, w_lm, k_caches, v_caches, block
     hidden.append(n)
     gamma = np.asarray(draft_ids).shape[1]
     res, logits64 = lm_head_accept(n, w_lm, draft_ids, cu, gamma)
+    if return_stages:
+        return res, logits64, hidden, caches, stages
     return res, logits64, hidden, caches
