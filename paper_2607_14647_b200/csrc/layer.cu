@@ -892,10 +892,12 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
         if (ga.force >= 0 && (ga.force > 22 || (ga.force & 7) == 7 || !((ga.bn_mask >> (ga.force & 7)) & 1) || (ga.force >= 8 && !ga.pairs) ||
                               (ga.force >= 16 && !((MODE == kPlain || MODE == kResidual) && ga.K >= 2 * BK))))
             ga.force = -1;
+        const int m_cap = (T_cap + BM - 1) / BM;   // no launch has more row blocks than that: the rest of the table repeats
         for (int m = 1; m <= kPlanRows; ++m)
-            ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, ga.pairs != 0,
-                                                           ga.pairs != 0 && (MODE == kPlain || MODE == kResidual) && ga.K >= 2 * BK,
-                                                           ga.force, MODE == kSwiGLU, grid);
+            ga.plan_by_m[m - 1] = m > m_cap && m > 1 ? ga.plan_by_m[m - 2]
+                                                    : (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, ga.pairs != 0,
+                                                                               ga.pairs != 0 && (MODE == kPlain || MODE == kResidual) && ga.K >= 2 * BK,
+                                                                               ga.force, MODE == kSwiGLU, grid);
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
@@ -913,7 +915,9 @@ dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, con
         return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, gemm_tcgen05_kernel<MODE>, a, b, b2, ga), "launch gemm_tcgen05_kernel");
     }
     for (int m = 1; m <= kPlanRows; ++m)
-        ga.plan_by_m[m - 1] = (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, false, false, ga.force, MODE == kSwiGLU, grid);
+        ga.plan_by_m[m - 1] = m > (T_cap + BM - 1) / BM && m > 1
+                                  ? ga.plan_by_m[m - 2]
+                                  : (unsigned char)gemm_plan(m, ga.N_out, ga.bn_mask, false, false, ga.force, MODE == kSwiGLU, grid);
     return dcut_check_cuda(ctx, dcut_launch_pdl(gemm_tcgen05_kernel<MODE>, dim3(grid), dim3(kGemmThreads), kGemmSmem, stream, a, b, b2, ga),
                            "launch gemm_tcgen05_kernel");
 }
