@@ -141,3 +141,32 @@ def test_argument_errors():
                         dev(sel.ctx_lens), dev(wl.cu_q_from_depths(depths)), cfg.t_cap)
     assert e.value.status == binding.ECAPACITY
     ctx.close()
+
+
+@pytest.mark.parametrize("tp", [2, 4])
+def test_kv_head_sharding_reproduces_the_unsharded_result(tp):
+    """Tensor-parallel sharding of the attention step as the paper's TP deployments would do it: rank r owns kv heads
+    r * Hkv/tp .. and their query heads, holds its own slice of the paged cache, and runs the same call on a context
+    created for its share of the heads; no exchange inside the step.  Heads are independent, so the concatenated
+    shards equal the unsharded output bit for bit (the ranks run one after the other here, on one GPU)."""
+    cfg = wl.custom_config(B=9, gamma=16, n_q_heads=16, n_kv_heads=4, head_dim=128, ctx_lo=3, ctx_hi=900)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    depths = np.array([16, 0, 5, 16, 1, 9, 16, 2, 7], np.int32)
+    q, cu, full, full_lse = _run(cfg, sel, kv, depths)
+    group = cfg.n_q_heads // cfg.n_kv_heads
+    hk = cfg.n_kv_heads // tp
+    shard_cfg = wl.custom_config(B=cfg.B, gamma=cfg.gamma, n_q_heads=hk * group, n_kv_heads=hk, head_dim=cfg.head_dim,
+                                 ctx_lo=cfg.ctx_lo, ctx_hi=cfg.ctx_hi)
+    outs = []
+    for r in range(tp):
+        ctx = make_ctx(shard_cfg, max_pages=kv.max_pages_per_req)
+        q_r = q[:, r * hk * group:(r + 1) * hk * group].contiguous()
+        k_r = kv.k_cache[:, r * hk:(r + 1) * hk].contiguous()
+        v_r = kv.v_cache[:, r * hk:(r + 1) * hk].contiguous()
+        out = ctx.verify_attn(dev(q_r), dev(k_r), dev(v_r), dev(kv.block_table), dev(sel.ctx_lens), dev(cu), cfg.t_cap)
+        torch.cuda.synchronize()
+        assert ctx.poll_device_status() == 0
+        ctx.close()
+        outs.append(out.float().cpu().numpy())
+    assert np.array_equal(np.concatenate(outs, axis=1), full)
