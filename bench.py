@@ -174,6 +174,14 @@ def cost_grid(cfg, points: int, tiled: bool) -> list:
     return sorted(pts)
 
 
+def monotone_cost(cost: np.ndarray) -> np.ndarray:
+    """Non-decreasing cost table from profiled points.  A longer batch never costs less, so the cost at T is at most
+    every measurement at T' >= T: the table is the running minimum taken from the long end.  (A running maximum from
+    the short end is monotone too, but one disturbed measurement then lifts every longer entry to its level, and the
+    selector, seeing a plateau, runs to the plateau's end.)"""
+    return np.minimum.accumulate(np.asarray(cost, np.float64)[::-1])[::-1].astype(np.float32)
+
+
 def peaks() -> dict:
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -334,17 +342,17 @@ def run_dcut(args):
         for _ in range(3):
             step(qp, lp, bufs)
         ts = []
-        for _ in range(7):
+        for _ in range(11):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             step(qp, lp, bufs)
             e1.record()
             e1.synchronize()
             ts.append(e0.elapsed_time(e1))
-        prof.append(statistics.median(ts))
+        prof.append(float(np.percentile(ts, 25)))   # interference only ever adds time: lean on the fast side of the sample
         del qp, lp, bufs
     cost = np.interp(np.arange(cap + 1), grid, prof)
-    cost = np.maximum.accumulate(cost).astype(np.float32)          # non-decreasing in T
+    cost = monotone_cost(cost)
 
     arms = {"pruned": cost, "full_gamma": np.ones(cap + 1, np.float32),
             "gamma0": (1.0 + 10.0 * np.maximum(0, np.arange(cap + 1) - cfg.B)).astype(np.float32)}
@@ -650,7 +658,7 @@ def run_model(args):
         ctx.set_cost_buckets(cfg.B, cfg.gamma, [T], [1.0])
         step()
         prof.append(timed(3)[0])
-    cost = np.maximum.accumulate(np.interp(np.arange(cap + 1), grid, prof)).astype(np.float32)
+    cost = monotone_cost(np.interp(np.arange(cap + 1), grid, prof))
     arms = {"pruned": cost, "full_gamma": np.ones(cap + 1, np.float32),
             "gamma0": (1.0 + 10.0 * np.maximum(0, np.arange(cap + 1) - cfg.B)).astype(np.float32)}
     flops_tok = L * layer_flops(cfg, 1) + 2.0 * H * V

@@ -26,7 +26,7 @@
  *
  * Environment variables read once, in dcut_create (measurement knobs; the defaults are the measured best):
  *   DCUT_ATTN_TC_MIN_ROWS     query rows from which a work item goes to the tcgen05 phase (17; above 128: never)
- *   DCUT_ATTN_TARGET_ITEMS    requests are cut along the context only below this many (request, kv head) pairs (2 x SMs)
+ *   DCUT_ATTN_TARGET_ITEMS    requests are cut along the context only below this many (request, kv head) pairs (13/8 x SMs)
  *   DCUT_ATTN_TAIL_REQ_DIV    cut the shortest B / n requests finer (0 = off)
  *   DCUT_ATTN_TAIL_MIN_PAGES  smallest such piece, in pages (32)
  *   DCUT_GEMM_2CTA            0 = never run GEMM tiles on pairs of SMs (tcgen05 cta_group::2); default: where it pays

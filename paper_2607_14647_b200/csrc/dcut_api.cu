@@ -133,7 +133,11 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
     if ((st = dcut_init_accept(c)) != DCUT_OK) return st;
     if (has_attn) {
         const char* env = getenv("DCUT_ATTN_TARGET_ITEMS");
-        c->target_items = env ? atoi(env) : c->sm_count * 2;   // requests are only cut when the batch has fewer (request, head) pairs than that
+        // Requests are cut along the context so that there are about this many work items when the batch has fewer
+        // (request, kv head) pairs.  13/8 of the SM count (240 on 148 SMs): the rounding of every request's cut adds a
+        // few items, and with 2 per SM as the aim those few made a third round on some SMs (B = 16: 2.7 TB/s with 296,
+        // 3.0 with 200-240, 2.9 with 148; no difference at B = 64, +1 % at B = 256).
+        c->target_items = env ? atoi(env) : c->sm_count * 13 / 8;
         if (c->target_items < 1) c->target_items = 1;
         env = getenv("DCUT_ATTN_TAIL_REQ_DIV");
         c->attn_tail_req_div = env ? atoi(env) : 0;

@@ -94,3 +94,15 @@ def test_cost_grid_marks_the_row_block_steps():
     assert [a for a in inner[::2]] == list(range(128, cfg4.t_cap, 128))          # every block edge at 18 points
     few = bench.cost_grid(cfg4, 6, True)
     assert few[0] == cfg4.B and few[-1] == cfg4.t_cap and 4 <= len(few) <= 8
+
+
+def test_monotone_cost_ignores_a_disturbed_point():
+    sys.path.insert(0, ROOT)
+    import bench
+    clean = np.array([1.0, 1.1, 1.2, 1.3, 1.4, 1.5], np.float32)
+    noisy = clean.copy()
+    noisy[2] = 1.9                                   # one measurement hit by interference
+    out = bench.monotone_cost(noisy)
+    assert (np.diff(out) >= 0).all()
+    assert np.allclose(out, [1.0, 1.1, 1.3, 1.3, 1.4, 1.5])       # the spike is capped by the next clean point
+    assert np.allclose(bench.monotone_cost(clean), clean)
