@@ -262,6 +262,34 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     if (tail_chunk < a.tail_min_pages) tail_chunk = a.tail_min_pages;
     if (tail_chunk > chunk_pages) tail_chunk = chunk_pages;
 
+    // The item kernel works through the tcgen05 queue first and the warp-level queue after it.  When the second
+    // holds only a small part of the pages (a few shallow requests among deep ones), its few long items would start
+    // late on a few SMs with the rest idle (measured at B = 64: +15 us per call while 3-8 % of the pages were in
+    // it): below one eighth of the pages everything goes to the tcgen05 queue.
+    __shared__ int w_tc_s, w_mma_s;
+    if (tid == 0) {
+        w_tc_s = 0;
+        w_mma_s = 0;
+    }
+    __syncthreads();
+    {
+        int w_tc = 0, w_mma = 0;
+        for (int i = tid; i < a.B; i += nthr) {
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+            const int M = (d + 1) * group;
+            const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
+            const int tc_rb = (a.max_item_rows >= a.tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= a.tc_min_rows) ? 1 : 0);
+            const int n_rb = n_full + (rem > 0 ? 1 : 0);
+            w_tc += pages * tc_rb;
+            w_mma += pages * (n_rb - tc_rb);
+        }
+        if (w_tc) atomicAdd(&w_tc_s, w_tc);
+        if (w_mma) atomicAdd(&w_mma_s, w_mma);
+    }
+    __syncthreads();
+    const int tc_min_rows = (a.tc_min_rows <= a.max_item_rows && w_tc_s > 0 && 8LL * w_mma_s < (long long)w_tc_s + w_mma_s) ? 1 : a.tc_min_rows;
+
     const int per = (a.B + nthr - 1) / nthr;
     const int j0 = tid * per;
     int my_tc = 0, my_mma = 0, my_rows = 0;
@@ -277,7 +305,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             // tcgen05 queue or to the warp-level queue by its number of rows
             const int M = (d + 1) * group;
             const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
-            const int tc_rb = (a.max_item_rows >= a.tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= a.tc_min_rows) ? 1 : 0);
+            const int tc_rb = (a.max_item_rows >= tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= tc_min_rows) ? 1 : 0);
             const int n_rb = n_full + (rem > 0 ? 1 : 0);
             my_tc += nc * a.n_kv_heads * tc_rb;
             my_mma += nc * a.n_kv_heads * (n_rb - tc_rb);
@@ -337,7 +365,7 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
                         it.q0 = q0;
                         it.depth = d;
                         it.ctx_len = ctx_len;
-                        const bool tc = rows >= a.tc_min_rows;
+                        const bool tc = rows >= tc_min_rows;
                         it.pad[0] = tc ? 1 : 0;   // which queue the item is in
                         it.pad[1] = row0;         // first query row of the item within the request's tile
                         it.pad[2] = rows;         // query rows of the item
