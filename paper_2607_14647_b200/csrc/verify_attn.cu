@@ -196,7 +196,7 @@ __device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* to
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     extern __shared__ unsigned long long order[];   // [npad] (inverted cost << 32 | request), sorted ascending
     __shared__ int ws[33];
-    __shared__ int total_s, tail_s;
+    __shared__ int total_s, tail_s, w_tc_s, w_mma_s;
     const int tid = threadIdx.x, nthr = blockDim.x;   // 256 threads for small batches: cheaper barriers
     dcut_pdl_wait();
     STAMP_MIN(0);
@@ -205,14 +205,24 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     if (tid == 0) {
         total_s = 0;
         tail_s = 0;
+        w_tc_s = 0;
+        w_mma_s = 0;
     }
     __syncthreads();
-    int local = 0;
+    int local = 0, w_tc = 0, w_mma = 0;   // pages in all; pages whose items would go to the tcgen05 / warp-level queue
     for (int i = tid; i < a.B; i += nthr) {
         const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-        local += (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+        const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+        local += pages;
+        const int M = (d + 1) * group;
+        const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
+        const int tc_rb = (a.max_item_rows >= a.tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= a.tc_min_rows) ? 1 : 0);
+        w_tc += pages * tc_rb;
+        w_mma += pages * (n_full + (rem > 0 ? 1 : 0) - tc_rb);
     }
     if (local) atomicAdd(&total_s, local);
+    if (w_tc) atomicAdd(&w_tc_s, w_tc);
+    if (w_mma) atomicAdd(&w_mma_s, w_mma);
     __syncthreads();
     const int total_pages = total_s;
     const long long units = (long long)total_pages * a.n_kv_heads;
@@ -266,28 +276,6 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     // holds only a small part of the pages (a few shallow requests among deep ones), its few long items would start
     // late on a few SMs with the rest idle (measured at B = 64: +15 us per call while 3-8 % of the pages were in
     // it): below one eighth of the pages everything goes to the tcgen05 queue.
-    __shared__ int w_tc_s, w_mma_s;
-    if (tid == 0) {
-        w_tc_s = 0;
-        w_mma_s = 0;
-    }
-    __syncthreads();
-    {
-        int w_tc = 0, w_mma = 0;
-        for (int i = tid; i < a.B; i += nthr) {
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-            const int M = (d + 1) * group;
-            const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
-            const int tc_rb = (a.max_item_rows >= a.tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= a.tc_min_rows) ? 1 : 0);
-            const int n_rb = n_full + (rem > 0 ? 1 : 0);
-            w_tc += pages * tc_rb;
-            w_mma += pages * (n_rb - tc_rb);
-        }
-        if (w_tc) atomicAdd(&w_tc_s, w_tc);
-        if (w_mma) atomicAdd(&w_mma_s, w_mma);
-    }
-    __syncthreads();
     const int tc_min_rows = (a.tc_min_rows <= a.max_item_rows && w_tc_s > 0 && 8LL * w_mma_s < (long long)w_tc_s + w_mma_s) ? 1 : a.tc_min_rows;
 
     const int per = (a.B + nthr - 1) / nthr;
