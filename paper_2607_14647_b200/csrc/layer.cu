@@ -35,7 +35,8 @@ constexpr int kBTile = BN * BK * 2;            // 32 KB
 constexpr int kGemmStageBytes = kATile + kBTile;
 constexpr int kGemmThreads = 192;              // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int kTmemCols = 512;              // two 128 x 256 fp32 accumulators
-constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 256 /* two sets of barriers, tmem ptr */;
+constexpr int kMaxStages = 12;                 // a narrow tile's stage is smaller: more of them fit the same operand area
+constexpr int kGemmSmem = kGemmStages * kGemmStageBytes + 1024 /* align */ + 512 /* two sets of barriers, tmem ptr */;
 constexpr int kWaitLimit = 1 << 22;
 
 enum GemmMode { kPlain = 0, kResidual = 1, kSwiGLU = 2, kArgmax = 3 };
@@ -48,6 +49,11 @@ constexpr int kNumBn = 7;
 __host__ __device__ constexpr int bn_of(int i) { return BN - 32 * i; }
 struct BMaps {
     CUtensorMap m[kNumBn];
+};
+// The activations' tensor map with the full 128-row box and with a 64-row box: with at most 64 packed rows a tile's
+// lower half would only be fetched to be ignored (at T = 64 the A tiles were more than half of what the SMs took in).
+struct AMaps {
+    CUtensorMap full, half;
 };
 constexpr unsigned kBnMaskAll = (1u << kNumBn) - 1;
 constexpr int kPlanRows = 72;
@@ -365,28 +371,28 @@ static_assert(kGemmStages * kGemmStageBytes == kG2Stages * kG2StageBytes, "both 
 
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ BMaps b_maps,
+gemm_tcgen05_kernel(const __grid_constant__ AMaps a_maps, const __grid_constant__ BMaps b_maps,
                     const __grid_constant__ BMaps b2_maps, GemmArgs g) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + kGemmStages * kGemmStageBytes);
-    unsigned long long* bars2 = bars + 2 * kGemmStages + 4;                 // the pair mode's set
+    unsigned long long* bars2 = bars + 2 * kMaxStages + 4;                  // the pair mode's set
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars2 + 2 * kG2Stages + 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_kb = g.K / BK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kGemmStages; ++s) {
+        for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(smem_u32(bars + s), 1);
-            mbar_init(smem_u32(bars + kGemmStages + s), 1);
+            mbar_init(smem_u32(bars + kMaxStages + s), 1);
         }
         for (int s = 0; s < kG2Stages; ++s) {
             mbar_init(smem_u32(bars2 + s), 1);                 // the leader's expect_tx arrival (bytes of both CTAs)
             mbar_init(smem_u32(bars2 + kG2Stages + s), 1);     // the leader's multicast commit
         }
         for (int k = 0; k < 2; ++k) {
-            mbar_init(smem_u32(bars + 2 * kGemmStages + k), 1);
-            mbar_init(smem_u32(bars + 2 * kGemmStages + 2 + k), 128);   // the four epilogue warps
+            mbar_init(smem_u32(bars + 2 * kMaxStages + k), 1);
+            mbar_init(smem_u32(bars + 2 * kMaxStages + 2 + k), 128);   // the four epilogue warps
             mbar_init(smem_u32(bars2 + 2 * kG2Stages + k), 1);          // the leader's multicast commit
             mbar_init(smem_u32(bars2 + 2 * kG2Stages + 2 + k), 256);    // (leader's copy) the epilogue threads of both CTAs
         }
@@ -399,6 +405,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
     const int T = g.cu_q[g.B];
+    // rows 64..127 of the A tile are not loaded when no row of them exists: they hold whatever shared memory held, and
+    // the accumulator rows computed from them are never stored (one-SM and split modes; a pair always loads full boxes)
+    const bool a_half = T <= BM / 2;
+    const CUtensorMap* a_map1 = a_half ? &a_maps.half : &a_maps.full;
+    const uint32_t a_bytes = a_half ? kATile / 2 : kATile;
     const int m_blocks = (T + BM - 1) / BM;
     const int plan_all = m_blocks > 0 ? g.plan_by_m[(m_blocks < kPlanRows ? m_blocks : kPlanRows) - 1] : 0;
     const bool split = plan_all >= kPlanSplit;                      // the pair shares one 128-row tile, half of K each
@@ -407,6 +418,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     const int bn = bn_of(plan), half_rows = bn >> 1;                // tile width; a B tile is loaded as two halves
     const int per = MODE == kSwiGLU ? half_rows : bn;               // output columns per tile
     const int n_tiles = (g.N_out + per - 1) / per;
+    // one-SM and split modes: a stage is this tile's A and B bytes, and as many stages as fit the operand area (a
+    // 64-wide tile at T <= 64 moves 8 KB of weights per stage: with four stages too few bytes were in flight per SM to
+    // cover the DRAM latency)
+    const uint32_t stage_stride = a_bytes + (uint32_t)bn * BK * 2;                         // multiples of 1 KB
+    const int n_stages = min(kMaxStages, (int)((uint32_t)(kGemmStages * kGemmStageBytes) / stage_stride));
     if (warp == 1) {   // tensor memory: two 128 x 256 fp32 accumulators (per CTA; allocated for the pair in pair mode)
         if (pairs) {
             asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(kTmemCols) : "memory");
@@ -436,44 +452,50 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
         const uint32_t rank = cluster_ctarank();
         const int n_tile = has_tile ? w / m_tiles : 0, m0 = has_tile ? (w - n_tile * m_tiles) * BM : 0;
         const int kb_mid = (n_kb + 1) >> 1, kb0 = rank ? kb_mid : 0, kb1 = rank ? n_kb : kb_mid;
-        const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
-        const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages);
+        const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kMaxStages);
+        const uint32_t acc_full = smem_u32(bars + 2 * kMaxStages);
         if (has_tile && warp == 0) {
             const CUtensorMap* b_map = pick_map(b_maps, plan);
-            const uint32_t stage_tx = kATile + bn * BK * 2;
-            for (int kb = kb0, kc = 0; kb < kb1; ++kb, ++kc) {
-                const int s = kc % kGemmStages;
-                if (kc >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kGemmStages) - 1) & 1))) {
+            const uint32_t stage_tx = a_bytes + bn * BK * 2;
+            for (int kb = kb0, kc = 0, s = 0, use = 0; kb < kb1; ++kb, ++kc) {
+                if (use > 0 && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, (use - 1) & 1))) {
                     failed = true;
                     break;
                 }
                 if (elect_one()) {
-                    const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
+                    const uint32_t a_dst = smem_u32(smem + s * stage_stride), b_dst = a_dst + a_bytes;
                     const uint32_t bar = full_bar + 8 * s;
                     mbar_arrive_expect_tx(bar, stage_tx);
-                    tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
+                    tma_load_2d(a_dst, a_map1, kb * BK, m0, bar);
                     tma_load_2d(b_dst, b_map, kb * BK, n_tile * bn, bar);
                     tma_load_2d(b_dst + half_rows * BK * 2, b_map, kb * BK, n_tile * bn + half_rows, bar);
                 }
                 __syncwarp();
+                if (++s == n_stages) {
+                    s = 0;
+                    ++use;
+                }
             }
         } else if (has_tile && warp == 1) {
             const uint32_t idesc = kIdescNoN | ((uint32_t)(bn >> 3) << 17);
-            for (int kb = kb0, kc = 0; kb < kb1; ++kb, ++kc) {
-                const int s = kc % kGemmStages;
-                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kGemmStages) & 1))) {
+            for (int kb = kb0, kc = 0, s = 0, use = 0; kb < kb1; ++kb, ++kc) {
+                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, use & 1))) {
                     failed = true;
                     break;
                 }
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
-                    const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
+                    const uint32_t a_addr = smem_u32(smem + s * stage_stride);
+                    const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + a_bytes);
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k) tc_mma(tmem_base, da + 2 * k, db + 2 * k, idesc, (kc | k) ? 1u : 0u);
                     tc_commit(empty_bar + 8 * s);
                 }
                 __syncwarp();
+                if (++s == n_stages) {
+                    s = 0;
+                    ++use;
+                }
             }
             if (!failed && elect_one()) tc_commit(acc_full);    // this CTA's partial sums are complete
             __syncwarp();
@@ -545,27 +567,26 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
     } else if (!pairs) {
         const int m_tiles = (T + BM - 1) / BM;
         const int n_work = m_tiles * n_tiles;                      // (a CTA without work falls through the loops below)
-        const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kGemmStages);
-        const uint32_t acc_full = smem_u32(bars + 2 * kGemmStages), acc_empty = acc_full + 16;
+        const uint32_t full_bar = smem_u32(bars), empty_bar = smem_u32(bars + kMaxStages);
+        const uint32_t acc_full = smem_u32(bars + 2 * kMaxStages), acc_empty = acc_full + 16;
         if (warp == 0) {
             // ---------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
             const CUtensorMap* b_map = pick_map(b_maps, plan);
             const CUtensorMap* b2_map = pick_map(b2_maps, plan);
-            const uint32_t stage_tx = kATile + bn * BK * 2;
-            int kc = 0;   // k-blocks issued so far, over all tiles
+            const uint32_t stage_tx = a_bytes + bn * BK * 2;
+            int s = 0, use = 0;   // stage of the next k-block, and how often the ring has gone round (over all tiles)
             for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x) {
                 const int n_tile = w / m_tiles, m0 = (w - n_tile * m_tiles) * BM;
-                for (int kb = 0; kb < n_kb; ++kb, ++kc) {
-                    const int s = kc % kGemmStages;
-                    if (kc >= kGemmStages && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, ((kc / kGemmStages) - 1) & 1))) {
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    if (use > 0 && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * s, (use - 1) & 1))) {
                         failed = true;
                         break;
                     }
                     if (elect_one()) {
-                        const uint32_t a_dst = smem_u32(smem + s * kGemmStageBytes), b_dst = a_dst + kATile;
+                        const uint32_t a_dst = smem_u32(smem + s * stage_stride), b_dst = a_dst + a_bytes;
                         const uint32_t bar = full_bar + 8 * s;
                         mbar_arrive_expect_tx(bar, stage_tx);
-                        tma_load_2d(a_dst, &a_map, kb * BK, m0, bar);
+                        tma_load_2d(a_dst, a_map1, kb * BK, m0, bar);
                         if (MODE == kSwiGLU) {   // the gate rows, then the up rows of the same features
                             tma_load_2d(b_dst, b_map, kb * BK, n_tile * half_rows, bar);
                             tma_load_2d(b_dst + half_rows * BK * 2, b2_map, kb * BK, n_tile * half_rows, bar);
@@ -575,12 +596,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                         }
                     }
                     __syncwarp();
+                    if (++s == n_stages) {
+                        s = 0;
+                        ++use;
+                    }
                 }
             }
         } else if (warp == 1) {
             // ---------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
             const uint32_t idesc = kIdescNoN | ((uint32_t)(bn >> 3) << 17);
-            int kc = 0, it = 0;
+            int s = 0, use = 0, it = 0;
             for (int w = blockIdx.x; w < n_work && !failed; w += gridDim.x, ++it) {
                 const int acc = it & 1;
                 // the epilogue must have drained this accumulator (used by tile it - 2)
@@ -590,22 +615,25 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                 }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + acc * BN;
-                for (int kb = 0; kb < n_kb; ++kb, ++kc) {
-                    const int s = kc % kGemmStages;
-                    if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, (kc / kGemmStages) & 1))) {
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * s, use & 1))) {
                         failed = true;
                         break;
                     }
                     tc_fence_after();
                     if (elect_one()) {
-                        const uint32_t a_addr = smem_u32(smem + s * kGemmStageBytes);
-                        const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + kATile);
+                        const uint32_t a_addr = smem_u32(smem + s * stage_stride);
+                        const uint64_t da = umma_desc_sw128(a_addr), db = umma_desc_sw128(a_addr + a_bytes);
     #pragma unroll
                         for (int k = 0; k < BK / 16; ++k)   // 32 bytes along K per step = 2 descriptor address units
                             tc_mma(tmem_d, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
                         tc_commit(empty_bar + 8 * s);       // the stage is free once these MMAs have read it
                     }
                     __syncwarp();
+                    if (++s == n_stages) {
+                        s = 0;
+                        ++use;
+                    }
                 }
                 if (failed) break;
                 if (elect_one()) tc_commit(acc_full + 8 * acc);   // accumulator complete
@@ -657,7 +685,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_cons
                         const uint32_t a_dst = smem_u32(smem + s * kG2StageBytes), b_dst = a_dst + kATile;
                         if (rank == 0) mbar_arrive_expect_tx(full_bar + 8 * s, pair_tx);
                         const uint32_t bar = lead_full + 8 * s;
-                        tma_load_2d_pair(a_dst, &a_map, kb * BK, m0, bar);
+                        tma_load_2d_pair(a_dst, &a_maps.full, kb * BK, m0, bar);
                         if (MODE == kSwiGLU)      // the leader's half: 128 gate rows; the peer's: the 128 up rows of the same features
                             tma_load_2d_pair(b_dst, rank == 0 ? b_map : b2_map, kb * BK, n_tile * half_rows, bar);
                         else
@@ -858,6 +886,12 @@ dcut_status make_kmajor_map(dcut_ctx* ctx, CUtensorMap* map, const void* base, l
     return DCUT_OK;
 }
 
+dcut_status make_act_maps(dcut_ctx* ctx, AMaps* maps, const void* base, long long rows, long long cols) {
+    dcut_status st = make_kmajor_map(ctx, &maps->full, base, rows, cols, BM);
+    if (st != DCUT_OK) return st;
+    return make_kmajor_map(ctx, &maps->half, base, rows, cols, BM / 2);
+}
+
 // The weight's tensor maps for the tile widths in `mask` (box = half the width in rows)
 dcut_status make_weight_maps(dcut_ctx* ctx, BMaps* maps, const void* w, long long rows, long long cols, unsigned mask) {
     for (int i = 0; i < kNumBn; ++i) {
@@ -869,7 +903,7 @@ dcut_status make_weight_maps(dcut_ctx* ctx, BMaps* maps, const void* w, long lon
 }
 
 template <int MODE>
-dcut_status launch_gemm(dcut_ctx* ctx, const CUtensorMap& a, const BMaps& b, const BMaps& b2, int n_tiles,
+dcut_status launch_gemm(dcut_ctx* ctx, const AMaps& a, const BMaps& b, const BMaps& b2, int n_tiles,
                         int T_cap, unsigned bn_mask, const GemmArgs& g, cudaStream_t stream) {
     GemmArgs ga = g;
     ga.n_tiles = n_tiles;
@@ -930,7 +964,7 @@ struct WeightMaps {
 };
 constexpr int kLayerCache = 64;
 struct LayerMaps {
-    CUtensorMap act[4]; // norm out, attention out, norm-2 out, mlp activation
+    AMaps act[4];       // norm out, attention out, norm-2 out, mlp activation
     bool act_ready;
     WeightMaps cache[kLayerCache];
 };
@@ -1032,9 +1066,9 @@ dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_
 // logits = x . w_lm^T reduced on the fly to one (maximum, first column) word per row: the [T, V] logits never exist
 dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void* w_lm, int V, int K, const int* cu_q, int B,
                                        int T_cap, unsigned long long* row_key, cudaStream_t stream) {
-    CUtensorMap am;
+    AMaps am;
     BMaps bm;
-    dcut_status st = make_kmajor_map(ctx, &am, x, T_cap, K, BM);
+    dcut_status st = make_act_maps(ctx, &am, x, T_cap, K);
     if (st != DCUT_OK) return st;
     // rows past V read as zeros; hundreds of tiles per row block: only the full width is offered
     if ((st = make_weight_maps(ctx, &bm, w_lm, V, K, 1u)) != DCUT_OK) return st;
@@ -1055,12 +1089,12 @@ dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void*
 dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const void* w2, int mode, int N, int K,
                              const int* cu_q, int B, int T_cap, void* out, const void* residual, cudaStream_t stream) {
     // generic entry used by dcut_gemm_bf16 (tests, benchmarks): encodes its maps on every call
-    CUtensorMap am;
+    AMaps am;
     BMaps bm, b2m;
-    dcut_status st = make_kmajor_map(ctx, &am, a, T_cap, K, BM);
+    dcut_status st = make_act_maps(ctx, &am, a, T_cap, K);
     if (st != DCUT_OK) return st;
     const unsigned mask = (mode == kSwiGLU ? ctx->ly_gemm_bn_mask & kBnMaskSwiGLU : ctx->ly_gemm_bn_mask) | 1u;
-    for (int i = 0; i < kNumBn; ++i) bm.m[i] = am;     // entries outside the mask are never used; keep them defined
+    for (int i = 0; i < kNumBn; ++i) bm.m[i] = am.full;   // entries outside the mask are never used; keep them defined
     if ((st = make_weight_maps(ctx, &bm, w, N, K, mask)) != DCUT_OK) return st;
     b2m = bm;
     if (mode == kSwiGLU && (st = make_weight_maps(ctx, &b2m, w2, N, K, mask)) != DCUT_OK) return st;
@@ -1090,10 +1124,10 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     LayerMaps* lm = static_cast<LayerMaps*>(ctx->layer_maps);
     dcut_status st;
     if (!lm->act_ready) {
-        if ((st = make_kmajor_map(ctx, &lm->act[0], ctx->ly_norm, max_T, H, BM)) != DCUT_OK) return st;
-        if ((st = make_kmajor_map(ctx, &lm->act[1], ctx->ly_attn, max_T, q_w, BM)) != DCUT_OK) return st;
-        if ((st = make_kmajor_map(ctx, &lm->act[2], ctx->ly_norm2, max_T, H, BM)) != DCUT_OK) return st;
-        if ((st = make_kmajor_map(ctx, &lm->act[3], ctx->ly_act, max_T, I, BM)) != DCUT_OK) return st;
+        if ((st = make_act_maps(ctx, &lm->act[0], ctx->ly_norm, max_T, H)) != DCUT_OK) return st;
+        if ((st = make_act_maps(ctx, &lm->act[1], ctx->ly_attn, max_T, q_w)) != DCUT_OK) return st;
+        if ((st = make_act_maps(ctx, &lm->act[2], ctx->ly_norm2, max_T, H)) != DCUT_OK) return st;
+        if ((st = make_act_maps(ctx, &lm->act[3], ctx->ly_act, max_T, I)) != DCUT_OK) return st;
         lm->act_ready = true;
     }
     const void* wp[5] = {w->w_qkv, w->w_o, w->w_gate, w->w_up, w->w_down};
