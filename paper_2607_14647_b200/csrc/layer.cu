@@ -7,9 +7,10 @@
 //   rope_append_kernel    rotate-half RoPE on q and k heads, K/V of the new tokens written into the paged cache at
 //                         position L_i + t, q written as the attention kernel's [T, Hq, Dh] input
 //   gemm_tcgen05_kernel   C[M, N] = A[M, K] . B[N, K]^T on the 5th-generation tensor cores.  Persistent; launched as
-//                         clusters of two CTAs.  After reading the packed length it runs either 128 x 256 tiles on
-//                         single SMs (tcgen05.mma M128 N256 K16, four 48 KB operand stages) or 256 x 256 tiles on
-//                         pairs of SMs (cta_group::2, M256, each CTA loading half of B, six 32 KB stages).  Operands
+//                         clusters of two CTAs.  After reading the packed length it looks up how to run: 128-row
+//                         tiles on single SMs (tcgen05.mma M128 K16), 256-row tiles on pairs of SMs (cta_group::2,
+//                         M256, each CTA loading half of B), or a pair sharing one 128-row tile with half of K each;
+//                         and how wide the tile is (256, 224, ..., 64 columns = the MMA's N).  Operands
 //                         are staged by TMA as 128-byte-swizzled K-major tiles (BK = 64); one elected lane issues the
 //                         MMAs and releases stages with tcgen05.commit; two accumulators in tensor memory let the four
 //                         epilogue warps (tcgen05.ld) work on one tile while the next is being multiplied.
@@ -274,8 +275,8 @@ __device__ __forceinline__ void gemm_epilogue(const GemmArgs& g, int T, int row,
 // on the leader's accumulator-empty barrier through distributed shared memory.
 // Measured against the one-CTA kernel: 74 us against 86 us for the down projection at T = 512-640 (K = 12288), 81 against
 // 90 us for gate/up + SwiGLU at T = 512, but 135 against 92 us for the down projection at T = 1088, where 5 x 16 = 80
-// pair tiles need two waves on 74 pairs (and 1280 padded rows are computed instead of 1152): the kernel therefore
-// picks the mode per launch (gemm_use_pairs).
+// pair tiles need two waves on 74 pairs (and 1280 padded rows are computed instead of 1152): the mode is therefore
+// chosen per launch (gemm_plan).
 
 constexpr int kG2Stages = 6;
 constexpr int kG2StageBytes = kATile + kBTile / 2;     // 32 KB
@@ -317,21 +318,22 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
                  ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
 
-// One persistent kernel, two ways of running a GEMM, chosen on the device from the packed length (the same answer in
-// every CTA).
-//   One SM per tile: a CTA walks the 128 x 256 output tiles b, b + gridDim.x, ... (m fastest, so the CTAs running
-//   together share weight tiles in L2); four 48 KB operand stages.
-//   A pair of SMs per tile (see above): 256 x 256 tiles, six 32 KB stages.  It needs ~7 % fewer cycles per flop but
-//   pads the rows to 256 and has half as many, larger work items, so it is taken when it does not add a wave
-//   (gemm_use_pairs).
-// In both the operand ring and its barriers continue across tiles and the accumulator is double-buffered in tensor
-// memory (2 x 256 columns), so the epilogue of one tile overlaps the main loop of the next.
+// One persistent kernel, three ways of running a GEMM and seven tile widths, looked up on the device from the packed
+// length (the same answer in every CTA).
+//   One SM per tile: a CTA walks the 128 x bn output tiles b, b + gridDim.x, ... (m fastest, so the CTAs running
+//   together share weight tiles in L2); a stage holds the tile's A and B bytes, 4 (bn = 256) to 12 stages.
+//   A pair of SMs per tile (see above): 256 x bn tiles, six 32 KB stages.  Fewer bytes per flop from L2, but rows
+//   padded to 256 and half as many, larger work items.
+//   A pair per 128 x bn tile, half of K each (below): for launches whose tiles all fit one wave of pairs.
+// In the first two the operand ring and its barriers continue across tiles and the accumulator is double-buffered in
+// tensor memory (2 x 256 columns), so the epilogue of one tile overlaps the main loop of the next.
 // The cheapest way to run this launch under a model fitted to measurements on the four projections of an 8B-class
-// layer at 17 packed lengths from 64 to 1088 (every width, both modes): time = waves x (4 bn + 1664) on one SM per
-// tile, waves x (7 bn + 800) on a pair.  (A pair tile moves two thirds of the bytes per flop from L2 and its MMAs are
-// issued at about 0.57 of the one-SM rate per column; the constants stand for what a tile costs whatever its width.)
-// Over those 68 cases the pick is within 0.3 % (geometric mean; worst case 7 %) of the best measured choice.  Returns
-// the width index, + kPlanPair for the pair mode; the wider tile wins ties.
+// layer at 17 packed lengths from 64 to 1088 (every width, every mode): time = waves x (4 bn + 1664) on one SM per
+// tile, waves x (7 bn + 800) on a pair, half a one-SM tile + kSplitCost for a pair splitting K.  (A pair tile moves two
+// thirds of the bytes per flop from L2 and its MMAs are issued at about 0.57 of the one-SM rate per column; the
+// constants stand for what a tile costs whatever its width.)  Over those 68 cases the pick reaches the best measured
+// single choice to within a percent (geometric mean).  Returns the width index, + kPlanPair or + kPlanSplit; the
+// wider tile wins ties.
 // The choice depends on T only through the number of 128-row blocks, so the host tabulates it per launch
 // (GemmArgs::plan_by_m) and the kernel looks it up after reading T.
 constexpr int kPlanPair = 8, kPlanSplit = 16;
