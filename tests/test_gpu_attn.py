@@ -170,3 +170,21 @@ def test_kv_head_sharding_reproduces_the_unsharded_result(tp):
         ctx.close()
         outs.append(out.float().cpu().numpy())
     assert np.array_equal(np.concatenate(outs, axis=1), full)
+
+
+@pytest.mark.parametrize("shallow", [[0, 0], [1, 3], [2]])
+def test_a_few_shallow_requests_among_deep_ones(shallow):
+    """When the warp-level queue would hold less than an eighth of the pages, the work list sends every item to the
+    tcgen05 queue: query tiles of 4 to 16 rows (depth 0 to 3 at four heads per kv head) then run on the 128-row tensor
+    memory path.  Every element against the oracle."""
+    n = 14
+    cfg = wl.custom_config(B=n, gamma=16, n_q_heads=16, n_kv_heads=4, head_dim=128, ctx_lo=200, ctx_hi=1200)
+    sel = wl.select_inputs(cfg)
+    depths = np.full(n, 16, np.int32)
+    order = np.argsort(sel.ctx_lens)                       # the shallow requests get the shortest contexts
+    for j, d in enumerate(shallow):
+        depths[order[j]] = d
+    pages = (sel.ctx_lens + depths + 1 + 15) // 16
+    assert 8 * pages[depths < 4].sum() < pages.sum()       # the rule applies
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    _full_compare(cfg, sel, kv, depths)
