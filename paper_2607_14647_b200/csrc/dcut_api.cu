@@ -77,6 +77,9 @@ void free_all(dcut_ctx* c) {
     cudaFree(c->hs_out);
     cudaFree(c->hs_logits);
     if (c->hs_host_cu_q) cudaFreeHost(c->hs_host_cu_q);
+    if (c->hs_copy_stream) cudaStreamDestroy(c->hs_copy_stream);
+    if (c->hs_ev_fork) cudaEventDestroy(c->hs_ev_fork);
+    if (c->hs_ev_join) cudaEventDestroy(c->hs_ev_join);
 }
 
 }  // namespace
@@ -505,6 +508,9 @@ dcut_status ensure_host_step_buffers(dcut_ctx* c, int V) {
         if ((st = dmalloc(c, &c->hs_out, max_T * l.n_q_heads * l.head_dim, "cudaMalloc(step out)")) != DCUT_OK) return st;
         cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&c->hs_host_cu_q), sizeof(int) * ((size_t)l.max_B + 1));
         if (e != cudaSuccess) return dcut_check_cuda(c, e, "cudaMallocHost(step cu_q)");
+        if ((e = cudaStreamCreateWithFlags(&c->hs_copy_stream, cudaStreamNonBlocking)) != cudaSuccess) return dcut_check_cuda(c, e, "cudaStreamCreate(step copy)");
+        if ((e = cudaEventCreateWithFlags(&c->hs_ev_fork, cudaEventDisableTiming)) != cudaSuccess) return dcut_check_cuda(c, e, "cudaEventCreate(step)");
+        if ((e = cudaEventCreateWithFlags(&c->hs_ev_join, cudaEventDisableTiming)) != cudaSuccess) return dcut_check_cuda(c, e, "cudaEventCreate(step)");
     }
     if (c->hs_logits) cudaFree(c->hs_logits);
     c->hs_logits = nullptr;
@@ -548,18 +554,30 @@ extern "C" dcut_status dcut_verify_step_host(dcut_ctx* c, const dcut_host_step* 
     const int* cu = c->hs_host_cu_q;
     long long h2d = (long long)(sizeof(float) + sizeof(int)) * B * g + 2ll * sizeof(int) * B +
                     (long long)sizeof(int) * B * s->block_table_stride;
+    // The logits (the bulk of the bytes) travel on a second stream while the query rows are copied and attention
+    // runs on the caller's; acceptance waits for both.  (The previous call ended with a synchronisation, so nothing
+    // still reads the buffers that are being overwritten.)
+    if ((st = dcut_check_cuda(c, cudaEventRecord(c->hs_ev_fork, cs), "cudaEventRecord(step fork)")) != DCUT_OK) return st;
+    if ((st = dcut_check_cuda(c, cudaStreamWaitEvent(c->hs_copy_stream, c->hs_ev_fork, 0), "cudaStreamWaitEvent(step fork)")) != DCUT_OK) return st;
     for (int i = 0; i < B; ++i) {
         const size_t rows = (size_t)(cu[i + 1] - cu[i]);
         DCUT_CP(reinterpret_cast<char*>(c->hs_q) + (size_t)cu[i] * q_row,
                 static_cast<const char*>(s->q_rows) + (size_t)i * (g + 1) * q_row, rows * q_row, cudaMemcpyHostToDevice);
-        DCUT_CP(reinterpret_cast<char*>(c->hs_logits) + (size_t)cu[i] * lg_row,
-                static_cast<const char*>(s->logits_rows) + (size_t)i * (g + 1) * lg_row, rows * lg_row, cudaMemcpyHostToDevice);
         h2d += (long long)(rows * (q_row + lg_row));
     }
+    for (int i = 0; i < B; ++i) {
+        const size_t rows = (size_t)(cu[i + 1] - cu[i]);
+        if ((st = dcut_check_cuda(c, cudaMemcpyAsync(reinterpret_cast<char*>(c->hs_logits) + (size_t)cu[i] * lg_row,
+                                                     static_cast<const char*>(s->logits_rows) + (size_t)i * (g + 1) * lg_row,
+                                                     rows * lg_row, cudaMemcpyHostToDevice, c->hs_copy_stream),
+                                  "cudaMemcpyAsync(step logits)")) != DCUT_OK) return st;
+    }
+    if ((st = dcut_check_cuda(c, cudaEventRecord(c->hs_ev_join, c->hs_copy_stream), "cudaEventRecord(step join)")) != DCUT_OK) return st;
     const int T_cap = B * (g + 1);
     st = dcut_verify_attn(c, c->hs_q, s->k_cache, s->v_cache, s->num_pages, c->hs_block_table, s->block_table_stride,
                           c->hs_ctx_lens, c->hs_cu_q, B, T_cap, s->scale, c->hs_out, nullptr, stream);
     if (st != DCUT_OK) return st;
+    if ((st = dcut_check_cuda(c, cudaStreamWaitEvent(cs, c->hs_ev_join, 0), "cudaStreamWaitEvent(step join)")) != DCUT_OK) return st;
     int* acc = c->hs_accept;            // [B] accept_len, [B] bonus, [B*(g+1)] tokens, [1] total
     st = dcut_accept(c, c->hs_logits, V, c->hs_draft, c->hs_cu_q, B, g, T_cap, acc, acc + B, acc + 2 * B,
                      acc + 2 * B + B * (g + 1), stream);
