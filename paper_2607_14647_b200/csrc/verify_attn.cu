@@ -447,6 +447,17 @@ __device__ __forceinline__ uint64_t desc_kmajor(uint32_t addr) {
     return (uint64_t)((addr & 0x3ffff) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) |
            ((uint64_t)2 << 61);
 }
+// the same with the 8-row groups 2048 bytes apart: the two 64-column halves of a 128-wide K row sit side by side
+// (group, half, row), which is the order one 4-D TMA box per page delivers
+__device__ __forceinline__ uint64_t desc_kmajor_2k(uint32_t addr) {
+    return (uint64_t)((addr & 0x3ffff) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(2048 >> 4) << 32) | ((uint64_t)1 << 46) |
+           ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
 // MN-major tile (rows = K index, 128 bytes = 64 consecutive MN elements per row): the next 64 MN elements are
 // 2048 bytes on (leading byte offset), the next 8 K rows 1024 bytes on (stride byte offset)
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t addr) {
@@ -952,8 +963,8 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
                         if (j < np) {
-                            tma_load_2d(dst + j * 2048, &k2_map, 0, rows[j], bar);            // K columns 0..63 of page j
-                            tma_load_2d(dst + 8192 + j * 2048, &k2_map, 64, rows[j], bar);    // K columns 64..127
+                            // page j of K as one 4 KB box: (two 8-row groups) x (two 64-column halves) x 8 rows x 128 bytes
+                            tma_load_4d(dst + j * 4096, &k2_map, 0, 0, 0, rows[j] >> 3, bar);
                             tma_load_tile(dst + 4 * kTcPageBytes + j * kTcPageBytes, &v_map, rows[j], bar);
                         }
                 }
@@ -993,7 +1004,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                     const uint32_t k_addr = smem_u32(ring + gs * kTcGroupBytes);
                     const uint32_t d = tmem_o + kTcColS + 64 * b;
                     const uint32_t idesc = kIdescBase | ((uint32_t)(np * kPage >> 3) << 17);
-                    const uint64_t dk0 = desc_kmajor(k_addr), dk1 = desc_kmajor(k_addr + 8192);
+                    const uint64_t dk0 = desc_kmajor_2k(k_addr), dk1 = desc_kmajor_2k(k_addr + 1024);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)    // 16 head-dim elements = 8 words of Q, 32 bytes along a K row
                         tc_mma_ts(d, tmem_q + ks * 8, dk0 + 2 * ks, idesc, ks ? 1u : 0u);
@@ -1453,12 +1464,15 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     st = make_cache_map(ctx, &vm, v_cache, num_pages);
     if (st != DCUT_OK) return st;
     k2m = km;
-    if (ctx->lim.head_dim == 128) {   // the K cache as a plain 2-D matrix of token rows, {64 columns, 16 rows} boxes
-        cuuint64_t dims[2] = {128, (cuuint64_t)num_pages * ctx->lim.n_kv_heads * kPage};
-        cuuint64_t strides[1] = {256};
-        cuuint32_t box[2] = {64, kPage}, estr[2] = {1, 1};
+    if (ctx->lim.head_dim == 128) {
+        // The K cache for the tcgen05 phase: token rows of 128 columns seen as (64 columns, 8 rows, 2 halves, groups of
+        // 8 rows), so that a {64, 8, 2, 2} box (one page: 16 rows, 4 KB) arrives as [group][half][row][64 columns]:
+        // each half is a K-major tile of 128-byte rows whose 8-row groups are 2048 bytes apart.
+        cuuint64_t dims[4] = {64, 8, 2, (cuuint64_t)num_pages * ctx->lim.n_kv_heads * kPage / 8};
+        cuuint64_t strides[3] = {256, 128, 2048};
+        cuuint32_t box[4] = {64, 8, 2, 2}, estr[4] = {1, 1, 1, 1};
         CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
-            &k2m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(k_cache), dims, strides, box, estr,
+            &k2m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(k_cache), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return dcut_fail(ctx, DCUT_ECUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
