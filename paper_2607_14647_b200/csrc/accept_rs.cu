@@ -97,28 +97,33 @@ __global__ void __launch_bounds__(kStatThreads) rs_stats_kernel(RsArgs a) {
                 const int k = k0 + u * kStatThreads + threadIdx.x;
                 w[u] = k < nvec ? ld_stream_v4(vp + k) : make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
             }
+            // Two values per word: NaN is turned into -inf (weight 0) and the batch maximum is taken on the packed
+            // words (max.bf16x2 returns the other operand for a NaN), one instruction per two values each
             float x[8 * kUnroll];
-            float vmax = -INFINITY;
+            unsigned int wmax = 0xff80ff80u;
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const unsigned int ws[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    x[8 * u + 2 * e] = __uint_as_float(ws[e] << 16);
-                    x[8 * u + 2 * e + 1] = __uint_as_float(ws[e] & 0xffff0000u);
-                    vmax = fmaxf(vmax, fmaxf(x[8 * u + 2 * e], x[8 * u + 2 * e + 1]));   // fmaxf drops NaN
+                    unsigned int c;
+                    asm("max.bf16x2 %0, %1, %2;" : "=r"(c) : "r"(ws[e]), "r"(0xff80ff80u));
+                    asm("max.bf16x2 %0, %1, %2;" : "=r"(wmax) : "r"(wmax), "r"(c));
+                    x[8 * u + 2 * e] = __uint_as_float(c << 16);
+                    x[8 * u + 2 * e + 1] = __uint_as_float(c & 0xffff0000u);
                 }
             }
+            const float vmax = fmaxf(__uint_as_float(wmax << 16), __uint_as_float(wmax & 0xffff0000u));
             const float mn = fmaxf(m, vmax);
             if (mn > -INFINITY) {
-                // exp(x - mn) = 2^(x * log2(e) - mn * log2(e)): one FMA, one clamp that turns NaN into -inf (weight 0),
-                // one special-function operation, one add per value; two partial sums for instruction-level parallelism
+                // exp(x - mn) = 2^(x * log2(e) - mn * log2(e)): one FMA, one special-function operation, one add per
+                // value; two partial sums for instruction-level parallelism
                 const float kL2e = 1.4426950408889634f, off = -mn * kL2e;
                 float add0 = 0.0f, add1 = 0.0f;
 #pragma unroll
                 for (int e = 0; e < 8 * kUnroll; e += 2) {
-                    add0 += exp2f_fast(fmaxf(fmaf(x[e], kL2e, off), -INFINITY));
-                    add1 += exp2f_fast(fmaxf(fmaf(x[e + 1], kL2e, off), -INFINITY));
+                    add0 += exp2f_fast(fmaf(x[e], kL2e, off));
+                    add1 += exp2f_fast(fmaf(x[e + 1], kL2e, off));
                 }
                 s = s * __expf(m - mn) + (add0 + add1);
                 m = mn;
