@@ -324,7 +324,10 @@ dcut_status dcut_model_verify(dcut_ctx* ctx, const dcut_model* model, long long 
  * (64 KB) on every GPU that loads the library, held until the process exits.
  *
  * Same arguments, same results and same DEVICE / caller-owned buffers as dcut_accept; the device that
- * holds the buffers must be current.  T_cap > DCUT_ACCEPT_STATIC_MAX_ROWS returns DCUT_ECAPACITY
+ * holds the buffers must be current.  cu_q[B] <= T_cap is the caller's contract, as for dcut_accept; this
+ * call has no status word to report a breach through, but it never touches a row at or past T_cap (such
+ * rows are left out of the prefix match, a request with no row left reports accept_len 0 and bonus 0), so
+ * nothing outside the first T_cap words of the fixed array is read or written.  T_cap > DCUT_ACCEPT_STATIC_MAX_ROWS returns DCUT_ECAPACITY
  * (use dcut_accept then).  errbuf (HOST, may be NULL) receives a message when the status is not
  * DCUT_OK.  The call never calls cudaMalloc, cudaFree or any allocating routine; it issues one
  * cudaMemsetAsync and two kernels on `stream`.
@@ -385,7 +388,9 @@ dcut_status dcut_verify_step_host(dcut_ctx* ctx, const dcut_host_step* step, voi
  * and clears it.  A non-zero code also makes this call return DCUT_EDEVICE.  Codes: 1 = a bounded
  * wait in the attention kernel gave up, 2 = a block-table entry outside [0, num_pages) (page 0 was
  * read instead), 3 = the attention work list did not fit the scratch, 4 = a bounded wait in the GEMM
- * kernel gave up, 5 = dcut_commit ran out of room, 6 = dcut_model_verify met a token id outside [0, vocab). */
+ * kernel gave up, 5 = dcut_commit ran out of room, 6 = dcut_model_verify met a token id outside [0, vocab),
+ * 7 = an acceptance call met a cu_q that is not a packing of B requests of 1 .. gamma + 1 rows inside T_cap
+ * (rows at or past T_cap were left out: nothing outside the caller's T_cap rows is read or written). */
 dcut_status dcut_poll_device_status(dcut_ctx* ctx, int* code, void* stream);
 
 #ifdef __cplusplus

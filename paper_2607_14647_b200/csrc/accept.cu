@@ -47,7 +47,7 @@ __global__ void __launch_bounds__(kArgmaxThreads) accept_argmax_kernel(
     unsigned long long* __restrict__ row_key) {
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
-    const int row = blockIdx.y;
+    const int row = blockIdx.y;   // < T_cap, the rows the per-row words are sized for
     if (row >= cu_q[B]) return;
     const int start = blockIdx.x * seg_elems;
     if (start >= V) return;
@@ -107,11 +107,14 @@ __device__ int slow_first_valid(const unsigned short* rp, int V) {
 
 // One warp per request: the lanes fetch the row results of t = lane, lane + 32, ... together, a ballot finds the
 // first row whose argmax differs from the draft (or the last row), and the per-row words are cleared on the way.
+// Only rows below row_cap (the T_cap the words and the scan were sized for) exist: a cu_q that runs past it breaks the
+// caller's contract, so those rows are neither read nor cleared, the request's scan ends at the last row that
+// exists (a request with none reports accept_len 0 and bonus 0), and the status word, if there is one, says so.
 __global__ void __launch_bounds__(1024) accept_match_kernel(
     const unsigned short* __restrict__ logits, int V, const int* __restrict__ draft_ids,
-    const int* __restrict__ cu_q, int B, int gamma, unsigned long long* __restrict__ row_key,
+    const int* __restrict__ cu_q, int B, int gamma, int row_cap, unsigned long long* __restrict__ row_key,
     int* __restrict__ accept_len, int* __restrict__ bonus, int* __restrict__ out_tokens,
-    int* __restrict__ n_accepted_total, int* __restrict__ row_argmax) {
+    int* __restrict__ n_accepted_total, int* __restrict__ row_argmax, int* __restrict__ status) {
     __shared__ int total_s;
     if (threadIdx.x == 0) total_s = 0;
     __syncthreads();
@@ -120,8 +123,14 @@ __global__ void __launch_bounds__(1024) accept_match_kernel(
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     int local = 0;
     for (int i = warp; i < B; i += n_warps) {
-        const int a = cu_q[i], d = cu_q[i + 1] - a - 1;
-        int m = -1, bon = 0;
+        const int a = cu_q[i];
+        int d = cu_q[i + 1] - a - 1;
+        if (a < 0 || d < 0 || d > gamma || a + d >= row_cap) {
+            if (lane == 0 && status) atomicExch(status, DCUT_DEV_BAD_CU_Q);
+            d = min(min(d, gamma), row_cap - 1 - a);       // rows [a, a + d] exist; none if d < 0 or a < 0
+            if (a < 0) d = -1;
+        }
+        int m = d < 0 ? 0 : -1, bon = 0;
         for (int t0 = 0; t0 <= d; t0 += 32) {
             const int t = t0 + lane;
             int am = 0;
@@ -182,18 +191,20 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
                                      "launch accept_argmax_kernel");
     if (st != DCUT_OK) return st;
     return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
-                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, row_key,
-                                                accept_len, bonus, out_tokens, n_accepted_total, static_cast<int*>(nullptr)),
+                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
+                                                row_key, accept_len, bonus, out_tokens, n_accepted_total,
+                                                static_cast<int*>(nullptr), ctx->d_status),
                            "launch accept_match_kernel");
 }
 
 dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
-                                     int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
+                                     int B, int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
                                      int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
                                      cudaStream_t stream) {
     return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
-                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, row_key,
-                                                accept_len, bonus, out_tokens, n_accepted_total, row_argmax),
+                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
+                                                row_key, accept_len, bonus, out_tokens, n_accepted_total, row_argmax,
+                                                ctx->d_status),
                            "launch accept_match_kernel");
 }
 
@@ -230,6 +241,10 @@ extern "C" dcut_status dcut_accept_static(const void* logits, int V, const int* 
     }
     if (B < 1 || gamma < 1 || V < 1 || T_cap < B) {
         static_msg(errbuf, errbuf_len, "dcut_accept_static: need B, gamma, V >= 1 and T_cap >= B");
+        return DCUT_EINVAL;
+    }
+    if (reinterpret_cast<uintptr_t>(logits) & 1) {
+        static_msg(errbuf, errbuf_len, "dcut_accept_static: logits must be 2-byte aligned");
         return DCUT_EINVAL;
     }
     if (T_cap > DCUT_ACCEPT_STATIC_MAX_ROWS || B > 1024 * 64) {
@@ -286,8 +301,9 @@ extern "C" dcut_status dcut_accept_static(const void* logits, int V, const int* 
     dim3 grid(splits, T_cap);
     accept_argmax_kernel<<<grid, kArgmaxThreads, 0, cs>>>(static_cast<const unsigned short*>(logits), V, cu_q, B, seg, keys);
     if ((e = cudaGetLastError()) == cudaSuccess) {
-        accept_match_kernel<<<1, 1024, 0, cs>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma,
-                                               keys, accept_len, bonus, out_tokens, n_accepted_total, nullptr);
+        // rows at or past T_cap are never touched, so nothing outside the first T_cap words of the array is
+        accept_match_kernel<<<1, 1024, 0, cs>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
+                                               keys, accept_len, bonus, out_tokens, n_accepted_total, nullptr, nullptr);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) {

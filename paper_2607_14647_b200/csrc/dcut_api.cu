@@ -416,7 +416,7 @@ dcut_status dcut_lm_head_accept(dcut_ctx* c, const void* x, const void* w_lm, in
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     dcut_status st = dcut_launch_lm_head_argmax(c, x, w_lm, V, c->lim.hidden, cu_q, B, T_cap, c->d_row_key, s);
     if (st != DCUT_OK) return st;
-    return dcut_launch_accept_match(c, nullptr, V, draft_ids, cu_q, B, gamma, accept_len, bonus, out_tokens,
+    return dcut_launch_accept_match(c, nullptr, V, draft_ids, cu_q, B, gamma, T_cap, accept_len, bonus, out_tokens,
                                     n_accepted_total, row_argmax, c->d_row_key, s);
 }
 

@@ -18,6 +18,7 @@
 #define DCUT_DEV_GEMM_WAIT_TIMEOUT 4    // a bounded mbarrier wait in the GEMM kernel gave up
 #define DCUT_DEV_COMMIT_OVERFLOW 5      // dcut_commit: a context or a token stream ran out of room
 #define DCUT_DEV_BAD_TOKEN 6            // dcut_model_verify: a token id outside [0, vocab)
+#define DCUT_DEV_BAD_CU_Q 7             // acceptance: cu_q is not a packing of B requests of 1..gamma+1 rows within T_cap
 
 // One split-KV work item of the attention kernel: one (request, kv head, page range).
 struct __align__(16) AttnItem {
@@ -58,7 +59,8 @@ struct dcut_ctx {
     int target_items;
     int attn_tail_req_div;  // the shortest max(1, B / this) requests are cut finer (0: none)
     int attn_tail_min_pages;
-    int attn_tc_min_rows;   // items with at least this many query rows (and <= 128) use the tcgen05 kernel
+    int attn_tc_min_rows;   // items with at least this many query rows use the tcgen05 phase
+    int attn_tail_rows;     // a query tile of up to 128 + this many rows stays one item (0: cut at 128)
 
     // accept scratch
     unsigned long long* d_row_key;   // [max_T] packed (ordered max, ~index); zero between calls
@@ -160,7 +162,7 @@ dcut_status dcut_launch_lm_head_argmax(dcut_ctx* ctx, const void* x, const void*
                                        int T_cap, unsigned long long* row_key, cudaStream_t stream);
 // second half of dcut_accept on per-row words that are already filled (logits may be null: rows without a word give 0)
 dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids, const int* cu_q,
-                                     int B, int gamma, int* accept_len, int* bonus, int* out_tokens,
+                                     int B, int gamma, int T_cap, int* accept_len, int* bonus, int* out_tokens,
                                      int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
                                      cudaStream_t stream);
 dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_pages, const int* block_table,

@@ -1061,7 +1061,7 @@ dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_
                                                    static_cast<const __nv_bfloat16*>(m->g_final), cu_q, B, H, eps, ctx->ly_norm),
                               "launch rmsnorm_kernel")) != DCUT_OK) return st;
     if ((st = dcut_launch_lm_head_argmax(ctx, ctx->ly_norm, m->w_lm, m->vocab, H, cu_q, B, T_cap, ctx->d_row_key, stream)) != DCUT_OK) return st;
-    return dcut_launch_accept_match(ctx, nullptr, m->vocab, draft_ids, cu_q, B, gamma, accept_len, bonus, out_tokens,
+    return dcut_launch_accept_match(ctx, nullptr, m->vocab, draft_ids, cu_q, B, gamma, T_cap, accept_len, bonus, out_tokens,
                                     n_accepted_total, row_argmax, ctx->d_row_key, stream);
 }
 

@@ -14,12 +14,6 @@
 #include <limits.h>
 
 #include "dcut_internal.h"
-#ifdef DCUT_PROFILE_SEL
-#include <stdio.h>
-#define SELP(...) __VA_ARGS__
-#else
-#define SELP(...)
-#endif
 
 namespace {
 
@@ -181,7 +175,6 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
 
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
-    SELP(long long t0 = clock64();)
     // 1. prefix scores and sort keys.  The confidences come in through shared memory with coalesced loads
     // (the later prefix-sum array is free at this point), so the per-request product chain reads no global memory.
     float* conf_s = reinterpret_cast<float*>(qs);
@@ -204,13 +197,10 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     for (int r = n + tid; r < npad; r += kThreads) keys[r] = ~0ull;
     for (int i = tid; i < B; i += kThreads) depth_s[i] = 0;
     __syncthreads();
-
-    SELP(long long t1 = clock64();)
     // 2. bitonic sort, ascending, over S = max(npad, 1024) keys held in registers: thread t owns elements
     // e * 1024 + t.  Compare-exchange distances below 32 go through warp shuffles, distances 32..512 through a
     // double-buffered shared array (one barrier per stage), distances >= 1024 stay inside the thread.
     sort_keys(keys, xbuf, npad);
-    SELP(long long t2 = clock64();)
     // 3. fixed-point prefix sums Q[0..n]; ranks
     {
         const int per = (npad + kThreads - 1) / kThreads;
@@ -241,8 +231,6 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
         }
     }
     __syncthreads();
-
-    SELP(long long t3 = clock64();)
     // 4. objective over the candidates
     if (a.causal && a.n_buckets == 0) {
         // Causal early-stopping scan (Appendix B): positions are admitted in ranked order while the objective strictly
@@ -314,8 +302,6 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
         __syncthreads();
     }
     const int n_star = best_s.N;
-
-    SELP(long long t4 = clock64();)
     // 5. depths, cu_q, packed token metadata
     for (int r = tid; r < n_star; r += kThreads) atomicAdd(&depth_s[(int)(keys[r] & 0xffffu)], 1);
     __syncthreads();
@@ -358,7 +344,6 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
             if (a.tok_id) a.tok_id[idx] = -1;
         }
     }
-    SELP(if (tid == 0) printf("select cycles: load+products %lld sort %lld scan %lld objective %lld depths+meta %lld\n", t1 - t0, t2 - t1, t3 - t2, t4 - t3, clock64() - t4);)
     if (tid == 0 && a.info) {
         dcut_select_info out;
         out.n_star = n_star;

@@ -28,37 +28,13 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <stdlib.h>
-#ifdef DCUT_PROFILE_STAMPS
-// profiling builds only: wall-clock stamps (ns) of the three kernels of one call
-__device__ unsigned long long g_attn_stamps[8];   // plan start/end, item first start/last end, combine first start/last end, item first-CTA-after-wait
-__device__ __forceinline__ unsigned long long gtime() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-#define STAMP_MIN(i) do { if (threadIdx.x == 0) atomicMin(&g_attn_stamps[i], gtime()); } while (0)
-#define STAMP_MAX(i) do { if (threadIdx.x == 0) atomicMax(&g_attn_stamps[i], gtime()); } while (0)
-extern "C" void dcut_debug_attn_stamps(unsigned long long* out) {
-    cudaMemcpyFromSymbol(out, g_attn_stamps, sizeof(unsigned long long) * 8);
-    unsigned long long init[8] = {~0ull, 0, ~0ull, 0, ~0ull, 0, ~0ull, 0};
-    cudaMemcpyToSymbol(g_attn_stamps, init, sizeof(init));
-}
-#else
-#define STAMP_MIN(i)
-#define STAMP_MAX(i)
-#endif
-#ifdef DCUT_PROFILE_TC
-#include <stdio.h>
-#define TCP(...) __VA_ARGS__
-#else
-#define TCP(...)
-#endif
+#include <type_traits>
 
 #include "dcut_internal.h"
 
 namespace {
 
-constexpr int kThreads = 320;        // tcgen05 phase: TMA warp, MMA warp, 8 softmax warps; warp-level phase: 8 consumer warps + 1 producer
+constexpr int kThreads = 384;        // tcgen05 phase: TMA warp, MMA warp, 8 softmax warps, 2 tail-row warps; warp-level phase: 8 consumer warps + 1 producer
 constexpr int kMmaWarps = 8;         // consumer warps of the warp-level MMA phase
 constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kMmaStages = 16;       // page stages in its ring (8 KB each at head_dim 128)
@@ -131,6 +107,18 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// the same without `volatile`: a pure function of its operands, which the compiler may move across the loads around it
+__device__ __forceinline__ void mma_bf16_pure(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// transposes an 8 x 8 matrix of 16-bit elements held one row per four lanes (lane 4 g + t: row g, elements 2 t, 2 t + 1)
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
+    uint32_t r;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(v));
+    return r;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -147,6 +135,11 @@ __device__ __forceinline__ uint32_t tile_off(int r, int c16) {
     return (uint32_t)(((c16 >> 3) << 11) + (r << 7) + (((c16 & 7) ^ (r & 7)) << 4));
 }
 
+// the same for a K page of the tcgen05 phase, which one 4-D TMA box delivers as [8-row group][half][8 rows][64 columns]
+__device__ __forceinline__ uint32_t tile_off_k4(int r, int c16) {
+    return (uint32_t)(((r >> 3) << 11) + ((c16 >> 3) << 10) + ((r & 7) << 7) + (((c16 & 7) ^ (r & 7)) << 4));
+}
+
 // ------------------------------------------------------------------------------------------------
 // plan
 
@@ -155,6 +148,7 @@ struct PlanArgs {
     const int* cu_q;
     int B, n_q_heads, n_kv_heads;
     int target_items, min_chunk_pages, max_items, npad, tc_min_rows, max_item_rows;
+    int tail_rows;                      // a remainder of at most this many rows rides with the last full row block (0: never)
     int tail_req_div, tail_min_pages;   // the shortest B / tail_req_div requests are cut finer (0: none)
     long long part_rows_cap;
     int* status;
@@ -191,6 +185,18 @@ __device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* to
     return res;
 }
 
+// Row blocks of a query tile of M rows: full blocks of max_rows rows and one remainder.  A remainder of at most
+// tail_rows rows does not become an item of its own (which would stream the request's K/V a second time): it rides
+// with the last full block, whose item then has up to max_rows + tail_rows rows (the tail warps of the tcgen05 phase
+// take the rows past max_rows from the same staged pages).
+__device__ __forceinline__ int plan_row_blocks(int M, int max_rows, int tail_rows) {
+    const int n_full = M / max_rows, rem = M - n_full * max_rows;
+    return n_full + ((rem > 0 && !(n_full > 0 && rem <= tail_rows)) ? 1 : 0);
+}
+__device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, int rb) {
+    return rb == n_rb - 1 ? M - rb * max_rows : max_rows;
+}
+
 // Requests are ordered by the estimated duration of their items, longest first, so the CTAs that
 // start last are the short ones (the hardware hands items to SMs in index order as SMs free up).
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
@@ -199,7 +205,6 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
     __shared__ int total_s, tail_s, w_tc_s, w_mma_s;
     const int tid = threadIdx.x, nthr = blockDim.x;   // 256 threads for small batches: cheaper barriers
     dcut_pdl_wait();
-    STAMP_MIN(0);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the item kernel's CTAs may take their SMs now
     const int group = a.n_q_heads / a.n_kv_heads;
     if (tid == 0) {
@@ -215,10 +220,11 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
         const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
         local += pages;
         const int M = (d + 1) * group;
-        const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
-        const int tc_rb = (a.max_item_rows >= a.tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= a.tc_min_rows) ? 1 : 0);
+        const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
+        int tc_rb = 0;
+        for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= a.tc_min_rows ? 1 : 0;
         w_tc += pages * tc_rb;
-        w_mma += pages * (n_full + (rem > 0 ? 1 : 0) - tc_rb);
+        w_mma += pages * (n_rb - tc_rb);
     }
     if (local) atomicAdd(&total_s, local);
     if (w_tc) atomicAdd(&w_tc_s, w_tc);
@@ -292,9 +298,9 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             // row blocks of the query tile: full blocks of max_item_rows rows and one remainder; each goes to the
             // tcgen05 queue or to the warp-level queue by its number of rows
             const int M = (d + 1) * group;
-            const int n_full = M / a.max_item_rows, rem = M - n_full * a.max_item_rows;
-            const int tc_rb = (a.max_item_rows >= tc_min_rows ? n_full : 0) + ((rem > 0 && rem >= tc_min_rows) ? 1 : 0);
-            const int n_rb = n_full + (rem > 0 ? 1 : 0);
+            const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
+            int tc_rb = 0;
+            for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= tc_min_rows ? 1 : 0;
             my_tc += nc * a.n_kv_heads * tc_rb;
             my_mma += nc * a.n_kv_heads * (n_rb - tc_rb);
             if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
@@ -316,9 +322,6 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
         a.plan[5] = overflow ? 0 : n_tc;     // items [0, n_tc): tcgen05 queue; [n_tc, n_items): warp-level queue
         a.plan[8] = 0;                       // next item of the tcgen05 queue (claimed by the CTAs of the item kernel)
         a.plan[9] = overflow ? 0 : n_tc;     // next item of the warp-level queue
-#ifdef DCUT_PROFILE_STAMPS
-        atomicMax(&g_attn_stamps[1], gtime());
-#endif
         if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
     }
     if (overflow) return;
@@ -336,13 +339,13 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
             const int M = (d + 1) * group;
             a.req_part[2 * i] = row_off;
             a.req_part[2 * i + 1] = nc;
-            // a query tile above max_item_rows rows (head_dim 128: the 128 lanes of tensor memory) is cut into row
-            // blocks, each its own item over the same pages
-            const int n_rb = (M + a.max_item_rows - 1) / a.max_item_rows;
+            // a query tile above max_item_rows (+ tail_rows) rows is cut into row blocks, each its own item over the
+            // same pages
+            const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
             for (int c = 0; c < nc; ++c)
                 for (int h = 0; h < a.n_kv_heads; ++h)
                     for (int rb = 0; rb < n_rb; ++rb) {
-                        const int row0 = rb * a.max_item_rows, rows = min(a.max_item_rows, M - row0);
+                        const int row0 = rb * a.max_item_rows, rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
                         AttnItem it;
                         it.req = i;
                         it.kv_head = h;
@@ -382,10 +385,21 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
 // Both MMAs therefore stream only K and V from shared memory.  Warp 0: TMA producer (lanes 0-3 look up the
 // group's pages, one elected lane issues its loads), warp 1: MMA issuer and tensor-memory owner, warps 2-5 and
 // 6-9: the two softmax teams, which also write the output.
+//   tail rows   a query tile of 129..144 rows (8 q heads per kv head at depth 16: 136) does not fit the 128 lanes of
+//                 tensor memory.  Cutting it into two items would stream the request's K/V twice; instead the item
+//                 keeps all its rows and warps 10-11 take rows 128.. as one m16 tile of warp-level MMAs
+//                 (mma.sync, as in the warp-level phase) on the very pages the ring holds for the tcgen05 MMAs: the
+//                 two warps take the item's pages alternately and merge their (m, l, O) at the end of the item.  A
+//                 ring stage is released by three arrivals: the commit of its last PV MMA and the two tail warps
+//                 (which arrive as soon as the stage is full when the item has no tail rows).
 constexpr int kTcGroupStages = 6;                  // ring of page groups (192 KB in flight)
 constexpr int kTcSBufs = 3;                        // S/P buffers in tensor memory: groups in flight between QK^T and PV
 constexpr int kTcSoftmaxThreads = 256;             // two teams of 128: one thread per row and team
-static_assert(kThreads == 64 + kTcSoftmaxThreads, "roles of the tcgen05 phase");
+constexpr int kTcTailWarps = 2;                    // warps 10, 11: query rows 128..143 of an item, by warp-level MMA
+constexpr int kTcTailRows = 16;                    // one m16 tile
+constexpr int kTcTailStride = 128 + 8;             // floats per row of the tail warps' merge buffer
+constexpr int kTcTailBytes = (kTcTailRows * kTcTailStride + kTcTailRows * 2) * 4;
+static_assert(kThreads == 64 + kTcSoftmaxThreads + 32 * kTcTailWarps, "roles of the tcgen05 phase");
 constexpr int kTcPageBytes = kPage * 128 * 2;      // 4 KB: one K or V page tile
 constexpr int kTcGroupBytes = 8 * kTcPageBytes;    // K of 4 pages (16 KB, [half][64 rows][64]) + V of 4 pages
 constexpr int kTcRingBytes = kTcGroupStages * kTcGroupBytes;
@@ -906,8 +920,8 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
 // current item is still being finished; only Q and O (single-buffered in tensor memory) serialise at an item boundary,
 // through the q_ready and o_free barriers.
 __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtensorMap& v_map, const AttnArgs& a,
-                                         unsigned char* ring, Ctrl* c, float (*xm)[128], float (*xl)[128],
-                                         int* counter, int end) {
+                                         unsigned char* ring, float* tail_buf, Ctrl* c, float (*xm)[128],
+                                         float (*xl)[128], int* counter, int end) {
     constexpr int kPhase = 0;
     const uint32_t full_bar = smem_u32(c->ring_full), empty_bar = smem_u32(c->ring_empty);
     const uint32_t s_full = smem_u32(c->s_full), p_full = smem_u32(c->p_full), pv_done = smem_u32(c->pv_done);
@@ -935,18 +949,15 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             const int n_groups = (n_pages + 3) >> 2;
             const int* bt = a.block_table + (size_t)item.req * a.block_table_stride + item.page_begin;
             int next = (lane < 4 && lane < n_pages) ? bt[lane] : 0;
-            TCP(long long t_we = 0; long long t_all = clock64();)
             for (int g = 0; g < n_groups; ++g) {
                 int page_id = next;
                 const int pn = 4 * (g + 1) + lane;
                 if (lane < 4 && pn < n_pages) next = bt[pn];
                 const int gc = G0 + g, gs = gc % kTcGroupStages, use = gc / kTcGroupStages;
-                TCP(long long c0 = clock64();)
                 if (use > 0 && !__all_sync(0xffffffffu, mbar_wait(empty_bar + 8 * gs, (use - 1) & 1, &c->abort))) {
                     failed = true;
                     break;
                 }
-                TCP(t_we += clock64() - c0;)
                 const int np = min(4, n_pages - 4 * g);
                 if (lane < np && (page_id < 0 || page_id >= a.num_pages)) {
                     atomicExch(a.status, DCUT_DEV_BAD_PAGE);
@@ -970,7 +981,6 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                 }
                 __syncwarp();
             }
-            TCP(if (blockIdx.x == 0 && lane == 0) printf("producer: groups %d total %lld wait_empty %lld\n", n_groups, clock64() - t_all, t_we);)
             if (failed || ABORTED(c)) {
                 failed = true;
                 break;
@@ -1074,7 +1084,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             }
             if (idx < 0) break;
             const int q0 = item.q0, ctx_len = item.ctx_len, kvh = item.kv_head;
-            const int row0 = item.pad[1], M = item.pad[2];   // this item's rows of the request's query tile
+            const int row0 = item.pad[1], M = min(item.pad[2], 128);   // this item's rows of the request's query tile (rows past 128: tail warps)
             const int n_pages = item.page_end - item.page_begin;
             const int n_groups = (n_pages + 3) >> 2;
             {
@@ -1233,6 +1243,405 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             sched_release(c, kPhase, n);
             G0 += n_groups;
         }
+    } else if (warp < 2 + kTcSoftmaxThreads / 32 + kTcTailWarps) {
+        // ---------------------------------------------------------------- tail rows (128 .. 143 of the item)
+        // One m16 tile by warp-level MMA on the staged pages; warp tw takes the item's pages p with p mod 2 = tw.
+        // Both warps walk every group of every item, because every stage of the ring waits for their arrival.
+        const int tw = warp - (2 + kTcSoftmaxThreads / 32);
+        const float cs = a.scale_log2;
+        float* t_o = tail_buf;
+        float* t_ml = tail_buf + kTcTailRows * kTcTailStride;
+        const int r_lo = lane >> 2, c0 = (lane & 3) << 1;
+        const int kmat = lane >> 3;
+        const int k_tok = ((kmat >> 1) << 3) + (lane & 7), k_chunk = kmat & 1;
+        const int v_tok = ((kmat & 1) << 3) + (lane & 7), v_chunk = kmat >> 1;
+        for (int n = 0;; ++n) {
+            const int idx = sched_wait(c, kPhase, n, item);
+            if (idx == -2) failed = true;
+            // also: warp 10 has read what warp 11 left in the merge buffer for the previous item
+            if (bar_any(6, 32 * kTcTailWarps, failed || ABORTED(c))) {
+                failed = true;
+                break;
+            }
+            if (idx < 0) break;
+            const int q0 = item.q0, ctx_len = item.ctx_len, kvh = item.kv_head;
+            const int row0 = item.pad[1] + 128, M = item.pad[2] - 128;   // the tail's first row within the request's tile, its rows
+            const int n_pages = item.page_end - item.page_begin;
+            const int n_groups = (n_pages + 3) >> 2;
+            const bool has_tail = M > 0;
+            uint32_t qf[8][4];
+            float o[16][4];
+            float m_run[2] = {-INFINITY, -INFINITY};
+            float l_run[2] = {0.0f, 0.0f};
+            int jmax_lo = 0, jmax_hi = 0;
+            // A tail of at most 8 rows (8 q heads per kv head at depth 16) runs with the operands swapped: S^T = K Q^T and
+            // O^T = V^T P^T, the tail rows as the MMA's n = 8 and the keys / head dimension as its m = 16, which takes half
+            // the MMAs of a 16-row tile that is half padding.
+            const bool swapped = has_tail && M <= 8;
+            if (swapped) {
+                // B fragments of Q^T: lane 4 g + t holds row g, head-dim elements 2 t, 2 t + 1 (+ 8) of every k-step
+                const int R = row0 + min(r_lo, M - 1), tq = R / group;
+                const uint32_t* qr = reinterpret_cast<const uint32_t*>(a.q + ((size_t)(q0 + tq) * a.n_q_heads + kvh * group + (R - tq * group)) * 128);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    qf[ks][0] = qr[ks * 8 + (lane & 3)];
+                    qf[ks][1] = qr[ks * 8 + 4 + (lane & 3)];
+                }
+                // the two rows whose scores this lane holds: 2 t and 2 t + 1
+                jmax_lo = ctx_len + (row0 + min(c0, M - 1)) / group;
+                jmax_hi = ctx_len + (row0 + min(c0 + 1, M - 1)) / group;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
+            } else if (has_tail) {
+                // A fragments straight from global memory (16 rows of 256 bytes, once per item); rows past the tail
+                // repeat its last row and are never written
+                const int R_lo = row0 + min(r_lo, M - 1), R_hi = row0 + min(r_lo + 8, M - 1);
+                const int t_l = R_lo / group, t_h = R_hi / group;
+                const uint32_t* q_l = reinterpret_cast<const uint32_t*>(a.q + ((size_t)(q0 + t_l) * a.n_q_heads + kvh * group + (R_lo - t_l * group)) * 128);
+                const uint32_t* q_h = reinterpret_cast<const uint32_t*>(a.q + ((size_t)(q0 + t_h) * a.n_q_heads + kvh * group + (R_hi - t_h * group)) * 128);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    qf[ks][0] = q_l[ks * 8 + (lane & 3)];
+                    qf[ks][1] = q_h[ks * 8 + (lane & 3)];
+                    qf[ks][2] = q_l[ks * 8 + 4 + (lane & 3)];
+                    qf[ks][3] = q_h[ks * 8 + 4 + (lane & 3)];
+                }
+                jmax_lo = ctx_len + t_l;     // query token t sees cache positions j <= ctx_len + t
+                jmax_hi = ctx_len + t_h;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
+            }
+            // NP pages (8 KB apart in the stage: this warp's page of the group and the one two further on) = 16 NP keys.
+            // The ldmatrix loads run one step ahead of the MMAs that use them (a warp issues in order, and with two
+            // tail warps per SM nothing else hides the shared-memory latency).
+            auto tail_step = [&](auto npc, uint32_t k_base, int pg) {
+                constexpr int NP = decltype(npc)::value, NT = 2 * NP;
+                float s[NT][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) s[nt][e] = 0.0f;
+                {
+                    uint32_t kf[2][NP][4];
+#pragma unroll
+                    for (int pp = 0; pp < NP; ++pp) ldmatrix_x4(k_base + pp * 2 * kTcPageBytes + tile_off_k4(k_tok, k_chunk), kf[0][pp]);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        if (ks + 1 < 8) {
+#pragma unroll
+                            for (int pp = 0; pp < NP; ++pp)
+                                ldmatrix_x4(k_base + pp * 2 * kTcPageBytes + tile_off_k4(k_tok, 2 * (ks + 1) + k_chunk), kf[(ks + 1) & 1][pp]);
+                        }
+#pragma unroll
+                        for (int pp = 0; pp < NP; ++pp) {
+                            mma_bf16_pure(s[2 * pp], qf[ks], kf[ks & 1][pp][0], kf[ks & 1][pp][1]);
+                            mma_bf16_pure(s[2 * pp + 1], qf[ks], kf[ks & 1][pp][2], kf[ks & 1][pp][3]);
+                        }
+                    }
+                }
+                if ((pg + 2 * (NP - 1)) * kPage + kPage - 1 > ctx_len) {   // only pages that reach past the cached context hold hidden keys
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int j0 = (pg + 2 * (nt >> 1)) * kPage + (nt & 1) * 8 + c0;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (j0 + (e & 1) > ((e < 2) ? jmax_lo : jmax_hi)) s[nt][e] = -INFINITY;
+                    }
+                }
+                float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    mx[0] = fmaxf(mx[0], fmaxf(s[nt][0], s[nt][1]));
+                    mx[1] = fmaxf(mx[1], fmaxf(s[nt][2], s[nt][3]));
+                }
+                float alpha[2], mc[2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+                    mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+                    const float m_new = fmaxf(m_run[r], mx[r]);
+                    const float msafe = (m_new == -INFINITY) ? 0.0f : m_new;
+                    alpha[r] = fast_exp2((m_run[r] - msafe) * cs);
+                    mc[r] = msafe * cs;
+                    m_run[r] = m_new;
+                }
+                // the first V fragments travel while the exponentials are computed
+                const uint32_t v_base = k_base + 4 * kTcPageBytes;
+                constexpr int NV = 8 * NP;               // V fragment loads of the step: (page pp, 16 columns jj)
+                uint32_t vf[3][4];
+                ldmatrix_x4_trans(v_base + tile_off(v_tok, v_chunk), vf[0]);
+                ldmatrix_x4_trans(v_base + tile_off(v_tok, 2 + v_chunk), vf[1]);
+                float sum[2] = {0.0f, 0.0f};
+                uint32_t pf[NP][4];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const float p0 = fast_exp2(fmaf(s[nt][0], cs, -mc[0])), p1 = fast_exp2(fmaf(s[nt][1], cs, -mc[0]));
+                    const float p2 = fast_exp2(fmaf(s[nt][2], cs, -mc[1])), p3 = fast_exp2(fmaf(s[nt][3], cs, -mc[1]));
+                    sum[0] += p0 + p1;
+                    sum[1] += p2 + p3;
+                    pf[nt >> 1][2 * (nt & 1)] = pack_bf16(p0, p1);
+                    pf[nt >> 1][2 * (nt & 1) + 1] = pack_bf16(p2, p3);
+                }
+                l_run[0] = l_run[0] * alpha[0] + sum[0];
+                l_run[1] = l_run[1] * alpha[1] + sum[1];
+                if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
+#pragma unroll
+                    for (int jo = 0; jo < 16; ++jo) {
+                        o[jo][0] *= alpha[0];
+                        o[jo][1] *= alpha[0];
+                        o[jo][2] *= alpha[1];
+                        o[jo][3] *= alpha[1];
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int pp = i >> 3, jj = i & 7;
+                    if (i + 2 < NV) {
+                        const int pn = (i + 2) >> 3, jn = (i + 2) & 7;
+                        ldmatrix_x4_trans(v_base + pn * 2 * kTcPageBytes + tile_off(v_tok, 2 * jn + v_chunk), vf[(i + 2) % 3]);
+                    }
+                    mma_bf16_pure(o[2 * jj], pf[pp], vf[i % 3][0], vf[i % 3][1]);
+                    mma_bf16_pure(o[2 * jj + 1], pf[pp], vf[i % 3][2], vf[i % 3][3]);
+                }
+            };
+            // The same step with the operands swapped (tails of at most 8 rows).  S^T[16 keys, 8 rows] per page: A = the K
+            // page (keys x head dim, as stored), B = Q^T; this lane holds keys g and g + 8 of rows 2 t and 2 t + 1, so
+            // a row's maximum is taken over the lanes of equal t.  P^T becomes the B operand of O^T += V^T P^T through
+            // movmatrix (key-major pairs -> row-major pairs); A = the V page read transposed (head dim x keys).
+            // o[mt] holds O^T: head-dim elements 16 mt + g and + 8 of rows 2 t and 2 t + 1.
+            auto tail_step8 = [&](auto npc, uint32_t k_base, int pg) {
+                constexpr int NP = decltype(npc)::value;   // consecutive pages of the group
+                constexpr int DK = 4, DV = 6;              // fragment loads in flight ahead of the MMAs
+                float s[NP][4];
+#pragma unroll
+                for (int pp = 0; pp < NP; ++pp)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) s[pp][e] = 0.0f;
+                {
+                    uint32_t kf[DK][NP][4];
+#pragma unroll
+                    for (int ks = 0; ks < DK - 1; ++ks)
+#pragma unroll
+                        for (int pp = 0; pp < NP; ++pp) ldmatrix_x4(k_base + pp * kTcPageBytes + tile_off_k4(v_tok, 2 * ks + v_chunk), kf[ks][pp]);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        if (ks + DK - 1 < 8) {
+#pragma unroll
+                            for (int pp = 0; pp < NP; ++pp)
+                                ldmatrix_x4(k_base + pp * kTcPageBytes + tile_off_k4(v_tok, 2 * (ks + DK - 1) + v_chunk), kf[(ks + DK - 1) % DK][pp]);
+                        }
+#pragma unroll
+                        for (int pp = 0; pp < NP; ++pp) mma_bf16_pure(s[pp], kf[ks % DK][pp], qf[ks][0], qf[ks][1]);
+                    }
+                }
+                if ((pg + NP - 1) * kPage + kPage - 1 > ctx_len) {
+#pragma unroll
+                    for (int pp = 0; pp < NP; ++pp) {
+                        const int j0 = (pg + pp) * kPage + r_lo;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (j0 + ((e >> 1) << 3) > ((e & 1) ? jmax_hi : jmax_lo)) s[pp][e] = -INFINITY;
+                    }
+                }
+                float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+                for (int pp = 0; pp < NP; ++pp) {
+                    mx[0] = fmaxf(mx[0], fmaxf(s[pp][0], s[pp][2]));
+                    mx[1] = fmaxf(mx[1], fmaxf(s[pp][1], s[pp][3]));
+                }
+#pragma unroll
+                for (int sh = 4; sh < 32; sh <<= 1) {
+                    mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], sh));
+                    mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], sh));
+                }
+                float alpha[2], mc[2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const float m_new = fmaxf(m_run[r], mx[r]);
+                    const float msafe = (m_new == -INFINITY) ? 0.0f : m_new;
+                    alpha[r] = fast_exp2((m_run[r] - msafe) * cs);
+                    mc[r] = msafe * cs;
+                    m_run[r] = m_new;
+                }
+                // the first V fragments travel while the exponentials are computed
+                const uint32_t v_base = k_base + 4 * kTcPageBytes;
+                constexpr int NV = 8 * NP;               // V fragment loads of the step: (page pp, 16 head-dim elements mt)
+                uint32_t vf[DV][4];
+#pragma unroll
+                for (int i = 0; i < DV - 1; ++i) ldmatrix_x4_trans(v_base + (i >> 3) * kTcPageBytes + tile_off(k_tok, 2 * (i & 7) + k_chunk), vf[i]);
+                float sum[2] = {0.0f, 0.0f};
+                uint32_t pb[NP][2];
+#pragma unroll
+                for (int pp = 0; pp < NP; ++pp) {
+                    const float p0 = fast_exp2(fmaf(s[pp][0], cs, -mc[0])), p1 = fast_exp2(fmaf(s[pp][1], cs, -mc[1]));
+                    const float p2 = fast_exp2(fmaf(s[pp][2], cs, -mc[0])), p3 = fast_exp2(fmaf(s[pp][3], cs, -mc[1]));
+                    sum[0] += p0 + p2;
+                    sum[1] += p1 + p3;
+                    pb[pp][0] = movmatrix_trans(pack_bf16(p0, p1));      // keys 0-7: (row g; keys 2 t, 2 t + 1)
+                    pb[pp][1] = movmatrix_trans(pack_bf16(p2, p3));      // keys 8-15
+                }
+                l_run[0] = l_run[0] * alpha[0] + sum[0];                 // this lane's keys only; summed over the lanes at the end
+                l_run[1] = l_run[1] * alpha[1] + sum[1];
+                if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
+#pragma unroll
+                    for (int mt = 0; mt < 8; ++mt) {
+                        o[mt][0] *= alpha[0];
+                        o[mt][1] *= alpha[1];
+                        o[mt][2] *= alpha[0];
+                        o[mt][3] *= alpha[1];
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int pp = i >> 3, mt = i & 7;
+                    if (i + DV - 1 < NV) {
+                        const int in = i + DV - 1;
+                        ldmatrix_x4_trans(v_base + (in >> 3) * kTcPageBytes + tile_off(k_tok, 2 * (in & 7) + k_chunk), vf[in % DV]);
+                    }
+                    mma_bf16_pure(o[mt], vf[i % DV], pb[pp][0], pb[pp][1]);
+                }
+            };
+            for (int g = 0; g < n_groups; ++g) {
+                const int gc = G0 + g, gs = gc % kTcGroupStages;
+                if (!__all_sync(0xffffffffu, mbar_wait(full_bar + 8 * gs, (gc / kTcGroupStages) & 1, &c->abort))) {
+                    failed = true;
+                    break;
+                }
+                if (swapped) {
+                    const int np = min(4, n_pages - 4 * g);
+                    const uint32_t k_grp = smem_u32(ring + gs * kTcGroupBytes);
+                    // the warps take the groups alternately, a whole group (64 keys) per softmax step
+                    if ((gc & 1) == tw) {
+                        if (np == 4) tail_step8(std::integral_constant<int, 4>(), k_grp, item.page_begin + 4 * g);
+                        else
+                            for (int j = 0; j < np; ++j) tail_step8(std::integral_constant<int, 1>(), k_grp + j * kTcPageBytes, item.page_begin + 4 * g + j);
+                    }
+                } else if (has_tail) {
+                    const int np = min(4, n_pages - 4 * g);
+                    const uint32_t k_grp = smem_u32(ring + gs * kTcGroupBytes);
+                    // this warp's pages of the group, tw and tw + 2, go through one softmax step together: twice as
+                    // many independent MMA chains per step and half as many steps
+                    if (tw + 2 < np) tail_step(std::integral_constant<int, 2>(), k_grp + tw * kTcPageBytes, item.page_begin + 4 * g + tw);
+                    else if (tw < np) tail_step(std::integral_constant<int, 1>(), k_grp + tw * kTcPageBytes, item.page_begin + 4 * g + tw);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar + 8 * gs);     // this warp is done with the group's stage
+            }
+            if (failed) c->abort = 1;
+            if (swapped) {
+                // both warps leave (m, l, O) in the merge buffer: [warp][row][head dim]
+#pragma unroll
+                for (int sh = 4; sh < 32; sh <<= 1) {
+                    l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], sh);
+                    l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], sh);
+                }
+                float* mo = t_o + tw * 8 * kTcTailStride;
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    mo[c0 * kTcTailStride + 16 * mt + r_lo] = o[mt][0];
+                    mo[(c0 + 1) * kTcTailStride + 16 * mt + r_lo] = o[mt][1];
+                    mo[c0 * kTcTailStride + 16 * mt + r_lo + 8] = o[mt][2];
+                    mo[(c0 + 1) * kTcTailStride + 16 * mt + r_lo + 8] = o[mt][3];
+                }
+                if (r_lo == 0) {
+                    t_ml[(tw * 8 + c0) * 2] = m_run[0];
+                    t_ml[(tw * 8 + c0) * 2 + 1] = l_run[0];
+                    t_ml[(tw * 8 + c0 + 1) * 2] = m_run[1];
+                    t_ml[(tw * 8 + c0 + 1) * 2 + 1] = l_run[1];
+                }
+            } else if (has_tail) {
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
+                    l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
+                }
+                if (tw == 1) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        *reinterpret_cast<float2*>(t_o + r_lo * kTcTailStride + j * 8 + c0) = make_float2(o[j][0], o[j][1]);
+                        *reinterpret_cast<float2*>(t_o + (r_lo + 8) * kTcTailStride + j * 8 + c0) = make_float2(o[j][2], o[j][3]);
+                    }
+                    if ((lane & 3) == 0) {
+                        t_ml[2 * r_lo] = m_run[0];
+                        t_ml[2 * r_lo + 1] = l_run[0];
+                        t_ml[2 * (r_lo + 8)] = m_run[1];
+                        t_ml[2 * (r_lo + 8) + 1] = l_run[1];
+                    }
+                }
+            }
+            if (bar_any(6, 32 * kTcTailWarps, failed)) {
+                failed = true;
+                break;
+            }
+            if (swapped) {
+                // the 64 threads merge the two warps' rows and write them out, four head-dim elements at a time
+                for (int i = (warp - (2 + kTcSoftmaxThreads / 32)) * 32 + lane; i < M * 32; i += 32 * kTcTailWarps) {
+                    const int rr = i >> 5, c4 = (i & 31) << 2;
+                    const float m0 = t_ml[rr * 2], l0 = t_ml[rr * 2 + 1], m1 = t_ml[(8 + rr) * 2], l1 = t_ml[(8 + rr) * 2 + 1];
+                    const float m_all = fmaxf(m0, m1);
+                    const float w0 = m0 == -INFINITY ? 0.0f : fast_exp2((m0 - m_all) * cs);
+                    const float w1 = m1 == -INFINITY ? 0.0f : fast_exp2((m1 - m_all) * cs);
+                    const float l_all = l0 * w0 + l1 * w1;
+                    const float inv = l_all > 0.0f ? 1.0f / l_all : 0.0f;
+                    const float f0 = w0 * inv, f1 = w1 * inv;
+                    const float4 v0 = *reinterpret_cast<const float4*>(t_o + rr * kTcTailStride + c4);
+                    const float4 v1 = *reinterpret_cast<const float4*>(t_o + (8 + rr) * kTcTailStride + c4);
+                    const float4 v = make_float4(v0.x * f0 + v1.x * f1, v0.y * f0 + v1.y * f1, v0.z * f0 + v1.z * f1, v0.w * f0 + v1.w * f1);
+                    const int R = row0 + rr;
+                    const int t = R / group, hl = R - t * group;
+                    const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+                    const float lse_nat = l_all > 0.0f ? (m_all * cs + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+                    if (item.n_chunks == 1) {
+                        *reinterpret_cast<uint2*>(a.out + orow * 128 + c4) = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+                        if (a.lse && c4 == 0) a.lse[orow] = lse_nat;
+                    } else {
+                        const size_t prow = (size_t)item.part_row + 128 + rr;
+                        *reinterpret_cast<float4*>(a.part_o + prow * 128 + c4) = v;
+                        if (c4 == 0) a.part_lse[prow] = lse_nat;
+                    }
+                }
+            } else if (has_tail && tw == 0) {
+                // each lane merges the elements it holds with the ones the same lane of the other warp held
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+                    const int rr = r_lo + 8 * r;
+                    const float m_o = t_ml[2 * rr], l_o = t_ml[2 * rr + 1];
+                    const float m_all = fmaxf(m_run[r], m_o);
+                    const float w_s = m_run[r] == -INFINITY ? 0.0f : fast_exp2((m_run[r] - m_all) * cs);
+                    const float w_o = m_o == -INFINITY ? 0.0f : fast_exp2((m_o - m_all) * cs);
+                    const float l_all = l_run[r] * w_s + l_o * w_o;
+                    const float inv = l_all > 0.0f ? 1.0f / l_all : 0.0f;
+                    const float f_s = w_s * inv, f_o = w_o * inv;
+                    if (rr < M) {
+                        const int R = row0 + rr;
+                        const int t = R / group, hl = R - t * group;
+                        const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+                        const float lse_nat = l_all > 0.0f ? (m_all * cs + log2f(l_all)) * 0.6931471805599453f : -INFINITY;
+                        const float* po = t_o + rr * kTcTailStride + c0;
+                        if (item.n_chunks == 1) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float2 v = *reinterpret_cast<const float2*>(po + j * 8);
+                                *reinterpret_cast<uint32_t*>(a.out + orow * 128 + j * 8 + c0) =
+                                    pack_bf16(o[j][2 * r] * f_s + v.x * f_o, o[j][2 * r + 1] * f_s + v.y * f_o);
+                            }
+                            if (a.lse && (lane & 3) == 0) a.lse[orow] = lse_nat;
+                        } else {
+                            const size_t prow = (size_t)item.part_row + 128 + rr;
+                            float* pd = a.part_o + prow * 128 + c0;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float2 v = *reinterpret_cast<const float2*>(po + j * 8);
+                                *reinterpret_cast<float2*>(pd + j * 8) = make_float2(o[j][2 * r] * f_s + v.x * f_o, o[j][2 * r + 1] * f_s + v.y * f_o);
+                            }
+                            if ((lane & 3) == 0) a.part_lse[prow] = lse_nat;
+                        }
+                    }
+                }
+            }
+            sched_release(c, kPhase, n);
+            G0 += n_groups;
+        }
     }
     if (failed) {
         atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
@@ -1244,7 +1653,9 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
 template <int DH>
 constexpr int kDataBytes = (DH == 128 && kTcRingBytes > MmaSmem<DH>::kTotal) ? kTcRingBytes : MmaSmem<DH>::kTotal;
 template <int DH>
-constexpr int kSmemBytes = kDataBytes<DH> + 1024 /* alignment slack */ + 1024 /* control block */;
+constexpr int kTailPad = DH == 128 ? ((kTcTailBytes + 1023) / 1024) * 1024 : 0;   // merge buffer of the tcgen05 phase's tail warps
+template <int DH>
+constexpr int kSmemBytes = kDataBytes<DH> + kTailPad<DH> + 1024 /* alignment slack */ + 1024 /* control block */;
 static_assert(sizeof(Ctrl) <= 1024, "control block");
 
 // Persistent kernel: one CTA per SM takes work items from two queues, first the tcgen05-path items, then the
@@ -1255,14 +1666,14 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
                  const __grid_constant__ CUtensorMap k2_map, AttnArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    Ctrl* c = reinterpret_cast<Ctrl*>(smem + kDataBytes<DH>);
+    Ctrl* c = reinterpret_cast<Ctrl*>(smem + kDataBytes<DH> + kTailPad<DH>);
     __shared__ float xm[2][128];       // [team][row]: the teams' running maxima at the end of an item (tcgen05 phase)
     __shared__ float xl[2][128];       // [team][row]: their running sums
     const int warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) {
             mbar_init(smem_u32(&c->ring_full[s]), 1);    // tcgen05 phase: one arrival (with the group's byte count)
-            mbar_init(smem_u32(&c->ring_empty[s]), 1);
+            mbar_init(smem_u32(&c->ring_empty[s]), 1 + kTcTailWarps);   // the commit of the stage's last MMA + the tail warps
         }
         for (int b = 0; b < kTcSBufs; ++b) {
             mbar_init(smem_u32(&c->s_full[b]), 1);
@@ -1274,7 +1685,7 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&c->sched_full[0][s]), 1);
             mbar_init(smem_u32(&c->sched_full[1][s]), 1);
-            mbar_init(smem_u32(&c->sched_empty[0][s]), 1 + kTcSoftmaxThreads / 32);   // MMA warp + softmax warps
+            mbar_init(smem_u32(&c->sched_empty[0][s]), 1 + kTcSoftmaxThreads / 32 + kTcTailWarps);   // MMA warp + softmax warps + tail warps
             mbar_init(smem_u32(&c->sched_empty[1][s]), kMmaWarps);
         }
         mbar_init(smem_u32(&c->geom_a), kMmaWarps + 1);
@@ -1292,12 +1703,10 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
     tc_fence_after();
     // launched with programmatic stream serialization: everything above overlaps the plan kernel; nothing it writes
     // is read before this wait
-    STAMP_MIN(2);
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    STAMP_MIN(6);
     const int n_items = a.plan[0], n_tc = a.plan[5];
     if (DH == 128 && n_tc > 0) {
-        tc_phase(k2_map, v_map, a, smem, c, xm, xl, a.plan + 8, n_tc);
+        tc_phase(k2_map, v_map, a, smem, reinterpret_cast<float*>(smem + kDataBytes<DH>), c, xm, xl, a.plan + 8, n_tc);
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
@@ -1306,7 +1715,6 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may take this SM
     tc_fence_before();
     __syncthreads();
-    STAMP_MAX(3);
     if (DH == 128 && warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c->tmem_base), "n"(kTcCols) : "memory");
@@ -1331,10 +1739,8 @@ template <int DH>
 __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
     // grid: x = request * (gamma_max + 1) + block position t, y = group of blockDim.x / 32 q heads; warp = one head.
     // Launched with programmatic stream serialization (see attn_item_kernel).
-    STAMP_MIN(4);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    STAMP_MAX(5);
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
         // the item kernel has drained both queues: rewind them, so that the same plan can serve another launch over
         // the same batch (the layers of one model forward)
@@ -1442,6 +1848,8 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
     {
         const char* env = getenv("DCUT_ATTN_TC_MIN_ROWS");   // query rows from which an item goes to the tcgen05 kernel
         ctx->attn_tc_min_rows = env ? atoi(env) : 17;
+        env = getenv("DCUT_ATTN_TAIL_ROWS");     // 0: a query tile above 128 rows becomes two items (experiments)
+        ctx->attn_tail_rows = env ? (atoi(env) > 0 ? kTcTailRows : 0) : kTcTailRows;
     }
     e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS);
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn plan)");
@@ -1493,6 +1901,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     pa.status = ctx->d_status;
     pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
     pa.max_item_rows = 128;
+    pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? ctx->attn_tail_rows : 0;
     pa.max_items = ctx->max_items;
     pa.part_rows_cap = ctx->part_rows_cap;
     pa.items = ctx->d_items;

@@ -108,3 +108,37 @@ def test_unaligned_logits_base():
         al, bo, _, _ = ctx.accept(view, dev(np.zeros((T, 1), np.int32)), dev(cu), T)
         assert np.array_equal(bo.cpu().numpy(), ref.bonus)
     ctx.close()
+
+
+def _past_cap_case():
+    """B = 4 requests of 3 rows each (cu_q[B] = 12) handed over with T_cap = 8: the caller's contract is broken.
+    Rows 0..7 exist.  Request 2 has rows 6, 7 left (of 6, 7, 8); request 3 has none."""
+    V, g = 300, 2
+    rng = np.random.default_rng(11)
+    x = torch.from_numpy(rng.standard_normal((12, V), dtype=np.float32)).to(torch.bfloat16)
+    draft = rng.integers(0, V, size=(4, g)).astype(np.int32)
+    for i in range(4):
+        for t in range(g):
+            x[3 * i + t, draft[i, t]] = 8.0                  # every draft matches wherever its row is looked at
+    cu = np.array([0, 3, 6, 9, 12], np.int32)
+    am = x.float().argmax(dim=1).numpy()
+    want_len = np.array([2, 2, 1, 0], np.int32)             # request 2: row 6 matches, row 7 is its last existing row
+    want_bonus = np.array([am[2], am[5], am[7], 0], np.int32)
+    return x, draft, cu, g, want_len, want_bonus
+
+
+def test_cu_q_past_T_cap_is_clamped_and_reported():
+    """cu_q[B] > T_cap: rows at or past T_cap are neither read nor cleared, the outputs are defined, and the
+    device status word reports code 7.  (Nothing faults: the logits buffer does hold 12 rows.)"""
+    x, draft, cu, g, want_len, want_bonus = _past_cap_case()
+    cfg = wl.custom_config(B=4, gamma=g, vocab=x.shape[1])
+    ctx = make_ctx(cfg, n_q_heads=0)
+    al, bo, toks, total = ctx.accept(dev(x), dev(draft), dev(cu), 8)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 7
+    assert np.array_equal(al.cpu().numpy(), want_len) and np.array_equal(bo.cpu().numpy(), want_bonus)
+    assert int(total.item()) == int(want_len.sum()) + 4
+    # the context is still good and its scratch clean: a valid call right after gives the oracle's answer
+    _check(ctx, x, draft, cu, g, 12)
+    assert ctx.poll_device_status() == 0
+    ctx.close()

@@ -56,6 +56,27 @@ def test_mid_size_every_element(shape):
         _full_compare(cfg, sel, kv, depths)
 
 
+@pytest.mark.parametrize("shape,B,gamma,ctx_hi", [
+    (dict(n_q_heads=64, n_kv_heads=8, head_dim=128), 5, 16, 1500),     # few requests: cut into chunks, partial results merged
+    (dict(n_q_heads=64, n_kv_heads=8, head_dim=128), 40, 16, 400),     # many requests: whole requests per item
+    (dict(n_q_heads=16, n_kv_heads=2, head_dim=128), 24, 17, 700),     # 18 tokens x 8 heads = 144 rows: a full 16-row tail
+    (dict(n_q_heads=18, n_kv_heads=2, head_dim=128), 10, 15, 900),     # 9 heads per kv head: tails of 7 and 16 rows, ragged groups
+])
+def test_query_tiles_above_128_rows_every_element(shape, B, gamma, ctx_hi):
+    """A request whose (1 + d_i) x (q heads per kv head) query rows exceed the 128 rows of the tensor-memory tile
+    (8 heads per kv head at depth 16: 136 rows) stays ONE work item: rows 128.. are computed by the tail warps from
+    the same staged pages.  Depths straddle the boundary (127/128/129.. rows), every element against the oracle."""
+    cfg = wl.custom_config(B=B, gamma=gamma, ctx_lo=0, ctx_hi=ctx_hi, **shape)
+    sel = wl.select_inputs(cfg)
+    sel.ctx_lens[:3] = [0, 15, 16]
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    rng = np.random.default_rng(2)
+    mixed = rng.integers(max(0, gamma - 3), gamma + 1, cfg.B).astype(np.int32)
+    mixed[::5] = rng.integers(0, gamma + 1, len(mixed[::5]))
+    for depths in (np.full(cfg.B, gamma, np.int32), mixed):
+        _full_compare(cfg, sel, kv, depths)
+
+
 def test_unused_slots_are_never_read():
     cfg = wl.custom_config(B=6, gamma=16, n_q_heads=8, n_kv_heads=2, head_dim=128, ctx_lo=10, ctx_hi=300)
     sel = wl.select_inputs(cfg)
@@ -107,6 +128,7 @@ def test_b256_long_tail_sampled():
     kv = wl.paged_kv(cfg, sel.ctx_lens)
     _sampled_compare(cfg, sel, kv, _pruned_depths(cfg, sel), 160)
     _sampled_compare(cfg, sel, kv, np.full(cfg.B, cfg.gamma, np.int32), 96, seed=1)
+    _sampled_compare(cfg, sel, kv, np.zeros(cfg.B, np.int32), 96, seed=2)
 
 
 def test_repeated_runs_are_bit_identical():

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import dcut_oracle as orc
 from paper_2607_14647_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -38,7 +39,29 @@ def test_static_scratch_matches_context_scratch_on_two_calls_in_a_row():
         torch.cuda.synchronize()
         for g, w in zip(got, want):
             assert torch.equal(g, w)
+        ref = orc.accept(logits, sel.draft_ids, wl.cu_q_from_depths(depths), cfg.gamma)   # and both equal the oracle
+        assert np.array_equal(got[0].cpu().numpy(), ref.accept_len) and np.array_equal(got[1].cpu().numpy(), ref.bonus)
+        assert np.array_equal(got[2].cpu().numpy(), ref.out_tokens) and int(got[3].item()) == ref.n_accepted_total
     ctx.close()
+
+
+def test_rows_past_T_cap_are_left_alone():
+    """A cu_q that runs past T_cap breaks the caller's contract; the call must still stay inside the first T_cap
+    words of the shared array.  T_cap = 8 with cu_q[B] = 12: rows 8..11 are left out, the outputs are defined,
+    and a valid call right after (which would see any stray write to words 8..11) still matches the oracle."""
+    from paper_2607_14647_b200 import binding
+    from tests.test_gpu_accept import _past_cap_case
+    x, draft, cu, g, want_len, want_bonus = _past_cap_case()
+    i32 = dict(dtype=torch.int32, device="cuda")
+    d_x, d_draft, d_cu = x.cuda(), torch.from_numpy(draft).cuda(), torch.from_numpy(cu).cuda()
+    out = (torch.full((4,), -7, **i32), torch.full((4,), -7, **i32), torch.full((4, g + 1), -7, **i32), torch.full((1,), -7, **i32))
+    binding.accept_static(d_x, d_draft, d_cu, 8, *out)
+    torch.cuda.synchronize()
+    assert np.array_equal(out[0].cpu().numpy(), want_len) and np.array_equal(out[1].cpu().numpy(), want_bonus)
+    binding.accept_static(d_x, d_draft, d_cu, 12, *out)
+    torch.cuda.synchronize()
+    ref = orc.accept(x, draft, cu, g)
+    assert np.array_equal(out[0].cpu().numpy(), ref.accept_len) and np.array_equal(out[1].cpu().numpy(), ref.bonus)
 
 
 def test_rows_beyond_the_fixed_scratch_are_refused():
