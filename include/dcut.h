@@ -203,6 +203,20 @@ dcut_status dcut_layer_forward(dcut_ctx* ctx, const dcut_layer_weights* weights,
                                int T_cap, void* stream);
 
 /*
+ * Selection and the attention work list in one launch (Algorithm 1 hands the packed batch straight to the target
+ * forward; Appendix C folds the packing cost into verification).  The work list of dcut_verify_attn (how the requests'
+ * page lists are cut into items and in which order they run) depends on ctx_lens, cu_q, B and the context's shapes only.
+ * After dcut_enable_plan_in_select(ctx, 1), every dcut_select / dcut_select_causal call that is given ctx_lens also
+ * builds that list in the selector kernel's tail, for the batch it has just packed; the attention calls that follow
+ * (dcut_verify_attn, dcut_layer_forward, dcut_model_verify, any number of them) and are given the SAME cu_q and
+ * ctx_lens pointers and the same B use it and launch no work-list kernel of their own.  Contract: between such a
+ * select and those calls the caller changes neither the contents of cu_q nor of ctx_lens, and issues them on the same
+ * stream (or one ordered after it).  Any other attention call builds its own list, as before.  Results are identical
+ * either way (the list is the same).  Off by default; needs a context with attention shapes.
+ */
+dcut_status dcut_enable_plan_in_select(dcut_ctx* ctx, int on);
+
+/*
  * Stochastic variant, selection (Appendix B "Causality under Rejection Sampling").  Same arguments and outputs as
  * dcut_select, with two differences.  (1) The ranking score of draft depth k is the SHIFTED score of Eq. 7,
  * s~_{i,1} = 1, s~_{i,k} = prod_{t<k} c_{i,t}: it does not depend on the proposal at depth k itself (scores_out

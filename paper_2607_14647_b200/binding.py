@@ -29,7 +29,8 @@ STATUS_NAMES = ["DCUT_OK", "DCUT_EINVAL", "DCUT_ECAPACITY", "DCUT_ECUDA", "DCUT_
 EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dense", "dcut_set_cost_buckets",
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
            "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_lm_head_accept",
-           "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_model_verify", "dcut_poll_device_status"]
+           "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_model_verify", "dcut_poll_device_status",
+           "dcut_enable_plan_in_select"]
 
 
 class Limits(C.Structure):
@@ -63,6 +64,7 @@ _lib.dcut_set_cost_buckets.argtypes = [_vp, _i, _i, _vp, _vp, _i]
 _lib.dcut_budget_from_ratio.argtypes = [_i, _i, _i, _i, C.POINTER(_i)]
 _lib.dcut_select.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
 _lib.dcut_select_causal.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
+_lib.dcut_enable_plan_in_select.argtypes = [_vp, _i]
 _lib.dcut_accept_rs.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i] + [_vp] * 8
 _lib.dcut_commit.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.dcut_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _i, _i, _f, _vp, _vp, _vp]
@@ -201,6 +203,10 @@ class Context:
         a = np.ascontiguousarray(cost_ms, dtype=np.float32)
         assert len(k) == len(a)
         self._check(_lib.dcut_set_cost_buckets(self._h, B, gamma, k.ctypes.data, a.ctypes.data, len(a)))
+
+    def enable_plan_in_select(self, on: bool = True):
+        """dcut_enable_plan_in_select: the selector also builds the attention work list of the batch it packs."""
+        self._check(_lib.dcut_enable_plan_in_select(self._h, 1 if on else 0))
 
     # -- hot path ------------------------------------------------------------------------------
     def select(self, conf, draft_ids, bonus_ids, ctx_lens, out: Optional[SelectOut] = None,

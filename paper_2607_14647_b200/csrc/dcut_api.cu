@@ -261,8 +261,22 @@ static dcut_status select_common(dcut_ctx* c, const float* conf, int B, int gamm
     } else if (c->cost_n < B * (gamma + 1) + 1) {
         return dcut_fail(c, DCUT_ECOST, "dense cost table has %d entries, need %d", c->cost_n, B * (gamma + 1) + 1);
     }
-    return dcut_launch_select(c, conf, B, gamma, draft_ids, bonus_ids, ctx_lens, depths, cu_q, tok_req, tok_pos, tok_id,
-                              info, scores_out, ranks_out, causal, static_cast<cudaStream_t>(stream));
+    const int with_plan = c->plan_in_select && ctx_lens && c->lim.n_q_heads > 0;
+    dcut_status st = dcut_launch_select(c, conf, B, gamma, draft_ids, bonus_ids, ctx_lens, depths, cu_q, tok_req, tok_pos,
+                                        tok_id, info, scores_out, ranks_out, causal, with_plan, static_cast<cudaStream_t>(stream));
+    // the attention calls that get these very buffers next use the list instead of building their own
+    c->plan_cu_q = (st == DCUT_OK && with_plan) ? cu_q : nullptr;
+    c->plan_ctx_lens = ctx_lens;
+    c->plan_B = B;
+    return st;
+}
+
+dcut_status dcut_enable_plan_in_select(dcut_ctx* c, int on) {
+    if (!c) return DCUT_EINVAL;
+    if (on && c->lim.n_q_heads <= 0) return dcut_fail(c, DCUT_EINVAL, "context was created without attention shapes");
+    c->plan_in_select = on ? 1 : 0;
+    c->plan_cu_q = nullptr;
+    return DCUT_OK;
 }
 
 dcut_status dcut_select(dcut_ctx* c, const float* conf, int B, int gamma, const int* draft_ids, const int* bonus_ids,

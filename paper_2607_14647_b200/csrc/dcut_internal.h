@@ -61,6 +61,11 @@ struct dcut_ctx {
     int attn_tail_min_pages;
     int attn_tc_min_rows;   // items with at least this many query rows use the tcgen05 phase
     int attn_tail_rows;     // a query tile of up to 128 + this many rows stays one item (0: cut at 128)
+    // work list left ready by the selector (dcut_enable_plan_in_select): the batch it was made for
+    int plan_in_select;
+    const int* plan_cu_q;
+    const int* plan_ctx_lens;
+    int plan_B;
 
     // accept scratch
     unsigned long long* d_row_key;   // [max_T] packed (ordered max, ~index); zero between calls
@@ -141,7 +146,7 @@ void dcut_free_layer(dcut_ctx* ctx);
 dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
                                const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q,
                                int* tok_req, int* tok_pos, int* tok_id, dcut_select_info* info,
-                               float* scores_out, int* ranks_out, int causal, cudaStream_t stream);
+                               float* scores_out, int* ranks_out, int causal, int with_plan, cudaStream_t stream);
 dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids,
                                const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
                                int* out_tokens, int* n_accepted_total, unsigned long long* row_key,

@@ -14,6 +14,7 @@
 #include <limits.h>
 
 #include "dcut_internal.h"
+#include "attn_plan.cuh"
 
 namespace {
 
@@ -38,6 +39,8 @@ struct SelectArgs {
     dcut_select_info* info;
     float* scores_out;
     int* ranks_out;
+    int with_plan;               // also build the attention work list of the packed batch (plan holds its arguments)
+    dcut_plan::PlanArgs plan;
 };
 
 __device__ __forceinline__ float clamp_conf(float c) {
@@ -354,6 +357,13 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
         out.objective = best_s.obj;
         *a.info = out;
     }
+    if (a.with_plan) {
+        // 6. the attention work list of the batch just packed: it depends on ctx_lens, cu_q and the shapes only, and
+        // this CTA has them at hand, so the attention call that follows need not launch a one-CTA kernel of its own.
+        // The sort keys are dead by now: their shared memory holds the plan's ordering keys (npad >= B entries).
+        __syncthreads();            // every thread's cu_q writes are visible to the CTA; nobody reads `keys` any more
+        dcut_plan::attn_plan_body(a.plan, keys);
+    }
 }
 
 size_t select_smem_bytes(int B, int npad) {
@@ -373,7 +383,7 @@ dcut_status dcut_init_select(dcut_ctx* ctx) {
 dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamma, const int* draft_ids,
                                const int* bonus_ids, const int* ctx_lens, int* depths, int* cu_q,
                                int* tok_req, int* tok_pos, int* tok_id, dcut_select_info* info,
-                               float* scores_out, int* ranks_out, int causal, cudaStream_t stream) {
+                               float* scores_out, int* ranks_out, int causal, int with_plan, cudaStream_t stream) {
     const int n = B * gamma;
     int npad = 32;
     while (npad < n) npad <<= 1;
@@ -397,6 +407,8 @@ dcut_status dcut_launch_select(dcut_ctx* ctx, const float* conf, int B, int gamm
     a.info = info;
     a.scores_out = scores_out;
     a.ranks_out = ranks_out;
+    a.with_plan = with_plan;
+    if (with_plan) dcut_fill_plan_args(ctx, ctx_lens, cu_q, B, &a.plan);
     const size_t smem = select_smem_bytes(B, npad);
     return dcut_check_cuda(ctx, dcut_launch_pdl(dcut_select_kernel, dim3(1), dim3(kThreads), smem, stream, a), "launch dcut_select_kernel");
 }

@@ -31,6 +31,7 @@
 #include <type_traits>
 
 #include "dcut_internal.h"
+#include "attn_plan.cuh"
 
 namespace {
 
@@ -39,7 +40,7 @@ constexpr int kMmaWarps = 8;         // consumer warps of the warp-level MMA pha
 constexpr int kMmaThreads = kMmaWarps * 32;
 constexpr int kMmaStages = 16;       // page stages in its ring (8 KB each at head_dim 128)
 constexpr int kMaxProducerLanes = 8;
-constexpr int kPage = 16;            // tokens per page
+constexpr int kPage = dcut_plan::kPage;   // tokens per page
 constexpr int kMaxMTiles = 8;        // query rows per item <= 128
 constexpr int kPlanThreads = 1024;
 constexpr int kSpinLimit = 1 << 21;   // bounded waits: ~1 s, then the CTA reports and leaves
@@ -141,230 +142,15 @@ __device__ __forceinline__ uint32_t tile_off_k4(int r, int c16) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// plan
+// plan (the body lives in attn_plan.cuh: the selector kernel can run it too)
 
-struct PlanArgs {
-    const int* ctx_lens;
-    const int* cu_q;
-    int B, n_q_heads, n_kv_heads;
-    int target_items, min_chunk_pages, max_items, npad, tc_min_rows, max_item_rows;
-    int tail_rows;                      // a remainder of at most this many rows rides with the last full row block (0: never)
-    int tail_req_div, tail_min_pages;   // the shortest B / tail_req_div requests are cut finer (0: none)
-    long long part_rows_cap;
-    int* status;
-    AttnItem* items;
-    int* plan;       // [0] n_items, [1] chunk_pages, [2] total_pages, [3] partial rows used, [4] overflow, [5] n_tc, [8], [9] queue heads
-    int* req_part;   // [B][2]: first partial row, n_chunks
-};
+using dcut_plan::PlanArgs;
 
-template <typename T>
-__device__ __forceinline__ T plan_warp_scan(T v, int lane) {
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        T u = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= o) v += u;
-    }
-    return v;
-}
-
-__device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int inc = plan_warp_scan(v, lane);
-    if (lane == 31) ws[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        int w = lane < (int)(blockDim.x >> 5) ? ws[lane] : 0;
-        int winc = plan_warp_scan(w, lane);
-        ws[lane] = winc - w;
-        if (lane == 31) ws[32] = winc;
-    }
-    __syncthreads();
-    int res = ws[warp] + inc - v;
-    *total = ws[32];
-    __syncthreads();
-    return res;
-}
-
-// Row blocks of a query tile of M rows: full blocks of max_rows rows and one remainder.  A remainder of at most
-// tail_rows rows does not become an item of its own (which would stream the request's K/V a second time): it rides
-// with the last full block, whose item then has up to max_rows + tail_rows rows (the tail warps of the tcgen05 phase
-// take the rows past max_rows from the same staged pages).
-__device__ __forceinline__ int plan_row_blocks(int M, int max_rows, int tail_rows) {
-    const int n_full = M / max_rows, rem = M - n_full * max_rows;
-    return n_full + ((rem > 0 && !(n_full > 0 && rem <= tail_rows)) ? 1 : 0);
-}
-__device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, int rb) {
-    return rb == n_rb - 1 ? M - rb * max_rows : max_rows;
-}
-
-// Requests are ordered by the estimated duration of their items, longest first, so the CTAs that
-// start last are the short ones (the hardware hands items to SMs in index order as SMs free up).
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
-    extern __shared__ unsigned long long order[];   // [npad] (inverted cost << 32 | request), sorted ascending
-    __shared__ int ws[33];
-    __shared__ int total_s, tail_s, w_tc_s, w_mma_s;
-    const int tid = threadIdx.x, nthr = blockDim.x;   // 256 threads for small batches: cheaper barriers
+    extern __shared__ unsigned long long plan_order[];
     dcut_pdl_wait();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the item kernel's CTAs may take their SMs now
-    const int group = a.n_q_heads / a.n_kv_heads;
-    if (tid == 0) {
-        total_s = 0;
-        tail_s = 0;
-        w_tc_s = 0;
-        w_mma_s = 0;
-    }
-    __syncthreads();
-    int local = 0, w_tc = 0, w_mma = 0;   // pages in all; pages whose items would go to the tcgen05 / warp-level queue
-    for (int i = tid; i < a.B; i += nthr) {
-        const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-        const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-        local += pages;
-        const int M = (d + 1) * group;
-        const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
-        int tc_rb = 0;
-        for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= a.tc_min_rows ? 1 : 0;
-        w_tc += pages * tc_rb;
-        w_mma += pages * (n_rb - tc_rb);
-    }
-    if (local) atomicAdd(&total_s, local);
-    if (w_tc) atomicAdd(&w_tc_s, w_tc);
-    if (w_mma) atomicAdd(&w_mma_s, w_mma);
-    __syncthreads();
-    const int total_pages = total_s;
-    const long long units = (long long)total_pages * a.n_kv_heads;
-    int chunk_pages = (int)((units + a.target_items - 1) / a.target_items);
-    if (chunk_pages < a.min_chunk_pages) chunk_pages = a.min_chunk_pages;
-
-    for (int i = tid; i < a.npad; i += nthr) {
-        unsigned long long key = ~0ull;
-        if (i < a.B) {
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-            const int nc = (pages + chunk_pages - 1) / chunk_pages;
-            const int cp = (pages + nc - 1) / nc;
-            const int MT = ((d + 1) * group + 15) >> 4;
-            // per page: memory-bound below about two m-tiles, then time grows with the m-tiles
-            const unsigned int cost = (unsigned int)cp * (unsigned int)max(7, 3 * MT);
-            key = ((unsigned long long)(0xffffffffu - cost) << 32) | (unsigned int)i;
-        }
-        order[i] = key;
-    }
-    __syncthreads();
-    for (int k = 2; k <= a.npad; k <<= 1)
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < (a.npad >> 1); t += nthr) {
-                const int i = 2 * t - (t & (j - 1)), l = i + j;
-                const bool up = (i & k) == 0;
-                const unsigned long long x = order[i], y = order[l];
-                if ((x > y) == up) {
-                    order[i] = y;
-                    order[l] = x;
-                }
-            }
-            __syncthreads();
-        }
-
-    // The items that start last decide how unevenly the SMs finish: the requests at the end of the order are cut
-    // into about target_items pieces altogether, so every SM ends on a short item.
-    const int n_tail = a.tail_req_div > 0 ? (a.B + a.tail_req_div - 1) / a.tail_req_div : 0;
-    const int tail_from = a.B - n_tail;
-    for (int j = tail_from + tid; j < a.B; j += nthr) {
-        const int i = (int)(order[j] & 0xffffffffu);
-        const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-        atomicAdd(&tail_s, (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage);
-    }
-    __syncthreads();
-    int tail_chunk = (int)(((long long)tail_s * a.n_kv_heads + a.target_items - 1) / a.target_items);
-    if (tail_chunk < a.tail_min_pages) tail_chunk = a.tail_min_pages;
-    if (tail_chunk > chunk_pages) tail_chunk = chunk_pages;
-
-    // The item kernel works through the tcgen05 queue first and the warp-level queue after it.  When the second
-    // holds only a small part of the pages (a few shallow requests among deep ones), its few long items would start
-    // late on a few SMs with the rest idle (measured at B = 64: +15 us per call while 3-8 % of the pages were in
-    // it): below one eighth of the pages everything goes to the tcgen05 queue.
-    const int tc_min_rows = (a.tc_min_rows <= a.max_item_rows && w_tc_s > 0 && 8LL * w_mma_s < (long long)w_tc_s + w_mma_s) ? 1 : a.tc_min_rows;
-
-    const int per = (a.B + nthr - 1) / nthr;
-    const int j0 = tid * per;
-    int my_tc = 0, my_mma = 0, my_rows = 0;
-    for (int e = 0; e < per; ++e) {
-        const int j = j0 + e;
-        if (j < a.B) {
-            const int i = (int)(order[j] & 0xffffffffu);
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-            const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
-            const int nc = (pages + cpj - 1) / cpj;
-            // row blocks of the query tile: full blocks of max_item_rows rows and one remainder; each goes to the
-            // tcgen05 queue or to the warp-level queue by its number of rows
-            const int M = (d + 1) * group;
-            const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
-            int tc_rb = 0;
-            for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= tc_min_rows ? 1 : 0;
-            my_tc += nc * a.n_kv_heads * tc_rb;
-            my_mma += nc * a.n_kv_heads * (n_rb - tc_rb);
-            if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
-        }
-    }
-    int n_tc, n_mma, n_rows;
-    int tc_off = plan_block_exclusive_scan(my_tc, ws, &n_tc);
-    int mma_off = plan_block_exclusive_scan(my_mma, ws, &n_mma);
-    int row_off = plan_block_exclusive_scan(my_rows, ws, &n_rows);
-    const int n_items = n_tc + n_mma;
-    mma_off += n_tc;
-    const bool overflow = n_items > a.max_items || (long long)n_rows > a.part_rows_cap;
-    if (tid == 0) {
-        a.plan[0] = overflow ? 0 : n_items;
-        a.plan[1] = chunk_pages;
-        a.plan[2] = total_pages;
-        a.plan[3] = n_rows;
-        a.plan[4] = overflow ? 1 : 0;
-        a.plan[5] = overflow ? 0 : n_tc;     // items [0, n_tc): tcgen05 queue; [n_tc, n_items): warp-level queue
-        a.plan[8] = 0;                       // next item of the tcgen05 queue (claimed by the CTAs of the item kernel)
-        a.plan[9] = overflow ? 0 : n_tc;     // next item of the warp-level queue
-        if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
-    }
-    if (overflow) return;
-    for (int e = 0; e < per; ++e) {
-        const int j = j0 + e;
-        if (j < a.B) {
-            const int i = (int)(order[j] & 0xffffffffu);
-            const int q0 = a.cu_q[i];
-            const int d = a.cu_q[i + 1] - q0 - 1;
-            const int ctx_len = a.ctx_lens[i];
-            const int pages = (ctx_len + d + 1 + kPage - 1) / kPage;
-            const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
-            const int nc = (pages + cpj - 1) / cpj;
-            const int cp = (pages + nc - 1) / nc;   // near-equal chunks
-            const int M = (d + 1) * group;
-            a.req_part[2 * i] = row_off;
-            a.req_part[2 * i + 1] = nc;
-            // a query tile above max_item_rows (+ tail_rows) rows is cut into row blocks, each its own item over the
-            // same pages
-            const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
-            for (int c = 0; c < nc; ++c)
-                for (int h = 0; h < a.n_kv_heads; ++h)
-                    for (int rb = 0; rb < n_rb; ++rb) {
-                        const int row0 = rb * a.max_item_rows, rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
-                        AttnItem it;
-                        it.req = i;
-                        it.kv_head = h;
-                        it.page_begin = c * cp;
-                        it.page_end = min(pages, (c + 1) * cp);
-                        it.n_chunks = nc;
-                        it.part_row = nc > 1 ? row_off + (c * a.n_kv_heads + h) * M + row0 : -1;
-                        it.q0 = q0;
-                        it.depth = d;
-                        it.ctx_len = ctx_len;
-                        const bool tc = rows >= tc_min_rows;
-                        it.pad[0] = tc ? 1 : 0;   // which queue the item is in
-                        it.pad[1] = row0;         // first query row of the item within the request's tile
-                        it.pad[2] = rows;         // query rows of the item
-                        a.items[tc ? tc_off++ : mma_off++] = it;
-                    }
-            if (nc > 1) row_off += nc * (d + 1) * a.n_q_heads;
-        }
-    }
+    dcut_plan::attn_plan_body(a, plan_order);                         // 256 threads for small batches: cheaper barriers
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -579,9 +365,11 @@ __device__ __forceinline__ void sched_release(Ctrl* c, int phase, int n) {
 // warp-level MMA phase (items with few query rows, or any item when head_dim is not 128)
 //
 // kMmaWarps consumer warps + one producer warp.  The ring of page stages is cut into one sub-ring per page slot
-// (nslots = kMmaWarps / m-tiles of the item); pages are numbered through consecutive items, so the producer keeps
-// loading the next item's pages while the consumers still merge the current one.  Only when the number of m-tiles
-// changes between two items is the ring drained and its barriers set up again.
+// (nslots = kMmaWarps / m-tiles of the item); page p of an item goes to slot p mod nslots, and every slot's pages are
+// numbered through consecutive items, so the producer keeps loading the next item's pages while the consumers still
+// merge the current one and an item's result does not depend on what its CTA worked on before (the same bits on
+// every run).  Only when the number of m-tiles changes between two items is the ring drained and its barriers set
+// up again.
 
 template <int DH>
 __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnArgs& a,
@@ -601,7 +389,7 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
 
     AttnItem item;
     int cur_mt = -1, n_geom = 0;
-    long long P0 = 0;                           // pages of the earlier items since the ring was last set up
+    long long slot_pages = 0;                   // producer lanes: pages of this lane's slot since the ring was last set up
     bool failed = false;
 
     if (warp == kMmaWarps) {
@@ -624,24 +412,28 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
                 }
                 ++n_geom;
                 cur_mt = MT;
-                P0 = 0;
+                slot_pages = 0;
             }
             const int n_pages = item.page_end - item.page_begin;
-            int G = kMaxProducerLanes;
-            while (ring_n % G) --G;
-            if (lane < G) {
-                // lane l issues the pages whose running number is l modulo G: a stage is always refilled by the
-                // same lane, whose waits on it are therefore ordered
+            static_assert(kMaxProducerLanes == 8 && kMmaStages == 16, "lane / slot / stage arithmetic below");
+            (void)ring_n;
+            if (lane < kMaxProducerLanes) {
+                // Page p of the item belongs to slot p mod nslots, whatever came before it (the split of an item's
+                // pages over the slots, and with it the rounding of its result, must not depend on which items this
+                // CTA happened to take earlier).  A slot's pages go through its sub-ring in order; the slot is served
+                // by 8 / nslots lanes, lane l = slot + nslots j taking the slot's positions q with q mod (8 / nslots)
+                // = j: a stage is always refilled by the same lane, whose waits on it are therefore ordered.
+                const int sl = lane % nslots, ksub = kMaxProducerLanes / nslots, jsub = lane / nslots;
+                const int cnt = sl < n_pages ? (n_pages - sl + nslots - 1) / nslots : 0;   // this item's pages of the slot
                 const int* bt = a.block_table + (size_t)item.req * a.block_table_stride + item.page_begin;
-                int p = (int)(((long long)lane - P0 % G + G) % G);
-                int next = p < n_pages ? bt[p] : 0;
-                for (; p < n_pages; p += G) {
+                int k = (int)((jsub - slot_pages % ksub + ksub) % ksub);
+                int next = k < cnt ? bt[sl + nslots * k] : 0;
+                for (; k < cnt; k += ksub) {
                     int page_id = next;
-                    if (p + G < n_pages) next = bt[p + G];
-                    const long long P = P0 + p;
-                    const int in_ring = (int)(P % ring_n);
-                    const long long use = P / ring_n;
-                    const int sl = in_ring % nslots, r = in_ring / nslots;   // r-th stage of slot sl
+                    if (k + ksub < cnt) next = bt[sl + nslots * (k + ksub)];
+                    const long long q = slot_pages + k;               // position in the slot's sub-ring since it was set up
+                    const int r = (int)(q % depth_s);
+                    const long long use = q / depth_s;
                     const int stage = sl * depth_s + r;
                     if (use > 0 && !mbar_wait(empty_bar + 8 * stage, (uint32_t)((use - 1) & 1), &c->abort)) {
                         failed = true;
@@ -664,7 +456,10 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
                 failed = true;
                 break;
             }
-            P0 += n_pages;
+            {
+                const int sl = lane % nslots;
+                slot_pages += sl < n_pages ? (n_pages - sl + nslots - 1) / nslots : 0;
+            }
         }
         if (failed) {
             atomicExch(a.status, DCUT_DEV_ATTN_WAIT_TIMEOUT);
@@ -707,7 +502,6 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
             if (!mbar_wait(geom_b, n_geom & 1, &c->abort)) failed = true;
             ++n_geom;
             cur_mt = MT;
-            P0 = 0;
             r_stage = 0;
             parity = 0;
         }
@@ -755,9 +549,9 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
             const int v_tok = ((kmat & 1) << 3) + (lane & 7);
             const int v_chunk = kmat >> 1;
 
-            // this warp's pages of the item: running number = slot modulo nslots, in order through the slot's sub-ring
+            // this warp's pages of the item: p = slot modulo nslots, in order through the slot's sub-ring
             const float c_log2 = a.scale_log2;
-            for (int p = (int)(((long long)slot - P0 % nslots + nslots) % nslots); p < n_pages; p += nslots) {
+            for (int p = slot; p < n_pages; p += nslots) {
                 const int stage = slot * depth_s + r_stage;
                 if (!mbar_wait(full_bar + 8 * stage, parity, &c->abort)) {
                     failed = true;
@@ -846,7 +640,6 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
             }
         }
         if (failed) c->abort = 1;
-        P0 += n_pages;
 
         // ---------------------------------------------------------------- merge the slots
         // (the merge buffer is not part of the ring: the producer is already loading the next item)
@@ -1511,7 +1304,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                     const int np = min(4, n_pages - 4 * g);
                     const uint32_t k_grp = smem_u32(ring + gs * kTcGroupBytes);
                     // the warps take the groups alternately, a whole group (64 keys) per softmax step
-                    if ((gc & 1) == tw) {
+                    if ((g & 1) == tw) {
                         if (np == 4) tail_step8(std::integral_constant<int, 4>(), k_grp, item.page_begin + 4 * g);
                         else
                             for (int j = 0; j < np; ++j) tail_step8(std::integral_constant<int, 1>(), k_grp + j * kTcPageBytes, item.page_begin + 4 * g + j);
@@ -1862,6 +1655,30 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
     return DCUT_OK;
 }
 
+void dcut_fill_plan_args(dcut_ctx* ctx, const int* ctx_lens, const int* cu_q, int B, dcut_plan::PlanArgs* out) {
+    dcut_plan::PlanArgs& pa = *out;
+    pa.ctx_lens = ctx_lens;
+    pa.cu_q = cu_q;
+    pa.B = B;
+    pa.n_q_heads = ctx->lim.n_q_heads;
+    pa.n_kv_heads = ctx->lim.n_kv_heads;
+    pa.target_items = ctx->target_items;
+    pa.min_chunk_pages = 8;
+    pa.tail_req_div = ctx->attn_tail_req_div;
+    pa.tail_min_pages = ctx->attn_tail_min_pages;
+    pa.npad = 32;
+    while (pa.npad < B) pa.npad <<= 1;
+    pa.status = ctx->d_status;
+    pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
+    pa.max_item_rows = 128;
+    pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? ctx->attn_tail_rows : 0;
+    pa.max_items = ctx->max_items;
+    pa.part_rows_cap = ctx->part_rows_cap;
+    pa.items = ctx->d_items;
+    pa.plan = ctx->d_plan;
+    pa.req_part = ctx->d_req_part;
+}
+
 dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
                                     long long num_pages, const int* block_table, int block_table_stride,
                                     const int* ctx_lens, const int* cu_q, int B, int T_cap, float scale,
@@ -1887,27 +1704,11 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     }
 
     PlanArgs pa;
-    pa.ctx_lens = ctx_lens;
-    pa.cu_q = cu_q;
-    pa.B = B;
-    pa.n_q_heads = ctx->lim.n_q_heads;
-    pa.n_kv_heads = ctx->lim.n_kv_heads;
-    pa.target_items = ctx->target_items;
-    pa.min_chunk_pages = 8;
-    pa.tail_req_div = ctx->attn_tail_req_div;
-    pa.tail_min_pages = ctx->attn_tail_min_pages;
-    pa.npad = 32;
-    while (pa.npad < B) pa.npad <<= 1;
-    pa.status = ctx->d_status;
-    pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
-    pa.max_item_rows = 128;
-    pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? ctx->attn_tail_rows : 0;
-    pa.max_items = ctx->max_items;
-    pa.part_rows_cap = ctx->part_rows_cap;
-    pa.items = ctx->d_items;
-    pa.plan = ctx->d_plan;
-    pa.req_part = ctx->d_req_part;
+    dcut_fill_plan_args(ctx, ctx_lens, cu_q, B, &pa);
+    // the selector may have left the work list of exactly this batch ready (dcut_enable_plan_in_select)
+    if (ctx->plan_in_select && ctx->plan_cu_q == cu_q && ctx->plan_ctx_lens == ctx_lens && ctx->plan_B == B) reuse_plan = 1;
     if (!reuse_plan) {   // reuse_plan: the previous launch on this stream had the same ctx_lens, cu_q and B (its work list stands)
+        ctx->plan_cu_q = nullptr;   // the list now belongs to this call's batch
         st = dcut_check_cuda(ctx, dcut_launch_pdl(attn_plan_kernel, dim3(1), dim3(B <= 256 ? 256 : kPlanThreads),
                                                   sizeof(unsigned long long) * pa.npad, stream, pa), "launch attn_plan_kernel");
         if (st != DCUT_OK) return st;

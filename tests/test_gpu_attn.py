@@ -131,11 +131,14 @@ def test_b256_long_tail_sampled():
     _sampled_compare(cfg, sel, kv, np.zeros(cfg.B, np.int32), 96, seed=2)
 
 
-def test_repeated_runs_are_bit_identical():
-    cfg = wl.custom_config(B=8, gamma=16, n_q_heads=32, n_kv_heads=8, head_dim=128, ctx_lo=100, ctx_hi=3000)
+@pytest.mark.parametrize("B,depths", [(8, [3, 16, 0, 8, 12, 1, 5, 16]), (20, [0] * 20), (20, [0, 1, 2, 3, 7] * 4)])
+def test_repeated_runs_are_bit_identical(B, depths):
+    """The persistent CTAs take work items in whatever order they come free; an item's result must not depend on
+    what its CTA worked on before (shallow batches go through the warp-level phase, where it once did)."""
+    cfg = wl.custom_config(B=B, gamma=16, n_q_heads=32, n_kv_heads=8, head_dim=128, ctx_lo=100, ctx_hi=3000)
     sel = wl.select_inputs(cfg)
     kv = wl.paged_kv(cfg, sel.ctx_lens)
-    depths = np.array([3, 16, 0, 8, 12, 1, 5, 16], np.int32)
+    depths = np.array(depths, np.int32)
     ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req)
     args = (dev(wl.q_rows(cfg, depths)), dev(kv.k_cache), dev(kv.v_cache), dev(kv.block_table), dev(sel.ctx_lens),
             dev(wl.cu_q_from_depths(depths)), cfg.t_cap)
