@@ -203,6 +203,37 @@ dcut_status dcut_layer_forward(dcut_ctx* ctx, const dcut_layer_weights* weights,
                                int T_cap, void* stream);
 
 /*
+ * Start-up cost table C(B, rho) (Eq. 4-5; Appendix C, "Cost-table profiling protocol"; Table 3 shows two such
+ * tables).  The paper's system builds it once before serving: for every batch size B it captures a graph for and
+ * every ratio bucket rho it runs dummy speculative steps with the budget K_rho(B) and records the median step
+ * latency; at decode time the selector reads the row of the current batch size, and a batch size between captured
+ * points uses the nearest captured row.  dcut_cost_grid is that table as a HOST object: the caller runs and times the
+ * steps (they go through this library's own calls; paper_2607_14647_b200/profiler.py does it with CUDA events) and
+ * records the samples; the library keeps the medians, finds the nearest row and installs it as the bucket table.
+ *   batch_sizes ascending, >= 1; ratios num/den ascending in (0, 1]; all HOST arrays, copied.
+ *   dcut_cost_grid_budget   K_rho(B) of Eq. 4 for any live B (ceiling in exact integer arithmetic, clamp to [B, B(gamma+1)]).
+ *   dcut_cost_grid_record   cell (b, r) := median of n > 0 positive finite samples (an even n: mean of the two middle
+ *                           ones, computed in double); DCUT_ECOST on a bad sample.
+ *   dcut_cost_grid_nearest  index of the captured batch size nearest to B; the paper does not say how a tie breaks:
+ *                           here the larger captured batch wins (its graph can hold the batch and its cost is not an
+ *                           underestimate).
+ *   dcut_cost_grid_buckets  the bucket table a live batch of B gets: budgets K_rho(B), costs of the nearest row; ratios
+ *                           that give the same budget (small B) are merged and keep the smaller cost.  K_out / cost_out
+ *                           hold one entry per ratio at most.  DCUT_ECOST if the row has an unrecorded cell.
+ *   dcut_set_cost_from_grid the same table handed to dcut_set_cost_buckets(ctx, B, gamma, ...).
+ */
+typedef struct dcut_cost_grid dcut_cost_grid;
+dcut_status dcut_cost_grid_create(dcut_cost_grid** out, const int* batch_sizes, int n_batch, const int* ratio_num,
+                                  const int* ratio_den, int n_ratios, int gamma);
+dcut_status dcut_cost_grid_destroy(dcut_cost_grid* grid);
+dcut_status dcut_cost_grid_budget(const dcut_cost_grid* grid, int B, int r, int* K);
+dcut_status dcut_cost_grid_record(dcut_cost_grid* grid, int b, int r, const float* samples_ms, int n);
+dcut_status dcut_cost_grid_get(const dcut_cost_grid* grid, int b, int r, float* cost_ms);
+dcut_status dcut_cost_grid_nearest(const dcut_cost_grid* grid, int B, int* b);
+dcut_status dcut_cost_grid_buckets(const dcut_cost_grid* grid, int B, int* K_out, float* cost_out, int* n_out);
+dcut_status dcut_set_cost_from_grid(dcut_ctx* ctx, const dcut_cost_grid* grid, int B);
+
+/*
  * Selection and the attention work list in one launch (Algorithm 1 hands the packed batch straight to the target
  * forward; Appendix C folds the packing cost into verification).  The work list of dcut_verify_attn (how the requests'
  * page lists are cut into items and in which order they run) depends on ctx_lens, cu_q, B and the context's shapes only.

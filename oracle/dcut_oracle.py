@@ -1,9 +1,11 @@
 """ctypes front end of the CPU oracle (`dcut_oracle.c`).  TEST INFRASTRUCTURE ONLY.
 
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
-It marshals numpy / torch-CPU arrays to the C functions and does no arithmetic of its own
-(what each C function computes, and the passage of the paper it follows, is in the C file).
-It imports nothing from the CUDA package.
+It marshals numpy / torch-CPU arrays to the C functions (what each C function computes, and the passage
+of the paper it follows, is in the C file).  A few definitions that are only bookkeeping around those
+functions are written out here in plain Python, each citing its passage: `commit` (end of a step),
+`cost_grid_*` (the start-up cost table), and the compositions `lm_head_accept`, `layer_forward`,
+`model_verify`.  It imports nothing from the CUDA package.
 """
 from __future__ import annotations
 
@@ -152,6 +154,41 @@ def commit(accept_len, out_tokens, ctx_lens, streams):
         nxt[i] = out_tokens[i, m]
         streams[i].extend(int(t) for t in out_tokens[i, : m + 1])
     return new_ctx, nxt
+
+
+# ---------------------------------------------------------------------------------------------
+# Start-up cost table C(B, rho)  (Appendix C, "Cost-table profiling protocol"; Eq. 4; Table 3)
+
+def cost_grid_median(samples_ms) -> np.float32:
+    """"Median per-step latency over a small number of repetitions": the middle sample; for an even count the
+    mean of the two middle samples (a reading: the paper does not say), in double, rounded once to fp32."""
+    v = sorted(float(np.float32(x)) for x in samples_ms)
+    n = len(v)
+    return np.float32(v[n // 2]) if n % 2 else np.float32((v[n // 2 - 1] + v[n // 2]) * 0.5)
+
+
+def cost_grid_nearest(batch_sizes: Sequence[int], B: int) -> int:
+    """"Batch sizes that fall between captured points reuse the nearest captured entry": index of the captured
+    size with the smallest |B_c - B|.  A tie (the paper is silent) goes to the larger captured batch."""
+    best = None
+    for b, bc in enumerate(batch_sizes):
+        d = abs(int(bc) - int(B))
+        if best is None or d < best[0] or (d == best[0] and bc > batch_sizes[best[1]]):
+            best = (d, b)
+    return best[1]
+
+
+def cost_grid_buckets(batch_sizes, ratios, gamma: int, table, B: int):
+    """The bucket table a live batch of B requests reads: budgets K_rho(B) by Eq. 4 for the live B, latencies from
+    the row of the nearest captured batch size.  Ratios whose budgets coincide (small B) are one candidate; it
+    keeps the smaller latency (a reading: the objective of Eq. 5 then prefers it anyway)."""
+    row = table[cost_grid_nearest(batch_sizes, B)]
+    out = {}
+    for (num, den), c in zip(ratios, row):
+        K = budget(B, gamma, num, den)
+        out[K] = min(out.get(K, np.inf), float(np.float32(c)))
+    Ks = sorted(out)
+    return np.array(Ks, np.int32), np.array([out[k] for k in Ks], np.float32)
 
 
 def scores_shifted(conf: np.ndarray) -> np.ndarray:

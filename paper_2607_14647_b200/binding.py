@@ -10,7 +10,7 @@ from __future__ import annotations
 import ctypes as C
 import os
 from dataclasses import dataclass
-from typing import Optional, Sequence
+from typing import Optional, Sequence, Tuple
 
 import numpy as np
 import torch
@@ -30,7 +30,9 @@ EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dens
            "dcut_budget_from_ratio", "dcut_select", "dcut_verify_attn", "dcut_accept", "dcut_verify_step_host",
            "dcut_accept_static", "dcut_gemm_bf16", "dcut_layer_forward", "dcut_lm_head_accept",
            "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_model_verify", "dcut_poll_device_status",
-           "dcut_enable_plan_in_select"]
+           "dcut_enable_plan_in_select", "dcut_cost_grid_create", "dcut_cost_grid_destroy", "dcut_cost_grid_budget",
+           "dcut_cost_grid_record", "dcut_cost_grid_get", "dcut_cost_grid_nearest", "dcut_cost_grid_buckets",
+           "dcut_set_cost_from_grid"]
 
 
 class Limits(C.Structure):
@@ -65,6 +67,14 @@ _lib.dcut_budget_from_ratio.argtypes = [_i, _i, _i, _i, C.POINTER(_i)]
 _lib.dcut_select.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
 _lib.dcut_select_causal.argtypes = [_vp, _vp, _i, _i] + [_vp] * 11 + [_vp]
 _lib.dcut_enable_plan_in_select.argtypes = [_vp, _i]
+_lib.dcut_cost_grid_create.argtypes = [C.POINTER(_vp), _vp, _i, _vp, _vp, _i, _i]
+_lib.dcut_cost_grid_destroy.argtypes = [_vp]
+_lib.dcut_cost_grid_budget.argtypes = [_vp, _i, _i, C.POINTER(_i)]
+_lib.dcut_cost_grid_record.argtypes = [_vp, _i, _i, _vp, _i]
+_lib.dcut_cost_grid_get.argtypes = [_vp, _i, _i, C.POINTER(_f)]
+_lib.dcut_cost_grid_nearest.argtypes = [_vp, _i, C.POINTER(_i)]
+_lib.dcut_cost_grid_buckets.argtypes = [_vp, _i, _vp, _vp, C.POINTER(_i)]
+_lib.dcut_set_cost_from_grid.argtypes = [_vp, _vp, _i]
 _lib.dcut_accept_rs.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i] + [_vp] * 8
 _lib.dcut_commit.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.dcut_verify_attn.argtypes = [_vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _i, _i, _f, _vp, _vp, _vp]
@@ -153,6 +163,65 @@ class SelectOut:
     ranks: Optional[torch.Tensor]
 
 
+class CostGrid:
+    """dcut_cost_grid: the start-up cost table C(B, rho), a host object (works without a GPU)."""
+
+    def __init__(self, batch_sizes: Sequence[int], ratios: Sequence[Tuple[int, int]], gamma: int):
+        self.batch_sizes, self.ratios, self.gamma = [int(b) for b in batch_sizes], [(int(n), int(d)) for n, d in ratios], int(gamma)
+        b = np.ascontiguousarray(self.batch_sizes, dtype=np.int32)
+        num = np.ascontiguousarray([r[0] for r in self.ratios], dtype=np.int32)
+        den = np.ascontiguousarray([r[1] for r in self.ratios], dtype=np.int32)
+        self._h = _vp(None)
+        st = _lib.dcut_cost_grid_create(C.byref(self._h), b.ctypes.data, len(b), num.ctypes.data, den.ctypes.data, len(num), gamma)
+        if st != OK:
+            raise DcutError(st, "dcut_cost_grid_create: batch sizes and ratios must ascend; ratios in (0, 1]; gamma >= 1")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            _lib.dcut_cost_grid_destroy(self._h)
+            self._h = _vp(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int, what: str):
+        if st != OK:
+            raise DcutError(st, what)
+
+    def budget(self, B: int, r: int) -> int:
+        k = _i(0)
+        self._check(_lib.dcut_cost_grid_budget(self._h, B, r, C.byref(k)), "dcut_cost_grid_budget")
+        return k.value
+
+    def record(self, b: int, r: int, samples_ms: Sequence[float]):
+        a = np.ascontiguousarray(samples_ms, dtype=np.float32)
+        self._check(_lib.dcut_cost_grid_record(self._h, b, r, a.ctypes.data, len(a)), "dcut_cost_grid_record: bad cell or sample")
+
+    def get(self, b: int, r: int) -> float:
+        v = _f(0.0)
+        self._check(_lib.dcut_cost_grid_get(self._h, b, r, C.byref(v)), "dcut_cost_grid_get")
+        return v.value
+
+    def table(self) -> np.ndarray:
+        return np.array([[self.get(b, r) for r in range(len(self.ratios))] for b in range(len(self.batch_sizes))], np.float32)
+
+    def nearest(self, B: int) -> int:
+        b = _i(0)
+        self._check(_lib.dcut_cost_grid_nearest(self._h, B, C.byref(b)), "dcut_cost_grid_nearest")
+        return b.value
+
+    def buckets(self, B: int):
+        K = np.zeros(len(self.ratios), np.int32)
+        c = np.zeros(len(self.ratios), np.float32)
+        n = _i(0)
+        self._check(_lib.dcut_cost_grid_buckets(self._h, B, K.ctypes.data, c.ctypes.data, C.byref(n)),
+                    "dcut_cost_grid_buckets: the nearest row is not fully recorded")
+        return K[: n.value].copy(), c[: n.value].copy()
+
+
 def read_info(info: torch.Tensor) -> SelectInfo:
     """Copies the device record to the host (synchronises)."""
     raw = info.cpu().numpy().tobytes()
@@ -207,6 +276,10 @@ class Context:
     def enable_plan_in_select(self, on: bool = True):
         """dcut_enable_plan_in_select: the selector also builds the attention work list of the batch it packs."""
         self._check(_lib.dcut_enable_plan_in_select(self._h, 1 if on else 0))
+
+    def set_cost_from_grid(self, grid: "CostGrid", B: int):
+        """dcut_set_cost_from_grid: bucket mode with the budgets of a live batch of B and the nearest captured row."""
+        self._check(_lib.dcut_set_cost_from_grid(self._h, grid._h, B))
 
     # -- hot path ------------------------------------------------------------------------------
     def select(self, conf, draft_ids, bonus_ids, ctx_lens, out: Optional[SelectOut] = None,

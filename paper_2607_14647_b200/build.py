@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libdcut.so")
-SOURCES = ["dcut_api.cu", "select.cu", "accept.cu", "accept_rs.cu", "commit.cu", "verify_attn.cu", "layer.cu"]
+SOURCES = ["dcut_api.cu", "cost_grid.cu", "select.cu", "accept.cu", "accept_rs.cu", "commit.cu", "verify_attn.cu", "layer.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
 
