@@ -33,22 +33,66 @@ __device__ __forceinline__ T plan_warp_scan(T v, int lane) {
     return v;
 }
 
-__device__ __forceinline__ int plan_block_exclusive_scan(int v, int* ws, int* total) {
+// three exclusive scans over the CTA at once (one value of each per thread): prefixes in o0..o2, totals in t0..t2
+__device__ __forceinline__ void plan_block_exclusive_scan3(int v0, int v1, int v2, int (*ws)[33], int& o0, int& o1, int& o2,
+                                                           int& t0, int& t1, int& t2) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int inc = plan_warp_scan(v, lane);
-    if (lane == 31) ws[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        int w = lane < (int)(blockDim.x >> 5) ? ws[lane] : 0;
-        int winc = plan_warp_scan(w, lane);
-        ws[lane] = winc - w;
-        if (lane == 31) ws[32] = winc;
+    const int i0 = plan_warp_scan(v0, lane), i1 = plan_warp_scan(v1, lane), i2 = plan_warp_scan(v2, lane);
+    if (lane == 31) {
+        ws[0][warp] = i0;
+        ws[1][warp] = i1;
+        ws[2][warp] = i2;
     }
     __syncthreads();
-    int res = ws[warp] + inc - v;
-    *total = ws[32];
+    if (warp < 3) {
+        const int w = lane < (int)(blockDim.x >> 5) ? ws[warp][lane] : 0;
+        const int winc = plan_warp_scan(w, lane);
+        ws[warp][lane] = winc - w;
+        if (lane == 31) ws[warp][32] = winc;
+    }
     __syncthreads();
-    return res;
+    o0 = ws[0][warp] + i0 - v0;
+    o1 = ws[1][warp] + i1 - v1;
+    o2 = ws[2][warp] + i2 - v2;
+    t0 = ws[0][32];
+    t1 = ws[1][32];
+    t2 = ws[2][32];
+}
+
+// ascending bitonic sort of 32 E keys by one warp: lane l holds elements e * 32 + l
+template <int E>
+__device__ __forceinline__ void plan_warp_sort(unsigned long long* keys, int lane) {
+    unsigned long long k[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) k[e] = keys[e * 32 + lane];
+#pragma unroll
+    for (int kk = 2; kk <= 32 * E; kk <<= 1) {
+#pragma unroll
+        for (int j = kk >> 1; j > 0; j >>= 1) {
+            if (j >= 32) {                          // partner in the same lane
+                const int je = j >> 5;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if ((e & je) == 0) {
+                        const bool up = (((e * 32 + lane) & kk) == 0);
+                        const unsigned long long x = k[e], y = k[e | je];
+                        const bool swap = (x > y) == up;
+                        k[e] = swap ? y : x;
+                        k[e | je] = swap ? x : y;
+                    }
+                }
+            } else {                                // partner in another lane
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, k[e], j);
+                    const bool keep_min = (((e * 32 + lane) & kk) == 0) == ((lane & j) == 0);
+                    k[e] = ((k[e] < other) == keep_min) ? k[e] : other;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) keys[e * 32 + lane] = k[e];
 }
 
 // Row blocks of a query tile of M rows: full blocks of max_rows rows and one remainder.  A remainder of at most
@@ -68,7 +112,7 @@ __device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, in
 // Every thread of the CTA calls this (it synchronises the CTA).  `order` is shared memory for a.npad 64-bit keys:
 // (inverted cost << 32 | request), sorted ascending.
 __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, unsigned long long* order) {
-    __shared__ int ws[33];
+    __shared__ int ws3[3][33];
     __shared__ int total_s, tail_s, w_tc_s, w_mma_s;
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -115,30 +159,43 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, unsigned long 
         order[i] = key;
     }
     __syncthreads();
-    for (int k = 2; k <= a.npad; k <<= 1)
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int t = tid; t < (a.npad >> 1); t += nthr) {
-                const int i = 2 * t - (t & (j - 1)), l = i + j;
-                const bool up = (i & k) == 0;
-                const unsigned long long x = order[i], y = order[l];
-                if ((x > y) == up) {
-                    order[i] = y;
-                    order[l] = x;
-                }
-            }
-            __syncthreads();
+    if (a.npad <= 256) {
+        // up to 256 requests: one warp sorts the keys in registers (element e * 32 + lane), without a single barrier
+        if (tid < 32) {
+            if (a.npad <= 32) plan_warp_sort<1>(order, tid);
+            else if (a.npad <= 64) plan_warp_sort<2>(order, tid);
+            else if (a.npad <= 128) plan_warp_sort<4>(order, tid);
+            else plan_warp_sort<8>(order, tid);
         }
+        __syncthreads();
+    } else {
+        for (int k = 2; k <= a.npad; k <<= 1)
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int t = tid; t < (a.npad >> 1); t += nthr) {
+                    const int i = 2 * t - (t & (j - 1)), l = i + j;
+                    const bool up = (i & k) == 0;
+                    const unsigned long long x = order[i], y = order[l];
+                    if ((x > y) == up) {
+                        order[i] = y;
+                        order[l] = x;
+                    }
+                }
+                __syncthreads();
+            }
+    }
 
     // The items that start last decide how unevenly the SMs finish: the requests at the end of the order are cut
     // into about target_items pieces altogether, so every SM ends on a short item.
     const int n_tail = a.tail_req_div > 0 ? (a.B + a.tail_req_div - 1) / a.tail_req_div : 0;
     const int tail_from = a.B - n_tail;
-    for (int j = tail_from + tid; j < a.B; j += nthr) {
-        const int i = (int)(order[j] & 0xffffffffu);
-        const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-        atomicAdd(&tail_s, (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage);
+    if (n_tail > 0) {   // (the same answer in every thread)
+        for (int j = tail_from + tid; j < a.B; j += nthr) {
+            const int i = (int)(order[j] & 0xffffffffu);
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            atomicAdd(&tail_s, (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage);
+        }
+        __syncthreads();
     }
-    __syncthreads();
     int tail_chunk = (int)(((long long)tail_s * a.n_kv_heads + a.target_items - 1) / a.target_items);
     if (tail_chunk < a.tail_min_pages) tail_chunk = a.tail_min_pages;
     if (tail_chunk > chunk_pages) tail_chunk = chunk_pages;
@@ -172,9 +229,8 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, unsigned long 
         }
     }
     int n_tc, n_mma, n_rows;
-    int tc_off = plan_block_exclusive_scan(my_tc, ws, &n_tc);
-    int mma_off = plan_block_exclusive_scan(my_mma, ws, &n_mma);
-    int row_off = plan_block_exclusive_scan(my_rows, ws, &n_rows);
+    int tc_off, mma_off, row_off;
+    plan_block_exclusive_scan3(my_tc, my_mma, my_rows, ws3, tc_off, mma_off, row_off, n_tc, n_mma, n_rows);
     const int n_items = n_tc + n_mma;
     mma_off += n_tc;
     const bool overflow = n_items > a.max_items || (long long)n_rows > a.part_rows_cap;

@@ -147,9 +147,17 @@ __device__ __forceinline__ uint32_t tile_off_k4(int r, int c16) {
 using dcut_plan::PlanArgs;
 
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
-    extern __shared__ unsigned long long plan_order[];
+    extern __shared__ unsigned long long plan_order[];                // [npad] keys, then cu_q [B + 1] and ctx_lens [B]
     dcut_pdl_wait();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the item kernel's CTAs may take their SMs now
+    // the body reads every request's cu_q and ctx_lens several times: from shared memory, not through L2
+    int* cu_s = reinterpret_cast<int*>(plan_order + a.npad);
+    int* ctx_s = cu_s + a.B + 1;
+    for (int i = threadIdx.x; i <= a.B; i += blockDim.x) cu_s[i] = a.cu_q[i];
+    for (int i = threadIdx.x; i < a.B; i += blockDim.x) ctx_s[i] = a.ctx_lens[i];
+    __syncthreads();
+    a.cu_q = cu_s;
+    a.ctx_lens = ctx_s;
     dcut_plan::attn_plan_body(a, plan_order);                         // 256 threads for small batches: cheaper barriers
 }
 
@@ -1644,7 +1652,7 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
         env = getenv("DCUT_ATTN_TAIL_ROWS");     // 0: a query tile above 128 rows becomes two items (experiments)
         ctx->attn_tail_rows = env ? (atoi(env) > 0 ? kTcTailRows : 0) : kTcTailRows;
     }
-    e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS);
+    e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS + 4 * (2 * DCUT_MAX_KEYS + 1));
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn plan)");
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -1710,7 +1718,8 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     if (!reuse_plan) {   // reuse_plan: the previous launch on this stream had the same ctx_lens, cu_q and B (its work list stands)
         ctx->plan_cu_q = nullptr;   // the list now belongs to this call's batch
         st = dcut_check_cuda(ctx, dcut_launch_pdl(attn_plan_kernel, dim3(1), dim3(B <= 256 ? 256 : kPlanThreads),
-                                                  sizeof(unsigned long long) * pa.npad, stream, pa), "launch attn_plan_kernel");
+                                                  sizeof(unsigned long long) * pa.npad + sizeof(int) * (2 * B + 1), stream, pa),
+                             "launch attn_plan_kernel");
         if (st != DCUT_OK) return st;
     }
 
