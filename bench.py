@@ -43,9 +43,9 @@ METRIC = "accepted_tokens_per_s_per_verify_step_B64"
 UNIT = "tokens/s"
 L2_BYTES = 126e6
 # DRAM bytes per algorithmic byte of attn_item_kernel, from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum of
-# one launch) summarised in profiles/attn_item_kernel_dram_traffic.md: 1.03 at workload 2's pruned packing, 1.02-1.06 over
-# the other arms and workload 3; the kernel's traffic is proportional to the KV it streams
-ATTN_TRAFFIC_RATIO = 1.03
+# one launch) summarised in profiles/attn_item_kernel_dram_traffic.md: 1.001-1.005 over the three arms of workload 2 at
+# full size and of workload 3's shapes at B = 48; the kernel's traffic is proportional to the KV it streams
+ATTN_TRAFFIC_RATIO = 1.003
 RATIO_BUCKETS = [(1, 4), (1, 2), (3, 4), (1, 1)]          # the paper's ratio set R (Eq. 4; Table 3)
 COST_PROFILE_DIR = os.path.join(ROOT, "paper_2607_14647_b200", "cost_profiles")
 
@@ -74,6 +74,7 @@ def parse_args():
     ap.add_argument("--multistep", type=int, default=8, help="steps chained on the device (select..commit) in the multi-step arm; 0: skip")
     ap.add_argument("--attn-only", action="store_true",
                     help="run only dcut_verify_attn, `--steps` launches per arm after `--warmup` (the command ncu captures)")
+    ap.add_argument("--batch", type=int, default=0, help="with --attn-only: this many requests instead of the config's B (small ncu captures)")
     ap.add_argument("--write-cost-profile", action="store_true",
                     help="store the profiled cost points under paper_2607_14647_b200/cost_profiles/ (read by --impl reference)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -815,6 +816,8 @@ def run_attn_only(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     cfg = wl.config(args.config)
+    if args.batch > 0:
+        cfg = dataclasses.replace(cfg, B=args.batch, name=f"{cfg.name}_B{args.batch}")
     w = Workload(cfg, dev, kv_copies=1)
     cost = wl.cost_table_linear(cfg.t_cap + 1, 0.2, 0.0001)
     out = {}
