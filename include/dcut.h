@@ -16,6 +16,9 @@
  *   - The context owns only its scratch memory, allocated once in dcut_create from dcut_limits;
  *     no call on the hot path allocates.  One context serves one stream at a time: calls that
  *     overlap on the GPU share the scratch and race.
+ *   - A context belongs to the device it was created on.  Every call that launches work checks that
+ *     this device is the current one (cudaGetDevice) and returns DCUT_EINVAL otherwise: a launch on
+ *     another device would hand that device this context's scratch pointers.
  *   - Every call returns a dcut_status.  Errors the host can see (null pointer, a size over the
  *     limits, a bad cost table) are returned before anything is launched.  Nothing aborts or traps;
  *     dcut_last_error gives a message for the last failing call on that context.
@@ -94,6 +97,9 @@ const char* dcut_last_error(const dcut_ctx* ctx);
  * B <= K[r] <= B*(gamma+1), total positions including the B bonus positions) and their costs;
  * valid for exactly this B and gamma.  n_buckets <= 64.
  * Any cost <= 0, NaN or inf gives DCUT_ECOST.  Setting one form replaces the other.
+ * The table lives in one device buffer that the copy overwrites in place (a synchronous copy that is not
+ * ordered against work on other streams): no dcut_select of this context may be running or enqueued when the
+ * table is replaced.  A captured CUDA graph of a step reads whatever table is in the buffer when it is replayed.
  */
 dcut_status dcut_set_cost_dense(dcut_ctx* ctx, const float* cost_ms, int n);
 dcut_status dcut_set_cost_buckets(dcut_ctx* ctx, int B, int gamma, const int* K, const float* cost_ms,

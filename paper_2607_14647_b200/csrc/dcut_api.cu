@@ -36,6 +36,20 @@ struct DeviceGuard {
     }
 };
 
+// a launch with another device current would run there with this context's scratch pointers
+dcut_status check_device(dcut_ctx* c) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return dcut_fail(c, DCUT_ECUDA, "cudaGetDevice failed");
+    if (dev != c->device)
+        return dcut_fail(c, DCUT_EINVAL, "device %d is current, but this context belongs to device %d (cudaSetDevice first)", dev, c->device);
+    return DCUT_OK;
+}
+#define DCUT_ON_DEVICE(c)                                   \
+    do {                                                    \
+        const dcut_status dev_st_ = check_device(c);        \
+        if (dev_st_ != DCUT_OK) return dev_st_;             \
+    } while (0)
+
 template <typename T>
 dcut_status dmalloc(dcut_ctx* ctx, T** p, size_t count, const char* what) {
     cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), sizeof(T) * (count ? count : 1));
@@ -246,6 +260,7 @@ static dcut_status select_common(dcut_ctx* c, const float* conf, int B, int gamm
                                  const int* ctx_lens, int* depths, int* cu_q, int* tok_req, int* tok_pos, int* tok_id,
                                  dcut_select_info* info, float* scores_out, int* ranks_out, int causal, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (causal && c->n_buckets > 1)
         return dcut_fail(c, DCUT_ECOST, "the causal selector takes a dense cost table or exactly one bucket (a budget fixed beforehand)");
     if (!conf || !depths || !cu_q) return dcut_fail(c, DCUT_EINVAL, "conf, depths and cu_q must not be null");
@@ -298,6 +313,7 @@ dcut_status dcut_verify_attn(dcut_ctx* c, const void* q, const void* k_cache, co
                              const int* block_table, int block_table_stride, const int* ctx_lens, const int* cu_q, int B,
                              int T_cap, float scale, void* out, float* lse, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (c->lim.n_q_heads <= 0) return dcut_fail(c, DCUT_EINVAL, "context was created without attention shapes");
     if (!q || !k_cache || !v_cache || !block_table || !ctx_lens || !cu_q || !out)
         return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
@@ -319,6 +335,7 @@ dcut_status dcut_verify_attn(dcut_ctx* c, const void* q, const void* k_cache, co
 dcut_status dcut_accept(dcut_ctx* c, const void* logits, int V, const int* draft_ids, const int* cu_q, int B, int gamma,
                         int T_cap, int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (!logits || !draft_ids || !cu_q || !accept_len || !bonus) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
     if (B < 1 || gamma < 1 || V < 1 || T_cap < B) return dcut_fail(c, DCUT_EINVAL, "need B, gamma, V >= 1 and T_cap >= B");
     if (B > c->lim.max_B || gamma > c->lim.max_gamma || T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
@@ -333,6 +350,7 @@ dcut_status dcut_accept_rs(dcut_ctx* c, const void* target_logits, const void* d
                            const int* cu_q, int B, int gamma, int T_cap, const float* u_accept, const float* u_sample,
                            int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, float* prob, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (!c->d_rs_scratch) return dcut_fail(c, DCUT_EINVAL, "context was created with vocab = 0");
     if (!target_logits || !draft_logits || !draft_ids || !cu_q || !u_accept || !u_sample || !accept_len || !bonus)
         return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
@@ -352,6 +370,7 @@ dcut_status dcut_model_verify(dcut_ctx* c, const dcut_model* m, long long num_pa
                               int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total, int* row_argmax,
                               void* hidden_out, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (c->lim.hidden <= 0 || !c->ly_x[0]) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
     if (!m || !m->embed || !m->g_final || !m->w_lm || m->n_layers < 0 || (m->n_layers > 0 && (!m->layers || !m->k_caches || !m->v_caches)))
         return dcut_fail(c, DCUT_EINVAL, "incomplete model description");
@@ -392,6 +411,7 @@ dcut_status dcut_model_verify(dcut_ctx* c, const dcut_model* m, long long num_pa
 dcut_status dcut_commit(dcut_ctx* c, const int* accept_len, const int* out_tokens, int B, int gamma, int max_ctx,
                         int* ctx_lens, int* bonus_ids, int* stream_tokens, int* stream_len, int stream_cap, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (!accept_len || !out_tokens || !ctx_lens || !bonus_ids) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
     if ((stream_tokens != nullptr) != (stream_len != nullptr) || (stream_tokens && stream_cap < 1))
         return dcut_fail(c, DCUT_EINVAL, "stream_tokens, stream_len and stream_cap go together");
@@ -404,6 +424,7 @@ dcut_status dcut_commit(dcut_ctx* c, const int* accept_len, const int* out_token
 dcut_status dcut_gemm_bf16(dcut_ctx* c, const void* a, const void* w, const void* w2, int mode, int N, int K,
                            const int* cu_q, int B, int T_cap, void* out, const void* residual, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (!c->layer_maps) return dcut_fail(c, DCUT_EINVAL, "context was created without attention shapes (no tensor-map encoder)");
     if (!a || !w || !cu_q || !out || (mode == 2 && !w2) || (mode == 1 && !residual) || mode < 0 || mode > 2)
         return dcut_fail(c, DCUT_EINVAL, "null pointer or bad mode");
@@ -419,6 +440,7 @@ dcut_status dcut_lm_head_accept(dcut_ctx* c, const void* x, const void* w_lm, in
                                 const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
                                 int* out_tokens, int* n_accepted_total, int* row_argmax, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (c->lim.hidden <= 0 || !c->layer_maps) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
     if (!x || !w_lm || !draft_ids || !cu_q || !accept_len || !bonus) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
     if (V < 1 || c->lim.hidden % 64) return dcut_fail(c, DCUT_EINVAL, "need V >= 1 and hidden %% 64 == 0");
@@ -434,15 +456,15 @@ dcut_status dcut_lm_head_accept(dcut_ctx* c, const void* x, const void* w_lm, in
                                     n_accepted_total, row_argmax, c->d_row_key, s);
 }
 
-// first call (or a new theta): build the RoPE inverse-frequency table in fp64, round once to fp32
+// first call (or a new theta): build the RoPE inverse-frequency table in fp64, round once to fp32.  The host copy of
+// the table lives in the context: if this first call is being captured into a CUDA graph, the copy node reads it again
+// at every replay, and the context outlives the graph's use of it.
 static dcut_status dcut_prepare_rope(dcut_ctx* c, float rope_theta, cudaStream_t stream) {
     if (c->ly_theta == rope_theta) return DCUT_OK;
     const int half = c->lim.head_dim / 2;
-    float tab[128];
-    for (int e = 0; e < half; ++e) tab[e] = (float)pow((double)rope_theta, -2.0 * e / c->lim.head_dim);
-    // the table is read by kernels of this stream only; a pageable source is copied before the call returns
-    dcut_status st = dcut_check_cuda(c, cudaMemcpyAsync(c->ly_inv_freq, tab, sizeof(float) * half, cudaMemcpyHostToDevice, stream),
-                                     "cudaMemcpyAsync(inv_freq)");
+    for (int e = 0; e < half; ++e) c->ly_inv_freq_host[e] = (float)pow((double)rope_theta, -2.0 * e / c->lim.head_dim);
+    dcut_status st = dcut_check_cuda(c, cudaMemcpyAsync(c->ly_inv_freq, c->ly_inv_freq_host, sizeof(float) * half,
+                                                        cudaMemcpyHostToDevice, stream), "cudaMemcpyAsync(inv_freq)");
     if (st != DCUT_OK) return st;
     c->ly_theta = rope_theta;
     return DCUT_OK;
@@ -453,6 +475,7 @@ dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const v
                                const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
                                int T_cap, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (c->lim.hidden <= 0 || !c->ly_norm) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
     if (!w || !w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down || !w->g_attn || !w->g_mlp || !x || !y ||
         !k_cache || !v_cache || !block_table || !ctx_lens || !cu_q || !tok_req || !tok_pos)
@@ -538,6 +561,7 @@ dcut_status ensure_host_step_buffers(dcut_ctx* c, int V) {
 
 extern "C" dcut_status dcut_verify_step_host(dcut_ctx* c, const dcut_host_step* s, void* stream) {
     if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
     if (!s || !s->conf || !s->draft_ids || !s->bonus_ids || !s->ctx_lens || !s->block_table || !s->q_rows ||
         !s->logits_rows || !s->k_cache || !s->v_cache || !s->depths || !s->accept_len || !s->bonus || !s->out_tokens ||
         !s->n_accepted_total)

@@ -87,6 +87,7 @@ struct dcut_ctx {
     int ly_gemm_force;      // experiments: -1 = gemm_plan chooses; 0..6 a width on one SM; 8..14 on a pair
     unsigned ly_gemm_bn_mask;   // tile widths the one-SM mode may choose from (bit i: 256 - 32 i columns)
     float* ly_inv_freq;     // [head_dim / 2]
+    float ly_inv_freq_host[64];   // its host copy (head_dim <= 128), the source of the upload
     float ly_theta;         // theta the table was built for (0 = none yet)
     void* layer_maps;       // cached tensor maps (layer.cu)
 

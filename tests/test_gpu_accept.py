@@ -45,6 +45,30 @@ def test_workload_configs(idx, arms):
     ctx.close()
 
 
+def test_b256_full_depth_on_a_sub_batch():
+    """Workload 3 at full depth has 4352 rows of 151 936 logits (1.3 GB): the device scans all of them; the oracle
+    checks every fourth request (64 requests, 1088 rows) cut out of the same rows.  Rows are generated per (i, t),
+    so a request's rows are the same in the sub-batch."""
+    cfg = wl.config(3)
+    sel = wl.select_inputs(cfg)
+    depths = np.full(cfg.B, cfg.gamma, np.int32)
+    cu = wl.cu_q_from_depths(depths)
+    logits = wl.logits_rows(cfg, sel, depths)
+    ctx = make_ctx(cfg, n_q_heads=0)
+    al, bo, toks, total = ctx.accept(dev(logits), dev(sel.draft_ids), dev(cu), cfg.t_cap)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    al, bo, toks = al.cpu().numpy(), bo.cpu().numpy(), toks.cpu().numpy()
+    assert np.array_equal(al, np.minimum(sel.reject_index, depths))            # the planted acceptance, every request
+    assert int(total.item()) == int(al.sum()) + cfg.B
+    sub = np.arange(0, cfg.B, 4)
+    rows = np.concatenate([np.arange(cu[i], cu[i + 1]) for i in sub])
+    ref = orc.accept(logits[torch.from_numpy(rows)], sel.draft_ids[sub], wl.cu_q_from_depths(depths[sub]), cfg.gamma)
+    assert np.array_equal(al[sub], ref.accept_len) and np.array_equal(bo[sub], ref.bonus)
+    assert np.array_equal(toks[sub], ref.out_tokens)
+    ctx.close()
+
+
 def test_ties_nan_inf_signed_zero_rows():
     V = 4099                                   # odd: rows start at every 2-byte alignment
     rng = np.random.default_rng(4)

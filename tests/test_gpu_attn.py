@@ -213,3 +213,41 @@ def test_a_few_shallow_requests_among_deep_ones(shallow):
     assert 8 * pages[depths < 4].sum() < pages.sum()       # the rule applies
     kv = wl.paged_kv(cfg, sel.ctx_lens)
     _full_compare(cfg, sel, kv, depths)
+
+
+def test_block_table_entry_outside_the_cache_reads_page_0_and_is_reported():
+    """Device status 2.  A block-table entry outside [0, num_pages) must not become an address: the kernel reads
+    page 0 in its place, finishes, and the status word says so.  Every other input is valid, so nothing faults; the
+    requests whose tables are intact still match the oracle, and the context works normally afterwards."""
+    cfg = wl.custom_config(B=6, gamma=16, n_q_heads=8, n_kv_heads=2, head_dim=128, ctx_lo=40, ctx_hi=600)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    depths = np.array([0, 16, 3, 16, 0, 7], np.int32)         # request 0 runs on the warp-level phase, request 1 on tcgen05
+    bad = kv.block_table.copy()
+    bad[0, 1] = kv.num_pages + 5                              # past the cache
+    bad[1, 0] = -3                                            # negative, in a slot that is in use
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req)
+    q = wl.q_rows(cfg, depths)
+    cu = wl.cu_q_from_depths(depths)
+    args = (dev(q), dev(kv.k_cache), dev(kv.v_cache))
+    out = ctx.verify_attn(*args, dev(bad), dev(sel.ctx_lens), dev(cu), cfg.t_cap)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 2
+    assert torch.isfinite(out.float()).all()
+    # what the kernel computed is the attention over the table with page 0 substituted
+    sub = bad.copy()
+    sub[0, 1] = 0
+    sub[1, 0] = 0
+    ref, _ = orc.verify_attn(q, kv.k_cache, kv.v_cache, sub, sel.ctx_lens, cu, cfg.n_q_heads, cfg.n_kv_heads,
+                             cfg.head_dim, cfg.page_size)
+    ok, worst = attn_tolerance_ok(out.float().cpu().numpy(), ref)
+    assert ok, f"worst err/limit {worst}"
+    # the status word was cleared by the poll; a valid call on the same context is clean
+    out2 = ctx.verify_attn(*args, dev(kv.block_table), dev(sel.ctx_lens), dev(cu), cfg.t_cap)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    ref2, _ = orc.verify_attn(q, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, cu, cfg.n_q_heads, cfg.n_kv_heads,
+                              cfg.head_dim, cfg.page_size)
+    ok, worst = attn_tolerance_ok(out2.float().cpu().numpy(), ref2)
+    assert ok, f"worst err/limit {worst}"
+    ctx.close()

@@ -114,6 +114,22 @@ def test_full_layer_workload_on_sampled_requests():
     _layer_case(cfg, depths, cfg.hidden, cfg.intermediate, sub=[0, 1, 37])
 
 
+@pytest.mark.parametrize("arm", ["full_gamma", "T512"])
+def test_full_layer_workload_at_the_bench_s_packed_lengths(arm):
+    """The two packed lengths the benchmark times on the layer workload: T = 1088 (full depth: the length at which the
+    GEMM plan picks pair tiles for the wide projections) and T = 512 (the pruned arm: the selector forced to the
+    budget the profiled table leads to), through dcut_layer_forward at the full shapes, on three sampled requests."""
+    cfg = wl.config(4)
+    sel = wl.select_inputs(cfg)
+    if arm == "full_gamma":
+        depths = np.full(cfg.B, cfg.gamma, np.int32)
+    else:
+        depths = orc.select(sel.conf, sel.draft_ids, sel.bonus_ids, sel.ctx_lens, np.ones(1, np.float32), bucket_K=[512]).depths
+        assert int(depths.sum()) + cfg.B == 512
+    deep = int(np.argmax(depths))
+    _layer_case(cfg, depths, cfg.hidden, cfg.intermediate, sub=[2, deep, 61])
+
+
 @pytest.mark.parametrize("T,N,K,mode", [(300, 512, 1024, 0), (257, 256, 4096, 1), (640, 1024, 512, 2), (100, 256, 128, 0)])
 def test_single_sm_mode_matches_the_oracle(T, N, K, mode, monkeypatch):
     """The GEMM with its pair mode (cta_group::2) switched off when the context is created: single-SM tiles only.
@@ -246,4 +262,49 @@ def test_split_k_mode_at_every_tile_width(width_bit, mode, T, K, monkeypatch):
     want = orc.linear(a[:T], w) + (res[:T].double().numpy() if mode == 1 else 0.0)
     _close(out[:T], want, f"split-K, width bit {width_bit}, epilogue {mode}")
     assert (out[T:].float() == 7.0).all()
+    ctx.close()
+
+
+def test_first_layer_call_captured_in_a_graph_replays_correctly():
+    """The first layer call on a context uploads the RoPE frequency table from host memory.  Captured into a CUDA
+    graph, that upload is a node that runs again at every replay, so its source must outlive the call (it lives in
+    the context): two replays of a graph whose capture was the context's very first call equal the eager result."""
+    cfg = wl.custom_config(B=5, gamma=16, n_q_heads=4, n_kv_heads=2, head_dim=128, ctx_lo=5, ctx_hi=300, conf_kind="skew_halves")
+    hidden, inter = 512, 1024
+    depths = np.array([16, 0, 3, 9, 1], np.int32)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    w = wl.layer_weights(cfg, hidden, inter)
+    wd = {n: dev(getattr(w, n)) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")}
+    x = dev(wl.layer_x_rows(cfg, depths, hidden))
+    cu = dev(wl.cu_q_from_depths(depths))
+    tok_req = dev(np.concatenate([np.full(d + 1, i) for i, d in enumerate(depths)]).astype(np.int32))
+    tok_pos = dev(np.concatenate([sel.ctx_lens[i] + np.arange(d + 1) for i, d in enumerate(depths)]).astype(np.int32))
+    d_bt, d_ctx = dev(kv.block_table), dev(sel.ctx_lens)
+
+    def run(ctx, y, k, v):
+        ctx.layer_forward(wd, x, y, k, v, d_bt, d_ctx, cu, tok_req, tok_pos, cfg.t_cap, cfg.rms_eps, cfg.rope_theta)
+
+    eager_ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req, hidden=hidden, intermediate=inter, vocab=0)
+    y_eager = torch.empty((int(depths.sum()) + cfg.B, hidden), dtype=torch.bfloat16, device="cuda")
+    k_e, v_e = dev(kv.k_cache), dev(kv.v_cache)
+    run(eager_ctx, y_eager, k_e, v_e)
+    torch.cuda.synchronize()
+    eager_ctx.close()
+
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req, hidden=hidden, intermediate=inter, vocab=0)
+    y = torch.zeros_like(y_eager)
+    k_g, v_g = dev(kv.k_cache), dev(kv.v_cache)
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            run(ctx, y, k_g, v_g)                      # the context's first layer call happens inside the capture
+    torch.cuda.synchronize()
+    for _ in range(2):
+        y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.poll_device_status() == 0
+        assert torch.equal(y, y_eager) and torch.equal(k_g, k_e) and torch.equal(v_g, v_e)
     ctx.close()

@@ -166,6 +166,15 @@ def test_accept_rs_full_vocab_sub_batch():
     _check_rs(cfg, 151936, depths, noise=0.3)
 
 
+def test_accept_rs_b64_full_vocab():
+    """The batch size the benchmark times (B = 64, V = 151 936), ragged depths with both extremes."""
+    cfg = wl.custom_config(B=64, gamma=16, index=2, vocab=151936)
+    rng = np.random.default_rng(64)
+    depths = rng.integers(0, 17, 64).astype(np.int32)
+    depths[:4] = [16, 0, 16, 1]
+    _check_rs(cfg, 151936, depths, noise=0.3)
+
+
 def test_accept_rs_identical_distributions_accept_everything():
     cfg = wl.custom_config(B=5, gamma=6, index=305, vocab=500)
     sel = wl.select_inputs(cfg)
