@@ -1,6 +1,18 @@
-// Work list of the verification attention (split-KV flash-decoding plan), as a device function that runs in ONE CTA:
-// the stand-alone attn_plan_kernel of dcut_verify_attn, or the tail of the selector kernel, which has just written
-// cu_q and can leave the list ready for the attention call that follows (dcut_enable_plan_in_select).
+// Work partition of the verification attention, as a device function that runs in ONE CTA: the stand-alone
+// attn_plan_kernel of dcut_verify_attn, or the tail of the selector kernel, which has just written cu_q and can leave
+// the partition ready for the attention call that follows (dcut_enable_plan_in_select).
+//
+// The work of a call is a stream of (request, row block, kv head) items, each a run of KV pages; its cost is known
+// up front (pages x a per-page weight that depends on how the item runs, plus a fixed cost per item).  The stream is
+// cut into one segment of equal cost per SM: a CTA of the persistent item kernel owns a contiguous piece of the
+// stream, which may begin or end in the middle of an item.  An item that a boundary cuts is computed in pieces (one
+// per segment it touches) whose partial results the combine kernel merges; at most one item is cut per boundary, so
+// there are fewer cut items than SMs whatever the batch.  This replaces both the split of long contexts into chunks
+// for small batches and a dynamic item queue: every SM ends within the cost model's error of every other, and the
+// assignment (hence the rounding of every result) is the same on every run.
+//
+// The plan only writes the table of entries (one per (request, row block): n_kv_heads items of equal cost) and the
+// n_sm + 1 segment boundaries; the item kernel walks its segment and builds its items on the fly.
 #pragma once
 
 #include "dcut_internal.h"
@@ -8,19 +20,36 @@
 namespace dcut_plan {
 
 constexpr int kPage = 16;            // tokens per page
+constexpr int kSlotRows = 144;       // rows of a partial-result slot (the largest query tile of an item)
+constexpr int kMaxSegs = 256;        // segments (SMs) the plan handles
+
+// Cost model, nanoseconds on B200, fitted to the busy time of the item kernel's CTAs against the items and pages of
+// their segments (least squares over the 148 CTAs of batches of equal query tiles).  Per page: 168-171 on the
+// warp-level phase (4- and 8-row tiles), 186 on the tcgen05 phase at 68 rows, 209 at 136 rows (128 + tail rows).  Per
+// item, beyond its pages: 2.4-2.6 us on the warp-level phase, 4.4 us (68 rows) to 6.3 us (136 rows) on the tcgen05
+// phase, where Q and O are single-buffered in tensor memory and the pipeline drains at an item boundary.  Only ratios
+// matter for the partition.
+__device__ __forceinline__ int cost_per_page(int rows, int tc) {
+    if (tc) return rows > 128 ? 209 : 186;                 // every lane of tensor memory is processed, whatever the valid rows
+    const int mt = (rows + 15) >> 4;                       // m-tiles of the warp-level phase: memory-bound up to two
+    return 169 * max(7, 3 * mt) / 7;
+}
+__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 6300 : 4400) : 2500; }
 
 struct PlanArgs {
     const int* ctx_lens;
     const int* cu_q;
     int B, n_q_heads, n_kv_heads;
-    int target_items, min_chunk_pages, max_items, npad, tc_min_rows, max_item_rows;
+    int n_sm;                           // segments = CTAs of the item kernel
+    int min_chunk_pages;                // no piece of a cut item is shorter than this
+    int tc_min_rows, max_item_rows;
     int tail_rows;                      // a remainder of at most this many rows rides with the last full row block (0: never)
-    int tail_req_div, tail_min_pages;   // the shortest B / tail_req_div requests are cut finer (0: none)
-    long long part_rows_cap;
+    int max_entries;
     int* status;
-    AttnItem* items;
-    int* plan;       // [0] n_items, [1] chunk_pages, [2] total_pages, [3] partial rows used, [4] overflow, [5] n_tc, [8], [9] queue heads
-    int* req_part;   // [B][2]: first partial row, n_chunks
+    AttnEntry* entries;                 // [max_entries]
+    AttnSeg* segs;                      // [n_sm + 1]
+    AttnCut* cuts;                      // [n_sm]: entry b describes the merge the combine kernel does at boundary b
+    int* plan;                          // [0] n_entries, [1] first entry of the warp-level part, [2] total pages
 };
 
 template <typename T>
@@ -33,66 +62,23 @@ __device__ __forceinline__ T plan_warp_scan(T v, int lane) {
     return v;
 }
 
-// three exclusive scans over the CTA at once (one value of each per thread): prefixes in o0..o2, totals in t0..t2
-__device__ __forceinline__ void plan_block_exclusive_scan3(int v0, int v1, int v2, int (*ws)[33], int& o0, int& o1, int& o2,
-                                                           int& t0, int& t1, int& t2) {
+// exclusive scan over the CTA of one value per thread; prefix in `o`, total in `t` (`ws`: 33 values of shared memory)
+template <typename T>
+__device__ __forceinline__ void plan_block_exclusive_scan(T v, T* ws, T& o, T& t) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int i0 = plan_warp_scan(v0, lane), i1 = plan_warp_scan(v1, lane), i2 = plan_warp_scan(v2, lane);
-    if (lane == 31) {
-        ws[0][warp] = i0;
-        ws[1][warp] = i1;
-        ws[2][warp] = i2;
+    const T inc = plan_warp_scan(v, lane);
+    if (lane == 31) ws[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const T w = lane < (int)(blockDim.x >> 5) ? ws[lane] : T(0);
+        const T winc = plan_warp_scan(w, lane);
+        ws[lane] = winc - w;
+        if (lane == 31) ws[32] = winc;
     }
     __syncthreads();
-    if (warp < 3) {
-        const int w = lane < (int)(blockDim.x >> 5) ? ws[warp][lane] : 0;
-        const int winc = plan_warp_scan(w, lane);
-        ws[warp][lane] = winc - w;
-        if (lane == 31) ws[warp][32] = winc;
-    }
+    o = ws[warp] + inc - v;
+    t = ws[32];
     __syncthreads();
-    o0 = ws[0][warp] + i0 - v0;
-    o1 = ws[1][warp] + i1 - v1;
-    o2 = ws[2][warp] + i2 - v2;
-    t0 = ws[0][32];
-    t1 = ws[1][32];
-    t2 = ws[2][32];
-}
-
-// ascending bitonic sort of 32 E keys by one warp: lane l holds elements e * 32 + l
-template <int E>
-__device__ __forceinline__ void plan_warp_sort(unsigned long long* keys, int lane) {
-    unsigned long long k[E];
-#pragma unroll
-    for (int e = 0; e < E; ++e) k[e] = keys[e * 32 + lane];
-#pragma unroll
-    for (int kk = 2; kk <= 32 * E; kk <<= 1) {
-#pragma unroll
-        for (int j = kk >> 1; j > 0; j >>= 1) {
-            if (j >= 32) {                          // partner in the same lane
-                const int je = j >> 5;
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    if ((e & je) == 0) {
-                        const bool up = (((e * 32 + lane) & kk) == 0);
-                        const unsigned long long x = k[e], y = k[e | je];
-                        const bool swap = (x > y) == up;
-                        k[e] = swap ? y : x;
-                        k[e | je] = swap ? x : y;
-                    }
-                }
-            } else {                                // partner in another lane
-#pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, k[e], j);
-                    const bool keep_min = (((e * 32 + lane) & kk) == 0) == ((lane & j) == 0);
-                    k[e] = ((k[e] < other) == keep_min) ? k[e] : other;
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int e = 0; e < E; ++e) keys[e * 32 + lane] = k[e];
 }
 
 // Row blocks of a query tile of M rows: full blocks of max_rows rows and one remainder.  A remainder of at most
@@ -107,188 +93,189 @@ __device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, in
     return rb == n_rb - 1 ? M - rb * max_rows : max_rows;
 }
 
-// Requests are ordered by the estimated duration of their items, longest first, so the CTAs that
-// start last are the short ones (the hardware hands items to SMs in index order as SMs free up).
-// Every thread of the CTA calls this (it synchronises the CTA).  `order` is shared memory for a.npad 64-bit keys:
-// (inverted cost << 32 | request), sorted ascending.
-__device__ __forceinline__ void attn_plan_body(const PlanArgs& a, unsigned long long* order) {
-    __shared__ int ws3[3][33];
-    __shared__ int total_s, tail_s, w_tc_s, w_mma_s;
+// Every thread of the CTA calls this (it synchronises the CTA).  `prefix` is shared memory for 2 B + 1 64-bit values:
+// the cost of the stream before each entry.
+__device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* prefix) {
+    __shared__ long long ws64[33];
+    __shared__ int ws32[33];
+    __shared__ int total_s, w_tc_s, w_mma_s;
+    __shared__ AttnSeg seg_s[kMaxSegs + 1];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int group = a.n_q_heads / a.n_kv_heads;
     if (tid == 0) {
         total_s = 0;
-        tail_s = 0;
         w_tc_s = 0;
         w_mma_s = 0;
     }
     __syncthreads();
-    int local = 0, w_tc = 0, w_mma = 0;   // pages in all; pages whose items would go to the tcgen05 / warp-level queue
-    for (int i = tid; i < a.B; i += nthr) {
-        const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-        const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-        local += pages;
-        const int M = (d + 1) * group;
-        const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
-        int tc_rb = 0;
-        for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= a.tc_min_rows ? 1 : 0;
-        w_tc += pages * tc_rb;
-        w_mma += pages * (n_rb - tc_rb);
-    }
-    if (local) atomicAdd(&total_s, local);
-    if (w_tc) atomicAdd(&w_tc_s, w_tc);
-    if (w_mma) atomicAdd(&w_mma_s, w_mma);
-    __syncthreads();
-    const int total_pages = total_s;
-    const long long units = (long long)total_pages * a.n_kv_heads;
-    int chunk_pages = (int)((units + a.target_items - 1) / a.target_items);
-    if (chunk_pages < a.min_chunk_pages) chunk_pages = a.min_chunk_pages;
-
-    for (int i = tid; i < a.npad; i += nthr) {
-        unsigned long long key = ~0ull;
-        if (i < a.B) {
+    // pass 1: pages in all, and how they would split over the two phases of the item kernel
+    {
+        int local = 0, w_tc = 0, w_mma = 0;
+        for (int i = tid; i < a.B; i += nthr) {
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-            const int nc = (pages + chunk_pages - 1) / chunk_pages;
-            const int cp = (pages + nc - 1) / nc;
-            const int MT = ((d + 1) * group + 15) >> 4;
-            // per page: memory-bound below about two m-tiles, then time grows with the m-tiles
-            const unsigned int cost = (unsigned int)cp * (unsigned int)max(7, 3 * MT);
-            key = ((unsigned long long)(0xffffffffu - cost) << 32) | (unsigned int)i;
-        }
-        order[i] = key;
-    }
-    __syncthreads();
-    if (a.npad <= 256) {
-        // up to 256 requests: one warp sorts the keys in registers (element e * 32 + lane), without a single barrier
-        if (tid < 32) {
-            if (a.npad <= 32) plan_warp_sort<1>(order, tid);
-            else if (a.npad <= 64) plan_warp_sort<2>(order, tid);
-            else if (a.npad <= 128) plan_warp_sort<4>(order, tid);
-            else plan_warp_sort<8>(order, tid);
-        }
-        __syncthreads();
-    } else {
-        for (int k = 2; k <= a.npad; k <<= 1)
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                for (int t = tid; t < (a.npad >> 1); t += nthr) {
-                    const int i = 2 * t - (t & (j - 1)), l = i + j;
-                    const bool up = (i & k) == 0;
-                    const unsigned long long x = order[i], y = order[l];
-                    if ((x > y) == up) {
-                        order[i] = y;
-                        order[l] = x;
-                    }
-                }
-                __syncthreads();
-            }
-    }
-
-    // The items that start last decide how unevenly the SMs finish: the requests at the end of the order are cut
-    // into about target_items pieces altogether, so every SM ends on a short item.
-    const int n_tail = a.tail_req_div > 0 ? (a.B + a.tail_req_div - 1) / a.tail_req_div : 0;
-    const int tail_from = a.B - n_tail;
-    if (n_tail > 0) {   // (the same answer in every thread)
-        for (int j = tail_from + tid; j < a.B; j += nthr) {
-            const int i = (int)(order[j] & 0xffffffffu);
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            atomicAdd(&tail_s, (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage);
-        }
-        __syncthreads();
-    }
-    int tail_chunk = (int)(((long long)tail_s * a.n_kv_heads + a.target_items - 1) / a.target_items);
-    if (tail_chunk < a.tail_min_pages) tail_chunk = a.tail_min_pages;
-    if (tail_chunk > chunk_pages) tail_chunk = chunk_pages;
-
-    // The item kernel works through the tcgen05 queue first and the warp-level queue after it.  When the second
-    // holds only a small part of the pages (a few shallow requests among deep ones), its few long items would start
-    // late on a few SMs with the rest idle (measured at B = 64: +15 us per call while 3-8 % of the pages were in
-    // it): below one eighth of the pages everything goes to the tcgen05 queue.
-    const int tc_min_rows = (a.tc_min_rows <= a.max_item_rows && w_tc_s > 0 && 8LL * w_mma_s < (long long)w_tc_s + w_mma_s) ? 1 : a.tc_min_rows;
-
-    const int per = (a.B + nthr - 1) / nthr;
-    const int j0 = tid * per;
-    int my_tc = 0, my_mma = 0, my_rows = 0;
-    for (int e = 0; e < per; ++e) {
-        const int j = j0 + e;
-        if (j < a.B) {
-            const int i = (int)(order[j] & 0xffffffffu);
-            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
-            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
-            const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
-            const int nc = (pages + cpj - 1) / cpj;
-            // row blocks of the query tile: full blocks of max_item_rows rows and one remainder; each goes to the
-            // tcgen05 queue or to the warp-level queue by its number of rows
+            local += pages;
             const int M = (d + 1) * group;
             const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
             int tc_rb = 0;
-            for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= tc_min_rows ? 1 : 0;
-            my_tc += nc * a.n_kv_heads * tc_rb;
-            my_mma += nc * a.n_kv_heads * (n_rb - tc_rb);
-            if (nc > 1) my_rows += nc * (d + 1) * a.n_q_heads;
+            for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= a.tc_min_rows ? 1 : 0;
+            w_tc += pages * tc_rb;
+            w_mma += pages * (n_rb - tc_rb);
+        }
+        if (local) atomicAdd(&total_s, local);
+        if (w_tc) atomicAdd(&w_tc_s, w_tc);
+        if (w_mma) atomicAdd(&w_mma_s, w_mma);
+    }
+    __syncthreads();
+    // The item kernel runs a segment's tcgen05 items first and its warp-level items after them.  When the second kind
+    // holds only a small part of the pages (a few shallow requests among deep ones), every item takes the tcgen05
+    // path: one kind of item, one cost weight, and no switch of phase inside the CTAs.
+    const int tc_min_rows = (a.tc_min_rows <= a.max_item_rows && w_tc_s > 0 && 8LL * w_mma_s < (long long)w_tc_s + w_mma_s) ? 1 : a.tc_min_rows;
+
+    // pass 2: entries of each request in either part of the stream, and their cost
+    const int per = (a.B + nthr - 1) / nthr;
+    const int i0 = tid * per;
+    int my_tc = 0, my_mma = 0;
+    long long c_tc = 0, c_mma = 0;
+    for (int e = 0; e < per; ++e) {
+        const int i = i0 + e;
+        if (i < a.B) {
+            const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
+            const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
+            const int M = (d + 1) * group;
+            const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
+            for (int rb = 0; rb < n_rb; ++rb) {
+                const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
+                const int tc = rows >= tc_min_rows;
+                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc));
+                if (tc) {
+                    ++my_tc;
+                    c_tc += c;
+                } else {
+                    ++my_mma;
+                    c_mma += c;
+                }
+            }
         }
     }
-    int n_tc, n_mma, n_rows;
-    int tc_off, mma_off, row_off;
-    plan_block_exclusive_scan3(my_tc, my_mma, my_rows, ws3, tc_off, mma_off, row_off, n_tc, n_mma, n_rows);
-    const int n_items = n_tc + n_mma;
-    mma_off += n_tc;
-    const bool overflow = n_items > a.max_items || (long long)n_rows > a.part_rows_cap;
+    int off_tc, off_mma, n_tc, n_mma;
+    long long pre_tc, pre_mma, tot_tc, tot_mma;
+    plan_block_exclusive_scan<int>(my_tc, ws32, off_tc, n_tc);
+    plan_block_exclusive_scan<int>(my_mma, ws32, off_mma, n_mma);
+    plan_block_exclusive_scan<long long>(c_tc, ws64, pre_tc, tot_tc);
+    plan_block_exclusive_scan<long long>(c_mma, ws64, pre_mma, tot_mma);
+    const int n_entries = n_tc + n_mma;
+    const long long total = tot_tc + tot_mma;
+    const bool overflow = n_entries > a.max_entries;      // cannot happen with a context sized for the batch; defensive
     if (tid == 0) {
-        a.plan[0] = overflow ? 0 : n_items;
-        a.plan[1] = chunk_pages;
-        a.plan[2] = total_pages;
-        a.plan[3] = n_rows;
-        a.plan[4] = overflow ? 1 : 0;
-        a.plan[5] = overflow ? 0 : n_tc;     // items [0, n_tc): tcgen05 queue; [n_tc, n_items): warp-level queue
-        a.plan[8] = 0;                       // next item of the tcgen05 queue (claimed by the CTAs of the item kernel)
-        a.plan[9] = overflow ? 0 : n_tc;     // next item of the warp-level queue
+        a.plan[0] = overflow ? 0 : n_entries;
+        a.plan[1] = overflow ? 0 : n_tc;
+        a.plan[2] = total_s;
         if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
     }
-    if (overflow) return;
+    if (overflow) {
+        for (int s = tid; s <= a.n_sm; s += nthr) {
+            a.segs[s] = AttnSeg{0, 0, 0, 0};
+            if (s < a.n_sm) a.cuts[s] = AttnCut{0, 0, 0, 0, 0, {0, 0, 0}};
+        }
+        return;
+    }
+    off_mma += n_tc;
+    pre_mma += tot_tc;
     for (int e = 0; e < per; ++e) {
-        const int j = j0 + e;
-        if (j < a.B) {
-            const int i = (int)(order[j] & 0xffffffffu);
+        const int i = i0 + e;
+        if (i < a.B) {
             const int q0 = a.cu_q[i];
             const int d = a.cu_q[i + 1] - q0 - 1;
             const int ctx_len = a.ctx_lens[i];
             const int pages = (ctx_len + d + 1 + kPage - 1) / kPage;
-            const int cpj = j >= tail_from ? tail_chunk : chunk_pages;
-            const int nc = (pages + cpj - 1) / cpj;
-            const int cp = (pages + nc - 1) / nc;   // near-equal chunks
             const int M = (d + 1) * group;
-            a.req_part[2 * i] = row_off;
-            a.req_part[2 * i + 1] = nc;
-            // a query tile above max_item_rows (+ tail_rows) rows is cut into row blocks, each its own item over the
-            // same pages
             const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
-            for (int c = 0; c < nc; ++c)
-                for (int h = 0; h < a.n_kv_heads; ++h)
-                    for (int rb = 0; rb < n_rb; ++rb) {
-                        const int row0 = rb * a.max_item_rows, rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
-                        AttnItem it;
-                        it.req = i;
-                        it.kv_head = h;
-                        it.page_begin = c * cp;
-                        it.page_end = min(pages, (c + 1) * cp);
-                        it.n_chunks = nc;
-                        it.part_row = nc > 1 ? row_off + (c * a.n_kv_heads + h) * M + row0 : -1;
-                        it.q0 = q0;
-                        it.depth = d;
-                        it.ctx_len = ctx_len;
-                        const bool tc = rows >= tc_min_rows;
-                        it.pad[0] = tc ? 1 : 0;   // which queue the item is in
-                        it.pad[1] = row0;         // first query row of the item within the request's tile
-                        it.pad[2] = rows;         // query rows of the item
-                        a.items[tc ? tc_off++ : mma_off++] = it;
-                    }
-            if (nc > 1) row_off += nc * (d + 1) * a.n_q_heads;
+            for (int rb = 0; rb < n_rb; ++rb) {
+                const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
+                const int tc = rows >= tc_min_rows;
+                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc));
+                AttnEntry en;
+                en.req = i;
+                en.row0 = rb * a.max_item_rows;
+                en.rows = rows;
+                en.pages = pages;
+                en.q0 = q0;
+                en.depth = d;
+                en.ctx_len = ctx_len;
+                en.tc = tc;
+                const int idx = tc ? off_tc++ : off_mma++;
+                a.entries[idx] = en;
+                prefix[idx] = tc ? pre_tc : pre_mma;
+                if (tc) pre_tc += c; else pre_mma += c;
+            }
         }
+    }
+    if (tid == 0) prefix[n_entries] = total;
+    __syncthreads();
+    // segment boundaries: position s / n_sm of the total cost, mapped to (entry, kv head, page) and moved to the nearest
+    // place where an item may be cut (no piece shorter than min_chunk_pages; tcgen05 items at multiples of 4 pages)
+    for (int s = tid; s <= a.n_sm; s += nthr) {
+        AttnSeg sg = {n_entries, 0, 0, 0};
+        if (s == 0) {
+            sg.e = 0;                                        // the stream's beginning, whatever its first item looks like
+        } else if (s < a.n_sm && n_entries > 0) {
+            const long long pos = (total / a.n_sm) * s + (total % a.n_sm) * s / a.n_sm;
+            int lo = 0, hi = n_entries;                      // largest e < n_entries with prefix[e] <= pos
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (prefix[mid] <= pos) lo = mid; else hi = mid;
+            }
+            int e = lo;
+            const AttnEntry en = a.entries[e];               // written by this CTA before the barrier above
+            const long long item_cost = (prefix[e + 1] - prefix[e]) / a.n_kv_heads;
+            const long long rem = pos - prefix[e];
+            int h = (int)(rem / item_cost);
+            if (h >= a.n_kv_heads) h = a.n_kv_heads - 1;
+            const long long in_item = rem - (long long)h * item_cost - cost_per_item(en.rows, en.tc);
+            // Cuts inside an item fall on multiples of min_chunk_pages.  Two boundaries must never cut an item at the same
+            // page (the segment between them would hold an empty piece that nobody writes): consecutive positions are
+            // at least total / n_sm apart, so they land on different multiples as long as a segment is worth at least
+            // min_chunk_pages of this item; below that (tiny batches) the item is not cut at all.
+            const long long quantum = (long long)a.min_chunk_pages * cost_per_page(en.rows, en.tc);
+            int p = (in_item <= 0 || total / a.n_sm < quantum) ? 0 : (int)(in_item / quantum) * a.min_chunk_pages;
+            if (en.pages - p < a.min_chunk_pages) {          // the rest is too short to be a piece: the boundary moves to the next item
+                p = 0;
+                if (++h == a.n_kv_heads) {
+                    h = 0;
+                    ++e;
+                }
+            }
+            sg.e = e;
+            sg.h = h;
+            sg.p = p;
+        }
+        a.segs[s] = sg;
+        seg_s[s] = sg;
+    }
+    __syncthreads();
+    // what the combine kernel merges at each boundary: the item a boundary cuts is merged at the first boundary inside it
+    for (int b = tid; b < a.n_sm; b += nthr) {
+        AttnCut cut = {0, 0, 0, 0, 0, {0, 0, 0}};
+        const AttnSeg sg = seg_s[b];
+        if (b > 0 && sg.p > 0 && sg.e < n_entries) {
+            const AttnSeg pv = seg_s[b - 1];
+            if (!(pv.e == sg.e && pv.h == sg.h && pv.p > 0)) {
+                int m = 1;                                    // boundaries b .. b + m - 1 cut the item: m + 1 pieces
+                while (b + m < a.n_sm && seg_s[b + m].e == sg.e && seg_s[b + m].h == sg.h && seg_s[b + m].p > 0) ++m;
+                const AttnEntry en = a.entries[sg.e];
+                cut.pieces = m + 1;
+                cut.rows = en.rows;
+                cut.row0 = en.row0;
+                cut.q0 = en.q0;
+                cut.kv_head = sg.h;
+            }
+        }
+        a.cuts[b] = cut;
     }
 }
 
 }  // namespace dcut_plan
 
-// fills the arguments of the work-list builder for this batch from the context's shapes and scratch (verify_attn.cu)
+// fills the arguments of the partition builder for this batch from the context's shapes and scratch (verify_attn.cu)
 void dcut_fill_plan_args(dcut_ctx* ctx, const int* ctx_lens, const int* cu_q, int B, dcut_plan::PlanArgs* pa);

@@ -60,9 +60,10 @@ dcut_status dmalloc(dcut_ctx* ctx, T** p, size_t count, const char* what) {
 void free_all(dcut_ctx* c) {
     cudaFree(c->d_cost);
     cudaFree(c->d_bucket_K);
-    cudaFree(c->d_items);
+    cudaFree(c->d_entries);
+    cudaFree(c->d_segs);
+    cudaFree(c->d_cuts);
     cudaFree(c->d_plan);
-    cudaFree(c->d_req_part);
     cudaFree(c->d_part_o);
     cudaFree(c->d_part_lse);
     cudaFree(c->d_row_key);
@@ -149,28 +150,22 @@ dcut_status dcut_create(dcut_ctx** out, const dcut_limits* lim, int device) {
     if ((st = dcut_init_select(c)) != DCUT_OK) return st;
     if ((st = dcut_init_accept(c)) != DCUT_OK) return st;
     if (has_attn) {
-        const char* env = getenv("DCUT_ATTN_TARGET_ITEMS");
-        // Requests are cut along the context so that there are about this many work items when the batch has fewer
-        // (request, kv head) pairs.  13/8 of the SM count (240 on 148 SMs): the rounding of every request's cut adds a
-        // few items, and with 2 per SM as the aim those few made a third round on some SMs (B = 16: 2.7 TB/s with 296,
-        // 3.0 with 200-240, 2.9 with 148; no difference at B = 64, +1 % at B = 256).
-        c->target_items = env ? atoi(env) : c->sm_count * 13 / 8;
-        if (c->target_items < 1) c->target_items = 1;
-        env = getenv("DCUT_ATTN_TAIL_REQ_DIV");
-        c->attn_tail_req_div = env ? atoi(env) : 0;
-        env = getenv("DCUT_ATTN_TAIL_MIN_PAGES");
-        c->attn_tail_min_pages = env ? atoi(env) : 32;
-        if (c->attn_tail_min_pages < 8) c->attn_tail_min_pages = 8;
-        // whole-batch cut (<= target_items + pairs) + tail cut (<= target_items + pairs); x2: query tiles above 128
-        // rows are cut in two
-        c->max_items = 2 * (2 * lim->max_B * lim->n_kv_heads + 2 * c->target_items);
-        const int group = lim->n_q_heads / lim->n_kv_heads;
-        c->part_rows_cap = (long long)c->max_items * (lim->max_gamma + 1) * group;
-        if ((st = dmalloc(c, &c->d_items, c->max_items, "cudaMalloc(items)")) != DCUT_OK) return st;
+        // The work of a call is cut into one segment per SM (attn_plan.cuh): a table of at most two entries per request
+        // (row blocks of its query tile), the segment boundaries, and two partial-result slots per segment (an item cut
+        // by the segment's first boundary, one cut by its last).
+        const char* env = getenv("DCUT_ATTN_MIN_CHUNK_PAGES");
+        c->attn_min_chunk_pages = env ? atoi(env) : 8;
+        if (c->attn_min_chunk_pages < 4) c->attn_min_chunk_pages = 4;
+        c->attn_min_chunk_pages = (c->attn_min_chunk_pages + 3) & ~3;      // the tcgen05 phase works in groups of four pages
+        if (c->sm_count > 256) return dcut_fail(c, DCUT_ECAPACITY, "the attention work partition handles at most 256 SMs, this device has %d", c->sm_count);
+        c->max_entries = 2 * lim->max_B;
+        const size_t slots = 2 * (size_t)c->sm_count;
+        if ((st = dmalloc(c, &c->d_entries, c->max_entries, "cudaMalloc(attention entries)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->d_segs, (size_t)c->sm_count + 1, "cudaMalloc(attention segments)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->d_cuts, (size_t)c->sm_count + 1, "cudaMalloc(attention cuts)")) != DCUT_OK) return st;
         if ((st = dmalloc(c, &c->d_plan, 16, "cudaMalloc(plan)")) != DCUT_OK) return st;
-        if ((st = dmalloc(c, &c->d_req_part, 2 * (size_t)lim->max_B, "cudaMalloc(req_part)")) != DCUT_OK) return st;
-        if ((st = dmalloc(c, &c->d_part_o, (size_t)c->part_rows_cap * lim->head_dim, "cudaMalloc(part_o)")) != DCUT_OK) return st;
-        if ((st = dmalloc(c, &c->d_part_lse, (size_t)c->part_rows_cap, "cudaMalloc(part_lse)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->d_part_o, slots * 144 * lim->head_dim, "cudaMalloc(part_o)")) != DCUT_OK) return st;
+        if ((st = dmalloc(c, &c->d_part_lse, slots * 144, "cudaMalloc(part_lse)")) != DCUT_OK) return st;
         if ((st = dcut_init_verify_attn(c)) != DCUT_OK) return st;
     }
     if (lim->hidden > 0) {

@@ -20,7 +20,30 @@
 #define DCUT_DEV_BAD_TOKEN 6            // dcut_model_verify: a token id outside [0, vocab)
 #define DCUT_DEV_BAD_CU_Q 7             // acceptance: cu_q is not a packing of B requests of 1..gamma+1 rows within T_cap
 
-// One split-KV work item of the attention kernel: one (request, kv head, page range).
+// One row of the attention work table: a (request, row block of its query tile); it stands for n_kv_heads work items of
+// equal cost, one per kv head, each over the request's `pages` KV pages.
+struct __align__(16) AttnEntry {
+    int32_t req;
+    int32_t row0;         // first query row of the block within the request's tile
+    int32_t rows;         // query rows of the block
+    int32_t pages;        // KV pages of the request (context + retained tokens)
+    int32_t q0;           // cu_q[req]: first packed token of the request
+    int32_t depth;        // d_i
+    int32_t ctx_len;      // L_i
+    int32_t tc;           // 1: the items run on the tcgen05 phase of the item kernel, 0: on the warp-level phase
+};
+// A boundary between two segments of the work stream: before page `p` of the item (entry `e`, kv head `h`).
+struct __align__(16) AttnSeg {
+    int32_t e, h, p, pad;
+};
+
+// What the combine kernel does at boundary b (between segments b - 1 and b): nothing (pieces = 0), or merge the
+// `pieces` partial results of the item that boundaries b .. b + pieces - 2 cut (the item begins in segment b - 1).
+struct __align__(16) AttnCut {
+    int32_t pieces, rows, row0, q0, kv_head, pad[3];
+};
+
+// One work item of the attention kernel as a CTA runs it: one (request, kv head, page range).
 struct __align__(16) AttnItem {
     int32_t req;
     int32_t kv_head;
@@ -49,16 +72,14 @@ struct dcut_ctx {
     int bucket_B, bucket_gamma;
 
     // attention scratch
-    AttnItem* d_items;      // [max_items]
-    int* d_plan;            // [8] plan header: n_items, chunk_pages, ...
-    int* d_req_part;        // [max_B * 2]: first partial row / n_chunks per request
-    float* d_part_o;        // [part_rows_cap, head_dim] fp32
-    float* d_part_lse;      // [part_rows_cap]
-    int max_items;
-    long long part_rows_cap;
-    int target_items;
-    int attn_tail_req_div;  // the shortest max(1, B / this) requests are cut finer (0: none)
-    int attn_tail_min_pages;
+    AttnEntry* d_entries;   // [max_entries] work table (one row per (request, row block))
+    AttnSeg* d_segs;        // [sm_count + 1] segment boundaries of the work stream, one segment per CTA of the item kernel
+    AttnCut* d_cuts;        // [sm_count] per boundary: the cut item whose pieces the combine kernel merges there
+    int* d_plan;            // [16] plan header: n_entries, first warp-level entry, total pages
+    float* d_part_o;        // [2 * sm_count slots][144 rows][head_dim] fp32: partial results of the items a boundary cuts
+    float* d_part_lse;      // [2 * sm_count slots][144 rows]
+    int max_entries;
+    int attn_min_chunk_pages;   // no piece of a cut item is shorter than this
     int attn_tc_min_rows;   // items with at least this many query rows use the tcgen05 phase
     int attn_tail_rows;     // a query tile of up to 128 + this many rows stays one item (0: cut at 128)
     // work list left ready by the selector (dcut_enable_plan_in_select): the batch it was made for

@@ -361,15 +361,17 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
         // 6. the attention work list of the batch just packed: it depends on ctx_lens, cu_q and the shapes only, and
         // this CTA has them at hand, so the attention call that follows need not launch a one-CTA kernel of its own.
         // The sort keys are dead by now: their shared memory holds the plan's ordering keys (npad >= B entries).
-        // cu_q is at hand in shared memory (cu_s); ctx_lens joins it in the dead prefix-sum array
-        __syncthreads();            // nobody reads `keys` or `qs` any more
-        int* ctx_s = reinterpret_cast<int*>(qs);
+        // cu_q is at hand in shared memory (cu_s); ctx_lens joins it in the dead depth array.  The sort keys and the
+        // prefix sums are dead too: their contiguous shared memory (16 npad + 8 bytes, npad >= B) holds the plan's
+        // 2 B + 1 cost prefixes.
+        __syncthreads();            // nobody reads `keys`, `qs` or `depth_s` any more
+        int* ctx_s = depth_s;
         for (int i = tid; i < B; i += kThreads) ctx_s[i] = a.ctx_lens[i];
         __syncthreads();
         dcut_plan::PlanArgs pa = a.plan;
         pa.cu_q = cu_s;
         pa.ctx_lens = ctx_s;
-        dcut_plan::attn_plan_body(pa, keys);
+        dcut_plan::attn_plan_body(pa, reinterpret_cast<long long*>(keys));
     }
 }
 

@@ -147,18 +147,18 @@ __device__ __forceinline__ uint32_t tile_off_k4(int r, int c16) {
 using dcut_plan::PlanArgs;
 
 __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
-    extern __shared__ unsigned long long plan_order[];                // [npad] keys, then cu_q [B + 1] and ctx_lens [B]
+    extern __shared__ long long plan_prefix[];                        // [2 B + 1] cost prefixes, then cu_q [B + 1] and ctx_lens [B]
     dcut_pdl_wait();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the item kernel's CTAs may take their SMs now
     // the body reads every request's cu_q and ctx_lens several times: from shared memory, not through L2
-    int* cu_s = reinterpret_cast<int*>(plan_order + a.npad);
+    int* cu_s = reinterpret_cast<int*>(plan_prefix + 2 * a.B + 1);
     int* ctx_s = cu_s + a.B + 1;
     for (int i = threadIdx.x; i <= a.B; i += blockDim.x) cu_s[i] = a.cu_q[i];
     for (int i = threadIdx.x; i < a.B; i += blockDim.x) ctx_s[i] = a.ctx_lens[i];
     __syncthreads();
     a.cu_q = cu_s;
     a.ctx_lens = ctx_s;
-    dcut_plan::attn_plan_body(a, plan_order);                         // 256 threads for small batches: cheaper barriers
+    dcut_plan::attn_plan_body(a, plan_prefix);                        // 256 threads for small batches: cheaper barriers
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -286,8 +286,9 @@ struct AttnArgs {
     int block_table_stride;
     const int* ctx_lens;
     const int* cu_q;
-    const AttnItem* items;
-    int* plan;
+    const AttnEntry* entries;  // work table and segment boundaries (attn_plan.cuh)
+    const AttnSeg* segs;
+    const int* plan;
     int n_q_heads, n_kv_heads;
     long long num_pages;
     float scale_log2;          // softmax scale * log2(e)
@@ -337,18 +338,58 @@ __device__ __forceinline__ bool bar_any(int id, int nthreads, bool pred) {
     return r != 0;
 }
 
-// Scheduler, producer side (whole warp, converged): claims the next item of the phase from the global counter and
-// posts it in slot n & 1 of the CTA's queue.  idx = -1 when the phase has no items left.
-__device__ __forceinline__ bool sched_fetch(Ctrl* c, const AttnArgs& a, int phase, int n, int* counter, int end,
+// Position in the work stream (entry, kv head, page), and the end of what this CTA runs in the current phase.
+struct SegCursor {
+    int e, h, p;
+    int e1, h1, p1;
+};
+__device__ __forceinline__ bool seg_before(int e, int h, int p, int e1, int h1, int p1) {
+    return e < e1 || (e == e1 && (h < h1 || (h == h1 && p < p1)));
+}
+// the part of this CTA's segment [s0, s1) that lies in [lo, hi) entries of the table (one phase of the kernel)
+__device__ __forceinline__ SegCursor seg_range(const AttnSeg& s0, const AttnSeg& s1, int e_lo, int e_hi) {
+    SegCursor c;
+    if (s0.e < e_lo) { c.e = e_lo; c.h = 0; c.p = 0; } else { c.e = s0.e; c.h = s0.h; c.p = s0.p; }
+    if (s1.e >= e_hi) { c.e1 = e_hi; c.h1 = 0; c.p1 = 0; } else { c.e1 = s1.e; c.h1 = s1.h; c.p1 = s1.p; }
+    return c;
+}
+
+// Scheduler, producer side (whole warp, converged): builds the next item of this CTA's segment and posts it in slot
+// n & 1 of the CTA's queue.  idx = -1 when the phase has no items left.  An item that a segment boundary cuts covers
+// only this segment's pages of it and leaves a partial result in one of the segment's two slots: slot 2 s when the
+// item began in an earlier segment, slot 2 s + 1 when it begins here and continues in the next.
+__device__ __forceinline__ bool sched_fetch(Ctrl* c, const AttnArgs& a, int phase, int n, SegCursor& cur,
                                             AttnItem& it, int& idx) {
     const int slot = n & 1, lane = threadIdx.x & 31;
     if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(smem_u32(&c->sched_empty[phase][slot]), ((n >> 1) - 1) & 1, &c->abort)))
         return false;
-    int i = 0;
-    if (lane == 0) i = atomicAdd(counter, 1);
-    i = __shfl_sync(0xffffffffu, i, 0);
-    idx = i < end ? i : -1;
-    if (idx >= 0) it = a.items[idx];
+    idx = seg_before(cur.e, cur.h, cur.p, cur.e1, cur.h1, cur.p1) ? n : -1;
+    if (idx >= 0) {
+        const AttnEntry en = a.entries[cur.e];
+        const bool last = cur.e == cur.e1 && cur.h == cur.h1;      // the segment ends inside this item
+        it.req = en.req;
+        it.kv_head = cur.h;
+        it.page_begin = cur.p;
+        it.page_end = last ? cur.p1 : en.pages;
+        const bool whole = it.page_begin == 0 && it.page_end == en.pages;
+        it.n_chunks = whole ? 1 : 2;
+        it.part_row = whole ? -1 : (2 * (int)blockIdx.x + (cur.p > 0 ? 0 : 1)) * dcut_plan::kSlotRows;
+        it.q0 = en.q0;
+        it.depth = en.depth;
+        it.ctx_len = en.ctx_len;
+        it.pad[0] = en.tc;
+        it.pad[1] = en.row0;      // first query row of the item within the request's tile
+        it.pad[2] = en.rows;      // query rows of the item
+        if (last) {
+            cur.p = cur.p1;
+        } else {
+            cur.p = 0;
+            if (++cur.h == a.n_kv_heads) {
+                cur.h = 0;
+                ++cur.e;
+            }
+        }
+    }
     if (lane == 0) {
         c->item_idx[slot] = idx;
         if (idx >= 0) c->item[slot] = it;
@@ -381,7 +422,7 @@ __device__ __forceinline__ void sched_release(Ctrl* c, int phase, int n) {
 
 template <int DH>
 __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtensorMap& v_map, const AttnArgs& a,
-                                          unsigned char* smem, Ctrl* c, int* counter, int end) {
+                                          unsigned char* smem, Ctrl* c, SegCursor cur) {
     using L = MmaSmem<DH>;
     unsigned char* ring = smem;
     float* merge = reinterpret_cast<float*>(smem + L::kRingBytes);
@@ -404,7 +445,7 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
         // ---------------------------------------------------------------- producer warp
         for (int n = 0;; ++n) {
             int idx;
-            if (!sched_fetch(c, a, kPhase, n, counter, end, item, idx)) {
+            if (!sched_fetch(c, a, kPhase, n, cur, item, idx)) {
                 failed = true;
                 break;
             }
@@ -722,7 +763,7 @@ __device__ __forceinline__ void mma_phase(const CUtensorMap& k_map, const CUtens
 // through the q_ready and o_free barriers.
 __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtensorMap& v_map, const AttnArgs& a,
                                          unsigned char* ring, float* tail_buf, Ctrl* c, float (*xm)[128],
-                                         float (*xl)[128], int* counter, int end) {
+                                         float (*xl)[128], SegCursor cur) {
     constexpr int kPhase = 0;
     const uint32_t full_bar = smem_u32(c->ring_full), empty_bar = smem_u32(c->ring_empty);
     const uint32_t s_full = smem_u32(c->s_full), p_full = smem_u32(c->p_full), pv_done = smem_u32(c->pv_done);
@@ -741,7 +782,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
         // load, which made the producer the slowest role).
         for (int n = 0;; ++n) {
             int idx;
-            if (!sched_fetch(c, a, kPhase, n, counter, end, item, idx)) {
+            if (!sched_fetch(c, a, kPhase, n, cur, item, idx)) {
                 failed = true;
                 break;
             }
@@ -1505,14 +1546,18 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
     // launched with programmatic stream serialization: everything above overlaps the plan kernel; nothing it writes
     // is read before this wait
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int n_items = a.plan[0], n_tc = a.plan[5];
-    if (DH == 128 && n_tc > 0) {
-        tc_phase(k2_map, v_map, a, smem, reinterpret_cast<float*>(smem + kDataBytes<DH>), c, xm, xl, a.plan + 8, n_tc);
+    // this CTA's segment of the work stream: its tcgen05 items first, then its warp-level items
+    const int n_entries = a.plan[0], e_split = a.plan[1];
+    const AttnSeg s0 = a.segs[blockIdx.x], s1 = a.segs[blockIdx.x + 1];
+    const SegCursor tc_cur = seg_range(s0, s1, 0, e_split), mma_cur = seg_range(s0, s1, e_split, n_entries);
+    if (DH == 128 && seg_before(tc_cur.e, tc_cur.h, tc_cur.p, tc_cur.e1, tc_cur.h1, tc_cur.p1)) {
+        tc_phase(k2_map, v_map, a, smem, reinterpret_cast<float*>(smem + kDataBytes<DH>), c, xm, xl, tc_cur);
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
     }
-    if (n_items > n_tc && !ABORTED(c)) mma_phase<DH>(k_map, v_map, a, smem, c, a.plan + 9, n_items);
+    if (seg_before(mma_cur.e, mma_cur.h, mma_cur.p, mma_cur.e1, mma_cur.h1, mma_cur.p1) && !ABORTED(c))
+        mma_phase<DH>(k_map, v_map, a, smem, c, mma_cur);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the combine kernel may take this SM
     tc_fence_before();
     __syncthreads();
@@ -1523,69 +1568,59 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
 }
 
 // ------------------------------------------------------------------------------------------------
-// combine the chunks of multi-chunk requests: one warp per (token, q head)
+// combine the pieces of the items that segment boundaries cut: one CTA per boundary
 
 struct CombineArgs {
-    const int* cu_q;
-    const int* req_part;
+    const AttnCut* cuts;
     const float* part_o;
     const float* part_lse;
-    int* plan;   // read; the two queue heads are rewound
-    int B, n_q_heads, n_kv_heads, tokens_per_req;
+    int n_q_heads, n_kv_heads;
     __nv_bfloat16* out;
     float* lse;
 };
 
 template <int DH>
 __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
-    // grid: x = request * (gamma_max + 1) + block position t, y = group of blockDim.x / 32 q heads; warp = one head.
+    // grid: x: boundary b = blockIdx.x + 1 between segments b - 1 and b; y: block of 32 query rows; a warp merges one row
+    // (the loads of a row depend on one another, so the rows must not queue up behind each other).
     // Launched with programmatic stream serialization (see attn_item_kernel).
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
-        // the item kernel has drained both queues: rewind them, so that the same plan can serve another launch over
-        // the same batch (the layers of one model forward)
-        a.plan[8] = 0;
-        a.plan[9] = a.plan[5];
-    }
-    if (a.plan[4] || a.plan[3] == 0) return;   // overflow, or no request was cut: nothing to merge
-    const int lane = threadIdx.x & 31;
-    const int h = blockIdx.y * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (h >= a.n_q_heads) return;
-    // grid-stride over (request, block position): the grid is capped at two CTAs per SM so that the usual case of an
-    // uncut batch costs a few hundred CTA launches, not B * (gamma + 1)
-    for (int k = blockIdx.x; k < a.B * a.tokens_per_req; k += gridDim.x) {
-    const int req = k / a.tokens_per_req, t = k - req * a.tokens_per_req;
-    const int nc = a.req_part[2 * req + 1];
-    if (nc <= 1 || t >= a.cu_q[req + 1] - a.cu_q[req]) continue;
-    const int tok = a.cu_q[req] + t;
+    const int b = blockIdx.x + 1;
+    const AttnCut en = a.cuts[b];
+    if (en.pieces == 0 || (int)blockIdx.y * 32 >= en.rows) return;   // no item to merge at this boundary, or no rows for this block
+    const int m = en.pieces - 1;
+    struct { int h; } sg = {en.kv_head};
     const int group = a.n_q_heads / a.n_kv_heads;
-    const int q0 = a.cu_q[req];
-    const int M = (a.cu_q[req + 1] - q0) * group;
-    const int kvh = h / group;
-    const int R = (tok - q0) * group + (h - kvh * group);
-    const size_t base = (size_t)a.req_part[2 * req];
-    float m_all = -INFINITY;
-    for (int c = 0; c < nc; ++c) m_all = fmaxf(m_all, a.part_lse[base + (size_t)(c * a.n_kv_heads + kvh) * M + R]);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int kPer = DH / 32;
-    float acc[kPer];
+    for (int R = blockIdx.y * 32 + warp; R < en.rows; R += 32 * gridDim.y) {
+        // piece 0 is in segment b - 1 (the item begins there: its second slot); piece c >= 1 in segment b + c - 1 (first slot)
+        float m_all = -INFINITY;
+        for (int c = 0; c <= m; ++c) {
+            const size_t prow = (size_t)(c == 0 ? 2 * (b - 1) + 1 : 2 * (b + c - 1)) * dcut_plan::kSlotRows + R;
+            m_all = fmaxf(m_all, a.part_lse[prow]);
+        }
+        float acc[kPer];
 #pragma unroll
-    for (int e = 0; e < kPer; ++e) acc[e] = 0.0f;
-    float wsum = 0.0f;
-    for (int c = 0; c < nc; ++c) {
-        const size_t prow = base + (size_t)(c * a.n_kv_heads + kvh) * M + R;
-        const float l = a.part_lse[prow];
-        const float w = (l == -INFINITY) ? 0.0f : __expf(l - m_all);
-        wsum += w;
-        const float* po = a.part_o + prow * DH + lane * kPer;
+        for (int e = 0; e < kPer; ++e) acc[e] = 0.0f;
+        float wsum = 0.0f;
+        for (int c = 0; c <= m; ++c) {
+            const size_t prow = (size_t)(c == 0 ? 2 * (b - 1) + 1 : 2 * (b + c - 1)) * dcut_plan::kSlotRows + R;
+            const float l = a.part_lse[prow];
+            const float w = (l == -INFINITY) ? 0.0f : __expf(l - m_all);
+            wsum += w;
+            const float* po = a.part_o + prow * DH + lane * kPer;
 #pragma unroll
-        for (int e = 0; e < kPer; ++e) acc[e] += w * po[e];
-    }
-    const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
-    __nv_bfloat16* op = a.out + ((size_t)tok * a.n_q_heads + h) * DH + lane * kPer;
+            for (int e = 0; e < kPer; ++e) acc[e] += w * po[e];
+        }
+        const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+        const int t = (en.row0 + R) / group, hl = (en.row0 + R) - t * group;
+        const size_t orow = (size_t)(en.q0 + t) * a.n_q_heads + sg.h * group + hl;
+        __nv_bfloat16* op = a.out + orow * DH + lane * kPer;
 #pragma unroll
-    for (int e = 0; e < kPer; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
-    if (a.lse && lane == 0) a.lse[(size_t)tok * a.n_q_heads + h] = wsum > 0.0f ? m_all + logf(wsum) : -INFINITY;
+        for (int e = 0; e < kPer; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
+        if (a.lse && lane == 0) a.lse[orow] = wsum > 0.0f ? m_all + logf(wsum) : -INFINITY;
     }
 }
 
@@ -1631,10 +1666,9 @@ dcut_status launch_t(dcut_ctx* ctx, const CUtensorMap& km, const CUtensorMap& vm
     dcut_status st = dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, attn_item_kernel<DH>, km, vm, k2m, aa), "launch attn_item_kernel");
     if (st != DCUT_OK) return st;
     (void)T_cap;
-    const int heads_per_cta = ctx->lim.n_q_heads < 32 ? ((ctx->lim.n_q_heads + 7) / 8) * 8 : 32;
-    const int cgrid = ca.B * ca.tokens_per_req < 2 * ctx->sm_count ? ca.B * ca.tokens_per_req : 2 * ctx->sm_count;
-    lc.gridDim = dim3(cgrid, (ctx->lim.n_q_heads + heads_per_cta - 1) / heads_per_cta);
-    lc.blockDim = dim3(32 * heads_per_cta);
+    if (ctx->sm_count < 2) return DCUT_OK;      // one segment: no boundary, nothing to merge
+    lc.gridDim = dim3(ctx->sm_count - 1, (dcut_plan::kSlotRows + 31) / 32);
+    lc.blockDim = dim3(1024);
     lc.dynamicSmemBytes = 0;
     return dcut_check_cuda(ctx, cudaLaunchKernelEx(&lc, attn_combine_kernel<DH>, ca), "launch attn_combine_kernel");
 }
@@ -1652,7 +1686,7 @@ dcut_status dcut_init_verify_attn(dcut_ctx* ctx) {
         env = getenv("DCUT_ATTN_TAIL_ROWS");     // 0: a query tile above 128 rows becomes two items (experiments)
         ctx->attn_tail_rows = env ? (atoi(env) > 0 ? kTcTailRows : 0) : kTcTailRows;
     }
-    e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * DCUT_MAX_KEYS + 4 * (2 * DCUT_MAX_KEYS + 1));
+    e = cudaFuncSetAttribute(attn_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * (2 * DCUT_MAX_KEYS + 1) + 4 * (2 * DCUT_MAX_KEYS + 1));
     if (e != cudaSuccess) return dcut_check_cuda(ctx, e, "cudaFuncSetAttribute(attn plan)");
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -1670,21 +1704,17 @@ void dcut_fill_plan_args(dcut_ctx* ctx, const int* ctx_lens, const int* cu_q, in
     pa.B = B;
     pa.n_q_heads = ctx->lim.n_q_heads;
     pa.n_kv_heads = ctx->lim.n_kv_heads;
-    pa.target_items = ctx->target_items;
-    pa.min_chunk_pages = 8;
-    pa.tail_req_div = ctx->attn_tail_req_div;
-    pa.tail_min_pages = ctx->attn_tail_min_pages;
-    pa.npad = 32;
-    while (pa.npad < B) pa.npad <<= 1;
+    pa.n_sm = ctx->sm_count;
+    pa.min_chunk_pages = ctx->attn_min_chunk_pages;
     pa.status = ctx->d_status;
     pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
     pa.max_item_rows = 128;
     pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? ctx->attn_tail_rows : 0;
-    pa.max_items = ctx->max_items;
-    pa.part_rows_cap = ctx->part_rows_cap;
-    pa.items = ctx->d_items;
+    pa.max_entries = ctx->max_entries;
+    pa.entries = ctx->d_entries;
+    pa.segs = ctx->d_segs;
+    pa.cuts = ctx->d_cuts;
     pa.plan = ctx->d_plan;
-    pa.req_part = ctx->d_req_part;
 }
 
 dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_cache, const void* v_cache,
@@ -1718,7 +1748,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     if (!reuse_plan) {   // reuse_plan: the previous launch on this stream had the same ctx_lens, cu_q and B (its work list stands)
         ctx->plan_cu_q = nullptr;   // the list now belongs to this call's batch
         st = dcut_check_cuda(ctx, dcut_launch_pdl(attn_plan_kernel, dim3(1), dim3(B <= 256 ? 256 : kPlanThreads),
-                                                  sizeof(unsigned long long) * pa.npad + sizeof(int) * (2 * B + 1), stream, pa),
+                                                  sizeof(long long) * (2 * B + 1) + sizeof(int) * (2 * B + 1), stream, pa),
                              "launch attn_plan_kernel");
         if (st != DCUT_OK) return st;
     }
@@ -1729,7 +1759,8 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     aa.block_table_stride = block_table_stride;
     aa.ctx_lens = ctx_lens;
     aa.cu_q = cu_q;
-    aa.items = ctx->d_items;
+    aa.entries = ctx->d_entries;
+    aa.segs = ctx->d_segs;
     aa.plan = ctx->d_plan;
     aa.n_q_heads = ctx->lim.n_q_heads;
     aa.n_kv_heads = ctx->lim.n_kv_heads;
@@ -1742,15 +1773,11 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     aa.status = ctx->d_status;
 
     CombineArgs ca;
-    ca.cu_q = cu_q;
-    ca.req_part = ctx->d_req_part;
+    ca.cuts = ctx->d_cuts;
     ca.part_o = ctx->d_part_o;
     ca.part_lse = ctx->d_part_lse;
-    ca.plan = ctx->d_plan;
-    ca.B = B;
     ca.n_q_heads = ctx->lim.n_q_heads;
     ca.n_kv_heads = ctx->lim.n_kv_heads;
-    ca.tokens_per_req = ctx->lim.max_gamma + 1;
     ca.out = static_cast<__nv_bfloat16*>(out);
     ca.lse = lse;
 

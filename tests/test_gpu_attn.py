@@ -173,7 +173,9 @@ def test_kv_head_sharding_reproduces_the_unsharded_result(tp):
     """Tensor-parallel sharding of the attention step as the paper's TP deployments would do it: rank r owns kv heads
     r * Hkv/tp .. and their query heads, holds its own slice of the paged cache, and runs the same call on a context
     created for its share of the heads; no exchange inside the step.  Heads are independent, so the concatenated
-    shards equal the unsharded output bit for bit (the ranks run one after the other here, on one GPU)."""
+    shards equal the unsharded output up to rounding: a shard's work is cut into per-SM segments at other places than
+    the unsharded call's, so the few items a boundary cuts merge their pieces in a different split (the ranks run one
+    after the other here, on one GPU)."""
     cfg = wl.custom_config(B=9, gamma=16, n_q_heads=16, n_kv_heads=4, head_dim=128, ctx_lo=3, ctx_hi=900)
     sel = wl.select_inputs(cfg)
     kv = wl.paged_kv(cfg, sel.ctx_lens)
@@ -194,7 +196,12 @@ def test_kv_head_sharding_reproduces_the_unsharded_result(tp):
         assert ctx.poll_device_status() == 0
         ctx.close()
         outs.append(out.float().cpu().numpy())
-    assert np.array_equal(np.concatenate(outs, axis=1), full)
+    got = np.concatenate(outs, axis=1)
+    assert np.abs(got - full).max() <= 1e-2 and (got == full).mean() > 0.5       # rounding-level differences, and only in the cut items
+    ref, _ = orc.verify_attn(q, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, cu, cfg.n_q_heads, cfg.n_kv_heads,
+                             cfg.head_dim, cfg.page_size)
+    ok, worst = attn_tolerance_ok(got, ref)
+    assert ok, f"worst err/limit {worst}"
 
 
 @pytest.mark.parametrize("shallow", [[0, 0], [1, 3], [2]])
