@@ -917,6 +917,28 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
         const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
         const uint32_t t_mine = t_lane + kTcColOB * team, t_other = t_lane + kTcColOB * (team ^ 1);
         const float cs = a.scale_log2;
+        // an item's query tile goes to tensor memory: row R = lane of tensor memory, 128 bf16 = 64 words, 32 per team
+        auto store_q = [&](const AttnItem& it) {
+            uint32_t qw[32];
+            const int rows = min(it.pad[2], 128);
+            if (R < rows) {
+                const int t = (it.pad[1] + R) / group, hl = (it.pad[1] + R) - t * group;
+                const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(it.q0 + t) * a.n_q_heads + it.kv_head * group + hl) * 128) + 8 * team;
+#pragma unroll
+                for (int cc = 0; cc < 8; ++cc) {
+                    const uint4 v = src[cc];
+                    qw[4 * cc] = v.x; qw[4 * cc + 1] = v.y; qw[4 * cc + 2] = v.z; qw[4 * cc + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int cc = 0; cc < 32; ++cc) qw[cc] = 0;
+            }
+            tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * team, qw);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(q_ready);
+        };
+        bool q_staged = false;                   // this item's query tile was stored while the previous item was finishing
         for (int n = 0;; ++n) {
             const int idx = sched_wait(c, kPhase, n, item);
             if (idx == -2) failed = true;
@@ -929,27 +951,8 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             const int row0 = item.pad[1], M = min(item.pad[2], 128);   // this item's rows of the request's query tile (rows past 128: tail warps)
             const int n_pages = item.page_end - item.page_begin;
             const int n_groups = (n_pages + 3) >> 2;
-            {
-                // the query tile goes to tensor memory (every MMA of the previous item has completed: both teams
-                // waited for its last PV): row R = lane of tensor memory, 128 bf16 = 64 words, 32 per team
-                uint32_t qw[32];
-                if (R < M) {
-                    const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
-                    const uint4* src = reinterpret_cast<const uint4*>(a.q + ((size_t)(q0 + t) * a.n_q_heads + kvh * group + hl) * 128) + 8 * team;
-#pragma unroll
-                    for (int cc = 0; cc < 8; ++cc) {
-                        const uint4 v = src[cc];
-                        qw[4 * cc] = v.x; qw[4 * cc + 1] = v.y; qw[4 * cc + 2] = v.z; qw[4 * cc + 3] = v.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int cc = 0; cc < 32; ++cc) qw[cc] = 0;
-                }
-                tc_st32(tmem_q + ((uint32_t)(quarter * 32) << 16) + 32 * team, qw);
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(q_ready);
-            }
+            if (!q_staged) store_q(item);
+            q_staged = false;
             const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
             float m_run = -INFINITY, l_run = 0.0f;
             for (int g = team; g < n_groups; g += 2) {
@@ -1021,9 +1024,24 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                 tc_fence_before();
                 mbar_arrive(p_full + 8 * b);
             }
+            const int gl = G0 + n_groups - 1;
+            // The next item's query tile, before this item's epilogue: Q's columns are free as soon as the last QK^T of
+            // this item has completed (s_full of its last group; the team that did not own that group waits for it
+            // here), and the scheduler posted the next item when it issued this item's last load.  The MMA warp can
+            // then issue the next item's first QK^T products while the epilogue below runs, instead of after it.
+            if (!failed) {
+                AttnItem nxt;
+                const int idx_n = sched_wait(c, kPhase, n + 1, nxt);
+                if (idx_n == -2) failed = true;
+                if (idx_n >= 0 && !mbar_wait(s_full + 8 * (gl % kTcSBufs), (gl / kTcSBufs) & 1, &c->abort)) failed = true;
+                if (!__any_sync(0xffffffffu, failed) && idx_n >= 0) {
+                    tc_fence_after();
+                    store_q(nxt);
+                    q_staged = true;
+                }
+            }
             // epilogue: every MMA of the item has completed once its last PV has; the two teams' (m, l, O) are merged
             // and normalised; this thread writes columns [64 * team, 64 * team + 64) of its row
-            const int gl = G0 + n_groups - 1;
             if (!failed && !mbar_wait(pv_done + 8 * (gl % kTcSBufs), (gl / kTcSBufs) & 1, &c->abort)) failed = true;
             failed = __any_sync(0xffffffffu, failed);
             tc_fence_after();
