@@ -209,6 +209,33 @@ dcut_status dcut_layer_forward(dcut_ctx* ctx, const dcut_layer_weights* weights,
                                int T_cap, void* stream);
 
 /*
+ * The decoder layer cut where a tensor-parallel deployment exchanges (Appendix D runs the targets at TP 1/4/8).  A
+ * rank holds its share of the heads and of the MLP width: w_qkv = the rows of its q heads, then of its k heads, then
+ * of its v heads; w_o = the matching columns [hidden, n_q_heads_local * head_dim]; w_gate / w_up = its rows
+ * [intermediate_local, hidden]; w_down = the matching columns [hidden, intermediate_local]; its own slice of the paged
+ * cache [num_pages, n_kv_heads_local, page, head_dim]; a context created with the LOCAL head counts and intermediate
+ * width and the full hidden size.  Every rank runs
+ *     dcut_layer_attn_part:  o_part = Attn(RoPE(Wqkv . RMSNorm(x))) . Wo^T      (no residual)
+ *     -- all-reduce (sum) of o_part over the ranks: the caller's exchange --
+ *     dcut_residual_add:     h1 = x + o_sum
+ *     dcut_layer_mlp_part:   d_part = (SiLU(Wg . RMSNorm(h1)) * (Wu . RMSNorm(h1))) . Wd^T   (no residual)
+ *     -- all-reduce (sum) of d_part --
+ *     dcut_residual_add:     y = h1 + d_sum
+ * and gets dcut_layer_forward's y up to the rounding of the bf16 partial sums.  The library makes no collective of its
+ * own: the exchange is the caller's (NCCL or its own kernels), so these calls run on one GPU as they stand.  Arguments
+ * as dcut_layer_forward (all five weight pointers of `weights` must be set in both halves: the layer's tensor maps are
+ * cached together).  dcut_residual_add: out = a + b over the rows < cu_q[B] of bf16 [T, width] tensors, width % 8 == 0.
+ */
+dcut_status dcut_layer_attn_part(dcut_ctx* ctx, const dcut_layer_weights* weights, const void* x, void* o_part, void* k_cache,
+                                 void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                                 const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                                 int T_cap, void* stream);
+dcut_status dcut_layer_mlp_part(dcut_ctx* ctx, const dcut_layer_weights* weights, const void* h1, void* d_part, const int* cu_q,
+                                int B, int T_cap, void* stream);
+dcut_status dcut_residual_add(dcut_ctx* ctx, const void* a, const void* b, void* out, int width, const int* cu_q, int B,
+                              int T_cap, void* stream);
+
+/*
  * Start-up cost table C(B, rho) (Eq. 4-5; Appendix C, "Cost-table profiling protocol"; Table 3 shows two such
  * tables).  The paper's system builds it once before serving: for every batch size B it captures a graph for and
  * every ratio bucket rho it runs dummy speculative steps with the budget K_rho(B) and records the median step

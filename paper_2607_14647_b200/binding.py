@@ -32,7 +32,7 @@ EXPORTS = ["dcut_create", "dcut_destroy", "dcut_last_error", "dcut_set_cost_dens
            "dcut_select_causal", "dcut_accept_rs", "dcut_commit", "dcut_model_verify", "dcut_poll_device_status",
            "dcut_enable_plan_in_select", "dcut_cost_grid_create", "dcut_cost_grid_destroy", "dcut_cost_grid_budget",
            "dcut_cost_grid_record", "dcut_cost_grid_get", "dcut_cost_grid_nearest", "dcut_cost_grid_buckets",
-           "dcut_set_cost_from_grid"]
+           "dcut_set_cost_from_grid", "dcut_layer_attn_part", "dcut_layer_mlp_part", "dcut_residual_add"]
 
 
 class Limits(C.Structure):
@@ -102,6 +102,9 @@ _lib.dcut_gemm_bf16.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _vp, _i, _i, _vp
 _lib.dcut_lm_head_accept.argtypes = [_vp, _vp, _vp, _i, _vp, _vp, _i, _i, _i, _vp, _vp, _vp, _vp, _vp, _vp]
 _lib.dcut_layer_forward.argtypes = [_vp, C.POINTER(LayerWeights), _vp, _vp, _vp, _vp, _ll, _vp, _i, _vp, _vp, _vp, _vp,
                                     _i, _i, _vp]
+_lib.dcut_layer_attn_part.argtypes = _lib.dcut_layer_forward.argtypes
+_lib.dcut_layer_mlp_part.argtypes = [_vp, C.POINTER(LayerWeights), _vp, _vp, _vp, _i, _i, _vp]
+_lib.dcut_residual_add.argtypes = [_vp, _vp, _vp, _vp, _i, _vp, _i, _i, _vp]
 
 
 @dataclass
@@ -425,6 +428,33 @@ class Context:
                                             _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32),
                                             _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32), B, T_cap, _stream()))
         return y
+
+    def layer_attn_part(self, weights: dict, x, o_part, k_cache, v_cache, block_table, ctx_lens, cu_q, tok_req, tok_pos,
+                        T_cap: int, rms_eps: float = 1e-6, rope_theta: float = 1e6):
+        """dcut_layer_attn_part: a tensor-parallel rank's attention half of the layer (its partial O projection, no residual)."""
+        lw = LayerWeights(*[_ptr(weights[n], torch.bfloat16) for n in
+                            ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")], rms_eps, rope_theta)
+        B = ctx_lens.shape[0]
+        self._check(_lib.dcut_layer_attn_part(self._h, C.byref(lw), _ptr(x, torch.bfloat16), _ptr(o_part, torch.bfloat16),
+                                              _ptr(k_cache, torch.bfloat16), _ptr(v_cache, torch.bfloat16),
+                                              k_cache.shape[0], _ptr(block_table, torch.int32), block_table.shape[1],
+                                              _ptr(ctx_lens, torch.int32), _ptr(cu_q, torch.int32),
+                                              _ptr(tok_req, torch.int32), _ptr(tok_pos, torch.int32), B, T_cap, _stream()))
+        return o_part
+
+    def layer_mlp_part(self, weights: dict, h1, d_part, cu_q, T_cap: int, rms_eps: float = 1e-6, rope_theta: float = 1e6):
+        """dcut_layer_mlp_part: the rank's MLP half (its partial down projection, no residual)."""
+        lw = LayerWeights(*[_ptr(weights[n], torch.bfloat16) for n in
+                            ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")], rms_eps, rope_theta)
+        self._check(_lib.dcut_layer_mlp_part(self._h, C.byref(lw), _ptr(h1, torch.bfloat16), _ptr(d_part, torch.bfloat16),
+                                             _ptr(cu_q, torch.int32), cu_q.shape[0] - 1, T_cap, _stream()))
+        return d_part
+
+    def residual_add(self, a, b, out, cu_q, T_cap: int):
+        """dcut_residual_add: out = a + b over the packed rows in use."""
+        self._check(_lib.dcut_residual_add(self._h, _ptr(a, torch.bfloat16), _ptr(b, torch.bfloat16), _ptr(out, torch.bfloat16),
+                                           a.shape[1], _ptr(cu_q, torch.int32), cu_q.shape[0] - 1, T_cap, _stream()))
+        return out
 
     def make_model(self, layers: list, embed, g_final, w_lm, k_caches: list, v_caches: list, rms_eps: float = 1e-6,
                    rope_theta: float = 1e6) -> "PreparedModel":

@@ -465,19 +465,24 @@ static dcut_status dcut_prepare_rope(dcut_ctx* c, float rope_theta, cudaStream_t
     return DCUT_OK;
 }
 
-dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
-                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
-                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
-                               int T_cap, void* stream) {
+static dcut_status layer_common(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
+                                void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                                const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                                int T_cap, int part, void* stream) {
     if (!c) return DCUT_EINVAL;
     DCUT_ON_DEVICE(c);
     if (c->lim.hidden <= 0 || !c->ly_norm) return dcut_fail(c, DCUT_EINVAL, "context was created without layer shapes");
-    if (!w || !w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down || !w->g_attn || !w->g_mlp || !x || !y ||
-        !k_cache || !v_cache || !block_table || !ctx_lens || !cu_q || !tok_req || !tok_pos)
+    const bool attn = part != 2, mlp = part != 1;
+    if (!w || !x || !y || !cu_q) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (attn && (!w->w_qkv || !w->w_o || !w->g_attn || !k_cache || !v_cache || !block_table || !ctx_lens || !tok_req || !tok_pos))
         return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (mlp && (!w->w_gate || !w->w_up || !w->w_down || !w->g_mlp)) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    // the tensor-map cache of a layer is keyed by w_qkv and holds all five projections: every weight pointer must be given
+    if (!w->w_qkv || !w->w_o || !w->w_gate || !w->w_up || !w->w_down)
+        return dcut_fail(c, DCUT_EINVAL, "all five weight pointers of the layer must be set (also for one half of it)");
     if (B < 1 || T_cap < B || B > c->lim.max_B || T_cap > c->lim.max_B * (c->lim.max_gamma + 1))
         return dcut_fail(c, DCUT_ECAPACITY, "B = %d, T_cap = %d outside the limits", B, T_cap);
-    if (block_table_stride < 1 || block_table_stride > c->lim.max_pages_per_req)
+    if (attn && (block_table_stride < 1 || block_table_stride > c->lim.max_pages_per_req))
         return dcut_fail(c, DCUT_ECAPACITY, "block_table_stride = %d outside [1, %d]", block_table_stride, c->lim.max_pages_per_req);
     if (!(w->rope_theta > 1.0f) || !(w->rms_eps >= 0.0f)) return dcut_fail(c, DCUT_EINVAL, "rope_theta must exceed 1, rms_eps >= 0");
     const uintptr_t al = reinterpret_cast<uintptr_t>(w->w_qkv) | reinterpret_cast<uintptr_t>(w->w_o) |
@@ -487,12 +492,44 @@ dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const v
     if ((al & 127) || ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) |
                         reinterpret_cast<uintptr_t>(w->g_attn) | reinterpret_cast<uintptr_t>(w->g_mlp)) & 15))
         return dcut_fail(c, DCUT_EINVAL, "weights and caches must be 128-byte aligned, x / y / gains 16-byte aligned");
-    {
+    if (attn) {
         dcut_status st = dcut_prepare_rope(c, w->rope_theta, static_cast<cudaStream_t>(stream));
         if (st != DCUT_OK) return st;
     }
     return dcut_launch_layer(c, w, x, y, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q,
-                             tok_req, tok_pos, B, T_cap, 0, static_cast<cudaStream_t>(stream));
+                             tok_req, tok_pos, B, T_cap, 0, part, static_cast<cudaStream_t>(stream));
+}
+
+dcut_status dcut_layer_forward(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
+                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                               int T_cap, void* stream) {
+    return layer_common(c, w, x, y, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q, tok_req,
+                        tok_pos, B, T_cap, 0, stream);
+}
+
+dcut_status dcut_layer_attn_part(dcut_ctx* c, const dcut_layer_weights* w, const void* x, void* o_part, void* k_cache,
+                                 void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
+                                 const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
+                                 int T_cap, void* stream) {
+    return layer_common(c, w, x, o_part, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens, cu_q, tok_req,
+                        tok_pos, B, T_cap, 1, stream);
+}
+
+dcut_status dcut_layer_mlp_part(dcut_ctx* c, const dcut_layer_weights* w, const void* h1, void* d_part, const int* cu_q, int B,
+                                int T_cap, void* stream) {
+    return layer_common(c, w, h1, d_part, nullptr, nullptr, 0, nullptr, 0, nullptr, cu_q, nullptr, nullptr, B, T_cap, 2, stream);
+}
+
+dcut_status dcut_residual_add(dcut_ctx* c, const void* a, const void* b, void* out, int width, const int* cu_q, int B,
+                              int T_cap, void* stream) {
+    if (!c) return DCUT_EINVAL;
+    DCUT_ON_DEVICE(c);
+    if (!a || !b || !out || !cu_q) return dcut_fail(c, DCUT_EINVAL, "null pointer argument");
+    if (B < 1 || T_cap < B || width < 8 || width % 8) return dcut_fail(c, DCUT_EINVAL, "need B >= 1, T_cap >= B, width a positive multiple of 8");
+    if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(out)) & 15)
+        return dcut_fail(c, DCUT_EINVAL, "operands must be 16-byte aligned");
+    return dcut_launch_residual_add(c, a, b, out, width, cu_q, B, T_cap, static_cast<cudaStream_t>(stream));
 }
 
 dcut_status dcut_poll_device_status(dcut_ctx* c, int* code, void* stream) {

@@ -203,4 +203,6 @@ dcut_status dcut_launch_commit(dcut_ctx* ctx, const int* accept_len, const int* 
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
-                              int T_cap, int reuse_plan, cudaStream_t stream);
+                              int T_cap, int reuse_plan, int part, cudaStream_t stream);
+dcut_status dcut_launch_residual_add(dcut_ctx* ctx, const void* a, const void* b, void* out, int width, const int* cu_q, int B,
+                                     int T_cap, cudaStream_t stream);

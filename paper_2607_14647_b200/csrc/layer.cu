@@ -1051,7 +1051,7 @@ dcut_status dcut_launch_model(dcut_ctx* ctx, const dcut_model* m, long long num_
         __nv_bfloat16* y = (l == m->n_layers - 1 && user) ? user : ctx->ly_x[(l + 1) & 1];
         st = dcut_launch_layer(ctx, &m->layers[l], x, y, m->k_caches[l], m->v_caches[l], num_pages,
                                block_table, block_table_stride, ctx_lens, cu_q, tok_req, tok_pos, B, T_cap,
-                               l > 0 /* the attention work list of layer 0 serves every layer */, stream);
+                               l > 0 /* the attention work list of layer 0 serves every layer */, 0, stream);
         if (st != DCUT_OK) return st;
         x = y;
     }
@@ -1118,7 +1118,10 @@ dcut_status dcut_launch_gemm(dcut_ctx* ctx, const void* a, const void* w, const 
 dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const void* x, void* y, void* k_cache,
                               void* v_cache, long long num_pages, const int* block_table, int block_table_stride,
                               const int* ctx_lens, const int* cu_q, const int* tok_req, const int* tok_pos, int B,
-                              int T_cap, int reuse_plan, cudaStream_t stream) {
+                              int T_cap, int reuse_plan, int part, cudaStream_t stream) {
+    // part 0: the whole layer.  Tensor-parallel halves (a rank's shard of the heads / of the intermediate width, the
+    // projections that close a half WITHOUT the residual, so that the ranks' outputs can be summed first):
+    // part 1: y = Attn(RoPE(Wqkv . RMSNorm(x))) . Wo^T;  part 2: y = (SiLU(Wg . n) * (Wu . n)) . Wd^T with n = RMSNorm(x).
     const dcut_limits& l = ctx->lim;
     const int H = l.hidden, I = l.intermediate, Dh = l.head_dim;
     const int qkv_w = (l.n_q_heads + 2 * l.n_kv_heads) * Dh, q_w = l.n_q_heads * Dh;
@@ -1148,6 +1151,7 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     g.V = 0;
     g.status = ctx->d_status;
 
+    if (part != 2) {
     // 1. n = RMSNorm(x)
     if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(x),
                                                    static_cast<const __nv_bfloat16*>(w->g_attn), cu_q, B, H, w->rms_eps, ctx->ly_norm),
@@ -1166,17 +1170,62 @@ dcut_status dcut_launch_layer(dcut_ctx* ctx, const dcut_layer_weights* w, const 
     st = dcut_launch_verify_attn(ctx, ctx->ly_q, k_cache, v_cache, num_pages, block_table, block_table_stride, ctx_lens,
                                  cu_q, B, T_cap, 1.0f / sqrtf((float)Dh), ctx->ly_attn, nullptr, reuse_plan, stream);
     if (st != DCUT_OK) return st;
-    // 5. h1 = x + attn . Wo^T
-    g.N_out = H; g.K = q_w; g.out = ctx->ly_h1; g.residual = static_cast<const __nv_bfloat16*>(x);
+    // 5. h1 = x + attn . Wo^T   (a tensor-parallel half: the rank's partial product alone, into y)
+    g.N_out = H; g.K = q_w;
+    if (part == 1) {
+        g.out = static_cast<__nv_bfloat16*>(y); g.residual = nullptr;
+        return launch_gemm<kPlain>(ctx, lm->act[1], wm->m[1], wm->m[1], H / BN, T_cap, wmask[1], g, stream);
+    }
+    g.out = ctx->ly_h1; g.residual = static_cast<const __nv_bfloat16*>(x);
     if ((st = launch_gemm<kResidual>(ctx, lm->act[1], wm->m[1], wm->m[1], H / BN, T_cap, wmask[1], g, stream)) != DCUT_OK) return st;
-    // 6. n2 = RMSNorm(h1)
-    if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream, static_cast<const __nv_bfloat16*>(ctx->ly_h1),
+    }
+    // 6. n2 = RMSNorm(h1)   (the MLP half of a tensor-parallel layer starts here, from the caller's h1)
+    const __nv_bfloat16* h1 = part == 2 ? static_cast<const __nv_bfloat16*>(x) : ctx->ly_h1;
+    if ((st = dcut_check_cuda(ctx, dcut_launch_pdl(rmsnorm_kernel, dim3(T_cap), dim3(256), 0, stream, h1,
                                                    static_cast<const __nv_bfloat16*>(w->g_mlp), cu_q, B, H, w->rms_eps, ctx->ly_norm2),
                               "launch rmsnorm_kernel")) != DCUT_OK) return st;
     // 7. act = SiLU(n2 . Wg^T) * (n2 . Wu^T)
     g.N_out = I; g.K = H; g.out = ctx->ly_act; g.residual = nullptr;
     if ((st = launch_gemm<kSwiGLU>(ctx, lm->act[2], wm->m[2], wm->m[3], I / (BN / 2), T_cap, wmask[2], g, stream)) != DCUT_OK) return st;
     // 8. y = h1 + act . Wd^T
-    g.N_out = H; g.K = I; g.out = static_cast<__nv_bfloat16*>(y); g.residual = ctx->ly_h1;
+    g.N_out = H; g.K = I; g.out = static_cast<__nv_bfloat16*>(y);
+    if (part == 2) {
+        g.residual = nullptr;
+        return launch_gemm<kPlain>(ctx, lm->act[3], wm->m[4], wm->m[4], H / BN, T_cap, wmask[4], g, stream);
+    }
+    g.residual = ctx->ly_h1;
     return launch_gemm<kResidual>(ctx, lm->act[3], wm->m[4], wm->m[4], H / BN, T_cap, wmask[4], g, stream);
+}
+
+namespace {
+// out = a + b over the rows in use (bf16, one 16-byte vector per thread and step)
+__global__ void __launch_bounds__(256) residual_add_kernel(const uint4* __restrict__ a, const uint4* __restrict__ b, uint4* __restrict__ out,
+                                                           const int* __restrict__ cu_q, int B, int vec_per_row) {
+    dcut_pdl_wait();
+    dcut_pdl_launch_dependents();
+    const long long n = (long long)cu_q[B] * vec_per_row;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const uint4 x = a[i], y = b[i];
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+        uint32_t r[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat162 u = *reinterpret_cast<const __nv_bfloat162*>(&xs[e]), v = *reinterpret_cast<const __nv_bfloat162*>(&ys[e]);
+            const __nv_bfloat162 s = __floats2bfloat162_rn(__low2float(u) + __low2float(v), __high2float(u) + __high2float(v));
+            r[e] = *reinterpret_cast<const uint32_t*>(&s);
+        }
+        out[i] = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+}
+}  // namespace
+
+dcut_status dcut_launch_residual_add(dcut_ctx* ctx, const void* a, const void* b, void* out, int width, const int* cu_q, int B,
+                                     int T_cap, cudaStream_t stream) {
+    const long long cap = (long long)T_cap * (width / 8);
+    int grid = (int)((cap + 255) / 256);
+    if (grid > 4 * ctx->sm_count) grid = 4 * ctx->sm_count;
+    if (grid < 1) grid = 1;
+    return dcut_check_cuda(ctx, dcut_launch_pdl(residual_add_kernel, dim3(grid), dim3(256), 0, stream, static_cast<const uint4*>(a),
+                                                static_cast<const uint4*>(b), static_cast<uint4*>(out), cu_q, B, width / 8),
+                           "launch residual_add_kernel");
 }

@@ -308,3 +308,75 @@ def test_first_layer_call_captured_in_a_graph_replays_correctly():
         assert ctx.poll_device_status() == 0
         assert torch.equal(y, y_eager) and torch.equal(k_g, k_e) and torch.equal(v_g, v_e)
     ctx.close()
+
+
+@pytest.mark.parametrize("tp", [2, 4])
+def test_tensor_parallel_halves_reproduce_the_layer(tp):
+    """dcut_layer_attn_part / dcut_layer_mlp_part / dcut_residual_add: the decoder layer cut where a tensor-parallel
+    deployment exchanges.  Rank r holds the q / k / v heads, O columns, gate / up rows and down columns of its share
+    and its slice of the paged cache; the ranks run one after the other on this one GPU and a float32 sum stands in
+    for the two all-reduces (the exchange is the caller's).  The result must match the oracle's layer like the
+    unsharded call does, and the appended K/V slices must be the unsharded call's (same arithmetic per head)."""
+    cfg = wl.custom_config(B=6, gamma=16, n_q_heads=8, n_kv_heads=4, head_dim=128, ctx_lo=5, ctx_hi=400, conf_kind="skew_halves")
+    hidden, inter = 512, 1024
+    depths = np.array([16, 0, 3, 9, 1, 16], np.int32)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    w = wl.layer_weights(cfg, hidden, inter)
+    wd = {n: getattr(w, n) for n in ("w_qkv", "w_o", "w_gate", "w_up", "w_down", "g_attn", "g_mlp")}
+    x = wl.layer_x_rows(cfg, depths, hidden)
+    cu = wl.cu_q_from_depths(depths)
+    T = int(cu[-1])
+    tok_req = np.concatenate([np.full(d + 1, i) for i, d in enumerate(depths)]).astype(np.int32)
+    tok_pos = np.concatenate([sel.ctx_lens[i] + np.arange(d + 1) for i, d in enumerate(depths)]).astype(np.int32)
+    d_x, d_cu, d_bt, d_ctx = dev(x), dev(cu), dev(kv.block_table), dev(sel.ctx_lens)
+    d_req, d_pos = dev(tok_req), dev(tok_pos)
+    Dh, Hq, Hkv = cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads
+    hq, hk, it = Hq // tp, Hkv // tp, inter // tp
+    shard_cfg = wl.custom_config(B=cfg.B, gamma=cfg.gamma, n_q_heads=hq, n_kv_heads=hk, head_dim=Dh, ctx_lo=cfg.ctx_lo, ctx_hi=cfg.ctx_hi)
+    ranks = []
+    for r in range(tp):
+        q_rows = wd["w_qkv"][r * hq * Dh:(r + 1) * hq * Dh]
+        k_rows = wd["w_qkv"][Hq * Dh + r * hk * Dh: Hq * Dh + (r + 1) * hk * Dh]
+        v_rows = wd["w_qkv"][(Hq + Hkv) * Dh + r * hk * Dh: (Hq + Hkv) * Dh + (r + 1) * hk * Dh]
+        ws = dict(w_qkv=torch.cat([q_rows, k_rows, v_rows]).contiguous(), w_o=wd["w_o"][:, r * hq * Dh:(r + 1) * hq * Dh].contiguous(),
+                  w_gate=wd["w_gate"][r * it:(r + 1) * it].contiguous(), w_up=wd["w_up"][r * it:(r + 1) * it].contiguous(),
+                  w_down=wd["w_down"][:, r * it:(r + 1) * it].contiguous(), g_attn=wd["g_attn"], g_mlp=wd["g_mlp"])
+        ranks.append(dict(ctx=make_ctx(shard_cfg, max_pages=kv.max_pages_per_req, hidden=hidden, intermediate=it, vocab=0),
+                          w={k: dev(v) for k, v in ws.items()},
+                          k=dev(kv.k_cache[:, r * hk:(r + 1) * hk].contiguous()), v=dev(kv.v_cache[:, r * hk:(r + 1) * hk].contiguous())))
+    bf = dict(dtype=torch.bfloat16, device="cuda")
+    # attention half on every rank, then the first all-reduce
+    parts = []
+    for rk in ranks:
+        o = torch.empty((T, hidden), **bf)
+        rk["ctx"].layer_attn_part(rk["w"], d_x, o, rk["k"], rk["v"], d_bt, d_ctx, d_cu, d_req, d_pos, cfg.t_cap, cfg.rms_eps, cfg.rope_theta)
+        parts.append(o)
+    o_sum = torch.stack([p.float() for p in parts]).sum(0).to(torch.bfloat16)
+    ys = []
+    for rk in ranks:                                       # every rank computes h1 and its MLP half from the same sum
+        h1 = rk["ctx"].residual_add(d_x, o_sum, torch.empty((T, hidden), **bf), d_cu, cfg.t_cap)
+        rk["h1"] = h1
+        rk["d"] = rk["ctx"].layer_mlp_part(rk["w"], h1, torch.empty((T, hidden), **bf), d_cu, cfg.t_cap, cfg.rms_eps, cfg.rope_theta)
+    d_sum = torch.stack([rk["d"].float() for rk in ranks]).sum(0).to(torch.bfloat16)
+    for rk in ranks:
+        ys.append(rk["ctx"].residual_add(rk["h1"], d_sum, torch.empty((T, hidden), **bf), d_cu, cfg.t_cap))
+    torch.cuda.synchronize()
+    for rk in ranks:
+        assert rk["ctx"].poll_device_status() == 0
+    assert all(torch.equal(ys[0], y) for y in ys[1:])
+    ref = orc.layer_forward(x, wd, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, depths, Hq, Hkv, Dh, cfg.page_size,
+                            cfg.rms_eps, cfg.rope_theta)
+    _close(ys[0], ref["y"], "tensor-parallel layer output y")
+    # the unsharded call on the same inputs: same output within the layer's tolerance, same appended K/V bit for bit
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req, hidden=hidden, intermediate=inter, vocab=0)
+    y_full = torch.empty((T, hidden), **bf)
+    k_full, v_full = dev(kv.k_cache), dev(kv.v_cache)
+    ctx.layer_forward({k: dev(v) for k, v in wd.items()}, d_x, y_full, k_full, v_full, d_bt, d_ctx, d_cu, d_req, d_pos, cfg.t_cap,
+                      cfg.rms_eps, cfg.rope_theta)
+    torch.cuda.synchronize()
+    _close(ys[0], y_full.float().cpu(), "tensor-parallel against unsharded")
+    for r, rk in enumerate(ranks):
+        assert torch.equal(rk["k"], k_full[:, r * hk:(r + 1) * hk]) and torch.equal(rk["v"], v_full[:, r * hk:(r + 1) * hk])
+        rk["ctx"].close()
+    ctx.close()
