@@ -539,20 +539,24 @@ def run_arms(w: Workload, args, world: int, arms: dict, light: bool):
         n_ev = max(steps, 40 if light else 100)
         for c in range(w.kv_copies):
             w.step(qp, lp, bufs, c)
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ev)]
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n_ev)]
         barrier(world)
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         start.record()
         for k in range(n_ev):
-            so = w.select()
             ev[k][0].record()
-            w.middle(qp, so, bufs, k % w.kv_copies)
+            so = w.select()
             ev[k][1].record()
+            w.middle(qp, so, bufs, k % w.kv_copies)
+            ev[k][2].record()
             w.accept(lp, so, bufs)
+            ev[k][3].record()
         end.record()
         barrier(world)
         eager_ms = max_over_ranks(start.elapsed_time(end), world) / n_ev
-        mid = [a.elapsed_time(b) for a, b in ev]
+        mid = [e[1].elapsed_time(e[2]) for e in ev]
+        sel_ms = statistics.median(e[0].elapsed_time(e[1]) for e in ev)
+        acc_ms = statistics.median(e[2].elapsed_time(e[3]) for e in ev)
         # (b) the same step captured once per KV copy in a CUDA graph and replayed: the packed length is read on the
         # device, so one graph serves whatever depth vector the selector produces
         runs, keep = w.graphs(qp, lp, bufs, not args.no_graph)
@@ -561,7 +565,7 @@ def run_arms(w: Workload, args, world: int, arms: dict, light: bool):
         assert w.ctx.poll_device_status() == 0
         res[name] = dict(T=T, accepted=accepted, ms_per_step=mean_ms, per_step=stats_ms(per_step), rounds=len(round_ms),
                          timed_steps=len(round_ms) * steps, eager_ms=eager_ms, mid_ms=statistics.mean(mid), mid=stats_ms(mid),
-                         tokens_per_s=world * accepted / (mean_ms * 1e-3),
+                         tokens_per_s=world * accepted / (mean_ms * 1e-3), sel_ms=sel_ms, acc_ms=acc_ms,
                          attn_bytes=attn_algorithmic_bytes(cfg, w.sel.ctx_lens, d), depths=d)
         del qp, lp, bufs, runs, keep
     return res
@@ -573,7 +577,9 @@ def arms_json(w: Workload, res: dict, pk: dict) -> dict:
         e = {"T": v["T"], "accepted_tokens": v["accepted"], "ms_per_step": round(v["ms_per_step"], 4),
              "ms_per_step_median": v["per_step"]["median"], "ms_per_step_p95": v["per_step"]["p95"],
              "timed_steps": v["timed_steps"], "ms_per_step_kernel_by_kernel": round(v["eager_ms"], 4),
-             "tokens_per_s": round(v["tokens_per_s"], 1)}
+             "tokens_per_s": round(v["tokens_per_s"], 1), "select_us_median": round(v["sel_ms"] * 1e3, 1),
+             "accept_us_median": round(v["acc_ms"] * 1e3, 1),
+             "accept_gbs": round(v["T"] * w.cfg.vocab * 2 / (v["acc_ms"] * 1e-3) / 1e9, 1)}
         if w.is_layer:
             e["forward_ms"] = round(v["mid_ms"], 4)
             e["forward_ms_median"] = v["mid"]["median"]
@@ -708,6 +714,43 @@ def stochastic_extra(w: Workload, cost):
         return out
     except Exception as exc:   # the extra measurement must not take the bench line down
         return {"error": repr(exc)[:200]}
+
+
+def e2e_hidden_form(w: "Workload", args, cost, h: dict, want_accepted: int, hidden: int = 4096):
+    """The end-to-end step again, in the host call's hidden-state form: the kept rows of the last hidden states
+    (8 KB each) cross the bus instead of the kept logits rows (300 KB each), and the step ends in the LM head fused
+    with acceptance (the LM head's weights are resident like the cache).  A longer step (it contains the LM-head GEMM)
+    that is no longer bound by the bus."""
+    from paper_2607_14647_b200 import binding
+    cfg, dev = w.cfg, w.dev
+    ctx = binding.Context(max_B=cfg.B, max_gamma=cfg.gamma, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                          head_dim=cfg.head_dim, page_size=cfg.page_size, max_pages_per_req=w.kv.block_table.shape[1],
+                          vocab=cfg.vocab, hidden=hidden, intermediate=hidden)
+    try:
+        ctx.set_cost_dense(cost)
+        w_lm = wl.lm_head_weight(cfg, vocab=cfg.vocab, hidden=hidden)
+        full = np.full(cfg.B, cfg.gamma, np.int32)
+        x_all = wl.lm_head_x_rows(cfg, w.sel, full, w_lm).view(cfg.B, cfg.gamma + 1, hidden).contiguous().pin_memory()
+        d_w = w_lm.to(dev)
+        hout = ctx.host_step_outputs(cfg.B, cfg.gamma)
+        call = lambda: ctx.verify_step_host(h["conf"], h["draft"], h["bonus"], h["ctx"], h["bt"], h["q"], None, w.d_k[0], w.d_v[0],
+                                            out=hout, hidden_rows=x_all, w_lm=d_w)
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            call()
+        torch.cuda.synchronize()
+        dt = (time.perf_counter() - t0) / args.e2e_steps
+        acc = int(hout["n_accepted_total"].item())
+        assert ctx.poll_device_status() == 0
+        return {"value": acc / dt, "unit": UNIT, "ms_per_step": round(dt * 1e3, 4), "accepted_tokens": acc,
+                "accepted_tokens_of_the_logits_form": want_accepted, "h2d_bytes_per_step": hout["h2d_bytes"],
+                "d2h_bytes_per_step": hout["d2h_bytes"], "hidden": hidden,
+                "api": "dcut_verify_step_host with hidden_rows + w_lm (select, attention, LM head fused with acceptance)"}
+    finally:
+        ctx.close()
 
 
 def multistep_arm(cfg, dev, args, world, cost, n_chain: int):
@@ -892,6 +935,12 @@ def run_dcut(args):
                    "h2d_bytes_per_step": hout["h2d_bytes"], "d2h_bytes_per_step": hout["d2h_bytes"],
                    "api": "dcut_verify_step_host (pinned host buffers; KV cache resident)"}
         stochastic = stochastic_extra(w, cost) if (not is_layer and rank == 0) else None
+        e2e_hidden = None
+        if not is_layer and world == 1 and args.e2e_steps > 0:
+            try:
+                e2e_hidden = e2e_hidden_form(w, args, cost, h, res["pruned"]["accepted"])
+            except Exception as exc:   # the extra measurement must not take the bench line down
+                e2e_hidden = {"error": repr(exc)[:300]}
     finally:
         w.close()
     del w
@@ -974,6 +1023,8 @@ def run_dcut(args):
             "kernel": "gemm_tcgen05_kernel (4 projections of the layer, full-gamma arm, timed alone)", "bound": "tensor",
             "achieved": g["tflops"], "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": round(g["tflops"] / pk["bf16_tflops"], 4),
             "peak_source": f"of {pk['source']} (burst)", "traffic": None}
+    if e2e_hidden is not None:
+        line["e2e_hidden_state_form"] = e2e_hidden
     if stochastic is not None:
         line["stochastic"] = stochastic
     if multistep is not None:

@@ -437,6 +437,12 @@ dcut_status dcut_accept_static(const void* logits, int V, const int* draft_ids, 
  *   [1]; attn_out bf16 [T, n_q_heads, head_dim] or NULL; h2d_bytes / d2h_bytes (bytes copied, or NULL).
  * Uses the cost table set on the context.  The first call (and a call with a larger vocab) allocates
  * device staging buffers; later calls allocate nothing.
+ * Hidden-state form: a bf16 logits row is 300 KB at V = 151 936 and the kept rows of a step are what fills the bus.
+ * With hidden_rows (HOST bf16 [B, gamma+1, hidden], the last hidden state of every block position) and w_lm (DEVICE
+ * bf16 [vocab, hidden], resident like the cache) set, and logits_rows NULL, the call copies the kept rows of
+ * hidden_rows instead (8 KB each at hidden 4096) and ends in dcut_lm_head_accept (Section 3.1: the target's
+ * prediction at every retained position, here from its LM head), so the logits exist neither on the host nor in HBM.
+ * Needs a context with layer shapes (hidden > 0).
  */
 typedef struct {
     int B, gamma, vocab, block_table_stride;
@@ -459,6 +465,8 @@ typedef struct {
     void* attn_out;
     long long* h2d_bytes;
     long long* d2h_bytes;
+    const void* hidden_rows;   /* hidden-state form (else NULL) */
+    const void* w_lm;
 } dcut_host_step;
 dcut_status dcut_verify_step_host(dcut_ctx* ctx, const dcut_host_step* step, void* stream);
 

@@ -53,7 +53,7 @@ class HostStep(C.Structure):
                 ("scale", _f)] + [(n, _vp) for n in (
                     "conf", "draft_ids", "bonus_ids", "ctx_lens", "block_table", "q_rows", "logits_rows", "k_cache",
                     "v_cache", "depths", "accept_len", "bonus", "out_tokens", "n_accepted_total", "attn_out",
-                    "h2d_bytes", "d2h_bytes")]
+                    "h2d_bytes", "d2h_bytes", "hidden_rows", "w_lm")]
 
 
 _lib.dcut_verify_step_host.argtypes = [_vp, C.POINTER(HostStep), _vp]
@@ -361,13 +361,15 @@ class Context:
                                      _ptr(accept_len), _ptr(bonus), _ptr(out_tokens), _ptr(total), _stream()))
 
     def verify_step_host(self, conf, draft_ids, bonus_ids, ctx_lens, block_table, q_rows, logits_rows, k_cache,
-                         v_cache, out: Optional[dict] = None, scale: Optional[float] = None, want_attn_out=False):
+                         v_cache, out: Optional[dict] = None, scale: Optional[float] = None, want_attn_out=False,
+                         hidden_rows=None, w_lm=None):
         """Whole step from HOST tensors (CPU torch tensors, ideally pinned); k_cache / v_cache are the
-        device-resident cache.  Returns a dict of CPU tensors plus the bytes copied each way."""
+        device-resident cache.  Returns a dict of CPU tensors plus the bytes copied each way.
+        Hidden-state form: logits_rows=None, hidden_rows (CPU bf16 [B, gamma+1, hidden]) and w_lm (CUDA bf16 [V, hidden])."""
         B, gamma = conf.shape
-        V = logits_rows.shape[-1]
-        for t in (conf, draft_ids, bonus_ids, ctx_lens, block_table, q_rows, logits_rows):
-            assert not t.is_cuda and t.is_contiguous()
+        V = logits_rows.shape[-1] if logits_rows is not None else w_lm.shape[0]
+        for t in (conf, draft_ids, bonus_ids, ctx_lens, block_table, q_rows, logits_rows, hidden_rows):
+            assert t is None or (not t.is_cuda and t.is_contiguous())
         if out is None:
             out = self.host_step_outputs(B, gamma, want_attn_out)
         if scale is None:
@@ -375,11 +377,12 @@ class Context:
         h2d, d2h = _ll(0), _ll(0)
         hs = HostStep(B, gamma, V, block_table.shape[1], k_cache.shape[0], float(scale), conf.data_ptr(),
                       draft_ids.data_ptr(), bonus_ids.data_ptr(), ctx_lens.data_ptr(), block_table.data_ptr(),
-                      q_rows.data_ptr(), logits_rows.data_ptr(), _ptr(k_cache, torch.bfloat16),
+                      q_rows.data_ptr(), logits_rows.data_ptr() if logits_rows is not None else None, _ptr(k_cache, torch.bfloat16),
                       _ptr(v_cache, torch.bfloat16), out["depths"].data_ptr(), out["accept_len"].data_ptr(),
                       out["bonus"].data_ptr(), out["out_tokens"].data_ptr(), out["n_accepted_total"].data_ptr(),
                       out["attn_out"].data_ptr() if out.get("attn_out") is not None else None,
-                      C.addressof(h2d), C.addressof(d2h))
+                      C.addressof(h2d), C.addressof(d2h), hidden_rows.data_ptr() if hidden_rows is not None else None,
+                      _ptr(w_lm, torch.bfloat16))
         self._check(_lib.dcut_verify_step_host(self._h, C.byref(hs), _stream()))
         out["h2d_bytes"], out["d2h_bytes"] = h2d.value, d2h.value
         return out

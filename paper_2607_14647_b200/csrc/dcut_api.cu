@@ -91,6 +91,7 @@ void free_all(dcut_ctx* c) {
     cudaFree(c->hs_q);
     cudaFree(c->hs_out);
     cudaFree(c->hs_logits);
+    cudaFree(c->hs_hidden);
     if (c->hs_host_cu_q) cudaFreeHost(c->hs_host_cu_q);
     if (c->hs_copy_stream) cudaStreamDestroy(c->hs_copy_stream);
     if (c->hs_ev_fork) cudaEventDestroy(c->hs_ev_fork);
@@ -558,8 +559,12 @@ dcut_status dcut_poll_device_status(dcut_ctx* c, int* code, void* stream) {
 
 namespace {
 
-dcut_status ensure_host_step_buffers(dcut_ctx* c, int V) {
-    if (c->hs_ready && c->hs_vocab >= V) return DCUT_OK;
+dcut_status ensure_host_step_buffers(dcut_ctx* c, int V, bool hidden_form) {
+    if (hidden_form && c->hs_ready) {
+        if (c->hs_hidden) return DCUT_OK;
+        return dmalloc(c, &c->hs_hidden, (size_t)c->lim.max_B * (c->lim.max_gamma + 1) * c->lim.hidden, "cudaMalloc(step hidden)");
+    }
+    if (c->hs_ready && (hidden_form || c->hs_vocab >= V)) return DCUT_OK;
     const dcut_limits& l = c->lim;
     const size_t max_T = (size_t)l.max_B * (l.max_gamma + 1);
     const size_t keys = (size_t)l.max_B * l.max_gamma;
@@ -581,10 +586,14 @@ dcut_status ensure_host_step_buffers(dcut_ctx* c, int V) {
         if ((e = cudaEventCreateWithFlags(&c->hs_ev_fork, cudaEventDisableTiming)) != cudaSuccess) return dcut_check_cuda(c, e, "cudaEventCreate(step)");
         if ((e = cudaEventCreateWithFlags(&c->hs_ev_join, cudaEventDisableTiming)) != cudaSuccess) return dcut_check_cuda(c, e, "cudaEventCreate(step)");
     }
-    if (c->hs_logits) cudaFree(c->hs_logits);
-    c->hs_logits = nullptr;
-    if ((st = dmalloc(c, &c->hs_logits, max_T * (size_t)V, "cudaMalloc(step logits)")) != DCUT_OK) return st;
-    c->hs_vocab = V;
+    if (hidden_form) {
+        if (!c->hs_hidden && (st = dmalloc(c, &c->hs_hidden, max_T * (size_t)l.hidden, "cudaMalloc(step hidden)")) != DCUT_OK) return st;
+    } else {
+        if (c->hs_logits) cudaFree(c->hs_logits);
+        c->hs_logits = nullptr;
+        if ((st = dmalloc(c, &c->hs_logits, max_T * (size_t)V, "cudaMalloc(step logits)")) != DCUT_OK) return st;
+        c->hs_vocab = V;
+    }
     c->hs_ready = 1;
     return DCUT_OK;
 }
@@ -595,19 +604,26 @@ extern "C" dcut_status dcut_verify_step_host(dcut_ctx* c, const dcut_host_step* 
     if (!c) return DCUT_EINVAL;
     DCUT_ON_DEVICE(c);
     if (!s || !s->conf || !s->draft_ids || !s->bonus_ids || !s->ctx_lens || !s->block_table || !s->q_rows ||
-        !s->logits_rows || !s->k_cache || !s->v_cache || !s->depths || !s->accept_len || !s->bonus || !s->out_tokens ||
-        !s->n_accepted_total)
+        !s->k_cache || !s->v_cache || !s->depths || !s->accept_len || !s->bonus || !s->out_tokens || !s->n_accepted_total)
         return dcut_fail(c, DCUT_EINVAL, "null pointer in dcut_host_step");
+    const bool hidden_form = s->hidden_rows != nullptr;
+    if (hidden_form ? (s->logits_rows != nullptr || !s->w_lm) : !s->logits_rows)
+        return dcut_fail(c, DCUT_EINVAL, "dcut_host_step needs either logits_rows, or hidden_rows with w_lm");
+    if (hidden_form && (c->lim.hidden <= 0 || !c->layer_maps))
+        return dcut_fail(c, DCUT_EINVAL, "the hidden-state form needs a context created with layer shapes");
     const int B = s->B, g = s->gamma, V = s->vocab;
     const dcut_limits& l = c->lim;
     if (B < 1 || g < 1 || V < 1) return dcut_fail(c, DCUT_EINVAL, "need B, gamma, vocab >= 1");
     if (B > l.max_B || g > l.max_gamma || s->block_table_stride > l.max_pages_per_req || s->block_table_stride < 1)
         return dcut_fail(c, DCUT_ECAPACITY, "B, gamma or block_table_stride exceed the limits");
     if (l.n_q_heads <= 0) return dcut_fail(c, DCUT_EINVAL, "context was created without attention shapes");
-    dcut_status st = ensure_host_step_buffers(c, V);
+    dcut_status st = ensure_host_step_buffers(c, V, hidden_form);
     if (st != DCUT_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    const size_t q_row = (size_t)l.n_q_heads * l.head_dim * 2, lg_row = (size_t)V * 2;
+    // per block position the second stream carries a logits row, or (hidden-state form) a last-hidden-state row
+    const size_t q_row = (size_t)l.n_q_heads * l.head_dim * 2, lg_row = hidden_form ? (size_t)l.hidden * 2 : (size_t)V * 2;
+    const char* lg_src = static_cast<const char*>(hidden_form ? s->hidden_rows : s->logits_rows);
+    char* lg_dst = reinterpret_cast<char*>(hidden_form ? c->hs_hidden : c->hs_logits);
 #define DCUT_CP(dst, src, bytes, kind)                                                                   \
     if ((st = dcut_check_cuda(c, cudaMemcpyAsync(dst, src, bytes, kind, cs), "cudaMemcpyAsync(step)")) != DCUT_OK) return st
     DCUT_CP(c->hs_conf, s->conf, sizeof(float) * B * g, cudaMemcpyHostToDevice);
@@ -637,8 +653,7 @@ extern "C" dcut_status dcut_verify_step_host(dcut_ctx* c, const dcut_host_step* 
     }
     for (int i = 0; i < B; ++i) {
         const size_t rows = (size_t)(cu[i + 1] - cu[i]);
-        if ((st = dcut_check_cuda(c, cudaMemcpyAsync(reinterpret_cast<char*>(c->hs_logits) + (size_t)cu[i] * lg_row,
-                                                     static_cast<const char*>(s->logits_rows) + (size_t)i * (g + 1) * lg_row,
+        if ((st = dcut_check_cuda(c, cudaMemcpyAsync(lg_dst + (size_t)cu[i] * lg_row, lg_src + (size_t)i * (g + 1) * lg_row,
                                                      rows * lg_row, cudaMemcpyHostToDevice, c->hs_copy_stream),
                                   "cudaMemcpyAsync(step logits)")) != DCUT_OK) return st;
     }
@@ -649,8 +664,12 @@ extern "C" dcut_status dcut_verify_step_host(dcut_ctx* c, const dcut_host_step* 
     if (st != DCUT_OK) return st;
     if ((st = dcut_check_cuda(c, cudaStreamWaitEvent(cs, c->hs_ev_join, 0), "cudaStreamWaitEvent(step join)")) != DCUT_OK) return st;
     int* acc = c->hs_accept;            // [B] accept_len, [B] bonus, [B*(g+1)] tokens, [1] total
-    st = dcut_accept(c, c->hs_logits, V, c->hs_draft, c->hs_cu_q, B, g, T_cap, acc, acc + B, acc + 2 * B,
-                     acc + 2 * B + B * (g + 1), stream);
+    if (hidden_form)
+        st = dcut_lm_head_accept(c, c->hs_hidden, s->w_lm, V, c->hs_draft, c->hs_cu_q, B, g, T_cap, acc, acc + B, acc + 2 * B,
+                                 acc + 2 * B + B * (g + 1), nullptr, stream);
+    else
+        st = dcut_accept(c, c->hs_logits, V, c->hs_draft, c->hs_cu_q, B, g, T_cap, acc, acc + B, acc + 2 * B,
+                         acc + 2 * B + B * (g + 1), stream);
     if (st != DCUT_OK) return st;
     DCUT_CP(s->depths, c->hs_depths, sizeof(int) * B, cudaMemcpyDeviceToHost);
     DCUT_CP(s->accept_len, acc, sizeof(int) * B, cudaMemcpyDeviceToHost);

@@ -116,7 +116,7 @@ struct dcut_ctx {
     int hs_ready, hs_vocab;
     float* hs_conf;
     int *hs_draft, *hs_bonus, *hs_ctx_lens, *hs_block_table, *hs_depths, *hs_cu_q, *hs_accept;
-    unsigned short *hs_q, *hs_out, *hs_logits;
+    unsigned short *hs_q, *hs_out, *hs_logits, *hs_hidden;
     int* hs_host_cu_q;      // pinned
     cudaStream_t hs_copy_stream;   // dcut_verify_step_host: the logits travel on this stream while attention runs
     cudaEvent_t hs_ev_fork, hs_ev_join;
