@@ -258,3 +258,51 @@ def test_block_table_entry_outside_the_cache_reads_page_0_and_is_reported():
     ok, worst = attn_tolerance_ok(out2.float().cpu().numpy(), ref2)
     assert ok, f"worst err/limit {worst}"
     ctx.close()
+
+
+@pytest.mark.parametrize("B,shape,ctx_lo,ctx_hi,depths_kind", [
+    (1, dict(n_q_heads=8, n_kv_heads=1, head_dim=128), 30000, 30000, "full"),     # one item cut into a piece per SM
+    (1, dict(n_q_heads=8, n_kv_heads=1, head_dim=128), 30000, 30000, "zero"),
+    (2, dict(n_q_heads=32, n_kv_heads=8, head_dim=128), 9000, 20000, "mixed"),    # 16 items, every one cut many times
+    (3, dict(n_q_heads=4, n_kv_heads=1, head_dim=64), 4000, 9000, "full"),        # head_dim 64: warp-level pieces with 5 m-tiles
+    (480, dict(n_q_heads=8, n_kv_heads=2, head_dim=128), 0, 40, "mixed"),         # many tiny items, several per segment, none cut
+])
+def test_extreme_batch_shapes_sampled(B, shape, ctx_lo, ctx_hi, depths_kind):
+    """The work partition at its extremes: a single long request (one item per kv head, cut into as many pieces as
+    there are SMs and merged from that many partial results), and hundreds of one-page requests (segments of many
+    whole items).  The selector builds the partition (dcut_enable_plan_in_select)."""
+    cfg = wl.custom_config(B=B, gamma=16, ctx_lo=ctx_lo, ctx_hi=ctx_hi, vocab=64, **shape)
+    sel = wl.select_inputs(cfg)
+    kv = wl.paged_kv(cfg, sel.ctx_lens)
+    rng = np.random.default_rng(B)
+    depths = {"full": np.full(B, 16, np.int32), "zero": np.zeros(B, np.int32), "mixed": rng.integers(0, 17, B).astype(np.int32)}[depths_kind]
+    ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req)
+    ctx.enable_plan_in_select(True)
+    # force the selector to these depths: confidences 1 on the kept drafts, 0 beyond, and a flat cost
+    conf = np.zeros((B, 16), np.float32)
+    for i, d in enumerate(depths):
+        conf[i, :d] = 1.0
+    ctx.set_cost_buckets(B, 16, [int(depths.sum()) + B], [1.0])
+    so = ctx.select(dev(conf), dev(sel.draft_ids), dev(sel.bonus_ids), dev(sel.ctx_lens))
+    assert np.array_equal(so.depths.cpu().numpy(), depths)
+    q = wl.q_rows(cfg, depths)
+    cu = wl.cu_q_from_depths(depths)
+    T = int(cu[-1])
+    lse = torch.empty((T, cfg.n_q_heads), dtype=torch.float32, device="cuda")
+    out = ctx.verify_attn(dev(q), dev(kv.k_cache), dev(kv.v_cache), dev(kv.block_table), dev(sel.ctx_lens), so.cu_q, cfg.t_cap, lse=lse)
+    torch.cuda.synchronize()
+    assert ctx.poll_device_status() == 0
+    out2 = ctx.verify_attn(dev(q), dev(kv.k_cache), dev(kv.v_cache), dev(kv.block_table), dev(sel.ctx_lens), so.cu_q, cfg.t_cap)
+    assert torch.equal(out, out2)                                   # same partition, same bits
+    ctx.close()
+    n = min(T * cfg.n_q_heads, 96)
+    tok = rng.integers(0, T, n).astype(np.int32)
+    head = rng.integers(0, cfg.n_q_heads, n).astype(np.int32)
+    tok[:2] = [0, T - 1]
+    ref, ref_lse = orc.verify_attn(q, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, cu, cfg.n_q_heads, cfg.n_kv_heads,
+                                   cfg.head_dim, cfg.page_size, sample_tok=tok, sample_head=head)
+    got = out.float().cpu().numpy()
+    ok, worst = attn_tolerance_ok(got[tok, head], ref)
+    assert ok, f"worst err/limit {worst}"
+    np.testing.assert_allclose(lse.cpu().numpy()[tok, head], ref_lse, rtol=2e-3, atol=2e-3)
+    assert np.isfinite(got).all()
