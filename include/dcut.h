@@ -29,9 +29,8 @@
  *
  * Environment variables read once, in dcut_create (measurement knobs; the defaults are the measured best):
  *   DCUT_ATTN_TC_MIN_ROWS     query rows from which a work item goes to the tcgen05 phase (17; above 128: never)
- *   DCUT_ATTN_TARGET_ITEMS    requests are cut along the context only below this many (request, kv head) pairs (13/8 x SMs)
- *   DCUT_ATTN_TAIL_REQ_DIV    cut the shortest B / n requests finer (0 = off)
- *   DCUT_ATTN_TAIL_MIN_PAGES  smallest such piece, in pages (32)
+ *   DCUT_ATTN_MIN_CHUNK_PAGES a work item that a segment boundary cuts is cut at multiples of this many pages (8)
+ *   DCUT_ATTN_TAIL_ROWS       0 = a query tile above 128 rows becomes two work items instead of one with tail rows
  *   DCUT_GEMM_2CTA            0 = never run GEMM tiles on pairs of SMs (tcgen05 cta_group::2); default: where it pays
  *   DCUT_GEMM_WIDTHS          bit mask of the GEMM tile widths that may be chosen (bit i: 256 - 32 i columns; default 0x7f)
  *   DCUT_GEMM_FORCE           experiments: 0..6 = that width on one SM per tile, 8..14 = on a pair, 16..22 = a pair splitting K,

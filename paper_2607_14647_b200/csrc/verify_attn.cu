@@ -3,13 +3,14 @@
 // HBM-bound by design: every K/V byte of every request is read once per step, so the kernels are organised around
 // keeping 100-200 KB of page loads in flight per SM, all the time.
 //
-//   attn_plan_kernel     one CTA.  Cuts the requests' page lists into work items (flash-decoding split-KV, only when the
-//                        batch has fewer (request, kv head) pairs than two per SM); an item is one (request, kv head,
-//                        page range, block of query rows).  Items go to one of two queues, each ordered longest first:
-//                        query tiles of 17+ rows to the tcgen05 queue, smaller ones to the warp-level queue.
-//   attn_item_kernel     persistent, one CTA per SM.  A CTA claims items from the tcgen05 queue, then from the warp-level
-//                        queue, through a global counter.  In both phases the TMA producer warp claims the next item as
-//                        soon as it has issued the current item's last load and keeps streaming into the same ring of
+//   work partition       one CTA (attn_plan.cuh): the tail of the selector kernel, or the stand-alone attn_plan_kernel.
+//                        The call's work is a stream of (request, row block, kv head) items, each a run of KV pages of
+//                        known cost; it is cut into one segment of equal cost per SM.  A segment may begin or end inside
+//                        an item: that item is computed in pieces.  Query tiles of 17+ rows form the tcgen05 part of the
+//                        stream, smaller ones the warp-level part.
+//   attn_item_kernel     persistent, one CTA per SM.  A CTA walks its segment: its tcgen05 items, then its warp-level
+//                        items.  In both phases the TMA producer warp builds the next item from the work table as soon
+//                        as it has issued the current item's last load and keeps streaming into the same ring of
 //                        stages (stages, tensor-memory buffers and their mbarriers are numbered through consecutive
 //                        items), so the loads never pause at an item boundary.
 //       tcgen05 phase    Q and P in tensor memory, page groups of four (64 keys), S = Q K^T and O += P V as tcgen05.mma,
@@ -19,9 +20,9 @@
 //                        every nslots-th page (mma.sync m16n8k16 bf16, fp32 accumulate, ldmatrix from the swizzled
 //                        tiles), in order from its slot's sub-ring; the slots' (m, l, O) are merged through shared
 //                        memory (see mma_phase).
-//       output           an item of an uncut request writes bf16 output directly, otherwise normalised fp32 partials
-//                        and their log-sum-exp.
-//   attn_combine_kernel  merges the chunks of cut requests.
+//       output           an item that no segment boundary cuts writes bf16 output directly, a piece of a cut item
+//                        normalised fp32 partials and their log-sum-exp.
+//   attn_combine_kernel  merges the pieces of the cut items (one per boundary at most).
 //
 // The three kernels are chained with programmatic dependent launch.  Every mbarrier wait is bounded; on expiry the CTA
 // sets the device status word and every role leaves at a point where none is left waiting at a named barrier.
@@ -1518,8 +1519,8 @@ template <int DH>
 constexpr int kSmemBytes = kDataBytes<DH> + kTailPad<DH> + 1024 /* alignment slack */ + 1024 /* control block */;
 static_assert(sizeof(Ctrl) <= 1024, "control block");
 
-// Persistent kernel: one CTA per SM takes work items from two queues, first the tcgen05-path items, then the
-// warp-level-MMA items (each queue longest first, so the items that start last are the short ones).
+// Persistent kernel: one CTA per SM runs its segment of the work stream, first its tcgen05-path items, then its
+// warp-level-MMA items.
 template <int DH>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constant__ CUtensorMap v_map,
