@@ -293,6 +293,7 @@ struct AttnArgs {
     int n_q_heads, n_kv_heads;
     long long num_pages;
     float scale_log2;          // softmax scale * log2(e)
+    int q_row_bytes;           // head_dim * 2
     __nv_bfloat16* out;
     float* lse;                // [T, Hq] or null
     float* part_o;
@@ -381,6 +382,16 @@ __device__ __forceinline__ bool sched_fetch(Ctrl* c, const AttnArgs& a, int phas
         it.pad[0] = en.tc;
         it.pad[1] = en.row0;      // first query row of the item within the request's tile
         it.pad[2] = en.rows;      // query rows of the item
+        {
+            // the item's query rows will be fetched when the item before it ends: ask L2 for them now (256 bytes per
+            // row at head_dim 128; rows of one token are contiguous across the group's heads)
+            const int group = a.n_q_heads / a.n_kv_heads, dh_bytes = (int)(a.q_row_bytes);
+            for (int r = lane; r < en.rows; r += 32) {
+                const int t = (en.row0 + r) / group, hl = (en.row0 + r) - t * group;
+                const char* p = reinterpret_cast<const char*>(a.q) + ((size_t)(en.q0 + t) * a.n_q_heads + cur.h * group + hl) * dh_bytes;
+                for (int o = 0; o < dh_bytes; o += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + o));
+            }
+        }
         if (last) {
             cur.p = cur.p1;
         } else {
@@ -1785,6 +1796,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     aa.n_kv_heads = ctx->lim.n_kv_heads;
     aa.num_pages = num_pages;
     aa.scale_log2 = scale * 1.4426950408889634f;
+    aa.q_row_bytes = ctx->lim.head_dim * 2;
     aa.out = static_cast<__nv_bfloat16*>(out);
     aa.lse = lse;
     aa.part_o = ctx->d_part_o;
