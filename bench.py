@@ -913,7 +913,7 @@ def run_dcut(args):
     e2e = None
     try:
         w.ctx.set_cost_dense(cost)
-        if not is_layer:
+        if not is_layer and args.e2e_steps > 0:
             pin = lambda t: t.contiguous().pin_memory()
             h = dict(conf=pin(torch.from_numpy(sel.conf)), draft=pin(torch.from_numpy(sel.draft_ids)),
                      bonus=pin(torch.from_numpy(sel.bonus_ids)), ctx=pin(torch.from_numpy(sel.ctx_lens)),
