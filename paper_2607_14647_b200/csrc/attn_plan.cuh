@@ -62,23 +62,53 @@ __device__ __forceinline__ T plan_warp_scan(T v, int lane) {
     return v;
 }
 
-// exclusive scan over the CTA of one value per thread; prefix in `o`, total in `t` (`ws`: 33 values of shared memory)
-template <typename T>
-__device__ __forceinline__ void plan_block_exclusive_scan(T v, T* ws, T& o, T& t) {
+// exclusive scan over the CTA of two counts and two costs per thread at once (one pass of barriers): prefixes in `o`,
+// totals in `t`; `w0`..`w3`: 33 values of shared memory each
+struct PlanScan4 {
+    int n0, n1;
+    long long c0, c1;
+};
+__device__ __forceinline__ void plan_block_exclusive_scan4(const PlanScan4& v, int* w0, int* w1, long long* w2, long long* w3,
+                                                           PlanScan4& o, PlanScan4& t) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const T inc = plan_warp_scan(v, lane);
-    if (lane == 31) ws[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        const T w = lane < (int)(blockDim.x >> 5) ? ws[lane] : T(0);
-        const T winc = plan_warp_scan(w, lane);
-        ws[lane] = winc - w;
-        if (lane == 31) ws[32] = winc;
+    PlanScan4 inc;
+    inc.n0 = plan_warp_scan(v.n0, lane);
+    inc.n1 = plan_warp_scan(v.n1, lane);
+    inc.c0 = plan_warp_scan(v.c0, lane);
+    inc.c1 = plan_warp_scan(v.c1, lane);
+    if (lane == 31) {
+        w0[warp] = inc.n0;
+        w1[warp] = inc.n1;
+        w2[warp] = inc.c0;
+        w3[warp] = inc.c1;
     }
     __syncthreads();
-    o = ws[warp] + inc - v;
-    t = ws[32];
+    if (warp == 0) {
+        const bool in = lane < (int)(blockDim.x >> 5);
+        const int a0 = in ? w0[lane] : 0, a1 = in ? w1[lane] : 0;
+        const long long a2 = in ? w2[lane] : 0, a3 = in ? w3[lane] : 0;
+        const int s0 = plan_warp_scan(a0, lane), s1 = plan_warp_scan(a1, lane);
+        const long long s2 = plan_warp_scan(a2, lane), s3 = plan_warp_scan(a3, lane);
+        w0[lane] = s0 - a0;
+        w1[lane] = s1 - a1;
+        w2[lane] = s2 - a2;
+        w3[lane] = s3 - a3;
+        if (lane == 31) {
+            w0[32] = s0;
+            w1[32] = s1;
+            w2[32] = s2;
+            w3[32] = s3;
+        }
+    }
     __syncthreads();
+    o.n0 = w0[warp] + inc.n0 - v.n0;
+    o.n1 = w1[warp] + inc.n1 - v.n1;
+    o.c0 = w2[warp] + inc.c0 - v.c0;
+    o.c1 = w3[warp] + inc.c1 - v.c1;
+    t.n0 = w0[32];
+    t.n1 = w1[32];
+    t.c0 = w2[32];
+    t.c1 = w3[32];
 }
 
 // Row blocks of a query tile of M rows: full blocks of max_rows rows and one remainder.  A remainder of at most
@@ -96,8 +126,8 @@ __device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, in
 // Every thread of the CTA calls this (it synchronises the CTA).  `prefix` is shared memory for 2 B + 1 64-bit values:
 // the cost of the stream before each entry.
 __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* prefix) {
-    __shared__ long long ws64[33];
-    __shared__ int ws32[33];
+    __shared__ long long ws64[33], ws64b[33];
+    __shared__ int ws32[33], ws32b[33];
     __shared__ int total_s, w_tc_s, w_mma_s;
     __shared__ AttnSeg seg_s[kMaxSegs + 1];
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -158,12 +188,12 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             }
         }
     }
-    int off_tc, off_mma, n_tc, n_mma;
-    long long pre_tc, pre_mma, tot_tc, tot_mma;
-    plan_block_exclusive_scan<int>(my_tc, ws32, off_tc, n_tc);
-    plan_block_exclusive_scan<int>(my_mma, ws32, off_mma, n_mma);
-    plan_block_exclusive_scan<long long>(c_tc, ws64, pre_tc, tot_tc);
-    plan_block_exclusive_scan<long long>(c_mma, ws64, pre_mma, tot_mma);
+    PlanScan4 sc_o, sc_t;
+    plan_block_exclusive_scan4(PlanScan4{my_tc, my_mma, c_tc, c_mma}, ws32, ws32b, ws64, ws64b, sc_o, sc_t);
+    int off_tc = sc_o.n0, off_mma = sc_o.n1;
+    const int n_tc = sc_t.n0, n_mma = sc_t.n1;
+    long long pre_tc = sc_o.c0, pre_mma = sc_o.c1;
+    const long long tot_tc = sc_t.c0, tot_mma = sc_t.c1;
     const int n_entries = n_tc + n_mma;
     const long long total = tot_tc + tot_mma;
     const bool overflow = n_entries > a.max_entries;      // cannot happen with a context sized for the batch; defensive

@@ -50,6 +50,8 @@ __device__ __forceinline__ float clamp_conf(float c) {
     return c;
 }
 
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 template <typename T>
 __device__ __forceinline__ T warp_inclusive_scan(T v, int lane) {
 #pragma unroll
@@ -86,70 +88,84 @@ __device__ __forceinline__ unsigned long long cx(unsigned long long mine, unsign
     return ((mine < other) == keep_min) ? mine : other;
 }
 
-template <int E>
-__device__ __forceinline__ void sort_keys_e(unsigned long long* keys, unsigned long long (*xbuf)[kThreads], int npad) {
+// order a pair held by one thread: ascending if `up`
+__device__ __forceinline__ void cx_pair(unsigned long long& a, unsigned long long& b, bool up) {
+    const unsigned long long x = a, y = b;
+    const bool swap = (x > y) == up;
+    a = swap ? y : x;
+    b = swap ? x : y;
+}
+
+// Bitonic sort, ascending, of the npad keys in `keys` (shared memory), held in registers meanwhile: KPT consecutive
+// keys per thread of the first S / KPT threads (S = max(npad, 32 KPT) keys with padding); the other warps wait at the
+// closing barrier.  Compare-exchange distances below KPT stay inside a thread, the next five are warp shuffles, the
+// rest cross warps through shared memory: `keys` itself and `alt` (npad words, free during the sort) alternate as the
+// exchange buffer, with one named barrier of the sorting warps per stage.  One loop per kind of stage keeps the code
+// small: the kernel starts with cold instruction caches in every step, and a network unrolled for each size, though
+// a third faster once warm, made the step slower.
+template <int KPT>
+__device__ __forceinline__ void sort_keys_blocked(unsigned long long* keys, unsigned long long* alt, int npad) {
     const int tid = threadIdx.x;
-    unsigned long long k[E];
+    int S = 32 * KPT;
+    while (S < npad) S <<= 1;
+    const int nt = S / KPT;                              // sorting threads: a multiple of 32
+    if (tid < nt) {
+        unsigned long long k[KPT];
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const int idx = e * kThreads + tid;
-        k[e] = idx < npad ? keys[idx] : ~0ull;
-    }
-    __syncthreads();
-    int p = 0;
-    constexpr int S = E * kThreads;
-    for (int kk = 2; kk <= S; kk <<= 1) {
-        for (int j = kk >> 1; j > 0; j >>= 1) {
-            if (j >= kThreads) {                      // partner in the same thread
+        for (int e = 0; e < KPT; ++e) {
+            const int idx = KPT * tid + e;
+            k[e] = idx < npad ? keys[idx] : ~0ull;
+        }
+        int p = 0;
+        for (int kk = 2; kk <= S; kk <<= 1) {
+            const bool up_t = ((KPT * tid) & kk) == 0;   // direction of this thread's keys in the stages across threads
+            int j = kk >> 1;
+            for (; j >= 32 * KPT; j >>= 1) {             // partner thread in another warp (then S = npad >= 64 KPT)
+                const int jt = j / KPT;
+                const bool keep_min = up_t == ((tid & jt) == 0);
+                unsigned long long* xb = p ? keys : alt;
+                unsigned long long o[KPT];
 #pragma unroll
-                for (int je = E / 2; je >= 1; je >>= 1) {
-                    if (j == je * kThreads) {
+                for (int e = 0; e < KPT; ++e) xb[e * nt + tid] = k[e];
+                asm volatile("bar.sync 1, %0;" ::"r"(nt) : "memory");
 #pragma unroll
-                        for (int e = 0; e < E; ++e) {
-                            if ((e & je) == 0) {
-                                const int idx = e * kThreads + tid;
-                                const bool up = (idx & kk) == 0;
-                                const unsigned long long a = k[e], b = k[e | je];
-                                const bool swap = (a > b) == up;
-                                k[e] = swap ? b : a;
-                                k[e | je] = swap ? a : b;
-                            }
-                        }
-                    }
-                }
-            } else if (j >= 32) {                     // partner in another warp: through shared memory
+                for (int e = 0; e < KPT; ++e) o[e] = xb[e * nt + (tid ^ jt)];
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    xbuf[p][tid] = k[e];
-                    __syncthreads();
-                    const unsigned long long other = xbuf[p][tid ^ j];
-                    const int idx = e * kThreads + tid;
-                    k[e] = cx(k[e], other, ((idx & kk) == 0) == ((tid & j) == 0));
-                    p ^= 1;
-                }
-            } else {                                  // partner in the same warp
+                for (int e = 0; e < KPT; ++e) k[e] = cx(k[e], o[e], keep_min);
+                p ^= 1;
+            }
+            for (; j >= KPT; j >>= 1) {                  // partner thread in the same warp; same slot e
+                const int jt = j / KPT;
+                const bool keep_min = up_t == ((tid & jt) == 0);
+                unsigned long long o[KPT];
 #pragma unroll
-                for (int e = 0; e < E; ++e) {
-                    const unsigned long long other = __shfl_xor_sync(0xffffffffu, k[e], j);
-                    const int idx = e * kThreads + tid;
-                    k[e] = cx(k[e], other, ((idx & kk) == 0) == ((tid & j) == 0));
+                for (int e = 0; e < KPT; ++e) o[e] = __shfl_xor_sync(0xffffffffu, k[e], jt);
+#pragma unroll
+                for (int e = 0; e < KPT; ++e) k[e] = cx(k[e], o[e], keep_min);
+            }
+#pragma unroll
+            for (int je = KPT / 2; je >= 1; je >>= 1) {  // partner key in the same thread (constant register indices)
+                if (je <= j) {
+#pragma unroll
+                    for (int e = 0; e < KPT; ++e)
+                        if ((e & je) == 0) cx_pair(k[e], k[e | je], ((KPT * tid + e) & kk) == 0);
                 }
             }
         }
-    }
+        // the last exchange buffer may have been `keys`: everybody has read it before the sorted keys go there
+        asm volatile("bar.sync 1, %0;" ::"r"(nt) : "memory");
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const int idx = e * kThreads + tid;
-        if (idx < npad) keys[idx] = k[e];
+        for (int e = 0; e < KPT; ++e) {
+            const int idx = KPT * tid + e;
+            if (idx < npad) keys[idx] = k[e];
+        }
     }
     __syncthreads();
 }
 
-__device__ __forceinline__ void sort_keys(unsigned long long* keys, unsigned long long (*xbuf)[kThreads], int npad) {
-    if (npad <= kThreads) sort_keys_e<1>(keys, xbuf, npad);
-    else if (npad <= 2 * kThreads) sort_keys_e<2>(keys, xbuf, npad);
-    else if (npad <= 4 * kThreads) sort_keys_e<4>(keys, xbuf, npad);
-    else sort_keys_e<8>(keys, xbuf, npad);
+__device__ __forceinline__ void sort_keys(unsigned long long* keys, unsigned long long* alt, int npad) {
+    if (npad <= 4 * kThreads) sort_keys_blocked<4>(keys, alt, npad);
+    else sort_keys_blocked<8>(keys, alt, npad);
 }
 
 struct Best {
@@ -169,7 +185,6 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     long long* qs = reinterpret_cast<long long*>(keys + npad);                       // [npad + 1]
     int* depth_s = reinterpret_cast<int*>(qs + npad + 1);                            // [B]
     int* cu_s = depth_s + B;                                                         // [B + 1]
-    __shared__ unsigned long long xbuf[2][kThreads];
     __shared__ long long ws64[kWarps + 1];
     __shared__ int ws32[kWarps + 1];
     __shared__ Best wbest[kWarps];
@@ -178,6 +193,20 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
 
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
+    // What the later steps read from global memory, each after a barrier and hence with its full latency exposed:
+    // ask for it now (between two steps of a serving loop the KV stream has pushed all of it out of L2).
+    {
+        const size_t cost_bytes = sizeof(float) * (size_t)(a.n_buckets > 0 ? a.n_buckets : n + 1);
+        const char* cost0 = reinterpret_cast<const char*>(a.cost + (a.n_buckets > 0 ? 0 : B));
+        for (size_t off = (size_t)tid * 128; off < cost_bytes; off += (size_t)kThreads * 128) prefetch_l2(cost0 + off);
+        for (size_t off = (size_t)tid * 128; off < sizeof(int) * (size_t)n; off += (size_t)kThreads * 128)
+            prefetch_l2(reinterpret_cast<const char*>(a.draft_ids) + off);
+        for (size_t off = (size_t)tid * 128; off < sizeof(int) * (size_t)B; off += (size_t)kThreads * 128) {
+            prefetch_l2(reinterpret_cast<const char*>(a.ctx_lens) + off);
+            prefetch_l2(reinterpret_cast<const char*>(a.bonus_ids) + off);
+        }
+        if (a.n_buckets > 0 && tid == 0) prefetch_l2(a.bucket_K);
+    }
     // 1. prefix scores and sort keys.  The confidences come in through shared memory with coalesced loads
     // (the later prefix-sum array is free at this point), so the per-request product chain reads no global memory.
     float* conf_s = reinterpret_cast<float*>(qs);
@@ -200,10 +229,9 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
     for (int r = n + tid; r < npad; r += kThreads) keys[r] = ~0ull;
     for (int i = tid; i < B; i += kThreads) depth_s[i] = 0;
     __syncthreads();
-    // 2. bitonic sort, ascending, over S = max(npad, 1024) keys held in registers: thread t owns elements
-    // e * 1024 + t.  Compare-exchange distances below 32 go through warp shuffles, distances 32..512 through a
-    // double-buffered shared array (one barrier per stage), distances >= 1024 stay inside the thread.
-    sort_keys(keys, xbuf, npad);
+    // 2. bitonic sort, ascending, with the keys held in registers (sort_keys_blocked); the prefix-sum array is free
+    // until step 3 and serves as the second exchange buffer
+    sort_keys(keys, reinterpret_cast<unsigned long long*>(qs), npad);
     // 3. fixed-point prefix sums Q[0..n]; ranks
     {
         const int per = (npad + kThreads - 1) / kThreads;
