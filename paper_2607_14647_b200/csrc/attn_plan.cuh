@@ -24,17 +24,18 @@ constexpr int kSlotRows = 144;       // rows of a partial-result slot (the large
 constexpr int kMaxSegs = 256;        // segments (SMs) the plan handles
 
 // Cost model, nanoseconds on B200, fitted to the busy time of the item kernel's CTAs against the items and pages of
-// their segments (least squares over the 148 CTAs of batches of equal query tiles).  Per page: 168-171 on the
-// warp-level phase (4- and 8-row tiles), 186 on the tcgen05 phase at 68 rows, 209 at 136 rows (128 + tail rows).  Per
-// item, beyond its pages: 2.4-2.6 us on the warp-level phase, 3.6 us (68 rows) to 5.5 us (136 rows) on the tcgen05
-// phase, where O is single-buffered in tensor memory and the softmax -> PV chain drains at an item boundary (4.4 / 6.3
-// before the next item's query tile was staged ahead of the epilogue).  Only ratios matter for the partition.
+// their segments (least squares over the 148 CTAs, batches of mixed and of equal query tiles).  With every SM streaming,
+// a page costs what the shared HBM gives each SM, whatever the phase: 176-191 on the tcgen05 phase (188), 193-202 with
+// tail rows (196), 161-176 on the warp-level phase (180 balances mixed batches best: CTAs with only warp-level items
+// finished 5 % late at 169).  Per item, beyond its pages: 2.1-2.8 us on the warp-level phase, 2.9-3.5 us on the
+// tcgen05 phase, 5.9-6.8 us with tail rows (O is single-buffered in tensor memory and the softmax -> PV chain drains
+// at an item boundary; CTAs with many short tail-row items were the last to finish at 5.5).  Only ratios matter.
 __device__ __forceinline__ int cost_per_page(int rows, int tc) {
-    if (tc) return rows > 128 ? 209 : 186;                 // every lane of tensor memory is processed, whatever the valid rows
+    if (tc) return rows > 128 ? 196 : 188;                 // every lane of tensor memory is processed, whatever the valid rows
     const int mt = (rows + 15) >> 4;                       // m-tiles of the warp-level phase: memory-bound up to two
-    return 169 * max(7, 3 * mt) / 7;
+    return 180 * max(7, 3 * mt) / 7;
 }
-__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 5500 : 3600) : 2500; }
+__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 7500 : 3800) : 2500; }
 
 struct PlanArgs {
     const int* ctx_lens;

@@ -131,6 +131,32 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Two fp32 values in one 64-bit register and the sm_100 instructions that work on both at once: the softmax warps of
+// the tcgen05 phase are short of issue slots, not of arithmetic.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// maximum of three (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 // byte offset of 16-byte chunk `c16` (0 .. DH/8-1) of token/row `r` (0..15) inside a swizzled
 // [DH/64][16][64] bf16 tile (what two 64-column TMA boxes with 128-byte swizzle produce)
 __device__ __forceinline__ uint32_t tile_off(int r, int c16) {
@@ -984,15 +1010,12 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                 if (ncols < 64 || j0 + 63 > ctx_len) {                  // a partial group or one that holds hidden keys
                     const int lim = min(ncols - 1, jmax - j0);          // columns 0..lim are visible
 #pragma unroll
-                    for (int e = 0; e < 64; ++e) {
-                        const float v = e <= lim ? __uint_as_float(sr[e]) : -INFINITY;
-                        sr[e] = __float_as_uint(v);
-                        mx4[e & 3] = fmaxf(mx4[e & 3], v);
-                    }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 64; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sr[e]));
+                    for (int e = 0; e < 64; ++e) sr[e] = e <= lim ? sr[e] : 0xff800000u;   // -inf
                 }
+#pragma unroll
+                for (int e = 0; e < 64; e += 8)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) mx4[k] = fmax3(mx4[k], __uint_as_float(sr[e + k]), __uint_as_float(sr[e + 4 + k]));
                 const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 // the running maximum only moves (and O is only rescaled) when it would grow by more than 2^8
                 float alpha = 1.0f;
@@ -1021,16 +1044,23 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
                     tc_wait_st();
                 }
                 const float mc = (m_run == -INFINITY ? 0.0f : m_run) * cs;
-                float sum4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                const unsigned long long cs2 = pack_f32x2(cs, cs), nmc2 = pack_f32x2(-mc, -mc);
+                unsigned long long sum2[2] = {0ull, 0ull};                // four partial sums, two per register
                 uint32_t pw[32];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[2 * e]), cs, -mc));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[2 * e + 1]), cs, -mc));
-                    sum4[e & 3] += p0 + p1;
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[2 * e]), __uint_as_float(sr[2 * e + 1])), cs2, nmc2), x0, x1);
+                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                    sum2[e & 1] = add_f32x2(sum2[e & 1], pack_f32x2(p0, p1));
                     pw[e] = pack_bf16(p0, p1);
                 }
-                l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+                {
+                    float s0, s1, s2, s3;
+                    unpack_f32x2(sum2[0], s0, s1);
+                    unpack_f32x2(sum2[1], s2, s3);
+                    l_run += (s0 + s1) + (s2 + s3);
+                }
                 tc_st32(t_s, pw);                                         // P over the columns S occupied
                 tc_wait_st();
                 tc_fence_before();
