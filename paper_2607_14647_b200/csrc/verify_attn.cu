@@ -992,12 +992,20 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             if (!q_staged) store_q(item);
             q_staged = false;
             const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
+            const bool live = quarter * 32 < M;                          // (warp-uniform) some of this warp's rows exist
             float m_run = -INFINITY, l_run = 0.0f;
             for (int g = team; g < n_groups; g += 2) {
                 const int gc = G0 + g, b = gc % kTcSBufs;
                 if (!failed && !mbar_wait(s_full + 8 * b, (gc / kTcSBufs) & 1, &c->abort)) failed = true;
                 failed = __any_sync(0xffffffffu, failed);
                 if (failed) break;
+                if (!live) {
+                    // None of this warp's 32 rows exists (a query tile of at most 96, 64 or 32 rows): nothing to compute.
+                    // Its lanes of P keep the raw scores and its rows of O whatever the MMAs make of them; rows of
+                    // the accumulators are independent and these are never read.
+                    mbar_arrive(p_full + 8 * b);
+                    continue;
+                }
                 const uint32_t t_s = t_lane + kTcColS + 64 * b;
                 uint32_t sr[64];
                 tc_fence_after();
@@ -1104,8 +1112,12 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             const float f_s = w_s * inv, f_o = w_o * inv;
             const int t = (row0 + R) / group, hl = (row0 + R) - t * group;
             const size_t orow = (size_t)(q0 + t) * a.n_q_heads + kvh * group + hl;
+            if (!live) {
+                tc_fence_before();
+                mbar_arrive(o_free);
+            }
 #pragma unroll 1
-            for (int hh = 0; hh < 2; ++hh) {
+            for (int hh = 0; live && hh < 2; ++hh) {
                 const int cc = 64 * team + 32 * hh;
                 uint32_t os[32], oo[32];
                 tc_ld32(t_mine + cc, os);
