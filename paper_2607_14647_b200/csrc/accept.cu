@@ -27,6 +27,12 @@ __device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
 
 __device__ __forceinline__ unsigned int ordered_bits(float f) { return dcut_ordered_bits(f); }
 
+__device__ __forceinline__ unsigned int max_bf16x2(unsigned int x, unsigned int y) {   // a NaN operand is ignored
+    unsigned int r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(x), "r"(y));
+    return r;
+}
+
 __device__ __forceinline__ void take(float f, int idx, float& best, int& bidx) {
     if (f > best) {   // strict: the first of equal values stays; NaN never passes
         best = f;
@@ -74,14 +80,24 @@ __global__ void __launch_bounds__(kArgmaxThreads) accept_argmax_kernel(
     const int tail0 = body0 + (nvec << 3);
     if ((int)threadIdx.x < head)
         take(__uint_as_float((unsigned int)rp[start + threadIdx.x] << 16), start + threadIdx.x, best, bidx);
+    // A thread keeps the packed bf16x2 maximum of the vectors it has seen (one max.bf16x2 per 4 bytes, NaNs ignored);
+    // only a batch of loads that raises one of its halves can hold a value above `best`, and only such a batch is
+    // looked at value by value for (maximum, first index).  After the first few batches that is rare.
     const uint4* vp = reinterpret_cast<const uint4*>(rp + body0);
+    unsigned int best2 = 0xff80ff80u;                 // (-inf, -inf)
     int v = threadIdx.x;
     for (; v + (kUnroll - 1) * kArgmaxThreads < nvec; v += kUnroll * kArgmaxThreads) {
         uint4 x[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) x[u] = ld_stream_v4(vp + v + u * kArgmaxThreads);
+        unsigned int m2 = best2;
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) take8(x[u], body0 + ((v + u * kArgmaxThreads) << 3), best, bidx);
+        for (int u = 0; u < kUnroll; ++u) m2 = max_bf16x2(m2, max_bf16x2(max_bf16x2(x[u].x, x[u].y), max_bf16x2(x[u].z, x[u].w)));
+        if (m2 != best2) {
+            best2 = m2;
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) take8(x[u], body0 + ((v + u * kArgmaxThreads) << 3), best, bidx);
+        }
     }
     for (; v < nvec; v += kArgmaxThreads) take8(ld_stream_v4(vp + v), body0 + (v << 3), best, bidx);
     // a thread's indices ascend except for the tail, which lies past every body index
