@@ -1,7 +1,8 @@
 """Decoder-layer path against the oracle: the tcgen05 GEMM by itself (all three epilogues), RMSNorm + RoPE + cache
 append through the whole layer on a small shape (every element, every stage that is visible), and the full-layer
 workload on a sub-batch of requests the oracle can afford.  Tolerance 2e-2 + 2e-2 |ref| (bf16 tensors, fp32
-accumulation over K up to 12 288; the paper gives none)."""
+accumulation over K up to 12 288; the paper gives none); for the layer output, |ref| is the larger of the output and of
+the residual stream h1 it is added to, since both terms of that sum are rounded to bf16 before it."""
 import numpy as np
 import pytest
 import torch
@@ -13,11 +14,17 @@ from tests.gpu_helpers import dev, make_ctx
 pytestmark = pytest.mark.gpu
 
 
-def _close(got, want, what):
-    got = got.float().cpu().numpy().astype(np.float64)
-    want = want.float().numpy().astype(np.float64) if isinstance(want, torch.Tensor) else np.asarray(want, np.float64)
+def _f64(t):
+    return t.float().cpu().numpy().astype(np.float64) if isinstance(t, torch.Tensor) else np.asarray(t, np.float64)
+
+
+def _close(got, want, what, size=None):
+    """|got - want| <= 2e-2 + 2e-2 s elementwise, s = |want|, or the larger of |want| and |size| where the value is a
+    sum whose terms were rounded to bf16 on their own (the layer output y = h1 + MLP: an element that is 1.24 after
+    attention and 0.10 after the MLP carries the rounding step of 1.24)."""
+    got, want = _f64(got), _f64(want)
     err = np.abs(got - want)
-    lim = 2e-2 + 2e-2 * np.abs(want)
+    lim = 2e-2 + 2e-2 * (np.abs(want) if size is None else np.maximum(np.abs(want), np.abs(_f64(size))))
     assert (err <= lim).all(), f"{what}: worst err/limit {(err / lim).max():.2f} at {np.unravel_index((err / lim).argmax(), err.shape)}"
 
 
@@ -83,7 +90,7 @@ def _layer_case(cfg, depths, hidden, inter, sub=None):
     rows = np.concatenate([np.arange(cu[i], cu[i + 1]) for i in sub])
     ref = orc.layer_forward(x[rows], wd, kv.k_cache, kv.v_cache, kv.block_table[sub], sel.ctx_lens[sub], depths[sub],
                             cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.page_size, cfg.rms_eps, cfg.rope_theta)
-    _close(y[rows], ref["y"], "layer output y")
+    _close(y[rows], ref["y"], "layer output y", size=ref["h1"])
     # the appended K/V of the new tokens (the rest of the cache must be untouched)
     kc, vc = d_k.cpu(), d_v.cpu()
     for n_, i in enumerate(sub):
@@ -367,7 +374,7 @@ def test_tensor_parallel_halves_reproduce_the_layer(tp):
     assert all(torch.equal(ys[0], y) for y in ys[1:])
     ref = orc.layer_forward(x, wd, kv.k_cache, kv.v_cache, kv.block_table, sel.ctx_lens, depths, Hq, Hkv, Dh, cfg.page_size,
                             cfg.rms_eps, cfg.rope_theta)
-    _close(ys[0], ref["y"], "tensor-parallel layer output y")
+    _close(ys[0], ref["y"], "tensor-parallel layer output y", size=ref["h1"])
     # the unsharded call on the same inputs: same output within the layer's tolerance, same appended K/V bit for bit
     ctx = make_ctx(cfg, max_pages=kv.max_pages_per_req, hidden=hidden, intermediate=inter, vocab=0)
     y_full = torch.empty((T, hidden), **bf)
