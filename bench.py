@@ -45,7 +45,7 @@ L2_BYTES = 126e6
 # DRAM bytes per algorithmic byte of attn_item_kernel, from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum of
 # one launch) summarised in profiles/attn_item_kernel_dram_traffic.md: 1.001-1.005 over the three arms of workload 2 at
 # full size and of workload 3's shapes at B = 48; the kernel's traffic is proportional to the KV it streams
-ATTN_TRAFFIC_RATIO = 1.003
+ATTN_TRAFFIC_RATIO = 1.004
 RATIO_BUCKETS = [(1, 4), (1, 2), (3, 4), (1, 1)]          # the paper's ratio set R (Eq. 4; Table 3)
 COST_PROFILE_DIR = os.path.join(ROOT, "paper_2607_14647_b200", "cost_profiles")
 
