@@ -25,17 +25,19 @@ constexpr int kMaxSegs = 256;        // segments (SMs) the plan handles
 
 // Cost model, nanoseconds on B200, fitted to the busy time of the item kernel's CTAs against the items and pages of
 // their segments (least squares over the 148 CTAs, batches of mixed and of equal query tiles).  With every SM streaming,
-// a page costs what the shared HBM gives each SM, whatever the phase: 176-191 on the tcgen05 phase (188), 193-202 with
-// tail rows (196), 161-176 on the warp-level phase (180 balances mixed batches best: CTAs with only warp-level items
-// finished 5 % late at 169).  Per item, beyond its pages: 2.1-2.8 us on the warp-level phase, 2.9-3.5 us on the
-// tcgen05 phase, 5.9-6.8 us with tail rows (O is single-buffered in tensor memory and the softmax -> PV chain drains
-// at an item boundary; CTAs with many short tail-row items were the last to finish at 5.5).  Only ratios matter.
-__device__ __forceinline__ int cost_per_page(int rows, int tc) {
-    if (tc) return rows > 128 ? 196 : 188;                 // every lane of tensor memory is processed, whatever the valid rows
+// a page costs about what the shared HBM gives each SM, a little less for the CTAs that can take more.  tcgen05 phase:
+// 188 per page, 196 with tail rows, but 166 when the shapes never have tail rows (`tc_alone`: the producer and the MMA
+// issuer then run on schedulers that hold no busy softmax warps, and CTAs with only such items finished 10 % early at
+// 188); warp-level phase 176.  Per item, beyond its pages: 3.8 us on the tcgen05 phase, 7.5 us with tail rows (O is
+// single-buffered in tensor memory and the softmax -> PV chain drains at an item boundary; the tail warps add their
+// merge), 3 us on the warp-level phase (2.1-2.8 in batches of such items only; CTAs with two or three short warp-level
+// items among tcgen05 CTAs were the last to finish on small batches at 2.5).  Only ratios matter for the partition.
+__device__ __forceinline__ int cost_per_page(int rows, int tc, int tc_alone) {
+    if (tc) return rows > 128 ? 196 : (tc_alone ? 166 : 188);   // every lane of tensor memory is processed, whatever the valid rows
     const int mt = (rows + 15) >> 4;                       // m-tiles of the warp-level phase: memory-bound up to two
-    return 180 * max(7, 3 * mt) / 7;
+    return 176 * max(7, 3 * mt) / 7;
 }
-__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 7500 : 3800) : 2500; }
+__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 7500 : 3800) : 3000; }
 
 struct PlanArgs {
     const int* ctx_lens;
@@ -43,6 +45,7 @@ struct PlanArgs {
     int B, n_q_heads, n_kv_heads;
     int n_sm;                           // segments = CTAs of the item kernel
     int min_chunk_pages;                // no piece of a cut item is shorter than this
+    int tc_alone;                       // the shapes never give a query tile above 128 rows (see the cost model)
     int tc_min_rows, max_item_rows;
     int tail_rows;                      // a remainder of at most this many rows rides with the last full row block (0: never)
     int max_entries;
@@ -129,7 +132,7 @@ __device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, in
 __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* prefix) {
     __shared__ long long ws64[33], ws64b[33];
     __shared__ int ws32[33], ws32b[33];
-    __shared__ int total_s, w_tc_s, w_mma_s;
+    __shared__ int total_s, w_tc_s, w_mma_s, w_tall_s;
     __shared__ AttnSeg seg_s[kMaxSegs + 1];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -137,11 +140,12 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
         total_s = 0;
         w_tc_s = 0;
         w_mma_s = 0;
+        w_tall_s = 0;
     }
     __syncthreads();
     // pass 1: pages in all, and how they would split over the two phases of the item kernel
     {
-        int local = 0, w_tc = 0, w_mma = 0;
+        int local = 0, w_tc = 0, w_mma = 0, w_tall = 0;
         for (int i = tid; i < a.B; i += nthr) {
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
@@ -149,13 +153,18 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             const int M = (d + 1) * group;
             const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
             int tc_rb = 0;
-            for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= a.tc_min_rows ? 1 : 0;
+            for (int rb = 0; rb < n_rb; ++rb) {
+                const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
+                tc_rb += rows >= a.tc_min_rows ? 1 : 0;
+                w_tall += rows > 96 ? pages : 0;               // rows in the last lane quarter of tensor memory
+            }
             w_tc += pages * tc_rb;
             w_mma += pages * (n_rb - tc_rb);
         }
         if (local) atomicAdd(&total_s, local);
         if (w_tc) atomicAdd(&w_tc_s, w_tc);
         if (w_mma) atomicAdd(&w_mma_s, w_mma);
+        if (w_tall) atomicAdd(&w_tall_s, w_tall);
     }
     __syncthreads();
     // The item kernel runs a segment's tcgen05 items first and its warp-level items after them.  When the second kind
@@ -178,7 +187,7 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             for (int rb = 0; rb < n_rb; ++rb) {
                 const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
                 const int tc = rows >= tc_min_rows;
-                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc));
+                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc, a.tc_alone));
                 if (tc) {
                     ++my_tc;
                     c_tc += c;
@@ -202,6 +211,9 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
         a.plan[0] = overflow ? 0 : n_entries;
         a.plan[1] = overflow ? 0 : n_tc;
         a.plan[2] = total_s;
+        // Which warps of the item kernel's tcgen05 phase run the producer and the MMA issuer (see tc_phase): the ones on
+        // the schedulers of lane quarters 2 and 3 when most pages belong to query tiles that leave quarter 3 empty.
+        a.plan[3] = 2 * w_tall_s < w_tc_s ? 1 : 0;
         if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
     }
     if (overflow) {
@@ -225,7 +237,7 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             for (int rb = 0; rb < n_rb; ++rb) {
                 const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
                 const int tc = rows >= tc_min_rows;
-                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc));
+                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc, a.tc_alone));
                 AttnEntry en;
                 en.req = i;
                 en.row0 = rb * a.max_item_rows;
@@ -268,7 +280,7 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             // page (the segment between them would hold an empty piece that nobody writes): consecutive positions are
             // at least total / n_sm apart, so they land on different multiples as long as a segment is worth at least
             // min_chunk_pages of this item; below that (tiny batches) the item is not cut at all.
-            const long long quantum = (long long)a.min_chunk_pages * cost_per_page(en.rows, en.tc);
+            const long long quantum = (long long)a.min_chunk_pages * cost_per_page(en.rows, en.tc, a.tc_alone);
             int p = (in_item <= 0 || total / a.n_sm < quantum) ? 0 : (int)(in_item / quantum) * a.min_chunk_pages;
             if (en.pages - p < a.min_chunk_pages) {          // the rest is too short to be a piece: the boundary moves to the next item
                 p = 0;

@@ -320,6 +320,7 @@ struct AttnArgs {
     long long num_pages;
     float scale_log2;          // softmax scale * log2(e)
     int q_row_bytes;           // head_dim * 2
+    int tail_on;               // query tiles above 128 rows can occur with this context's shapes: the tail warps take part
     __nv_bfloat16* out;
     float* lse;                // [T, Hq] or null
     float* part_o;
@@ -806,7 +807,18 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
     const uint32_t full_bar = smem_u32(c->ring_full), empty_bar = smem_u32(c->ring_empty);
     const uint32_t s_full = smem_u32(c->s_full), p_full = smem_u32(c->p_full), pv_done = smem_u32(c->pv_done);
     const uint32_t q_ready = smem_u32(&c->q_ready), o_free = smem_u32(&c->o_free);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
+    // Role of this warp.  A softmax warp must be the warp whose number mod 4 is its lane quarter of tensor memory, which
+    // is also its scheduler: warps 2-9.  The producer (role 0) and the MMA issuer (role 1) run on warps 0 and 1 and the
+    // tail warps (roles 10, 11) on warps 10 and 11 when the query tiles fill all four lane quarters: the schedulers
+    // prefer their lower-numbered warps, so the issuer goes ahead of the softmax warps it shares a scheduler with and
+    // the instruction-heavy tail warps behind them (the other way round full-depth 136-row tiles lost 8 %).  When most
+    // pages belong to tiles that leave quarter 3 empty (32q/8kv at depth 16: 68 rows; pruned batches) the plan says so
+    // and the two pairs swap: producer and issuer get schedulers 2 and 3 to themselves instead of sharing 0 and 1 with
+    // the softmax warps that always have rows (scheduler 3 issued 6 % of the time on 68-row tiles): +9 % at full depth
+    // on the 32q/8kv workload.
+    const int pw = tid >> 5;
+    const int warp = a.plan[3] ? (pw >= 10 ? pw - 10 : (pw < 2 ? pw + 10 : pw)) : pw;
     const int group = a.n_q_heads / a.n_kv_heads;
     const uint32_t tmem_o = c->tmem_base;
     AttnItem item;
@@ -1157,8 +1169,10 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             sched_release(c, kPhase, n);
             G0 += n_groups;
         }
-    } else if (warp < 2 + kTcSoftmaxThreads / 32 + kTcTailWarps) {
+    } else if (a.tail_on) {
         // ---------------------------------------------------------------- tail rows (128 .. 143 of the item)
+        // (with shapes whose query tiles never exceed 128 rows these two warps have no part in the phase: no stage and
+        // no item waits for them)
         // One m16 tile by warp-level MMA on the staged pages; warp tw takes the item's pages p with p mod 2 = tw.
         // Both warps walk every group of every item, because every stage of the ring waits for their arrival.
         const int tw = warp - (2 + kTcSoftmaxThreads / 32);
@@ -1587,7 +1601,7 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) {
             mbar_init(smem_u32(&c->ring_full[s]), 1);    // tcgen05 phase: one arrival (with the group's byte count)
-            mbar_init(smem_u32(&c->ring_empty[s]), 1 + kTcTailWarps);   // the commit of the stage's last MMA + the tail warps
+            mbar_init(smem_u32(&c->ring_empty[s]), 1 + (a.tail_on ? kTcTailWarps : 0));   // the commit of the stage's last MMA + the tail warps
         }
         for (int b = 0; b < kTcSBufs; ++b) {
             mbar_init(smem_u32(&c->s_full[b]), 1);
@@ -1599,7 +1613,7 @@ attn_item_kernel(const __grid_constant__ CUtensorMap k_map, const __grid_constan
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&c->sched_full[0][s]), 1);
             mbar_init(smem_u32(&c->sched_full[1][s]), 1);
-            mbar_init(smem_u32(&c->sched_empty[0][s]), 1 + kTcSoftmaxThreads / 32 + kTcTailWarps);   // MMA warp + softmax warps + tail warps
+            mbar_init(smem_u32(&c->sched_empty[0][s]), 1 + kTcSoftmaxThreads / 32 + (a.tail_on ? kTcTailWarps : 0));   // MMA warp + softmax warps + tail warps
             mbar_init(smem_u32(&c->sched_empty[1][s]), kMmaWarps);
         }
         mbar_init(smem_u32(&c->geom_a), kMmaWarps + 1);
@@ -1782,6 +1796,7 @@ void dcut_fill_plan_args(dcut_ctx* ctx, const int* ctx_lens, const int* cu_q, in
     pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
     pa.max_item_rows = 128;
     pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? ctx->attn_tail_rows : 0;
+    pa.tc_alone = !(ctx->attn_tail_rows > 0 && (ctx->lim.max_gamma + 1) * (ctx->lim.n_q_heads / ctx->lim.n_kv_heads) > 128);
     pa.max_entries = ctx->max_entries;
     pa.entries = ctx->d_entries;
     pa.segs = ctx->d_segs;
@@ -1839,6 +1854,7 @@ dcut_status dcut_launch_verify_attn(dcut_ctx* ctx, const void* q, const void* k_
     aa.num_pages = num_pages;
     aa.scale_log2 = scale * 1.4426950408889634f;
     aa.q_row_bytes = ctx->lim.head_dim * 2;
+    aa.tail_on = ctx->attn_tail_rows > 0 && (ctx->lim.max_gamma + 1) * (ctx->lim.n_q_heads / ctx->lim.n_kv_heads) > 128;
     aa.out = static_cast<__nv_bfloat16*>(out);
     aa.lse = lse;
     aa.part_o = ctx->d_part_o;
