@@ -2,8 +2,7 @@
 //
 // Two launches.
 //   accept_argmax_kernel  HBM-bound scan of the bf16 logits [T, V].  Each row is cut into
-//       segments, one CTA per (segment, row); the grid is sized for T_cap rows and the kernel cuts
-//       the T rows it finds into as many segments as that grid can serve.  Threads read
+//       segments, one CTA per (segment, row), so small batches still fill 148 SMs.  Threads read
 //       16-byte vectors with streaming loads, several in flight per thread, and keep (max, first
 //       index); the CTA result is merged into one 64-bit word per row with atomicMax on
 //       (ordered value << 32 | ~index): the largest value wins and, among equals, the lowest
@@ -50,21 +49,13 @@ __device__ __forceinline__ void take8(const uint4& v, int base, float& best, int
 }
 
 __global__ void __launch_bounds__(kArgmaxThreads) accept_argmax_kernel(
-    const unsigned short* __restrict__ logits, int V, const int* __restrict__ cu_q, int B, int max_splits,
+    const unsigned short* __restrict__ logits, int V, const int* __restrict__ cu_q, int B, int seg_elems,
     unsigned long long* __restrict__ row_key) {
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
-    // The grid is sized for T_cap rows; the batch has T = cu_q[B] of them.  The fewer rows, the more segments a row is
-    // cut into (down to ~16 KB each), so a shallow batch still spreads over the CTAs that a deep one would use.
-    const int n_ctas = gridDim.x * gridDim.y;                    // gridDim.y = T_cap, the rows the per-row words are sized for
-    const int T = min(cu_q[B], (int)gridDim.y);
-    if (T <= 0) return;
-    const int splits = max(1, min(max_splits, n_ctas / T));
-    const int cta = blockIdx.y * gridDim.x + blockIdx.x;
-    if (cta >= T * splits) return;
-    const int row = cta / splits;
-    const int seg_elems = ((V + splits - 1) / splits + 7) & ~7;
-    const int start = (cta - row * splits) * seg_elems;
+    const int row = blockIdx.y;   // < T_cap, the rows the per-row words are sized for
+    if (row >= cu_q[B]) return;
+    const int start = blockIdx.x * seg_elems;
     if (start >= V) return;
     const int end = min(V, start + seg_elems);
     const unsigned short* rp = logits + (size_t)row * V;
@@ -207,9 +198,12 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
     const int max_splits = (V + 8191) / 8192;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
+    int seg = (V + splits - 1) / splits;
+    seg = (seg + 7) & ~7;
+    splits = (V + seg - 1) / seg;
     dim3 grid(splits, T_cap);
     dcut_status st = dcut_check_cuda(ctx, dcut_launch_pdl(accept_argmax_kernel, grid, dim3(kArgmaxThreads), 0, stream,
-                                                          static_cast<const unsigned short*>(logits), V, cu_q, B, max_splits, row_key),
+                                                          static_cast<const unsigned short*>(logits), V, cu_q, B, seg, row_key),
                                      "launch accept_argmax_kernel");
     if (st != DCUT_OK) return st;
     return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
@@ -317,8 +311,11 @@ extern "C" dcut_status dcut_accept_static(const void* logits, int V, const int* 
     const int max_splits = (V + 8191) / 8192;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
+    int seg = (V + splits - 1) / splits;
+    seg = (seg + 7) & ~7;
+    splits = (V + seg - 1) / seg;
     dim3 grid(splits, T_cap);
-    accept_argmax_kernel<<<grid, kArgmaxThreads, 0, cs>>>(static_cast<const unsigned short*>(logits), V, cu_q, B, max_splits, keys);
+    accept_argmax_kernel<<<grid, kArgmaxThreads, 0, cs>>>(static_cast<const unsigned short*>(logits), V, cu_q, B, seg, keys);
     if ((e = cudaGetLastError()) == cudaSuccess) {
         // rows at or past T_cap are never touched, so nothing outside the first T_cap words of the array is
         accept_match_kernel<<<1, 1024, 0, cs>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
