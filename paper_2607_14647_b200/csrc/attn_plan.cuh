@@ -132,7 +132,7 @@ __device__ __forceinline__ int plan_block_rows(int M, int max_rows, int n_rb, in
 __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* prefix) {
     __shared__ long long ws64[33], ws64b[33];
     __shared__ int ws32[33], ws32b[33];
-    __shared__ int total_s, w_tc_s, w_mma_s, w_tall_s;
+    __shared__ int total_s, w_tc_s, w_mma_s;
     __shared__ AttnSeg seg_s[kMaxSegs + 1];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const int group = a.n_q_heads / a.n_kv_heads;
@@ -140,12 +140,11 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
         total_s = 0;
         w_tc_s = 0;
         w_mma_s = 0;
-        w_tall_s = 0;
     }
     __syncthreads();
     // pass 1: pages in all, and how they would split over the two phases of the item kernel
     {
-        int local = 0, w_tc = 0, w_mma = 0, w_tall = 0;
+        int local = 0, w_tc = 0, w_mma = 0;
         for (int i = tid; i < a.B; i += nthr) {
             const int d = a.cu_q[i + 1] - a.cu_q[i] - 1;
             const int pages = (a.ctx_lens[i] + d + 1 + kPage - 1) / kPage;
@@ -153,18 +152,13 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             const int M = (d + 1) * group;
             const int n_rb = plan_row_blocks(M, a.max_item_rows, a.tail_rows);
             int tc_rb = 0;
-            for (int rb = 0; rb < n_rb; ++rb) {
-                const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
-                tc_rb += rows >= a.tc_min_rows ? 1 : 0;
-                w_tall += rows > 96 ? pages : 0;               // rows in the last lane quarter of tensor memory
-            }
+            for (int rb = 0; rb < n_rb; ++rb) tc_rb += plan_block_rows(M, a.max_item_rows, n_rb, rb) >= a.tc_min_rows ? 1 : 0;
             w_tc += pages * tc_rb;
             w_mma += pages * (n_rb - tc_rb);
         }
         if (local) atomicAdd(&total_s, local);
         if (w_tc) atomicAdd(&w_tc_s, w_tc);
         if (w_mma) atomicAdd(&w_mma_s, w_mma);
-        if (w_tall) atomicAdd(&w_tall_s, w_tall);
     }
     __syncthreads();
     // The item kernel runs a segment's tcgen05 items first and its warp-level items after them.  When the second kind
@@ -211,9 +205,6 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
         a.plan[0] = overflow ? 0 : n_entries;
         a.plan[1] = overflow ? 0 : n_tc;
         a.plan[2] = total_s;
-        // Which warps of the item kernel's tcgen05 phase run the producer and the MMA issuer (see tc_phase): the ones on
-        // the schedulers of lane quarters 2 and 3 when most pages belong to query tiles that leave quarter 3 empty.
-        a.plan[3] = 2 * w_tall_s < w_tc_s ? 1 : 0;
         if (overflow) atomicExch(a.status, DCUT_DEV_PLAN_OVERFLOW);
     }
     if (overflow) {

@@ -808,17 +808,14 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
     const uint32_t s_full = smem_u32(c->s_full), p_full = smem_u32(c->p_full), pv_done = smem_u32(c->pv_done);
     const uint32_t q_ready = smem_u32(&c->q_ready), o_free = smem_u32(&c->o_free);
     const int tid = threadIdx.x, lane = tid & 31;
-    // Role of this warp.  A softmax warp must be the warp whose number mod 4 is its lane quarter of tensor memory, which
-    // is also its scheduler: warps 2-9.  The producer (role 0) and the MMA issuer (role 1) run on warps 0 and 1 and the
-    // tail warps (roles 10, 11) on warps 10 and 11 when the query tiles fill all four lane quarters: the schedulers
-    // prefer their lower-numbered warps, so the issuer goes ahead of the softmax warps it shares a scheduler with and
-    // the instruction-heavy tail warps behind them (the other way round full-depth 136-row tiles lost 8 %).  When most
-    // pages belong to tiles that leave quarter 3 empty (32q/8kv at depth 16: 68 rows; pruned batches) the plan says so
-    // and the two pairs swap: producer and issuer get schedulers 2 and 3 to themselves instead of sharing 0 and 1 with
-    // the softmax warps that always have rows (scheduler 3 issued 6 % of the time on 68-row tiles): +9 % at full depth
-    // on the 32q/8kv workload.
-    const int pw = tid >> 5;
-    const int warp = a.plan[3] ? (pw >= 10 ? pw - 10 : (pw < 2 ? pw + 10 : pw)) : pw;
+    // Roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-3 tail rows, warps 4-11 softmax (team 0: 4-7, team 1: 8-11).
+    // A softmax warp's number mod 4 is its lane quarter of tensor memory and its scheduler, and a scheduler prefers its
+    // lower-numbered warps.  Query row r lives in lane (r + 64) mod 128: rows 0-63, which every tcgen05 item has, belong
+    // to quarters 2 and 3, so the producer and the issuer (schedulers 0 and 1, first in line there) share a scheduler
+    // only with the softmax warps of rows 64-127, which short query tiles (32q/8kv at depth 16: 68 rows; pruned
+    // batches) leave idle.  With row r in lane r the issuer and the producer shared schedulers 0 and 1 with the softmax
+    // warps that always have rows, and one scheduler issued 6 % of the time on 68-row tiles.
+    const int warp = tid >> 5;
     const int group = a.n_q_heads / a.n_kv_heads;
     const uint32_t tmem_o = c->tmem_base;
     AttnItem item;
@@ -954,20 +951,20 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             sched_release(c, kPhase, n);
             G0 += n_groups;
         }
-    } else if (warp < 2 + kTcSoftmaxThreads / 32) {
+    } else if (warp >= 2 + kTcTailWarps) {
         // ---------------------------------------------------------------- softmax + epilogue
         // Two teams of 128 threads (warps 2-5 and 6-9) take the page groups of an item alternately; each has its own
         // running (maximum, sum) per row and its own O accumulator, so while one team works through the latency chain
         // of its group (tcgen05.ld, maximum, exponentials, tcgen05.st) the other team's group is in flight too.
-        // Row R = tensor-memory lane; a thread owns the whole row (64 columns) of its team's S tiles.  The two threads
+        // Row R sits in tensor-memory lane (R + 64) mod 128; a thread owns the whole row (64 columns) of its team's S tiles.  The two threads
         // of a row (one per team) meet at a named barrier at the top and at the end of an item only.
         const uint32_t tmem_q = tmem_o + kTcColQ;
-        const int quarter = warp & 3, team = (warp - 2) >> 2;     // lane quarter of tensor memory; team 0 / 1
-        const int R = quarter * 32 + lane;
+        const int quarter = warp & 3, team = (warp - 2 - kTcTailWarps) >> 2;   // lane quarter of tensor memory; team 0 / 1
+        const int R = (quarter * 32 + lane + 64) & 127;            // the query row in this thread's lane
         const uint32_t t_lane = tmem_o + ((uint32_t)(quarter * 32) << 16);
         const uint32_t t_mine = t_lane + kTcColOB * team, t_other = t_lane + kTcColOB * (team ^ 1);
         const float cs = a.scale_log2;
-        // an item's query tile goes to tensor memory: row R = lane of tensor memory, 128 bf16 = 64 words, 32 per team
+        // an item's query tile goes to tensor memory: row R into this thread's lane, 128 bf16 = 64 words, 32 per team
         auto store_q = [&](const AttnItem& it) {
             uint32_t qw[32];
             const int rows = min(it.pad[2], 128);
@@ -1004,7 +1001,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             if (!q_staged) store_q(item);
             q_staged = false;
             const int jmax = ctx_len + (row0 + min(R, M - 1)) / group;  // last visible cache position
-            const bool live = quarter * 32 < M;                          // (warp-uniform) some of this warp's rows exist
+            const bool live = ((quarter * 32 + 64) & 127) < M;           // (warp-uniform) some of this warp's rows exist
             float m_run = -INFINITY, l_run = 0.0f;
             for (int g = team; g < n_groups; g += 2) {
                 const int gc = G0 + g, b = gc % kTcSBufs;
@@ -1175,7 +1172,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
         // no item waits for them)
         // One m16 tile by warp-level MMA on the staged pages; warp tw takes the item's pages p with p mod 2 = tw.
         // Both warps walk every group of every item, because every stage of the ring waits for their arrival.
-        const int tw = warp - (2 + kTcSoftmaxThreads / 32);
+        const int tw = warp - 2;
         const float cs = a.scale_log2;
         float* t_o = tail_buf;
         float* t_ml = tail_buf + kTcTailRows * kTcTailStride;
@@ -1503,7 +1500,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
             }
             if (swapped) {
                 // the 64 threads merge the two warps' rows and write them out, four head-dim elements at a time
-                for (int i = (warp - (2 + kTcSoftmaxThreads / 32)) * 32 + lane; i < M * 32; i += 32 * kTcTailWarps) {
+                for (int i = tw * 32 + lane; i < M * 32; i += 32 * kTcTailWarps) {
                     const int rr = i >> 5, c4 = (i & 31) << 2;
                     const float m0 = t_ml[rr * 2], l0 = t_ml[rr * 2 + 1], m1 = t_ml[(8 + rr) * 2], l1 = t_ml[(8 + rr) * 2 + 1];
                     const float m_all = fmaxf(m0, m1);
