@@ -23,21 +23,23 @@ constexpr int kPage = 16;            // tokens per page
 constexpr int kSlotRows = 144;       // rows of a partial-result slot (the largest query tile of an item)
 constexpr int kMaxSegs = 256;        // segments (SMs) the plan handles
 
-// Cost model, nanoseconds on B200, fitted to the busy time of the item kernel's CTAs against the items and pages of
-// their segments (least squares over the 148 CTAs, batches of mixed and of equal query tiles).  With every SM streaming,
-// a page costs about what the shared HBM gives each SM, a little less for the CTAs that can take more.  tcgen05 phase:
-// 188 per page, 196 with tail rows, but 166 when the shapes never have tail rows (`tc_alone`: the producer and the MMA
-// issuer then run on schedulers that hold no busy softmax warps, and CTAs with only such items finished 10 % early at
-// 188); warp-level phase 176.  Per item, beyond its pages: 3.8 us on the tcgen05 phase, 7.5 us with tail rows (O is
-// single-buffered in tensor memory and the softmax -> PV chain drains at an item boundary; the tail warps add their
-// merge), 3 us on the warp-level phase (2.1-2.8 in batches of such items only; CTAs with two or three short warp-level
-// items among tcgen05 CTAs were the last to finish on small batches at 2.5).  Only ratios matter for the partition.
-__device__ __forceinline__ int cost_per_page(int rows, int tc, int tc_alone) {
-    if (tc) return rows > 128 ? 196 : (tc_alone ? 166 : 188);   // every lane of tensor memory is processed, whatever the valid rows
+// Cost model, nanoseconds on B200, fitted to the busy time of the item kernel's CTAs (`%globaltimer` at the start and
+// the end of every CTA) against the items and pages of their segments by class of item (least squares over the 148
+// CTAs of batches with random depths).  With every SM streaming, a page costs about what the shared HBM gives each SM;
+// what differs is how many softmax warps share schedulers with the producer and the MMA issuer.  tcgen05 phase, query
+// tiles of up to 96 rows (lane quarter 1 of tensor memory empty, so the issuer has its scheduler to itself): 178 per
+// page (fits 178-179 for tiles of <= 32, <= 64, <= 96 rows); 97-128 rows: 197; with tail rows: 204; warp-level phase:
+// as the short tiles (163-170 against 166 in the same batches).  Per item, beyond its pages: 3.2-3.8 us up to 96 rows,
+// 4.7 to 128, 5.6-7.5 with tail rows (O is single-buffered in tensor memory and the softmax -> PV chain drains at an
+// item boundary; the tail warps add their merge), 3.6-4.3 us on the warp-level phase next to tcgen05 CTAs.  Only
+// ratios matter for the partition.  With one cost for all tiles up to 128 rows, CTAs whose items had 97-128 rows
+// finished 8 % after the mean on workload 3 with mixed depths.
+__device__ __forceinline__ int cost_per_page(int rows, int tc) {
+    if (tc) return rows > 128 ? 204 : (rows > 96 ? 197 : 178);
     const int mt = (rows + 15) >> 4;                       // m-tiles of the warp-level phase: memory-bound up to two
-    return 176 * max(7, 3 * mt) / 7;
+    return 178 * max(7, 3 * mt) / 7;
 }
-__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 7500 : 3800) : 3000; }
+__device__ __forceinline__ int cost_per_item(int rows, int tc) { return tc ? (rows > 128 ? 6500 : (rows > 96 ? 4700 : 3500)) : 4000; }
 
 struct PlanArgs {
     const int* ctx_lens;
@@ -45,7 +47,6 @@ struct PlanArgs {
     int B, n_q_heads, n_kv_heads;
     int n_sm;                           // segments = CTAs of the item kernel
     int min_chunk_pages;                // no piece of a cut item is shorter than this
-    int tc_alone;                       // the shapes never give a query tile above 128 rows (see the cost model)
     int tc_min_rows, max_item_rows;
     int tail_rows;                      // a remainder of at most this many rows rides with the last full row block (0: never)
     int max_entries;
@@ -181,7 +182,7 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             for (int rb = 0; rb < n_rb; ++rb) {
                 const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
                 const int tc = rows >= tc_min_rows;
-                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc, a.tc_alone));
+                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc));
                 if (tc) {
                     ++my_tc;
                     c_tc += c;
@@ -228,7 +229,7 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             for (int rb = 0; rb < n_rb; ++rb) {
                 const int rows = plan_block_rows(M, a.max_item_rows, n_rb, rb);
                 const int tc = rows >= tc_min_rows;
-                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc, a.tc_alone));
+                const long long c = (long long)a.n_kv_heads * (cost_per_item(rows, tc) + (long long)pages * cost_per_page(rows, tc));
                 AttnEntry en;
                 en.req = i;
                 en.row0 = rb * a.max_item_rows;
@@ -271,7 +272,7 @@ __device__ __forceinline__ void attn_plan_body(const PlanArgs& a, long long* pre
             // page (the segment between them would hold an empty piece that nobody writes): consecutive positions are
             // at least total / n_sm apart, so they land on different multiples as long as a segment is worth at least
             // min_chunk_pages of this item; below that (tiny batches) the item is not cut at all.
-            const long long quantum = (long long)a.min_chunk_pages * cost_per_page(en.rows, en.tc, a.tc_alone);
+            const long long quantum = (long long)a.min_chunk_pages * cost_per_page(en.rows, en.tc);
             int p = (in_item <= 0 || total / a.n_sm < quantum) ? 0 : (int)(in_item / quantum) * a.min_chunk_pages;
             if (en.pages - p < a.min_chunk_pages) {          // the rest is too short to be a piece: the boundary moves to the next item
                 p = 0;
