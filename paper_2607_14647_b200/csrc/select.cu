@@ -199,11 +199,12 @@ __global__ void __launch_bounds__(kThreads, 1) dcut_select_kernel(SelectArgs a) 
         const size_t cost_bytes = sizeof(float) * (size_t)(a.n_buckets > 0 ? a.n_buckets : n + 1);
         const char* cost0 = reinterpret_cast<const char*>(a.cost + (a.n_buckets > 0 ? 0 : B));
         for (size_t off = (size_t)tid * 128; off < cost_bytes; off += (size_t)kThreads * 128) prefetch_l2(cost0 + off);
-        for (size_t off = (size_t)tid * 128; off < sizeof(int) * (size_t)n; off += (size_t)kThreads * 128)
-            prefetch_l2(reinterpret_cast<const char*>(a.draft_ids) + off);
+        if (a.draft_ids)      // (the three arrays are optional: a caller that wants only depths and cu_q passes none)
+            for (size_t off = (size_t)tid * 128; off < sizeof(int) * (size_t)n; off += (size_t)kThreads * 128)
+                prefetch_l2(reinterpret_cast<const char*>(a.draft_ids) + off);
         for (size_t off = (size_t)tid * 128; off < sizeof(int) * (size_t)B; off += (size_t)kThreads * 128) {
-            prefetch_l2(reinterpret_cast<const char*>(a.ctx_lens) + off);
-            prefetch_l2(reinterpret_cast<const char*>(a.bonus_ids) + off);
+            if (a.ctx_lens) prefetch_l2(reinterpret_cast<const char*>(a.ctx_lens) + off);
+            if (a.bonus_ids) prefetch_l2(reinterpret_cast<const char*>(a.bonus_ids) + off);
         }
         if (a.n_buckets > 0 && tid == 0) prefetch_l2(a.bucket_K);
     }
