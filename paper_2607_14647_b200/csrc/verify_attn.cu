@@ -204,19 +204,20 @@ __global__ void __launch_bounds__(kPlanThreads) attn_plan_kernel(PlanArgs a) {
 //   O_team[128, 128] += P . V_page  one MMA (M128 N128 K16) per page: A = P from tensor memory, B = the V tile
 //                 read MN-major (transposed by its descriptor); one accumulator per team in tensor memory.
 // Both MMAs therefore stream only K and V from shared memory.  Warp 0: TMA producer (lanes 0-3 look up the
-// group's pages, one elected lane issues its loads), warp 1: MMA issuer and tensor-memory owner, warps 2-5 and
-// 6-9: the two softmax teams, which also write the output.
+// group's pages, one elected lane issues its loads), warp 1: MMA issuer and tensor-memory owner, warps 2-3: tail rows
+// (below), warps 4-7 and 8-11: the two softmax teams, which also write the output (why this order: tc_phase).
 //   tail rows   a query tile of 129..144 rows (8 q heads per kv head at depth 16: 136) does not fit the 128 lanes of
 //                 tensor memory.  Cutting it into two items would stream the request's K/V twice; instead the item
-//                 keeps all its rows and warps 10-11 take rows 128.. as one m16 tile of warp-level MMAs
+//                 keeps all its rows and warps 2-3 take rows 128.. as one m16 tile of warp-level MMAs
 //                 (mma.sync, as in the warp-level phase) on the very pages the ring holds for the tcgen05 MMAs: the
 //                 two warps take the item's pages alternately and merge their (m, l, O) at the end of the item.  A
 //                 ring stage is released by three arrivals: the commit of its last PV MMA and the two tail warps
-//                 (which arrive as soon as the stage is full when the item has no tail rows).
+//                 (which arrive as soon as the stage is full when the item has no tail rows; with shapes that
+//                 never give more than 128 rows they take no part and the commit alone releases a stage).
 constexpr int kTcGroupStages = 6;                  // ring of page groups (192 KB in flight)
 constexpr int kTcSBufs = 3;                        // S/P buffers in tensor memory: groups in flight between QK^T and PV
 constexpr int kTcSoftmaxThreads = 256;             // two teams of 128: one thread per row and team
-constexpr int kTcTailWarps = 2;                    // warps 10, 11: query rows 128..143 of an item, by warp-level MMA
+constexpr int kTcTailWarps = 2;                    // warps 2, 3: query rows 128..143 of an item, by warp-level MMA
 constexpr int kTcTailRows = 16;                    // one m16 tile
 constexpr int kTcTailStride = 128 + 8;             // floats per row of the tail warps' merge buffer
 constexpr int kTcTailBytes = (kTcTailRows * kTcTailStride + kTcTailRows * 2) * 4;
@@ -953,7 +954,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
         }
     } else if (warp >= 2 + kTcTailWarps) {
         // ---------------------------------------------------------------- softmax + epilogue
-        // Two teams of 128 threads (warps 2-5 and 6-9) take the page groups of an item alternately; each has its own
+        // Two teams of 128 threads (warps 4-7 and 8-11) take the page groups of an item alternately; each has its own
         // running (maximum, sum) per row and its own O accumulator, so while one team works through the latency chain
         // of its group (tcgen05.ld, maximum, exponentials, tcgen05.st) the other team's group is in flight too.
         // Row R sits in tensor-memory lane (R + 64) mod 128; a thread owns the whole row (64 columns) of its team's S tiles.  The two threads
@@ -1183,7 +1184,7 @@ __device__ __forceinline__ void tc_phase(const CUtensorMap& k2_map, const CUtens
         for (int n = 0;; ++n) {
             const int idx = sched_wait(c, kPhase, n, item);
             if (idx == -2) failed = true;
-            // also: warp 10 has read what warp 11 left in the merge buffer for the previous item
+            // also: the first tail warp has read what the second left in the merge buffer for the previous item
             if (bar_any(6, 32 * kTcTailWarps, failed || ABORTED(c))) {
                 failed = true;
                 break;
