@@ -47,6 +47,7 @@ L2_BYTES = 126e6
 # full size and of workload 3's shapes at B = 48; the kernel's traffic is proportional to the KV it streams
 ATTN_TRAFFIC_RATIO = 1.004
 RATIO_BUCKETS = [(1, 4), (1, 2), (3, 4), (1, 1)]          # the paper's ratio set R (Eq. 4; Table 3)
+COST_INNER = 4        # steps per timed sample of the cost profile (CUDA event stamps step by 1-2 us)
 COST_PROFILE_DIR = os.path.join(ROOT, "paper_2607_14647_b200", "cost_profiles")
 
 
@@ -485,7 +486,7 @@ def profile_dense_cost(w: Workload, args, points: int, reps: int):
         def run():
             runs[k[0] % len(runs)]()
             k[0] += 1
-        ts = profiler.time_replays(run, reps, 3)
+        ts = profiler.time_replays(run, reps, 3, COST_INNER)
         med.append(float(np.median(ts)))
         p25.append(float(np.percentile(ts, 25)))
         del qp, lp, bufs, runs, keep
@@ -517,7 +518,7 @@ def profile_bucket_cost(w: Workload, args, reps: int):
             k[0] += 1
         run._keep = (qp, lp, bufs, keep)
         return run
-    table = profiler.profile_cost_grid(grid, make_step, reps=reps, warmup=3)
+    table = profiler.profile_cost_grid(grid, make_step, reps=reps, warmup=3, inner=COST_INNER)
     return grid, table
 
 
@@ -841,7 +842,7 @@ def bench_workload(cfg, dev, args, world, rank, local, headline: bool):
                    "cost_table": {"points_T": grid, "median_ms": [round(x, 4) for x in med], "p25_ms": [round(x, 4) for x in p25],
                                   "table_ms_at_points": [round(float(cost[t]), 4) for t in grid],
                                   "fit": "running minimum from the long end" if w.is_layer else "isotonic (non-decreasing least squares)",
-                                  "reps_per_point": reps},
+                                  "reps_per_point": reps, "steps_per_rep": COST_INNER},
                    "bucket_cost_table": {"B": cfg.B, "ratios": [f"{n}/{d}" for n, d in RATIO_BUCKETS],
                                          "K": [bucket_grid.budget(cfg.B, r) for r in range(len(RATIO_BUCKETS))],
                                          "median_ms": [round(float(x), 4) for x in bucket_table[0]]}}
@@ -983,7 +984,7 @@ def run_dcut(args):
         ct = section["cost_table"]
         json.dump({"B": cfg.B, "gamma": cfg.gamma, "workload": workload_name(cfg), "T": ct["points_T"], "median_ms": ct["median_ms"],
                    "protocol": "bench.py profile_dense_cost: selector forced to T, the step's CUDA graph replayed, median of "
-                               f"{ct['reps_per_point']} replays per point", "gpu": torch.cuda.get_device_name(local)},
+                               f"{ct['reps_per_point']} samples of {ct['steps_per_rep']} back-to-back replays per point", "gpu": torch.cuda.get_device_name(local)},
                   open(os.path.join(COST_PROFILE_DIR, f"b200_config{cfg.index}_gamma{cfg.gamma}.json"), "w"), indent=1)
     line = {
         "metric": METRIC, "value": p["tokens_per_s"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
