@@ -1793,7 +1793,9 @@ void dcut_fill_plan_args(dcut_ctx* ctx, const int* ctx_lens, const int* cu_q, in
     pa.status = ctx->d_status;
     pa.tc_min_rows = ctx->lim.head_dim == 128 ? ctx->attn_tc_min_rows : 1 << 30;
     pa.max_item_rows = 128;
-    pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128) ? ctx->attn_tail_rows : 0;
+    // (no tail-row items when the shapes cannot need them: the item kernel then runs without its tail warps)
+    const bool tail_on = ctx->attn_tail_rows > 0 && (ctx->lim.max_gamma + 1) * (ctx->lim.n_q_heads / ctx->lim.n_kv_heads) > 128;
+    pa.tail_rows = (ctx->lim.head_dim == 128 && ctx->attn_tc_min_rows <= 128 && tail_on) ? ctx->attn_tail_rows : 0;
     pa.max_entries = ctx->max_entries;
     pa.entries = ctx->d_entries;
     pa.segs = ctx->d_segs;
