@@ -1680,6 +1680,32 @@ __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
     constexpr int kPer = DH / 32;
     for (int R = blockIdx.y * 32 + warp; R < en.rows; R += 32 * gridDim.y) {
         // piece 0 is in segment b - 1 (the item begins there: its second slot); piece c >= 1 in segment b + c - 1 (first slot)
+        const int t = (en.row0 + R) / group, hl = (en.row0 + R) - t * group;
+        const size_t orow = (size_t)(en.q0 + t) * a.n_q_heads + sg.h * group + hl;
+        __nv_bfloat16* op = a.out + orow * DH + lane * kPer;
+        if (m == 1) {
+            // two pieces (nearly every cut): the four loads leave together, one trip to L2 instead of two per piece;
+            // the same arithmetic in the same order as the general loop below
+            const size_t r0 = (size_t)(2 * (b - 1) + 1) * dcut_plan::kSlotRows + R, r1 = (size_t)(2 * b) * dcut_plan::kSlotRows + R;
+            const float l0 = __ldcg(a.part_lse + r0), l1 = __ldcg(a.part_lse + r1);
+            float o0[kPer], o1[kPer];
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) {
+                o0[e] = __ldcg(a.part_o + r0 * DH + lane * kPer + e);
+                o1[e] = __ldcg(a.part_o + r1 * DH + lane * kPer + e);
+            }
+            const float m_all = fmaxf(l0, l1);
+            const float w0 = (l0 == -INFINITY) ? 0.0f : __expf(l0 - m_all), w1 = (l1 == -INFINITY) ? 0.0f : __expf(l1 - m_all);
+            const float wsum = (0.0f + w0) + w1;
+            const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
+#pragma unroll
+            for (int e = 0; e < kPer; e += 2) {
+                const float x0 = fmaf(w1, o1[e], fmaf(w0, o0[e], 0.0f)), x1 = fmaf(w1, o1[e + 1], fmaf(w0, o0[e + 1], 0.0f));
+                *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(x0 * inv, x1 * inv);
+            }
+            if (a.lse && lane == 0) a.lse[orow] = wsum > 0.0f ? m_all + logf(wsum) : -INFINITY;
+            continue;
+        }
         float m_all = -INFINITY;
         for (int c = 0; c <= m; ++c) {
             const size_t prow = (size_t)(c == 0 ? 2 * (b - 1) + 1 : 2 * (b + c - 1)) * dcut_plan::kSlotRows + R;
@@ -1699,9 +1725,6 @@ __global__ void __launch_bounds__(1024) attn_combine_kernel(CombineArgs a) {
             for (int e = 0; e < kPer; ++e) acc[e] += w * po[e];
         }
         const float inv = wsum > 0.0f ? 1.0f / wsum : 0.0f;
-        const int t = (en.row0 + R) / group, hl = (en.row0 + R) - t * group;
-        const size_t orow = (size_t)(en.q0 + t) * a.n_q_heads + sg.h * group + hl;
-        __nv_bfloat16* op = a.out + orow * DH + lane * kPer;
 #pragma unroll
         for (int e = 0; e < kPer; e += 2) *reinterpret_cast<uint32_t*>(op + e) = pack_bf16(acc[e] * inv, acc[e + 1] * inv);
         if (a.lse && lane == 0) a.lse[orow] = wsum > 0.0f ? m_all + logf(wsum) : -INFINITY;
