@@ -121,64 +121,126 @@ __device__ int slow_first_valid(const unsigned short* rp, int V) {
     return 0;
 }
 
+constexpr int kMatchR = 1;   // requests a warp of the matching kernel has in flight (2: 0.4 us less at B = 64, 0.35 us more at B = 16; 4: slower)
+
+struct MatchArgs {
+    const unsigned short* logits;   // only read for rows whose scan found nothing above -inf; may be null
+    int V;
+    const int* draft_ids;
+    const int* cu_q;
+    int B, gamma, row_cap;
+    unsigned long long* row_key;
+    int* accept_len;
+    int* bonus;
+    int* out_tokens;
+    int* n_accepted_total;
+    int* row_argmax;
+    int* status;
+};
+
 // One warp per request: the lanes fetch the row results of t = lane, lane + 32, ... together, a ballot finds the
 // first row whose argmax differs from the draft (or the last row), and the per-row words are cleared on the way.
+// A warp works on R requests at a time: their loads (offsets, then row words and drafts) are issued together, so the
+// two global-memory latencies of the chain are paid once per R requests.
 // Only rows below row_cap (the T_cap the words and the scan were sized for) exist: a cu_q that runs past it breaks the
 // caller's contract, so those rows are neither read nor cleared, the request's scan ends at the last row that
 // exists (a request with none reports accept_len 0 and bonus 0), and the status word, if there is one, says so.
-__global__ void __launch_bounds__(1024) accept_match_kernel(
-    const unsigned short* __restrict__ logits, int V, const int* __restrict__ draft_ids,
-    const int* __restrict__ cu_q, int B, int gamma, int row_cap, unsigned long long* __restrict__ row_key,
-    int* __restrict__ accept_len, int* __restrict__ bonus, int* __restrict__ out_tokens,
-    int* __restrict__ n_accepted_total, int* __restrict__ row_argmax, int* __restrict__ status) {
+// Returns this lane's share of the accepted-token total (lane 0 of each warp carries it).
+template <int R>
+__device__ __forceinline__ int match_requests(const MatchArgs& g, int warp, int n_warps, int lane) {
+    int local = 0;
+    const int gamma = g.gamma;
+    for (int i0 = warp * R; i0 < g.B; i0 += n_warps * R) {
+        int a_[R], d_[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int i = i0 + r;
+            a_[r] = 0;
+            d_[r] = -2;                       // -2: no such request
+            if (i < g.B) {
+                a_[r] = g.cu_q[i];
+                d_[r] = g.cu_q[i + 1] - a_[r] - 1;
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (d_[r] == -2) continue;
+            int a = a_[r], d = d_[r];
+            if (a < 0 || d < 0 || d > gamma || a + d >= g.row_cap) {
+                if (lane == 0 && g.status) atomicExch(g.status, DCUT_DEV_BAD_CU_Q);
+                d = min(min(d, gamma), g.row_cap - 1 - a);       // rows [a, a + d] exist; none if d < 0 or a < 0
+                if (a < 0 || d < 0) d = -1;
+                d_[r] = d;
+            }
+        }
+        unsigned long long key_[R];
+        int dr_[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {         // the first 32 rows of each request
+            key_[r] = 0;
+            dr_[r] = -1;
+            if (lane <= d_[r]) {
+                key_[r] = __ldcg(g.row_key + a_[r] + lane);
+                if (lane < d_[r]) dr_[r] = g.draft_ids[(size_t)(i0 + r) * gamma + lane];
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            if (d_[r] == -2) continue;
+            const int i = i0 + r, a = a_[r], d = d_[r];
+            int m = d < 0 ? 0 : -1, bon = 0;
+            for (int t0 = 0; t0 <= d; t0 += 32) {
+                const int t = t0 + lane;
+                int am = 0;
+                bool stop = false;
+                if (t <= d) {
+                    unsigned long long key;
+                    int dr;
+                    if (t0 == 0) {
+                        key = key_[r];
+                        dr = dr_[r];
+                    } else {
+                        key = __ldcg(g.row_key + a + t);
+                        dr = t < d ? g.draft_ids[(size_t)i * gamma + t] : -1;
+                    }
+                    g.row_key[a + t] = 0;
+                    am = key ? (int)(0xffffffffu - (unsigned int)key)
+                             : (g.logits ? slow_first_valid(g.logits + (size_t)(a + t) * g.V, g.V) : 0);
+                    if (g.row_argmax) g.row_argmax[a + t] = am;
+                    stop = (t == d) || am != dr;
+                }
+                const unsigned int mask = __ballot_sync(0xffffffffu, stop);
+                if (m < 0 && mask) {
+                    const int first = __ffs(mask) - 1;
+                    m = t0 + first;
+                    bon = __shfl_sync(0xffffffffu, am, first);
+                }
+            }
+            if (lane == 0) {
+                g.accept_len[i] = m;
+                g.bonus[i] = bon;
+                local += m + 1;
+            }
+            if (g.out_tokens) {
+                int* o = g.out_tokens + (size_t)i * (gamma + 1);
+                for (int t = lane; t <= gamma; t += 32)
+                    o[t] = t < m ? ((t < 32 && t < d) ? dr_[r] : g.draft_ids[(size_t)i * gamma + t]) : (t == m ? bon : -1);
+            }
+        }
+    }
+    return local;
+}
+
+__global__ void __launch_bounds__(1024) accept_match_kernel(MatchArgs g) {
     __shared__ int total_s;
     if (threadIdx.x == 0) total_s = 0;
     __syncthreads();
     dcut_pdl_wait();
     dcut_pdl_launch_dependents();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    int local = 0;
-    for (int i = warp; i < B; i += n_warps) {
-        const int a = cu_q[i];
-        int d = cu_q[i + 1] - a - 1;
-        if (a < 0 || d < 0 || d > gamma || a + d >= row_cap) {
-            if (lane == 0 && status) atomicExch(status, DCUT_DEV_BAD_CU_Q);
-            d = min(min(d, gamma), row_cap - 1 - a);       // rows [a, a + d] exist; none if d < 0 or a < 0
-            if (a < 0) d = -1;
-        }
-        int m = d < 0 ? 0 : -1, bon = 0;
-        for (int t0 = 0; t0 <= d; t0 += 32) {
-            const int t = t0 + lane;
-            int am = 0;
-            bool stop = false;
-            if (t <= d) {
-                const unsigned long long key = row_key[a + t];
-                row_key[a + t] = 0;
-                am = key ? (int)(0xffffffffu - (unsigned int)key)
-                         : (logits ? slow_first_valid(logits + (size_t)(a + t) * V, V) : 0);
-                if (row_argmax) row_argmax[a + t] = am;
-                stop = (t == d) || am != draft_ids[(size_t)i * gamma + t];
-            }
-            const unsigned int mask = __ballot_sync(0xffffffffu, stop);
-            if (m < 0 && mask) {
-                const int first = __ffs(mask) - 1;
-                m = t0 + first;
-                bon = __shfl_sync(0xffffffffu, am, first);
-            }
-        }
-        if (lane == 0) {
-            accept_len[i] = m;
-            bonus[i] = bon;
-            local += m + 1;
-        }
-        if (out_tokens) {
-            int* o = out_tokens + (size_t)i * (gamma + 1);
-            for (int t = lane; t <= gamma; t += 32) o[t] = t < m ? draft_ids[(size_t)i * gamma + t] : (t == m ? bon : -1);
-        }
-    }
+    const int local = match_requests<kMatchR>(g, threadIdx.x >> 5, blockDim.x >> 5, threadIdx.x & 31);
     if (local) atomicAdd(&total_s, local);
     __syncthreads();
-    if (threadIdx.x == 0 && n_accepted_total) *n_accepted_total = total_s;
+    if (threadIdx.x == 0 && g.n_accepted_total) *g.n_accepted_total = total_s;
 }
 
 }  // namespace
@@ -187,6 +249,29 @@ dcut_status dcut_init_accept(dcut_ctx* ctx) {
     (void)ctx;
     return DCUT_OK;
 }
+
+namespace {
+MatchArgs match_args(const void* logits, int V, const int* draft_ids, const int* cu_q, int B, int gamma, int T_cap,
+                     unsigned long long* row_key, int* accept_len, int* bonus, int* out_tokens, int* n_accepted_total,
+                     int* row_argmax, int* status) {
+    MatchArgs m;
+    m.logits = static_cast<const unsigned short*>(logits);
+    m.V = V;
+    m.draft_ids = draft_ids;
+    m.cu_q = cu_q;
+    m.B = B;
+    m.gamma = gamma;
+    m.row_cap = T_cap;
+    m.row_key = row_key;
+    m.accept_len = accept_len;
+    m.bonus = bonus;
+    m.out_tokens = out_tokens;
+    m.n_accepted_total = n_accepted_total;
+    m.row_argmax = row_argmax;
+    m.status = status;
+    return m;
+}
+}  // namespace
 
 dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const int* draft_ids,
                                const int* cu_q, int B, int gamma, int T_cap, int* accept_len, int* bonus,
@@ -207,9 +292,8 @@ dcut_status dcut_launch_accept(dcut_ctx* ctx, const void* logits, int V, const i
                                      "launch accept_argmax_kernel");
     if (st != DCUT_OK) return st;
     return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
-                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
-                                                row_key, accept_len, bonus, out_tokens, n_accepted_total,
-                                                static_cast<int*>(nullptr), ctx->d_status),
+                                                match_args(logits, V, draft_ids, cu_q, B, gamma, T_cap, row_key, accept_len, bonus,
+                                                           out_tokens, n_accepted_total, nullptr, ctx->d_status)),
                            "launch accept_match_kernel");
 }
 
@@ -218,9 +302,8 @@ dcut_status dcut_launch_accept_match(dcut_ctx* ctx, const void* logits, int V, c
                                      int* n_accepted_total, int* row_argmax, unsigned long long* row_key,
                                      cudaStream_t stream) {
     return dcut_check_cuda(ctx, dcut_launch_pdl(accept_match_kernel, dim3(1), dim3(1024), 0, stream,
-                                                static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
-                                                row_key, accept_len, bonus, out_tokens, n_accepted_total, row_argmax,
-                                                ctx->d_status),
+                                                match_args(logits, V, draft_ids, cu_q, B, gamma, T_cap, row_key, accept_len, bonus,
+                                                           out_tokens, n_accepted_total, row_argmax, ctx->d_status)),
                            "launch accept_match_kernel");
 }
 
@@ -318,8 +401,8 @@ extern "C" dcut_status dcut_accept_static(const void* logits, int V, const int* 
     accept_argmax_kernel<<<grid, kArgmaxThreads, 0, cs>>>(static_cast<const unsigned short*>(logits), V, cu_q, B, seg, keys);
     if ((e = cudaGetLastError()) == cudaSuccess) {
         // rows at or past T_cap are never touched, so nothing outside the first T_cap words of the array is
-        accept_match_kernel<<<1, 1024, 0, cs>>>(static_cast<const unsigned short*>(logits), V, draft_ids, cu_q, B, gamma, T_cap,
-                                               keys, accept_len, bonus, out_tokens, n_accepted_total, nullptr, nullptr);
+        accept_match_kernel<<<1, 1024, 0, cs>>>(match_args(logits, V, draft_ids, cu_q, B, gamma, T_cap, keys, accept_len, bonus,
+                                                          out_tokens, n_accepted_total, nullptr, nullptr));
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) {
