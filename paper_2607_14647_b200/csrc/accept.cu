@@ -14,7 +14,7 @@
 namespace {
 
 constexpr int kArgmaxThreads = 256;
-constexpr int kUnroll = 4;
+constexpr int kUnroll = 8;   // 16-byte loads in flight per thread (4: 35-37 us at T = 600 of the 64-request workload, 8: 30-31; 50 against 51 us at T = 1088)
 
 __device__ __forceinline__ uint4 ld_stream_v4(const uint4* p) {
     uint4 r;
